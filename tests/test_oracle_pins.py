@@ -1,0 +1,356 @@
+"""Pins for the CPU oracle: every oracle function is checked against something other than itself --
+a worked example, closed forms, invariants that determine the answer uniquely, brute force on tiny
+inputs, and special cases that reduce to torch/numpy fp64 library routines.  CPU only."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import mok_ref
+from paper_2609_36070_b200 import inputs
+from paper_2609_36070_b200.inputs import MoEConfig, bf16_bits_to_f64, f32_to_bf16_bits
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "worked_example.txt")
+
+
+def bits(a):
+    """float array (exactly representable in bf16, or to be rounded) -> bf16 bit patterns."""
+    return f32_to_bf16_bits(np.asarray(a, np.float32))
+
+
+def small_inputs(T=24, H=16, E=6, k=3, I=8, I_s=8, seed=3, bias="none"):
+    cfg = MoEConfig("small", T=T, H=H, E=E, k=k, I=I, I_s=I_s, bias=bias, seed=seed)
+    d = inputs.make_inputs(cfg, threads=1)
+    # larger weights than the 0.02 recipe so that every term matters at fp64 tolerances
+    rng = np.random.default_rng(seed)
+    d["W_r"] = rng.standard_normal((E, H)).astype(np.float32)
+    d["W_gate_up"] = bits(rng.standard_normal((E, 2 * I, H)) * 0.5)
+    d["W_down"] = bits(rng.standard_normal((E, H, I)) * 0.5)
+    if I_s:
+        d["W_sgu"] = bits(rng.standard_normal((2 * I_s, H)) * 0.5)
+        d["W_sd"] = bits(rng.standard_normal((H, I_s)) * 0.5)
+    return cfg, d
+
+
+def t64(b):
+    return torch.from_numpy(bf16_bits_to_f64(b))
+
+
+def dense_ffn(v, Wgu, Wd):
+    """Library restatement of one expert FFN on a batch: torch fp64 matmuls + torch's own SiLU."""
+    I = Wgu.shape[0] // 2
+    g = v @ Wgu[:I].T
+    u = v @ Wgu[I:].T
+    return (torch.nn.functional.silu(g) * u) @ Wd.T
+
+
+# ----------------------------------------------------------------------------- worked example
+def read_golden():
+    vals = {}
+    for line in open(GOLDEN):
+        if line.startswith("#") or not line.strip():
+            continue
+        name, *nums = line.split()
+        vals[name] = np.array([float(v) for v in nums])
+    return vals
+
+
+def test_worked_example_routing_schedule_output():
+    g = read_golden()
+    T, H, E, k, I = 4, 2, 3, 2, 1
+    x = bits(g["x"].reshape(T, H))
+    W_r = g["W_r"].reshape(E, H).astype(np.float32)
+    Wgu = bits(np.concatenate([g["W_gate"].reshape(E, I, H), g["W_up"].reshape(E, I, H)], axis=1))
+    Wd = bits(g["W_down"].reshape(E, H, I))
+    Sgu = bits(np.concatenate([g["S_gate"].reshape(1, H), g["S_up"].reshape(1, H)], axis=0))
+    Sd = bits(g["S_down"].reshape(H, 1))
+    idx, w, gap, lg = mok_ref.route(x, W_r, None, k)
+    assert np.array_equal(lg.ravel(), g["logits"])                  # exact: all products are dyadic
+    assert np.array_equal(idx.ravel(), g["idx"].astype(np.int32))    # token 2 is a 3-way tie -> experts 0,1
+    np.testing.assert_allclose(w.ravel(), g["w"], rtol=0, atol=2e-12)
+    assert gap[2] == 0.0 and gap[0] == 0.25
+    counts, offsets, perm, inv = mok_ref.schedule(idx.ravel(), E)
+    assert np.array_equal(counts, g["counts"]) and np.array_equal(offsets, g["offsets"])
+    assert np.array_equal(perm, g["perm"])
+    out, idx2, w2 = mok_ref.forward(x, W_r, None, Wgu, Wd, Sgu, Sd, k)
+    np.testing.assert_allclose(out.ravel(), g["out"], rtol=0, atol=2e-12)
+    assert np.array_equal(idx2, idx) and np.array_equal(w2, w)
+
+
+# ----------------------------------------------------------------------------- routing
+def test_equal_logits_pick_first_k_with_equal_weights():
+    T, H, E, k = 5, 8, 7, 3
+    x = bits(np.random.default_rng(0).standard_normal((T, H)))
+    idx, w, gap, lg = mok_ref.route(x, np.zeros((E, H), np.float32), None, k)
+    assert np.array_equal(idx, np.tile(np.arange(k, dtype=np.int32), (T, 1)))
+    assert np.array_equal(w, np.full((T, k), 1.0 / k))
+    assert np.all(gap == 0.0)
+
+
+def test_routing_matches_torch_library_when_no_ties():
+    cfg, d = small_inputs(T=64, H=32, E=16, k=4, bias="normal")
+    idx, w, gap, lg = mok_ref.route(d["x"], d["W_r"], d["bias"], cfg.k)
+    tl = t64(d["x"]) @ torch.from_numpy(d["W_r"]).double().T + torch.from_numpy(d["bias"]).double()
+    np.testing.assert_allclose(lg, tl.numpy(), rtol=0, atol=1e-12)
+    assert gap.min() > 1e-9                                   # no ties in this draw
+    tv, ti = torch.topk(tl, cfg.k, dim=1)                     # library top-k: descending values
+    assert np.array_equal(idx, ti.numpy().astype(np.int32))
+    p = torch.softmax(tl, dim=1).gather(1, ti)
+    np.testing.assert_allclose(w, (p / p.sum(1, keepdim=True)).numpy(), rtol=0, atol=1e-14)
+    # closed form: softmax over all E then renormalised == softmax over the selected logits alone
+    np.testing.assert_allclose(w, torch.softmax(tv, dim=1).numpy(), rtol=0, atol=1e-14)
+    assert np.allclose(w.sum(1), 1.0, atol=1e-15) and (w > 0).all()
+    assert (np.diff(w, axis=1) <= 0).all()                    # slots are in descending-logit order
+
+
+def test_one_hot_tokens_read_topk_off_the_router_matrix():
+    H, E, k = 6, 9, 4
+    W_r = np.random.default_rng(1).standard_normal((E, H)).astype(np.float32)
+    x = bits(np.eye(H))
+    idx, w, gap, lg = mok_ref.route(x, W_r, None, k)
+    assert np.array_equal(lg, W_r.T.astype(np.float64))
+    for h in range(H):
+        col = W_r[:, h].astype(np.float64)
+        assert np.array_equal(idx[h], np.argsort(-col, kind="stable")[:k])
+        assert gap[h] == np.sort(col)[::-1][k - 1] - np.sort(col)[::-1][k]
+
+
+def test_topk_brute_force_with_many_ties():
+    rng = np.random.default_rng(2)
+    for E, k in [(5, 1), (5, 5), (8, 3), (13, 6)]:
+        lg = rng.integers(-2, 3, size=(40, E)).astype(np.float64) * 0.5     # heavy ties
+        idx, gap = mok_ref.topk(lg, k)
+        for t in range(lg.shape[0]):
+            order = sorted(range(E), key=lambda e: (-lg[t, e], e))
+            assert list(idx[t]) == order[:k]
+            want = np.inf if k == E else lg[t, order[k - 1]] - lg[t, order[k]]
+            assert gap[t] == want
+
+
+def test_expert_relabelling_commutes_with_routing():
+    cfg, d = small_inputs(T=32, H=16, E=10, k=3)
+    idx, w, gap, _ = mok_ref.route(d["x"], d["W_r"], None, cfg.k)
+    sigma = np.random.default_rng(5).permutation(cfg.E)          # new id of old expert e is sigma[e]
+    W2 = np.empty_like(d["W_r"])
+    W2[sigma] = d["W_r"]
+    idx2, w2, _, _ = mok_ref.route(d["x"], W2, None, cfg.k)
+    assert gap.min() > 0
+    assert np.array_equal(idx2, sigma[idx].astype(np.int32))
+    np.testing.assert_allclose(w2, w, rtol=0, atol=1e-15)
+
+
+def test_bias_enters_selection_and_weights():
+    cfg, d = small_inputs(T=16, H=16, E=8, k=2)
+    idx0, w0, _, lg0 = mok_ref.route(d["x"], d["W_r"], None, 2)
+    b = np.zeros(cfg.E, np.float32)
+    b[5] = 100.0
+    idx1, w1, _, lg1 = mok_ref.route(d["x"], d["W_r"], b, 2)
+    assert (idx1[:, 0] == 5).all() and (w1[:, 0] > 0.999999).all()
+    np.testing.assert_allclose(lg1 - lg0, np.tile(b.astype(np.float64), (16, 1)), atol=1e-12)
+    # a constant bias changes neither the selection nor the weights (softmax shift invariance)
+    idx2, w2, _, _ = mok_ref.route(d["x"], d["W_r"], np.full(cfg.E, 3.0, np.float32), 2)
+    assert np.array_equal(idx2, idx0)
+    np.testing.assert_allclose(w2, w0, rtol=0, atol=1e-13)
+
+
+# ----------------------------------------------------------------------------- schedule
+def check_schedule_invariants(a, E, counts, offsets, perm, inv):
+    n = a.size
+    assert counts.sum() == n and offsets[0] == 0 and offsets[E] == n
+    assert np.array_equal(np.sort(perm), np.arange(n))                      # bijection
+    assert np.array_equal(inv[perm], np.arange(n))
+    for e in range(E):
+        seg = perm[offsets[e]:offsets[e + 1]]
+        assert seg.size == counts[e]
+        assert (a[seg] == e).all()
+        assert (np.diff(seg) > 0).all()                                      # stable: ascending route ids
+
+
+@pytest.mark.parametrize("n,E", [(0, 4), (1, 1), (37, 5), (1000, 16), (4096, 256)])
+def test_schedule_equals_stable_counting_sort(n, E):
+    rng = np.random.default_rng(n + E)
+    a = rng.integers(0, E, size=n).astype(np.int32)
+    if n > 10:
+        a[a == 1] = 0                                                        # an empty expert
+    counts, offsets, perm, inv = mok_ref.schedule(a, E)
+    check_schedule_invariants(a, E, counts, offsets, perm, inv)
+    assert np.array_equal(counts, np.bincount(a, minlength=E))
+    assert np.array_equal(offsets[1:], np.cumsum(np.bincount(a, minlength=E)))
+    assert np.array_equal(perm, np.argsort(a, kind="stable"))
+
+
+def test_alg1_single_rank_is_the_schedule():
+    rng = np.random.default_rng(7)
+    a = rng.integers(0, 6, size=200).astype(np.int32)
+    counts, offsets, perm, inv = mok_ref.schedule(a, 6)
+    S, pr, pi = mok_ref.alg1(a.reshape(1, -1), L=6, c=0)
+    assert np.array_equal(S, offsets) and (pr == 0).all() and np.array_equal(pi, perm)
+
+
+@pytest.mark.parametrize("R,NK,L", [(2, 30, 3), (4, 64, 2), (5, 17, 4), (3, 1, 1)])
+def test_alg1_matches_sort_by_expert_ordinal_rank(R, NK, L):
+    """Algorithm 1's closed-form position against its own restatement as a sort (Section 3.1), for every rank."""
+    rng = np.random.default_rng(R * 100 + NK)
+    A = rng.integers(0, R * L, size=(R, NK)).astype(np.int32)
+    A[0, A[0] == 0] = 1 % (R * L)                                           # make one (rank, expert) pair empty
+    for c in range(R):
+        S, pr, pi = mok_ref.alg1(A, L, c)
+        keys = []
+        for r in range(R):
+            seen = {}
+            for j in range(NK):
+                g = int(A[r, j])
+                o = seen.get(g, 0)
+                seen[g] = o + 1
+                if g // L == c:
+                    keys.append((g - c * L, o, r, j))
+        keys.sort()
+        assert S[L] == len(keys)
+        assert [q[2] for q in keys] == list(pr) and [q[3] for q in keys] == list(pi)
+        # the three properties a pull schedule must have (Section 3.1)
+        experts = A[pr, pi] - c * L
+        assert (np.diff(experts) >= 0).all()                                 # non-decreasing local expert
+        for l in range(L):                                                   # contiguous fill of [S_l, S_l+1)
+            assert (experts[S[l]:S[l + 1]] == l).all()
+            ranks = pr[S[l]:S[l + 1]]
+            remaining = np.array([(A[r] == c * L + l).sum() for r in range(R)])
+            pos = 0
+            while pos < ranks.size:                                          # round-robin over ranks that still have routes
+                alive = [r for r in range(R) if remaining[r] > 0]
+                assert list(ranks[pos:pos + len(alive)]) == alive
+                remaining[alive] -= 1
+                pos += len(alive)
+
+
+# ----------------------------------------------------------------------------- expert FFN + combine
+def test_zero_routed_down_projection_reduces_to_dense_shared_expert():
+    cfg, d = small_inputs()
+    d["W_down"][:] = 0
+    out, _, _ = mok_ref.forward(d["x"], d["W_r"], None, d["W_gate_up"], d["W_down"], d["W_sgu"], d["W_sd"], cfg.k)
+    want = dense_ffn(t64(d["x"]), t64(d["W_sgu"]), t64(d["W_sd"])).numpy()
+    np.testing.assert_allclose(out, want, rtol=1e-12, atol=1e-12)
+
+
+def test_identical_experts_make_routing_irrelevant():
+    cfg, d = small_inputs(T=40, E=5, k=2)
+    d["W_gate_up"][:] = d["W_gate_up"][0]
+    d["W_down"][:] = d["W_down"][0]
+    out, _, w = mok_ref.forward(d["x"], d["W_r"], None, d["W_gate_up"], d["W_down"], d["W_sgu"], d["W_sd"], cfg.k)
+    v = t64(d["x"])
+    want = dense_ffn(v, t64(d["W_sgu"]), t64(d["W_sd"])) + dense_ffn(v, t64(d["W_gate_up"][0]), t64(d["W_down"][0]))
+    np.testing.assert_allclose(out, want.numpy(), rtol=1e-12, atol=1e-12)       # weights sum to 1
+
+
+def test_k_equals_E_is_the_dense_softmax_mixture():
+    cfg, d = small_inputs(T=20, E=4, k=4, I_s=0)
+    out, idx, w = mok_ref.forward(d["x"], d["W_r"], None, d["W_gate_up"], d["W_down"], None, None, 4)
+    v = t64(d["x"])
+    p = torch.softmax(v @ torch.from_numpy(d["W_r"]).double().T, dim=1)
+    fe = torch.stack([dense_ffn(v, t64(d["W_gate_up"][e]), t64(d["W_down"][e])) for e in range(4)], dim=1)
+    want = torch.einsum("te,teh->th", p, fe)
+    np.testing.assert_allclose(out, want.numpy(), rtol=1e-12, atol=1e-12)
+
+
+def test_zero_input_gives_zero_output():
+    cfg, d = small_inputs()
+    d["x"][:] = 0
+    out, _, _ = mok_ref.forward(d["x"], d["W_r"], None, d["W_gate_up"], d["W_down"], d["W_sgu"], d["W_sd"], cfg.k)
+    assert np.array_equal(out, np.zeros_like(out))
+
+
+def test_linearity_in_down_projection_and_combine_weights():
+    cfg, d = small_inputs(I_s=0)
+    idx, w, _, _ = mok_ref.route(d["x"], d["W_r"], None, cfg.k)
+    tok = np.arange(cfg.T, dtype=np.int32)
+    base = mok_ref.ffn_tokens(d["x"], d["W_gate_up"], d["W_down"], None, None, idx, w, tok)
+    Wd2 = bits(bf16_bits_to_f64(d["W_down"]) * 2.0)                           # x2 is exact in bf16
+    np.testing.assert_array_equal(mok_ref.ffn_tokens(d["x"], d["W_gate_up"], Wd2, None, None, idx, w, tok), 2 * base)
+    np.testing.assert_allclose(mok_ref.ffn_tokens(d["x"], d["W_gate_up"], d["W_down"], None, None, idx, 0.5 * w, tok),
+                               0.5 * base, rtol=1e-15)
+    # with one-hot combine weights the output is a single expert's dense FFN
+    w1 = np.zeros_like(w)
+    w1[:, 1] = 1.0
+    got = mok_ref.ffn_tokens(d["x"], d["W_gate_up"], d["W_down"], None, None, idx, w1, tok)
+    v = t64(d["x"])
+    for t in range(cfg.T):
+        e = idx[t, 1]
+        want = dense_ffn(v[t:t + 1], t64(d["W_gate_up"][e]), t64(d["W_down"][e]))[0].numpy()
+        np.testing.assert_allclose(got[t], want, rtol=1e-12, atol=1e-12)
+
+
+def test_token_permutation_equivariance_and_sampling():
+    cfg, d = small_inputs()
+    out, idx, w = mok_ref.forward(d["x"], d["W_r"], None, d["W_gate_up"], d["W_down"], d["W_sgu"], d["W_sd"], cfg.k)
+    pi = np.random.default_rng(9).permutation(cfg.T)
+    out2, _, _ = mok_ref.forward(np.ascontiguousarray(d["x"][pi]), d["W_r"], None, d["W_gate_up"], d["W_down"],
+                                 d["W_sgu"], d["W_sd"], cfg.k)
+    assert np.array_equal(out2, out[pi])
+    tok = np.array([5, 0, 17, 5], np.int32)
+    sub = mok_ref.ffn_tokens(d["x"], d["W_gate_up"], d["W_down"], d["W_sgu"], d["W_sd"], idx, w, tok)
+    assert np.array_equal(sub, out[tok])
+
+
+def test_scalar_brute_force_of_the_definition():
+    """Pure-Python scalar loops with math.exp, transcribed from the equation, on a tiny shape with a bias."""
+    import math
+    cfg, d = small_inputs(T=6, H=4, E=3, k=2, I=3, I_s=2, bias="normal")
+    out, idx, w = mok_ref.forward(d["x"], d["W_r"], d["bias"], d["W_gate_up"], d["W_down"], d["W_sgu"], d["W_sd"], 2)
+    x = bf16_bits_to_f64(d["x"])
+    Wgu, Wd = bf16_bits_to_f64(d["W_gate_up"]), bf16_bits_to_f64(d["W_down"])
+    Sgu, Sd = bf16_bits_to_f64(d["W_sgu"]), bf16_bits_to_f64(d["W_sd"])
+
+    def ffn(v, gu, dn, I):
+        hid = []
+        for i in range(I):
+            g = sum(gu[i][h] * v[h] for h in range(cfg.H))
+            u = sum(gu[I + i][h] * v[h] for h in range(cfg.H))
+            hid.append(g / (1.0 + math.exp(-g)) * u)
+        return [sum(dn[h][i] * hid[i] for i in range(I)) for h in range(cfg.H)]
+
+    for t in range(cfg.T):
+        lg = [sum(x[t][h] * float(d["W_r"][e][h]) for h in range(cfg.H)) + float(d["bias"][e]) for e in range(cfg.E)]
+        order = sorted(range(cfg.E), key=lambda e: (-lg[e], e))[:2]
+        assert order == list(idx[t])
+        ex = [math.exp(v - max(lg)) for v in lg]
+        s = [ex[e] / sum(ex) for e in order]
+        acc = ffn(x[t], Sgu, Sd, cfg.I_s)
+        for e, se in zip(order, s):
+            f = ffn(x[t], Wgu[e], Wd[e], cfg.I)
+            acc = [a + se / sum(s) * fv for a, fv in zip(acc, f)]
+        np.testing.assert_allclose(out[t], acc, rtol=1e-12, atol=1e-13)
+
+
+def test_bf16_mimic_mode_is_close_but_not_identical():
+    cfg, d = small_inputs(T=32, H=64, I=32, I_s=0)
+    idx, w, _, _ = mok_ref.route(d["x"], d["W_r"], None, cfg.k)
+    tok = np.arange(cfg.T, dtype=np.int32)
+    a = mok_ref.ffn_tokens(d["x"], d["W_gate_up"], d["W_down"], None, None, idx, w, tok)
+    b = mok_ref.ffn_tokens(d["x"], d["W_gate_up"], d["W_down"], None, None, idx, w, tok, mimic_bf16=True)
+    rel = np.abs(a - b).mean() / np.abs(a).mean()
+    assert 0 < rel < 5e-3
+
+
+# ----------------------------------------------------------------------------- input generator (host logic)
+def test_bf16_rounding_matches_torch_and_is_seeded():
+    a = np.random.default_rng(0).standard_normal(10000).astype(np.float32)
+    a[:4] = [1.00390625, 1.01171875, -1.00390625, 3.0e-39]                     # ties to even, a subnormal
+    want = torch.from_numpy(a).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    assert np.array_equal(f32_to_bf16_bits(a), want)
+    cfg = inputs.CONFIGS["tiny"]
+    d1, d2 = inputs.make_inputs(cfg), inputs.make_inputs(cfg, threads=1)
+    for key in d1:
+        assert (d1[key] is None and d2[key] is None) or np.array_equal(d1[key], d2[key])
+    x_short = inputs.make_x(cfg.with_tokens(100))
+    assert np.array_equal(x_short, d1["x"][:100])
+    assert abs(bf16_bits_to_f64(d1["W_gate_up"]).std() - 0.02) < 2e-4
+    assert abs(bf16_bits_to_f64(d1["x"]).std() - 1.0) < 2e-2
+
+
+def test_token_sample_covers_every_used_expert():
+    cfg = MoEConfig("s", T=2000, H=8, E=64, k=2, I=8)
+    idx = np.random.default_rng(0).integers(0, 40, size=(cfg.T, 2)).astype(np.int32)   # experts 40..63 unused
+    idx[1999] = [62, 63]                                                     # two experts used by one late token only
+    s = inputs.sample_tokens(cfg, idx, 64)
+    assert set(np.unique(idx)) == set(np.unique(idx[s])) and 1999 in s
+    assert np.array_equal(s, np.unique(s)) and (s[:64 if s.size > 64 else s.size] >= 0).all()
