@@ -1,0 +1,153 @@
+/*
+ * mok.h -- C ABI of libmok: the fused Mixture-of-Experts layer forward pass on one B200 (sm_100a).
+ *
+ * The layer (paper, Section 2.1):
+ *     MoE(x, s) = f_shared(x) + sum_{i in top-k} s_i / (sum_j s_j) * f_i(x),
+ *     f_i(x)    = W_down_i ( silu(W_gate_i x) .* (W_up_i x) ).
+ * One call runs, on the device and without any host synchronisation or count readback (Section 3.3):
+ *   router projection and top-k with normalised weights (Section 2.1; Figure 1, right),
+ *   dispatch schedule construction (Algorithm 1 with one rank: counts, offsets, stable permutation),
+ *   the token gather in expert order ("pull dispatch", Section 3.1),
+ *   the routed and shared SwiGLU expert FFNs as grouped bf16 GEMMs (Section 2.1),
+ *   and the deterministic weighted combine back to token order ("push combine" + router-weighted sum,
+ *   Sections 3.1 and 3.4 "Determinism").
+ *
+ * General rules for every entry point
+ *   - Pointers are DEVICE pointers unless the argument is documented as HOST.  The caller owns every
+ *     buffer; the library borrows it for the duration of the enqueued work and never frees it.
+ *   - bf16 tensors are row-major with the last index contiguous; they must be 16-byte aligned and
+ *     H, I, I_shared must be multiples of 8 (16-byte rows).
+ *   - Work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = default stream).  Calls return
+ *     as soon as the work is enqueued, unless stated otherwise.
+ *   - Return value: MOK_OK (0) or a negative mok_status.  Nothing throws or exits.  Argument errors are
+ *     detected before anything is launched.
+ *   - Inputs must be finite; behaviour on NaN/Inf is unspecified.
+ *   - Limits: 1 <= k <= 32, k <= E <= 512, T*k < 2^31 / 256.
+ */
+#ifndef MOK_H_
+#define MOK_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum mok_status {
+    MOK_OK = 0,
+    MOK_ERR_NULL = -1,       /* a required pointer is NULL */
+    MOK_ERR_SHAPE = -2,      /* unsupported or inconsistent sizes */
+    MOK_ERR_ALIGN = -3,      /* a tensor pointer is not 16-byte aligned */
+    MOK_ERR_WORKSPACE = -4,  /* workspace missing, misaligned or too small */
+    MOK_ERR_CUDA = -5,       /* a CUDA runtime/driver call failed; see mok_last_cuda_error() */
+    MOK_ERR_TIMEOUT = -6,    /* device side: a bounded wait inside a kernel ran out (reported by mok_read_status) */
+    MOK_ERR_SCHEDULE = -7,   /* device side: the schedule failed its consistency check */
+    MOK_ERR_UNSUPPORTED = -8 /* the device is not an sm_100 part */
+} mok_status;
+
+/* Which grouped-GEMM kernel runs the expert FFNs. */
+enum {
+    MOK_IMPL_TCGEN05 = 0, /* warp-specialised persistent kernel: TMA -> smem ring -> tcgen05.mma -> TMEM (default) */
+    MOK_IMPL_SIMT = 1     /* plain shared-memory FMA kernel; slow; the on-device cross-check of the above */
+};
+
+/* Optional tuning / debugging knobs.  Zero-initialise for defaults. */
+typedef struct mok_config {
+    int32_t impl;         /* MOK_IMPL_* */
+    int32_t grid;         /* persistent grid size override for the tcgen05 kernels (0 = number of SMs).  The
+                             output bits do not depend on it (Section 3.4 "Determinism"). */
+    int32_t router_impl;  /* 0 = default, 1 = fp32 FMA router, 2 = split-bf16 tensor-core router */
+    int32_t reserved[5];
+} mok_config;
+
+/*
+ * Arguments of mok_moe_forward_ex.  Zero-initialise, then fill.  Shapes follow the paper's notation:
+ * T tokens, H hidden size (D in the paper), I expert intermediate size, E routed experts, k routes/token.
+ */
+typedef struct mok_args {
+    /* inputs */
+    const void*  x;                 /* bf16 [T, H] */
+    const float* W_router;          /* fp32 [E, H] */
+    const float* router_bias;       /* fp32 [E] or NULL: logit[t,e] += bias[e] (enters selection and weights) */
+    const void*  W_gate_up;         /* bf16 [E, 2I, H]: rows 0..I-1 = W_gate, rows I..2I-1 = W_up */
+    const void*  W_down;            /* bf16 [E, H, I] */
+    const void*  W_shared_gate_up;  /* bf16 [2*I_shared, H] or NULL */
+    const void*  W_shared_down;     /* bf16 [H, I_shared]   or NULL */
+    int32_t T, H, I, I_shared, E, k;
+    /* output */
+    void* out;                      /* bf16 [T, H] */
+    /* scratch, caller-owned: >= mok_workspace_bytes(...) bytes, 256-byte aligned.  Its contents are
+       undefined between calls; calls that share a workspace must not overlap on the device. */
+    void*  workspace;
+    size_t workspace_bytes;
+    /* optional stage outputs (NULL = not wanted); written by the same enqueued work */
+    int32_t* topk_idx;   /* [T, k]  selected experts, descending logit, ties to the lowest id */
+    float*   topk_w;     /* [T, k]  normalised router weights (sum to 1 per token) */
+    int32_t* counts;     /* [E]     routes per expert */
+    int32_t* offsets;    /* [E+1]   exclusive prefix sum of counts (unpadded) */
+    int32_t* perm;       /* [T*k]   route id (t*k+s) at dispatch-buffer position p: Algorithm 1's table for one rank */
+    int32_t* inv_perm;   /* [T*k]   inverse of perm */
+    const mok_config* config;       /* NULL = defaults */
+    void* stream;
+} mok_args;
+
+/*
+ * The MoE layer forward (Section 2.1 equation; Figure 1).  out[t,:] = f_shared(x[t]) + sum_s w[t,s] f_{idx[t,s]}(x[t]).
+ * Scores are softmax over all E router logits, the k largest are selected (ties to the lowest expert id) and
+ * renormalised.  I_shared == 0 <=> both shared pointers NULL.  T == 0 returns MOK_OK without launching.
+ * Uses a library-owned per-device workspace that grows on demand with cudaMalloc (so the first call for a
+ * new size is not capturable and not thread-safe); use mok_moe_forward_ex to supply your own.
+ */
+int mok_moe_forward(const void* x, const float* W_router,
+                    const void* W_gate_up, const void* W_down,
+                    const void* W_shared_gate_up, const void* W_shared_down,
+                    int T, int H, int I, int I_shared, int E, int k,
+                    void* out, void* stream);
+
+/* Bytes of scratch mok_moe_forward_ex needs for these sizes (0 if the sizes are invalid). */
+size_t mok_workspace_bytes(int T, int H, int I, int I_shared, int E, int k);
+
+/* Same layer with a router bias, caller-owned workspace, stage outputs and knobs (see mok_args). */
+int mok_moe_forward_ex(const mok_args* args);
+
+/*
+ * Same layer with the activations in HOST memory: x_host (bf16 [T,H]) is copied to the device, the layer
+ * runs, and out_host (bf16 [T,H]) is copied back; the call returns after the result has arrived (it
+ * synchronises `stream`).  Pinned host buffers make the copies asynchronous DMA.  Weights, bias and
+ * workspace stay DEVICE pointers as in mok_args; args->x and args->out are ignored.  The workspace must
+ * have mok_workspace_bytes(...) + 2 * T*H*2 bytes (the staging copies of x and out live at its end).
+ */
+int mok_moe_forward_host(const mok_args* args, const void* x_host, void* out_host);
+
+/*
+ * Stage entry points (used by tests and profiling; each is the corresponding step of mok_moe_forward_ex).
+ *   mok_route    : router projection + top-k + weights (Section 2.1)          -> topk_idx [T,k], topk_w [T,k]
+ *   mok_schedule : Algorithm 1 for one rank from topk_idx [T*k]               -> counts, offsets, perm, inv_perm
+ * `workspace` as for mok_moe_forward_ex (same size query).
+ */
+int mok_route(const void* x, const float* W_router, const float* router_bias, int T, int H, int E, int k,
+              int32_t* topk_idx, float* topk_w, void* workspace, size_t workspace_bytes,
+              const mok_config* config, void* stream);
+int mok_schedule(const int32_t* topk_idx, int T, int E, int k,
+                 int32_t* counts, int32_t* offsets, int32_t* perm, int32_t* inv_perm,
+                 void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Reads the device-side status word of a workspace after synchronising `stream` -- the only call besides
+ * mok_moe_forward_host that blocks the host.  Returns MOK_OK, MOK_ERR_TIMEOUT or MOK_ERR_SCHEDULE
+ * (or MOK_ERR_CUDA if the stream itself is in error).
+ */
+int mok_read_status(const void* workspace, void* stream);
+
+/* Number of kernels (and memset nodes) one mok_moe_forward_ex call enqueues for these arguments; 0 on bad sizes. */
+int mok_launch_count(int T, int H, int I, int I_shared, int E, int k, const mok_config* config);
+
+int mok_last_cuda_error(void);          /* cudaError_t of the most recent failed CUDA call on this thread */
+const char* mok_status_string(int status);
+int mok_version(void);                  /* major*10000 + minor*100 + patch */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MOK_H_ */

@@ -1,0 +1,375 @@
+// Grouped expert GEMMs on the 5th-generation tensor cores (paper, Section 2.1: f_i(x) = W_down(phi(W_gate x) .* W_up x);
+// Section 3.2: expert FFNs run as persistent, fused kernels that keep the tensor cores fed by pipelining operands).
+//
+// One persistent CTA per SM, 192 threads, warp-specialised:
+//   warp 0      TMA producer : A tile [128 x 64] and B tile [256 x 64] (bf16, 128-byte swizzle) -> 4-stage smem ring
+//   warp 1      MMA issuer   : tcgen05.mma.cta_group::1.kind::f16, M=128 N=256 K=16, fp32 accumulators in TMEM
+//                              (2 accumulator stages x 256 columns = all 512 TMEM columns)
+//   warps 2..5  epilogue     : tcgen05.ld -> registers -> (SwiGLU) -> bf16 -> global
+// Tiles are handed out statically (tile L -> CTA L mod grid) in the order expert-major, then N tile, then M tile,
+// so that CTAs running side by side share the same weight tile through L2 and an expert's activations stay L2
+// resident while its N tiles stream.  The tile tables come from the on-device schedule; nothing is read back.
+// Every output element is produced by exactly one tile with a fixed k order, so results do not depend on the
+// grid size or on timing (Section 3.4 "Determinism").
+//
+//   SWIGLU : B = [E, 2N, K]; the 256-wide B tile is 128 gate rows followed by the matching 128 up rows and the
+//            epilogue writes C[:, n*128 .. n*128+127] = silu(gate) * up.
+//   else   : B = [E, N, K]; C[:, n*256 .. n*256+255] = A . B^T.
+// All mbarrier waits are bounded: on a timeout the CTA records MOK_ERR_TIMEOUT and leaves cleanly.
+#include "mok_internal.cuh"
+
+namespace mok {
+namespace tc {
+
+constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4, UMMA_K = 16;
+constexpr int A_BYTES = BM * BK * 2;           // 16 KB
+constexpr int B_BYTES = BN * BK * 2;           // 32 KB
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES; // 48 KB
+constexpr int ACC_STAGES = 2, TMEM_COLS = 512;
+constexpr int THREADS = 192;
+constexpr int SMEM_CTRL = 256;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + SMEM_CTRL + 1024;   // + slack for 1024-byte alignment
+constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;            // 2 s
+
+struct Ctrl {
+    uint64_t full[STAGES];
+    uint64_t empty[STAGES];
+    uint64_t tfull[ACC_STAGES];
+    uint64_t tempty[ACC_STAGES];
+    uint32_t tmem_base;
+    uint32_t abort;
+};
+static_assert(sizeof(Ctrl) <= SMEM_CTRL, "control block too large");
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ unsigned long long globaltimer() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false if the CTA is aborting (this or another thread ran out of time).
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                            WsHeader* hdr, int site) {
+    const unsigned long long t0 = globaltimer();
+    uint32_t spins = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++spins & 127u) == 0u) {
+            if (*abort_flag) return false;
+            if (globaltimer() - t0 > WAIT_LIMIT_NS) {
+                *abort_flag = 1u;
+                atomicCAS(&hdr->status, 0, (int)MOK_ERR_TIMEOUT);
+                hdr->where = site;
+                return false;
+            }
+        }
+    }
+    return true;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                          WsHeader* hdr, int site) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, abort_flag, hdr, site);
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]^T, M=128, N=256, K=16, bf16 inputs, fp32 accumulate.
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// 32 lanes x 32 consecutive fp32 columns: thread i of the warp gets lane (base + i), registers = columns.
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor for a K-major bf16 tile whose rows are 128 bytes (64 elements) with the
+// 128-byte swizzle: 8-row groups are 1024 bytes apart (stride byte offset); the leading byte offset is unused.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3FFFFu) >> 4);          // start address, 16-byte units
+    d |= (uint64_t)1 << 16;                           // leading byte offset (ignored for swizzled K-major)
+    d |= (uint64_t)(1024 >> 4) << 32;                 // stride byte offset
+    d |= (uint64_t)1 << 46;                           // descriptor version (sm_100)
+    d |= (uint64_t)2 << 61;                           // 128-byte swizzle
+    return d;
+}
+// Instruction descriptor: D fp32, A/B bf16, both K-major, dense, M=128, N=256.
+constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+
+struct Tile { int row0, n, e; };
+
+__device__ __forceinline__ Tile decode_tile(const GemmArgs& a, int L, int n_nt, int n_mt_total) {
+    Tile t;
+    int mt0, m_cnt;
+    if (a.dense_rows > 0) {
+        t.e = 0; mt0 = 0; m_cnt = n_mt_total;
+    } else {
+        t.e = __ldg(a.tile_expert + L / n_nt);
+        mt0 = __ldg(a.mt_start + t.e);
+        m_cnt = __ldg(a.mt_start + t.e + 1) - mt0;
+    }
+    const int r = L - n_nt * mt0;
+    t.n = r / m_cnt;
+    t.row0 = (mt0 + (r - t.n * m_cnt)) * BM;
+    return t;
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+template <bool SWIGLU>
+__global__ void __launch_bounds__(THREADS, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
+               const GemmArgs a, const int n_nt, const int k_blocks) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t* smem = smem_raw + (base - raw);
+    Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem + STAGES * STAGE_BYTES);
+    volatile uint32_t* abort_flag = &ctrl->abort;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    int n_mt_total = (a.dense_rows > 0) ? (a.dense_rows + BM - 1) / BM : *a.n_mtiles;
+    if (n_mt_total > a.max_mt) n_mt_total = a.max_mt;
+    const int total = n_mt_total * n_nt;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(smem_u32(&ctrl->full[s]), 1); mbar_init(smem_u32(&ctrl->empty[s]), 1); }
+        for (int s = 0; s < ACC_STAGES; ++s) { mbar_init(smem_u32(&ctrl->tfull[s]), 1); mbar_init(smem_u32(&ctrl->tempty[s]), 128); }
+        ctrl->abort = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&ctrl->tmem_base)), "r"((uint32_t)TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = ctrl->tmem_base;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            int s = 0;
+            uint32_t ph = 0;
+            const int b_rows_per_expert = (SWIGLU ? 2 : 1) * a.N;
+            for (int L = blockIdx.x; L < total; L += gridDim.x) {
+                const Tile t = decode_tile(a, L, n_nt, n_mt_total);
+                const int brow0 = t.e * b_rows_per_expert + (SWIGLU ? t.n * (BN / 2) : t.n * BN);
+                const int brow1 = SWIGLU ? brow0 + a.N : brow0 + BN / 2;
+                bool ok = true;
+                for (int kb = 0; kb < k_blocks; ++kb) {
+                    ok = mbar_wait(smem_u32(&ctrl->empty[s]), ph ^ 1u, abort_flag, a.header, 1);
+                    if (!ok) break;
+                    const uint32_t full = smem_u32(&ctrl->full[s]);
+                    const uint32_t sa = base + s * STAGE_BYTES, sb = sa + A_BYTES;
+                    mbar_expect_tx(full, STAGE_BYTES);
+                    tma_load_2d(sa, &tmapA, full, kb * BK, t.row0);
+                    tma_load_2d(sb, &tmapB, full, kb * BK, brow0);
+                    tma_load_2d(sb + B_BYTES / 2, &tmapB, full, kb * BK, brow1);
+                    if (++s == STAGES) { s = 0; ph ^= 1u; }
+                }
+                if (!ok) break;
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            int s = 0, as = 0;
+            uint32_t ph = 0, aph = 0;
+            for (int L = blockIdx.x; L < total; L += gridDim.x) {
+                bool ok = mbar_wait(smem_u32(&ctrl->tempty[as]), aph ^ 1u, abort_flag, a.header, 2);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(as * BN);
+                for (int kb = 0; kb < k_blocks; ++kb) {
+                    ok = mbar_wait(smem_u32(&ctrl->full[s]), ph, abort_flag, a.header, 3);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t sa = base + s * STAGE_BYTES, sb = sa + A_BYTES;
+                    const uint64_t adesc = make_smem_desc(sa), bdesc = make_smem_desc(sb);
+#pragma unroll
+                    for (int j = 0; j < BK / UMMA_K; ++j)   // +32 bytes per K=16 step inside the 128-byte swizzle row
+                        tc_mma(d_tmem, adesc + (uint64_t)(j * 2), bdesc + (uint64_t)(j * 2), IDESC, (kb | j) ? 1u : 0u);
+                    tc_commit(smem_u32(&ctrl->empty[s]));     // frees the smem stage when these MMAs retire
+                    if (++s == STAGES) { s = 0; ph ^= 1u; }
+                }
+                if (!ok) break;
+                tc_commit(smem_u32(&ctrl->tfull[as]));        // accumulator complete
+                if (++as == ACC_STAGES) { as = 0; aph ^= 1u; }
+            }
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------------------ epilogue (warps 2..5)
+        const int quad = warp & 3;                            // TMEM lane quadrant this warp may access
+        int as = 0;
+        uint32_t aph = 0;
+        for (int L = blockIdx.x; L < total; L += gridDim.x) {
+            const Tile t = decode_tile(a, L, n_nt, n_mt_total);
+            bool ok = mbar_wait(smem_u32(&ctrl->tfull[as]), aph, abort_flag, a.header, 4);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(as * BN);
+            __nv_bfloat16* crow = a.C + (size_t)(t.row0 + quad * 32 + lane) * a.N;
+            if (SWIGLU) {
+                const int c0 = t.n * (BN / 2);
+#pragma unroll 1
+                for (int c = 0; c < BN / 2; c += 32) {
+                    uint32_t g[32], u[32];
+                    tc_ld32(taddr + c, g);
+                    tc_ld32(taddr + BN / 2 + c, u);
+                    tc_wait_ld();
+                    uint32_t o[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        float g0 = __uint_as_float(g[2 * i]), g1 = __uint_as_float(g[2 * i + 1]);
+                        float h0 = (g0 / (1.f + __expf(-g0))) * __uint_as_float(u[2 * i]);
+                        float h1 = (g1 / (1.f + __expf(-g1))) * __uint_as_float(u[2 * i + 1]);
+                        o[i] = pack_bf16(h0, h1);
+                    }
+#pragma unroll
+                    for (int v = 0; v < 4; ++v) {
+                        const int col = c0 + c + v * 8;
+                        if (col < a.N)
+                            *reinterpret_cast<uint4*>(crow + col) = make_uint4(o[4 * v], o[4 * v + 1], o[4 * v + 2], o[4 * v + 3]);
+                    }
+                }
+            } else {
+                const int c0 = t.n * BN;
+#pragma unroll 1
+                for (int c = 0; c < BN; c += 32) {
+                    uint32_t r[32];
+                    tc_ld32(taddr + c, r);
+                    tc_wait_ld();
+                    uint32_t o[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) o[i] = pack_bf16(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
+#pragma unroll
+                    for (int v = 0; v < 4; ++v) {
+                        const int col = c0 + c + v * 8;
+                        if (col < a.N)
+                            *reinterpret_cast<uint4*>(crow + col) = make_uint4(o[4 * v], o[4 * v + 1], o[4 * v + 2], o[4 * v + 3]);
+                    }
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(smem_u32(&ctrl->tempty[as]));
+            if (++as == ACC_STAGES) { as = 0; aph ^= 1u; }
+        }
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    if (*abort_flag) {   // failure path only: give copies and MMAs already in flight time to land before leaving
+        const unsigned long long t0 = globaltimer();
+        while (globaltimer() - t0 < 200000ull) { }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS) : "memory");
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn get_encode() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// 2D bf16 row-major tensor [rows, cols] -> tensor map with a [box_rows x 64] box and 128-byte swizzle.
+static bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+    EncodeTiledFn enc = get_encode();
+    if (!enc) return false;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols * 2};
+    cuuint32_t box[2] = {(cuuint32_t)BK, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace tc
+
+cudaError_t launch_gemm_tc(const GemmArgs& a, bool swiglu, int grid, cudaStream_t s) {
+    using namespace tc;
+    CUtensorMap mA, mB;
+    const uint64_t b_rows = (uint64_t)a.E * (swiglu ? 2 : 1) * a.N;
+    if (!make_map(&mA, a.A, (uint64_t)a.a_rows, (uint64_t)a.K, BM)) return cudaErrorInvalidValue;
+    if (!make_map(&mB, a.B, b_rows, (uint64_t)a.K, BN / 2)) return cudaErrorInvalidValue;
+    const int n_nt = swiglu ? (a.N + BN / 2 - 1) / (BN / 2) : (a.N + BN - 1) / BN;
+    const int k_blocks = (a.K + BK - 1) / BK;
+    static int sm_count = 0;
+    if (!sm_count) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
+        cudaFuncSetAttribute(gemm_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+        cudaFuncSetAttribute(gemm_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    }
+    if (grid <= 0 || grid > sm_count) grid = sm_count;
+    if (swiglu) gemm_tc_kernel<true><<<grid, THREADS, SMEM_BYTES, s>>>(mA, mB, a, n_nt, k_blocks);
+    else gemm_tc_kernel<false><<<grid, THREADS, SMEM_BYTES, s>>>(mA, mB, a, n_nt, k_blocks);
+    return cudaGetLastError();
+}
+
+}  // namespace mok

@@ -1,0 +1,300 @@
+// Host side of libmok: argument validation, workspace layout and the launch sequence of the MoE layer forward
+// (paper, Figure 1: router projection + top-k, dispatch scheduling, then dispatch / expert FFNs / combine).
+// Nothing here synchronises with the device or reads counts back (Section 3.3), except mok_read_status and
+// mok_moe_forward_host, which say so.
+#include "mok_internal.cuh"
+#include <string.h>
+
+namespace mok {
+
+static thread_local int g_last_cuda_error = 0;
+
+static int cuda_fail(cudaError_t e) {
+    g_last_cuda_error = (int)e;
+    return MOK_ERR_CUDA;
+}
+
+static bool sizes_ok(int T, int H, int I, int Is, int E, int k) {
+    if (T < 0 || H <= 0 || I <= 0 || Is < 0 || E <= 0 || k < 1) return false;
+    if (k > E || k > MAX_K || E > MAX_E) return false;
+    if ((H % 8) || (I % 8) || (Is % 8)) return false;
+    if ((long long)T * k >= (1ll << 31) / 256) return false;
+    return true;
+}
+
+bool ws_layout(int T, int H, int I, int Is, int E, int k, WsLayout* L) {
+    if (!sizes_ok(T, H, I, Is, E, k)) return false;
+    memset(L, 0, sizeof(*L));
+    const long long R = (long long)T * k;
+    const long long nonempty_max = R < E ? R : E;
+    long long Rpad = (R + nonempty_max * (TILE_M - 1) + TILE_M - 1) / TILE_M * TILE_M;
+    if (Rpad < TILE_M) Rpad = TILE_M;
+    L->R = (int32_t)R;
+    L->Rpad = (int32_t)Rpad;
+    L->max_mt = (int32_t)(Rpad / TILE_M);
+    L->Tpad = (T + TILE_M - 1) / TILE_M * TILE_M;
+    if (L->Tpad < TILE_M) L->Tpad = TILE_M;
+    L->n_blk = (int32_t)((R + SCHED_CHUNK - 1) / SCHED_CHUNK);
+    if (L->n_blk < 1) L->n_blk = 1;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    L->header = take(sizeof(WsHeader));
+    L->idx = take(sizeof(int32_t) * (size_t)(R > 0 ? R : 1));
+    L->w = take(sizeof(float) * (size_t)(R > 0 ? R : 1));
+    L->counts = take(sizeof(int32_t) * E);
+    L->offsets = take(sizeof(int32_t) * (E + 1));
+    L->pad_offsets = take(sizeof(int32_t) * (E + 1));
+    L->mt_start = take(sizeof(int32_t) * (E + 1));
+    L->tile_expert = take(sizeof(int32_t) * (size_t)L->max_mt);
+    L->perm = take(sizeof(int32_t) * (size_t)(R > 0 ? R : 1));
+    L->inv = take(sizeof(int32_t) * (size_t)(R > 0 ? R : 1));
+    L->pos = take(sizeof(int32_t) * (size_t)(R > 0 ? R : 1));
+    L->blk_hist = take(sizeof(int32_t) * (size_t)L->n_blk * E);
+    L->wr_split = take(2 * (size_t)3 * E * H);
+    L->logits = take(sizeof(float) * (size_t)L->Tpad * 3 * E);
+    L->xg = take(2 * (size_t)Rpad * H);
+    L->h = take(2 * (size_t)Rpad * I);
+    L->y = take(2 * (size_t)Rpad * H);
+    L->hs = take(Is > 0 ? 2 * (size_t)L->Tpad * Is : 0);
+    L->ysh = take(Is > 0 ? 2 * (size_t)L->Tpad * H : 0);
+    L->total = off;
+    return true;
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static int validate(const mok_args* a, WsLayout* L, size_t extra_ws) {
+    if (!a) return MOK_ERR_NULL;
+    if (!ws_layout(a->T, a->H, a->I, a->I_shared, a->E, a->k, L)) return MOK_ERR_SHAPE;
+    if ((a->I_shared > 0) != (a->W_shared_gate_up != nullptr) || (a->I_shared > 0) != (a->W_shared_down != nullptr))
+        return MOK_ERR_SHAPE;
+    if (a->T == 0) return MOK_OK;
+    if (!a->W_router || !a->W_gate_up || !a->W_down) return MOK_ERR_NULL;
+    if (!aligned16(a->W_router) || !aligned16(a->W_gate_up) || !aligned16(a->W_down) ||
+        !aligned16(a->W_shared_gate_up) || !aligned16(a->W_shared_down))
+        return MOK_ERR_ALIGN;
+    if (!a->workspace || (reinterpret_cast<uintptr_t>(a->workspace) & 255u) || a->workspace_bytes < L->total + extra_ws)
+        return MOK_ERR_WORKSPACE;
+    if (a->config && (a->config->impl < 0 || a->config->impl > 1 || a->config->grid < 0)) return MOK_ERR_SHAPE;
+    return MOK_OK;
+}
+
+static int run_gemm(const GemmArgs& g, bool swiglu, const mok_config* cfg, cudaStream_t s) {
+    cudaError_t e = (cfg && cfg->impl == MOK_IMPL_SIMT) ? launch_gemm_simt(g, swiglu, s)
+                                                          : launch_gemm_tc(g, swiglu, cfg ? cfg->grid : 0, s);
+    return e == cudaSuccess ? MOK_OK : cuda_fail(e);
+}
+
+static int route_stage(const mok_args* a, const WsLayout& L, char* ws, const __nv_bfloat16* x, cudaStream_t s) {
+    int32_t* idx = reinterpret_cast<int32_t*>(ws + L.idx);
+    float* w = reinterpret_cast<float*>(ws + L.w);
+    cudaError_t e = launch_router_simt(x, a->W_router, a->router_bias, a->T, a->H, a->E, a->k, idx, w, s);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (a->topk_idx) {
+        e = cudaMemcpyAsync(a->topk_idx, idx, sizeof(int32_t) * (size_t)L.R, cudaMemcpyDeviceToDevice, s);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    if (a->topk_w) {
+        e = cudaMemcpyAsync(a->topk_w, w, sizeof(float) * (size_t)L.R, cudaMemcpyDeviceToDevice, s);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    return MOK_OK;
+}
+
+// The whole layer on device pointers.  x / out may differ from a->x / a->out (host-buffer variant).
+static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloat16* x, __nv_bfloat16* out) {
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(a->stream);
+    char* ws = reinterpret_cast<char*>(a->workspace);
+    WsHeader* hdr = reinterpret_cast<WsHeader*>(ws + L.header);
+    cudaError_t e = cudaMemsetAsync(hdr, 0, sizeof(WsHeader), s);
+    if (e != cudaSuccess) return cuda_fail(e);
+    int rc = route_stage(a, L, ws, x, s);
+    if (rc) return rc;
+    e = launch_schedule(reinterpret_cast<const int32_t*>(ws + L.idx), a->T, a->E, a->k, L, ws,
+                        a->counts, a->offsets, a->perm, a->inv_perm, s);
+    if (e != cudaSuccess) return cuda_fail(e);
+    e = launch_gather(x, a->H, a->k, L, ws, s);
+    if (e != cudaSuccess) return cuda_fail(e);
+
+    GemmArgs g;
+    memset(&g, 0, sizeof(g));
+    g.header = hdr;
+    g.n_mtiles = &hdr->n_mtiles;
+    g.tile_expert = reinterpret_cast<const int32_t*>(ws + L.tile_expert);
+    g.mt_start = reinterpret_cast<const int32_t*>(ws + L.mt_start);
+    g.max_mt = L.max_mt;
+    // routed experts: h = silu(Xg Wg^T) * (Xg Wu^T);  y = h Wd^T
+    g.A = reinterpret_cast<const __nv_bfloat16*>(ws + L.xg);
+    g.B = reinterpret_cast<const __nv_bfloat16*>(a->W_gate_up);
+    g.C = reinterpret_cast<__nv_bfloat16*>(ws + L.h);
+    g.K = a->H; g.N = a->I; g.E = a->E; g.rows_pad = L.Rpad; g.a_rows = L.Rpad; g.dense_rows = 0;
+    if ((rc = run_gemm(g, true, a->config, s))) return rc;
+    g.A = reinterpret_cast<const __nv_bfloat16*>(ws + L.h);
+    g.B = reinterpret_cast<const __nv_bfloat16*>(a->W_down);
+    g.C = reinterpret_cast<__nv_bfloat16*>(ws + L.y);
+    g.K = a->I; g.N = a->H;
+    if ((rc = run_gemm(g, false, a->config, s))) return rc;
+    if (a->I_shared > 0) {   // shared expert: every token in natural order, no gather
+        g.A = x;
+        g.B = reinterpret_cast<const __nv_bfloat16*>(a->W_shared_gate_up);
+        g.C = reinterpret_cast<__nv_bfloat16*>(ws + L.hs);
+        g.K = a->H; g.N = a->I_shared; g.E = 1; g.rows_pad = L.Tpad; g.a_rows = a->T; g.dense_rows = a->T;
+        if ((rc = run_gemm(g, true, a->config, s))) return rc;
+        g.A = reinterpret_cast<const __nv_bfloat16*>(ws + L.hs);
+        g.B = reinterpret_cast<const __nv_bfloat16*>(a->W_shared_down);
+        g.C = reinterpret_cast<__nv_bfloat16*>(ws + L.ysh);
+        g.K = a->I_shared; g.N = a->H; g.a_rows = L.Tpad;
+        if ((rc = run_gemm(g, false, a->config, s))) return rc;
+    }
+    e = launch_combine(L, ws, a->T, a->H, a->k, a->I_shared > 0, out, s);
+    return e == cudaSuccess ? MOK_OK : cuda_fail(e);
+}
+
+// Library-owned workspace of mok_moe_forward, one per device, grown on demand.
+struct OwnedWs { void* ptr; size_t bytes; };
+static OwnedWs g_owned[64];
+
+}  // namespace mok
+
+using namespace mok;
+
+extern "C" {
+
+size_t mok_workspace_bytes(int T, int H, int I, int I_shared, int E, int k) {
+    WsLayout L;
+    return ws_layout(T, H, I, I_shared, E, k, &L) ? L.total : 0;
+}
+
+int mok_moe_forward_ex(const mok_args* a) {
+    WsLayout L;
+    int rc = validate(a, &L, 0);
+    if (rc || a->T == 0) return rc;
+    if (!a->x || !a->out) return MOK_ERR_NULL;
+    if (!aligned16(a->x) || !aligned16(a->out)) return MOK_ERR_ALIGN;
+    return forward_device(a, L, reinterpret_cast<const __nv_bfloat16*>(a->x), reinterpret_cast<__nv_bfloat16*>(a->out));
+}
+
+int mok_moe_forward_host(const mok_args* a, const void* x_host, void* out_host) {
+    WsLayout L;
+    if (!a) return MOK_ERR_NULL;
+    const size_t act = 2 * (size_t)(a->T > 0 ? a->T : 0) * (size_t)(a->H > 0 ? a->H : 0);
+    const size_t act_al = align_up(act, 256);
+    int rc = validate(a, &L, 2 * act_al);
+    if (rc || a->T == 0) return rc;
+    if (!x_host || !out_host) return MOK_ERR_NULL;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(a->stream);
+    char* ws = reinterpret_cast<char*>(a->workspace);
+    __nv_bfloat16* xd = reinterpret_cast<__nv_bfloat16*>(ws + L.total);
+    __nv_bfloat16* od = reinterpret_cast<__nv_bfloat16*>(ws + L.total + act_al);
+    cudaError_t e = cudaMemcpyAsync(xd, x_host, act, cudaMemcpyHostToDevice, s);
+    if (e != cudaSuccess) return cuda_fail(e);
+    rc = forward_device(a, L, xd, od);
+    if (rc) return rc;
+    e = cudaMemcpyAsync(out_host, od, act, cudaMemcpyDeviceToHost, s);
+    if (e != cudaSuccess) return cuda_fail(e);
+    e = cudaStreamSynchronize(s);
+    return e == cudaSuccess ? MOK_OK : cuda_fail(e);
+}
+
+int mok_moe_forward(const void* x, const float* W_router, const void* W_gate_up, const void* W_down,
+                    const void* W_shared_gate_up, const void* W_shared_down,
+                    int T, int H, int I, int I_shared, int E, int k, void* out, void* stream) {
+    WsLayout L;
+    if (!ws_layout(T, H, I, I_shared, E, k, &L)) return MOK_ERR_SHAPE;
+    if (T == 0) return MOK_OK;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (dev < 0 || dev >= 64) return MOK_ERR_UNSUPPORTED;
+    OwnedWs& o = g_owned[dev];
+    if (o.bytes < L.total) {
+        if (o.ptr) {
+            e = cudaStreamSynchronize(reinterpret_cast<cudaStream_t>(stream));
+            if (e != cudaSuccess) return cuda_fail(e);
+            cudaFree(o.ptr);
+            o.ptr = nullptr;
+            o.bytes = 0;
+        }
+        e = cudaMalloc(&o.ptr, L.total);
+        if (e != cudaSuccess) { o.ptr = nullptr; return cuda_fail(e); }
+        o.bytes = L.total;
+    }
+    mok_args a;
+    memset(&a, 0, sizeof(a));
+    a.x = x; a.W_router = W_router; a.W_gate_up = W_gate_up; a.W_down = W_down;
+    a.W_shared_gate_up = W_shared_gate_up; a.W_shared_down = W_shared_down;
+    a.T = T; a.H = H; a.I = I; a.I_shared = I_shared; a.E = E; a.k = k;
+    a.out = out; a.workspace = o.ptr; a.workspace_bytes = o.bytes; a.stream = stream;
+    return mok_moe_forward_ex(&a);
+}
+
+int mok_route(const void* x, const float* W_router, const float* router_bias, int T, int H, int E, int k,
+              int32_t* topk_idx, float* topk_w, void* workspace, size_t workspace_bytes,
+              const mok_config* config, void* stream) {
+    WsLayout L;
+    if (!ws_layout(T, H, 8, 0, E, k, &L)) return MOK_ERR_SHAPE;
+    if (T == 0) return MOK_OK;
+    if (!x || !W_router || !topk_idx || !topk_w) return MOK_ERR_NULL;
+    if (!aligned16(x) || !aligned16(W_router)) return MOK_ERR_ALIGN;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < L.total) return MOK_ERR_WORKSPACE;
+    mok_args a;
+    memset(&a, 0, sizeof(a));
+    a.W_router = W_router; a.router_bias = router_bias; a.T = T; a.H = H; a.E = E; a.k = k;
+    a.topk_idx = topk_idx; a.topk_w = topk_w; a.config = config;
+    return route_stage(&a, L, reinterpret_cast<char*>(workspace), reinterpret_cast<const __nv_bfloat16*>(x),
+                       reinterpret_cast<cudaStream_t>(stream));
+}
+
+int mok_schedule(const int32_t* topk_idx, int T, int E, int k, int32_t* counts, int32_t* offsets, int32_t* perm,
+                 int32_t* inv_perm, void* workspace, size_t workspace_bytes, void* stream) {
+    WsLayout L;
+    if (!ws_layout(T, 8, 8, 0, E, k, &L)) return MOK_ERR_SHAPE;
+    if (T == 0) return MOK_OK;
+    if (!topk_idx) return MOK_ERR_NULL;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < L.total) return MOK_ERR_WORKSPACE;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    char* ws = reinterpret_cast<char*>(workspace);
+    cudaError_t e = cudaMemsetAsync(ws + L.header, 0, sizeof(WsHeader), s);
+    if (e != cudaSuccess) return cuda_fail(e);
+    e = launch_schedule(topk_idx, T, E, k, L, ws, counts, offsets, perm, inv_perm, s);
+    return e == cudaSuccess ? MOK_OK : cuda_fail(e);
+}
+
+int mok_read_status(const void* workspace, void* stream) {
+    if (!workspace) return MOK_ERR_NULL;
+    cudaError_t e = cudaStreamSynchronize(reinterpret_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(e);
+    WsHeader h;
+    e = cudaMemcpy(&h, workspace, sizeof(h), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(e);
+    return h.status;
+}
+
+int mok_launch_count(int T, int H, int I, int I_shared, int E, int k, const mok_config* config) {
+    WsLayout L;
+    (void)config;
+    if (!ws_layout(T, H, I, I_shared, E, k, &L) || T == 0) return 0;
+    // header memset, router, 3 schedule kernels, gather, 2 routed GEMMs, (2 shared GEMMs), combine
+    return 1 + 1 + 3 + 1 + 2 + (I_shared > 0 ? 2 : 0) + 1;
+}
+
+int mok_last_cuda_error(void) { return g_last_cuda_error; }
+
+const char* mok_status_string(int status) {
+    switch (status) {
+        case MOK_OK: return "ok";
+        case MOK_ERR_NULL: return "a required pointer is NULL";
+        case MOK_ERR_SHAPE: return "unsupported or inconsistent sizes";
+        case MOK_ERR_ALIGN: return "a tensor pointer is not 16-byte aligned";
+        case MOK_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case MOK_ERR_CUDA: return "a CUDA call failed";
+        case MOK_ERR_TIMEOUT: return "a bounded wait inside a kernel ran out";
+        case MOK_ERR_SCHEDULE: return "the dispatch schedule failed its consistency check";
+        case MOK_ERR_UNSUPPORTED: return "unsupported device";
+        default: return "unknown status";
+    }
+}
+
+int mok_version(void) { return 100; }
+
+}  // extern "C"

@@ -1,0 +1,74 @@
+// Internal declarations shared by the translation units of libmok (not part of the public ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <cuda.h>
+#include <stdint.h>
+#include <stddef.h>
+#include "mok.h"
+
+namespace mok {
+
+constexpr int TILE_M = 128;          // rows of one GEMM tile; expert segments are padded to this internally
+constexpr int SCHED_CHUNK = 2048;    // routes handled by one block of the schedule kernels
+constexpr int MAX_E = 512;
+constexpr int MAX_K = 32;
+
+// Device-side control block at the start of the workspace (one 256-byte slot).
+struct WsHeader {
+    int32_t status;        // 0 or a negative mok_status written by a kernel
+    int32_t n_mtiles;      // number of 128-row tiles of the padded dispatch buffer (written by the schedule)
+    int32_t where;         // diagnostic: which wait gave up (role * 1000 + site)
+    int32_t pad[61];
+};
+
+// Byte offsets of every workspace region, computed on the host from the sizes alone (no readback).
+struct WsLayout {
+    size_t header, idx, w, counts, offsets, pad_offsets, mt_start, tile_expert, perm, inv, pos, blk_hist;
+    size_t wr_split;      // bf16 [3E, H]: W_r split into hi/mid/lo parts for the tensor-core router
+    size_t logits;        // fp32 [T, 3E] partial logits of the tensor-core router
+    size_t xg, h, y, hs, ysh;
+    size_t total;
+    int32_t R;            // T*k
+    int32_t Rpad;         // upper bound on padded rows (multiple of 128)
+    int32_t max_mt;       // Rpad / 128
+    int32_t Tpad;         // T rounded up to 128
+    int32_t n_blk;        // schedule blocks
+};
+
+bool ws_layout(int T, int H, int I, int Is, int E, int k, WsLayout* L);
+
+// Arguments of the grouped GEMM (both implementations).  Rows live in a padded space: expert e owns rows
+// [128*mt_start[e], 128*mt_start[e+1]); tile q belongs to expert tile_expert[q].  In dense mode (shared
+// expert) there is one expert and ceil(dense_rows/128) tiles.
+struct GemmArgs {
+    const __nv_bfloat16* A;      // [rows_pad, K]
+    const __nv_bfloat16* B;      // SWIGLU: [E, 2*N, K] (gate rows then up rows); else [E, N, K]
+    __nv_bfloat16* C;            // [rows_pad, N]
+    int32_t K, N, E;
+    int32_t rows_pad;            // allocated rows of C (multiple of 128)
+    int32_t a_rows;              // allocated rows of A (reads beyond it are treated as zero)
+    int32_t dense_rows;          // > 0: dense mode with this many valid rows
+    const int32_t* n_mtiles;     // device (routed mode)
+    const int32_t* tile_expert;  // device [max_mt]
+    const int32_t* mt_start;     // device [E+1]
+    int32_t max_mt;
+    WsHeader* header;
+};
+
+// kernels' host launchers (each returns a cudaError_t from the launch)
+cudaError_t launch_router_simt(const __nv_bfloat16* x, const float* Wr, const float* bias, int T, int H, int E, int k,
+                               int32_t* idx, float* w, cudaStream_t s);
+cudaError_t launch_schedule(const int32_t* idx, int T, int E, int k, const WsLayout& L, char* ws,
+                            int32_t* counts_out, int32_t* offsets_out, int32_t* perm_out, int32_t* inv_out,
+                            cudaStream_t s);
+cudaError_t launch_gather(const __nv_bfloat16* x, int H, int k, const WsLayout& L, char* ws, cudaStream_t s);
+cudaError_t launch_combine(const WsLayout& L, char* ws, int T, int H, int k, bool shared, __nv_bfloat16* out,
+                           cudaStream_t s);
+cudaError_t launch_gemm_simt(const GemmArgs& a, bool swiglu, cudaStream_t s);
+cudaError_t launch_gemm_tc(const GemmArgs& a, bool swiglu, int grid, cudaStream_t s);
+int gemm_tc_launches(void);
+
+inline __host__ __device__ size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+}  // namespace mok

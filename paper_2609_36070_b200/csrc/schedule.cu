@@ -1,0 +1,162 @@
+// Dispatch schedule construction on the device: Algorithm 1 of the paper for one rank.
+//
+// With a single source rank Algorithm 1 reduces to a stable counting sort of the routes by expert:
+// M_{0,l} = counts[l], S_l = exclusive prefix sum, the ordinal o of a route is the number of earlier routes
+// to the same expert and its position is p = o, so Phi[S_l + o] = route.  Three kernels, no host readback
+// (Section 3.3), integer arithmetic only, hence bit-reproducible:
+//   1. sched_hist    per-block expert histograms of SCHED_CHUNK consecutive routes
+//   2. sched_scan    one block: per-expert prefix over blocks, counts, offsets, and the internal tile tables
+//                    (each expert's segment padded to a multiple of 128 rows: pad_offsets, mt_start, tile_expert)
+//   3. sched_scatter stable ranks inside each block (warp match + per-warp running counters) -> perm, inv, pos
+// Exported offsets/perm are unpadded; the padding is internal to the GEMM row space.
+#include "mok_internal.cuh"
+
+namespace mok {
+
+constexpr int SCHED_THREADS = 256;
+constexpr int SCHED_WARPS = SCHED_THREADS / 32;
+constexpr int ROUTES_PER_WARP = SCHED_CHUNK / SCHED_WARPS;   // contiguous routes owned by one warp
+
+__global__ void __launch_bounds__(SCHED_THREADS)
+sched_hist_kernel(const int32_t* __restrict__ a, int n, int E, int32_t* __restrict__ blk_hist) {
+    __shared__ int32_t hist[MAX_E];
+    for (int e = threadIdx.x; e < E; e += SCHED_THREADS) hist[e] = 0;
+    __syncthreads();
+    int base = blockIdx.x * SCHED_CHUNK;
+    for (int i = threadIdx.x; i < SCHED_CHUNK; i += SCHED_THREADS) {
+        int j = base + i;
+        if (j < n && (unsigned)a[j] < (unsigned)E) atomicAdd(&hist[a[j]], 1);   // integer atomics: order-independent result
+    }
+    __syncthreads();
+    for (int e = threadIdx.x; e < E; e += SCHED_THREADS) blk_hist[(size_t)blockIdx.x * E + e] = hist[e];
+}
+
+// One block of MAX_E threads.  Thread e walks the blocks for expert e (exclusive prefix, in place), then the
+// block scans over experts.
+__global__ void __launch_bounds__(MAX_E)
+sched_scan_kernel(int32_t* __restrict__ blk_hist, int n_blk, int E, int max_mt,
+                  int32_t* __restrict__ counts, int32_t* __restrict__ offsets, int32_t* __restrict__ pad_offsets,
+                  int32_t* __restrict__ mt_start, int32_t* __restrict__ tile_expert, WsHeader* __restrict__ hdr,
+                  int32_t* __restrict__ counts_out, int32_t* __restrict__ offsets_out) {
+    __shared__ int32_t s_cnt[MAX_E], s_off[MAX_E + 1], s_mt[MAX_E + 1];
+    const int e = threadIdx.x;
+    int32_t total = 0;
+    if (e < E) {
+        for (int b = 0; b < n_blk; ++b) {
+            int32_t c = blk_hist[(size_t)b * E + e];
+            blk_hist[(size_t)b * E + e] = total;
+            total += c;
+        }
+        s_cnt[e] = total;
+    }
+    __syncthreads();
+    if (e == 0) {   // E <= 512: a serial scan by one thread is a few hundred cycles
+        int32_t off = 0, mt = 0;
+        for (int i = 0; i < E; ++i) {
+            s_off[i] = off;
+            s_mt[i] = mt;
+            off += s_cnt[i];
+            mt += (s_cnt[i] + TILE_M - 1) / TILE_M;
+        }
+        s_off[E] = off;
+        s_mt[E] = mt;
+        hdr->n_mtiles = mt;
+        if (mt > max_mt) hdr->status = MOK_ERR_SCHEDULE;
+    }
+    __syncthreads();
+    if (e < E) {
+        counts[e] = s_cnt[e];
+        offsets[e] = s_off[e];
+        pad_offsets[e] = s_mt[e] * TILE_M;
+        mt_start[e] = s_mt[e];
+        if (counts_out) counts_out[e] = s_cnt[e];
+        if (offsets_out) offsets_out[e] = s_off[e];
+        for (int q = s_mt[e]; q < s_mt[e + 1] && q < max_mt; ++q) tile_expert[q] = e;
+    }
+    if (e == 0) {
+        offsets[E] = s_off[E];
+        pad_offsets[E] = s_mt[E] * TILE_M;
+        mt_start[E] = s_mt[E];
+        if (offsets_out) offsets_out[E] = s_off[E];
+    }
+}
+
+__global__ void __launch_bounds__(SCHED_THREADS)
+sched_scatter_kernel(const int32_t* __restrict__ a, int n, int E,
+                     const int32_t* __restrict__ blk_base, const int32_t* __restrict__ offsets,
+                     const int32_t* __restrict__ pad_offsets,
+                     int32_t* __restrict__ perm, int32_t* __restrict__ inv, int32_t* __restrict__ pos,
+                     int32_t* __restrict__ perm_out, int32_t* __restrict__ inv_out) {
+    extern __shared__ int32_t ssm[];                 // [SCHED_WARPS][E] running counters per warp
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    int32_t* mine = ssm + warp * E;
+    for (int e = threadIdx.x; e < SCHED_WARPS * E; e += SCHED_THREADS) ssm[e] = 0;
+    __syncthreads();
+    const int wbase = blockIdx.x * SCHED_CHUNK + warp * ROUTES_PER_WARP;
+    // pass 1: this warp's histogram over its contiguous routes
+    for (int i = 0; i < ROUTES_PER_WARP; i += 32) {
+        int j = wbase + i + lane;
+        bool valid = j < n;
+        int e = valid ? a[j] : -1 - lane;            // invalid lanes get unique keys
+        if ((unsigned)e >= (unsigned)E) { valid = false; e = -1 - lane; }
+        unsigned peers = __match_any_sync(0xffffffffu, e);
+        if (valid && lane == __ffs(peers) - 1) mine[e] += __popc(peers);
+        __syncwarp();
+    }
+    __syncthreads();
+    // warp-exclusive prefix over warps, plus the block's base for each expert -> starting rank per (warp, expert)
+    for (int e = threadIdx.x; e < E; e += SCHED_THREADS) {
+        int32_t run = blk_base[(size_t)blockIdx.x * E + e];
+        for (int wi = 0; wi < SCHED_WARPS; ++wi) {
+            int32_t c = ssm[wi * E + e];
+            ssm[wi * E + e] = run;
+            run += c;
+        }
+    }
+    __syncthreads();
+    // pass 2: ranks in route order
+    for (int i = 0; i < ROUTES_PER_WARP; i += 32) {
+        int j = wbase + i + lane;
+        bool valid = j < n;
+        int e = valid ? a[j] : -1 - lane;
+        if ((unsigned)e >= (unsigned)E) { valid = false; e = -1 - lane; }
+        unsigned peers = __match_any_sync(0xffffffffu, e);
+        int before = __popc(peers & ((1u << lane) - 1u));
+        int32_t rank = 0;
+        if (valid) rank = mine[e] + before;          // ordinal o of Algorithm 1
+        __syncwarp();
+        if (valid && lane == __ffs(peers) - 1) mine[e] += __popc(peers);
+        __syncwarp();
+        if (valid) {
+            int32_t p = offsets[e] + rank;           // Phi[S_l + o] = route j
+            perm[p] = j;
+            inv[j] = p;
+            pos[j] = pad_offsets[e] + rank;          // row in the padded GEMM space
+            if (perm_out) perm_out[p] = j;
+            if (inv_out) inv_out[j] = p;
+        }
+    }
+}
+
+cudaError_t launch_schedule(const int32_t* idx, int T, int E, int k, const WsLayout& L, char* ws,
+                            int32_t* counts_out, int32_t* offsets_out, int32_t* perm_out, int32_t* inv_out,
+                            cudaStream_t s) {
+    const int n = T * k;
+    int32_t* blk_hist = reinterpret_cast<int32_t*>(ws + L.blk_hist);
+    int32_t* counts = reinterpret_cast<int32_t*>(ws + L.counts);
+    int32_t* offsets = reinterpret_cast<int32_t*>(ws + L.offsets);
+    int32_t* pad_offsets = reinterpret_cast<int32_t*>(ws + L.pad_offsets);
+    int32_t* mt_start = reinterpret_cast<int32_t*>(ws + L.mt_start);
+    int32_t* tile_expert = reinterpret_cast<int32_t*>(ws + L.tile_expert);
+    WsHeader* hdr = reinterpret_cast<WsHeader*>(ws + L.header);
+    sched_hist_kernel<<<L.n_blk, SCHED_THREADS, 0, s>>>(idx, n, E, blk_hist);
+    sched_scan_kernel<<<1, MAX_E, 0, s>>>(blk_hist, L.n_blk, E, L.max_mt, counts, offsets, pad_offsets, mt_start,
+                                          tile_expert, hdr, counts_out, offsets_out);
+    sched_scatter_kernel<<<L.n_blk, SCHED_THREADS, sizeof(int32_t) * SCHED_WARPS * E, s>>>(
+        idx, n, E, blk_hist, offsets, pad_offsets,
+        reinterpret_cast<int32_t*>(ws + L.perm), reinterpret_cast<int32_t*>(ws + L.inv),
+        reinterpret_cast<int32_t*>(ws + L.pos), perm_out, inv_out);
+    return cudaGetLastError();
+}
+
+}  // namespace mok

@@ -1,0 +1,233 @@
+"""Thin Python binding over the C-ABI library libmok.so (see include/mok.h).
+
+Argument marshalling only: every step of the layer runs in the library's CUDA kernels.  PyTorch is used for
+device memory and streams.  Importing this module fails loudly if the library has not been built
+(`python -m paper_2609_36070_b200.build`); there is no CPU or PyTorch fallback.
+"""
+import ctypes
+import os
+
+import torch
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libmok.so")
+if not os.path.exists(_LIB_PATH):
+    raise ImportError(f"{_LIB_PATH} is missing: build it with `python -m paper_2609_36070_b200.build`")
+_lib = ctypes.CDLL(_LIB_PATH)
+
+MOK_OK = 0
+MOK_ERR_NULL, MOK_ERR_SHAPE, MOK_ERR_ALIGN, MOK_ERR_WORKSPACE = -1, -2, -3, -4
+MOK_ERR_CUDA, MOK_ERR_TIMEOUT, MOK_ERR_SCHEDULE, MOK_ERR_UNSUPPORTED = -5, -6, -7, -8
+MOK_IMPL_TCGEN05, MOK_IMPL_SIMT = 0, 1
+
+EXPORTS = ["mok_moe_forward", "mok_workspace_bytes", "mok_moe_forward_ex", "mok_moe_forward_host", "mok_route",
+           "mok_schedule", "mok_read_status", "mok_launch_count", "mok_last_cuda_error", "mok_status_string",
+           "mok_version"]
+
+
+class mok_config(ctypes.Structure):
+    _fields_ = [("impl", ctypes.c_int32), ("grid", ctypes.c_int32), ("router_impl", ctypes.c_int32),
+                ("reserved", ctypes.c_int32 * 5)]
+
+
+class mok_args(ctypes.Structure):
+    _fields_ = [("x", ctypes.c_void_p), ("W_router", ctypes.c_void_p), ("router_bias", ctypes.c_void_p),
+                ("W_gate_up", ctypes.c_void_p), ("W_down", ctypes.c_void_p),
+                ("W_shared_gate_up", ctypes.c_void_p), ("W_shared_down", ctypes.c_void_p),
+                ("T", ctypes.c_int32), ("H", ctypes.c_int32), ("I", ctypes.c_int32), ("I_shared", ctypes.c_int32),
+                ("E", ctypes.c_int32), ("k", ctypes.c_int32),
+                ("out", ctypes.c_void_p), ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
+                ("topk_idx", ctypes.c_void_p), ("topk_w", ctypes.c_void_p), ("counts", ctypes.c_void_p),
+                ("offsets", ctypes.c_void_p), ("perm", ctypes.c_void_p), ("inv_perm", ctypes.c_void_p),
+                ("config", ctypes.POINTER(mok_config)), ("stream", ctypes.c_void_p)]
+
+
+_lib.mok_workspace_bytes.restype = ctypes.c_size_t
+_lib.mok_workspace_bytes.argtypes = [ctypes.c_int] * 6
+_lib.mok_moe_forward.restype = ctypes.c_int
+_lib.mok_moe_forward.argtypes = [ctypes.c_void_p] * 6 + [ctypes.c_int] * 6 + [ctypes.c_void_p] * 2
+_lib.mok_moe_forward_ex.restype = ctypes.c_int
+_lib.mok_moe_forward_ex.argtypes = [ctypes.POINTER(mok_args)]
+_lib.mok_moe_forward_host.restype = ctypes.c_int
+_lib.mok_moe_forward_host.argtypes = [ctypes.POINTER(mok_args), ctypes.c_void_p, ctypes.c_void_p]
+_lib.mok_route.restype = ctypes.c_int
+_lib.mok_route.argtypes = ([ctypes.c_void_p] * 3 + [ctypes.c_int] * 4 + [ctypes.c_void_p] * 3 +
+                           [ctypes.c_size_t, ctypes.POINTER(mok_config), ctypes.c_void_p])
+_lib.mok_schedule.restype = ctypes.c_int
+_lib.mok_schedule.argtypes = ([ctypes.c_void_p] + [ctypes.c_int] * 3 + [ctypes.c_void_p] * 5 +
+                              [ctypes.c_size_t, ctypes.c_void_p])
+_lib.mok_read_status.restype = ctypes.c_int
+_lib.mok_read_status.argtypes = [ctypes.c_void_p, ctypes.c_void_p]
+_lib.mok_launch_count.restype = ctypes.c_int
+_lib.mok_launch_count.argtypes = [ctypes.c_int] * 6 + [ctypes.POINTER(mok_config)]
+_lib.mok_last_cuda_error.restype = ctypes.c_int
+_lib.mok_status_string.restype = ctypes.c_char_p
+_lib.mok_status_string.argtypes = [ctypes.c_int]
+_lib.mok_version.restype = ctypes.c_int
+
+
+class MokError(RuntimeError):
+    def __init__(self, status):
+        self.status = status
+        msg = _lib.mok_status_string(status).decode()
+        if status == MOK_ERR_CUDA:
+            msg += f" (cudaError {_lib.mok_last_cuda_error()})"
+        super().__init__(f"libmok: {msg} [{status}]")
+
+
+def _check(status):
+    if status != MOK_OK:
+        raise MokError(status)
+
+
+def _p(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def _config(impl=0, grid=0, router_impl=0):
+    c = mok_config()
+    c.impl, c.grid, c.router_impl = impl, grid, router_impl
+    return c
+
+
+def mok_version():
+    return int(_lib.mok_version())
+
+
+def mok_status_string(status):
+    return _lib.mok_status_string(status).decode()
+
+
+def mok_workspace_bytes(T, H, I, I_shared, E, k):
+    return int(_lib.mok_workspace_bytes(T, H, I, I_shared, E, k))
+
+
+def mok_launch_count(T, H, I, I_shared, E, k):
+    return int(_lib.mok_launch_count(T, H, I, I_shared, E, k, None))
+
+
+def alloc_workspace(T, H, I, I_shared, E, k, device="cuda", host_staging=False):
+    """A torch uint8 buffer large enough for mok_moe_forward_ex (plus the x/out staging copies of the host variant)."""
+    n = mok_workspace_bytes(T, H, I, I_shared, E, k)
+    if n == 0:
+        raise MokError(MOK_ERR_SHAPE)
+    if host_staging:
+        n += 2 * ((2 * T * H + 255) // 256 * 256)
+    return torch.empty(n + 256, dtype=torch.uint8, device=device)
+
+
+def _aligned_ws(ws):
+    off = (-ws.data_ptr()) % 256
+    return ws.data_ptr() + off, ws.numel() - off
+
+
+def _shapes(x_shape, W_router, W_gate_up, W_shared_gate_up, k):
+    T, H = x_shape
+    E = W_router.shape[0]
+    I = W_gate_up.shape[1] // 2
+    I_s = 0 if W_shared_gate_up is None else W_shared_gate_up.shape[0] // 2
+    return T, H, I, I_s, E, k
+
+
+def mok_moe_forward(x, W_router, W_gate_up, W_down, W_shared_gate_up, W_shared_down, k, out=None, stream=None):
+    """The 14-argument entry point (library-owned workspace, no router bias).  Returns out (bf16 [T,H])."""
+    T, H, I, I_s, E, k = _shapes(x.shape, W_router, W_gate_up, W_shared_gate_up, k)
+    if out is None:
+        out = torch.empty_like(x)
+    _check(_lib.mok_moe_forward(_p(x), _p(W_router), _p(W_gate_up), _p(W_down), _p(W_shared_gate_up),
+                                _p(W_shared_down), T, H, I, I_s, E, k, _p(out), _stream(stream)))
+    return out
+
+
+def _fill_args(x_shape, W_router, router_bias, W_gate_up, W_down, W_shared_gate_up, W_shared_down, k, workspace,
+               stages, config, stream, device):
+    T, H, I, I_s, E, k = _shapes(x_shape, W_router, W_gate_up, W_shared_gate_up, k)
+    a = mok_args()
+    a.W_router = W_router.data_ptr()
+    a.router_bias = None if router_bias is None else router_bias.data_ptr()
+    a.W_gate_up, a.W_down = W_gate_up.data_ptr(), W_down.data_ptr()
+    a.W_shared_gate_up = None if W_shared_gate_up is None else W_shared_gate_up.data_ptr()
+    a.W_shared_down = None if W_shared_down is None else W_shared_down.data_ptr()
+    a.T, a.H, a.I, a.I_shared, a.E, a.k = T, H, I, I_s, E, k
+    a.workspace, a.workspace_bytes = _aligned_ws(workspace)
+    res = {}
+    if stages:
+        R = T * k
+        res = {"topk_idx": torch.empty((T, k), dtype=torch.int32, device=device),
+               "topk_w": torch.empty((T, k), dtype=torch.float32, device=device),
+               "counts": torch.empty((E,), dtype=torch.int32, device=device),
+               "offsets": torch.empty((E + 1,), dtype=torch.int32, device=device),
+               "perm": torch.empty((R,), dtype=torch.int32, device=device),
+               "inv_perm": torch.empty((R,), dtype=torch.int32, device=device)}
+        for name, t in res.items():
+            setattr(a, name, t.data_ptr())
+    if config is not None:
+        a.config = ctypes.pointer(config)
+    a.stream = _stream(stream).value
+    return a, res
+
+
+def mok_moe_forward_ex(x, W_router, router_bias, W_gate_up, W_down, W_shared_gate_up, W_shared_down, k, workspace,
+                       out=None, stages=False, config=None, stream=None):
+    """The layer with router bias, caller-owned workspace, optional stage outputs and knobs.
+
+    Returns out, or (out, dict of stage tensors) when stages=True.
+    """
+    if out is None:
+        out = torch.empty_like(x)
+    a, res = _fill_args(x.shape, W_router, router_bias, W_gate_up, W_down, W_shared_gate_up, W_shared_down, k,
+                        workspace, stages, config, stream, x.device)
+    a.x, a.out = x.data_ptr(), out.data_ptr()
+    _check(_lib.mok_moe_forward_ex(ctypes.byref(a)))
+    return (out, res) if stages else out
+
+
+def mok_moe_forward_host(x_host, out_host, W_router, router_bias, W_gate_up, W_down, W_shared_gate_up, W_shared_down,
+                         k, workspace, config=None, stream=None):
+    """Host-buffer variant: x_host / out_host are CPU (ideally pinned) bf16 tensors; blocks until out_host is filled."""
+    assert not x_host.is_cuda and not out_host.is_cuda
+    a, _ = _fill_args(x_host.shape, W_router, router_bias, W_gate_up, W_down, W_shared_gate_up, W_shared_down, k,
+                      workspace, False, config, stream, W_router.device)
+    _check(_lib.mok_moe_forward_host(ctypes.byref(a), ctypes.c_void_p(x_host.data_ptr()),
+                                     ctypes.c_void_p(out_host.data_ptr())))
+    return out_host
+
+
+def mok_route(x, W_router, router_bias, k, workspace, config=None, stream=None):
+    T, H = x.shape
+    E = W_router.shape[0]
+    idx = torch.empty((T, k), dtype=torch.int32, device=x.device)
+    w = torch.empty((T, k), dtype=torch.float32, device=x.device)
+    wp, wn = _aligned_ws(workspace)
+    _check(_lib.mok_route(_p(x), _p(W_router), _p(router_bias), T, H, E, k, _p(idx), _p(w), wp, wn,
+                          None if config is None else ctypes.pointer(config), _stream(stream)))
+    return idx, w
+
+
+def mok_schedule(topk_idx, E, workspace, stream=None):
+    T, k = topk_idx.shape
+    dev = topk_idx.device
+    counts = torch.empty((E,), dtype=torch.int32, device=dev)
+    offsets = torch.empty((E + 1,), dtype=torch.int32, device=dev)
+    perm = torch.empty((T * k,), dtype=torch.int32, device=dev)
+    inv = torch.empty((T * k,), dtype=torch.int32, device=dev)
+    wp, wn = _aligned_ws(workspace)
+    _check(_lib.mok_schedule(_p(topk_idx), T, E, k, _p(counts), _p(offsets), _p(perm), _p(inv), wp, wn,
+                             _stream(stream)))
+    return counts, offsets, perm, inv
+
+
+def mok_read_status(workspace, stream=None):
+    wp, _ = _aligned_ws(workspace)
+    return int(_lib.mok_read_status(wp, _stream(stream)))
+
+
+def to_device_bf16(bits, device="cuda"):
+    """numpy uint16 bf16 bit patterns -> torch bf16 tensor on the device (a byte copy, no arithmetic)."""
+    import numpy as np
+    return torch.from_numpy(bits.view(np.int16)).to(device).view(torch.bfloat16)

@@ -1,0 +1,134 @@
+"""GPU parity tests: the CUDA path (through the C-ABI binding) against the CPU oracle, element by element on
+small seeded inputs that span several tiles and ragged tails, and on sampled tokens at the full workload sizes."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2609_36070_b200 import inputs
+from paper_2609_36070_b200.inputs import MoEConfig
+
+import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+
+def mok():
+    from paper_2609_36070_b200 import mok as m
+    return m
+
+
+SMALL = [
+    # name, T, H, E, k, I, I_s, bias  -- ragged tails everywhere: T, H (not a multiple of 64), I (not of 128)
+    MoEConfig("ragged", T=333, H=200, E=6, k=2, I=136, I_s=72, seed=11),
+    MoEConfig("k1", T=257, H=128, E=5, k=1, I=128, I_s=0, seed=12),
+    MoEConfig("k_eq_E", T=130, H=64, E=4, k=4, I=64, I_s=64, seed=13),
+    MoEConfig("one_token", T=1, H=64, E=8, k=2, I=64, I_s=0, seed=14),
+    MoEConfig("wide_n", T=300, H=520, E=3, k=2, I=264, I_s=0, seed=15),            # 3 GEMM2 N tiles, 3 GEMM1 N tiles
+    MoEConfig("many_experts", T=512, H=256, E=256, k=8, I=128, I_s=0, bias="normal", seed=16),
+    MoEConfig("zipf_skew", T=700, H=256, E=64, k=4, I=256, I_s=128, bias="zipf", seed=17),  # empty experts + a hot one
+]
+
+
+@pytest.mark.parametrize("cfg", SMALL, ids=[c.name for c in SMALL])
+@pytest.mark.parametrize("impl", ["tcgen05", "simt"])
+def test_small_shapes_every_token(cfg, impl):
+    m = mok()
+    conf = m._config(impl=m.MOK_IMPL_SIMT if impl == "simt" else m.MOK_IMPL_TCGEN05)
+    out, st, rep = pu.full_parity(cfg, config=conf)
+    print(cfg.name, impl, rep)
+
+
+def test_all_routes_to_one_expert():
+    """Degenerate dispatch: a huge bias sends every token's first route to expert 3; other experts get the rest."""
+    cfg = MoEConfig("hot", T=400, H=128, E=8, k=2, I=128, I_s=0, seed=21)
+    d = inputs.make_inputs(cfg)
+    d["bias"] = np.zeros(cfg.E, np.float32)
+    d["bias"][3] = 50.0
+    out, st, rep = pu.full_parity(cfg, d=d)
+    assert st["counts"].cpu().numpy()[3] == cfg.T
+
+
+def test_tiny_config_every_token_and_determinism():
+    cfg = inputs.CONFIGS["tiny"]
+    d = inputs.make_inputs(cfg)
+    g = pu.upload(d)
+    out, st, rep = pu.full_parity(cfg, d=d, g=g)
+    print("tiny", rep)
+    m = mok()
+    out2 = pu.run_gpu(cfg, g, stages=False)
+    assert torch.equal(out.view(torch.int16), out2.view(torch.int16))            # run-to-run bitwise identity
+    for grid in (1, 7, 148):                                                       # bits do not depend on the grid
+        o = pu.run_gpu(cfg, g, config=m._config(grid=grid), stages=False)
+        assert torch.equal(out.view(torch.int16), o.view(torch.int16)), grid
+
+
+def test_fourteen_argument_entry_point_matches_ex():
+    m = mok()
+    cfg = inputs.CONFIGS["tiny"]
+    d = inputs.make_inputs(cfg)
+    g = pu.upload(d)
+    out_ex = pu.run_gpu(cfg, g, stages=False)
+    out = m.mok_moe_forward(g["x"], g["W_r"], g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], cfg.k)
+    torch.cuda.synchronize()
+    assert torch.equal(out.view(torch.int16), out_ex.view(torch.int16))
+    # a second, larger problem makes the library-owned workspace grow
+    cfg2 = SMALL[-1]
+    d2 = inputs.make_inputs(cfg2)
+    d2["bias"] = None
+    g2 = pu.upload(d2)
+    out2 = m.mok_moe_forward(g2["x"], g2["W_r"], g2["W_gate_up"], g2["W_down"], g2["W_sgu"], g2["W_sd"], cfg2.k)
+    ref2 = pu.run_gpu(cfg2, g2, stages=False)
+    torch.cuda.synchronize()
+    assert torch.equal(out2.view(torch.int16), ref2.view(torch.int16))
+
+
+def test_host_buffer_entry_point():
+    m = mok()
+    cfg = inputs.CONFIGS["tiny"]
+    d = inputs.make_inputs(cfg)
+    g = pu.upload(d)
+    ref = pu.run_gpu(cfg, g, stages=False)
+    ws = m.alloc_workspace(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k, host_staging=True)
+    xh = g["x"].cpu().pin_memory()
+    oh = torch.empty_like(xh).pin_memory()
+    m.mok_moe_forward_host(xh, oh, g["W_r"], g["bias"], g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], cfg.k, ws)
+    assert torch.equal(oh.view(torch.int16), ref.cpu().view(torch.int16))
+
+
+def test_stage_entry_points():
+    m = mok()
+    cfg = SMALL[-1]
+    d = inputs.make_inputs(cfg)
+    g = pu.upload(d)
+    ws = m.alloc_workspace(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k)
+    idx, w = m.mok_route(g["x"], g["W_r"], g["bias"], cfg.k, ws)
+    counts, offsets, perm, inv = m.mok_schedule(idx, cfg.E, ws)
+    st = {"topk_idx": idx, "topk_w": w, "counts": counts, "offsets": offsets, "perm": perm, "inv_perm": inv}
+    assert m.mok_read_status(ws) == 0
+    pu.check_routing_and_schedule(cfg, d, st)
+
+
+def test_argument_errors_launch_nothing():
+    m = mok()
+    cfg = inputs.CONFIGS["tiny"]
+    d = inputs.make_inputs(cfg)
+    g = pu.upload(d)
+    ws = m.alloc_workspace(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k)
+    args = (g["x"], g["W_r"], g["bias"], g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"])
+    with pytest.raises(m.MokError) as e:
+        m.mok_moe_forward_ex(*args, cfg.E + 1, ws)                                  # k > E
+    assert e.value.status == m.MOK_ERR_SHAPE
+    with pytest.raises(m.MokError) as e:
+        m.mok_moe_forward_ex(*args, cfg.k, torch.empty(1024, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == m.MOK_ERR_WORKSPACE
+    with pytest.raises(m.MokError) as e:                                             # shared weights without both halves
+        m.mok_moe_forward_ex(g["x"], g["W_r"], None, g["W_gate_up"], g["W_down"], g["W_sgu"], None, cfg.k, ws)
+    assert e.value.status == m.MOK_ERR_SHAPE
+    with pytest.raises(m.MokError) as e:                                             # misaligned activation pointer
+        xm = torch.empty(cfg.T * cfg.H + 8, dtype=torch.bfloat16, device="cuda")[1:1 + cfg.T * cfg.H].view(cfg.T, cfg.H)
+        m.mok_moe_forward_ex(xm, *args[1:], cfg.k, ws)
+    assert e.value.status == m.MOK_ERR_ALIGN
+    # T == 0 is a no-op
+    x0 = torch.empty((0, cfg.H), dtype=torch.bfloat16, device="cuda")
+    out0 = m.mok_moe_forward_ex(x0, *args[1:], cfg.k, ws)
+    assert out0.shape == (0, cfg.H)
