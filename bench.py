@@ -1,0 +1,296 @@
+"""Benchmark of the MoE layer forward pass (one "step" = the whole hot path over one synthetic batch).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl mok|reference]
+
+Prints ONE JSON line.  Default workload: the Qwen3-30B-A3B-like layer (T=16384, H=2048, E=128, k=8, I=768,
+Zipf-skewed routing), synthetic seeded inputs.  With N > 1 (launched by torch.distributed.run) every rank holds a
+full copy of the weights and its own batch of T tokens (token-sharded replicas: no data-path collective), the step
+time is the max over ranks and `value` is the aggregate tokens/s ("weak" scaling).
+
+`--impl reference` times the CPU oracle (the fp64 definition of the layer) on the host cores on a bounded token
+sample of the same workload; it is a deliberately slow baseline, not a target.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "moe_layer_fwd_tokens_per_s"
+UNIT = "tokens/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# dram bytes (read + write) of one launch of the dominant kernel from the committed ncu capture, keyed by config
+# (None until a capture exists for that workload; see profiles/).
+NCU_TRAFFIC_BYTES = {}
+
+
+def parse():
+    p = argparse.ArgumentParser()
+    p.add_argument("--gpus", type=int, default=1)
+    p.add_argument("--steps", type=int, default=300)
+    p.add_argument("--warmup", type=int, default=20)
+    p.add_argument("--config", default="qwen3_30b_a3b")
+    p.add_argument("--impl", default="mok", choices=["mok", "reference"])
+    p.add_argument("--tokens", type=int, default=0, help="override T (small-T sweeps)")
+    p.add_argument("--cpu-sample", type=int, default=0, help="tokens of the CPU-oracle sample (0 = auto)")
+    p.add_argument("--no-cpu-baseline", action="store_true")
+    return p.parse_args()
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return {k: float(d[k]) for k in FALLBACK_PEAKS if k in d} | {"source": "measured"}
+    return dict(FALLBACK_PEAKS, source="fallback")
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu = gpu_index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.06)
+        self.proc.terminate()
+        out, _ = self.proc.communicate(timeout=10)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [v.strip() for v in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def cpu_oracle_rate(cfg, d, sample):
+    """tokens/s of the oracle as it stands on the host cores: routing of all T tokens (its per-token share is
+    charged to the sample) plus the per-token FFN of `sample` tokens."""
+    import numpy as np
+    from oracle import mok_ref
+    t0 = time.perf_counter()
+    idx, w, gap, lg = mok_ref.route(d["x"], d["W_r"], d["bias"], cfg.k)
+    t_route = time.perf_counter() - t0
+    tokens = np.arange(min(sample, cfg.T), dtype=np.int32)
+    t0 = time.perf_counter()
+    mok_ref.ffn_tokens(d["x"], d["W_gate_up"], d["W_down"], d["W_sgu"], d["W_sd"], idx, w, tokens)
+    t_ffn = time.perf_counter() - t0
+    t = t_ffn + t_route * len(tokens) / cfg.T
+    return len(tokens) / t, t_ffn + t_route, mok_ref.num_threads()
+
+
+def auto_sample(cfg, cores):
+    # aim at ~15 s of CPU work assuming ~1.2 fp64 GFLOP/s per core for the scalar oracle
+    per_token = 6.0 * cfg.H * (cfg.k * cfg.I + cfg.I_s)
+    n = int(15.0 * 1.2e9 * cores / per_token)
+    return max(16, min(cfg.T, n))
+
+
+def run_reference(args, cfg, rank):
+    """The CPU oracle as the reference arm.  Rank 0 only."""
+    if rank != 0:
+        return
+    from paper_2609_36070_b200 import inputs
+    d = inputs.make_inputs(cfg)
+    cores = os.cpu_count() or 1
+    steps = max(1, min(args.steps, 3))
+    sample = args.cpu_sample or max(16, auto_sample(cfg, cores) // (steps + min(args.warmup, 1)))
+    for _ in range(min(args.warmup, 1)):
+        cpu_oracle_rate(cfg, d, sample)
+    rates = []
+    t_total = 0.0
+    for _ in range(steps):
+        r, t, threads = cpu_oracle_rate(cfg, d, sample)
+        rates.append(r)
+        t_total += t
+    value = sum(rates) / len(rates)
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "impl": "reference", "n_gpus": args.gpus, "steps": steps,
+            "warmup": min(args.warmup, 1), "ms_per_step": 1e3 * t_total / steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": cfg.name, "T": cfg.T, "H": cfg.H, "E": cfg.E, "k": cfg.k, "I": cfg.I, "I_shared": cfg.I_s},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
+                             "sample": f"routing of all {cfg.T} tokens (charged pro rata) + fp64 FFN of the first {sample} tokens per step"},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gflops": value * 6.0 * cfg.H * (cfg.k * cfg.I + cfg.I_s) / 1e9}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    args = parse()
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    from paper_2609_36070_b200 import inputs
+    cfg = inputs.CONFIGS[args.config]
+    if args.tokens:
+        cfg = cfg.with_tokens(args.tokens)
+    if args.impl == "reference":
+        run_reference(args, cfg, rank)
+        return
+
+    import numpy as np
+    import torch
+    from paper_2609_36070_b200 import mok
+    assert args.warmup >= 3, "timing rules: at least 3 warm-up steps"
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    # every rank: same weights, its own batch (seed offset by rank)
+    d = inputs.make_inputs(cfg)
+    if rank > 0:
+        from dataclasses import replace
+        d["x"] = inputs.make_x(replace(cfg, seed=cfg.seed + 1000 * rank))
+    g = {k: (None if d[k] is None else mok.to_device_bf16(d[k], dev)) for k in ("x", "W_gate_up", "W_down", "W_sgu", "W_sd")}
+    W_r = torch.from_numpy(d["W_r"]).to(dev)
+    bias = None if d["bias"] is None else torch.from_numpy(d["bias"]).to(dev)
+    ws = mok.alloc_workspace(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k, device=dev, host_staging=True)
+    out = torch.empty_like(g["x"])
+    conf = mok._config(profile=1)
+
+    def step():
+        mok.mok_moe_forward_ex(g["x"], W_r, bias, g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], cfg.k, ws,
+                               out=out, config=conf)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    status = mok.mok_read_status(ws)
+    assert status == 0, mok.mok_status_string(status)
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    mok.mok_profile_begin(args.steps)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ev0.record()
+    for _ in range(args.steps):
+        step()
+    ev1.record()
+    barrier()
+    total_ms = ev0.elapsed_time(ev1)
+    stage = mok.mok_profile_end(args.steps)
+    clocks = sampler.stop() if rank == 0 else None
+    status = mok.mok_read_status(ws)
+    assert status == 0, mok.mok_status_string(status)
+
+    if dist is not None:
+        t = torch.tensor([total_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * cfg.T / (ms_per_step * 1e-3)
+    flops = cfg.ffn_flops()
+    tflops = world * flops / (ms_per_step * 1e-3) / 1e12
+
+    # end to end through the host-buffer entry point: pinned host x -> device, layer, result -> pinned host
+    xh = g["x"].cpu().pin_memory()
+    oh = torch.empty_like(xh).pin_memory()
+    conf0 = mok._config()
+
+    def e2e_step():
+        mok.mok_moe_forward_host(xh, oh, W_r, bias, g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], cfg.k, ws,
+                                 config=conf0)
+
+    e2e_steps = max(5, min(args.steps, 50))
+    for _ in range(3):
+        e2e_step()
+    barrier()
+    ev0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    ev1.record()
+    barrier()
+    e2e_ms = ev0.elapsed_time(ev1) / e2e_steps
+    if dist is not None:
+        t = torch.tensor([e2e_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    act_bytes = 2 * cfg.T * cfg.H
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    pk = peaks()
+    mean = {s: float(np.mean([c[s] for c in stage])) for s in mok.STAGES}
+    # dominant kernel: the routed gate/up grouped GEMM with the SwiGLU epilogue (one launch per step)
+    g1_flops = 4.0 * cfg.T * cfg.k * cfg.H * cfg.I
+    g1_tflops = g1_flops / (mean["gemm1"] * 1e-3) / 1e12
+    peak_tf = pk.get("bf16_tflops_sustained", pk["bf16_tflops"])
+    ffn_ms = mean["gemm1"] + mean["gemm2"] + mean["shared_gemm1"] + mean["shared_gemm2"]
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": cfg.name, "T": cfg.T, "H": cfg.H, "E": cfg.E, "k": cfg.k, "I": cfg.I,
+                   "I_shared": cfg.I_s, "routing": cfg.bias, "parallelism": f"token-sharded replicas x{world}",
+                   "l2": "inputs larger than L2 (weights + activations >> 126 MB), no explicit flush"},
+        "tflops": tflops,
+        "tflops_frac_of_peak": tflops / world / pk["bf16_tflops"],
+        "ffn_phase": {"ms": ffn_ms, "tflops": flops / (ffn_ms * 1e-3) / 1e12,
+                      "frac_of_bf16_peak": flops / (ffn_ms * 1e-3) / 1e12 / pk["bf16_tflops"],
+                      "frac_of_bf16_sustained": flops / (ffn_ms * 1e-3) / 1e12 / peak_tf},
+        "stage_ms": mean,
+        "roofline": {"kernel": "gemm_tc_kernel<SWIGLU> (routed gate/up grouped GEMM + SwiGLU)", "bound": "tensor",
+                     "achieved": g1_tflops, "peak": peak_tf, "unit": "TFLOP/s", "frac": g1_tflops / peak_tf,
+                     "peak_source": f"{pk['source']} bf16_tflops_sustained",
+                     "traffic": NCU_TRAFFIC_BYTES.get(cfg.name)},
+        "e2e": {"value": world * cfg.T / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+                "h2d_bytes_per_step": act_bytes, "d2h_bytes_per_step": act_bytes},
+        "gpu_launches": args.steps * mok.mok_launch_count(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k),
+        "clocks": clocks,
+    }
+    if not args.no_cpu_baseline:
+        cores = os.cpu_count() or 1
+        sample = args.cpu_sample or auto_sample(cfg, cores)
+        rate, secs, threads = cpu_oracle_rate(cfg, d, sample)
+        line["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": threads, "kind": "oracle", "seconds": secs,
+                                "sample": f"routing of all {cfg.T} tokens (charged pro rata) + fp64 FFN of the first {min(sample, cfg.T)} tokens"}
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

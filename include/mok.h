@@ -58,7 +58,8 @@ typedef struct mok_config {
     int32_t grid;         /* persistent grid size override for the tcgen05 kernels (0 = number of SMs).  The
                              output bits do not depend on it (Section 3.4 "Determinism"). */
     int32_t router_impl;  /* 0 = default, 1 = fp32 FMA router, 2 = split-bf16 tensor-core router */
-    int32_t reserved[5];
+    int32_t profile;      /* != 0: record CUDA events around every stage of this call (see mok_profile_begin) */
+    int32_t reserved[4];
 } mok_config;
 
 /*
@@ -140,7 +141,23 @@ int mok_schedule(const int32_t* topk_idx, int T, int E, int k,
  */
 int mok_read_status(const void* workspace, void* stream);
 
-/* Number of kernels (and memset nodes) one mok_moe_forward_ex call enqueues for these arguments; 0 on bad sizes. */
+/*
+ * Per-stage device timing with CUDA events recorded on the call's stream (measurement aid; the paper reports
+ * CUDA-side latencies, Section 4.1).  mok_profile_begin reserves event sets for up to max_calls forward calls;
+ * every later forward call whose config has profile != 0 fills the next set without synchronising.
+ * mok_profile_end synchronises on the last recorded event, writes ms[call][stage] (row-major,
+ * MOK_STAGE_COUNT floats per call) for the calls recorded (at most max_calls_out rows), stores their number in
+ * *n_calls and releases the events.  Not thread-safe.
+ */
+enum {
+    MOK_STAGE_ROUTER = 0, MOK_STAGE_SCHEDULE, MOK_STAGE_GATHER, MOK_STAGE_GEMM1, MOK_STAGE_GEMM2,
+    MOK_STAGE_SHARED_GEMM1, MOK_STAGE_SHARED_GEMM2, MOK_STAGE_COMBINE, MOK_STAGE_COUNT
+};
+int mok_profile_begin(int max_calls);
+int mok_profile_end(float* ms, int max_calls_out, int* n_calls);
+
+/* Number of kernels one mok_moe_forward_ex call enqueues for these arguments (the 256-byte header memset is
+   not counted); 0 on bad sizes. */
 int mok_launch_count(int T, int H, int I, int I_shared, int E, int k, const mok_config* config);
 
 int mok_last_cuda_error(void);          /* cudaError_t of the most recent failed CUDA call on this thread */

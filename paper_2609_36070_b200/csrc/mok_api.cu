@@ -14,6 +14,18 @@ static int cuda_fail(cudaError_t e) {
     return MOK_ERR_CUDA;
 }
 
+// Event sets of the per-stage profiler (mok_profile_begin / mok_profile_end).
+struct Profiler {
+    cudaEvent_t* ev = nullptr;      // [max_calls][MOK_STAGE_COUNT + 1]
+    int max_calls = 0, n_calls = 0;
+};
+static Profiler g_prof;
+
+static cudaEvent_t* profile_slot(const mok_config* cfg) {
+    if (!cfg || !cfg->profile || !g_prof.ev || g_prof.n_calls >= g_prof.max_calls) return nullptr;
+    return g_prof.ev + (size_t)(g_prof.n_calls++) * (MOK_STAGE_COUNT + 1);
+}
+
 static bool sizes_ok(int T, int H, int I, int Is, int E, int k) {
     if (T < 0 || H <= 0 || I <= 0 || Is < 0 || E <= 0 || k < 1) return false;
     if (k > E || k > MAX_K || E > MAX_E) return false;
@@ -108,13 +120,19 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
     WsHeader* hdr = reinterpret_cast<WsHeader*>(ws + L.header);
     cudaError_t e = cudaMemsetAsync(hdr, 0, sizeof(WsHeader), s);
     if (e != cudaSuccess) return cuda_fail(e);
+    cudaEvent_t* pev = profile_slot(a->config);
+#define MOK_MARK(i) do { if (pev) cudaEventRecord(pev[i], s); } while (0)
+    MOK_MARK(0);
     int rc = route_stage(a, L, ws, x, s);
     if (rc) return rc;
+    MOK_MARK(MOK_STAGE_ROUTER + 1);
     e = launch_schedule(reinterpret_cast<const int32_t*>(ws + L.idx), a->T, a->E, a->k, L, ws,
                         a->counts, a->offsets, a->perm, a->inv_perm, s);
     if (e != cudaSuccess) return cuda_fail(e);
+    MOK_MARK(MOK_STAGE_SCHEDULE + 1);
     e = launch_gather(x, a->H, a->k, L, ws, s);
     if (e != cudaSuccess) return cuda_fail(e);
+    MOK_MARK(MOK_STAGE_GATHER + 1);
 
     GemmArgs g;
     memset(&g, 0, sizeof(g));
@@ -129,25 +147,35 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
     g.C = reinterpret_cast<__nv_bfloat16*>(ws + L.h);
     g.K = a->H; g.N = a->I; g.E = a->E; g.rows_pad = L.Rpad; g.a_rows = L.Rpad; g.dense_rows = 0;
     if ((rc = run_gemm(g, true, a->config, s))) return rc;
+    MOK_MARK(MOK_STAGE_GEMM1 + 1);
     g.A = reinterpret_cast<const __nv_bfloat16*>(ws + L.h);
     g.B = reinterpret_cast<const __nv_bfloat16*>(a->W_down);
     g.C = reinterpret_cast<__nv_bfloat16*>(ws + L.y);
     g.K = a->I; g.N = a->H;
     if ((rc = run_gemm(g, false, a->config, s))) return rc;
+    MOK_MARK(MOK_STAGE_GEMM2 + 1);
     if (a->I_shared > 0) {   // shared expert: every token in natural order, no gather
         g.A = x;
         g.B = reinterpret_cast<const __nv_bfloat16*>(a->W_shared_gate_up);
         g.C = reinterpret_cast<__nv_bfloat16*>(ws + L.hs);
         g.K = a->H; g.N = a->I_shared; g.E = 1; g.rows_pad = L.Tpad; g.a_rows = a->T; g.dense_rows = a->T;
         if ((rc = run_gemm(g, true, a->config, s))) return rc;
+        MOK_MARK(MOK_STAGE_SHARED_GEMM1 + 1);
         g.A = reinterpret_cast<const __nv_bfloat16*>(ws + L.hs);
         g.B = reinterpret_cast<const __nv_bfloat16*>(a->W_shared_down);
         g.C = reinterpret_cast<__nv_bfloat16*>(ws + L.ysh);
         g.K = a->I_shared; g.N = a->H; g.a_rows = L.Tpad;
         if ((rc = run_gemm(g, false, a->config, s))) return rc;
+        MOK_MARK(MOK_STAGE_SHARED_GEMM2 + 1);
+    } else {
+        MOK_MARK(MOK_STAGE_SHARED_GEMM1 + 1);
+        MOK_MARK(MOK_STAGE_SHARED_GEMM2 + 1);
     }
     e = launch_combine(L, ws, a->T, a->H, a->k, a->I_shared > 0, out, s);
-    return e == cudaSuccess ? MOK_OK : cuda_fail(e);
+    if (e != cudaSuccess) return cuda_fail(e);
+    MOK_MARK(MOK_STAGE_COMBINE + 1);
+#undef MOK_MARK
+    return MOK_OK;
 }
 
 // Library-owned workspace of mok_moe_forward, one per device, grown on demand.
@@ -274,8 +302,52 @@ int mok_launch_count(int T, int H, int I, int I_shared, int E, int k, const mok_
     WsLayout L;
     (void)config;
     if (!ws_layout(T, H, I, I_shared, E, k, &L) || T == 0) return 0;
-    // header memset, router, 3 schedule kernels, gather, 2 routed GEMMs, (2 shared GEMMs), combine
-    return 1 + 1 + 3 + 1 + 2 + (I_shared > 0 ? 2 : 0) + 1;
+    // router, 3 schedule kernels, gather, 2 routed GEMMs, (2 shared GEMMs), combine
+    return 1 + 3 + 1 + 2 + (I_shared > 0 ? 2 : 0) + 1;
+}
+
+int mok_profile_begin(int max_calls) {
+    if (max_calls <= 0) return MOK_ERR_SHAPE;
+    if (g_prof.ev) return MOK_ERR_SHAPE;            // a session is already open
+    const size_t n = (size_t)max_calls * (MOK_STAGE_COUNT + 1);
+    g_prof.ev = new cudaEvent_t[n];
+    for (size_t i = 0; i < n; ++i) {
+        cudaError_t e = cudaEventCreate(&g_prof.ev[i]);
+        if (e != cudaSuccess) {
+            for (size_t j = 0; j < i; ++j) cudaEventDestroy(g_prof.ev[j]);
+            delete[] g_prof.ev;
+            g_prof.ev = nullptr;
+            return cuda_fail(e);
+        }
+    }
+    g_prof.max_calls = max_calls;
+    g_prof.n_calls = 0;
+    return MOK_OK;
+}
+
+int mok_profile_end(float* ms, int max_calls_out, int* n_calls) {
+    if (!g_prof.ev) return MOK_ERR_SHAPE;
+    int rc = MOK_OK;
+    const int n = g_prof.n_calls < max_calls_out ? g_prof.n_calls : max_calls_out;
+    if (g_prof.n_calls > 0) {
+        cudaError_t e = cudaEventSynchronize(g_prof.ev[(size_t)(g_prof.n_calls - 1) * (MOK_STAGE_COUNT + 1) + MOK_STAGE_COUNT]);
+        if (e != cudaSuccess) rc = cuda_fail(e);
+    }
+    for (int c = 0; c < n && rc == MOK_OK && ms; ++c) {
+        cudaEvent_t* ev = g_prof.ev + (size_t)c * (MOK_STAGE_COUNT + 1);
+        for (int st = 0; st < MOK_STAGE_COUNT; ++st) {
+            float t = 0.f;
+            cudaError_t e = cudaEventElapsedTime(&t, ev[st], ev[st + 1]);
+            if (e != cudaSuccess) { rc = cuda_fail(e); break; }
+            ms[(size_t)c * MOK_STAGE_COUNT + st] = t;
+        }
+    }
+    if (n_calls) *n_calls = n;
+    const size_t total = (size_t)g_prof.max_calls * (MOK_STAGE_COUNT + 1);
+    for (size_t i = 0; i < total; ++i) cudaEventDestroy(g_prof.ev[i]);
+    delete[] g_prof.ev;
+    g_prof = Profiler();
+    return rc;
 }
 
 int mok_last_cuda_error(void) { return g_last_cuda_error; }

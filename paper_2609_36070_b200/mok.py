@@ -21,12 +21,13 @@ MOK_IMPL_TCGEN05, MOK_IMPL_SIMT = 0, 1
 
 EXPORTS = ["mok_moe_forward", "mok_workspace_bytes", "mok_moe_forward_ex", "mok_moe_forward_host", "mok_route",
            "mok_schedule", "mok_read_status", "mok_launch_count", "mok_last_cuda_error", "mok_status_string",
-           "mok_version"]
+           "mok_version", "mok_profile_begin", "mok_profile_end"]
+STAGES = ["router", "schedule", "gather", "gemm1", "gemm2", "shared_gemm1", "shared_gemm2", "combine"]
 
 
 class mok_config(ctypes.Structure):
     _fields_ = [("impl", ctypes.c_int32), ("grid", ctypes.c_int32), ("router_impl", ctypes.c_int32),
-                ("reserved", ctypes.c_int32 * 5)]
+                ("profile", ctypes.c_int32), ("reserved", ctypes.c_int32 * 4)]
 
 
 class mok_args(ctypes.Structure):
@@ -63,6 +64,10 @@ _lib.mok_last_cuda_error.restype = ctypes.c_int
 _lib.mok_status_string.restype = ctypes.c_char_p
 _lib.mok_status_string.argtypes = [ctypes.c_int]
 _lib.mok_version.restype = ctypes.c_int
+_lib.mok_profile_begin.restype = ctypes.c_int
+_lib.mok_profile_begin.argtypes = [ctypes.c_int]
+_lib.mok_profile_end.restype = ctypes.c_int
+_lib.mok_profile_end.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.POINTER(ctypes.c_int)]
 
 
 class MokError(RuntimeError):
@@ -89,10 +94,22 @@ def _stream(stream):
     return ctypes.c_void_p(stream.cuda_stream)
 
 
-def _config(impl=0, grid=0, router_impl=0):
+def _config(impl=0, grid=0, router_impl=0, profile=0):
     c = mok_config()
-    c.impl, c.grid, c.router_impl = impl, grid, router_impl
+    c.impl, c.grid, c.router_impl, c.profile = impl, grid, router_impl, profile
     return c
+
+
+def mok_profile_begin(max_calls):
+    _check(_lib.mok_profile_begin(max_calls))
+
+
+def mok_profile_end(max_calls):
+    """Returns a list of per-call dicts {stage name: milliseconds} for the calls recorded since mok_profile_begin."""
+    buf = (ctypes.c_float * (max_calls * len(STAGES)))()
+    n = ctypes.c_int(0)
+    _check(_lib.mok_profile_end(buf, max_calls, ctypes.byref(n)))
+    return [{s: buf[c * len(STAGES) + i] for i, s in enumerate(STAGES)} for c in range(n.value)]
 
 
 def mok_version():

@@ -1,7 +1,8 @@
 """Shared helpers of the GPU parity tests: run the CUDA layer through the C-ABI binding and compare every stage
 with the CPU oracle on the same seeded inputs.  Tolerances (stated by the benchmark spec):
   * top-k indices, counts, offsets, perm, inv_perm: bit-exact, except tokens whose k-th/(k+1)-th logit gap is
-    < 1e-4 (near-ties; counted and reported, and the schedule is then checked against the oracle's schedule of
+    < 1e-4, or whose selected logits contain an adjacent pair closer than 1e-4 (which decides the slot order)
+    (near-ties; counted and reported, and the schedule is then checked against the oracle's schedule of
     the device's own selection);
   * router weights: |w_gpu - w_ref| <= 1e-5;
   * outputs: max|gpu - ref| <= 1e-2 * max|ref| and mean|gpu - ref| / mean|ref| <= 5e-3.
@@ -49,13 +50,19 @@ def check_routing_and_schedule(cfg, d, st):
     idx_gpu = st["topk_idx"].cpu().numpy()
     w_gpu = st["topk_w"].cpu().numpy().astype(np.float64)
     differs = (idx_gpu != idx_ref).any(axis=1)
-    near = gap < NEAR_TIE
+    # Near-ties.  The selection is decided at the k-th/(k+1)-th boundary (gap); the slot ORDER inside the selection
+    # is decided by the same kind of comparison between adjacent selected logits, so the same 1e-4 rule applies:
+    # a token whose closest adjacent pair among its top-(k+1) logits is nearer than 1e-4 may differ, and is counted.
+    sel = np.take_along_axis(lg, idx_ref.astype(np.int64), axis=1)           # descending
+    inner = np.full(cfg.T, np.inf) if cfg.k == 1 else (sel[:, :-1] - sel[:, 1:]).min(axis=1)
+    near = np.minimum(gap, inner) < NEAR_TIE
     bad = differs & ~near
     assert not bad.any(), f"{bad.sum()} tokens with a different top-k that are not near-ties, first {np.flatnonzero(bad)[:5]}"
-    # a flipped near-tie must still be a valid selection: same set except members whose logits are within the gap
+    # a flipped near-tie must still be a valid selection in a valid order, both up to the tolerance
     for t in np.flatnonzero(differs):
-        lo = np.sort(lg[t, idx_gpu[t]])[0]
-        assert lo >= np.sort(lg[t])[::-1][cfg.k - 1] - NEAR_TIE
+        lsel = lg[t, idx_gpu[t]]
+        assert lsel.min() >= np.sort(lg[t])[::-1][cfg.k - 1] - NEAR_TIE
+        assert (np.diff(lsel) <= NEAR_TIE).all()
         assert len(set(idx_gpu[t])) == cfg.k
     w_sel = mok_ref.weights(lg, idx_gpu)
     werr = np.abs(w_gpu - w_sel).max()
