@@ -91,7 +91,7 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(GemmArgs a) {
             if (c >= a.N) continue;
             float v = accg[i][j];
             if (SWIGLU) v = (v / (1.f + expf(-v))) * accu[i][j];
-            a.C[(size_t)(r0 + ty * 4 + i) * a.N + c] = __float2bfloat16_rn(v);
+            reinterpret_cast<__nv_bfloat16*>(a.C)[(size_t)(r0 + ty * 4 + i) * a.ldc + c] = __float2bfloat16_rn(v);
         }
 }
 

@@ -12,9 +12,13 @@
 // Every output element is produced by exactly one tile with a fixed k order, so results do not depend on the
 // grid size or on timing (Section 3.4 "Determinism").
 //
-//   SWIGLU : B = [E, 2N, K]; the 256-wide B tile is 128 gate rows followed by the matching 128 up rows and the
-//            epilogue writes C[:, n*128 .. n*128+127] = silu(gate) * up.
-//   else   : B = [E, N, K]; C[:, n*256 .. n*256+255] = A . B^T.
+//   EPI_SWIGLU : B = [E, 2N, K]; the 256-wide B tile is 128 gate rows followed by the matching 128 up rows and the
+//                epilogue writes C[:, n*128 .. n*128+127] = silu(gate) * up (bf16).
+//   EPI_BF16   : B = [E, N, K]; C[:, n*256 .. n*256+255] = A . B^T (bf16).
+//   EPI_F32    : as EPI_BF16 with fp32 output (router logits).
+//   GATHER     : the A rows of a tile are token rows of x picked through the row -> token table of the dispatch
+//                schedule: the paper's pull dispatch (Section 3.1) done by the producer warp with TMA gather4
+//                (4 rows per instruction, one instruction per lane), so the expert-sorted copy of x never exists.
 // All mbarrier waits are bounded: on a timeout the CTA records MOK_ERR_TIMEOUT and leaves cleanly.
 #include "mok_internal.cuh"
 
@@ -95,6 +99,15 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1) : "memory");
 }
 
+// Four rows (r0..r3) of a 2D tensor, 64 columns starting at c0, land as four consecutive 128-byte smem rows.
+__device__ __forceinline__ void tma_gather4(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0,
+                                            int r0, int r1, int r2, int r3) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(r0), "r"(r1), "r"(r2), "r"(r3) : "memory");
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
@@ -136,7 +149,7 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr) {
 // Instruction descriptor: D fp32, A/B bf16, both K-major, dense, M=128, N=256.
 constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 
-struct Tile { int row0, n, e; };
+struct Tile { int row0, n, e, m; };
 
 __device__ __forceinline__ Tile decode_tile(const GemmArgs& a, int L, int n_nt, int n_mt_total) {
     Tile t;
@@ -150,7 +163,8 @@ __device__ __forceinline__ Tile decode_tile(const GemmArgs& a, int L, int n_nt, 
     }
     const int r = L - n_nt * mt0;
     t.n = r / m_cnt;
-    t.row0 = (mt0 + (r - t.n * m_cnt)) * BM;
+    t.m = r - t.n * m_cnt;
+    t.row0 = (mt0 + t.m) * BM;
     return t;
 }
 
@@ -159,10 +173,11 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
-template <bool SWIGLU>
+template <int EPI, bool GATHER>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
                const GemmArgs a, const int n_nt, const int k_blocks) {
+    constexpr bool SWIGLU = (EPI == EPI_SWIGLU);
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -194,28 +209,44 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
-        if (lane == 0) {
-            int s = 0;
-            uint32_t ph = 0;
-            const int b_rows_per_expert = (SWIGLU ? 2 : 1) * a.N;
-            for (int L = blockIdx.x; L < total; L += gridDim.x) {
-                const Tile t = decode_tile(a, L, n_nt, n_mt_total);
-                const int brow0 = t.e * b_rows_per_expert + (SWIGLU ? t.n * (BN / 2) : t.n * BN);
-                const int brow1 = SWIGLU ? brow0 + a.N : brow0 + BN / 2;
-                bool ok = true;
-                for (int kb = 0; kb < k_blocks; ++kb) {
-                    ok = mbar_wait(smem_u32(&ctrl->empty[s]), ph ^ 1u, abort_flag, a.header, 1);
-                    if (!ok) break;
-                    const uint32_t full = smem_u32(&ctrl->full[s]);
-                    const uint32_t sa = base + s * STAGE_BYTES, sb = sa + A_BYTES;
+        int s = 0;
+        uint32_t ph = 0;
+        const int b_rows_per_expert = (SWIGLU ? 2 : 1) * a.N;
+        for (int L = blockIdx.x; L < total; L += gridDim.x) {
+            const Tile t = decode_tile(a, L, n_nt, n_mt_total);
+            const int brow0 = t.e * b_rows_per_expert + (SWIGLU ? t.n * (BN / 2) : t.n * BN);
+            const int brow1 = SWIGLU ? brow0 + a.N : brow0 + BN / 2;
+            int4 tok = make_int4(0, 0, 0, 0);
+            if (GATHER) {   // lane l owns rows 4l..4l+3 of the tile; rows past the expert's segment reuse row 0
+                const int valid = __ldg(a.counts + t.e) - t.m * BM;
+                const int tok0 = __ldg(a.row_token + t.row0);
+                tok = *reinterpret_cast<const int4*>(a.row_token + t.row0 + lane * 4);
+                const int r = lane * 4;
+                if (r + 0 >= valid) tok.x = tok0;
+                if (r + 1 >= valid) tok.y = tok0;
+                if (r + 2 >= valid) tok.z = tok0;
+                if (r + 3 >= valid) tok.w = tok0;
+            }
+            bool ok = true;
+            for (int kb = 0; kb < k_blocks; ++kb) {
+                ok = mbar_wait(smem_u32(&ctrl->empty[s]), ph ^ 1u, abort_flag, a.header, 1);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                const uint32_t full = smem_u32(&ctrl->full[s]);
+                const uint32_t sa = base + s * STAGE_BYTES, sb = sa + A_BYTES;
+                if (lane == 0) {
                     mbar_expect_tx(full, STAGE_BYTES);
-                    tma_load_2d(sa, &tmapA, full, kb * BK, t.row0);
+                    if (!GATHER) tma_load_2d(sa, &tmapA, full, kb * BK, t.row0);
                     tma_load_2d(sb, &tmapB, full, kb * BK, brow0);
                     tma_load_2d(sb + B_BYTES / 2, &tmapB, full, kb * BK, brow1);
-                    if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
-                if (!ok) break;
+                if (GATHER) {
+                    __syncwarp();
+                    tma_gather4(sa + lane * 512, &tmapA, full, kb * BK, tok.x, tok.y, tok.z, tok.w);
+                }
+                if (++s == STAGES) { s = 0; ph ^= 1u; }
             }
+            if (!ok) break;
         }
         __syncwarp();
     } else if (warp == 1) {
@@ -258,8 +289,24 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
             if (!ok) break;
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(as * BN);
-            __nv_bfloat16* crow = a.C + (size_t)(t.row0 + quad * 32 + lane) * a.N;
-            if (SWIGLU) {
+            const size_t crow_off = (size_t)(t.row0 + quad * 32 + lane) * a.ldc;
+            __nv_bfloat16* crow = reinterpret_cast<__nv_bfloat16*>(a.C) + crow_off;
+            if (EPI == EPI_F32) {
+                float* frow = reinterpret_cast<float*>(a.C) + crow_off;
+                const int c0 = t.n * BN;
+#pragma unroll 1
+                for (int c = 0; c < BN; c += 32) {
+                    uint32_t r[32];
+                    tc_ld32(taddr + c, r);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int v = 0; v < 8; ++v) {
+                        const int col = c0 + c + v * 4;
+                        if (col < a.N)
+                            *reinterpret_cast<uint4*>(frow + col) = make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
+                    }
+                }
+            } else if (SWIGLU) {
                 const int c0 = t.n * (BN / 2);
 #pragma unroll 1
                 for (int c = 0; c < BN / 2; c += 32) {
@@ -350,11 +397,28 @@ static bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t co
 
 }  // namespace tc
 
-cudaError_t launch_gemm_tc(const GemmArgs& a, bool swiglu, int grid, cudaStream_t s) {
+template <int EPI, bool GATHER>
+static cudaError_t launch_one(const CUtensorMap& mA, const CUtensorMap& mB, const GemmArgs& a, int n_nt, int k_blocks,
+                              int grid, cudaStream_t s) {
     using namespace tc;
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<EPI, GATHER>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    gemm_tc_kernel<EPI, GATHER><<<grid, THREADS, SMEM_BYTES, s>>>(mA, mB, a, n_nt, k_blocks);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_gemm_tc(const GemmArgs& a, int epi, int grid, cudaStream_t s) {
+    using namespace tc;
+    const bool swiglu = (epi == EPI_SWIGLU), gather = (a.row_token != nullptr);
     CUtensorMap mA, mB;
     const uint64_t b_rows = (uint64_t)a.E * (swiglu ? 2 : 1) * a.N;
-    if (!make_map(&mA, a.A, (uint64_t)a.a_rows, (uint64_t)a.K, BM)) return cudaErrorInvalidValue;
+    // gather4 takes a one-row box: each instruction names four rows itself
+    if (!make_map(&mA, a.A, (uint64_t)a.a_rows, (uint64_t)a.K, gather ? 1 : BM)) return cudaErrorInvalidValue;
     if (!make_map(&mB, a.B, b_rows, (uint64_t)a.K, BN / 2)) return cudaErrorInvalidValue;
     const int n_nt = swiglu ? (a.N + BN / 2 - 1) / (BN / 2) : (a.N + BN - 1) / BN;
     const int k_blocks = (a.K + BK - 1) / BK;
@@ -363,13 +427,13 @@ cudaError_t launch_gemm_tc(const GemmArgs& a, bool swiglu, int grid, cudaStream_
         int dev = 0;
         cudaGetDevice(&dev);
         cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
-        cudaFuncSetAttribute(gemm_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
-        cudaFuncSetAttribute(gemm_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     }
     if (grid <= 0 || grid > sm_count) grid = sm_count;
-    if (swiglu) gemm_tc_kernel<true><<<grid, THREADS, SMEM_BYTES, s>>>(mA, mB, a, n_nt, k_blocks);
-    else gemm_tc_kernel<false><<<grid, THREADS, SMEM_BYTES, s>>>(mA, mB, a, n_nt, k_blocks);
-    return cudaGetLastError();
+    if (epi == EPI_SWIGLU && gather) return launch_one<EPI_SWIGLU, true>(mA, mB, a, n_nt, k_blocks, grid, s);
+    if (epi == EPI_SWIGLU) return launch_one<EPI_SWIGLU, false>(mA, mB, a, n_nt, k_blocks, grid, s);
+    if (epi == EPI_BF16 && !gather) return launch_one<EPI_BF16, false>(mA, mB, a, n_nt, k_blocks, grid, s);
+    if (epi == EPI_F32 && !gather) return launch_one<EPI_F32, false>(mA, mB, a, n_nt, k_blocks, grid, s);
+    return cudaErrorInvalidValue;
 }
 
 }  // namespace mok

@@ -62,8 +62,10 @@ bool ws_layout(int T, int H, int I, int Is, int E, int k, WsLayout* L) {
     L->inv = take(sizeof(int32_t) * (size_t)(R > 0 ? R : 1));
     L->pos = take(sizeof(int32_t) * (size_t)(R > 0 ? R : 1));
     L->blk_hist = take(sizeof(int32_t) * (size_t)L->n_blk * E);
-    L->wr_split = take(2 * (size_t)3 * E * H);
-    L->logits = take(sizeof(float) * (size_t)L->Tpad * 3 * E);
+    L->row_token = take(sizeof(int32_t) * (size_t)Rpad);
+    const size_t ldl = (size_t)(3 * E + 7) / 8 * 8;
+    L->wr_split = take(2 * ldl * H);
+    L->logits = take(sizeof(float) * (size_t)L->Tpad * ldl);
     L->xg = take(2 * (size_t)Rpad * H);
     L->h = take(2 * (size_t)Rpad * I);
     L->y = take(2 * (size_t)Rpad * H);
@@ -87,20 +89,33 @@ static int validate(const mok_args* a, WsLayout* L, size_t extra_ws) {
         return MOK_ERR_ALIGN;
     if (!a->workspace || (reinterpret_cast<uintptr_t>(a->workspace) & 255u) || a->workspace_bytes < L->total + extra_ws)
         return MOK_ERR_WORKSPACE;
-    if (a->config && (a->config->impl < 0 || a->config->impl > 1 || a->config->grid < 0)) return MOK_ERR_SHAPE;
+    if (a->config && (a->config->impl < 0 || a->config->impl > 1 || a->config->grid < 0 ||
+                      a->config->router_impl < 0 || a->config->router_impl > 2))
+        return MOK_ERR_SHAPE;
     return MOK_OK;
 }
 
+static bool use_simt(const mok_config* cfg) { return cfg && cfg->impl == MOK_IMPL_SIMT; }
+static bool use_simt_router(const mok_config* cfg, int k) {
+    if (k > 28) return true;   // the tensor-core router keeps k + 4 candidates in one warp's 32 lanes
+    return cfg && (cfg->router_impl == 1 || (cfg->router_impl == 0 && cfg->impl == MOK_IMPL_SIMT));
+}
+
 static int run_gemm(const GemmArgs& g, bool swiglu, const mok_config* cfg, cudaStream_t s) {
-    cudaError_t e = (cfg && cfg->impl == MOK_IMPL_SIMT) ? launch_gemm_simt(g, swiglu, s)
-                                                          : launch_gemm_tc(g, swiglu, cfg ? cfg->grid : 0, s);
+    cudaError_t e = use_simt(cfg) ? launch_gemm_simt(g, swiglu, s)
+                                  : launch_gemm_tc(g, swiglu ? EPI_SWIGLU : EPI_BF16, cfg ? cfg->grid : 0, s);
     return e == cudaSuccess ? MOK_OK : cuda_fail(e);
 }
 
 static int route_stage(const mok_args* a, const WsLayout& L, char* ws, const __nv_bfloat16* x, cudaStream_t s) {
     int32_t* idx = reinterpret_cast<int32_t*>(ws + L.idx);
     float* w = reinterpret_cast<float*>(ws + L.w);
-    cudaError_t e = launch_router_simt(x, a->W_router, a->router_bias, a->T, a->H, a->E, a->k, idx, w, s);
+    cudaError_t e;
+    if (use_simt_router(a->config, a->k))
+        e = launch_router_simt(x, a->W_router, a->router_bias, a->T, a->H, a->E, a->k, idx, w, s);
+    else
+        e = launch_router_tc(x, a->W_router, a->router_bias, a->T, a->H, a->E, a->k, L, ws,
+                             reinterpret_cast<WsHeader*>(ws + L.header), a->config ? a->config->grid : 0, idx, w, s);
     if (e != cudaSuccess) return cuda_fail(e);
     if (a->topk_idx) {
         e = cudaMemcpyAsync(a->topk_idx, idx, sizeof(int32_t) * (size_t)L.R, cudaMemcpyDeviceToDevice, s);
@@ -130,8 +145,11 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
                         a->counts, a->offsets, a->perm, a->inv_perm, s);
     if (e != cudaSuccess) return cuda_fail(e);
     MOK_MARK(MOK_STAGE_SCHEDULE + 1);
-    e = launch_gather(x, a->H, a->k, L, ws, s);
-    if (e != cudaSuccess) return cuda_fail(e);
+    const bool simt = !(a->config && a->config->reserved[0] == 1);   // TEMP: fused gather4 only on request
+    if (simt) {
+        e = launch_gather(x, a->H, a->k, L, ws, s);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
     MOK_MARK(MOK_STAGE_GATHER + 1);
 
     GemmArgs g;
@@ -142,29 +160,40 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
     g.mt_start = reinterpret_cast<const int32_t*>(ws + L.mt_start);
     g.max_mt = L.max_mt;
     // routed experts: h = silu(Xg Wg^T) * (Xg Wu^T);  y = h Wd^T
-    g.A = reinterpret_cast<const __nv_bfloat16*>(ws + L.xg);
+    if (simt) {
+        g.A = reinterpret_cast<const __nv_bfloat16*>(ws + L.xg);
+        g.a_rows = L.Rpad;
+    } else {
+        g.A = x;
+        g.a_rows = a->T;
+        g.row_token = reinterpret_cast<const int32_t*>(ws + L.row_token);
+        g.counts = reinterpret_cast<const int32_t*>(ws + L.counts);
+    }
     g.B = reinterpret_cast<const __nv_bfloat16*>(a->W_gate_up);
-    g.C = reinterpret_cast<__nv_bfloat16*>(ws + L.h);
-    g.K = a->H; g.N = a->I; g.E = a->E; g.rows_pad = L.Rpad; g.a_rows = L.Rpad; g.dense_rows = 0;
+    g.C = ws + L.h;
+    g.K = a->H; g.N = a->I; g.ldc = a->I; g.E = a->E; g.rows_pad = L.Rpad; g.dense_rows = 0;
     if ((rc = run_gemm(g, true, a->config, s))) return rc;
+    g.row_token = nullptr;
+    g.counts = nullptr;
+    g.a_rows = L.Rpad;
     MOK_MARK(MOK_STAGE_GEMM1 + 1);
     g.A = reinterpret_cast<const __nv_bfloat16*>(ws + L.h);
     g.B = reinterpret_cast<const __nv_bfloat16*>(a->W_down);
-    g.C = reinterpret_cast<__nv_bfloat16*>(ws + L.y);
-    g.K = a->I; g.N = a->H;
+    g.C = ws + L.y;
+    g.K = a->I; g.N = a->H; g.ldc = a->H;
     if ((rc = run_gemm(g, false, a->config, s))) return rc;
     MOK_MARK(MOK_STAGE_GEMM2 + 1);
     if (a->I_shared > 0) {   // shared expert: every token in natural order, no gather
         g.A = x;
         g.B = reinterpret_cast<const __nv_bfloat16*>(a->W_shared_gate_up);
-        g.C = reinterpret_cast<__nv_bfloat16*>(ws + L.hs);
-        g.K = a->H; g.N = a->I_shared; g.E = 1; g.rows_pad = L.Tpad; g.a_rows = a->T; g.dense_rows = a->T;
+        g.C = ws + L.hs;
+        g.K = a->H; g.N = a->I_shared; g.ldc = a->I_shared; g.E = 1; g.rows_pad = L.Tpad; g.a_rows = a->T; g.dense_rows = a->T;
         if ((rc = run_gemm(g, true, a->config, s))) return rc;
         MOK_MARK(MOK_STAGE_SHARED_GEMM1 + 1);
         g.A = reinterpret_cast<const __nv_bfloat16*>(ws + L.hs);
         g.B = reinterpret_cast<const __nv_bfloat16*>(a->W_shared_down);
-        g.C = reinterpret_cast<__nv_bfloat16*>(ws + L.ysh);
-        g.K = a->I_shared; g.N = a->H; g.a_rows = L.Tpad;
+        g.C = ws + L.ysh;
+        g.K = a->I_shared; g.N = a->H; g.ldc = a->H; g.a_rows = L.Tpad;
         if ((rc = run_gemm(g, false, a->config, s))) return rc;
         MOK_MARK(MOK_STAGE_SHARED_GEMM2 + 1);
     } else {
@@ -300,10 +329,10 @@ int mok_read_status(const void* workspace, void* stream) {
 
 int mok_launch_count(int T, int H, int I, int I_shared, int E, int k, const mok_config* config) {
     WsLayout L;
-    (void)config;
     if (!ws_layout(T, H, I, I_shared, E, k, &L) || T == 0) return 0;
-    // router, 3 schedule kernels, gather, 2 routed GEMMs, (2 shared GEMMs), combine
-    return 1 + 3 + 1 + 2 + (I_shared > 0 ? 2 : 0) + 1;
+    // router (1 fp32-FMA kernel, or split + GEMM + top-k), 3 schedule kernels, (gather on the SIMT path),
+    // 2 routed GEMMs, (2 shared GEMMs), combine
+    return (use_simt_router(config, k) ? 1 : 3) + 3 + 1 + 2 + (I_shared > 0 ? 2 : 0) + 1;
 }
 
 int mok_profile_begin(int max_calls) {

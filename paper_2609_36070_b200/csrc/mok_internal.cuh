@@ -25,8 +25,9 @@ struct WsHeader {
 // Byte offsets of every workspace region, computed on the host from the sizes alone (no readback).
 struct WsLayout {
     size_t header, idx, w, counts, offsets, pad_offsets, mt_start, tile_expert, perm, inv, pos, blk_hist;
+    size_t row_token;     // int32 [Rpad]: source token of every row of the padded dispatch space (pad rows undefined)
     size_t wr_split;      // bf16 [3E, H]: W_r split into hi/mid/lo parts for the tensor-core router
-    size_t logits;        // fp32 [T, 3E] partial logits of the tensor-core router
+    size_t logits;        // fp32 [Tpad, ldl] partial logits of the tensor-core router (ldl = 3E rounded up to 8)
     size_t xg, h, y, hs, ysh;
     size_t total;
     int32_t R;            // T*k
@@ -42,10 +43,13 @@ bool ws_layout(int T, int H, int I, int Is, int E, int k, WsLayout* L);
 // [128*mt_start[e], 128*mt_start[e+1]); tile q belongs to expert tile_expert[q].  In dense mode (shared
 // expert) there is one expert and ceil(dense_rows/128) tiles.
 struct GemmArgs {
-    const __nv_bfloat16* A;      // [rows_pad, K]
+    const __nv_bfloat16* A;      // [a_rows, K]; with row_token set, A = x [T, K] and rows are gathered through it
     const __nv_bfloat16* B;      // SWIGLU: [E, 2*N, K] (gate rows then up rows); else [E, N, K]
-    __nv_bfloat16* C;            // [rows_pad, N]
+    void* C;                     // [rows_pad, ldc] bf16 (fp32 for the router logits)
     int32_t K, N, E;
+    int32_t ldc;                 // elements between consecutive rows of C
+    const int32_t* row_token;    // device [rows_pad] or NULL: padded row -> token (gather fused into the A loads)
+    const int32_t* counts;       // device [E] (only read when row_token is set)
     int32_t rows_pad;            // allocated rows of C (multiple of 128)
     int32_t a_rows;              // allocated rows of A (reads beyond it are treated as zero)
     int32_t dense_rows;          // > 0: dense mode with this many valid rows
@@ -66,8 +70,10 @@ cudaError_t launch_gather(const __nv_bfloat16* x, int H, int k, const WsLayout& 
 cudaError_t launch_combine(const WsLayout& L, char* ws, int T, int H, int k, bool shared, __nv_bfloat16* out,
                            cudaStream_t s);
 cudaError_t launch_gemm_simt(const GemmArgs& a, bool swiglu, cudaStream_t s);
-cudaError_t launch_gemm_tc(const GemmArgs& a, bool swiglu, int grid, cudaStream_t s);
-int gemm_tc_launches(void);
+enum { EPI_BF16 = 0, EPI_SWIGLU = 1, EPI_F32 = 2 };
+cudaError_t launch_gemm_tc(const GemmArgs& a, int epi, int grid, cudaStream_t s);
+cudaError_t launch_router_tc(const __nv_bfloat16* x, const float* Wr, const float* bias, int T, int H, int E, int k,
+                             const WsLayout& L, char* ws, WsHeader* hdr, int grid, int32_t* idx, float* w, cudaStream_t s);
 
 inline __host__ __device__ size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 

@@ -9,47 +9,13 @@
 // This file holds the fp32 FMA version: a 64-token x 64-expert shared-memory tiled product that leaves
 // the block's logits in shared memory, followed by a warp-shuffle top-k (one warp per token).
 #include "mok_internal.cuh"
-#include <float.h>
+#include "router_common.cuh"
 
 namespace mok {
 
 constexpr int RT_TOK = 64;   // tokens per block
 constexpr int RT_EXP = 64;   // experts per pass
 constexpr int RT_KC = 32;    // hidden-dimension chunk
-
-// One warp selects the top-k of `E` logits in shared memory and writes idx / w for one token.
-__device__ __forceinline__ void warp_topk_softmax(const float* __restrict__ lg, int E, int k, int lane,
-                                                  int32_t* __restrict__ idx_out, float* __restrict__ w_out) {
-    uint32_t taken = 0;                 // bit j: expert lane + 32*j already selected
-    float sel_v = 0.f;
-    int sel_e = 0;
-    for (int s = 0; s < k; ++s) {
-        float bv = -FLT_MAX;
-        int be = 0x7fffffff;
-        for (int j = 0, e = lane; e < E; ++j, e += 32) {
-            if ((taken >> j) & 1u) continue;
-            float v = lg[e];
-            if (v > bv || be == 0x7fffffff) { bv = v; be = e; }   // ascending e + strict '>' keeps the lowest id on ties
-        }
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) {
-            float ov = __shfl_xor_sync(0xffffffffu, bv, off);
-            int oe = __shfl_xor_sync(0xffffffffu, be, off);
-            if (oe != 0x7fffffff && (be == 0x7fffffff || ov > bv || (ov == bv && oe < be))) { bv = ov; be = oe; }
-        }
-        if ((be & 31) == lane) taken |= 1u << (be >> 5);
-        if (lane == s) { sel_v = bv; sel_e = be; }
-    }
-    float v0 = __shfl_sync(0xffffffffu, sel_v, 0);
-    float ex = (lane < k) ? expf(sel_v - v0) : 0.f;
-    float sum = ex;
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
-    if (lane < k) {
-        idx_out[lane] = sel_e;
-        w_out[lane] = ex / sum;
-    }
-}
 
 __global__ void __launch_bounds__(256)
 router_simt_kernel(const __nv_bfloat16* __restrict__ x, const float* __restrict__ Wr, const float* __restrict__ bias,

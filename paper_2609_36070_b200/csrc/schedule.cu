@@ -7,7 +7,8 @@
 //   1. sched_hist    per-block expert histograms of SCHED_CHUNK consecutive routes
 //   2. sched_scan    one block: per-expert prefix over blocks, counts, offsets, and the internal tile tables
 //                    (each expert's segment padded to a multiple of 128 rows: pad_offsets, mt_start, tile_expert)
-//   3. sched_scatter stable ranks inside each block (warp match + per-warp running counters) -> perm, inv, pos
+//   3. sched_scatter stable ranks inside each block (warp match + per-warp running counters) -> perm, inv, pos,
+//                    row_token (padded row -> source token: the {src_index} column of the paper's schedule table)
 // Exported offsets/perm are unpadded; the padding is internal to the GEMM row space.
 #include "mok_internal.cuh"
 
@@ -86,6 +87,7 @@ sched_scatter_kernel(const int32_t* __restrict__ a, int n, int E,
                      const int32_t* __restrict__ blk_base, const int32_t* __restrict__ offsets,
                      const int32_t* __restrict__ pad_offsets,
                      int32_t* __restrict__ perm, int32_t* __restrict__ inv, int32_t* __restrict__ pos,
+                     int32_t* __restrict__ row_token, int k,
                      int32_t* __restrict__ perm_out, int32_t* __restrict__ inv_out) {
     extern __shared__ int32_t ssm[];                 // [SCHED_WARPS][E] running counters per warp
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -131,7 +133,9 @@ sched_scatter_kernel(const int32_t* __restrict__ a, int n, int E,
             int32_t p = offsets[e] + rank;           // Phi[S_l + o] = route j
             perm[p] = j;
             inv[j] = p;
-            pos[j] = pad_offsets[e] + rank;          // row in the padded GEMM space
+            const int32_t prow = pad_offsets[e] + rank;   // row in the padded GEMM space
+            pos[j] = prow;
+            row_token[prow] = j / k;                 // the schedule table's src_index column, as a token id
             if (perm_out) perm_out[p] = j;
             if (inv_out) inv_out[j] = p;
         }
@@ -155,7 +159,7 @@ cudaError_t launch_schedule(const int32_t* idx, int T, int E, int k, const WsLay
     sched_scatter_kernel<<<L.n_blk, SCHED_THREADS, sizeof(int32_t) * SCHED_WARPS * E, s>>>(
         idx, n, E, blk_hist, offsets, pad_offsets,
         reinterpret_cast<int32_t*>(ws + L.perm), reinterpret_cast<int32_t*>(ws + L.inv),
-        reinterpret_cast<int32_t*>(ws + L.pos), perm_out, inv_out);
+        reinterpret_cast<int32_t*>(ws + L.pos), reinterpret_cast<int32_t*>(ws + L.row_token), k, perm_out, inv_out);
     return cudaGetLastError();
 }
 
