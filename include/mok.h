@@ -59,7 +59,9 @@ typedef struct mok_config {
                              output bits do not depend on it (Section 3.4 "Determinism"). */
     int32_t router_impl;  /* 0 = default, 1 = fp32 FMA router, 2 = split-bf16 tensor-core router */
     int32_t profile;      /* != 0: record CUDA events around every stage of this call (see mok_profile_begin) */
-    int32_t reserved[4];
+    int32_t gather_mode;  /* token gather of the routed gate/up GEMM: 0 = choose by shape, 1 = fused into the GEMM's
+                             operand loads (no expert-sorted copy of x), 2 = separate gather kernel + TMA loads */
+    int32_t reserved[3];
 } mok_config;
 
 /*

@@ -17,8 +17,11 @@
 //   EPI_BF16   : B = [E, N, K]; C[:, n*256 .. n*256+255] = A . B^T (bf16).
 //   EPI_F32    : as EPI_BF16 with fp32 output (router logits).
 //   GATHER     : the A rows of a tile are token rows of x picked through the row -> token table of the dispatch
-//                schedule: the paper's pull dispatch (Section 3.1) done by the producer warp with TMA gather4
-//                (4 rows per instruction, one instruction per lane), so the expert-sorted copy of x never exists.
+//                schedule: the paper's pull dispatch (Section 3.1).  Four extra gather warps copy the rows with
+//                16-byte cp.async straight into the swizzled A stage (8 lanes cover one 128-byte row segment, so a
+//                warp instruction reads four whole segments), and the copies' completion arrives on the stage's
+//                mbarrier; the expert-sorted copy of x never exists.  (TMA tile::gather4 computes the same thing
+//                but measured 2x slower here: 32 instructions of 512 bytes per k-block outrun the TMA issue rate.)
 // All mbarrier waits are bounded: on a timeout the CTA records MOK_ERR_TIMEOUT and leaves cleanly.
 #include "mok_internal.cuh"
 
@@ -30,9 +33,12 @@ constexpr int A_BYTES = BM * BK * 2;           // 16 KB
 constexpr int B_BYTES = BN * BK * 2;           // 32 KB
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES; // 48 KB
 constexpr int ACC_STAGES = 2, TMEM_COLS = 512;
-constexpr int THREADS = 192;
+constexpr int THREADS = 192;                  // + 4 gather warps in the GATHER instantiation
+constexpr int GATHER_THREADS = 128;
+constexpr int GROUP_M = 16;                    // M tiles per rasterisation group
 constexpr int SMEM_CTRL = 256;
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + SMEM_CTRL + 1024;   // + slack for 1024-byte alignment
+constexpr int OUT_STAGE_BYTES = 4 * 8192;      // per epilogue warp: 32 rows x 128 bf16 columns, as two swizzled boxes
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + OUT_STAGE_BYTES + SMEM_CTRL + 1024;   // + slack for alignment
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;            // 2 s
 
 struct Ctrl {
@@ -99,13 +105,25 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1) : "memory");
 }
 
-// Four rows (r0..r3) of a 2D tensor, 64 columns starting at c0, land as four consecutive 128-byte smem rows.
-__device__ __forceinline__ void tma_gather4(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0,
-                                            int r0, int r1, int r2, int r3) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes"
-        " [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
-        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(r0), "r"(r1), "r"(r2), "r"(r3) : "memory");
+// 16-byte asynchronous global -> shared copy (src_bytes = 0 writes zeros), and the arrive that fires on the
+// mbarrier once all earlier cp.async of this thread have landed (it counts as one of the expected arrivals).
+__device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src, uint32_t src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_mbar_arrive(uint32_t bar) {
+    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// Shared -> global tile store (bulk async group); out-of-range rows / columns of the box are clipped by the map.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int c0, int c1) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(map), "r"(src), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -161,9 +179,15 @@ __device__ __forceinline__ Tile decode_tile(const GemmArgs& a, int L, int n_nt, 
         mt0 = __ldg(a.mt_start + t.e);
         m_cnt = __ldg(a.mt_start + t.e + 1) - mt0;
     }
+    // Inside an expert, M tiles are taken in groups of GROUP_M: all N tiles of a group before the next group, M
+    // fastest.  The group's activations (GROUP_M x 128 rows) then stay in L2 while the expert's weight tiles stream.
     const int r = L - n_nt * mt0;
-    t.n = r / m_cnt;
-    t.m = r - t.n * m_cnt;
+    const int per_group = GROUP_M * n_nt;
+    const int g = r / per_group;
+    const int rem = r - g * per_group;
+    const int in_group = min(GROUP_M, m_cnt - g * GROUP_M);
+    t.n = rem / in_group;
+    t.m = g * GROUP_M + (rem - t.n * in_group);
     t.row0 = (mt0 + t.m) * BM;
     return t;
 }
@@ -174,15 +198,15 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 }
 
 template <int EPI, bool GATHER>
-__global__ void __launch_bounds__(THREADS, 1)
+__global__ void __launch_bounds__(THREADS + (GATHER ? GATHER_THREADS : 0), 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
-               const GemmArgs a, const int n_nt, const int k_blocks) {
+               const __grid_constant__ CUtensorMap tmapC, const GemmArgs a, const int n_nt, const int k_blocks) {
     constexpr bool SWIGLU = (EPI == EPI_SWIGLU);
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t* smem = smem_raw + (base - raw);
-    Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem + STAGES * STAGE_BYTES);
+    Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem + STAGES * STAGE_BYTES + OUT_STAGE_BYTES);
     volatile uint32_t* abort_flag = &ctrl->abort;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -191,7 +215,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
     const int total = n_mt_total * n_nt;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) { mbar_init(smem_u32(&ctrl->full[s]), 1); mbar_init(smem_u32(&ctrl->empty[s]), 1); }
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(smem_u32(&ctrl->full[s]), GATHER ? 1 + GATHER_THREADS : 1);
+            mbar_init(smem_u32(&ctrl->empty[s]), 1);
+        }
         for (int s = 0; s < ACC_STAGES; ++s) { mbar_init(smem_u32(&ctrl->tfull[s]), 1); mbar_init(smem_u32(&ctrl->tempty[s]), 128); }
         ctrl->abort = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -209,44 +236,28 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
-        int s = 0;
-        uint32_t ph = 0;
-        const int b_rows_per_expert = (SWIGLU ? 2 : 1) * a.N;
-        for (int L = blockIdx.x; L < total; L += gridDim.x) {
-            const Tile t = decode_tile(a, L, n_nt, n_mt_total);
-            const int brow0 = t.e * b_rows_per_expert + (SWIGLU ? t.n * (BN / 2) : t.n * BN);
-            const int brow1 = SWIGLU ? brow0 + a.N : brow0 + BN / 2;
-            int4 tok = make_int4(0, 0, 0, 0);
-            if (GATHER) {   // lane l owns rows 4l..4l+3 of the tile; rows past the expert's segment reuse row 0
-                const int valid = __ldg(a.counts + t.e) - t.m * BM;
-                const int tok0 = __ldg(a.row_token + t.row0);
-                tok = *reinterpret_cast<const int4*>(a.row_token + t.row0 + lane * 4);
-                const int r = lane * 4;
-                if (r + 0 >= valid) tok.x = tok0;
-                if (r + 1 >= valid) tok.y = tok0;
-                if (r + 2 >= valid) tok.z = tok0;
-                if (r + 3 >= valid) tok.w = tok0;
-            }
-            bool ok = true;
-            for (int kb = 0; kb < k_blocks; ++kb) {
-                ok = mbar_wait(smem_u32(&ctrl->empty[s]), ph ^ 1u, abort_flag, a.header, 1);
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
-                const uint32_t full = smem_u32(&ctrl->full[s]);
-                const uint32_t sa = base + s * STAGE_BYTES, sb = sa + A_BYTES;
-                if (lane == 0) {
-                    mbar_expect_tx(full, STAGE_BYTES);
+        if (lane == 0) {
+            int s = 0;
+            uint32_t ph = 0;
+            const int b_rows_per_expert = (SWIGLU ? 2 : 1) * a.N;
+            for (int L = blockIdx.x; L < total; L += gridDim.x) {
+                const Tile t = decode_tile(a, L, n_nt, n_mt_total);
+                const int brow0 = t.e * b_rows_per_expert + (SWIGLU ? t.n * (BN / 2) : t.n * BN);
+                const int brow1 = SWIGLU ? brow0 + a.N : brow0 + BN / 2;
+                bool ok = true;
+                for (int kb = 0; kb < k_blocks; ++kb) {
+                    ok = mbar_wait(smem_u32(&ctrl->empty[s]), ph ^ 1u, abort_flag, a.header, 1);
+                    if (!ok) break;
+                    const uint32_t full = smem_u32(&ctrl->full[s]);
+                    const uint32_t sa = base + s * STAGE_BYTES, sb = sa + A_BYTES;
+                    mbar_expect_tx(full, GATHER ? B_BYTES : STAGE_BYTES);
                     if (!GATHER) tma_load_2d(sa, &tmapA, full, kb * BK, t.row0);
                     tma_load_2d(sb, &tmapB, full, kb * BK, brow0);
                     tma_load_2d(sb + B_BYTES / 2, &tmapB, full, kb * BK, brow1);
+                    if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
-                if (GATHER) {
-                    __syncwarp();
-                    tma_gather4(sa + lane * 512, &tmapA, full, kb * BK, tok.x, tok.y, tok.z, tok.w);
-                }
-                if (++s == STAGES) { s = 0; ph ^= 1u; }
+                if (!ok) break;
             }
-            if (!ok) break;
         }
         __syncwarp();
     } else if (warp == 1) {
@@ -277,9 +288,51 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
             }
         }
         __syncwarp();
+    } else if (GATHER && warp >= 6) {
+        // ------------------------------------------------------------------ gather warps 6..9 (pull dispatch)
+        // Warp gw owns tile rows 32 gw .. 32 gw + 31.  Lane = (sub-row 0..3, 16-byte chunk 0..7); pass i covers rows
+        // 32 gw + 4 i + sub-row.  Chunk c of row r lands at r*128 + ((c ^ (r & 7)) * 16): the 128-byte swizzle the
+        // UMMA descriptor expects.  Rows past the expert's segment re-read the tile's first row (never stored).
+        const int gw = warp - 6, sub = lane >> 3, chunk = lane & 7;
+        int s = 0;
+        uint32_t ph = 0;
+        for (int L = blockIdx.x; L < total; L += gridDim.x) {
+            const Tile t = decode_tile(a, L, n_nt, n_mt_total);
+            const int valid = __ldg(a.counts + t.e) - t.m * BM;
+            const int tok0 = __ldg(a.row_token + t.row0);
+            const __nv_bfloat16* src[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int r = gw * 32 + i * 4 + sub;
+                const int tok = (r < valid) ? __ldg(a.row_token + t.row0 + r) : tok0;
+                src[i] = a.A + (size_t)tok * a.K + chunk * 8;
+            }
+            bool ok = true;
+            for (int kb = 0; kb < k_blocks; ++kb) {
+                ok = mbar_wait(smem_u32(&ctrl->empty[s]), ph ^ 1u, abort_flag, a.header, 5);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                const uint32_t sa = base + s * STAGE_BYTES;
+                const bool in_k = (kb * BK + chunk * 8) < a.K;            // K tail: zero-fill
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int r = gw * 32 + i * 4 + sub;
+                    const uint32_t dst = sa + r * 128 + ((chunk ^ (r & 7)) << 4);
+                    cp_async_16(dst, in_k ? (const void*)(src[i] + kb * BK) : (const void*)a.A, in_k ? 16u : 0u);
+                }
+                cp_async_mbar_arrive(smem_u32(&ctrl->full[s]));
+                if (++s == STAGES) { s = 0; ph ^= 1u; }
+            }
+            if (!ok) break;
+        }
+        asm volatile("cp.async.wait_all;" ::: "memory");
     } else {
         // ------------------------------------------------------------------ epilogue (warps 2..5)
+        // TMEM -> registers -> (SwiGLU) -> bf16 -> this warp's swizzled staging slab -> TMA store.  Each warp owns
+        // 32 accumulator rows and stages 128 output columns at a time as two [32 rows x 64 columns] boxes, so the
+        // global writes are whole 128-byte lines and the warp only synchronises with itself.
         const int quad = warp & 3;                            // TMEM lane quadrant this warp may access
+        const uint32_t slab = base + STAGES * STAGE_BYTES + quad * 8192;
         int as = 0;
         uint32_t aph = 0;
         for (int L = blockIdx.x; L < total; L += gridDim.x) {
@@ -289,10 +342,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
             if (!ok) break;
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(as * BN);
-            const size_t crow_off = (size_t)(t.row0 + quad * 32 + lane) * a.ldc;
-            __nv_bfloat16* crow = reinterpret_cast<__nv_bfloat16*>(a.C) + crow_off;
+            const int row = t.row0 + quad * 32;
             if (EPI == EPI_F32) {
-                float* frow = reinterpret_cast<float*>(a.C) + crow_off;
+                float* frow = reinterpret_cast<float*>(a.C) + (size_t)(row + lane) * a.ldc;
                 const int c0 = t.n * BN;
 #pragma unroll 1
                 for (int c = 0; c < BN; c += 32) {
@@ -306,51 +358,63 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
                             *reinterpret_cast<uint4*>(frow + col) = make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
                     }
                 }
-            } else if (SWIGLU) {
-                const int c0 = t.n * (BN / 2);
-#pragma unroll 1
-                for (int c = 0; c < BN / 2; c += 32) {
-                    uint32_t g[32], u[32];
-                    tc_ld32(taddr + c, g);
-                    tc_ld32(taddr + BN / 2 + c, u);
-                    tc_wait_ld();
-                    uint32_t o[16];
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        float g0 = __uint_as_float(g[2 * i]), g1 = __uint_as_float(g[2 * i + 1]);
-                        float h0 = (g0 / (1.f + __expf(-g0))) * __uint_as_float(u[2 * i]);
-                        float h1 = (g1 / (1.f + __expf(-g1))) * __uint_as_float(u[2 * i + 1]);
-                        o[i] = pack_bf16(h0, h1);
-                    }
-#pragma unroll
-                    for (int v = 0; v < 4; ++v) {
-                        const int col = c0 + c + v * 8;
-                        if (col < a.N)
-                            *reinterpret_cast<uint4*>(crow + col) = make_uint4(o[4 * v], o[4 * v + 1], o[4 * v + 2], o[4 * v + 3]);
-                    }
-                }
+                tc_fence_before();
+                mbar_arrive(smem_u32(&ctrl->tempty[as]));
             } else {
-                const int c0 = t.n * BN;
+                constexpr int HALVES = SWIGLU ? 1 : 2;        // 128 output columns per pass
+                const int c0 = SWIGLU ? t.n * (BN / 2) : t.n * BN;
 #pragma unroll 1
-                for (int c = 0; c < BN; c += 32) {
-                    uint32_t r[32];
-                    tc_ld32(taddr + c, r);
-                    tc_wait_ld();
-                    uint32_t o[16];
+                for (int half = 0; half < HALVES; ++half) {
+                    if (lane == 0) tma_store_wait_read();     // the slab's previous stores have been read out
+                    __syncwarp();
+#pragma unroll 1
+                    for (int c = 0; c < 128; c += 32) {
+                        uint32_t o[16];
+                        if (SWIGLU) {
+                            uint32_t g[32], u[32];
+                            tc_ld32(taddr + c, g);
+                            tc_ld32(taddr + BN / 2 + c, u);
+                            tc_wait_ld();
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) o[i] = pack_bf16(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
+                            for (int i = 0; i < 16; ++i) {
+                                float g0 = __uint_as_float(g[2 * i]), g1 = __uint_as_float(g[2 * i + 1]);
+                                float h0 = (g0 / (1.f + __expf(-g0))) * __uint_as_float(u[2 * i]);
+                                float h1 = (g1 / (1.f + __expf(-g1))) * __uint_as_float(u[2 * i + 1]);
+                                o[i] = pack_bf16(h0, h1);
+                            }
+                        } else {
+                            uint32_t r[32];
+                            tc_ld32(taddr + half * 128 + c, r);
+                            tc_wait_ld();
 #pragma unroll
-                    for (int v = 0; v < 4; ++v) {
-                        const int col = c0 + c + v * 8;
-                        if (col < a.N)
-                            *reinterpret_cast<uint4*>(crow + col) = make_uint4(o[4 * v], o[4 * v + 1], o[4 * v + 2], o[4 * v + 3]);
+                            for (int i = 0; i < 16; ++i) o[i] = pack_bf16(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
+                        }
+                        // 32 columns = 4 chunks of 16 bytes in box (c / 64), chunk index ((c % 64) / 8 + v)
+                        const uint32_t box = slab + (c >> 6) * 4096 + lane * 128;
+#pragma unroll
+                        for (int v = 0; v < 4; ++v) {
+                            const int cc = ((c & 63) >> 3) + v;
+                            st_shared_v4(box + ((cc ^ (lane & 7)) << 4), o[4 * v], o[4 * v + 1], o[4 * v + 2], o[4 * v + 3]);
+                        }
+                    }
+                    if (half == HALVES - 1) {                 // all TMEM reads of this tile are done
+                        tc_fence_before();
+                        mbar_arrive(smem_u32(&ctrl->tempty[as]));
+                    }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) {
+                        const int col = c0 + half * 128;
+                        if (col < a.N) tma_store_2d(&tmapC, slab, col, row);
+                        if (col + 64 < a.N) tma_store_2d(&tmapC, slab + 4096, col + 64, row);
+                        tma_store_commit();
                     }
                 }
             }
-            tc_fence_before();
-            mbar_arrive(smem_u32(&ctrl->tempty[as]));
             if (++as == ACC_STAGES) { as = 0; aph ^= 1u; }
         }
+        if (lane == 0) tma_store_wait_all();
+        __syncwarp();
     }
 
     // ---------------------------------------------------------------------- teardown
@@ -383,11 +447,12 @@ static EncodeTiledFn get_encode() {
 }
 
 // 2D bf16 row-major tensor [rows, cols] -> tensor map with a [box_rows x 64] box and 128-byte swizzle.
-static bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+static bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows,
+                     uint64_t row_stride_elems = 0) {
     EncodeTiledFn enc = get_encode();
     if (!enc) return false;
     cuuint64_t dims[2] = {cols, rows};
-    cuuint64_t strides[1] = {cols * 2};
+    cuuint64_t strides[1] = {(row_stride_elems ? row_stride_elems : cols) * 2};
     cuuint32_t box[2] = {(cuuint32_t)BK, box_rows};
     cuuint32_t estr[2] = {1, 1};
     return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
@@ -398,8 +463,8 @@ static bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t co
 }  // namespace tc
 
 template <int EPI, bool GATHER>
-static cudaError_t launch_one(const CUtensorMap& mA, const CUtensorMap& mB, const GemmArgs& a, int n_nt, int k_blocks,
-                              int grid, cudaStream_t s) {
+static cudaError_t launch_one(const CUtensorMap& mA, const CUtensorMap& mB, const CUtensorMap& mC, const GemmArgs& a,
+                              int n_nt, int k_blocks, int grid, cudaStream_t s) {
     using namespace tc;
     static bool configured = false;
     if (!configured) {
@@ -408,18 +473,19 @@ static cudaError_t launch_one(const CUtensorMap& mA, const CUtensorMap& mB, cons
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    gemm_tc_kernel<EPI, GATHER><<<grid, THREADS, SMEM_BYTES, s>>>(mA, mB, a, n_nt, k_blocks);
+    gemm_tc_kernel<EPI, GATHER><<<grid, THREADS + (GATHER ? GATHER_THREADS : 0), SMEM_BYTES, s>>>(mA, mB, mC, a, n_nt, k_blocks);
     return cudaGetLastError();
 }
 
 cudaError_t launch_gemm_tc(const GemmArgs& a, int epi, int grid, cudaStream_t s) {
     using namespace tc;
     const bool swiglu = (epi == EPI_SWIGLU), gather = (a.row_token != nullptr);
-    CUtensorMap mA, mB;
+    CUtensorMap mA, mB, mC;
     const uint64_t b_rows = (uint64_t)a.E * (swiglu ? 2 : 1) * a.N;
-    // gather4 takes a one-row box: each instruction names four rows itself
-    if (!make_map(&mA, a.A, (uint64_t)a.a_rows, (uint64_t)a.K, gather ? 1 : BM)) return cudaErrorInvalidValue;
+    if (!make_map(&mA, a.A, (uint64_t)a.a_rows, (uint64_t)a.K, BM)) return cudaErrorInvalidValue;
     if (!make_map(&mB, a.B, b_rows, (uint64_t)a.K, BN / 2)) return cudaErrorInvalidValue;
+    if (epi == EPI_F32) mC = mB;      // the fp32 epilogue stores directly
+    else if (!make_map(&mC, a.C, (uint64_t)a.rows_pad, (uint64_t)a.N, 32, (uint64_t)a.ldc)) return cudaErrorInvalidValue;
     const int n_nt = swiglu ? (a.N + BN / 2 - 1) / (BN / 2) : (a.N + BN - 1) / BN;
     const int k_blocks = (a.K + BK - 1) / BK;
     static int sm_count = 0;
@@ -429,10 +495,10 @@ cudaError_t launch_gemm_tc(const GemmArgs& a, int epi, int grid, cudaStream_t s)
         cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
     }
     if (grid <= 0 || grid > sm_count) grid = sm_count;
-    if (epi == EPI_SWIGLU && gather) return launch_one<EPI_SWIGLU, true>(mA, mB, a, n_nt, k_blocks, grid, s);
-    if (epi == EPI_SWIGLU) return launch_one<EPI_SWIGLU, false>(mA, mB, a, n_nt, k_blocks, grid, s);
-    if (epi == EPI_BF16 && !gather) return launch_one<EPI_BF16, false>(mA, mB, a, n_nt, k_blocks, grid, s);
-    if (epi == EPI_F32 && !gather) return launch_one<EPI_F32, false>(mA, mB, a, n_nt, k_blocks, grid, s);
+    if (epi == EPI_SWIGLU && gather) return launch_one<EPI_SWIGLU, true>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
+    if (epi == EPI_SWIGLU) return launch_one<EPI_SWIGLU, false>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
+    if (epi == EPI_BF16 && !gather) return launch_one<EPI_BF16, false>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
+    if (epi == EPI_F32 && !gather) return launch_one<EPI_F32, false>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
     return cudaErrorInvalidValue;
 }
 

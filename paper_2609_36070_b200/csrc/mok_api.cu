@@ -90,7 +90,8 @@ static int validate(const mok_args* a, WsLayout* L, size_t extra_ws) {
     if (!a->workspace || (reinterpret_cast<uintptr_t>(a->workspace) & 255u) || a->workspace_bytes < L->total + extra_ws)
         return MOK_ERR_WORKSPACE;
     if (a->config && (a->config->impl < 0 || a->config->impl > 1 || a->config->grid < 0 ||
-                      a->config->router_impl < 0 || a->config->router_impl > 2))
+                      a->config->router_impl < 0 || a->config->router_impl > 2 ||
+                      a->config->gather_mode < 0 || a->config->gather_mode > 2))
         return MOK_ERR_SHAPE;
     return MOK_OK;
 }
@@ -99,6 +100,16 @@ static bool use_simt(const mok_config* cfg) { return cfg && cfg->impl == MOK_IMP
 static bool use_simt_router(const mok_config* cfg, int k) {
     if (k > 28) return true;   // the tensor-core router keeps k + 4 candidates in one warp's 32 lanes
     return cfg && (cfg->router_impl == 1 || (cfg->router_impl == 0 && cfg->impl == MOK_IMPL_SIMT));
+}
+
+// Whether the routed gate/up GEMM gathers its rows itself.  The fused path re-gathers the rows once per N tile
+// through the load/store units; the separate kernel writes the expert-sorted copy once and the GEMM then uses
+// plain TMA tile loads.  Measured on B200: fused wins at 6, 16 and 23 N tiles (ceil(I / 128)), loses at 112.
+static bool fused_gather(const mok_config* cfg, int I) {
+    if (use_simt(cfg)) return false;
+    if (cfg && cfg->gather_mode == 1) return true;
+    if (cfg && cfg->gather_mode == 2) return false;
+    return (I + 127) / 128 <= 32;
 }
 
 static int run_gemm(const GemmArgs& g, bool swiglu, const mok_config* cfg, cudaStream_t s) {
@@ -145,8 +156,8 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
                         a->counts, a->offsets, a->perm, a->inv_perm, s);
     if (e != cudaSuccess) return cuda_fail(e);
     MOK_MARK(MOK_STAGE_SCHEDULE + 1);
-    const bool simt = !(a->config && a->config->reserved[0] == 1);   // TEMP: fused gather4 only on request
-    if (simt) {
+    const bool simt = !fused_gather(a->config, a->I);
+    if (simt) {   // materialise the expert-sorted copy of x
         e = launch_gather(x, a->H, a->k, L, ws, s);
         if (e != cudaSuccess) return cuda_fail(e);
     }
@@ -332,7 +343,7 @@ int mok_launch_count(int T, int H, int I, int I_shared, int E, int k, const mok_
     if (!ws_layout(T, H, I, I_shared, E, k, &L) || T == 0) return 0;
     // router (1 fp32-FMA kernel, or split + GEMM + top-k), 3 schedule kernels, (gather on the SIMT path),
     // 2 routed GEMMs, (2 shared GEMMs), combine
-    return (use_simt_router(config, k) ? 1 : 3) + 3 + 1 + 2 + (I_shared > 0 ? 2 : 0) + 1;
+    return (use_simt_router(config, k) ? 1 : 3) + 3 + (fused_gather(config, I) ? 0 : 1) + 2 + (I_shared > 0 ? 2 : 0) + 1;
 }
 
 int mok_profile_begin(int max_calls) {

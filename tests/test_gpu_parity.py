@@ -30,10 +30,12 @@ SMALL = [
 
 
 @pytest.mark.parametrize("cfg", SMALL, ids=[c.name for c in SMALL])
-@pytest.mark.parametrize("impl", ["tcgen05", "simt"])
+@pytest.mark.parametrize("impl", ["tcgen05_fused_gather", "tcgen05_separate_gather", "simt"])
 def test_small_shapes_every_token(cfg, impl):
     m = mok()
-    conf = m._config(impl=m.MOK_IMPL_SIMT if impl == "simt" else m.MOK_IMPL_TCGEN05)
+    conf = {"simt": m._config(impl=m.MOK_IMPL_SIMT),
+            "tcgen05_fused_gather": m._config(gather_mode=1),
+            "tcgen05_separate_gather": m._config(gather_mode=2)}[impl]
     out, st, rep = pu.full_parity(cfg, config=conf)
     print(cfg.name, impl, rep)
 
