@@ -137,6 +137,23 @@ int mok_schedule(const int32_t* topk_idx, int T, int E, int k,
                  void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * mok_schedule without a workspace and without any allocation.  The paper has no counterpart of this entry point;
+ * it exists for callers that cannot allocate device memory where they need a schedule: serving loops that must not
+ * take cudaMalloc's device-wide synchronisation, processes whose framework already owns all of HBM, plug-ins that
+ * are handed only input and output buffers.  Inputs and outputs are as for mok_schedule (device pointers; any of the
+ * four outputs may be NULL).  The scratch lives in a fixed 1.25 MiB array inside the library image: one copy per GPU
+ * that loads the library, held until the process exits.
+ *   - Limit: T*k <= MOK_NOALLOC_MAX_ROUTES (and E <= 512); larger sizes return MOK_ERR_SHAPE and launch nothing.
+ *   - The first call on each device looks up the array's device address (a host-side set-up step); make that first
+ *     call outside of any stream capture.  No call allocates or frees memory.
+ *   - All calls on a device share the array and it keeps the previous call's contents (the words that must start at
+ *     zero are cleared by every call): calls that overlap on the device race, so serialise them on one stream.
+ */
+#define MOK_NOALLOC_MAX_ROUTES 32768
+int mok_schedule_noalloc(const int32_t* topk_idx, int T, int E, int k,
+                         int32_t* counts, int32_t* offsets, int32_t* perm, int32_t* inv_perm, void* stream);
+
+/*
  * Reads the device-side status word of a workspace after synchronising `stream` -- the only call besides
  * mok_moe_forward_host that blocks the host.  Returns MOK_OK, MOK_ERR_TIMEOUT or MOK_ERR_SCHEDULE
  * (or MOK_ERR_CUDA if the stream itself is in error).

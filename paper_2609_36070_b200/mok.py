@@ -21,7 +21,8 @@ MOK_IMPL_TCGEN05, MOK_IMPL_SIMT = 0, 1
 
 EXPORTS = ["mok_moe_forward", "mok_workspace_bytes", "mok_moe_forward_ex", "mok_moe_forward_host", "mok_route",
            "mok_schedule", "mok_read_status", "mok_launch_count", "mok_last_cuda_error", "mok_status_string",
-           "mok_version", "mok_profile_begin", "mok_profile_end"]
+           "mok_version", "mok_profile_begin", "mok_profile_end", "mok_schedule_noalloc"]
+MOK_NOALLOC_MAX_ROUTES = 32768
 STAGES = ["router", "schedule", "gather", "gemm1", "gemm2", "shared_gemm1", "shared_gemm2", "combine"]
 
 
@@ -56,6 +57,8 @@ _lib.mok_route.argtypes = ([ctypes.c_void_p] * 3 + [ctypes.c_int] * 4 + [ctypes.
 _lib.mok_schedule.restype = ctypes.c_int
 _lib.mok_schedule.argtypes = ([ctypes.c_void_p] + [ctypes.c_int] * 3 + [ctypes.c_void_p] * 5 +
                               [ctypes.c_size_t, ctypes.c_void_p])
+_lib.mok_schedule_noalloc.restype = ctypes.c_int
+_lib.mok_schedule_noalloc.argtypes = [ctypes.c_void_p] + [ctypes.c_int] * 3 + [ctypes.c_void_p] * 5
 _lib.mok_read_status.restype = ctypes.c_int
 _lib.mok_read_status.argtypes = [ctypes.c_void_p, ctypes.c_void_p]
 _lib.mok_launch_count.restype = ctypes.c_int
@@ -236,6 +239,21 @@ def mok_schedule(topk_idx, E, workspace, stream=None):
     wp, wn = _aligned_ws(workspace)
     _check(_lib.mok_schedule(_p(topk_idx), T, E, k, _p(counts), _p(offsets), _p(perm), _p(inv), wp, wn,
                              _stream(stream)))
+    return counts, offsets, perm, inv
+
+
+def mok_schedule_noalloc(topk_idx, E, stream=None):
+    """mok_schedule for callers that cannot allocate device memory: the scratch is a fixed array inside the library
+    (T*k <= MOK_NOALLOC_MAX_ROUTES).  The four result tensors are the caller's outputs, allocated here by torch only
+    because this is the Python convenience wrapper; the C entry point itself allocates nothing."""
+    T, k = topk_idx.shape
+    dev = topk_idx.device
+    counts = torch.empty((E,), dtype=torch.int32, device=dev)
+    offsets = torch.empty((E + 1,), dtype=torch.int32, device=dev)
+    perm = torch.empty((T * k,), dtype=torch.int32, device=dev)
+    inv = torch.empty((T * k,), dtype=torch.int32, device=dev)
+    _check(_lib.mok_schedule_noalloc(_p(topk_idx), T, E, k, _p(counts), _p(offsets), _p(perm), _p(inv),
+                                     _stream(stream)))
     return counts, offsets, perm, inv
 
 
