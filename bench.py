@@ -40,6 +40,7 @@ def parse():
     p.add_argument("--cpu-sample", type=int, default=0, help="tokens of the CPU-oracle sample (0 = auto)")
     p.add_argument("--no-cpu-baseline", action="store_true")
     p.add_argument("--gather-mode", type=int, default=0, help="0 auto, 1 fused into the GEMM, 2 separate kernel")
+    p.add_argument("--cta-group", type=int, default=0, help="0 default, 1 single CTAs, 2 CTA pairs")
     return p.parse_args()
 
 
@@ -180,7 +181,7 @@ def main():
     bias = None if d["bias"] is None else torch.from_numpy(d["bias"]).to(dev)
     ws = mok.alloc_workspace(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k, device=dev, host_staging=True)
     out = torch.empty_like(g["x"])
-    conf = mok._config(profile=1, gather_mode=args.gather_mode)
+    conf = mok._config(profile=1, gather_mode=args.gather_mode, cta_group=args.cta_group)
 
     def step():
         mok.mok_moe_forward_ex(g["x"], W_r, bias, g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], cfg.k, ws,

@@ -61,7 +61,9 @@ typedef struct mok_config {
     int32_t profile;      /* != 0: record CUDA events around every stage of this call (see mok_profile_begin) */
     int32_t gather_mode;  /* token gather of the routed gate/up GEMM: 0 = choose by shape, 1 = fused into the GEMM's
                              operand loads (no expert-sorted copy of x), 2 = separate gather kernel + TMA loads */
-    int32_t reserved[3];
+    int32_t cta_group;    /* tcgen05 GEMMs: 0 = default (1), 1 = one CTA per 128-row tile, 2 = CTA pairs sharing a
+                             256-row tile (cta_group::2; halves the weight traffic into each SM) */
+    int32_t reserved[2];
 } mok_config;
 
 /*
@@ -141,7 +143,7 @@ int mok_schedule(const int32_t* topk_idx, int T, int E, int k,
  * it exists for callers that cannot allocate device memory where they need a schedule: serving loops that must not
  * take cudaMalloc's device-wide synchronisation, processes whose framework already owns all of HBM, plug-ins that
  * are handed only input and output buffers.  Inputs and outputs are as for mok_schedule (device pointers; any of the
- * four outputs may be NULL).  The scratch lives in a fixed 1.25 MiB array inside the library image: one copy per GPU
+ * four outputs may be NULL).  The scratch lives in a fixed 1.5 MiB array inside the library image: one copy per GPU
  * that loads the library, held until the process exits.
  *   - Limit: T*k <= MOK_NOALLOC_MAX_ROUTES (and E <= 512); larger sizes return MOK_ERR_SHAPE and launch nothing.
  *   - The first call on each device looks up the array's device address (a host-side set-up step); make that first

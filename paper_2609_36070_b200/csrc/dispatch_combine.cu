@@ -11,16 +11,16 @@
 namespace mok {
 
 __global__ void __launch_bounds__(256)
-gather_kernel(const __nv_bfloat16* __restrict__ x, int H, int k,
+gather_kernel(const __nv_bfloat16* __restrict__ x, int H, int k, int tile_m,
               const WsHeader* __restrict__ hdr, const int32_t* __restrict__ tile_expert,
               const int32_t* __restrict__ pad_offsets, const int32_t* __restrict__ offsets,
               const int32_t* __restrict__ counts, const int32_t* __restrict__ perm,
               __nv_bfloat16* __restrict__ xg) {
     const int lane = threadIdx.x & 31;
-    const int rows = hdr->n_mtiles * TILE_M;
+    const int rows = hdr->n_mtiles * tile_m;
     const int chunks = H >> 3;
     for (int p = blockIdx.x * 8 + (threadIdx.x >> 5); p < rows; p += gridDim.x * 8) {
-        const int e = tile_expert[p / TILE_M];
+        const int e = tile_expert[p / tile_m];
         const int local = p - pad_offsets[e];
         uint4* dst = reinterpret_cast<uint4*>(xg + (size_t)p * H);
         if (local < counts[e]) {
@@ -81,10 +81,10 @@ combine_kernel(const __nv_bfloat16* __restrict__ y, const __nv_bfloat16* __restr
     }
 }
 
-cudaError_t launch_gather(const __nv_bfloat16* x, int H, int k, const WsLayout& L, char* ws, cudaStream_t s) {
+cudaError_t launch_gather(const __nv_bfloat16* x, int H, int k, int tile_m, const WsLayout& L, char* ws, cudaStream_t s) {
     int blocks = (L.Rpad + 7) / 8;
     if (blocks > 148 * 64) blocks = 148 * 64;
-    gather_kernel<<<blocks, 256, 0, s>>>(x, H, k, reinterpret_cast<const WsHeader*>(ws + L.header),
+    gather_kernel<<<blocks, 256, 0, s>>>(x, H, k, tile_m, reinterpret_cast<const WsHeader*>(ws + L.header),
                                          reinterpret_cast<const int32_t*>(ws + L.tile_expert),
                                          reinterpret_cast<const int32_t*>(ws + L.pad_offsets),
                                          reinterpret_cast<const int32_t*>(ws + L.offsets),

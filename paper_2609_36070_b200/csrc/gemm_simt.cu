@@ -15,9 +15,9 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(GemmArgs a) {
     __shared__ __align__(16) float Bu[SWIGLU ? 16 : 1][64];
     const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
     const int r0 = blockIdx.y * 64, c0 = blockIdx.x * 64;
-    const int n_rows = (a.dense_rows > 0) ? (a.dense_rows + TILE_M - 1) / TILE_M * TILE_M : *a.n_mtiles * TILE_M;
+    const int n_rows = (a.dense_rows > 0) ? (a.dense_rows + TILE_M - 1) / TILE_M * TILE_M : *a.n_mtiles * a.tile_m;
     if (r0 >= n_rows) return;
-    const int e = (a.dense_rows > 0) ? 0 : a.tile_expert[r0 / TILE_M];
+    const int e = (a.dense_rows > 0) ? 0 : a.tile_expert[r0 / a.tile_m];
     const size_t brow0 = (size_t)e * (SWIGLU ? 2 : 1) * a.N;
     const int lrow = tid >> 2, lk = (tid & 3) * 4;
 

@@ -1,16 +1,23 @@
 // Grouped expert GEMMs on the 5th-generation tensor cores (paper, Section 2.1: f_i(x) = W_down(phi(W_gate x) .* W_up x);
 // Section 3.2: expert FFNs run as persistent, fused kernels that keep the tensor cores fed by pipelining operands).
 //
-// One persistent CTA per SM, 192 threads, warp-specialised:
-//   warp 0      TMA producer : A tile [128 x 64] and B tile [256 x 64] (bf16, 128-byte swizzle) -> 4-stage smem ring
-//   warp 1      MMA issuer   : tcgen05.mma.cta_group::1.kind::f16, M=128 N=256 K=16, fp32 accumulators in TMEM
+// Persistent kernel, one CTA per SM, warp-specialised:
+//   warp 0      TMA producer : A tile [128 x 64] and B tile (bf16, 128-byte swizzle) -> shared-memory ring
+//   warp 1      MMA issuer   : tcgen05.mma.kind::f16, N = 256, K = 16, fp32 accumulators in TMEM
 //                              (2 accumulator stages x 256 columns = all 512 TMEM columns)
-//   warps 2..5  epilogue     : tcgen05.ld -> registers -> (SwiGLU) -> bf16 -> global
-// Tiles are handed out statically (tile L -> CTA L mod grid) in the order expert-major, then N tile, then M tile,
-// so that CTAs running side by side share the same weight tile through L2 and an expert's activations stay L2
-// resident while its N tiles stream.  The tile tables come from the on-device schedule; nothing is read back.
-// Every output element is produced by exactly one tile with a fixed k order, so results do not depend on the
-// grid size or on timing (Section 3.4 "Determinism").
+//   warps 2..5  epilogue     : tcgen05.ld -> registers -> (SwiGLU) -> bf16 -> swizzled smem slab -> TMA store
+//   warps 6..9  gather       : only in the GATHER instantiation, see below
+// CTAS = 1: every CTA computes 128 x 256 tiles on its own (cta_group::1, 4 stages of 48 KB).
+// CTAS = 2: two CTAs of a cluster compute one 256 x 256 tile with cta_group::2 MMAs issued by the even CTA: each CTA
+//           stages its own 128 rows of A and HALF of the B tile (128 of the 256 weight rows), so a k-block moves
+//           32 KB instead of 48 KB from L2 into each SM and the ring holds 6 stages.  The odd CTA's warp 1 forwards
+//           "my stage has landed" to the even CTA; tcgen05.commit multicasts "stage free" / "accumulator ready" to
+//           both CTAs; each CTA drains its own 128 accumulator rows.  No TMA multicast is used.
+// Tiles are handed out statically (tile L -> CTA or pair L mod grid) in the order expert, M group, N tile, M tile, so
+// that CTAs running side by side share the same weight tile through L2 while an expert's activations stay L2
+// resident.  The tile tables come from the on-device schedule; nothing is read back.  Every output element is
+// produced by exactly one tile with a fixed k order, so results do not depend on the grid size or on timing
+// (Section 3.4 "Determinism").
 //
 //   EPI_SWIGLU : B = [E, 2N, K]; the 256-wide B tile is 128 gate rows followed by the matching 128 up rows and the
 //                epilogue writes C[:, n*128 .. n*128+127] = silu(gate) * up (bf16).
@@ -28,24 +35,26 @@
 namespace mok {
 namespace tc {
 
-constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4, UMMA_K = 16;
+constexpr int BM = 128, BN = 256, BK = 64, UMMA_K = 16;
 constexpr int A_BYTES = BM * BK * 2;           // 16 KB
-constexpr int B_BYTES = BN * BK * 2;           // 32 KB
-constexpr int STAGE_BYTES = A_BYTES + B_BYTES; // 48 KB
+constexpr int B_BYTES = BN * BK * 2;           // 32 KB (whole tile; a CTA of a pair stages half of it)
+constexpr int MAX_STAGES = 6;
 constexpr int ACC_STAGES = 2, TMEM_COLS = 512;
-constexpr int THREADS = 192;                  // + 4 gather warps in the GATHER instantiation
+constexpr int THREADS = 192;                   // + 4 gather warps in the GATHER instantiation
 constexpr int GATHER_THREADS = 128;
-constexpr int GROUP_M = 16;                    // M tiles per rasterisation group
+constexpr int GROUP_ROWS = 2048;               // rows of one rasterisation group (16 tiles of 128 rows)
 constexpr int SMEM_CTRL = 256;
 constexpr int OUT_STAGE_BYTES = 4 * 8192;      // per epilogue warp: 32 rows x 128 bf16 columns, as two swizzled boxes
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + OUT_STAGE_BYTES + SMEM_CTRL + 1024;   // + slack for alignment
-constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;            // 2 s
+constexpr int RING_BYTES = 196608;             // 4 x 48 KB or 6 x 32 KB
+constexpr int SMEM_BYTES = RING_BYTES + OUT_STAGE_BYTES + SMEM_CTRL + 1024;   // + slack for 1024-byte alignment
+constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;                    // 2 s
 
 struct Ctrl {
-    uint64_t full[STAGES];
-    uint64_t empty[STAGES];
-    uint64_t tfull[ACC_STAGES];
-    uint64_t tempty[ACC_STAGES];
+    uint64_t full[MAX_STAGES];     // this CTA's stage has landed (TMA bytes + gather arrivals)
+    uint64_t pfull[MAX_STAGES];    // even CTA only: the odd CTA's stage has landed
+    uint64_t empty[MAX_STAGES];    // the MMAs reading the stage have retired
+    uint64_t tfull[ACC_STAGES];    // accumulator stage complete
+    uint64_t tempty[ACC_STAGES];   // accumulator stage drained by every epilogue warp (of both CTAs)
     uint32_t tmem_base;
     uint32_t abort;
 };
@@ -57,6 +66,14 @@ __device__ __forceinline__ unsigned long long globaltimer() {
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
@@ -66,11 +83,19 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
+// Arrive on the barrier at the same shared-memory offset in CTA `rank` of the cluster.
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t bar, uint32_t rank) {
+    asm volatile(
+        "{\n\t.reg .b32 ra;\n\t"
+        "mapa.shared::cluster.u32 ra, %0, %1;\n\t"
+        "mbarrier.arrive.release.cluster.shared::cluster.b64 _, [ra];\n\t}"
+        ::"r"(bar), "r"(rank) : "memory");
+}
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
@@ -104,7 +129,6 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
         ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1) : "memory");
 }
-
 // 16-byte asynchronous global -> shared copy (src_bytes = 0 writes zeros), and the arrive that fires on the
 // mbarrier once all earlier cp.async of this thread have landed (it counts as one of the expected arrivals).
 __device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src, uint32_t src_bytes) {
@@ -113,7 +137,6 @@ __device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src, uint3
 __device__ __forceinline__ void cp_async_mbar_arrive(uint32_t bar) {
     asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
 }
-
 // Shared -> global tile store (bulk async group); out-of-range rows / columns of the box are clipped by the map.
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int c0, int c1) {
     asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
@@ -128,16 +151,34 @@ __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// Arrive on `bar` once all MMAs issued so far by this thread have retired.  For a CTA pair the arrive is multicast
+// to the barrier at the same offset in both CTAs.
+template <int CTAS>
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    if (CTAS == 1) {
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    } else {
+        const uint16_t mask = 3;
+        asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                     ::"r"(bar), "h"(mask) : "memory");
+    }
 }
-// D[tmem] (+)= A[smem] * B[smem]^T, M=128, N=256, K=16, bf16 inputs, fp32 accumulate.
+// D[tmem] (+)= A[smem] * B[smem]^T, M = 128 x CTAS, N = 256, K = 16, bf16 inputs, fp32 accumulate.
+template <int CTAS>
 __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+    if (CTAS == 1) {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+    } else {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+    }
 }
 // 32 lanes x 32 consecutive fp32 columns: thread i of the warp gets lane (base + i), registers = columns.
 __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
@@ -164,12 +205,18 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr) {
     d |= (uint64_t)2 << 61;                           // 128-byte swizzle
     return d;
 }
-// Instruction descriptor: D fp32, A/B bf16, both K-major, dense, M=128, N=256.
-constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+// Instruction descriptor: D fp32, A/B bf16, both K-major, dense, M = 128 x CTAS, N = 256.
+template <int CTAS>
+__device__ __forceinline__ constexpr uint32_t make_idesc() {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((BM * CTAS) >> 4) << 24);
+}
 
-struct Tile { int row0, n, e, m; };
+struct Tile { int row0, n, e, m; };   // row0: first row of the (pair) tile in the padded row space
 
-__device__ __forceinline__ Tile decode_tile(const GemmArgs& a, int L, int n_nt, int n_mt_total) {
+// Tile L of the static schedule.  `tm` = rows per tile (128 x CTAS).  Inside an expert, M tiles are taken in groups
+// of GROUP_ROWS rows: all N tiles of a group before the next group, M fastest, so the group's activations stay in
+// L2 while the expert's weight tiles stream.
+__device__ __forceinline__ Tile decode_tile(const GemmArgs& a, int L, int n_nt, int n_mt_total, int tm) {
     Tile t;
     int mt0, m_cnt;
     if (a.dense_rows > 0) {
@@ -179,16 +226,15 @@ __device__ __forceinline__ Tile decode_tile(const GemmArgs& a, int L, int n_nt, 
         mt0 = __ldg(a.mt_start + t.e);
         m_cnt = __ldg(a.mt_start + t.e + 1) - mt0;
     }
-    // Inside an expert, M tiles are taken in groups of GROUP_M: all N tiles of a group before the next group, M
-    // fastest.  The group's activations (GROUP_M x 128 rows) then stay in L2 while the expert's weight tiles stream.
+    const int group_m = GROUP_ROWS / tm;
     const int r = L - n_nt * mt0;
-    const int per_group = GROUP_M * n_nt;
+    const int per_group = group_m * n_nt;
     const int g = r / per_group;
     const int rem = r - g * per_group;
-    const int in_group = min(GROUP_M, m_cnt - g * GROUP_M);
+    const int in_group = min(group_m, m_cnt - g * group_m);
     t.n = rem / in_group;
-    t.m = g * GROUP_M + (rem - t.n * in_group);
-    t.row0 = (mt0 + t.m) * BM;
+    t.m = g * group_m + (rem - t.n * in_group);
+    t.row0 = (mt0 + t.m) * tm;
     return t;
 }
 
@@ -197,40 +243,58 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
-template <int EPI, bool GATHER>
+template <int EPI, bool GATHER, int CTAS>
 __global__ void __launch_bounds__(THREADS + (GATHER ? GATHER_THREADS : 0), 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
                const __grid_constant__ CUtensorMap tmapC, const GemmArgs a, const int n_nt, const int k_blocks) {
     constexpr bool SWIGLU = (EPI == EPI_SWIGLU);
+    constexpr int STAGES = (CTAS == 2) ? 6 : 4;
+    constexpr int B_STAGE = B_BYTES / CTAS;                 // B bytes this CTA stages per k-block
+    constexpr int STAGE_BYTES = A_BYTES + B_STAGE;
+    constexpr int TM = BM * CTAS;                           // rows of one (pair) tile
+    static_assert(STAGES * STAGE_BYTES == RING_BYTES, "ring size");
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t* smem = smem_raw + (base - raw);
-    Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem + STAGES * STAGE_BYTES + OUT_STAGE_BYTES);
+    Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem + RING_BYTES + OUT_STAGE_BYTES);
     volatile uint32_t* abort_flag = &ctrl->abort;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int rank = (CTAS == 2) ? (int)cluster_ctarank() : 0;      // 0 = the CTA that issues the MMAs
+    const int unit = blockIdx.x / CTAS, n_units = gridDim.x / CTAS;   // CTA (or pair) index in the static schedule
 
-    int n_mt_total = (a.dense_rows > 0) ? (a.dense_rows + BM - 1) / BM : *a.n_mtiles;
+    int n_mt_total = (a.dense_rows > 0) ? (a.dense_rows + TM - 1) / TM : *a.n_mtiles;
     if (n_mt_total > a.max_mt) n_mt_total = a.max_mt;
     const int total = n_mt_total * n_nt;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(smem_u32(&ctrl->full[s]), GATHER ? 1 + GATHER_THREADS : 1);
+            mbar_init(smem_u32(&ctrl->pfull[s]), 1);
             mbar_init(smem_u32(&ctrl->empty[s]), 1);
         }
-        for (int s = 0; s < ACC_STAGES; ++s) { mbar_init(smem_u32(&ctrl->tfull[s]), 1); mbar_init(smem_u32(&ctrl->tempty[s]), 128); }
+        for (int s = 0; s < ACC_STAGES; ++s) {
+            mbar_init(smem_u32(&ctrl->tfull[s]), 1);
+            mbar_init(smem_u32(&ctrl->tempty[s]), 4 * CTAS);       // one arrive per epilogue warp of each CTA
+        }
         ctrl->abort = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(smem_u32(&ctrl->tmem_base)), "r"((uint32_t)TMEM_COLS) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        if (CTAS == 1) {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                         ::"r"(smem_u32(&ctrl->tmem_base)), "r"((uint32_t)TMEM_COLS) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                         ::"r"(smem_u32(&ctrl->tmem_base)), "r"((uint32_t)TMEM_COLS) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        }
     }
     tc_fence_before();
     __syncthreads();
+    if (CTAS == 2) cluster_sync();          // the peer's barriers exist before anyone arrives on them remotely
     tc_fence_after();
     const uint32_t tmem_base = ctrl->tmem_base;
 
@@ -240,8 +304,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
             int s = 0;
             uint32_t ph = 0;
             const int b_rows_per_expert = (SWIGLU ? 2 : 1) * a.N;
-            for (int L = blockIdx.x; L < total; L += gridDim.x) {
-                const Tile t = decode_tile(a, L, n_nt, n_mt_total);
+            for (int L = unit; L < total; L += n_units) {
+                const Tile t = decode_tile(a, L, n_nt, n_mt_total, TM);
+                // weight rows of this tile: [gate 128 | up 128] for SwiGLU, 256 consecutive rows otherwise; a CTA
+                // of a pair stages only its half (rank 0: first 128 rows, rank 1: second 128 rows)
                 const int brow0 = t.e * b_rows_per_expert + (SWIGLU ? t.n * (BN / 2) : t.n * BN);
                 const int brow1 = SWIGLU ? brow0 + a.N : brow0 + BN / 2;
                 bool ok = true;
@@ -250,10 +316,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
                     if (!ok) break;
                     const uint32_t full = smem_u32(&ctrl->full[s]);
                     const uint32_t sa = base + s * STAGE_BYTES, sb = sa + A_BYTES;
-                    mbar_expect_tx(full, GATHER ? B_BYTES : STAGE_BYTES);
-                    if (!GATHER) tma_load_2d(sa, &tmapA, full, kb * BK, t.row0);
-                    tma_load_2d(sb, &tmapB, full, kb * BK, brow0);
-                    tma_load_2d(sb + B_BYTES / 2, &tmapB, full, kb * BK, brow1);
+                    mbar_expect_tx(full, GATHER ? B_STAGE : STAGE_BYTES);
+                    if (!GATHER) tma_load_2d(sa, &tmapA, full, kb * BK, t.row0 + rank * BM);
+                    if (CTAS == 1) {
+                        tma_load_2d(sb, &tmapB, full, kb * BK, brow0);
+                        tma_load_2d(sb + B_BYTES / 2, &tmapB, full, kb * BK, brow1);
+                    } else {
+                        tma_load_2d(sb, &tmapB, full, kb * BK, rank == 0 ? brow0 : brow1);
+                    }
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
                 if (!ok) break;
@@ -261,30 +331,45 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
         }
         __syncwarp();
     } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        if (lane == 0 && rank == 0) {
+            // -------------------------------------------------------------- MMA issuer (even CTA of a pair)
+            constexpr uint32_t idesc = make_idesc<CTAS>();
             int s = 0, as = 0;
             uint32_t ph = 0, aph = 0;
-            for (int L = blockIdx.x; L < total; L += gridDim.x) {
+            for (int L = unit; L < total; L += n_units) {
                 bool ok = mbar_wait(smem_u32(&ctrl->tempty[as]), aph ^ 1u, abort_flag, a.header, 2);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(as * BN);
                 for (int kb = 0; kb < k_blocks; ++kb) {
                     ok = mbar_wait(smem_u32(&ctrl->full[s]), ph, abort_flag, a.header, 3);
+                    if (ok && CTAS == 2) ok = mbar_wait(smem_u32(&ctrl->pfull[s]), ph, abort_flag, a.header, 6);
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t sa = base + s * STAGE_BYTES, sb = sa + A_BYTES;
                     const uint64_t adesc = make_smem_desc(sa), bdesc = make_smem_desc(sb);
 #pragma unroll
                     for (int j = 0; j < BK / UMMA_K; ++j)   // +32 bytes per K=16 step inside the 128-byte swizzle row
-                        tc_mma(d_tmem, adesc + (uint64_t)(j * 2), bdesc + (uint64_t)(j * 2), IDESC, (kb | j) ? 1u : 0u);
-                    tc_commit(smem_u32(&ctrl->empty[s]));     // frees the smem stage when these MMAs retire
+                        tc_mma<CTAS>(d_tmem, adesc + (uint64_t)(j * 2), bdesc + (uint64_t)(j * 2), idesc, (kb | j) ? 1u : 0u);
+                    tc_commit<CTAS>(smem_u32(&ctrl->empty[s]));   // frees the smem stage (in both CTAs) when these MMAs retire
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
                 if (!ok) break;
-                tc_commit(smem_u32(&ctrl->tfull[as]));        // accumulator complete
+                tc_commit<CTAS>(smem_u32(&ctrl->tfull[as]));      // accumulator complete (in both CTAs)
                 if (++as == ACC_STAGES) { as = 0; aph ^= 1u; }
+            }
+        } else if (lane == 0 && CTAS == 2) {
+            // -------------------------------------------------------------- odd CTA: tell the even CTA that my stage landed
+            int s = 0;
+            uint32_t ph = 0;
+            bool ok = true;
+            for (int L = unit; L < total && ok; L += n_units) {
+                for (int kb = 0; kb < k_blocks; ++kb) {
+                    ok = mbar_wait(smem_u32(&ctrl->full[s]), ph, abort_flag, a.header, 7);
+                    if (!ok) break;
+                    mbar_arrive_remote(smem_u32(&ctrl->pfull[s]), 0);
+                    if (++s == STAGES) { s = 0; ph ^= 1u; }
+                }
             }
         }
         __syncwarp();
@@ -292,19 +377,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
         // ------------------------------------------------------------------ gather warps 6..9 (pull dispatch)
         // Warp gw owns tile rows 32 gw .. 32 gw + 31.  Lane = (sub-row 0..3, 16-byte chunk 0..7); pass i covers rows
         // 32 gw + 4 i + sub-row.  Chunk c of row r lands at r*128 + ((c ^ (r & 7)) * 16): the 128-byte swizzle the
-        // UMMA descriptor expects.  Rows past the expert's segment re-read the tile's first row (never stored).
+        // UMMA descriptor expects.  Rows past the expert's segment re-read the tile's first row (never combined).
         const int gw = warp - 6, sub = lane >> 3, chunk = lane & 7;
         int s = 0;
         uint32_t ph = 0;
-        for (int L = blockIdx.x; L < total; L += gridDim.x) {
-            const Tile t = decode_tile(a, L, n_nt, n_mt_total);
-            const int valid = __ldg(a.counts + t.e) - t.m * BM;
+        for (int L = unit; L < total; L += n_units) {
+            const Tile t = decode_tile(a, L, n_nt, n_mt_total, TM);
+            const int valid = __ldg(a.counts + t.e) - t.m * TM - rank * BM;
             const int tok0 = __ldg(a.row_token + t.row0);
+            const int* rows = a.row_token + t.row0 + rank * BM;
             const __nv_bfloat16* src[8];
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 const int r = gw * 32 + i * 4 + sub;
-                const int tok = (r < valid) ? __ldg(a.row_token + t.row0 + r) : tok0;
+                const int tok = (r < valid) ? __ldg(rows + r) : tok0;
                 src[i] = a.A + (size_t)tok * a.K + chunk * 8;
             }
             bool ok = true;
@@ -332,17 +418,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
         // 32 accumulator rows and stages 128 output columns at a time as two [32 rows x 64 columns] boxes, so the
         // global writes are whole 128-byte lines and the warp only synchronises with itself.
         const int quad = warp & 3;                            // TMEM lane quadrant this warp may access
-        const uint32_t slab = base + STAGES * STAGE_BYTES + quad * 8192;
+        const uint32_t slab = base + RING_BYTES + quad * 8192;
         int as = 0;
         uint32_t aph = 0;
-        for (int L = blockIdx.x; L < total; L += gridDim.x) {
-            const Tile t = decode_tile(a, L, n_nt, n_mt_total);
+        for (int L = unit; L < total; L += n_units) {
+            const Tile t = decode_tile(a, L, n_nt, n_mt_total, TM);
             bool ok = mbar_wait(smem_u32(&ctrl->tfull[as]), aph, abort_flag, a.header, 4);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(as * BN);
-            const int row = t.row0 + quad * 32;
+            const int row = t.row0 + rank * BM + quad * 32;
             if (EPI == EPI_F32) {
                 float* frow = reinterpret_cast<float*>(a.C) + (size_t)(row + lane) * a.ldc;
                 const int c0 = t.n * BN;
@@ -359,7 +445,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
                     }
                 }
                 tc_fence_before();
-                mbar_arrive(smem_u32(&ctrl->tempty[as]));
+                __syncwarp();
+                if (lane == 0) {
+                    if (rank == 0) mbar_arrive(smem_u32(&ctrl->tempty[as]));
+                    else mbar_arrive_remote(smem_u32(&ctrl->tempty[as]), 0);
+                }
             } else {
                 constexpr int HALVES = SWIGLU ? 1 : 2;        // 128 output columns per pass
                 const int c0 = SWIGLU ? t.n * (BN / 2) : t.n * BN;
@@ -397,13 +487,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
                             st_shared_v4(box + ((cc ^ (lane & 7)) << 4), o[4 * v], o[4 * v + 1], o[4 * v + 2], o[4 * v + 3]);
                         }
                     }
-                    if (half == HALVES - 1) {                 // all TMEM reads of this tile are done
-                        tc_fence_before();
-                        mbar_arrive(smem_u32(&ctrl->tempty[as]));
-                    }
+                    if (half == HALVES - 1) tc_fence_before();   // all TMEM reads of this tile are done
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     __syncwarp();
                     if (lane == 0) {
+                        if (half == HALVES - 1) {             // hand the accumulator stage back to the MMA issuer
+                            if (rank == 0) mbar_arrive(smem_u32(&ctrl->tempty[as]));
+                            else mbar_arrive_remote(smem_u32(&ctrl->tempty[as]), 0);
+                        }
                         const int col = c0 + half * 128;
                         if (col < a.N) tma_store_2d(&tmapC, slab, col, row);
                         if (col + 64 < a.N) tma_store_2d(&tmapC, slab + 4096, col + 64, row);
@@ -424,9 +515,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
     }
     tc_fence_before();
     __syncthreads();
+    if (CTAS == 2) cluster_sync();          // neither CTA frees TMEM or exits while the other may still touch it
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS) : "memory");
+        if (CTAS == 1)
+            asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS) : "memory");
+        else
+            asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS) : "memory");
     }
 }
 
@@ -462,24 +557,55 @@ static bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t co
 
 }  // namespace tc
 
-template <int EPI, bool GATHER>
+// Grid of the persistent kernel: one CTA per SM, or as many CTA pairs as can be co-resident.
+template <int EPI, bool GATHER, int CTAS>
 static cudaError_t launch_one(const CUtensorMap& mA, const CUtensorMap& mB, const CUtensorMap& mC, const GemmArgs& a,
                               int n_nt, int k_blocks, int grid, cudaStream_t s) {
     using namespace tc;
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<EPI, GATHER>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             SMEM_BYTES);
-        if (e != cudaSuccess) return e;
-        configured = true;
+    static int max_units = 0;
+    const int threads = THREADS + (GATHER ? GATHER_THREADS : 0);
+    auto kernel = gemm_tc_kernel<EPI, GATHER, CTAS>;
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    cfg.blockDim = dim3(threads);
+    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cfg.stream = s;
+    cfg.numAttrs = 0;
+    if (CTAS == 2) {
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
     }
-    gemm_tc_kernel<EPI, GATHER><<<grid, THREADS + (GATHER ? GATHER_THREADS : 0), SMEM_BYTES, s>>>(mA, mB, mC, a, n_nt, k_blocks);
-    return cudaGetLastError();
+    if (!max_units) {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        int dev = 0, sms = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (CTAS == 2) {
+            int clusters = 0;
+            cfg.gridDim = dim3(sms / 2 * 2);
+            e = cudaOccupancyMaxActiveClusters(&clusters, kernel, &cfg);
+            if (e != cudaSuccess) return e;
+            if (clusters < 1) return cudaErrorInvalidConfiguration;
+            max_units = clusters < sms / 2 ? clusters : sms / 2;
+        } else {
+            max_units = sms;
+        }
+    }
+    int units = (grid <= 0) ? max_units : (grid + CTAS - 1) / CTAS;
+    if (units > max_units) units = max_units;
+    cfg.gridDim = dim3(units * CTAS);
+    return cudaLaunchKernelEx(&cfg, kernel, mA, mB, mC, a, n_nt, k_blocks);
 }
 
 cudaError_t launch_gemm_tc(const GemmArgs& a, int epi, int grid, cudaStream_t s) {
     using namespace tc;
-    const bool swiglu = (epi == EPI_SWIGLU), gather = (a.row_token != nullptr);
+    const bool swiglu = (epi == EPI_SWIGLU), gather = (a.row_token != nullptr), pair = (a.tile_m == 2 * BM);
+    if (a.tile_m != BM && a.tile_m != 2 * BM) return cudaErrorInvalidValue;
     CUtensorMap mA, mB, mC;
     const uint64_t b_rows = (uint64_t)a.E * (swiglu ? 2 : 1) * a.N;
     if (!make_map(&mA, a.A, (uint64_t)a.a_rows, (uint64_t)a.K, BM)) return cudaErrorInvalidValue;
@@ -488,17 +614,17 @@ cudaError_t launch_gemm_tc(const GemmArgs& a, int epi, int grid, cudaStream_t s)
     else if (!make_map(&mC, a.C, (uint64_t)a.rows_pad, (uint64_t)a.N, 32, (uint64_t)a.ldc)) return cudaErrorInvalidValue;
     const int n_nt = swiglu ? (a.N + BN / 2 - 1) / (BN / 2) : (a.N + BN - 1) / BN;
     const int k_blocks = (a.K + BK - 1) / BK;
-    static int sm_count = 0;
-    if (!sm_count) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
+    if (pair) {
+        if (epi == EPI_SWIGLU && gather) return launch_one<EPI_SWIGLU, true, 2>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
+        if (epi == EPI_SWIGLU) return launch_one<EPI_SWIGLU, false, 2>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
+        if (epi == EPI_BF16 && !gather) return launch_one<EPI_BF16, false, 2>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
+        if (epi == EPI_F32 && !gather) return launch_one<EPI_F32, false, 2>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
+    } else {
+        if (epi == EPI_SWIGLU && gather) return launch_one<EPI_SWIGLU, true, 1>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
+        if (epi == EPI_SWIGLU) return launch_one<EPI_SWIGLU, false, 1>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
+        if (epi == EPI_BF16 && !gather) return launch_one<EPI_BF16, false, 1>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
+        if (epi == EPI_F32 && !gather) return launch_one<EPI_F32, false, 1>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
     }
-    if (grid <= 0 || grid > sm_count) grid = sm_count;
-    if (epi == EPI_SWIGLU && gather) return launch_one<EPI_SWIGLU, true>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
-    if (epi == EPI_SWIGLU) return launch_one<EPI_SWIGLU, false>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
-    if (epi == EPI_BF16 && !gather) return launch_one<EPI_BF16, false>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
-    if (epi == EPI_F32 && !gather) return launch_one<EPI_F32, false>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
     return cudaErrorInvalidValue;
 }
 

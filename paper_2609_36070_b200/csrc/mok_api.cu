@@ -39,13 +39,13 @@ bool ws_layout(int T, int H, int I, int Is, int E, int k, WsLayout* L) {
     memset(L, 0, sizeof(*L));
     const long long R = (long long)T * k;
     const long long nonempty_max = R < E ? R : E;
-    long long Rpad = (R + nonempty_max * (TILE_M - 1) + TILE_M - 1) / TILE_M * TILE_M;
-    if (Rpad < TILE_M) Rpad = TILE_M;
+    long long Rpad = (R + nonempty_max * (2 * TILE_M - 1) + 2 * TILE_M - 1) / (2 * TILE_M) * (2 * TILE_M);
+    if (Rpad < 2 * TILE_M) Rpad = 2 * TILE_M;
     L->R = (int32_t)R;
     L->Rpad = (int32_t)Rpad;
     L->max_mt = (int32_t)(Rpad / TILE_M);
-    L->Tpad = (T + TILE_M - 1) / TILE_M * TILE_M;
-    if (L->Tpad < TILE_M) L->Tpad = TILE_M;
+    L->Tpad = (T + 2 * TILE_M - 1) / (2 * TILE_M) * (2 * TILE_M);
+    if (L->Tpad < 2 * TILE_M) L->Tpad = 2 * TILE_M;
     L->n_blk = (int32_t)((R + SCHED_CHUNK - 1) / SCHED_CHUNK);
     if (L->n_blk < 1) L->n_blk = 1;
     size_t off = 0;
@@ -91,7 +91,8 @@ static int validate(const mok_args* a, WsLayout* L, size_t extra_ws) {
         return MOK_ERR_WORKSPACE;
     if (a->config && (a->config->impl < 0 || a->config->impl > 1 || a->config->grid < 0 ||
                       a->config->router_impl < 0 || a->config->router_impl > 2 ||
-                      a->config->gather_mode < 0 || a->config->gather_mode > 2))
+                      a->config->gather_mode < 0 || a->config->gather_mode > 2 ||
+                      a->config->cta_group < 0 || a->config->cta_group > 2))
         return MOK_ERR_SHAPE;
     return MOK_OK;
 }
@@ -112,6 +113,12 @@ static bool fused_gather(const mok_config* cfg, int I) {
     return (I + 127) / 128 <= 32;
 }
 
+// Rows of one tile of the padded row space: 256 when the GEMMs run on CTA pairs (cta_group::2), else 128.
+static int tile_rows(const mok_config* cfg) {
+    if (use_simt(cfg)) return TILE_M;
+    return (cfg && cfg->cta_group == 2) ? 2 * TILE_M : TILE_M;   // pairs are correct but not yet faster: off by default
+}
+
 static int run_gemm(const GemmArgs& g, bool swiglu, const mok_config* cfg, cudaStream_t s) {
     cudaError_t e = use_simt(cfg) ? launch_gemm_simt(g, swiglu, s)
                                   : launch_gemm_tc(g, swiglu ? EPI_SWIGLU : EPI_BF16, cfg ? cfg->grid : 0, s);
@@ -126,7 +133,8 @@ static int route_stage(const mok_args* a, const WsLayout& L, char* ws, const __n
         e = launch_router_simt(x, a->W_router, a->router_bias, a->T, a->H, a->E, a->k, idx, w, s);
     else
         e = launch_router_tc(x, a->W_router, a->router_bias, a->T, a->H, a->E, a->k, L, ws,
-                             reinterpret_cast<WsHeader*>(ws + L.header), a->config ? a->config->grid : 0, idx, w, s);
+                             reinterpret_cast<WsHeader*>(ws + L.header), a->config ? a->config->grid : 0,
+                             tile_rows(a->config), idx, w, s);
     if (e != cudaSuccess) return cuda_fail(e);
     if (a->topk_idx) {
         e = cudaMemcpyAsync(a->topk_idx, idx, sizeof(int32_t) * (size_t)L.R, cudaMemcpyDeviceToDevice, s);
@@ -152,13 +160,14 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
     int rc = route_stage(a, L, ws, x, s);
     if (rc) return rc;
     MOK_MARK(MOK_STAGE_ROUTER + 1);
-    e = launch_schedule(reinterpret_cast<const int32_t*>(ws + L.idx), a->T, a->E, a->k, L, ws,
+    const int tile_m = tile_rows(a->config);
+    e = launch_schedule(reinterpret_cast<const int32_t*>(ws + L.idx), a->T, a->E, a->k, tile_m, L, ws,
                         a->counts, a->offsets, a->perm, a->inv_perm, s);
     if (e != cudaSuccess) return cuda_fail(e);
     MOK_MARK(MOK_STAGE_SCHEDULE + 1);
     const bool simt = !fused_gather(a->config, a->I);
     if (simt) {   // materialise the expert-sorted copy of x
-        e = launch_gather(x, a->H, a->k, L, ws, s);
+        e = launch_gather(x, a->H, a->k, tile_m, L, ws, s);
         if (e != cudaSuccess) return cuda_fail(e);
     }
     MOK_MARK(MOK_STAGE_GATHER + 1);
@@ -170,6 +179,7 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
     g.tile_expert = reinterpret_cast<const int32_t*>(ws + L.tile_expert);
     g.mt_start = reinterpret_cast<const int32_t*>(ws + L.mt_start);
     g.max_mt = L.max_mt;
+    g.tile_m = tile_m;
     // routed experts: h = silu(Xg Wg^T) * (Xg Wu^T);  y = h Wd^T
     if (simt) {
         g.A = reinterpret_cast<const __nv_bfloat16*>(ws + L.xg);
@@ -324,7 +334,7 @@ int mok_schedule(const int32_t* topk_idx, int T, int E, int k, int32_t* counts, 
     char* ws = reinterpret_cast<char*>(workspace);
     cudaError_t e = cudaMemsetAsync(ws + L.header, 0, sizeof(WsHeader), s);
     if (e != cudaSuccess) return cuda_fail(e);
-    e = launch_schedule(topk_idx, T, E, k, L, ws, counts, offsets, perm, inv_perm, s);
+    e = launch_schedule(topk_idx, T, E, k, TILE_M, L, ws, counts, offsets, perm, inv_perm, s);
     return e == cudaSuccess ? MOK_OK : cuda_fail(e);
 }
 

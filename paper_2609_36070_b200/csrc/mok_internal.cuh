@@ -9,7 +9,8 @@
 
 namespace mok {
 
-constexpr int TILE_M = 128;          // rows of one GEMM tile; expert segments are padded to this internally
+constexpr int TILE_M = 128;          // rows of one CTA's GEMM tile; expert segments are padded internally to tile_m =
+                                     // 128 (single CTAs) or 256 (CTA pairs) rows
 constexpr int SCHED_CHUNK = 2048;    // routes handled by one block of the schedule kernels
 constexpr int MAX_E = 512;
 constexpr int MAX_K = 32;
@@ -31,9 +32,9 @@ struct WsLayout {
     size_t xg, h, y, hs, ysh;
     size_t total;
     int32_t R;            // T*k
-    int32_t Rpad;         // upper bound on padded rows (multiple of 128)
+    int32_t Rpad;         // upper bound on padded rows for either tile_m (multiple of 256)
     int32_t max_mt;       // Rpad / 128
-    int32_t Tpad;         // T rounded up to 128
+    int32_t Tpad;         // T rounded up to 256
     int32_t n_blk;        // schedule blocks
 };
 
@@ -57,23 +58,25 @@ struct GemmArgs {
     const int32_t* tile_expert;  // device [max_mt]
     const int32_t* mt_start;     // device [E+1]
     int32_t max_mt;
+    int32_t tile_m;              // rows of one tile of the padded row space: 128, or 256 for CTA pairs
     WsHeader* header;
 };
 
 // kernels' host launchers (each returns a cudaError_t from the launch)
 cudaError_t launch_router_simt(const __nv_bfloat16* x, const float* Wr, const float* bias, int T, int H, int E, int k,
                                int32_t* idx, float* w, cudaStream_t s);
-cudaError_t launch_schedule(const int32_t* idx, int T, int E, int k, const WsLayout& L, char* ws,
+cudaError_t launch_schedule(const int32_t* idx, int T, int E, int k, int tile_m, const WsLayout& L, char* ws,
                             int32_t* counts_out, int32_t* offsets_out, int32_t* perm_out, int32_t* inv_out,
                             cudaStream_t s);
-cudaError_t launch_gather(const __nv_bfloat16* x, int H, int k, const WsLayout& L, char* ws, cudaStream_t s);
+cudaError_t launch_gather(const __nv_bfloat16* x, int H, int k, int tile_m, const WsLayout& L, char* ws, cudaStream_t s);
 cudaError_t launch_combine(const WsLayout& L, char* ws, int T, int H, int k, bool shared, __nv_bfloat16* out,
                            cudaStream_t s);
 cudaError_t launch_gemm_simt(const GemmArgs& a, bool swiglu, cudaStream_t s);
 enum { EPI_BF16 = 0, EPI_SWIGLU = 1, EPI_F32 = 2 };
 cudaError_t launch_gemm_tc(const GemmArgs& a, int epi, int grid, cudaStream_t s);
 cudaError_t launch_router_tc(const __nv_bfloat16* x, const float* Wr, const float* bias, int T, int H, int E, int k,
-                             const WsLayout& L, char* ws, WsHeader* hdr, int grid, int32_t* idx, float* w, cudaStream_t s);
+                             const WsLayout& L, char* ws, WsHeader* hdr, int grid, int tile_m, int32_t* idx, float* w,
+                             cudaStream_t s);
 
 inline __host__ __device__ size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 

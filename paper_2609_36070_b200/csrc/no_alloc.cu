@@ -14,7 +14,7 @@
 
 namespace mok {
 
-constexpr size_t NOALLOC_SCRATCH_BYTES = 1280u << 10;  // 1.25 MiB: enough for MOK_NOALLOC_MAX_ROUTES routes with E = 512
+constexpr size_t NOALLOC_SCRATCH_BYTES = 1536u << 10;  // 1.5 MiB: enough for MOK_NOALLOC_MAX_ROUTES routes with E = 512
 static __device__ __align__(256) unsigned char g_noalloc_scratch[NOALLOC_SCRATCH_BYTES];
 
 // Device address of the scratch array, looked up once per device.  In host code `g_noalloc_scratch` is only a
@@ -55,6 +55,6 @@ extern "C" int mok_schedule_noalloc(const int32_t* topk_idx, int T, int E, int k
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     cudaError_t e = cudaMemsetAsync(ws + L.header, 0, sizeof(WsHeader), s);   // status / tile count start at zero
     if (e != cudaSuccess) return MOK_ERR_CUDA;
-    e = launch_schedule(topk_idx, T, E, k, L, ws, counts, offsets, perm, inv_perm, s);
+    e = launch_schedule(topk_idx, T, E, k, TILE_M, L, ws, counts, offsets, perm, inv_perm, s);
     return e == cudaSuccess ? MOK_OK : MOK_ERR_CUDA;
 }

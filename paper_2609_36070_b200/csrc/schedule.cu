@@ -6,7 +6,8 @@
 // (Section 3.3), integer arithmetic only, hence bit-reproducible:
 //   1. sched_hist    per-block expert histograms of SCHED_CHUNK consecutive routes
 //   2. sched_scan    one block: per-expert prefix over blocks, counts, offsets, and the internal tile tables
-//                    (each expert's segment padded to a multiple of 128 rows: pad_offsets, mt_start, tile_expert)
+//                    (each expert's segment padded to a multiple of tile_m = 128 or 256 rows: pad_offsets,
+//                    mt_start, tile_expert, all in units of tile_m)
 //   3. sched_scatter stable ranks inside each block (warp match + per-warp running counters) -> perm, inv, pos,
 //                    row_token (padded row -> source token: the {src_index} column of the paper's schedule table)
 // Exported offsets/perm are unpadded; the padding is internal to the GEMM row space.
@@ -35,7 +36,7 @@ sched_hist_kernel(const int32_t* __restrict__ a, int n, int E, int32_t* __restri
 // One block of MAX_E threads.  Thread e walks the blocks for expert e (exclusive prefix, in place), then the
 // block scans over experts.
 __global__ void __launch_bounds__(MAX_E)
-sched_scan_kernel(int32_t* __restrict__ blk_hist, int n_blk, int E, int max_mt,
+sched_scan_kernel(int32_t* __restrict__ blk_hist, int n_blk, int E, int max_mt, int tile_m,
                   int32_t* __restrict__ counts, int32_t* __restrict__ offsets, int32_t* __restrict__ pad_offsets,
                   int32_t* __restrict__ mt_start, int32_t* __restrict__ tile_expert, WsHeader* __restrict__ hdr,
                   int32_t* __restrict__ counts_out, int32_t* __restrict__ offsets_out) {
@@ -57,18 +58,18 @@ sched_scan_kernel(int32_t* __restrict__ blk_hist, int n_blk, int E, int max_mt,
             s_off[i] = off;
             s_mt[i] = mt;
             off += s_cnt[i];
-            mt += (s_cnt[i] + TILE_M - 1) / TILE_M;
+            mt += (s_cnt[i] + tile_m - 1) / tile_m;
         }
         s_off[E] = off;
         s_mt[E] = mt;
         hdr->n_mtiles = mt;
-        if (mt > max_mt) hdr->status = MOK_ERR_SCHEDULE;
+        if (mt * (tile_m / TILE_M) > max_mt) hdr->status = MOK_ERR_SCHEDULE;
     }
     __syncthreads();
     if (e < E) {
         counts[e] = s_cnt[e];
         offsets[e] = s_off[e];
-        pad_offsets[e] = s_mt[e] * TILE_M;
+        pad_offsets[e] = s_mt[e] * tile_m;
         mt_start[e] = s_mt[e];
         if (counts_out) counts_out[e] = s_cnt[e];
         if (offsets_out) offsets_out[e] = s_off[e];
@@ -76,7 +77,7 @@ sched_scan_kernel(int32_t* __restrict__ blk_hist, int n_blk, int E, int max_mt,
     }
     if (e == 0) {
         offsets[E] = s_off[E];
-        pad_offsets[E] = s_mt[E] * TILE_M;
+        pad_offsets[E] = s_mt[E] * tile_m;
         mt_start[E] = s_mt[E];
         if (offsets_out) offsets_out[E] = s_off[E];
     }
@@ -142,7 +143,7 @@ sched_scatter_kernel(const int32_t* __restrict__ a, int n, int E,
     }
 }
 
-cudaError_t launch_schedule(const int32_t* idx, int T, int E, int k, const WsLayout& L, char* ws,
+cudaError_t launch_schedule(const int32_t* idx, int T, int E, int k, int tile_m, const WsLayout& L, char* ws,
                             int32_t* counts_out, int32_t* offsets_out, int32_t* perm_out, int32_t* inv_out,
                             cudaStream_t s) {
     const int n = T * k;
@@ -154,7 +155,7 @@ cudaError_t launch_schedule(const int32_t* idx, int T, int E, int k, const WsLay
     int32_t* tile_expert = reinterpret_cast<int32_t*>(ws + L.tile_expert);
     WsHeader* hdr = reinterpret_cast<WsHeader*>(ws + L.header);
     sched_hist_kernel<<<L.n_blk, SCHED_THREADS, 0, s>>>(idx, n, E, blk_hist);
-    sched_scan_kernel<<<1, MAX_E, 0, s>>>(blk_hist, L.n_blk, E, L.max_mt, counts, offsets, pad_offsets, mt_start,
+    sched_scan_kernel<<<1, MAX_E, 0, s>>>(blk_hist, L.n_blk, E, L.max_mt, tile_m, counts, offsets, pad_offsets, mt_start,
                                           tile_expert, hdr, counts_out, offsets_out);
     sched_scatter_kernel<<<L.n_blk, SCHED_THREADS, sizeof(int32_t) * SCHED_WARPS * E, s>>>(
         idx, n, E, blk_hist, offsets, pad_offsets,

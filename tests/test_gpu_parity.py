@@ -30,12 +30,13 @@ SMALL = [
 
 
 @pytest.mark.parametrize("cfg", SMALL, ids=[c.name for c in SMALL])
-@pytest.mark.parametrize("impl", ["tcgen05_fused_gather", "tcgen05_separate_gather", "simt"])
+@pytest.mark.parametrize("impl", ["tcgen05_fused_gather", "tcgen05_separate_gather", "tcgen05_single_cta", "simt"])
 def test_small_shapes_every_token(cfg, impl):
     m = mok()
     conf = {"simt": m._config(impl=m.MOK_IMPL_SIMT),
             "tcgen05_fused_gather": m._config(gather_mode=1),
-            "tcgen05_separate_gather": m._config(gather_mode=2)}[impl]
+            "tcgen05_separate_gather": m._config(gather_mode=2),
+            "tcgen05_single_cta": m._config(cta_group=1)}[impl]
     out, st, rep = pu.full_parity(cfg, config=conf)
     print(cfg.name, impl, rep)
 
@@ -59,9 +60,10 @@ def test_tiny_config_every_token_and_determinism():
     m = mok()
     out2 = pu.run_gpu(cfg, g, stages=False)
     assert torch.equal(out.view(torch.int16), out2.view(torch.int16))            # run-to-run bitwise identity
-    for grid in (1, 7, 148):                                                       # bits do not depend on the grid
-        o = pu.run_gpu(cfg, g, config=m._config(grid=grid), stages=False)
-        assert torch.equal(out.view(torch.int16), o.view(torch.int16)), grid
+    for grid in (1, 2, 7, 148):                                                    # bits do not depend on the grid,
+        for cta_group in (1, 2):                                                   # nor on single CTAs vs CTA pairs
+            o = pu.run_gpu(cfg, g, config=m._config(grid=grid, cta_group=cta_group), stages=False)
+            assert torch.equal(out.view(torch.int16), o.view(torch.int16)), (grid, cta_group)
 
 
 def test_fourteen_argument_entry_point_matches_ex():

@@ -50,9 +50,9 @@ def test_workspace_size_query(lib):
     assert base > 0 and base % 256 == 0
     assert ws(512, 256, 512, 512, 8, 2) > base                # grows with T
     assert ws(256, 256, 512, 0, 8, 2) < base                  # no shared expert -> smaller
-    # buffers for the padded dispatch space: T*k rows + up to 127 pad rows per non-empty expert
+    # buffers for the padded dispatch space: T*k rows + up to 255 pad rows per non-empty expert (256-row pair tiles)
     T, H, I, E, k = 16384, 2048, 768, 128, 8
-    rows = T * k + 127 * E
+    rows = T * k + 255 * E
     need = 2 * rows * (2 * H + I)
     assert need <= ws(T, H, I, 0, E, k) <= need * 1.1 + (8 << 20)
     for bad in [(256, 250, 512, 0, 8, 2),     # H not a multiple of 8
