@@ -63,7 +63,8 @@ typedef struct mok_config {
                              operand loads (no expert-sorted copy of x), 2 = separate gather kernel + TMA loads */
     int32_t cta_group;    /* tcgen05 GEMMs: 0 = default (1), 1 = one CTA per 128-row tile, 2 = CTA pairs sharing a
                              256-row tile (cta_group::2; halves the weight traffic into each SM) */
-    int32_t reserved[2];
+    int32_t debug;        /* != 0: the tcgen05 GEMMs accumulate wait-time counters (see mok_debug_counters) */
+    int32_t reserved[1];
 } mok_config;
 
 /*
@@ -176,6 +177,15 @@ enum {
 };
 int mok_profile_begin(int max_calls);
 int mok_profile_end(float* ms, int max_calls_out, int* n_calls);
+
+/*
+ * Wait-time counters of the tcgen05 GEMM kernels of the last forward call that ran with config.debug != 0
+ * (measurement aid; Section 3 cost model: T_sync).  Synchronises `stream`, then writes 4 x 8 values: slot 1 = routed
+ * gate/up GEMM, 2 = routed down GEMM, 3 = shared GEMMs; per slot, SM cycles summed over CTAs: MMA issuer waiting for
+ * operands, for the peer CTA's operands, for a free accumulator; MMA issuer total; k-blocks issued; TMA producer
+ * waiting for a free stage; epilogue waiting for an accumulator; epilogue total.
+ */
+int mok_debug_counters(const void* workspace, void* stream, unsigned long long* out);
 
 /* Number of kernels one mok_moe_forward_ex call enqueues for these arguments (the 256-byte header memset is
    not counted); 0 on bad sizes. */

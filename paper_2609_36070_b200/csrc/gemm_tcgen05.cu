@@ -10,8 +10,8 @@
 // CTAS = 1: every CTA computes 128 x 256 tiles on its own (cta_group::1, 4 stages of 48 KB).
 // CTAS = 2: two CTAs of a cluster compute one 256 x 256 tile with cta_group::2 MMAs issued by the even CTA: each CTA
 //           stages its own 128 rows of A and HALF of the B tile (128 of the 256 weight rows), so a k-block moves
-//           32 KB instead of 48 KB from L2 into each SM and the ring holds 6 stages.  The odd CTA's warp 1 forwards
-//           "my stage has landed" to the even CTA; tcgen05.commit multicasts "stage free" / "accumulator ready" to
+//           32 KB instead of 48 KB from L2 into each SM and the ring holds 6 stages.  The odd CTA's TMA loads complete
+//           on the even CTA's mbarrier (its gathered rows are announced by its warp 1); tcgen05.commit multicasts "stage free" / "accumulator ready" to
 //           both CTAs; each CTA drains its own 128 accumulator rows.  No TMA multicast is used.
 // Tiles are handed out statically (tile L -> CTA or pair L mod grid) in the order expert, M group, N tile, M tile, so
 // that CTAs running side by side share the same weight tile through L2 while an expert's activations stay L2
@@ -88,14 +88,14 @@ __device__ __forceinline__ void mbar_arrive_remote(uint32_t bar, uint32_t rank) 
     asm volatile(
         "{\n\t.reg .b32 ra;\n\t"
         "mapa.shared::cluster.u32 ra, %0, %1;\n\t"
-        "mbarrier.arrive.release.cluster.shared::cluster.b64 _, [ra];\n\t}"
+        "mbarrier.arrive.shared::cluster.b64 _, [ra];\n\t}"
         ::"r"(bar), "r"(rank) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
@@ -127,6 +127,15 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+// Same load issued by the odd CTA of a pair: the bytes land in its own shared memory but complete on the barrier at
+// the same offset in the even CTA (cluster rank 0), which is the one the MMA issuer waits on.
+__device__ __forceinline__ void tma_load_2d_peer(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
+    asm volatile(
+        "{\n\t.reg .b32 rb;\n\t"
+        "mapa.shared::cluster.u32 rb, %2, 0;\n\t"
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [rb];\n\t}"
         ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1) : "memory");
 }
 // 16-byte asynchronous global -> shared copy (src_bytes = 0 writes zeros), and the arrive that fires on the
@@ -262,6 +271,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int rank = (CTAS == 2) ? (int)cluster_ctarank() : 0;      // 0 = the CTA that issues the MMAs
     const int unit = blockIdx.x / CTAS, n_units = gridDim.x / CTAS;   // CTA (or pair) index in the static schedule
+    const bool dbg = a.dbg_slot >= 0;
 
     int n_mt_total = (a.dense_rows > 0) ? (a.dense_rows + TM - 1) / TM : *a.n_mtiles;
     if (n_mt_total > a.max_mt) n_mt_total = a.max_mt;
@@ -269,7 +279,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
-            mbar_init(smem_u32(&ctrl->full[s]), GATHER ? 1 + GATHER_THREADS : 1);
+            // arrivals per phase: the producer's expect_tx (not in the odd CTA of a pair, whose TMA bytes complete on
+            // the even CTA's barrier) + one per gather thread
+            const int full_arrivals = ((CTAS == 2 && rank == 1) ? 0 : 1) + (GATHER ? GATHER_THREADS : 0);
+            mbar_init(smem_u32(&ctrl->full[s]), full_arrivals > 0 ? full_arrivals : 1);   // (unused when it would be 0)
             mbar_init(smem_u32(&ctrl->pfull[s]), 1);
             mbar_init(smem_u32(&ctrl->empty[s]), 1);
         }
@@ -303,6 +316,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
         if (lane == 0) {
             int s = 0;
             uint32_t ph = 0;
+            long long dbg_prod = 0;
             const int b_rows_per_expert = (SWIGLU ? 2 : 1) * a.N;
             for (int L = unit; L < total; L += n_units) {
                 const Tile t = decode_tile(a, L, n_nt, n_mt_total, TM);
@@ -312,22 +326,31 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
                 const int brow1 = SWIGLU ? brow0 + a.N : brow0 + BN / 2;
                 bool ok = true;
                 for (int kb = 0; kb < k_blocks; ++kb) {
+                    const long long w0 = dbg ? clock64() : 0;
                     ok = mbar_wait(smem_u32(&ctrl->empty[s]), ph ^ 1u, abort_flag, a.header, 1);
+                    if (dbg) dbg_prod += clock64() - w0;
                     if (!ok) break;
                     const uint32_t full = smem_u32(&ctrl->full[s]);
                     const uint32_t sa = base + s * STAGE_BYTES, sb = sa + A_BYTES;
-                    mbar_expect_tx(full, GATHER ? B_STAGE : STAGE_BYTES);
-                    if (!GATHER) tma_load_2d(sa, &tmapA, full, kb * BK, t.row0 + rank * BM);
                     if (CTAS == 1) {
+                        mbar_expect_tx(full, GATHER ? B_STAGE : STAGE_BYTES);
+                        if (!GATHER) tma_load_2d(sa, &tmapA, full, kb * BK, t.row0);
                         tma_load_2d(sb, &tmapB, full, kb * BK, brow0);
                         tma_load_2d(sb + B_BYTES / 2, &tmapB, full, kb * BK, brow1);
+                    } else if (rank == 0) {
+                        // the even CTA's barrier collects the TMA bytes of both CTAs of the pair
+                        mbar_expect_tx(full, 2 * (GATHER ? B_STAGE : STAGE_BYTES));
+                        if (!GATHER) tma_load_2d(sa, &tmapA, full, kb * BK, t.row0);
+                        tma_load_2d(sb, &tmapB, full, kb * BK, brow0);
                     } else {
-                        tma_load_2d(sb, &tmapB, full, kb * BK, rank == 0 ? brow0 : brow1);
+                        if (!GATHER) tma_load_2d_peer(sa, &tmapA, full, kb * BK, t.row0 + BM);
+                        tma_load_2d_peer(sb, &tmapB, full, kb * BK, brow1);
                     }
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
                 if (!ok) break;
             }
+            if (dbg) atomicAdd(&a.header->dbg[a.dbg_slot][DBG_PROD_WAIT_EMPTY], (unsigned long long)dbg_prod);
         }
         __syncwarp();
     } else if (warp == 1) {
@@ -336,14 +359,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
             constexpr uint32_t idesc = make_idesc<CTAS>();
             int s = 0, as = 0;
             uint32_t ph = 0, aph = 0;
+            long long d_full = 0, d_pfull = 0, d_tempty = 0, d_kb = 0;
+            const long long d_t0 = dbg ? clock64() : 0;
             for (int L = unit; L < total; L += n_units) {
+                long long w0 = dbg ? clock64() : 0;
                 bool ok = mbar_wait(smem_u32(&ctrl->tempty[as]), aph ^ 1u, abort_flag, a.header, 2);
+                if (dbg) d_tempty += clock64() - w0;
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(as * BN);
                 for (int kb = 0; kb < k_blocks; ++kb) {
+                    if (dbg) w0 = clock64();
                     ok = mbar_wait(smem_u32(&ctrl->full[s]), ph, abort_flag, a.header, 3);
-                    if (ok && CTAS == 2) ok = mbar_wait(smem_u32(&ctrl->pfull[s]), ph, abort_flag, a.header, 6);
+                    if (dbg) { const long long w1 = clock64(); d_full += w1 - w0; w0 = w1; ++d_kb; }
+                    if (ok && CTAS == 2 && GATHER) ok = mbar_wait(smem_u32(&ctrl->pfull[s]), ph, abort_flag, a.header, 6);
+                    if (dbg) d_pfull += clock64() - w0;
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t sa = base + s * STAGE_BYTES, sb = sa + A_BYTES;
@@ -358,7 +388,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
                 tc_commit<CTAS>(smem_u32(&ctrl->tfull[as]));      // accumulator complete (in both CTAs)
                 if (++as == ACC_STAGES) { as = 0; aph ^= 1u; }
             }
-        } else if (lane == 0 && CTAS == 2) {
+            if (dbg) {
+                unsigned long long* d = a.header->dbg[a.dbg_slot];
+                atomicAdd(d + DBG_MMA_WAIT_FULL, (unsigned long long)d_full);
+                atomicAdd(d + DBG_MMA_WAIT_PFULL, (unsigned long long)d_pfull);
+                atomicAdd(d + DBG_MMA_WAIT_TEMPTY, (unsigned long long)d_tempty);
+                atomicAdd(d + DBG_MMA_TOTAL, (unsigned long long)(clock64() - d_t0));
+                atomicAdd(d + DBG_KBLOCKS, (unsigned long long)d_kb);
+            }
+        } else if (lane == 0 && CTAS == 2 && GATHER) {
             // -------------------------------------------------------------- odd CTA: tell the even CTA that my stage landed
             int s = 0;
             uint32_t ph = 0;
@@ -421,9 +459,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
         const uint32_t slab = base + RING_BYTES + quad * 8192;
         int as = 0;
         uint32_t aph = 0;
+        long long d_tfull = 0;
+        const long long d_e0 = dbg ? clock64() : 0;
         for (int L = unit; L < total; L += n_units) {
             const Tile t = decode_tile(a, L, n_nt, n_mt_total, TM);
+            const long long w0 = dbg ? clock64() : 0;
             bool ok = mbar_wait(smem_u32(&ctrl->tfull[as]), aph, abort_flag, a.header, 4);
+            if (dbg) d_tfull += clock64() - w0;
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
@@ -506,6 +548,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
         }
         if (lane == 0) tma_store_wait_all();
         __syncwarp();
+        if (dbg && warp == 2 && lane == 0) {
+            atomicAdd(&a.header->dbg[a.dbg_slot][DBG_EPI_WAIT_TFULL], (unsigned long long)d_tfull);
+            atomicAdd(&a.header->dbg[a.dbg_slot][DBG_EPI_TOTAL], (unsigned long long)(clock64() - d_e0));
+        }
     }
 
     // ---------------------------------------------------------------------- teardown

@@ -180,6 +180,8 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
     g.mt_start = reinterpret_cast<const int32_t*>(ws + L.mt_start);
     g.max_mt = L.max_mt;
     g.tile_m = tile_m;
+    const bool dbg = a->config && a->config->debug;
+    g.dbg_slot = dbg ? 1 : -1;
     // routed experts: h = silu(Xg Wg^T) * (Xg Wu^T);  y = h Wd^T
     if (simt) {
         g.A = reinterpret_cast<const __nv_bfloat16*>(ws + L.xg);
@@ -197,6 +199,7 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
     g.row_token = nullptr;
     g.counts = nullptr;
     g.a_rows = L.Rpad;
+    g.dbg_slot = dbg ? 2 : -1;
     MOK_MARK(MOK_STAGE_GEMM1 + 1);
     g.A = reinterpret_cast<const __nv_bfloat16*>(ws + L.h);
     g.B = reinterpret_cast<const __nv_bfloat16*>(a->W_down);
@@ -204,6 +207,7 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
     g.K = a->I; g.N = a->H; g.ldc = a->H;
     if ((rc = run_gemm(g, false, a->config, s))) return rc;
     MOK_MARK(MOK_STAGE_GEMM2 + 1);
+    g.dbg_slot = dbg ? 3 : -1;
     if (a->I_shared > 0) {   // shared expert: every token in natural order, no gather
         g.A = x;
         g.B = reinterpret_cast<const __nv_bfloat16*>(a->W_shared_gate_up);
@@ -346,6 +350,17 @@ int mok_read_status(const void* workspace, void* stream) {
     e = cudaMemcpy(&h, workspace, sizeof(h), cudaMemcpyDeviceToHost);
     if (e != cudaSuccess) return cuda_fail(e);
     return h.status;
+}
+
+int mok_debug_counters(const void* workspace, void* stream, unsigned long long* out) {
+    if (!workspace || !out) return MOK_ERR_NULL;
+    cudaError_t e = cudaStreamSynchronize(reinterpret_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(e);
+    WsHeader h;
+    e = cudaMemcpy(&h, workspace, sizeof(h), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(e);
+    memcpy(out, h.dbg, sizeof(h.dbg));
+    return MOK_OK;
 }
 
 int mok_launch_count(int T, int H, int I, int I_shared, int E, int k, const mok_config* config) {

@@ -21,7 +21,11 @@ struct WsHeader {
     int32_t n_mtiles;      // number of 128-row tiles of the padded dispatch buffer (written by the schedule)
     int32_t where;         // diagnostic: which wait gave up (role * 1000 + site)
     int32_t pad[61];
+    // optional wait-time counters of the tcgen05 GEMMs (config.debug): [slot][counter], SM cycles summed over CTAs
+    unsigned long long dbg[4][8];
 };
+enum { DBG_MMA_WAIT_FULL = 0, DBG_MMA_WAIT_PFULL, DBG_MMA_WAIT_TEMPTY, DBG_MMA_TOTAL, DBG_KBLOCKS,
+       DBG_PROD_WAIT_EMPTY, DBG_EPI_WAIT_TFULL, DBG_EPI_TOTAL };
 
 // Byte offsets of every workspace region, computed on the host from the sizes alone (no readback).
 struct WsLayout {
@@ -59,6 +63,7 @@ struct GemmArgs {
     const int32_t* mt_start;     // device [E+1]
     int32_t max_mt;
     int32_t tile_m;              // rows of one tile of the padded row space: 128, or 256 for CTA pairs
+    int32_t dbg_slot;            // >= 0: accumulate wait-time counters into header->dbg[dbg_slot]
     WsHeader* header;
 };
 

@@ -125,6 +125,7 @@ cudaError_t launch_router_tc(const __nv_bfloat16* x, const float* Wr, const floa
     g.rows_pad = L.Tpad; g.a_rows = T; g.dense_rows = T;
     g.max_mt = L.Tpad / TILE_M;
     g.tile_m = tile_m;
+    g.dbg_slot = -1;
     g.header = hdr;
     e = launch_gemm_tc(g, EPI_F32, grid, s);
     if (e != cudaSuccess) return e;

@@ -21,7 +21,7 @@ MOK_IMPL_TCGEN05, MOK_IMPL_SIMT = 0, 1
 
 EXPORTS = ["mok_moe_forward", "mok_workspace_bytes", "mok_moe_forward_ex", "mok_moe_forward_host", "mok_route",
            "mok_schedule", "mok_read_status", "mok_launch_count", "mok_last_cuda_error", "mok_status_string",
-           "mok_version", "mok_profile_begin", "mok_profile_end", "mok_schedule_noalloc"]
+           "mok_version", "mok_profile_begin", "mok_profile_end", "mok_schedule_noalloc", "mok_debug_counters"]
 MOK_NOALLOC_MAX_ROUTES = 32768
 STAGES = ["router", "schedule", "gather", "gemm1", "gemm2", "shared_gemm1", "shared_gemm2", "combine"]
 
@@ -29,7 +29,7 @@ STAGES = ["router", "schedule", "gather", "gemm1", "gemm2", "shared_gemm1", "sha
 class mok_config(ctypes.Structure):
     _fields_ = [("impl", ctypes.c_int32), ("grid", ctypes.c_int32), ("router_impl", ctypes.c_int32),
                 ("profile", ctypes.c_int32), ("gather_mode", ctypes.c_int32), ("cta_group", ctypes.c_int32),
-                ("reserved", ctypes.c_int32 * 2)]
+                ("debug", ctypes.c_int32), ("reserved", ctypes.c_int32 * 1)]
 
 
 class mok_args(ctypes.Structure):
@@ -60,6 +60,8 @@ _lib.mok_schedule.argtypes = ([ctypes.c_void_p] + [ctypes.c_int] * 3 + [ctypes.c
                               [ctypes.c_size_t, ctypes.c_void_p])
 _lib.mok_schedule_noalloc.restype = ctypes.c_int
 _lib.mok_schedule_noalloc.argtypes = [ctypes.c_void_p] + [ctypes.c_int] * 3 + [ctypes.c_void_p] * 5
+_lib.mok_debug_counters.restype = ctypes.c_int
+_lib.mok_debug_counters.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
 _lib.mok_read_status.restype = ctypes.c_int
 _lib.mok_read_status.argtypes = [ctypes.c_void_p, ctypes.c_void_p]
 _lib.mok_launch_count.restype = ctypes.c_int
@@ -98,10 +100,11 @@ def _stream(stream):
     return ctypes.c_void_p(stream.cuda_stream)
 
 
-def _config(impl=0, grid=0, router_impl=0, profile=0, gather_mode=0, cta_group=0):
+def _config(impl=0, grid=0, router_impl=0, profile=0, gather_mode=0, cta_group=0, debug=0):
     c = mok_config()
     c.impl, c.grid, c.router_impl, c.profile, c.gather_mode = impl, grid, router_impl, profile, gather_mode
     c.cta_group = cta_group
+    c.debug = debug
     return c
 
 
@@ -257,6 +260,19 @@ def mok_schedule_noalloc(topk_idx, E, stream=None):
     _check(_lib.mok_schedule_noalloc(_p(topk_idx), T, E, k, _p(counts), _p(offsets), _p(perm), _p(inv),
                                      _stream(stream)))
     return counts, offsets, perm, inv
+
+
+DEBUG_COUNTERS = ["mma_wait_operands", "mma_wait_peer_operands", "mma_wait_accumulator", "mma_total", "k_blocks",
+                  "producer_wait_stage", "epilogue_wait_accumulator", "epilogue_total"]
+
+
+def mok_debug_counters(workspace, stream=None):
+    """{slot: {counter: cycles}} of the last forward call that ran with config.debug != 0."""
+    buf = (ctypes.c_ulonglong * 32)()
+    wp, _ = _aligned_ws(workspace)
+    _check(_lib.mok_debug_counters(wp, _stream(stream), buf))
+    names = {1: "gemm1", 2: "gemm2", 3: "shared"}
+    return {names[s]: {n: int(buf[s * 8 + i]) for i, n in enumerate(DEBUG_COUNTERS)} for s in names}
 
 
 def mok_read_status(workspace, stream=None):
