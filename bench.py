@@ -41,6 +41,7 @@ def parse():
     p.add_argument("--no-cpu-baseline", action="store_true")
     p.add_argument("--gather-mode", type=int, default=0, help="0 auto, 1 fused into the GEMM, 2 separate kernel")
     p.add_argument("--cta-group", type=int, default=0, help="0 default, 1 single CTAs, 2 CTA pairs")
+    p.add_argument("--host-chunks", type=int, default=0, help="token chunks of the host-buffer call (0 = auto)")
     return p.parse_args()
 
 
@@ -227,7 +228,7 @@ def main():
     # end to end through the host-buffer entry point: pinned host x -> device, layer, result -> pinned host
     xh = g["x"].cpu().pin_memory()
     oh = torch.empty_like(xh).pin_memory()
-    conf0 = mok._config()
+    conf0 = mok._config(gather_mode=args.gather_mode, cta_group=args.cta_group, host_chunks=args.host_chunks)
 
     def e2e_step():
         mok.mok_moe_forward_host(xh, oh, W_r, bias, g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], cfg.k, ws,

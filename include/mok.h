@@ -52,6 +52,8 @@ enum {
     MOK_IMPL_SIMT = 1     /* plain shared-memory FMA kernel; slow; the on-device cross-check of the above */
 };
 
+#define MOK_MAX_HOST_CHUNKS 8
+
 /* Optional tuning / debugging knobs.  Zero-initialise for defaults. */
 typedef struct mok_config {
     int32_t impl;         /* MOK_IMPL_* */
@@ -61,10 +63,11 @@ typedef struct mok_config {
     int32_t profile;      /* != 0: record CUDA events around every stage of this call (see mok_profile_begin) */
     int32_t gather_mode;  /* token gather of the routed gate/up GEMM: 0 = choose by shape, 1 = fused into the GEMM's
                              operand loads (no expert-sorted copy of x), 2 = separate gather kernel + TMA loads */
-    int32_t cta_group;    /* tcgen05 GEMMs: 0 = default (1), 1 = one CTA per 128-row tile, 2 = CTA pairs sharing a
+    int32_t cta_group;    /* tcgen05 GEMMs: 0 = choose by shape, 1 = one CTA per 128-row tile, 2 = CTA pairs sharing a
                              256-row tile (cta_group::2; halves the weight traffic into each SM) */
     int32_t debug;        /* != 0: the tcgen05 GEMMs accumulate wait-time counters (see mok_debug_counters) */
-    int32_t reserved[1];
+    int32_t host_chunks;  /* mok_moe_forward_host: token chunks whose copies overlap compute (0 = choose by T,
+                             at most MOK_MAX_HOST_CHUNKS) */
 } mok_config;
 
 /*
@@ -120,7 +123,11 @@ int mok_moe_forward_ex(const mok_args* args);
 /*
  * Same layer with the activations in HOST memory: x_host (bf16 [T,H]) is copied to the device, the layer
  * runs, and out_host (bf16 [T,H]) is copied back; the call returns after the result has arrived (it
- * synchronises `stream`).  Pinned host buffers make the copies asynchronous DMA.  Weights, bias and
+ * synchronises `stream`).  Pinned host buffers make the copies asynchronous DMA.  Because each token's output
+ * depends only on its own row of x, the batch is cut into token chunks (config.host_chunks) and the upload of the
+ * next chunk and the download of the previous one run on two library-owned copy streams while a chunk computes;
+ * the result bits do not depend on the number of chunks.  Stage outputs force a single chunk.  The first call on a
+ * device creates the copy streams and events.  Weights, bias and
  * workspace stay DEVICE pointers as in mok_args; args->x and args->out are ignored.  The workspace must
  * have mok_workspace_bytes(...) + 2 * T*H*2 bytes (the staging copies of x and out live at its end).
  */

@@ -11,8 +11,8 @@
 // CTAS = 2: two CTAs of a cluster compute one 256 x 256 tile with cta_group::2 MMAs issued by the even CTA: each CTA
 //           stages its own 128 rows of A and HALF of the B tile (128 of the 256 weight rows), so a k-block moves
 //           32 KB instead of 48 KB from L2 into each SM and the ring holds 6 stages.  The odd CTA's TMA loads complete
-//           on the even CTA's mbarrier (its gathered rows are announced by its warp 1); tcgen05.commit multicasts "stage free" / "accumulator ready" to
-//           both CTAs; each CTA drains its own 128 accumulator rows.  No TMA multicast is used.
+//           on the even CTA's mbarrier (its gathered rows are announced by its warp 1); tcgen05.commit multicasts
+//           "stage free" / "accumulator ready" to both CTAs; each CTA drains its own 128 accumulator rows.  No TMA multicast is used.
 // Tiles are handed out statically (tile L -> CTA or pair L mod grid) in the order expert, M group, N tile, M tile, so
 // that CTAs running side by side share the same weight tile through L2 while an expert's activations stay L2
 // resident.  The tile tables come from the on-device schedule; nothing is read back.  Every output element is
@@ -29,6 +29,8 @@
 //                warp instruction reads four whole segments), and the copies' completion arrives on the stage's
 //                mbarrier; the expert-sorted copy of x never exists.  (TMA tile::gather4 computes the same thing
 //                but measured 2x slower here: 32 instructions of 512 bytes per k-block outrun the TMA issue rate.)
+// Tried and dropped: cp.async.bulk.prefetch.tensor of the weight boxes 8-12 k-blocks ahead (by every CTA, or only by
+// the CTA holding a group's first M tile) made the operand waits longer, not shorter (+13 % kernel time).
 // All mbarrier waits are bounded: on a timeout the CTA records MOK_ERR_TIMEOUT and leaves cleanly.
 #include "mok_internal.cuh"
 

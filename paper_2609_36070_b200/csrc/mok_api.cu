@@ -92,7 +92,8 @@ static int validate(const mok_args* a, WsLayout* L, size_t extra_ws) {
     if (a->config && (a->config->impl < 0 || a->config->impl > 1 || a->config->grid < 0 ||
                       a->config->router_impl < 0 || a->config->router_impl > 2 ||
                       a->config->gather_mode < 0 || a->config->gather_mode > 2 ||
-                      a->config->cta_group < 0 || a->config->cta_group > 2))
+                      a->config->cta_group < 0 || a->config->cta_group > 2 ||
+                      a->config->host_chunks < 0 || a->config->host_chunks > MOK_MAX_HOST_CHUNKS))
         return MOK_ERR_SHAPE;
     return MOK_OK;
 }
@@ -114,9 +115,14 @@ static bool fused_gather(const mok_config* cfg, int I) {
 }
 
 // Rows of one tile of the padded row space: 256 when the GEMMs run on CTA pairs (cta_group::2), else 128.
-static int tile_rows(const mok_config* cfg) {
+// Measured on B200: pairs are 5-19 % faster per k-block for GEMMs whose A operand comes through TMA, but slower for
+// the fused-gather GEMM (its odd CTA has to announce its gathered rows in software) and they double the padding of
+// every expert segment.  So by default pairs are used exactly when the gather is a separate kernel.
+static int tile_rows(const mok_config* cfg, int I) {
     if (use_simt(cfg)) return TILE_M;
-    return (cfg && cfg->cta_group == 2) ? 2 * TILE_M : TILE_M;   // pairs are correct but not yet faster: off by default
+    if (cfg && cfg->cta_group == 2) return 2 * TILE_M;
+    if (cfg && cfg->cta_group == 1) return TILE_M;
+    return fused_gather(cfg, I) ? TILE_M : 2 * TILE_M;
 }
 
 static int run_gemm(const GemmArgs& g, bool swiglu, const mok_config* cfg, cudaStream_t s) {
@@ -134,7 +140,7 @@ static int route_stage(const mok_args* a, const WsLayout& L, char* ws, const __n
     else
         e = launch_router_tc(x, a->W_router, a->router_bias, a->T, a->H, a->E, a->k, L, ws,
                              reinterpret_cast<WsHeader*>(ws + L.header), a->config ? a->config->grid : 0,
-                             tile_rows(a->config), idx, w, s);
+                             tile_rows(a->config, a->I > 0 ? a->I : 8), idx, w, s);
     if (e != cudaSuccess) return cuda_fail(e);
     if (a->topk_idx) {
         e = cudaMemcpyAsync(a->topk_idx, idx, sizeof(int32_t) * (size_t)L.R, cudaMemcpyDeviceToDevice, s);
@@ -160,7 +166,7 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
     int rc = route_stage(a, L, ws, x, s);
     if (rc) return rc;
     MOK_MARK(MOK_STAGE_ROUTER + 1);
-    const int tile_m = tile_rows(a->config);
+    const int tile_m = tile_rows(a->config, a->I);
     e = launch_schedule(reinterpret_cast<const int32_t*>(ws + L.idx), a->T, a->E, a->k, tile_m, L, ws,
                         a->counts, a->offsets, a->perm, a->inv_perm, s);
     if (e != cudaSuccess) return cuda_fail(e);
@@ -256,6 +262,38 @@ int mok_moe_forward_ex(const mok_args* a) {
     return forward_device(a, L, reinterpret_cast<const __nv_bfloat16*>(a->x), reinterpret_cast<__nv_bfloat16*>(a->out));
 }
 
+// Copy streams and events of mok_moe_forward_host, created once per device.
+struct HostPipe {
+    cudaStream_t s_in = nullptr, s_out = nullptr;
+    cudaEvent_t start = nullptr, out_done = nullptr, in_done[MOK_MAX_HOST_CHUNKS] = {}, fwd_done[MOK_MAX_HOST_CHUNKS] = {};
+    bool ready = false;
+};
+static HostPipe g_pipe[64];
+
+static int host_pipe(HostPipe** out) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (dev < 0 || dev >= 64) return MOK_ERR_UNSUPPORTED;
+    HostPipe& p = g_pipe[dev];
+    if (!p.ready) {
+        if ((e = cudaStreamCreateWithFlags(&p.s_in, cudaStreamNonBlocking)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaStreamCreateWithFlags(&p.s_out, cudaStreamNonBlocking)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaEventCreateWithFlags(&p.start, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaEventCreateWithFlags(&p.out_done, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
+        for (int c = 0; c < MOK_MAX_HOST_CHUNKS; ++c) {
+            if ((e = cudaEventCreateWithFlags(&p.in_done[c], cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
+            if ((e = cudaEventCreateWithFlags(&p.fwd_done[c], cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
+        }
+        p.ready = true;
+    }
+    *out = &p;
+    return MOK_OK;
+}
+
+// Every token's output depends only on its own row of x, so the batch can be cut into token chunks: the upload of
+// chunk c+1 and the download of chunk c-1 run on two copy streams while chunk c computes.  The bits of the result
+// do not depend on the number of chunks.
 int mok_moe_forward_host(const mok_args* a, const void* x_host, void* out_host) {
     WsLayout L;
     if (!a) return MOK_ERR_NULL;
@@ -264,16 +302,50 @@ int mok_moe_forward_host(const mok_args* a, const void* x_host, void* out_host) 
     int rc = validate(a, &L, 2 * act_al);
     if (rc || a->T == 0) return rc;
     if (!x_host || !out_host) return MOK_ERR_NULL;
+    int chunks = a->config ? a->config->host_chunks : 0;
+    if (chunks < 0 || chunks > MOK_MAX_HOST_CHUNKS) return MOK_ERR_SHAPE;
+    const bool stages = a->topk_idx || a->topk_w || a->counts || a->offsets || a->perm || a->inv_perm;
+    if (chunks == 0) chunks = a->T >= 8192 ? 4 : (a->T >= 2048 ? 2 : 1);
+    if (stages) chunks = 1;                    // stage outputs describe one schedule over the whole batch
+    int rows_per_chunk = ((a->T + chunks - 1) / chunks + 2 * TILE_M - 1) / (2 * TILE_M) * (2 * TILE_M);
+    chunks = (a->T + rows_per_chunk - 1) / rows_per_chunk;
+    HostPipe* p = nullptr;
+    if ((rc = host_pipe(&p))) return rc;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(a->stream);
     char* ws = reinterpret_cast<char*>(a->workspace);
     __nv_bfloat16* xd = reinterpret_cast<__nv_bfloat16*>(ws + L.total);
     __nv_bfloat16* od = reinterpret_cast<__nv_bfloat16*>(ws + L.total + act_al);
-    cudaError_t e = cudaMemcpyAsync(xd, x_host, act, cudaMemcpyHostToDevice, s);
-    if (e != cudaSuccess) return cuda_fail(e);
-    rc = forward_device(a, L, xd, od);
-    if (rc) return rc;
-    e = cudaMemcpyAsync(out_host, od, act, cudaMemcpyDeviceToHost, s);
-    if (e != cudaSuccess) return cuda_fail(e);
+    const char* xh = reinterpret_cast<const char*>(x_host);
+    char* oh = reinterpret_cast<char*>(out_host);
+    cudaError_t e;
+    // the copy streams start after whatever already sits in the caller's stream (it may still use the staging area)
+    if ((e = cudaEventRecord(p->start, s)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaStreamWaitEvent(p->s_in, p->start, 0)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaStreamWaitEvent(p->s_out, p->start, 0)) != cudaSuccess) return cuda_fail(e);
+    for (int c = 0; c < chunks; ++c) {
+        const int t0 = c * rows_per_chunk, tc = (a->T - t0 < rows_per_chunk) ? a->T - t0 : rows_per_chunk;
+        const size_t off = 2 * (size_t)t0 * a->H, bytes = 2 * (size_t)tc * a->H;
+        if ((e = cudaMemcpyAsync(reinterpret_cast<char*>(xd) + off, xh + off, bytes, cudaMemcpyHostToDevice, p->s_in)) != cudaSuccess)
+            return cuda_fail(e);
+        if ((e = cudaEventRecord(p->in_done[c], p->s_in)) != cudaSuccess) return cuda_fail(e);
+    }
+    for (int c = 0; c < chunks; ++c) {
+        const int t0 = c * rows_per_chunk, tc = (a->T - t0 < rows_per_chunk) ? a->T - t0 : rows_per_chunk;
+        const size_t off = 2 * (size_t)t0 * a->H, bytes = 2 * (size_t)tc * a->H;
+        mok_args ac = *a;
+        ac.T = tc;
+        WsLayout Lc;
+        if (!ws_layout(tc, a->H, a->I, a->I_shared, a->E, a->k, &Lc)) return MOK_ERR_SHAPE;
+        if ((e = cudaStreamWaitEvent(s, p->in_done[c], 0)) != cudaSuccess) return cuda_fail(e);
+        rc = forward_device(&ac, Lc, xd + (size_t)t0 * a->H, od + (size_t)t0 * a->H);
+        if (rc) return rc;
+        if ((e = cudaEventRecord(p->fwd_done[c], s)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaStreamWaitEvent(p->s_out, p->fwd_done[c], 0)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaMemcpyAsync(oh + off, reinterpret_cast<char*>(od) + off, bytes, cudaMemcpyDeviceToHost, p->s_out)) != cudaSuccess)
+            return cuda_fail(e);
+    }
+    if ((e = cudaEventRecord(p->out_done, p->s_out)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaStreamWaitEvent(s, p->out_done, 0)) != cudaSuccess) return cuda_fail(e);
     e = cudaStreamSynchronize(s);
     return e == cudaSuccess ? MOK_OK : cuda_fail(e);
 }

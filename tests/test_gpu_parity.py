@@ -99,6 +99,22 @@ def test_host_buffer_entry_point():
     assert torch.equal(oh.view(torch.int16), ref.cpu().view(torch.int16))
 
 
+def test_host_buffer_entry_point_chunked_copies_give_the_same_bits():
+    """Token chunks (upload / compute / download overlapped) must not change a single bit of the result."""
+    m = mok()
+    cfg = MoEConfig("chunky", T=1500, H=256, E=16, k=4, I=256, I_s=128, bias="normal", seed=31)
+    d = inputs.make_inputs(cfg)
+    g = pu.upload(d)
+    ref = pu.run_gpu(cfg, g, stages=False).cpu()
+    ws = m.alloc_workspace(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k, host_staging=True)
+    xh = g["x"].cpu().pin_memory()
+    for chunks in (1, 2, 5):
+        oh = torch.zeros_like(xh).pin_memory()
+        m.mok_moe_forward_host(xh, oh, g["W_r"], g["bias"], g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], cfg.k,
+                               ws, config=m._config(host_chunks=chunks))
+        assert torch.equal(oh.view(torch.int16), ref.view(torch.int16)), chunks
+
+
 def test_stage_entry_points():
     m = mok()
     cfg = SMALL[-1]
