@@ -173,10 +173,10 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
 
     # every rank: same weights, its own batch (seed offset by rank)
+    from paper_2609_36070_b200 import sharding
     d = inputs.make_inputs(cfg)
     if rank > 0:
-        from dataclasses import replace
-        d["x"] = inputs.make_x(replace(cfg, seed=cfg.seed + 1000 * rank))
+        d["x"] = sharding.rank_tokens(cfg, rank)
     g = {k: (None if d[k] is None else mok.to_device_bf16(d[k], dev)) for k in ("x", "W_gate_up", "W_down", "W_sgu", "W_sd")}
     W_r = torch.from_numpy(d["W_r"]).to(dev)
     bias = None if d["bias"] is None else torch.from_numpy(d["bias"]).to(dev)
@@ -216,12 +216,9 @@ def main():
     status = mok.mok_read_status(ws)
     assert status == 0, mok.mok_status_string(status)
 
-    if dist is not None:
-        t = torch.tensor([total_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = sharding.max_over_ranks(total_ms, dist, dev)
     ms_per_step = total_ms / args.steps
-    value = world * cfg.T / (ms_per_step * 1e-3)
+    value = sharding.aggregate_tokens_per_s(cfg.T, world, ms_per_step)
     flops = cfg.ffn_flops()
     tflops = world * flops / (ms_per_step * 1e-3) / 1e12
 
@@ -244,10 +241,7 @@ def main():
     ev1.record()
     barrier()
     e2e_ms = ev0.elapsed_time(ev1) / e2e_steps
-    if dist is not None:
-        t = torch.tensor([e2e_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = sharding.max_over_ranks(e2e_ms, dist, dev)
     act_bytes = 2 * cfg.T * cfg.H
 
     if rank != 0:
