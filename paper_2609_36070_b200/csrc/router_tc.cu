@@ -34,26 +34,74 @@ router_split_kernel(const float* __restrict__ Wr, int E, int H, int ldl, __nv_bf
     }
 }
 
-// Exact (fp32 FMA) logit of one (token, expert) pair computed by a whole warp: lanes stride over h in 16-byte
-// pieces, then a shuffle tree.  Error ~1e-7 relative, far below the near-tie threshold.
-__device__ __forceinline__ float warp_exact_logit(const __nv_bfloat16* __restrict__ xrow, const float* __restrict__ wrow,
-                                                  int H, int lane) {
-    float acc = 0.f;
+// Exact (fp32 FMA) logits of one token against up to four experts at once, computed by a whole warp: lanes stride
+// over h in 16-byte pieces of x (read once for the four experts), then a shuffle tree per expert.  Four independent
+// weight streams keep enough loads in flight to hide the L2 latency.  Error ~1e-7 relative, far below the near-tie
+// threshold.
+__device__ __forceinline__ void warp_exact_logits4(const __nv_bfloat16* __restrict__ xrow, const float* __restrict__ Wr,
+                                                   const int (&e)[4], int n, int H, int lane, float (&out)[4]) {
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    const float* wrow[4];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) wrow[c] = Wr + (size_t)e[c < n ? c : 0] * H;
     for (int h = lane * 8; h < H; h += 256) {
         const uint4 raw = *reinterpret_cast<const uint4*>(xrow + h);
         const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&raw);
-        const float4 w0 = *reinterpret_cast<const float4*>(wrow + h);
-        const float4 w1 = *reinterpret_cast<const float4*>(wrow + h + 4);
         const float2 x0 = __bfloat1622float2(p[0]), x1 = __bfloat1622float2(p[1]);
         const float2 x2 = __bfloat1622float2(p[2]), x3 = __bfloat1622float2(p[3]);
-        acc = fmaf(x0.x, w0.x, acc); acc = fmaf(x0.y, w0.y, acc);
-        acc = fmaf(x1.x, w0.z, acc); acc = fmaf(x1.y, w0.w, acc);
-        acc = fmaf(x2.x, w1.x, acc); acc = fmaf(x2.y, w1.y, acc);
-        acc = fmaf(x3.x, w1.z, acc); acc = fmaf(x3.y, w1.w, acc);
+        float4 w0[4], w1[4];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            w0[c] = *reinterpret_cast<const float4*>(wrow[c] + h);
+            w1[c] = *reinterpret_cast<const float4*>(wrow[c] + h + 4);
+        }
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            float a = acc[c];
+            a = fmaf(x0.x, w0[c].x, a); a = fmaf(x0.y, w0[c].y, a);
+            a = fmaf(x1.x, w0[c].z, a); a = fmaf(x1.y, w0[c].w, a);
+            a = fmaf(x2.x, w1[c].x, a); a = fmaf(x2.y, w1[c].y, a);
+            a = fmaf(x3.x, w1[c].z, a); a = fmaf(x3.y, w1[c].w, a);
+            acc[c] = a;
+        }
     }
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
-    return acc;
+    for (int c = 0; c < 4; ++c) {
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) acc[c] += __shfl_xor_sync(0xffffffffu, acc[c], off);
+        out[c] = acc[c];
+    }
+}
+
+// Monotone map from float to unsigned: a > b  <=>  key(a) > key(b) (finite inputs).
+__device__ __forceinline__ unsigned float_key(float v) {
+    const unsigned u = __float_as_uint(v);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+// Selection with the logits in registers: lane l holds experts l, l+32, ... (VPL per lane).  One round = every lane's
+// best remaining value, a hardware warp max of the keys (redux.sync), and a warp min of the expert ids that attain it
+// (ties go to the lowest id): two reductions instead of a ten-shuffle tree.
+template <int VPL>
+__device__ __forceinline__ void reg_select(float (&v)[VPL], int lane, int s_begin, int s_end, float& slot_v, int& slot_e) {
+    for (int s = s_begin; s < s_end; ++s) {
+        float bv = v[0];
+        int bj = 0;
+#pragma unroll
+        for (int j = 1; j < VPL; ++j)
+            if (v[j] > bv) { bv = v[j]; bj = j; }             // strict '>' keeps the lowest id on ties inside a lane
+        const unsigned key = float_key(bv);
+        const unsigned kmax = __reduce_max_sync(0xffffffffu, key);
+        const int e_mine = (key == kmax) ? lane + 32 * bj : 0x7fffffff;
+        const int e_win = __reduce_min_sync(0xffffffffu, e_mine);
+        if (e_mine == e_win) {
+#pragma unroll
+            for (int j = 0; j < VPL; ++j)
+                if (j == bj) v[j] = -FLT_MAX;                    // taken
+        }
+        const float v_win = __shfl_sync(0xffffffffu, bv, e_win & 31);
+        if (lane == s) { slot_v = v_win; slot_e = e_win; }
+    }
 }
 
 // The tensor cores add the 16 products of one MMA step to the fp32 accumulator with truncation, so the logit
@@ -62,46 +110,61 @@ __device__ __forceinline__ float warp_exact_logit(const __nv_bfloat16* __restric
 // the error.  So: tokens whose top-(k+1) tensor-core logits contain an adjacent pair closer than
 //     guard = H * 2^-26 * (1 + max|logit|)      (four times the modelled bound (H/16) * 2^-24 * |acc|)
 // get the logits of their top-(k+4) candidates recomputed with plain fp32 FMAs and are selected again.
+template <int VPL>
 __global__ void __launch_bounds__(256)
 router_topk_kernel(const float* __restrict__ part, const float* __restrict__ bias,
                    const __nv_bfloat16* __restrict__ x, const float* __restrict__ Wr,
                    int T, int H, int E, int k, int ldl, int32_t* __restrict__ idx, float* __restrict__ w) {
-    extern __shared__ float tsm[];                      // [8][E]
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    float* lg = tsm + warp * E;
     const int n_check = (k + 1 < E) ? k + 1 : E;        // slots compared pairwise
     int n_cand = (k + 4 < E) ? k + 4 : E;               // candidates recomputed when a pair is too close
     if (n_cand > 32) n_cand = 32;
     const float guard_scale = (float)H * 1.4901161e-8f; // H * 2^-26
     for (int t = blockIdx.x * 8 + warp; t < T; t += gridDim.x * 8) {
         const float* row = part + (size_t)t * ldl;
-        for (int e = lane; e < E; e += 32) {
-            float v = (row[2 * E + e] + row[E + e]) + row[e];      // smallest terms first
-            if (bias) v += bias[e];
-            lg[e] = v;
+        float orig[VPL], v[VPL];
+#pragma unroll
+        for (int j = 0; j < VPL; ++j) {
+            const int e = lane + 32 * j;
+            float val = -FLT_MAX;
+            if (e < E) {
+                val = (row[2 * E + e] + row[E + e]) + row[e];      // smallest terms first
+                if (bias) val += bias[e];
+            }
+            orig[j] = val;
+            v[j] = val;
         }
-        __syncwarp();
         TopkState st = {0u, 0.f, 0};
-        warp_select(lg, E, 0, n_check, lane, st);
+        reg_select<VPL>(v, lane, 0, n_check, st.v, st.e);
         const float next_v = __shfl_down_sync(0xffffffffu, st.v, 1);
         float amax = (lane < n_check) ? fabsf(st.v) : 0.f;
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, off));
         const bool close = (lane + 1 < n_check) && (st.v - next_v < guard_scale * (1.f + amax));
         if (__any_sync(0xffffffffu, close)) {
-            warp_select(lg, E, n_check, n_cand, lane, st);
-            for (int c = 0; c < n_cand; ++c) {
-                const int e = __shfl_sync(0xffffffffu, st.e, c);
-                float v = warp_exact_logit(x + (size_t)t * H, Wr + (size_t)e * H, H, lane);
-                if (bias) v += bias[e];
-                if (lane == 0) lg[e] = v;
+            reg_select<VPL>(v, lane, n_check, n_cand, st.v, st.e);
+            for (int c0 = 0; c0 < n_cand; c0 += 4) {
+                int e[4];
+                float ex[4];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) e[c] = __shfl_sync(0xffffffffu, st.e, (c0 + c < n_cand) ? c0 + c : c0);
+                const int n = (n_cand - c0 < 4) ? n_cand - c0 : 4;
+                warp_exact_logits4(x + (size_t)t * H, Wr, e, n, H, lane, ex);
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    if (c < n && (e[c] & 31) == lane) {
+                        const float val = ex[c] + (bias ? bias[e[c]] : 0.f);
+#pragma unroll
+                        for (int j = 0; j < VPL; ++j)
+                            if (j == (e[c] >> 5)) orig[j] = val;
+                    }
+                }
             }
-            __syncwarp();
-            st.taken = 0u;
-            warp_select(lg, E, 0, k, lane, st);
+#pragma unroll
+            for (int j = 0; j < VPL; ++j) v[j] = orig[j];
+            reg_select<VPL>(v, lane, 0, k, st.v, st.e);
         }
         warp_write_topk(st, k, lane, idx + (size_t)t * k, w + (size_t)t * k);
-        __syncwarp();
     }
 }
 
@@ -131,7 +194,12 @@ cudaError_t launch_router_tc(const __nv_bfloat16* x, const float* Wr, const floa
     if (e != cudaSuccess) return e;
     int tblocks = (T + 7) / 8;
     if (tblocks > 148 * 16) tblocks = 148 * 16;
-    router_topk_kernel<<<tblocks, 256, sizeof(float) * 8 * E, s>>>(part, bias, x, Wr, T, H, E, k, ldl, idx, w);
+    const int vpl = (E + 31) / 32;
+    if (vpl <= 1) router_topk_kernel<1><<<tblocks, 256, 0, s>>>(part, bias, x, Wr, T, H, E, k, ldl, idx, w);
+    else if (vpl <= 2) router_topk_kernel<2><<<tblocks, 256, 0, s>>>(part, bias, x, Wr, T, H, E, k, ldl, idx, w);
+    else if (vpl <= 4) router_topk_kernel<4><<<tblocks, 256, 0, s>>>(part, bias, x, Wr, T, H, E, k, ldl, idx, w);
+    else if (vpl <= 8) router_topk_kernel<8><<<tblocks, 256, 0, s>>>(part, bias, x, Wr, T, H, E, k, ldl, idx, w);
+    else router_topk_kernel<16><<<tblocks, 256, 0, s>>>(part, bias, x, Wr, T, H, E, k, ldl, idx, w);
     return cudaGetLastError();
 }
 
