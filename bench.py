@@ -41,6 +41,7 @@ def parse():
     p.add_argument("--no-cpu-baseline", action="store_true")
     p.add_argument("--gather-mode", type=int, default=0, help="0 auto, 1 fused into the GEMM, 2 separate kernel")
     p.add_argument("--cta-group", type=int, default=0, help="0 default, 1 single CTAs, 2 CTA pairs")
+    p.add_argument("--gemm", type=int, default=0, help="0 tcgen05 (tokens on M), 2 tcgen05 (tokens on N), 1 SIMT")
     p.add_argument("--host-chunks", type=int, default=0, help="token chunks of the host-buffer call (0 = auto)")
     return p.parse_args()
 
@@ -182,7 +183,7 @@ def main():
     bias = None if d["bias"] is None else torch.from_numpy(d["bias"]).to(dev)
     ws = mok.alloc_workspace(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k, device=dev, host_staging=True)
     out = torch.empty_like(g["x"])
-    conf = mok._config(profile=1, gather_mode=args.gather_mode, cta_group=args.cta_group)
+    conf = mok._config(impl=args.gemm, profile=1, gather_mode=args.gather_mode, cta_group=args.cta_group)
 
     def step():
         mok.mok_moe_forward_ex(g["x"], W_r, bias, g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], cfg.k, ws,
@@ -225,7 +226,7 @@ def main():
     # end to end through the host-buffer entry point: pinned host x -> device, layer, result -> pinned host
     xh = g["x"].cpu().pin_memory()
     oh = torch.empty_like(xh).pin_memory()
-    conf0 = mok._config(gather_mode=args.gather_mode, cta_group=args.cta_group, host_chunks=args.host_chunks)
+    conf0 = mok._config(impl=args.gemm, gather_mode=args.gather_mode, cta_group=args.cta_group, host_chunks=args.host_chunks)
 
     def e2e_step():
         mok.mok_moe_forward_host(xh, oh, W_r, bias, g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], cfg.k, ws,

@@ -49,7 +49,8 @@ typedef enum mok_status {
 /* Which grouped-GEMM kernel runs the expert FFNs. */
 enum {
     MOK_IMPL_TCGEN05 = 0, /* warp-specialised persistent kernel: TMA -> smem ring -> tcgen05.mma -> TMEM (default) */
-    MOK_IMPL_SIMT = 1     /* plain shared-memory FMA kernel; slow; the on-device cross-check of the above */
+    MOK_IMPL_SIMT = 1,    /* plain shared-memory FMA kernel; slow; the on-device cross-check of the above */
+    MOK_IMPL_TCGEN05_TN = 2 /* tcgen05 kernel with the tokens on the MMA's N side (expert padding 16 rows, not 128) */
 };
 
 #define MOK_MAX_HOST_CHUNKS 8

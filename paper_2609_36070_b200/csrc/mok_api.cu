@@ -89,7 +89,7 @@ static int validate(const mok_args* a, WsLayout* L, size_t extra_ws) {
         return MOK_ERR_ALIGN;
     if (!a->workspace || (reinterpret_cast<uintptr_t>(a->workspace) & 255u) || a->workspace_bytes < L->total + extra_ws)
         return MOK_ERR_WORKSPACE;
-    if (a->config && (a->config->impl < 0 || a->config->impl > 1 || a->config->grid < 0 ||
+    if (a->config && (a->config->impl < 0 || a->config->impl > 2 || a->config->grid < 0 ||
                       a->config->router_impl < 0 || a->config->router_impl > 2 ||
                       a->config->gather_mode < 0 || a->config->gather_mode > 2 ||
                       a->config->cta_group < 0 || a->config->cta_group > 2 ||
@@ -99,6 +99,7 @@ static int validate(const mok_args* a, WsLayout* L, size_t extra_ws) {
 }
 
 static bool use_simt(const mok_config* cfg) { return cfg && cfg->impl == MOK_IMPL_SIMT; }
+static bool use_tn(const mok_config* cfg) { return cfg && cfg->impl == MOK_IMPL_TCGEN05_TN; }
 static bool use_simt_router(const mok_config* cfg, int k) {
     if (k > 28) return true;   // the tensor-core router keeps k + 4 candidates in one warp's 32 lanes
     return cfg && (cfg->router_impl == 1 || (cfg->router_impl == 0 && cfg->impl == MOK_IMPL_SIMT));
@@ -109,6 +110,7 @@ static bool use_simt_router(const mok_config* cfg, int k) {
 // plain TMA tile loads.  Measured on B200: fused wins at 6, 16 and 23 N tiles (ceil(I / 128)), loses at 112.
 static bool fused_gather(const mok_config* cfg, int I) {
     if (use_simt(cfg)) return false;
+    if (use_tn(cfg)) return true;
     if (cfg && cfg->gather_mode == 1) return true;
     if (cfg && cfg->gather_mode == 2) return false;
     return (I + 127) / 128 <= 32;
@@ -119,15 +121,16 @@ static bool fused_gather(const mok_config* cfg, int I) {
 // the fused-gather GEMM (its odd CTA has to announce its gathered rows in software) and they double the padding of
 // every expert segment.  So by default pairs are used exactly when the gather is a separate kernel.
 static int tile_rows(const mok_config* cfg, int I) {
-    if (use_simt(cfg)) return TILE_M;
+    if (use_simt(cfg) || use_tn(cfg)) return TILE_M;
     if (cfg && cfg->cta_group == 2) return 2 * TILE_M;
     if (cfg && cfg->cta_group == 1) return TILE_M;
     return fused_gather(cfg, I) ? TILE_M : 2 * TILE_M;
 }
 
 static int run_gemm(const GemmArgs& g, bool swiglu, const mok_config* cfg, cudaStream_t s) {
+    const int epi = swiglu ? EPI_SWIGLU : EPI_BF16, grid = cfg ? cfg->grid : 0;
     cudaError_t e = use_simt(cfg) ? launch_gemm_simt(g, swiglu, s)
-                                  : launch_gemm_tc(g, swiglu ? EPI_SWIGLU : EPI_BF16, cfg ? cfg->grid : 0, s);
+                    : use_tn(cfg) ? launch_gemm_tn(g, epi, grid, s) : launch_gemm_tc(g, epi, grid, s);
     return e == cudaSuccess ? MOK_OK : cuda_fail(e);
 }
 
@@ -140,7 +143,7 @@ static int route_stage(const mok_args* a, const WsLayout& L, char* ws, const __n
     else
         e = launch_router_tc(x, a->W_router, a->router_bias, a->T, a->H, a->E, a->k, L, ws,
                              reinterpret_cast<WsHeader*>(ws + L.header), a->config ? a->config->grid : 0,
-                             tile_rows(a->config, a->I > 0 ? a->I : 8), idx, w, s);
+                             tile_rows(a->config, a->I > 0 ? a->I : 8), use_tn(a->config), idx, w, s);
     if (e != cudaSuccess) return cuda_fail(e);
     if (a->topk_idx) {
         e = cudaMemcpyAsync(a->topk_idx, idx, sizeof(int32_t) * (size_t)L.R, cudaMemcpyDeviceToDevice, s);
@@ -167,7 +170,8 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
     if (rc) return rc;
     MOK_MARK(MOK_STAGE_ROUTER + 1);
     const int tile_m = tile_rows(a->config, a->I);
-    e = launch_schedule(reinterpret_cast<const int32_t*>(ws + L.idx), a->T, a->E, a->k, tile_m, L, ws,
+    const int pad_m = use_tn(a->config) ? 16 : tile_m;   // tokens on the MMA's N side need 16-row granularity only
+    e = launch_schedule(reinterpret_cast<const int32_t*>(ws + L.idx), a->T, a->E, a->k, tile_m, pad_m, L, ws,
                         a->counts, a->offsets, a->perm, a->inv_perm, s);
     if (e != cudaSuccess) return cuda_fail(e);
     MOK_MARK(MOK_STAGE_SCHEDULE + 1);
@@ -186,6 +190,8 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
     g.mt_start = reinterpret_cast<const int32_t*>(ws + L.mt_start);
     g.max_mt = L.max_mt;
     g.tile_m = tile_m;
+    g.pad_offsets = reinterpret_cast<const int32_t*>(ws + L.pad_offsets);
+    g.counts = reinterpret_cast<const int32_t*>(ws + L.counts);
     const bool dbg = a->config && a->config->debug;
     g.dbg_slot = dbg ? 1 : -1;
     // routed experts: h = silu(Xg Wg^T) * (Xg Wu^T);  y = h Wd^T
@@ -203,7 +209,6 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
     g.K = a->H; g.N = a->I; g.ldc = a->I; g.E = a->E; g.rows_pad = L.Rpad; g.dense_rows = 0;
     if ((rc = run_gemm(g, true, a->config, s))) return rc;
     g.row_token = nullptr;
-    g.counts = nullptr;
     g.a_rows = L.Rpad;
     g.dbg_slot = dbg ? 2 : -1;
     MOK_MARK(MOK_STAGE_GEMM1 + 1);
@@ -410,7 +415,7 @@ int mok_schedule(const int32_t* topk_idx, int T, int E, int k, int32_t* counts, 
     char* ws = reinterpret_cast<char*>(workspace);
     cudaError_t e = cudaMemsetAsync(ws + L.header, 0, sizeof(WsHeader), s);
     if (e != cudaSuccess) return cuda_fail(e);
-    e = launch_schedule(topk_idx, T, E, k, TILE_M, L, ws, counts, offsets, perm, inv_perm, s);
+    e = launch_schedule(topk_idx, T, E, k, TILE_M, TILE_M, L, ws, counts, offsets, perm, inv_perm, s);
     return e == cudaSuccess ? MOK_OK : cuda_fail(e);
 }
 

@@ -54,7 +54,8 @@ struct GemmArgs {
     int32_t K, N, E;
     int32_t ldc;                 // elements between consecutive rows of C
     const int32_t* row_token;    // device [rows_pad] or NULL: padded row -> token (gather fused into the A loads)
-    const int32_t* counts;       // device [E] (only read when row_token is set)
+    const int32_t* counts;       // device [E]
+    const int32_t* pad_offsets;  // device [E+1]: first row of each expert in the padded row space
     int32_t rows_pad;            // allocated rows of C (multiple of 128)
     int32_t a_rows;              // allocated rows of A (reads beyond it are treated as zero)
     int32_t dense_rows;          // > 0: dense mode with this many valid rows
@@ -70,7 +71,7 @@ struct GemmArgs {
 // kernels' host launchers (each returns a cudaError_t from the launch)
 cudaError_t launch_router_simt(const __nv_bfloat16* x, const float* Wr, const float* bias, int T, int H, int E, int k,
                                int32_t* idx, float* w, cudaStream_t s);
-cudaError_t launch_schedule(const int32_t* idx, int T, int E, int k, int tile_m, const WsLayout& L, char* ws,
+cudaError_t launch_schedule(const int32_t* idx, int T, int E, int k, int tile_m, int pad_m, const WsLayout& L, char* ws,
                             int32_t* counts_out, int32_t* offsets_out, int32_t* perm_out, int32_t* inv_out,
                             cudaStream_t s);
 cudaError_t launch_gather(const __nv_bfloat16* x, int H, int k, int tile_m, const WsLayout& L, char* ws, cudaStream_t s);
@@ -79,8 +80,10 @@ cudaError_t launch_combine(const WsLayout& L, char* ws, int T, int H, int k, boo
 cudaError_t launch_gemm_simt(const GemmArgs& a, bool swiglu, cudaStream_t s);
 enum { EPI_BF16 = 0, EPI_SWIGLU = 1, EPI_F32 = 2 };
 cudaError_t launch_gemm_tc(const GemmArgs& a, int epi, int grid, cudaStream_t s);
+cudaError_t launch_gemm_tn(const GemmArgs& a, int epi, int grid, cudaStream_t s);   // tokens on the MMA's N side
 cudaError_t launch_router_tc(const __nv_bfloat16* x, const float* Wr, const float* bias, int T, int H, int E, int k,
-                             const WsLayout& L, char* ws, WsHeader* hdr, int grid, int tile_m, int32_t* idx, float* w,
+                             const WsLayout& L, char* ws, WsHeader* hdr, int grid, int tile_m, bool tn, int32_t* idx,
+                             float* w,
                              cudaStream_t s);
 
 inline __host__ __device__ size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }

@@ -55,6 +55,6 @@ extern "C" int mok_schedule_noalloc(const int32_t* topk_idx, int T, int E, int k
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     cudaError_t e = cudaMemsetAsync(ws + L.header, 0, sizeof(WsHeader), s);   // status / tile count start at zero
     if (e != cudaSuccess) return MOK_ERR_CUDA;
-    e = launch_schedule(topk_idx, T, E, k, TILE_M, L, ws, counts, offsets, perm, inv_perm, s);
+    e = launch_schedule(topk_idx, T, E, k, TILE_M, TILE_M, L, ws, counts, offsets, perm, inv_perm, s);
     return e == cudaSuccess ? MOK_OK : MOK_ERR_CUDA;
 }

@@ -169,8 +169,8 @@ router_topk_kernel(const float* __restrict__ part, const float* __restrict__ bia
 }
 
 cudaError_t launch_router_tc(const __nv_bfloat16* x, const float* Wr, const float* bias, int T, int H, int E, int k,
-                             const WsLayout& L, char* ws, WsHeader* hdr, int grid, int tile_m, int32_t* idx, float* w,
-                             cudaStream_t s) {
+                             const WsLayout& L, char* ws, WsHeader* hdr, int grid, int tile_m, bool tn, int32_t* idx,
+                             float* w, cudaStream_t s) {
     const int ldl = (3 * E + 7) / 8 * 8;
     __nv_bfloat16* split = reinterpret_cast<__nv_bfloat16*>(ws + L.wr_split);
     float* part = reinterpret_cast<float*>(ws + L.logits);
@@ -190,7 +190,7 @@ cudaError_t launch_router_tc(const __nv_bfloat16* x, const float* Wr, const floa
     g.tile_m = tile_m;
     g.dbg_slot = -1;
     g.header = hdr;
-    e = launch_gemm_tc(g, EPI_F32, grid, s);
+    e = tn ? launch_gemm_tn(g, EPI_F32, grid, s) : launch_gemm_tc(g, EPI_F32, grid, s);
     if (e != cudaSuccess) return e;
     int tblocks = (T + 7) / 8;
     if (tblocks > 148 * 16) tblocks = 148 * 16;

@@ -6,8 +6,9 @@
 // (Section 3.3), integer arithmetic only, hence bit-reproducible:
 //   1. sched_hist    per-block expert histograms of SCHED_CHUNK consecutive routes
 //   2. sched_scan    one block: per-expert prefix over blocks, counts, offsets, and the internal tile tables
-//                    (each expert's segment padded to a multiple of tile_m = 128 or 256 rows: pad_offsets,
-//                    mt_start, tile_expert, all in units of tile_m)
+//                    (each expert's segment is padded to a multiple of pad_m rows -> pad_offsets; it is cut into
+//                    tiles of tile_m rows -> mt_start, tile_expert.  pad_m = tile_m = 128 or 256 when tokens sit on the
+//                    MMA's M side, pad_m = 16 and tile_m = 128 when they sit on its N side)
 //   3. sched_scatter stable ranks inside each block (warp match + per-warp running counters) -> perm, inv, pos,
 //                    row_token (padded row -> source token: the {src_index} column of the paper's schedule table)
 // Exported offsets/perm are unpadded; the padding is internal to the GEMM row space.
@@ -36,11 +37,11 @@ sched_hist_kernel(const int32_t* __restrict__ a, int n, int E, int32_t* __restri
 // One block of MAX_E threads.  Thread e walks the blocks for expert e (exclusive prefix, in place), then the
 // block scans over experts.
 __global__ void __launch_bounds__(MAX_E)
-sched_scan_kernel(int32_t* __restrict__ blk_hist, int n_blk, int E, int max_mt, int tile_m,
+sched_scan_kernel(int32_t* __restrict__ blk_hist, int n_blk, int E, int max_mt, int tile_m, int pad_m,
                   int32_t* __restrict__ counts, int32_t* __restrict__ offsets, int32_t* __restrict__ pad_offsets,
                   int32_t* __restrict__ mt_start, int32_t* __restrict__ tile_expert, WsHeader* __restrict__ hdr,
                   int32_t* __restrict__ counts_out, int32_t* __restrict__ offsets_out) {
-    __shared__ int32_t s_cnt[MAX_E], s_off[MAX_E + 1], s_mt[MAX_E + 1];
+    __shared__ int32_t s_cnt[MAX_E], s_off[MAX_E + 1], s_mt[MAX_E + 1], s_pad[MAX_E + 1];
     const int e = threadIdx.x;
     int32_t total = 0;
     if (e < E) {
@@ -58,15 +59,18 @@ sched_scan_kernel(int32_t* __restrict__ blk_hist, int n_blk, int E, int max_mt, 
     }
     __syncthreads();
     if (e == 0) {   // E <= 512: a serial scan by one thread is a few hundred cycles
-        int32_t off = 0, mt = 0;
+        int32_t off = 0, mt = 0, pad = 0;
         for (int i = 0; i < E; ++i) {
             s_off[i] = off;
             s_mt[i] = mt;
+            s_pad[i] = pad;
             off += s_cnt[i];
             mt += (s_cnt[i] + tile_m - 1) / tile_m;
+            pad += (s_cnt[i] + pad_m - 1) / pad_m * pad_m;
         }
         s_off[E] = off;
         s_mt[E] = mt;
+        s_pad[E] = pad;
         hdr->n_mtiles = mt;
         if (mt * (tile_m / TILE_M) > max_mt) hdr->status = MOK_ERR_SCHEDULE;
     }
@@ -74,7 +78,7 @@ sched_scan_kernel(int32_t* __restrict__ blk_hist, int n_blk, int E, int max_mt, 
     if (e < E) {
         counts[e] = s_cnt[e];
         offsets[e] = s_off[e];
-        pad_offsets[e] = s_mt[e] * tile_m;
+        pad_offsets[e] = s_pad[e];
         mt_start[e] = s_mt[e];
         if (counts_out) counts_out[e] = s_cnt[e];
         if (offsets_out) offsets_out[e] = s_off[e];
@@ -82,7 +86,7 @@ sched_scan_kernel(int32_t* __restrict__ blk_hist, int n_blk, int E, int max_mt, 
     }
     if (e == 0) {
         offsets[E] = s_off[E];
-        pad_offsets[E] = s_mt[E] * tile_m;
+        pad_offsets[E] = s_pad[E];
         mt_start[E] = s_mt[E];
         if (offsets_out) offsets_out[E] = s_off[E];
     }
@@ -148,7 +152,7 @@ sched_scatter_kernel(const int32_t* __restrict__ a, int n, int E,
     }
 }
 
-cudaError_t launch_schedule(const int32_t* idx, int T, int E, int k, int tile_m, const WsLayout& L, char* ws,
+cudaError_t launch_schedule(const int32_t* idx, int T, int E, int k, int tile_m, int pad_m, const WsLayout& L, char* ws,
                             int32_t* counts_out, int32_t* offsets_out, int32_t* perm_out, int32_t* inv_out,
                             cudaStream_t s) {
     const int n = T * k;
@@ -160,7 +164,7 @@ cudaError_t launch_schedule(const int32_t* idx, int T, int E, int k, int tile_m,
     int32_t* tile_expert = reinterpret_cast<int32_t*>(ws + L.tile_expert);
     WsHeader* hdr = reinterpret_cast<WsHeader*>(ws + L.header);
     sched_hist_kernel<<<L.n_blk, SCHED_THREADS, 0, s>>>(idx, n, E, blk_hist);
-    sched_scan_kernel<<<1, MAX_E, 0, s>>>(blk_hist, L.n_blk, E, L.max_mt, tile_m, counts, offsets, pad_offsets, mt_start,
+    sched_scan_kernel<<<1, MAX_E, 0, s>>>(blk_hist, L.n_blk, E, L.max_mt, tile_m, pad_m, counts, offsets, pad_offsets, mt_start,
                                           tile_expert, hdr, counts_out, offsets_out);
     sched_scatter_kernel<<<L.n_blk, SCHED_THREADS, sizeof(int32_t) * SCHED_WARPS * E, s>>>(
         idx, n, E, blk_hist, offsets, pad_offsets,

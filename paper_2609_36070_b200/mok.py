@@ -17,7 +17,7 @@ _lib = ctypes.CDLL(_LIB_PATH)
 MOK_OK = 0
 MOK_ERR_NULL, MOK_ERR_SHAPE, MOK_ERR_ALIGN, MOK_ERR_WORKSPACE = -1, -2, -3, -4
 MOK_ERR_CUDA, MOK_ERR_TIMEOUT, MOK_ERR_SCHEDULE, MOK_ERR_UNSUPPORTED = -5, -6, -7, -8
-MOK_IMPL_TCGEN05, MOK_IMPL_SIMT = 0, 1
+MOK_IMPL_TCGEN05, MOK_IMPL_SIMT, MOK_IMPL_TCGEN05_TN = 0, 1, 2
 
 EXPORTS = ["mok_moe_forward", "mok_workspace_bytes", "mok_moe_forward_ex", "mok_moe_forward_host", "mok_route",
            "mok_schedule", "mok_read_status", "mok_launch_count", "mok_last_cuda_error", "mok_status_string",

@@ -30,13 +30,14 @@ SMALL = [
 
 
 @pytest.mark.parametrize("cfg", SMALL, ids=[c.name for c in SMALL])
-@pytest.mark.parametrize("impl", ["tcgen05_fused_gather", "tcgen05_separate_gather", "tcgen05_single_cta", "simt"])
+@pytest.mark.parametrize("impl", ["tcgen05_fused_gather", "tcgen05_separate_gather", "tcgen05_single_cta", "tcgen05_tokens_as_n", "simt"])
 def test_small_shapes_every_token(cfg, impl):
     m = mok()
     conf = {"simt": m._config(impl=m.MOK_IMPL_SIMT),
             "tcgen05_fused_gather": m._config(gather_mode=1),
             "tcgen05_separate_gather": m._config(gather_mode=2),
-            "tcgen05_single_cta": m._config(cta_group=1)}[impl]
+            "tcgen05_single_cta": m._config(cta_group=1),
+            "tcgen05_tokens_as_n": m._config(impl=m.MOK_IMPL_TCGEN05_TN)}[impl]
     out, st, rep = pu.full_parity(cfg, config=conf)
     print(cfg.name, impl, rep)
 
