@@ -312,8 +312,21 @@ int mok_moe_forward_host(const mok_args* a, const void* x_host, void* out_host) 
     const bool stages = a->topk_idx || a->topk_w || a->counts || a->offsets || a->perm || a->inv_perm;
     if (chunks == 0) chunks = a->T >= 8192 ? 4 : (a->T >= 2048 ? 2 : 1);
     if (stages) chunks = 1;                    // stage outputs describe one schedule over the whole batch
-    int rows_per_chunk = ((a->T + chunks - 1) / chunks + 2 * TILE_M - 1) / (2 * TILE_M) * (2 * TILE_M);
-    chunks = (a->T + rows_per_chunk - 1) / rows_per_chunk;
+    // Chunk boundaries: with three or more chunks the first and the last get half the weight of the inner ones, so
+    // that the upload nobody can hide (first chunk) and the download nobody can hide (last chunk) are short.
+    int bound[MOK_MAX_HOST_CHUNKS + 1];
+    {
+        const int units = (chunks >= 3) ? 2 * chunks - 2 : chunks;
+        int acc_units = 0, n = 0;
+        bound[0] = 0;
+        for (int c = 0; c < chunks; ++c) {
+            acc_units += (chunks >= 3 && c > 0 && c < chunks - 1) ? 2 : 1;
+            int end = (int)(((long long)a->T * acc_units / units + 2 * TILE_M - 1) / (2 * TILE_M) * (2 * TILE_M));
+            if (end > a->T || c == chunks - 1) end = a->T;
+            if (end > bound[n]) bound[++n] = end;
+        }
+        chunks = n;
+    }
     HostPipe* p = nullptr;
     if ((rc = host_pipe(&p))) return rc;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(a->stream);
@@ -328,14 +341,14 @@ int mok_moe_forward_host(const mok_args* a, const void* x_host, void* out_host) 
     if ((e = cudaStreamWaitEvent(p->s_in, p->start, 0)) != cudaSuccess) return cuda_fail(e);
     if ((e = cudaStreamWaitEvent(p->s_out, p->start, 0)) != cudaSuccess) return cuda_fail(e);
     for (int c = 0; c < chunks; ++c) {
-        const int t0 = c * rows_per_chunk, tc = (a->T - t0 < rows_per_chunk) ? a->T - t0 : rows_per_chunk;
+        const int t0 = bound[c], tc = bound[c + 1] - bound[c];
         const size_t off = 2 * (size_t)t0 * a->H, bytes = 2 * (size_t)tc * a->H;
         if ((e = cudaMemcpyAsync(reinterpret_cast<char*>(xd) + off, xh + off, bytes, cudaMemcpyHostToDevice, p->s_in)) != cudaSuccess)
             return cuda_fail(e);
         if ((e = cudaEventRecord(p->in_done[c], p->s_in)) != cudaSuccess) return cuda_fail(e);
     }
     for (int c = 0; c < chunks; ++c) {
-        const int t0 = c * rows_per_chunk, tc = (a->T - t0 < rows_per_chunk) ? a->T - t0 : rows_per_chunk;
+        const int t0 = bound[c], tc = bound[c + 1] - bound[c];
         const size_t off = 2 * (size_t)t0 * a->H, bytes = 2 * (size_t)tc * a->H;
         mok_args ac = *a;
         ac.T = tc;
