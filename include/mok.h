@@ -195,8 +195,8 @@ int mok_profile_end(float* ms, int max_calls_out, int* n_calls);
  */
 int mok_debug_counters(const void* workspace, void* stream, unsigned long long* out);
 
-/* Number of kernels one mok_moe_forward_ex call enqueues for these arguments (the 256-byte header memset is
-   not counted); 0 on bad sizes. */
+/* Number of kernels one mok_moe_forward_ex call enqueues for these arguments (the memset of the workspace header
+   is not counted); 0 on bad sizes. */
 int mok_launch_count(int T, int H, int I, int I_shared, int E, int k, const mok_config* config);
 
 int mok_last_cuda_error(void);          /* cudaError_t of the most recent failed CUDA call on this thread */

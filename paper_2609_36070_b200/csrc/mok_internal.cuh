@@ -15,7 +15,7 @@ constexpr int SCHED_CHUNK = 2048;    // routes handled by one block of the sched
 constexpr int MAX_E = 512;
 constexpr int MAX_K = 32;
 
-// Device-side control block at the start of the workspace (one 256-byte slot).
+// Device-side control block at the start of the workspace.
 struct WsHeader {
     int32_t status;        // 0 or a negative mok_status written by a kernel
     int32_t n_mtiles;      // number of 128-row tiles of the padded dispatch buffer (written by the schedule)
