@@ -54,6 +54,7 @@ enum {
 };
 
 #define MOK_MAX_HOST_CHUNKS 8
+#define MOK_DEBUG_STARVE 2
 
 /* Optional tuning / debugging knobs.  Zero-initialise for defaults. */
 typedef struct mok_config {
@@ -66,7 +67,10 @@ typedef struct mok_config {
                              operand loads (no expert-sorted copy of x), 2 = separate gather kernel + TMA loads */
     int32_t cta_group;    /* tcgen05 GEMMs: 0 = choose by shape, 1 = one CTA per 128-row tile, 2 = CTA pairs sharing a
                              256-row tile (cta_group::2; halves the weight traffic into each SM) */
-    int32_t debug;        /* != 0: the tcgen05 GEMMs accumulate wait-time counters (see mok_debug_counters) */
+    int32_t debug;        /* 1: the tcgen05 GEMMs accumulate wait-time counters (see mok_debug_counters).
+                             MOK_DEBUG_STARVE: test hook for the bounded waits -- the gate/up GEMM's TMA producer
+                             issues nothing and every wait gives up after 2 ms, so the call must end with
+                             mok_read_status() == MOK_ERR_TIMEOUT and a usable context (output undefined) */
     int32_t host_chunks;  /* mok_moe_forward_host: token chunks whose copies overlap compute (0 = choose by T,
                              at most MOK_MAX_HOST_CHUNKS) */
 } mok_config;

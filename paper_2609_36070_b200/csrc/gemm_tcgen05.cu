@@ -156,7 +156,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
-        if (lane == 0) {
+        if (lane == 0 && !a.starve) {
             int s = 0;
             uint32_t ph = 0;
             long long dbg_prod = 0;

@@ -192,8 +192,15 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
     g.tile_m = tile_m;
     g.pad_offsets = reinterpret_cast<const int32_t*>(ws + L.pad_offsets);
     g.counts = reinterpret_cast<const int32_t*>(ws + L.counts);
-    const bool dbg = a->config && a->config->debug;
+    const bool dbg = a->config && a->config->debug == 1;
     g.dbg_slot = dbg ? 1 : -1;
+    if (a->config && a->config->debug == MOK_DEBUG_STARVE) {
+        // test hook (see mok.h): the gate/up GEMM's producer stays silent and every wait gives up after 2 ms
+        const uint32_t limit_us = 2000;
+        e = cudaMemcpyAsync(&hdr->wait_limit_us, &limit_us, sizeof(limit_us), cudaMemcpyHostToDevice, s);
+        if (e != cudaSuccess) return cuda_fail(e);
+        g.starve = 1;
+    }
     // routed experts: h = silu(Xg Wg^T) * (Xg Wu^T);  y = h Wd^T
     if (simt) {
         g.A = reinterpret_cast<const __nv_bfloat16*>(ws + L.xg);
@@ -209,6 +216,7 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
     g.K = a->H; g.N = a->I; g.ldc = a->I; g.E = a->E; g.rows_pad = L.Rpad; g.dense_rows = 0;
     if ((rc = run_gemm(g, true, a->config, s))) return rc;
     g.row_token = nullptr;
+    g.starve = 0;
     g.a_rows = L.Rpad;
     g.dbg_slot = dbg ? 2 : -1;
     MOK_MARK(MOK_STAGE_GEMM1 + 1);

@@ -19,8 +19,9 @@ constexpr int MAX_K = 32;
 struct WsHeader {
     int32_t status;        // 0 or a negative mok_status written by a kernel
     int32_t n_mtiles;      // number of 128-row tiles of the padded dispatch buffer (written by the schedule)
-    int32_t where;         // diagnostic: which wait gave up (role * 1000 + site)
-    int32_t pad[61];
+    int32_t where;         // diagnostic: which wait gave up (site number inside the kernel)
+    uint32_t wait_limit_us; // 0 = default (2 s): bound of every mbarrier wait, in microseconds
+    int32_t pad[60];
     // optional wait-time counters of the tcgen05 GEMMs (config.debug): [slot][counter], SM cycles summed over CTAs
     unsigned long long dbg[4][8];
 };
@@ -65,6 +66,7 @@ struct GemmArgs {
     int32_t max_mt;
     int32_t tile_m;              // rows of one tile of the padded row space: 128, or 256 for CTA pairs
     int32_t dbg_slot;            // >= 0: accumulate wait-time counters into header->dbg[dbg_slot]
+    int32_t starve;              // test hook: the TMA producer issues nothing, so the kernel's waits run out
     WsHeader* header;
 };
 

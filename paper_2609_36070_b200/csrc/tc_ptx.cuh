@@ -56,7 +56,8 @@ static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity
     while (!mbar_try_wait(bar, parity)) {
         if ((++spins & 127u) == 0u) {
             if (*abort_flag) return false;
-            if (globaltimer() - t0 > WAIT_LIMIT_NS) {
+            const unsigned long long limit = hdr->wait_limit_us ? 1000ull * hdr->wait_limit_us : WAIT_LIMIT_NS;
+            if (globaltimer() - t0 > limit) {
                 *abort_flag = 1u;
                 atomicCAS(&hdr->status, 0, (int)MOK_ERR_TIMEOUT);
                 hdr->where = site;

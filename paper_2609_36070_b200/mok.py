@@ -23,6 +23,7 @@ EXPORTS = ["mok_moe_forward", "mok_workspace_bytes", "mok_moe_forward_ex", "mok_
            "mok_schedule", "mok_read_status", "mok_launch_count", "mok_last_cuda_error", "mok_status_string",
            "mok_version", "mok_profile_begin", "mok_profile_end", "mok_schedule_noalloc", "mok_debug_counters"]
 MOK_NOALLOC_MAX_ROUTES = 32768
+MOK_DEBUG_STARVE = 2
 STAGES = ["router", "schedule", "gather", "gemm1", "gemm2", "shared_gemm1", "shared_gemm2", "combine"]
 
 

@@ -153,3 +153,20 @@ def test_argument_errors_launch_nothing():
     x0 = torch.empty((0, cfg.H), dtype=torch.bfloat16, device="cuda")
     out0 = m.mok_moe_forward_ex(x0, *args[1:], cfg.k, ws)
     assert out0.shape == (0, cfg.H)
+
+
+def test_bounded_waits_report_a_timeout_and_leave_the_context_usable():
+    """Failure detection without a fault: the test hook silences the gate/up GEMM's TMA producer, so its MMA issuer
+    waits for operands that never come.  Every wait is bounded (2 ms here), the kernel records MOK_ERR_TIMEOUT, frees
+    its tensor memory and returns; the next call on the same context must be correct again."""
+    m = mok()
+    cfg = inputs.CONFIGS["tiny"]
+    d = inputs.make_inputs(cfg)
+    g = pu.upload(d)
+    ws = m.alloc_workspace(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k)
+    good = pu.run_gpu(cfg, g, ws=ws, stages=False).clone()
+    m.mok_moe_forward_ex(g["x"], g["W_r"], g["bias"], g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], cfg.k, ws,
+                         config=m._config(debug=m.MOK_DEBUG_STARVE))
+    assert m.mok_read_status(ws) == m.MOK_ERR_TIMEOUT
+    again = pu.run_gpu(cfg, g, ws=ws, stages=False)
+    assert torch.equal(good.view(torch.int16), again.view(torch.int16))
