@@ -66,7 +66,8 @@ typedef struct mok_config {
     int32_t gather_mode;  /* token gather of the routed gate/up GEMM: 0 = choose by shape, 1 = fused into the GEMM's
                              operand loads (no expert-sorted copy of x), 2 = separate gather kernel + TMA loads */
     int32_t cta_group;    /* tcgen05 GEMMs: 0 = choose by shape, 1 = one CTA per 128-row tile, 2 = CTA pairs sharing a
-                             256-row tile (cta_group::2; halves the weight traffic into each SM) */
+                             256-row tile (cta_group::2; halves the weight traffic into each SM), 3 = one CTA per
+                             256-row tile with two accumulators (same traffic saving, no cross-CTA signalling) */
     int32_t debug;        /* 1: the tcgen05 GEMMs accumulate wait-time counters (see mok_debug_counters).
                              MOK_DEBUG_STARVE: test hook for the bounded waits -- the gate/up GEMM's TMA producer
                              issues nothing and every wait gives up after 2 ms, so the call must end with

@@ -1,0 +1,392 @@
+// Grouped expert GEMMs, 256-row tiles in ONE CTA (paper, Section 2.1: the expert FFN; Section 3 cost model: keep the
+// tensor cores fed, T_comp, against the memory system, T_mem).
+//
+// The 128 x 256 kernel (gemm_tcgen05.cu) moves 48 KB per k-block and can hold four such stages; measured on B200 that
+// is not enough bytes in flight to cover the ~1.4 us from TMA issue to landed data, and its MMA issuer waits for
+// operands 20-30 % of the time.  Here a tile is TWO 128-row halves that share one 256-row weight tile: per k-block
+// 16 + 16 KB of activations and 32 KB of weights feed twice the MMA work, so every stage in flight carries 1024
+// tensor-pipe cycles instead of 512 (three 64 KB stages), and a third less data crosses L2 -> SM per FLOP.  This is
+// what a CTA pair (cta_group::2) buys, without any cross-CTA signalling.  The price: both accumulators (2 x 256 TMEM
+// columns) belong to one tile, so the epilogue of a tile does not overlap the next tile's MMAs; eight epilogue warps
+// (four per accumulator) keep that bubble to the time it takes to read the accumulators out of TMEM.  The second half
+// of a tile is skipped when the expert's remaining rows fit in the first, so expert segments are still padded to 128
+// rows only.
+//
+//   warp 0        TMA producer : A halves (unless gathered) and the B tile -> 3-stage ring
+//   warp 1        MMA issuer   : per k-block 4 MMAs into accumulator 0 and, for a two-half tile, 4 into accumulator 1
+//   warps 2..5    epilogue of accumulator 0 (rows 0..127 of the tile);  warps 6..9: accumulator 1 (rows 128..255)
+//   warps 10..13  gather (GATHER only): token rows of x through the schedule's row -> token table (pull dispatch,
+//                 Section 3.1), 16-byte cp.async into the swizzled A halves
+// Tile order, epilogue variants (EPI_SWIGLU / EPI_BF16 / EPI_F32), determinism and the bounded waits are those of
+// gemm_tcgen05.cu.
+#include "mok_internal.cuh"
+#include "tc_ptx.cuh"
+
+namespace mok {
+namespace m2 {
+
+using namespace tc;
+
+constexpr int BM = 128, BN = 256, BK = 64, UMMA_K = 16, STAGES = 3;
+constexpr int A_BYTES = BM * BK * 2;           // 16 KB per half
+constexpr int B_BYTES = BN * BK * 2;           // 32 KB
+constexpr int STAGE_BYTES = 2 * A_BYTES + B_BYTES;   // 64 KB
+constexpr int TM = 2 * BM;                     // rows of a full tile
+constexpr int TMEM_COLS = 512;
+constexpr int EPI_WARPS = 8;
+constexpr int THREADS = 64 + 32 * EPI_WARPS;   // producer + MMA + epilogue warps = 320
+constexpr int GATHER_THREADS = 128;
+constexpr int GROUP_TILES = 8;                 // 2048 rows per rasterisation group
+constexpr int SLAB_BYTES = 4096;               // per epilogue warp: 32 rows x 64 bf16 columns (one swizzled box)
+constexpr int SMEM_CTRL = 256;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_WARPS * SLAB_BYTES + SMEM_CTRL + 1024;
+
+struct Ctrl {
+    uint64_t full[STAGES], empty[STAGES];
+    uint64_t tfull[2], tempty[2];              // per accumulator
+    uint32_t tmem_base, abort;
+};
+static_assert(sizeof(Ctrl) <= SMEM_CTRL, "control block too large");
+
+constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+
+struct Tile { int e, n, row0, valid; };        // valid: real rows of this tile (1..256); > 128 => both halves
+
+__device__ __forceinline__ Tile decode_tile(const GemmArgs& a, int L, int n_nt, int n_mt_total) {
+    Tile t;
+    int mt0, m_cnt, pad0, cnt;
+    if (a.dense_rows > 0) {
+        t.e = 0; mt0 = 0; m_cnt = n_mt_total; pad0 = 0; cnt = a.dense_rows;
+    } else {
+        t.e = __ldg(a.tile_expert + L / n_nt);
+        mt0 = __ldg(a.mt_start + t.e);
+        m_cnt = __ldg(a.mt_start + t.e + 1) - mt0;
+        pad0 = __ldg(a.pad_offsets + t.e);
+        cnt = __ldg(a.counts + t.e);
+    }
+    const int r = L - n_nt * mt0;
+    const int per_group = GROUP_TILES * n_nt;
+    const int g = r / per_group;
+    const int rem = r - g * per_group;
+    const int in_group = min(GROUP_TILES, m_cnt - g * GROUP_TILES);
+    t.n = rem / in_group;
+    const int m = g * GROUP_TILES + (rem - t.n * in_group);
+    t.row0 = pad0 + m * TM;
+    t.valid = min(TM, cnt - m * TM);
+    return t;
+}
+
+template <int EPI, bool GATHER>
+__global__ void __launch_bounds__(THREADS + (GATHER ? GATHER_THREADS : 0), 1)
+gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
+               const __grid_constant__ CUtensorMap tmapC, const GemmArgs a, const int n_nt, const int k_blocks) {
+    constexpr bool SWIGLU = (EPI == EPI_SWIGLU);
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t* smem = smem_raw + (base - raw);
+    Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem + STAGES * STAGE_BYTES + EPI_WARPS * SLAB_BYTES);
+    volatile uint32_t* abort_flag = &ctrl->abort;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    int n_mt_total = (a.dense_rows > 0) ? (a.dense_rows + TM - 1) / TM : *a.n_mtiles;
+    if (n_mt_total > a.max_mt) n_mt_total = a.max_mt;
+    const int total = n_mt_total * n_nt;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(smem_u32(&ctrl->full[s]), GATHER ? 1 + GATHER_THREADS : 1);
+            mbar_init(smem_u32(&ctrl->empty[s]), 1);
+        }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(smem_u32(&ctrl->tfull[s]), 1);
+            mbar_init(smem_u32(&ctrl->tempty[s]), 4);           // one arrive per epilogue warp of that accumulator
+        }
+        ctrl->abort = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&ctrl->tmem_base)), "r"((uint32_t)TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = ctrl->tmem_base;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0 && !a.starve) {
+            int s = 0;
+            uint32_t ph = 0;
+            const int b_rows_per_expert = (SWIGLU ? 2 : 1) * a.N;
+            for (int L = blockIdx.x; L < total; L += gridDim.x) {
+                const Tile t = decode_tile(a, L, n_nt, n_mt_total);
+                const bool two = t.valid > BM;
+                const int brow0 = t.e * b_rows_per_expert + (SWIGLU ? t.n * (BN / 2) : t.n * BN);
+                const int brow1 = SWIGLU ? brow0 + a.N : brow0 + BN / 2;
+                bool ok = true;
+                for (int kb = 0; kb < k_blocks; ++kb) {
+                    ok = mbar_wait(smem_u32(&ctrl->empty[s]), ph ^ 1u, abort_flag, a.header, 1);
+                    if (!ok) break;
+                    const uint32_t full = smem_u32(&ctrl->full[s]);
+                    const uint32_t sa = base + s * STAGE_BYTES, sb = sa + 2 * A_BYTES;
+                    mbar_expect_tx(full, B_BYTES + (GATHER ? 0 : (two ? 2 : 1) * A_BYTES));
+                    if (!GATHER) {
+                        tma_load_2d(sa, &tmapA, full, kb * BK, t.row0);
+                        if (two) tma_load_2d(sa + A_BYTES, &tmapA, full, kb * BK, t.row0 + BM);
+                    }
+                    tma_load_2d(sb, &tmapB, full, kb * BK, brow0);
+                    tma_load_2d(sb + B_BYTES / 2, &tmapB, full, kb * BK, brow1);
+                    if (++s == STAGES) { s = 0; ph ^= 1u; }
+                }
+                if (!ok) break;
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            int s = 0;
+            uint32_t ph = 0, ap0 = 0, ap1 = 0;        // phases of tempty[0], tempty[1]: they advance per use
+            for (int L = blockIdx.x; L < total; L += gridDim.x) {
+                const Tile t = decode_tile(a, L, n_nt, n_mt_total);
+                const bool two = t.valid > BM;
+                bool ok = mbar_wait(smem_u32(&ctrl->tempty[0]), ap0 ^ 1u, abort_flag, a.header, 2);
+                if (ok && two) ok = mbar_wait(smem_u32(&ctrl->tempty[1]), ap1 ^ 1u, abort_flag, a.header, 8);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t d0 = tmem_base, d1 = tmem_base + BN;
+                for (int kb = 0; kb < k_blocks; ++kb) {
+                    ok = mbar_wait(smem_u32(&ctrl->full[s]), ph, abort_flag, a.header, 3);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t sa = base + s * STAGE_BYTES;
+                    const uint64_t a0 = make_smem_desc(sa), a1 = make_smem_desc(sa + A_BYTES);
+                    const uint64_t bd = make_smem_desc(sa + 2 * A_BYTES);
+#pragma unroll
+                    for (int j = 0; j < BK / UMMA_K; ++j)
+                        tc_mma<1>(d0, a0 + (uint64_t)(j * 2), bd + (uint64_t)(j * 2), IDESC, (kb | j) ? 1u : 0u);
+                    if (two) {
+#pragma unroll
+                        for (int j = 0; j < BK / UMMA_K; ++j)
+                            tc_mma<1>(d1, a1 + (uint64_t)(j * 2), bd + (uint64_t)(j * 2), IDESC, (kb | j) ? 1u : 0u);
+                    }
+                    tc_commit<1>(smem_u32(&ctrl->empty[s]));
+                    if (++s == STAGES) { s = 0; ph ^= 1u; }
+                }
+                if (!ok) break;
+                tc_commit<1>(smem_u32(&ctrl->tfull[0]));
+                ap0 ^= 1u;
+                if (two) { tc_commit<1>(smem_u32(&ctrl->tfull[1])); ap1 ^= 1u; }
+            }
+        }
+        __syncwarp();
+    } else if (GATHER && warp >= 2 + EPI_WARPS) {
+        // ------------------------------------------------------------------ gather warps (pull dispatch)
+        // Warp gw owns rows 32 gw .. 32 gw + 31 of each half; lane = (sub-row 0..3, 16-byte chunk 0..7); pass i of half
+        // h covers row 128 h + 32 gw + 4 i + sub-row.  Chunk c of row r lands at r*128 + ((c ^ (r & 7)) * 16) inside
+        // its half.  Rows past the expert's segment re-read the tile's first row (computed, never combined).
+        const int gw = warp - (2 + EPI_WARPS), sub = lane >> 3, chunk = lane & 7;
+        int s = 0;
+        uint32_t ph = 0;
+        for (int L = blockIdx.x; L < total; L += gridDim.x) {
+            const Tile t = decode_tile(a, L, n_nt, n_mt_total);
+            const bool two = t.valid > BM;
+            const int tok0 = __ldg(a.row_token + t.row0);
+            const __nv_bfloat16* src[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const int r = (i >> 3) * BM + gw * 32 + (i & 7) * 4 + sub;
+                const int tok = (r < t.valid) ? __ldg(a.row_token + t.row0 + r) : tok0;
+                src[i] = a.A + (size_t)tok * a.K + chunk * 8;
+            }
+            bool ok = true;
+            for (int kb = 0; kb < k_blocks; ++kb) {
+                ok = mbar_wait(smem_u32(&ctrl->empty[s]), ph ^ 1u, abort_flag, a.header, 5);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                const uint32_t sa = base + s * STAGE_BYTES;
+                const bool in_k = (kb * BK + chunk * 8) < a.K;            // K tail: zero-fill
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    if (i < 8 || two) {
+                        const int rr = gw * 32 + (i & 7) * 4 + sub;       // row inside the half
+                        const uint32_t dst = sa + (i >> 3) * A_BYTES + rr * 128 + ((chunk ^ (rr & 7)) << 4);
+                        cp_async_16(dst, in_k ? (const void*)(src[i] + kb * BK) : (const void*)a.A, in_k ? 16u : 0u);
+                    }
+                }
+                cp_async_mbar_arrive(smem_u32(&ctrl->full[s]));
+                if (++s == STAGES) { s = 0; ph ^= 1u; }
+            }
+            if (!ok) break;
+        }
+        asm volatile("cp.async.wait_all;" ::: "memory");
+    } else {
+        // ------------------------------------------------------------------ epilogue: warps 2..5 -> accumulator 0,
+        // warps 6..9 -> accumulator 1.  TMEM -> registers -> (SwiGLU) -> bf16 -> this warp's swizzled slab (32 rows x
+        // 64 columns) -> TMA store; the accumulator is handed back right after its last TMEM read.
+        const int acc = (warp - 2) >> 2;                      // which accumulator / half of the tile
+        const int quad = warp & 3;                            // TMEM lane quadrant this warp may access
+        const uint32_t slab = base + STAGES * STAGE_BYTES + (warp - 2) * SLAB_BYTES;
+        uint32_t aph = 0;
+        for (int L = blockIdx.x; L < total; L += gridDim.x) {
+            const Tile t = decode_tile(a, L, n_nt, n_mt_total);
+            if (acc == 1 && t.valid <= BM) continue;          // this tile has no second half
+            bool ok = mbar_wait(smem_u32(&ctrl->tfull[acc]), aph, abort_flag, a.header, 4);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            aph ^= 1u;
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * BN);
+            const int row = t.row0 + acc * BM + quad * 32;
+            if (EPI == EPI_F32) {
+                float* frow = reinterpret_cast<float*>(a.C) + (size_t)(row + lane) * a.ldc;
+                const int c0 = t.n * BN;
+#pragma unroll 1
+                for (int c = 0; c < BN; c += 32) {
+                    uint32_t r[32];
+                    tc_ld32(taddr + c, r);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int v = 0; v < 8; ++v) {
+                        const int col = c0 + c + v * 4;
+                        if (col < a.N)
+                            *reinterpret_cast<uint4*>(frow + col) = make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&ctrl->tempty[acc]));
+            } else {
+                constexpr int PASSES = SWIGLU ? 2 : 4;        // 64 output columns per pass
+                const int c0 = SWIGLU ? t.n * (BN / 2) : t.n * BN;
+#pragma unroll 1
+                for (int pass = 0; pass < PASSES; ++pass) {
+                    if (lane == 0) tma_store_wait_read();     // the slab's previous store has been read out
+                    __syncwarp();
+#pragma unroll
+                    for (int c = 0; c < 64; c += 32) {
+                        uint32_t o[16];
+                        if (SWIGLU) {
+                            uint32_t g[32], u[32];
+                            tc_ld32(taddr + pass * 64 + c, g);
+                            tc_ld32(taddr + BN / 2 + pass * 64 + c, u);
+                            tc_wait_ld();
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) {
+                                float g0 = __uint_as_float(g[2 * i]), g1 = __uint_as_float(g[2 * i + 1]);
+                                float h0 = (g0 / (1.f + __expf(-g0))) * __uint_as_float(u[2 * i]);
+                                float h1 = (g1 / (1.f + __expf(-g1))) * __uint_as_float(u[2 * i + 1]);
+                                o[i] = pack_bf16(h0, h1);
+                            }
+                        } else {
+                            uint32_t r[32];
+                            tc_ld32(taddr + pass * 64 + c, r);
+                            tc_wait_ld();
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) o[i] = pack_bf16(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
+                        }
+                        const uint32_t line = slab + lane * 128;     // 32 columns = 4 chunks of 16 bytes, index c/8 + v
+#pragma unroll
+                        for (int v = 0; v < 4; ++v)
+                            st_shared_v4(line + ((((c >> 3) + v) ^ (lane & 7)) << 4), o[4 * v], o[4 * v + 1], o[4 * v + 2], o[4 * v + 3]);
+                    }
+                    if (pass == PASSES - 1) tc_fence_before();   // all TMEM reads of this accumulator are done
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) {
+                        if (pass == PASSES - 1) mbar_arrive(smem_u32(&ctrl->tempty[acc]));
+                        const int col = c0 + pass * 64;
+                        if (col < a.N) tma_store_2d(&tmapC, slab, col, row);
+                        tma_store_commit();
+                    }
+                }
+            }
+        }
+        if (lane == 0) tma_store_wait_all();
+        __syncwarp();
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    if (*abort_flag) {   // failure path only: give copies and MMAs already in flight time to land before leaving
+        const unsigned long long t0 = globaltimer();
+        while (globaltimer() - t0 < 200000ull) { }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS) : "memory");
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn get_encode() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+static bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows, uint64_t stride) {
+    EncodeTiledFn enc = get_encode();
+    if (!enc) return false;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {stride * 2};
+    cuuint32_t box[2] = {(cuuint32_t)BK, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int EPI, bool GATHER>
+static cudaError_t launch_one(const CUtensorMap& mA, const CUtensorMap& mB, const CUtensorMap& mC, const GemmArgs& a,
+                              int n_nt, int k_blocks, int grid, cudaStream_t s) {
+    static int sm_count = 0;
+    if (!sm_count) {
+        cudaError_t e = cudaFuncSetAttribute(gemm_m2_kernel<EPI, GATHER>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
+    }
+    if (grid <= 0 || grid > sm_count) grid = sm_count;
+    gemm_m2_kernel<EPI, GATHER><<<grid, THREADS + (GATHER ? GATHER_THREADS : 0), SMEM_BYTES, s>>>(mA, mB, mC, a, n_nt,
+                                                                                                 k_blocks);
+    return cudaGetLastError();
+}
+
+}  // namespace m2
+
+cudaError_t launch_gemm_m2(const GemmArgs& a, int epi, int grid, cudaStream_t s) {
+    using namespace m2;
+    const bool swiglu = (epi == EPI_SWIGLU), gather = (a.row_token != nullptr);
+    CUtensorMap mA, mB, mC;
+    const uint64_t b_rows = (uint64_t)a.E * (swiglu ? 2 : 1) * a.N;
+    if (!make_map(&mA, a.A, (uint64_t)a.a_rows, (uint64_t)a.K, BM, (uint64_t)a.K)) return cudaErrorInvalidValue;
+    if (!make_map(&mB, a.B, b_rows, (uint64_t)a.K, BN / 2, (uint64_t)a.K)) return cudaErrorInvalidValue;
+    if (epi == EPI_F32) mC = mB;      // the fp32 epilogue stores directly
+    else if (!make_map(&mC, a.C, (uint64_t)a.rows_pad, (uint64_t)a.N, 32, (uint64_t)a.ldc)) return cudaErrorInvalidValue;
+    const int n_nt = swiglu ? (a.N + BN / 2 - 1) / (BN / 2) : (a.N + BN - 1) / BN;
+    const int k_blocks = (a.K + BK - 1) / BK;
+    if (epi == EPI_SWIGLU && gather) return launch_one<EPI_SWIGLU, true>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
+    if (epi == EPI_SWIGLU) return launch_one<EPI_SWIGLU, false>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
+    if (epi == EPI_BF16 && !gather) return launch_one<EPI_BF16, false>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
+    if (epi == EPI_F32 && !gather) return launch_one<EPI_F32, false>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace mok

@@ -8,6 +8,7 @@
 namespace mok {
 
 static thread_local int g_last_cuda_error = 0;
+constexpr int M2_MIN_K = 1536;   // shortest K for which the 256-row-tile kernel is chosen by default
 
 static int cuda_fail(cudaError_t e) {
     g_last_cuda_error = (int)e;
@@ -58,6 +59,8 @@ bool ws_layout(int T, int H, int I, int Is, int E, int k, WsLayout* L) {
     L->pad_offsets = take(sizeof(int32_t) * (E + 1));
     L->mt_start = take(sizeof(int32_t) * (E + 1));
     L->tile_expert = take(sizeof(int32_t) * (size_t)L->max_mt);
+    L->mt_start2 = take(sizeof(int32_t) * (E + 1));
+    L->tile_expert2 = take(sizeof(int32_t) * (size_t)L->max_mt);
     L->perm = take(sizeof(int32_t) * (size_t)(R > 0 ? R : 1));
     L->inv = take(sizeof(int32_t) * (size_t)(R > 0 ? R : 1));
     L->pos = take(sizeof(int32_t) * (size_t)(R > 0 ? R : 1));
@@ -92,7 +95,7 @@ static int validate(const mok_args* a, WsLayout* L, size_t extra_ws) {
     if (a->config && (a->config->impl < 0 || a->config->impl > 2 || a->config->grid < 0 ||
                       a->config->router_impl < 0 || a->config->router_impl > 2 ||
                       a->config->gather_mode < 0 || a->config->gather_mode > 2 ||
-                      a->config->cta_group < 0 || a->config->cta_group > 2 ||
+                      a->config->cta_group < 0 || a->config->cta_group > 3 ||
                       a->config->host_chunks < 0 || a->config->host_chunks > MOK_MAX_HOST_CHUNKS))
         return MOK_ERR_SHAPE;
     return MOK_OK;
@@ -127,8 +130,26 @@ static int tile_rows(const mok_config* cfg, int I) {
     return fused_gather(cfg, I) ? TILE_M : 2 * TILE_M;
 }
 
-static int run_gemm(const GemmArgs& g, bool swiglu, const mok_config* cfg, cudaStream_t s) {
+// 256-row tiles with two accumulators in one CTA (gemm_tcgen05_m2.cu): used on the 128-padded row space through the
+// second tile table.  cta_group = 3 forces it; by default it serves GEMMs whose K is long enough to amortise the
+// accumulator hand-over between tiles.
+static bool use_m2(const mok_config* cfg, int K, int tile_m) {
+    if (use_simt(cfg) || use_tn(cfg) || tile_m != TILE_M) return false;
+    if (cfg && cfg->cta_group == 3) return true;
+    if (cfg && cfg->cta_group != 0) return false;
+    return K >= M2_MIN_K;
+}
+
+static int run_gemm(GemmArgs g, bool swiglu, const mok_config* cfg, const WsLayout& L, char* ws, cudaStream_t s) {
     const int epi = swiglu ? EPI_SWIGLU : EPI_BF16, grid = cfg ? cfg->grid : 0;
+    if (use_m2(cfg, g.K, g.tile_m)) {
+        WsHeader* hdr = reinterpret_cast<WsHeader*>(ws + L.header);
+        g.n_mtiles = &hdr->n_mtiles2;
+        g.mt_start = reinterpret_cast<const int32_t*>(ws + L.mt_start2);
+        g.tile_expert = reinterpret_cast<const int32_t*>(ws + L.tile_expert2);
+        cudaError_t e2 = launch_gemm_m2(g, epi, grid, s);
+        return e2 == cudaSuccess ? MOK_OK : cuda_fail(e2);
+    }
     cudaError_t e = use_simt(cfg) ? launch_gemm_simt(g, swiglu, s)
                     : use_tn(cfg) ? launch_gemm_tn(g, epi, grid, s) : launch_gemm_tc(g, epi, grid, s);
     return e == cudaSuccess ? MOK_OK : cuda_fail(e);
@@ -143,7 +164,9 @@ static int route_stage(const mok_args* a, const WsLayout& L, char* ws, const __n
     else
         e = launch_router_tc(x, a->W_router, a->router_bias, a->T, a->H, a->E, a->k, L, ws,
                              reinterpret_cast<WsHeader*>(ws + L.header), a->config ? a->config->grid : 0,
-                             tile_rows(a->config, a->I > 0 ? a->I : 8), use_tn(a->config), idx, w, s);
+                             tile_rows(a->config, a->I > 0 ? a->I : 8),
+                             use_tn(a->config) ? 2 : use_m2(a->config, a->H, tile_rows(a->config, a->I > 0 ? a->I : 8)) ? 3 : 0,
+                             idx, w, s);
     if (e != cudaSuccess) return cuda_fail(e);
     if (a->topk_idx) {
         e = cudaMemcpyAsync(a->topk_idx, idx, sizeof(int32_t) * (size_t)L.R, cudaMemcpyDeviceToDevice, s);
@@ -214,7 +237,7 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
     g.B = reinterpret_cast<const __nv_bfloat16*>(a->W_gate_up);
     g.C = ws + L.h;
     g.K = a->H; g.N = a->I; g.ldc = a->I; g.E = a->E; g.rows_pad = L.Rpad; g.dense_rows = 0;
-    if ((rc = run_gemm(g, true, a->config, s))) return rc;
+    if ((rc = run_gemm(g, true, a->config, L, ws, s))) return rc;
     g.row_token = nullptr;
     g.starve = 0;
     g.a_rows = L.Rpad;
@@ -224,7 +247,7 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
     g.B = reinterpret_cast<const __nv_bfloat16*>(a->W_down);
     g.C = ws + L.y;
     g.K = a->I; g.N = a->H; g.ldc = a->H;
-    if ((rc = run_gemm(g, false, a->config, s))) return rc;
+    if ((rc = run_gemm(g, false, a->config, L, ws, s))) return rc;
     MOK_MARK(MOK_STAGE_GEMM2 + 1);
     g.dbg_slot = dbg ? 3 : -1;
     if (a->I_shared > 0) {   // shared expert: every token in natural order, no gather
@@ -232,13 +255,13 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
         g.B = reinterpret_cast<const __nv_bfloat16*>(a->W_shared_gate_up);
         g.C = ws + L.hs;
         g.K = a->H; g.N = a->I_shared; g.ldc = a->I_shared; g.E = 1; g.rows_pad = L.Tpad; g.a_rows = a->T; g.dense_rows = a->T;
-        if ((rc = run_gemm(g, true, a->config, s))) return rc;
+        if ((rc = run_gemm(g, true, a->config, L, ws, s))) return rc;
         MOK_MARK(MOK_STAGE_SHARED_GEMM1 + 1);
         g.A = reinterpret_cast<const __nv_bfloat16*>(ws + L.hs);
         g.B = reinterpret_cast<const __nv_bfloat16*>(a->W_shared_down);
         g.C = ws + L.ysh;
         g.K = a->I_shared; g.N = a->H; g.ldc = a->H; g.a_rows = L.Tpad;
-        if ((rc = run_gemm(g, false, a->config, s))) return rc;
+        if ((rc = run_gemm(g, false, a->config, L, ws, s))) return rc;
         MOK_MARK(MOK_STAGE_SHARED_GEMM2 + 1);
     } else {
         MOK_MARK(MOK_STAGE_SHARED_GEMM1 + 1);

@@ -18,10 +18,11 @@ constexpr int MAX_K = 32;
 // Device-side control block at the start of the workspace.
 struct WsHeader {
     int32_t status;        // 0 or a negative mok_status written by a kernel
-    int32_t n_mtiles;      // number of 128-row tiles of the padded dispatch buffer (written by the schedule)
+    int32_t n_mtiles;      // number of tile_m-row tiles of the padded dispatch buffer (written by the schedule)
+    int32_t n_mtiles2;     // number of 2*tile_m-row tiles of the same buffer (second tile table)
     int32_t where;         // diagnostic: which wait gave up (site number inside the kernel)
     uint32_t wait_limit_us; // 0 = default (2 s): bound of every mbarrier wait, in microseconds
-    int32_t pad[60];
+    int32_t pad[59];
     // optional wait-time counters of the tcgen05 GEMMs (config.debug): [slot][counter], SM cycles summed over CTAs
     unsigned long long dbg[4][8];
 };
@@ -31,6 +32,7 @@ enum { DBG_MMA_WAIT_FULL = 0, DBG_MMA_WAIT_PFULL, DBG_MMA_WAIT_TEMPTY, DBG_MMA_T
 // Byte offsets of every workspace region, computed on the host from the sizes alone (no readback).
 struct WsLayout {
     size_t header, idx, w, counts, offsets, pad_offsets, mt_start, tile_expert, perm, inv, pos, blk_hist;
+    size_t mt_start2, tile_expert2;   // the same segments cut into tiles of 2*tile_m rows
     size_t row_token;     // int32 [Rpad]: source token of every row of the padded dispatch space (pad rows undefined)
     size_t wr_split;      // bf16 [3E, H]: W_r split into hi/mid/lo parts for the tensor-core router
     size_t logits;        // fp32 [Tpad, ldl] partial logits of the tensor-core router (ldl = 3E rounded up to 8)
@@ -83,8 +85,9 @@ cudaError_t launch_gemm_simt(const GemmArgs& a, bool swiglu, cudaStream_t s);
 enum { EPI_BF16 = 0, EPI_SWIGLU = 1, EPI_F32 = 2 };
 cudaError_t launch_gemm_tc(const GemmArgs& a, int epi, int grid, cudaStream_t s);
 cudaError_t launch_gemm_tn(const GemmArgs& a, int epi, int grid, cudaStream_t s);   // tokens on the MMA's N side
+cudaError_t launch_gemm_m2(const GemmArgs& a, int epi, int grid, cudaStream_t s);   // 256-row tiles, two accumulators
 cudaError_t launch_router_tc(const __nv_bfloat16* x, const float* Wr, const float* bias, int T, int H, int E, int k,
-                             const WsLayout& L, char* ws, WsHeader* hdr, int grid, int tile_m, bool tn, int32_t* idx,
+                             const WsLayout& L, char* ws, WsHeader* hdr, int grid, int tile_m, int variant, int32_t* idx,
                              float* w,
                              cudaStream_t s);
 

@@ -169,7 +169,7 @@ router_topk_kernel(const float* __restrict__ part, const float* __restrict__ bia
 }
 
 cudaError_t launch_router_tc(const __nv_bfloat16* x, const float* Wr, const float* bias, int T, int H, int E, int k,
-                             const WsLayout& L, char* ws, WsHeader* hdr, int grid, int tile_m, bool tn, int32_t* idx,
+                             const WsLayout& L, char* ws, WsHeader* hdr, int grid, int tile_m, int variant, int32_t* idx,
                              float* w, cudaStream_t s) {
     const int ldl = (3 * E + 7) / 8 * 8;
     __nv_bfloat16* split = reinterpret_cast<__nv_bfloat16*>(ws + L.wr_split);
@@ -190,7 +190,8 @@ cudaError_t launch_router_tc(const __nv_bfloat16* x, const float* Wr, const floa
     g.tile_m = tile_m;
     g.dbg_slot = -1;
     g.header = hdr;
-    e = tn ? launch_gemm_tn(g, EPI_F32, grid, s) : launch_gemm_tc(g, EPI_F32, grid, s);
+    e = variant == 2 ? launch_gemm_tn(g, EPI_F32, grid, s)
+        : variant == 3 ? launch_gemm_m2(g, EPI_F32, grid, s) : launch_gemm_tc(g, EPI_F32, grid, s);
     if (e != cudaSuccess) return e;
     int tblocks = (T + 7) / 8;
     if (tblocks > 148 * 16) tblocks = 148 * 16;

@@ -39,9 +39,10 @@ sched_hist_kernel(const int32_t* __restrict__ a, int n, int E, int32_t* __restri
 __global__ void __launch_bounds__(MAX_E)
 sched_scan_kernel(int32_t* __restrict__ blk_hist, int n_blk, int E, int max_mt, int tile_m, int pad_m,
                   int32_t* __restrict__ counts, int32_t* __restrict__ offsets, int32_t* __restrict__ pad_offsets,
-                  int32_t* __restrict__ mt_start, int32_t* __restrict__ tile_expert, WsHeader* __restrict__ hdr,
+                  int32_t* __restrict__ mt_start, int32_t* __restrict__ tile_expert,
+                  int32_t* __restrict__ mt_start2, int32_t* __restrict__ tile_expert2, WsHeader* __restrict__ hdr,
                   int32_t* __restrict__ counts_out, int32_t* __restrict__ offsets_out) {
-    __shared__ int32_t s_cnt[MAX_E], s_off[MAX_E + 1], s_mt[MAX_E + 1], s_pad[MAX_E + 1];
+    __shared__ int32_t s_cnt[MAX_E], s_off[MAX_E + 1], s_mt[MAX_E + 1], s_pad[MAX_E + 1], s_mt2[MAX_E + 1];
     const int e = threadIdx.x;
     int32_t total = 0;
     if (e < E) {
@@ -59,19 +60,23 @@ sched_scan_kernel(int32_t* __restrict__ blk_hist, int n_blk, int E, int max_mt, 
     }
     __syncthreads();
     if (e == 0) {   // E <= 512: a serial scan by one thread is a few hundred cycles
-        int32_t off = 0, mt = 0, pad = 0;
+        int32_t off = 0, mt = 0, pad = 0, mt2 = 0;
         for (int i = 0; i < E; ++i) {
             s_off[i] = off;
             s_mt[i] = mt;
+            s_mt2[i] = mt2;
             s_pad[i] = pad;
             off += s_cnt[i];
             mt += (s_cnt[i] + tile_m - 1) / tile_m;
+            mt2 += (s_cnt[i] + 2 * tile_m - 1) / (2 * tile_m);
             pad += (s_cnt[i] + pad_m - 1) / pad_m * pad_m;
         }
         s_off[E] = off;
         s_mt[E] = mt;
         s_pad[E] = pad;
+        s_mt2[E] = mt2;
         hdr->n_mtiles = mt;
+        hdr->n_mtiles2 = mt2;
         if (mt * (tile_m / TILE_M) > max_mt) hdr->status = MOK_ERR_SCHEDULE;
     }
     __syncthreads();
@@ -83,11 +88,14 @@ sched_scan_kernel(int32_t* __restrict__ blk_hist, int n_blk, int E, int max_mt, 
         if (counts_out) counts_out[e] = s_cnt[e];
         if (offsets_out) offsets_out[e] = s_off[e];
         for (int q = s_mt[e]; q < s_mt[e + 1] && q < max_mt; ++q) tile_expert[q] = e;
+        mt_start2[e] = s_mt2[e];
+        for (int q = s_mt2[e]; q < s_mt2[e + 1] && q < max_mt; ++q) tile_expert2[q] = e;
     }
     if (e == 0) {
         offsets[E] = s_off[E];
         pad_offsets[E] = s_pad[E];
         mt_start[E] = s_mt[E];
+        mt_start2[E] = s_mt2[E];
         if (offsets_out) offsets_out[E] = s_off[E];
     }
 }
@@ -165,7 +173,8 @@ cudaError_t launch_schedule(const int32_t* idx, int T, int E, int k, int tile_m,
     WsHeader* hdr = reinterpret_cast<WsHeader*>(ws + L.header);
     sched_hist_kernel<<<L.n_blk, SCHED_THREADS, 0, s>>>(idx, n, E, blk_hist);
     sched_scan_kernel<<<1, MAX_E, 0, s>>>(blk_hist, L.n_blk, E, L.max_mt, tile_m, pad_m, counts, offsets, pad_offsets, mt_start,
-                                          tile_expert, hdr, counts_out, offsets_out);
+                                          tile_expert, reinterpret_cast<int32_t*>(ws + L.mt_start2),
+                                          reinterpret_cast<int32_t*>(ws + L.tile_expert2), hdr, counts_out, offsets_out);
     sched_scatter_kernel<<<L.n_blk, SCHED_THREADS, sizeof(int32_t) * SCHED_WARPS * E, s>>>(
         idx, n, E, blk_hist, offsets, pad_offsets,
         reinterpret_cast<int32_t*>(ws + L.perm), reinterpret_cast<int32_t*>(ws + L.inv),

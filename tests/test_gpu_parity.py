@@ -30,13 +30,14 @@ SMALL = [
 
 
 @pytest.mark.parametrize("cfg", SMALL, ids=[c.name for c in SMALL])
-@pytest.mark.parametrize("impl", ["tcgen05_fused_gather", "tcgen05_separate_gather", "tcgen05_single_cta", "tcgen05_tokens_as_n", "simt"])
+@pytest.mark.parametrize("impl", ["tcgen05_fused_gather", "tcgen05_separate_gather", "tcgen05_single_cta", "tcgen05_256_row_tiles", "tcgen05_tokens_as_n", "simt"])
 def test_small_shapes_every_token(cfg, impl):
     m = mok()
     conf = {"simt": m._config(impl=m.MOK_IMPL_SIMT),
             "tcgen05_fused_gather": m._config(gather_mode=1),
             "tcgen05_separate_gather": m._config(gather_mode=2),
             "tcgen05_single_cta": m._config(cta_group=1),
+            "tcgen05_256_row_tiles": m._config(cta_group=3),
             "tcgen05_tokens_as_n": m._config(impl=m.MOK_IMPL_TCGEN05_TN)}[impl]
     out, st, rep = pu.full_parity(cfg, config=conf)
     print(cfg.name, impl, rep)
@@ -62,7 +63,7 @@ def test_tiny_config_every_token_and_determinism():
     out2 = pu.run_gpu(cfg, g, stages=False)
     assert torch.equal(out.view(torch.int16), out2.view(torch.int16))            # run-to-run bitwise identity
     for grid in (1, 2, 7, 148):                                                    # bits do not depend on the grid,
-        for cta_group in (1, 2):                                                   # nor on single CTAs vs CTA pairs
+        for cta_group in (1, 2, 3):                                                # nor on the tile / CTA arrangement
             o = pu.run_gpu(cfg, g, config=m._config(grid=grid, cta_group=cta_group), stages=False)
             assert torch.equal(out.view(torch.int16), o.view(torch.int16)), (grid, cta_group)
 
