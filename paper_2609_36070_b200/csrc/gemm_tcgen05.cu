@@ -353,8 +353,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
 #pragma unroll
                             for (int i = 0; i < 16; ++i) {
                                 float g0 = __uint_as_float(g[2 * i]), g1 = __uint_as_float(g[2 * i + 1]);
-                                float h0 = (g0 / (1.f + __expf(-g0))) * __uint_as_float(u[2 * i]);
-                                float h1 = (g1 / (1.f + __expf(-g1))) * __uint_as_float(u[2 * i + 1]);
+                                float h0 = swiglu(g0, __uint_as_float(u[2 * i]));
+                                float h1 = swiglu(g1, __uint_as_float(u[2 * i + 1]));
                                 o[i] = pack_bf16(h0, h1);
                             }
                         } else {

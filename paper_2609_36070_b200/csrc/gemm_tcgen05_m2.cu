@@ -151,16 +151,23 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
         if (lane == 0) {
             int s = 0;
             uint32_t ph = 0, ap0 = 0, ap1 = 0;        // phases of tempty[0], tempty[1]: they advance per use
+            const bool dbg = a.dbg_slot >= 0;
+            long long d_full = 0, d_tempty = 0, d_kb = 0;
+            const long long d_t0 = dbg ? clock64() : 0;
             for (int L = blockIdx.x; L < total; L += gridDim.x) {
                 const Tile t = decode_tile(a, L, n_nt, n_mt_total);
                 const bool two = t.valid > BM;
+                long long w0 = dbg ? clock64() : 0;
                 bool ok = mbar_wait(smem_u32(&ctrl->tempty[0]), ap0 ^ 1u, abort_flag, a.header, 2);
                 if (ok && two) ok = mbar_wait(smem_u32(&ctrl->tempty[1]), ap1 ^ 1u, abort_flag, a.header, 8);
+                if (dbg) d_tempty += clock64() - w0;
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t d0 = tmem_base, d1 = tmem_base + BN;
                 for (int kb = 0; kb < k_blocks; ++kb) {
+                    if (dbg) w0 = clock64();
                     ok = mbar_wait(smem_u32(&ctrl->full[s]), ph, abort_flag, a.header, 3);
+                    if (dbg) { d_full += clock64() - w0; d_kb += two ? 2 : 1; }
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t sa = base + s * STAGE_BYTES;
@@ -181,6 +188,13 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
                 tc_commit<1>(smem_u32(&ctrl->tfull[0]));
                 ap0 ^= 1u;
                 if (two) { tc_commit<1>(smem_u32(&ctrl->tfull[1])); ap1 ^= 1u; }
+            }
+            if (dbg) {   // k_blocks counted in 128-row units so that the figures compare with the 128-row kernel
+                unsigned long long* d = a.header->dbg[a.dbg_slot];
+                atomicAdd(d + DBG_MMA_WAIT_FULL, (unsigned long long)d_full);
+                atomicAdd(d + DBG_MMA_WAIT_TEMPTY, (unsigned long long)d_tempty);
+                atomicAdd(d + DBG_MMA_TOTAL, (unsigned long long)(clock64() - d_t0));
+                atomicAdd(d + DBG_KBLOCKS, (unsigned long long)d_kb);
             }
         }
         __syncwarp();
@@ -261,44 +275,56 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&ctrl->tempty[acc]));
             } else {
-                constexpr int PASSES = SWIGLU ? 2 : 4;        // 64 output columns per pass
+                // 64 output columns per pass.  The TMEM reads and the arithmetic of pass p+1 are done BEFORE waiting for
+                // the slab that pass p is about to overwrite, so the accumulator goes back to the MMA issuer as soon as
+                // its last column has been read, not after the stores.
+                constexpr int PASSES = SWIGLU ? 2 : 4;
                 const int c0 = SWIGLU ? t.n * (BN / 2) : t.n * BN;
-#pragma unroll 1
-                for (int pass = 0; pass < PASSES; ++pass) {
-                    if (lane == 0) tma_store_wait_read();     // the slab's previous store has been read out
-                    __syncwarp();
+                uint32_t cur[32], nxt[32];                    // one pass = 64 columns = 32 packed bf16 pairs per row
+                auto load_pass = [&](int pass, uint32_t (&o)[32]) {
 #pragma unroll
                     for (int c = 0; c < 64; c += 32) {
-                        uint32_t o[16];
                         if (SWIGLU) {
                             uint32_t g[32], u[32];
                             tc_ld32(taddr + pass * 64 + c, g);
                             tc_ld32(taddr + BN / 2 + pass * 64 + c, u);
                             tc_wait_ld();
 #pragma unroll
-                            for (int i = 0; i < 16; ++i) {
-                                float g0 = __uint_as_float(g[2 * i]), g1 = __uint_as_float(g[2 * i + 1]);
-                                float h0 = (g0 / (1.f + __expf(-g0))) * __uint_as_float(u[2 * i]);
-                                float h1 = (g1 / (1.f + __expf(-g1))) * __uint_as_float(u[2 * i + 1]);
-                                o[i] = pack_bf16(h0, h1);
-                            }
+                            for (int i = 0; i < 16; ++i)
+                                o[(c >> 1) + i] = pack_bf16(swiglu(__uint_as_float(g[2 * i]), __uint_as_float(u[2 * i])),
+                                                            swiglu(__uint_as_float(g[2 * i + 1]), __uint_as_float(u[2 * i + 1])));
                         } else {
                             uint32_t r[32];
                             tc_ld32(taddr + pass * 64 + c, r);
                             tc_wait_ld();
 #pragma unroll
-                            for (int i = 0; i < 16; ++i) o[i] = pack_bf16(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
+                            for (int i = 0; i < 16; ++i)
+                                o[(c >> 1) + i] = pack_bf16(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
                         }
-                        const uint32_t line = slab + lane * 128;     // 32 columns = 4 chunks of 16 bytes, index c/8 + v
-#pragma unroll
-                        for (int v = 0; v < 4; ++v)
-                            st_shared_v4(line + ((((c >> 3) + v) ^ (lane & 7)) << 4), o[4 * v], o[4 * v + 1], o[4 * v + 2], o[4 * v + 3]);
                     }
-                    if (pass == PASSES - 1) tc_fence_before();   // all TMEM reads of this accumulator are done
+                };
+                load_pass(0, nxt);
+#pragma unroll
+                for (int pass = 0; pass < PASSES; ++pass) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) cur[i] = nxt[i];
+                    if (pass + 1 < PASSES) {
+                        load_pass(pass + 1, nxt);
+                    }
+                    if (pass + 1 == PASSES - 1) {                 // the last TMEM read of this tile just happened
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(smem_u32(&ctrl->tempty[acc]));
+                    }
+                    if (lane == 0) tma_store_wait_read();     // the slab's previous store has been read out
+                    __syncwarp();
+                    const uint32_t line = slab + lane * 128;  // 64 columns = 8 chunks of 16 bytes
+#pragma unroll
+                    for (int v = 0; v < 8; ++v)
+                        st_shared_v4(line + ((v ^ (lane & 7)) << 4), cur[4 * v], cur[4 * v + 1], cur[4 * v + 2], cur[4 * v + 3]);
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     __syncwarp();
                     if (lane == 0) {
-                        if (pass == PASSES - 1) mbar_arrive(smem_u32(&ctrl->tempty[acc]));
                         const int col = c0 + pass * 64;
                         if (col < a.N) tma_store_2d(&tmapC, slab, col, row);
                         tma_store_commit();

@@ -281,7 +281,7 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap tmapW, const __grid_constant_
 #pragma unroll
                             for (int i = 0; i < 32; ++i) {
                                 const float gv = __uint_as_float(g[i]);
-                                const float hv = (gv / (1.f + __expf(-gv))) * __uint_as_float(u[i]);
+                                const float hv = swiglu(gv, __uint_as_float(u[i]));
                                 st_shared_b16(out_base + out_offset(c + i, f), bf16_bits(hv));
                             }
                         } else {

@@ -8,7 +8,7 @@
 namespace mok {
 
 static thread_local int g_last_cuda_error = 0;
-constexpr int M2_MIN_K = 1536;   // shortest K for which the 256-row-tile kernel is chosen by default
+constexpr int M2_MIN_K = 512;    // shortest K for which the 256-row-tile kernel is chosen by default
 
 static int cuda_fail(cudaError_t e) {
     g_last_cuda_error = (int)e;
@@ -120,14 +120,16 @@ static bool fused_gather(const mok_config* cfg, int I) {
 }
 
 // Rows of one tile of the padded row space: 256 when the GEMMs run on CTA pairs (cta_group::2), else 128.
-// Measured on B200: pairs are 5-19 % faster per k-block for GEMMs whose A operand comes through TMA, but slower for
-// the fused-gather GEMM (its odd CTA has to announce its gathered rows in software) and they double the padding of
-// every expert segment.  So by default pairs are used exactly when the gather is a separate kernel.
+// Measured on B200: pairs are 5-19 % faster per k-block than single 128-row tiles for GEMMs whose A operand comes
+// through TMA, but slower for the fused-gather GEMM (its odd CTA has to announce its gathered rows in software) and
+// they double the padding of every expert segment.  The 256-row tiles of ONE CTA (use_m2) get the same saving without
+// either drawback, so pairs are only used on request (cta_group = 2).
 static int tile_rows(const mok_config* cfg, int I) {
     if (use_simt(cfg) || use_tn(cfg)) return TILE_M;
     if (cfg && cfg->cta_group == 2) return 2 * TILE_M;
     if (cfg && cfg->cta_group == 1) return TILE_M;
-    return fused_gather(cfg, I) ? TILE_M : 2 * TILE_M;
+    (void)I;
+    return TILE_M;   // default: 128-row padding; the 256-row-tile kernel works on it through the second tile table
 }
 
 // 256-row tiles with two accumulators in one CTA (gemm_tcgen05_m2.cu): used on the 128-padded row space through the

@@ -163,6 +163,13 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr) {
     d |= (uint64_t)2 << 61;                           // 128-byte swizzle
     return d;
 }
+// silu(g) * u = g * u / (1 + exp(-g)) with two special-function instructions (ex2, rcp) and no IEEE division: the
+// epilogue warps share issue slots with the MMA issuer and the gather warps, and the result is rounded to bf16 anyway
+// (relative error of this form ~1e-6).  exp(-g) overflows to +inf for g < -88 and the quotient becomes -0: correct limit.
+__device__ __forceinline__ float swiglu(float g, float u) {
+    return __fdividef(g * u, 1.f + __expf(-g));
+}
+
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
