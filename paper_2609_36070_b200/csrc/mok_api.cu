@@ -135,16 +135,19 @@ static int tile_rows(const mok_config* cfg, int I) {
 // 256-row tiles with two accumulators in one CTA (gemm_tcgen05_m2.cu): used on the 128-padded row space through the
 // second tile table.  cta_group = 3 forces it; by default it serves GEMMs whose K is long enough to amortise the
 // accumulator hand-over between tiles.
-static bool use_m2(const mok_config* cfg, int K, int tile_m) {
+static bool use_m2(const mok_config* cfg, int K, int tile_m, long long rows, int experts) {
     if (use_simt(cfg) || use_tn(cfg) || tile_m != TILE_M) return false;
     if (cfg && cfg->cta_group == 3) return true;
     if (cfg && cfg->cta_group != 0) return false;
-    return K >= M2_MIN_K;
+    // With few rows per expert nearly every tile has one half only and the layer is bound by streaming the weights
+    // once: there the 128-row kernel, whose four stages are all weight and activation bytes, is the faster one
+    // (measured on the DeepSeek-like shape: 3.39 vs 3.62 ms at 2 rows per expert, 5.58 vs 5.31 ms at 128).
+    return K >= M2_MIN_K && rows >= 96ll * experts;
 }
 
 static int run_gemm(GemmArgs g, bool swiglu, const mok_config* cfg, const WsLayout& L, char* ws, cudaStream_t s) {
     const int epi = swiglu ? EPI_SWIGLU : EPI_BF16, grid = cfg ? cfg->grid : 0;
-    if (use_m2(cfg, g.K, g.tile_m)) {
+    if (use_m2(cfg, g.K, g.tile_m, g.dense_rows > 0 ? g.dense_rows : g.total_rows, g.dense_rows > 0 ? 1 : g.E)) {
         WsHeader* hdr = reinterpret_cast<WsHeader*>(ws + L.header);
         g.n_mtiles = &hdr->n_mtiles2;
         g.mt_start = reinterpret_cast<const int32_t*>(ws + L.mt_start2);
@@ -167,7 +170,7 @@ static int route_stage(const mok_args* a, const WsLayout& L, char* ws, const __n
         e = launch_router_tc(x, a->W_router, a->router_bias, a->T, a->H, a->E, a->k, L, ws,
                              reinterpret_cast<WsHeader*>(ws + L.header), a->config ? a->config->grid : 0,
                              tile_rows(a->config, a->I > 0 ? a->I : 8),
-                             use_tn(a->config) ? 2 : use_m2(a->config, a->H, tile_rows(a->config, a->I > 0 ? a->I : 8)) ? 3 : 0,
+                             use_tn(a->config) ? 2 : use_m2(a->config, a->H, tile_rows(a->config, a->I > 0 ? a->I : 8), a->T, 1) ? 3 : 0,
                              idx, w, s);
     if (e != cudaSuccess) return cuda_fail(e);
     if (a->topk_idx) {
@@ -239,6 +242,7 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
     g.B = reinterpret_cast<const __nv_bfloat16*>(a->W_gate_up);
     g.C = ws + L.h;
     g.K = a->H; g.N = a->I; g.ldc = a->I; g.E = a->E; g.rows_pad = L.Rpad; g.dense_rows = 0;
+    g.total_rows = L.R;
     if ((rc = run_gemm(g, true, a->config, L, ws, s))) return rc;
     g.row_token = nullptr;
     g.starve = 0;

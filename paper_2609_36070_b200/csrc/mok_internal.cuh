@@ -62,6 +62,7 @@ struct GemmArgs {
     int32_t rows_pad;            // allocated rows of C (multiple of 128)
     int32_t a_rows;              // allocated rows of A (reads beyond it are treated as zero)
     int32_t dense_rows;          // > 0: dense mode with this many valid rows
+    int32_t total_rows;          // routed mode: T*k (host-side hint for choosing the kernel; not read on the device)
     const int32_t* n_mtiles;     // device (routed mode)
     const int32_t* tile_expert;  // device [max_mt]
     const int32_t* mt_start;     // device [E+1]
