@@ -26,7 +26,7 @@ UNIT = "tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # dram bytes (read + write) of one launch of the dominant kernel from the committed ncu capture, keyed by config
 # (None until a capture exists for that workload; see profiles/).
-NCU_TRAFFIC_BYTES = {"qwen3_30b_a3b": 1.409e9}   # profiles/gemm_tc_kernel_qwen3_30b_a3b.md: 1.195 GB read + 0.214 GB written
+NCU_TRAFFIC_BYTES = {"qwen3_30b_a3b": 1.413e9}   # profiles/gemm_kernels_qwen3_30b_a3b.md: 1.183 GB read + 0.230 GB written
 
 
 def parse():
@@ -270,7 +270,7 @@ def main():
                       "frac_of_bf16_peak": flops / (ffn_ms * 1e-3) / 1e12 / pk["bf16_tflops"],
                       "frac_of_bf16_sustained": flops / (ffn_ms * 1e-3) / 1e12 / peak_tf},
         "stage_ms": mean,
-        "roofline": {"kernel": "gemm_tc_kernel<EPI_SWIGLU> (routed gate/up grouped GEMM + SwiGLU, token gather fused)",
+        "roofline": {"kernel": "routed gate/up grouped GEMM + SwiGLU, token gather fused (gemm_m2_kernel<EPI_SWIGLU, GATHER>)",
                      "bound": "tensor",
                      "achieved": g1_tflops, "peak": peak_tf, "unit": "TFLOP/s", "frac": g1_tflops / peak_tf,
                      "peak_source": f"{pk['source']} bf16_tflops_sustained",
