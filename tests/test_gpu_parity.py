@@ -43,6 +43,24 @@ def test_small_shapes_every_token(cfg, impl):
     print(cfg.name, impl, rep)
 
 
+EDGE = [
+    MoEConfig("min_dims", T=70, H=8, E=4, k=2, I=8, I_s=8, seed=41),                      # smallest legal H, I
+    MoEConfig("max_experts", T=300, H=64, E=512, k=6, I=64, I_s=0, bias="normal", seed=42),  # E at the limit, most experts empty
+    MoEConfig("k28", T=64, H=128, E=64, k=28, I=64, I_s=0, seed=43),                      # largest k of the tensor-core router
+    MoEConfig("k32", T=64, H=128, E=40, k=32, I=64, I_s=0, seed=44),                      # k > 28: fp32-FMA router takes over
+    MoEConfig("two_halves_exact", T=256, H=192, E=2, k=2, I=192, I_s=0, seed=45),         # every expert owns exactly 256 rows
+    MoEConfig("big_shared", T=513, H=128, E=4, k=1, I=64, I_s=640, seed=46),              # shared expert wider than routed
+]
+
+
+@pytest.mark.parametrize("cfg", EDGE, ids=[c.name for c in EDGE])
+@pytest.mark.parametrize("cta_group", [0, 3])
+def test_edge_shapes_every_token(cfg, cta_group):
+    m = mok()
+    out, st, rep = pu.full_parity(cfg, config=m._config(cta_group=cta_group))
+    print(cfg.name, cta_group, rep)
+
+
 def test_all_routes_to_one_expert():
     """Degenerate dispatch: a huge bias sends every token's first route to expert 3; other experts get the rest."""
     cfg = MoEConfig("hot", T=400, H=128, E=8, k=2, I=128, I_s=0, seed=21)
