@@ -114,9 +114,9 @@ def cpu_oracle_rate(cfg, d, sample):
 
 
 def auto_sample(cfg, cores):
-    # aim at ~15 s of CPU work assuming ~1.2 fp64 GFLOP/s per core for the scalar oracle
+    # aim at ~15 s of CPU work; the scalar oracle sustains about 4 fp64 GFLOP/s per core on the GPU hosts
     per_token = 6.0 * cfg.H * (cfg.k * cfg.I + cfg.I_s)
-    n = int(15.0 * 1.2e9 * cores / per_token)
+    n = int(15.0 * 4.0e9 * cores / per_token)
     return max(16, min(cfg.T, n))
 
 
