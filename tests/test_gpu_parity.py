@@ -189,3 +189,28 @@ def test_bounded_waits_report_a_timeout_and_leave_the_context_usable():
     assert m.mok_read_status(ws) == m.MOK_ERR_TIMEOUT
     again = pu.run_gpu(cfg, g, ws=ws, stages=False)
     assert torch.equal(good.view(torch.int16), again.view(torch.int16))
+
+
+def test_forward_can_be_captured_in_a_cuda_graph_and_replayed():
+    """The layer makes no host synchronisation and no allocation after its first call for a shape, so a whole
+    forward can be recorded once into a CUDA graph and replayed (launch-bound small batches): same bits."""
+    m = mok()
+    cfg = inputs.CONFIGS["tiny"]
+    d = inputs.make_inputs(cfg)
+    g = pu.upload(d)
+    ws = m.alloc_workspace(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k)
+    out = torch.empty_like(g["x"])
+    args = (g["x"], g["W_r"], g["bias"], g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], cfg.k, ws)
+    m.mok_moe_forward_ex(*args, out=out)                       # first call: one-time kernel attribute set-up
+    torch.cuda.synchronize()
+    want = out.clone()
+    graph = torch.cuda.CUDAGraph()
+    out.zero_()
+    with torch.cuda.graph(graph):
+        m.mok_moe_forward_ex(*args, out=out)
+    for _ in range(3):
+        out.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(out.view(torch.int16), want.view(torch.int16))
+    assert m.mok_read_status(ws) == 0
