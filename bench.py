@@ -113,6 +113,21 @@ def cpu_oracle_rate(cfg, d, sample):
     return len(tokens) / t, t_ffn + t_route, mok_ref.num_threads()
 
 
+def fingerprints(d, limit=1 << 31):
+    """SHA-256 of each input tensor as generated (tensors above `limit` bytes: of their first `limit` bytes)."""
+    import hashlib
+    import numpy as np
+    out = {"numpy": np.__version__}
+    for name in ("x", "W_r", "bias", "W_gate_up", "W_down", "W_sgu", "W_sd"):
+        a = d.get(name)
+        if a is None:
+            continue
+        raw = memoryview(np.ascontiguousarray(a)).cast("B")
+        part = raw[:limit]
+        out[name] = hashlib.sha256(part).hexdigest()[:16] + ("" if len(raw) <= limit else f" (first {limit} bytes)")
+    return out
+
+
 def auto_sample(cfg, cores):
     # aim at ~15 s of CPU work; the scalar oracle sustains about 4 fp64 GFLOP/s per core on the GPU hosts
     per_token = 6.0 * cfg.H * (cfg.k * cfg.I + cfg.I_s)
@@ -256,6 +271,7 @@ def main():
     g1_flops = 4.0 * cfg.T * cfg.k * cfg.H * cfg.I
     g1_tflops = g1_flops / (mean["gemm1"] * 1e-3) / 1e12
     peak_tf = pk.get("bf16_tflops_sustained", pk["bf16_tflops"])
+    per_step = sorted(sum(c[s] for s in mok.STAGES) for c in stage)
     ffn_ms = mean["gemm1"] + mean["gemm2"] + mean["shared_gemm1"] + mean["shared_gemm2"]
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -270,6 +286,8 @@ def main():
                       "frac_of_bf16_peak": flops / (ffn_ms * 1e-3) / 1e12 / pk["bf16_tflops"],
                       "frac_of_bf16_sustained": flops / (ffn_ms * 1e-3) / 1e12 / peak_tf},
         "stage_ms": mean,
+        "median_step_ms_from_stage_events": per_step[len(per_step) // 2],
+        "inputs": fingerprints(d),
         "roofline": {"kernel": "routed gate/up grouped GEMM + SwiGLU, token gather fused (gemm_m2_kernel<EPI_SWIGLU, GATHER>)",
                      "bound": "tensor",
                      "achieved": g1_tflops, "peak": peak_tf, "unit": "TFLOP/s", "frac": g1_tflops / peak_tf,

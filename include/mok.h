@@ -170,6 +170,73 @@ int mok_schedule_noalloc(const int32_t* topk_idx, int T, int E, int k,
                          int32_t* counts, int32_t* offsets, int32_t* perm, int32_t* inv_perm, void* stream);
 
 /*
+ * Expert parallelism over n_ranks GPUs of one NVLink domain (Sections 2.1 and 3.1-3.3; Algorithm 1 with R source
+ * ranks).  Rank c holds the L = E / n_ranks experts [cL, (c+1)L) and T_local tokens.  One layer is, on every rank:
+ *   1. mok_route on the rank's own tokens                                  -> topk_idx, topk_w      (local)
+ *   2. an all-gather of topk_idx over the ranks (the caller's collective; "all-gather of top-k routes")
+ *   3. mok_ep_expert_ffn: Algorithm 1 for this rank from the gathered routes (M, S, Phi; no host readback), then
+ *      the routed gate/up GEMM whose gather warps PULL each scheduled row straight from its source rank's token
+ *      buffer x_peers[src_rank] into shared memory ("pull dispatch": plain 16-byte asynchronous copies over NVLink,
+ *      never a multicast load), SwiGLU, and the down GEMM, which leaves this rank's expert outputs in y in schedule
+ *      order; pos tells every token owner where its routes' rows sit in this rank's y
+ *   4. a barrier over the ranks (the caller's; every rank's y and pos must be complete before any rank combines)
+ *   5. mok_ep_combine: each token owner reads its k rows from the serving ranks' y buffers and reduces them, with the
+ *      shared expert's output, in slot order in fp32 -- fixed order, no atomics, bitwise reproducible (Section 3.4).
+ *      The paper has the expert's rank push rows into a buffer of the owner, which the owner then reduces; here the
+ *      owner pulls the same rows, so each row still crosses NVLink once and the only cross-rank signal is step 4.
+ * x_peers / y_peers / pos_peers hold device pointers valid in the calling process: the rank's own buffers and the
+ * peers' buffers mapped into it (symmetric memory or IPC handles; the caller's plumbing).  On one GPU the same entry
+ * points serve any number of emulated ranks, since a local pointer is a valid peer pointer.
+ * Limits: n_ranks <= MOK_MAX_RANKS, E a multiple of n_ranks, and the sizes of mok_moe_forward_ex with
+ * T = n_ranks * T_local.  The dispatch buffers are sized for the worst case (every route of every rank served by this
+ * rank): mok_ep_y_rows rows.
+ */
+#define MOK_MAX_RANKS 16
+typedef struct mok_ep_args {
+    int32_t rank, n_ranks;
+    int32_t T_local, H, I, I_shared, E, k;
+    const void* x_peers[MOK_MAX_RANKS];  /* bf16 [T_local, H] of every rank; x_peers[rank] is this rank's own */
+    const int32_t* idx_all;              /* int32 [n_ranks, T_local*k]: gathered top-k expert ids, rank-major */
+    const void* W_gate_up;               /* bf16 [L, 2I, H]: this rank's experts */
+    const void* W_down;                  /* bf16 [L, H, I] */
+    const void* W_shared_gate_up;        /* bf16 [2*I_shared, H] or NULL: shared expert, run on the rank's own tokens */
+    const void* W_shared_down;           /* bf16 [H, I_shared] or NULL */
+    void* y;                             /* out: bf16 [y_rows, H] expert outputs in schedule order (peers read it) */
+    int64_t y_rows;                      /* rows allocated for y: at least mok_ep_y_rows(...) */
+    int32_t* pos;                        /* out: int32 [n_ranks*T_local*k]: row of y of every route this rank serves;
+                                            entries of routes served elsewhere are left untouched (peers read it) */
+    void* y_shared;                      /* out: bf16 [T_local rounded up to a multiple of 256, H]: the shared expert's
+                                            output for the rank's own tokens; required when I_shared > 0 */
+    void* workspace;                     /* mok_ep_workspace_bytes(...) bytes, 256-byte aligned */
+    size_t workspace_bytes;
+    /* optional outputs of Algorithm 1 (any may be NULL) */
+    int32_t* M;                          /* int32 [n_ranks, L]: routes from source rank r to local expert l */
+    int32_t* S;                          /* int32 [L+1]: exclusive prefix sums of the per-expert totals */
+    int32_t* phi_rank;                   /* int32 [n_ranks*T_local*k]: source rank of schedule row p < S[L] */
+    int32_t* phi_index;                  /* int32 [n_ranks*T_local*k]: source route index (token*k + slot) of row p */
+    int32_t schedule_only;               /* non-zero: stop after Algorithm 1 (y untouched; pos and the outputs written) */
+    const mok_config* config;            /* grid, cta_group 0/1/3, debug; impl must be MOK_IMPL_TCGEN05 */
+    void* stream;
+} mok_ep_args;
+
+typedef struct mok_ep_combine_args {
+    int32_t rank, n_ranks;
+    int32_t T_local, H, E, k;
+    const int32_t* topk_idx;             /* int32 [T_local, k]: this rank's routes */
+    const float* topk_w;                 /* fp32 [T_local, k] */
+    const void* y_peers[MOK_MAX_RANKS];  /* every rank's y */
+    const int32_t* pos_peers[MOK_MAX_RANKS]; /* every rank's pos */
+    const void* y_shared;                /* this rank's y_shared from mok_ep_expert_ffn, or NULL: no shared term */
+    void* out;                           /* bf16 [T_local, H] */
+    void* stream;
+} mok_ep_combine_args;
+
+size_t mok_ep_workspace_bytes(int n_ranks, int T_local, int H, int I, int I_shared, int E, int k);
+long long mok_ep_y_rows(int n_ranks, int T_local, int E, int k);
+int mok_ep_expert_ffn(const mok_ep_args* args);
+int mok_ep_combine(const mok_ep_combine_args* args);
+
+/*
  * Reads the device-side status word of a workspace after synchronising `stream` -- the only call besides
  * mok_moe_forward_host that blocks the host.  Returns MOK_OK, MOK_ERR_TIMEOUT or MOK_ERR_SCHEDULE
  * (or MOK_ERR_CUDA if the stream itself is in error).

@@ -98,7 +98,7 @@ __device__ __forceinline__ Tile decode_tile(const GemmArgs& a, int L, int n_nt, 
 template <int EPI, bool GATHER, int CTAS>
 __global__ void __launch_bounds__(THREADS + (GATHER ? GATHER_THREADS : 0), 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
-               const __grid_constant__ CUtensorMap tmapC, const GemmArgs a, const int n_nt, const int k_blocks) {
+               const __grid_constant__ CUtensorMap tmapC, const __grid_constant__ GemmArgs a, const int n_nt, const int k_blocks) {
     constexpr bool SWIGLU = (EPI == EPI_SWIGLU);
     constexpr int STAGES = (CTAS == 2) ? 6 : 4;
     constexpr int B_STAGE = B_BYTES / CTAS;                 // B bytes this CTA stages per k-block
@@ -272,7 +272,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
             for (int i = 0; i < 8; ++i) {
                 const int r = gw * 32 + i * 4 + sub;
                 const int tok = (r < valid) ? __ldg(rows + r) : tok0;
-                src[i] = a.A + (size_t)tok * a.K + chunk * 8;
+                src[i] = gather_row(a, tok) + chunk * 8;
             }
             bool ok = true;
             for (int kb = 0; kb < k_blocks; ++kb) {

@@ -79,7 +79,7 @@ __device__ __forceinline__ Tile decode_tile(const GemmArgs& a, int L, int n_nt, 
 template <int EPI, bool GATHER>
 __global__ void __launch_bounds__(THREADS + (GATHER ? GATHER_THREADS : 0), 1)
 gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
-               const __grid_constant__ CUtensorMap tmapC, const GemmArgs a, const int n_nt, const int k_blocks) {
+               const __grid_constant__ CUtensorMap tmapC, const __grid_constant__ GemmArgs a, const int n_nt, const int k_blocks) {
     constexpr bool SWIGLU = (EPI == EPI_SWIGLU);
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -215,7 +215,7 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
             for (int i = 0; i < 16; ++i) {
                 const int r = (i >> 3) * BM + gw * 32 + (i & 7) * 4 + sub;
                 const int tok = (r < t.valid) ? __ldg(a.row_token + t.row0 + r) : tok0;
-                src[i] = a.A + (size_t)tok * a.K + chunk * 8;
+                src[i] = gather_row(a, tok) + chunk * 8;
             }
             bool ok = true;
             for (int kb = 0; kb < k_blocks; ++kb) {

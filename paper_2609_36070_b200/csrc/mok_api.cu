@@ -10,7 +10,7 @@ namespace mok {
 static thread_local int g_last_cuda_error = 0;
 constexpr int M2_MIN_K = 512;    // shortest K for which the 256-row-tile kernel is chosen by default
 
-static int cuda_fail(cudaError_t e) {
+int cuda_fail(cudaError_t e) {
     g_last_cuda_error = (int)e;
     return MOK_ERR_CUDA;
 }
@@ -111,7 +111,7 @@ static bool use_simt_router(const mok_config* cfg, int k) {
 // Whether the routed gate/up GEMM gathers its rows itself.  The fused path re-gathers the rows once per N tile
 // through the load/store units; the separate kernel writes the expert-sorted copy once and the GEMM then uses
 // plain TMA tile loads.  Measured on B200: fused wins at 6, 16 and 23 N tiles (ceil(I / 128)), loses at 112.
-static bool fused_gather(const mok_config* cfg, int I) {
+bool fused_gather(const mok_config* cfg, int I) {
     if (use_simt(cfg)) return false;
     if (use_tn(cfg)) return true;
     if (cfg && cfg->gather_mode == 1) return true;
@@ -124,7 +124,7 @@ static bool fused_gather(const mok_config* cfg, int I) {
 // through TMA, but slower for the fused-gather GEMM (its odd CTA has to announce its gathered rows in software) and
 // they double the padding of every expert segment.  The 256-row tiles of ONE CTA (use_m2) get the same saving without
 // either drawback, so pairs are only used on request (cta_group = 2).
-static int tile_rows(const mok_config* cfg, int I) {
+int tile_rows(const mok_config* cfg, int I) {
     if (use_simt(cfg) || use_tn(cfg)) return TILE_M;
     if (cfg && cfg->cta_group == 2) return 2 * TILE_M;
     if (cfg && cfg->cta_group == 1) return TILE_M;
@@ -145,7 +145,7 @@ static bool use_m2(const mok_config* cfg, int K, int tile_m, long long rows, int
     return K >= M2_MIN_K && rows >= 96ll * experts;
 }
 
-static int run_gemm(GemmArgs g, bool swiglu, const mok_config* cfg, const WsLayout& L, char* ws, cudaStream_t s) {
+int run_gemm(GemmArgs g, bool swiglu, const mok_config* cfg, const WsLayout& L, char* ws, cudaStream_t s) {
     const int epi = swiglu ? EPI_SWIGLU : EPI_BF16, grid = cfg ? cfg->grid : 0;
     if (use_m2(cfg, g.K, g.tile_m, g.dense_rows > 0 ? g.dense_rows : g.total_rows, g.dense_rows > 0 ? 1 : g.E)) {
         WsHeader* hdr = reinterpret_cast<WsHeader*>(ws + L.header);

@@ -71,7 +71,21 @@ struct GemmArgs {
     int32_t dbg_slot;            // >= 0: accumulate wait-time counters into header->dbg[dbg_slot]
     int32_t starve;              // test hook: the TMA producer issues nothing, so the kernel's waits run out
     WsHeader* header;
+    // Expert-parallel pull dispatch (Section 3.1): with peer_tokens > 0 the ids in row_token are global,
+    // id = source_rank * peer_tokens + token, and row `id` is read from peer_x[source_rank] (this GPU's own tokens
+    // or a peer's, mapped into this process) with plain 16-byte asynchronous copies -- never a multicast load.
+    int32_t peer_tokens;
+    const __nv_bfloat16* peer_x[MOK_MAX_RANKS];
 };
+
+// Source row of the fused gather: row `tok` of A, or of the owning rank's token buffer in expert-parallel mode.
+__device__ __forceinline__ const __nv_bfloat16* gather_row(const GemmArgs& a, int tok) {
+    if (a.peer_tokens > 0) {
+        const int r = tok / a.peer_tokens;
+        return a.peer_x[r] + (size_t)(tok - r * a.peer_tokens) * a.K;
+    }
+    return a.A + (size_t)tok * a.K;
+}
 
 // kernels' host launchers (each returns a cudaError_t from the launch)
 cudaError_t launch_router_simt(const __nv_bfloat16* x, const float* Wr, const float* bias, int T, int H, int E, int k,
@@ -82,6 +96,13 @@ cudaError_t launch_schedule(const int32_t* idx, int T, int E, int k, int tile_m,
 cudaError_t launch_gather(const __nv_bfloat16* x, int H, int k, int tile_m, const WsLayout& L, char* ws, cudaStream_t s);
 cudaError_t launch_combine(const WsLayout& L, char* ws, int T, int H, int k, bool shared, __nv_bfloat16* out,
                            cudaStream_t s);
+cudaError_t launch_ep_schedule(const int32_t* idx_all, int n_ranks, int rank, int routes_per_rank, int k, int tokens_per_rank,
+                               int experts_local, int tile_m, const WsLayout& L, char* ws, int32_t* pos_out, int32_t* M_out,
+                               int32_t* S_out, int32_t* phi_rank_out, int32_t* phi_index_out, cudaStream_t s);
+int run_gemm(GemmArgs g, bool swiglu, const mok_config* cfg, const WsLayout& L, char* ws, cudaStream_t s);
+int tile_rows(const mok_config* cfg, int I);
+bool fused_gather(const mok_config* cfg, int I);
+int cuda_fail(cudaError_t e);
 cudaError_t launch_gemm_simt(const GemmArgs& a, bool swiglu, cudaStream_t s);
 enum { EPI_BF16 = 0, EPI_SWIGLU = 1, EPI_F32 = 2 };
 cudaError_t launch_gemm_tc(const GemmArgs& a, int epi, int grid, cudaStream_t s);

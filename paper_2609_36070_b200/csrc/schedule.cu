@@ -13,12 +13,9 @@
 //                    row_token (padded row -> source token: the {src_index} column of the paper's schedule table)
 // Exported offsets/perm are unpadded; the padding is internal to the GEMM row space.
 #include "mok_internal.cuh"
+#include "schedule_common.cuh"
 
 namespace mok {
-
-constexpr int SCHED_THREADS = 256;
-constexpr int SCHED_WARPS = SCHED_THREADS / 32;
-constexpr int ROUTES_PER_WARP = SCHED_CHUNK / SCHED_WARPS;   // contiguous routes owned by one warp
 
 __global__ void __launch_bounds__(SCHED_THREADS)
 sched_hist_kernel(const int32_t* __restrict__ a, int n, int E, int32_t* __restrict__ blk_hist) {
@@ -59,45 +56,8 @@ sched_scan_kernel(int32_t* __restrict__ blk_hist, int n_blk, int E, int max_mt, 
         s_cnt[e] = total;
     }
     __syncthreads();
-    if (e == 0) {   // E <= 512: a serial scan by one thread is a few hundred cycles
-        int32_t off = 0, mt = 0, pad = 0, mt2 = 0;
-        for (int i = 0; i < E; ++i) {
-            s_off[i] = off;
-            s_mt[i] = mt;
-            s_mt2[i] = mt2;
-            s_pad[i] = pad;
-            off += s_cnt[i];
-            mt += (s_cnt[i] + tile_m - 1) / tile_m;
-            mt2 += (s_cnt[i] + 2 * tile_m - 1) / (2 * tile_m);
-            pad += (s_cnt[i] + pad_m - 1) / pad_m * pad_m;
-        }
-        s_off[E] = off;
-        s_mt[E] = mt;
-        s_pad[E] = pad;
-        s_mt2[E] = mt2;
-        hdr->n_mtiles = mt;
-        hdr->n_mtiles2 = mt2;
-        if (mt * (tile_m / TILE_M) > max_mt) hdr->status = MOK_ERR_SCHEDULE;
-    }
-    __syncthreads();
-    if (e < E) {
-        counts[e] = s_cnt[e];
-        offsets[e] = s_off[e];
-        pad_offsets[e] = s_pad[e];
-        mt_start[e] = s_mt[e];
-        if (counts_out) counts_out[e] = s_cnt[e];
-        if (offsets_out) offsets_out[e] = s_off[e];
-        for (int q = s_mt[e]; q < s_mt[e + 1] && q < max_mt; ++q) tile_expert[q] = e;
-        mt_start2[e] = s_mt2[e];
-        for (int q = s_mt2[e]; q < s_mt2[e + 1] && q < max_mt; ++q) tile_expert2[q] = e;
-    }
-    if (e == 0) {
-        offsets[E] = s_off[E];
-        pad_offsets[E] = s_pad[E];
-        mt_start[E] = s_mt[E];
-        mt_start2[E] = s_mt2[E];
-        if (offsets_out) offsets_out[E] = s_off[E];
-    }
+    scan_tables(s_cnt, s_off, s_mt, s_pad, s_mt2, E, max_mt, tile_m, pad_m, counts, offsets, pad_offsets, mt_start,
+                tile_expert, mt_start2, tile_expert2, hdr, counts_out, offsets_out);
 }
 
 __global__ void __launch_bounds__(SCHED_THREADS)

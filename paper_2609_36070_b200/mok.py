@@ -21,7 +21,9 @@ MOK_IMPL_TCGEN05, MOK_IMPL_SIMT, MOK_IMPL_TCGEN05_TN = 0, 1, 2
 
 EXPORTS = ["mok_moe_forward", "mok_workspace_bytes", "mok_moe_forward_ex", "mok_moe_forward_host", "mok_route",
            "mok_schedule", "mok_read_status", "mok_launch_count", "mok_last_cuda_error", "mok_status_string",
-           "mok_version", "mok_profile_begin", "mok_profile_end", "mok_schedule_noalloc", "mok_debug_counters"]
+           "mok_version", "mok_profile_begin", "mok_profile_end", "mok_schedule_noalloc", "mok_debug_counters",
+           "mok_ep_workspace_bytes", "mok_ep_y_rows", "mok_ep_expert_ffn", "mok_ep_combine"]
+MOK_MAX_RANKS = 16
 MOK_NOALLOC_MAX_ROUTES = 32768
 MOK_DEBUG_STARVE = 2
 STAGES = ["router", "schedule", "gather", "gemm1", "gemm2", "shared_gemm1", "shared_gemm2", "combine"]
@@ -45,6 +47,37 @@ class mok_args(ctypes.Structure):
                 ("config", ctypes.POINTER(mok_config)), ("stream", ctypes.c_void_p)]
 
 
+class mok_ep_args(ctypes.Structure):
+    _fields_ = [("rank", ctypes.c_int32), ("n_ranks", ctypes.c_int32),
+                ("T_local", ctypes.c_int32), ("H", ctypes.c_int32), ("I", ctypes.c_int32), ("I_shared", ctypes.c_int32),
+                ("E", ctypes.c_int32), ("k", ctypes.c_int32),
+                ("x_peers", ctypes.c_void_p * MOK_MAX_RANKS), ("idx_all", ctypes.c_void_p),
+                ("W_gate_up", ctypes.c_void_p), ("W_down", ctypes.c_void_p),
+                ("W_shared_gate_up", ctypes.c_void_p), ("W_shared_down", ctypes.c_void_p),
+                ("y", ctypes.c_void_p), ("y_rows", ctypes.c_int64), ("pos", ctypes.c_void_p),
+                ("y_shared", ctypes.c_void_p),
+                ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
+                ("M", ctypes.c_void_p), ("S", ctypes.c_void_p), ("phi_rank", ctypes.c_void_p),
+                ("phi_index", ctypes.c_void_p), ("schedule_only", ctypes.c_int32),
+                ("config", ctypes.POINTER(mok_config)), ("stream", ctypes.c_void_p)]
+
+
+class mok_ep_combine_args(ctypes.Structure):
+    _fields_ = [("rank", ctypes.c_int32), ("n_ranks", ctypes.c_int32),
+                ("T_local", ctypes.c_int32), ("H", ctypes.c_int32), ("E", ctypes.c_int32), ("k", ctypes.c_int32),
+                ("topk_idx", ctypes.c_void_p), ("topk_w", ctypes.c_void_p),
+                ("y_peers", ctypes.c_void_p * MOK_MAX_RANKS), ("pos_peers", ctypes.c_void_p * MOK_MAX_RANKS),
+                ("y_shared", ctypes.c_void_p), ("out", ctypes.c_void_p), ("stream", ctypes.c_void_p)]
+
+
+_lib.mok_ep_workspace_bytes.restype = ctypes.c_size_t
+_lib.mok_ep_workspace_bytes.argtypes = [ctypes.c_int] * 7
+_lib.mok_ep_y_rows.restype = ctypes.c_longlong
+_lib.mok_ep_y_rows.argtypes = [ctypes.c_int] * 4
+_lib.mok_ep_expert_ffn.restype = ctypes.c_int
+_lib.mok_ep_expert_ffn.argtypes = [ctypes.POINTER(mok_ep_args)]
+_lib.mok_ep_combine.restype = ctypes.c_int
+_lib.mok_ep_combine.argtypes = [ctypes.POINTER(mok_ep_combine_args)]
 _lib.mok_workspace_bytes.restype = ctypes.c_size_t
 _lib.mok_workspace_bytes.argtypes = [ctypes.c_int] * 6
 _lib.mok_moe_forward.restype = ctypes.c_int
@@ -262,6 +295,68 @@ def mok_schedule_noalloc(topk_idx, E, stream=None):
     _check(_lib.mok_schedule_noalloc(_p(topk_idx), T, E, k, _p(counts), _p(offsets), _p(perm), _p(inv),
                                      _stream(stream)))
     return counts, offsets, perm, inv
+
+
+def mok_ep_workspace_bytes(n_ranks, T_local, H, I, I_shared, E, k):
+    return int(_lib.mok_ep_workspace_bytes(n_ranks, T_local, H, I, I_shared, E, k))
+
+
+def mok_ep_y_rows(n_ranks, T_local, E, k):
+    return int(_lib.mok_ep_y_rows(n_ranks, T_local, E, k))
+
+
+def mok_ep_expert_ffn(rank, x_peer_ptrs, idx_all, W_gate_up, W_down, W_shared_gate_up, W_shared_down, E, k, y, pos,
+                      y_shared, workspace, H, schedule_only=False, outputs=False, config=None, stream=None):
+    """Algorithm 1 for `rank` from the gathered routes idx_all [n_ranks, T_local*k], then this rank's expert FFNs with
+    the rows pulled from x_peer_ptrs (device addresses, one per rank).  Fills y, pos (and y_shared).  With
+    outputs=True also returns Algorithm 1's tables {M, S, phi_rank, phi_index}."""
+    n_ranks, n = idx_all.shape
+    T_local = n // k
+    a = mok_ep_args()
+    a.rank, a.n_ranks, a.T_local, a.H, a.E, a.k = rank, n_ranks, T_local, H, E, k
+    a.I = 8 if W_gate_up is None else W_gate_up.shape[1] // 2
+    a.I_shared = 0 if W_shared_gate_up is None else W_shared_gate_up.shape[0] // 2
+    for r, ptr in enumerate(x_peer_ptrs or []):
+        a.x_peers[r] = ptr
+    a.idx_all = idx_all.data_ptr()
+    for name, t in (("W_gate_up", W_gate_up), ("W_down", W_down), ("W_shared_gate_up", W_shared_gate_up),
+                    ("W_shared_down", W_shared_down), ("y", y), ("pos", pos), ("y_shared", y_shared)):
+        setattr(a, name, None if t is None else t.data_ptr())
+    a.y_rows = 0 if y is None else y.shape[0]
+    a.workspace, a.workspace_bytes = _aligned_ws(workspace)
+    res = {}
+    if outputs:
+        L = E // n_ranks
+        dev = idx_all.device
+        res = {"M": torch.empty((n_ranks, L), dtype=torch.int32, device=dev),
+               "S": torch.empty((L + 1,), dtype=torch.int32, device=dev),
+               "phi_rank": torch.full((n_ranks * n,), -1, dtype=torch.int32, device=dev),
+               "phi_index": torch.full((n_ranks * n,), -1, dtype=torch.int32, device=dev)}
+        for name, t in res.items():
+            setattr(a, name, t.data_ptr())
+    a.schedule_only = int(schedule_only)
+    if config is not None:
+        a.config = ctypes.pointer(config)
+    a.stream = _stream(stream).value
+    _check(_lib.mok_ep_expert_ffn(ctypes.byref(a)))
+    return res
+
+
+def mok_ep_combine(rank, n_ranks, topk_idx, topk_w, y_peer_ptrs, pos_peer_ptrs, y_shared, E, out, stream=None):
+    """Owner-side deterministic combine: out[t] = y_shared[t] + sum_s w[t,s] * (row of the serving rank's y)."""
+    a = mok_ep_combine_args()
+    a.rank, a.n_ranks = rank, n_ranks
+    a.T_local, a.k = topk_idx.shape
+    a.H, a.E = out.shape[1], E
+    a.topk_idx, a.topk_w = topk_idx.data_ptr(), topk_w.data_ptr()
+    for r in range(n_ranks):
+        a.y_peers[r] = y_peer_ptrs[r]
+        a.pos_peers[r] = pos_peer_ptrs[r]
+    a.y_shared = None if y_shared is None else y_shared.data_ptr()
+    a.out = out.data_ptr()
+    a.stream = _stream(stream).value
+    _check(_lib.mok_ep_combine(ctypes.byref(a)))
+    return out
 
 
 DEBUG_COUNTERS = ["mma_wait_operands", "mma_wait_peer_operands", "mma_wait_accumulator", "mma_total", "k_blocks",

@@ -1,0 +1,144 @@
+"""Expert parallelism on one GPU with emulated ranks: the device-side Algorithm 1 for R source ranks against the
+oracle's statement-by-statement version (bit-exact), and the whole expert-parallel layer (local routing, gathered
+routes, schedule, pull dispatch into the grouped GEMMs, owner-side combine) against the oracle's per-token
+definition and against the one-rank layer on the concatenated batch.  Every rank's buffers live on the same GPU, so a
+local pointer stands in for a peer pointer; kernels and schedules are exactly those of the multi-GPU path."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import mok_ref
+from paper_2609_36070_b200 import inputs
+from tests import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+
+def mok():
+    from paper_2609_36070_b200 import mok as m
+    return m
+
+
+def skewed_routes(rng, R, T_local, E, k, skew):
+    """Distinct experts per token; expert popularity ~ 1/(e+1)^skew, shifted per source rank so that ranks differ."""
+    idx = np.empty((R, T_local, k), np.int32)
+    base = 1.0 / np.arange(1, E + 1) ** skew
+    for r in range(R):
+        p = np.roll(base, 3 * r)
+        p = p / p.sum()
+        for t in range(T_local):
+            idx[r, t] = rng.choice(E, size=k, replace=False, p=p)
+    return idx.reshape(R, T_local * k)
+
+
+# (R, T_local, E, k, skew): ragged block tails, several blocks per rank, empty experts, one expert per rank, R = 1
+ALG1_CASES = [(2, 64, 8, 2, 0.0), (4, 300, 16, 4, 1.2), (8, 129, 64, 8, 1.1), (3, 1500, 12, 3, 2.0),
+              (2, 2100, 4, 2, 0.5), (8, 64, 8, 1, 0.0), (1, 777, 16, 4, 1.0), (16, 40, 32, 2, 3.0)]
+
+
+@pytest.mark.parametrize("R,T_local,E,k,skew", ALG1_CASES)
+def test_device_algorithm1_matches_oracle(R, T_local, E, k, skew):
+    m = mok()
+    rng = np.random.default_rng(1000 * R + T_local)
+    A = skewed_routes(rng, R, T_local, E, k, skew)
+    L = E // R
+    n = T_local * k
+    idx_all = torch.from_numpy(A).cuda()
+    ws = torch.empty(m.mok_ep_workspace_bytes(R, T_local, 64, 64, 0, E, k) + 256, dtype=torch.uint8, device="cuda")
+    for c in range(R):
+        pos = torch.full((R * n,), -7, dtype=torch.int32, device="cuda")
+        t = m.mok_ep_expert_ffn(c, None, idx_all, None, None, None, None, E, k, None, pos, None, ws, 64,
+                                schedule_only=True, outputs=True)
+        assert m.mok_read_status(ws) == 0
+        S, pr, pi = mok_ref.alg1(A, L, c)
+        total = int(S[L])
+        assert np.array_equal(t["S"].cpu().numpy(), S)
+        assert np.array_equal(t["phi_rank"].cpu().numpy()[:total], pr)
+        assert np.array_equal(t["phi_index"].cpu().numpy()[:total], pi)
+        # M is a plain count: routes of rank r to local expert l
+        M = np.stack([np.bincount(A[r][(A[r] >= c * L) & (A[r] < (c + 1) * L)] - c * L, minlength=L) for r in range(R)])
+        assert np.array_equal(t["M"].cpu().numpy(), M)
+        # pos: the row of y of every served route = its schedule position moved into the 128-row-padded space
+        counts = np.diff(S)
+        pad_off = np.concatenate([[0], np.cumsum((counts + 127) // 128 * 128)])
+        want = np.full(R * n, -7, np.int64)
+        for l in range(L):
+            p = np.arange(S[l], S[l + 1])
+            want[pr[p].astype(np.int64) * n + pi[p]] = pad_off[l] + (p - S[l])
+        assert np.array_equal(pos.cpu().numpy().astype(np.int64), want)
+
+
+def ep_case(cfg, R, config=None):
+    m = mok()
+    from paper_2609_36070_b200 import ep
+    d = inputs.make_inputs(cfg)
+    g = pu.upload(d)
+    T_local = cfg.T // R
+    xs = [g["x"][r * T_local:(r + 1) * T_local].contiguous() for r in range(R)]
+    outs = ep.forward_emulated(xs, g["W_r"], g["bias"], g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], cfg.k,
+                               config=config)
+    out = torch.cat(outs)
+    # the one-rank layer on the concatenated batch: same routing, same per-row arithmetic, same combine order
+    one, st = pu.run_gpu(cfg, g)
+    idx, w, rep = pu.check_routing_and_schedule(cfg, d, st)
+    rep.update(pu.check_output(cfg, d, out, idx, w, np.arange(cfg.T, dtype=np.int32)))
+    rep["bitwise_equal_to_one_rank"] = bool(torch.equal(out.view(torch.int16), one.view(torch.int16)))
+    return rep
+
+
+@pytest.mark.parametrize("R", [1, 2, 4, 8])
+def test_expert_parallel_layer_tiny(R):
+    rep = ep_case(inputs.CONFIGS["tiny"], R)
+    assert rep["bitwise_equal_to_one_rank"], rep
+
+
+EP_SHAPES = [
+    # name, T, H, E, k, I, I_s, bias, R
+    ("skewed_4_ranks", 1024, 512, 32, 4, 384, 0, "zipf", 4),
+    ("shared_expert_2_ranks", 768, 256, 16, 2, 256, 256, "none", 2),
+    ("one_expert_per_rank", 512, 256, 8, 2, 512, 0, "none", 8),
+    ("ragged_sizes_3_ranks", 3 * 150, 264, 12, 3, 200, 72, "normal", 3),
+]
+
+
+@pytest.mark.parametrize("name,T,H,E,k,I,I_s,bias,R", EP_SHAPES)
+def test_expert_parallel_layer_shapes(name, T, H, E, k, I, I_s, bias, R):
+    cfg = inputs.MoEConfig(name, T, H, E, k, I, I_s, bias=bias, seed=11)
+    rep = ep_case(cfg, R)
+    assert rep["bitwise_equal_to_one_rank"], rep
+
+
+def test_expert_parallel_is_reproducible_and_independent_of_the_kernel_choice():
+    cfg = inputs.MoEConfig("ep_repro", 1024, 512, 16, 4, 512, 0, bias="zipf", seed=5)
+    m = mok()
+    from paper_2609_36070_b200 import ep
+    d = inputs.make_inputs(cfg)
+    g = pu.upload(d)
+    xs = [g["x"][r * 256:(r + 1) * 256].contiguous() for r in range(4)]
+    runs = []
+    for config in (None, None, m._config(cta_group=1), m._config(cta_group=3), m._config(grid=7)):
+        outs = ep.forward_emulated(xs, g["W_r"], g["bias"], g["W_gate_up"], g["W_down"], None, None, cfg.k, config=config)
+        runs.append(torch.cat(outs).view(torch.int16).clone())
+    for r in runs[1:]:
+        assert torch.equal(r, runs[0])
+
+
+def test_expert_parallel_argument_errors():
+    m = mok()
+    a = m.mok_ep_args()
+    a.rank, a.n_ranks, a.T_local, a.H, a.I, a.E, a.k = 0, 3, 64, 64, 64, 8, 2      # E not a multiple of n_ranks
+    assert m._lib.mok_ep_expert_ffn(a) == m.MOK_ERR_SHAPE
+    a.n_ranks = 17
+    assert m._lib.mok_ep_expert_ffn(a) == m.MOK_ERR_SHAPE
+    a.n_ranks, a.rank = 2, 2
+    assert m._lib.mok_ep_expert_ffn(a) == m.MOK_ERR_SHAPE
+    a.rank = 1
+    assert m._lib.mok_ep_expert_ffn(a) == m.MOK_ERR_NULL                           # idx_all missing
+    assert m._lib.mok_ep_expert_ffn(None) == m.MOK_ERR_NULL
+    assert m.mok_ep_workspace_bytes(3, 64, 64, 64, 0, 8, 2) == 0
+    assert m.mok_ep_y_rows(2, 64, 8, 2) >= 2 * 64 * 2
+    c = m.mok_ep_combine_args()
+    c.rank, c.n_ranks, c.T_local, c.H, c.E, c.k = 0, 2, 64, 64, 8, 2
+    assert m._lib.mok_ep_combine(c) == m.MOK_ERR_NULL
+    c.E = 7
+    assert m._lib.mok_ep_combine(c) == m.MOK_ERR_SHAPE
