@@ -142,3 +142,21 @@ def test_expert_parallel_argument_errors():
     assert m._lib.mok_ep_combine(c) == m.MOK_ERR_NULL
     c.E = 7
     assert m._lib.mok_ep_combine(c) == m.MOK_ERR_SHAPE
+
+
+def test_distributed_driver_with_a_world_of_one_rank():
+    """The torch.distributed driver (symmetric-memory buffers, route all-gather, barriers) run as its own process with
+    one rank: the plumbing of the multi-GPU path on the one GPU available, checked bit for bit against the one-rank
+    layer by the module's own self-check."""
+    import json
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ, MASTER_ADDR="127.0.0.1", MASTER_PORT="29547", RANK="0", WORLD_SIZE="1", LOCAL_RANK="0",
+               NCCL_NVLS_ENABLE="0", TORCH_SYMM_MEM_DISABLE_MULTICAST="1")
+    r = subprocess.run([sys.executable, "-m", "paper_2609_36070_b200.ep", "--config", "tiny", "--steps", "3"],
+                       cwd=root, env=env, capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
+    line = json.loads([l for l in r.stdout.splitlines() if l.startswith("{")][-1])
+    assert line["bitwise_equal_to_one_rank_layer"] and line["n_ranks"] == 1
