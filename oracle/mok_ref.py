@@ -144,3 +144,73 @@ def forward(x, W_r, bias, W_gate_up, W_down, W_sgu, W_sd, k):
                                T, H, I, I_s, E, k, _ptr(out, np.float64), _ptr(idx, np.int32), _ptr(w, np.float64))
     _check(rc, "forward")
     return out, idx, w
+
+
+# ---- MXFP8 mode of the routed experts (Section 3.4 "MXFP8 Support"; oracle/mok_ref_mx.c) ----
+
+def e4m3_decode(codes):
+    """The real number of every E4M3 code (uint8 array) as fp64; NaN codes decode to NaN."""
+    lib().mok_ref_e4m3_decode.restype = ctypes.c_double
+    lib().mok_ref_e4m3_decode.argtypes = [ctypes.c_uint8]
+    c = np.asarray(codes, np.uint8)
+    return np.array([lib().mok_ref_e4m3_decode(int(v)) for v in c.ravel()], np.float64).reshape(c.shape)
+
+
+def e4m3_encode(values):
+    """Nearest E4M3 code of every finite fp64 value (ties to even, clamped to +-448)."""
+    lib().mok_ref_e4m3_encode.restype = ctypes.c_uint8
+    lib().mok_ref_e4m3_encode.argtypes = [ctypes.c_double]
+    v = np.asarray(values, np.float64)
+    return np.array([lib().mok_ref_e4m3_encode(float(a)) for a in v.ravel()], np.uint8).reshape(v.shape)
+
+
+def mx_quantize(values):
+    """fp64 [rows, cols] (cols % 32 == 0) -> (codes uint8 [rows, cols], scales uint8 [rows, cols/32])."""
+    v = np.ascontiguousarray(values, np.float64)
+    rows, cols = v.shape
+    codes = np.empty((rows, cols), np.uint8)
+    scales = np.empty((rows, cols // 32), np.uint8)
+    _check(lib().mok_ref_mx_quantize(_ptr(v, np.float64), ctypes.c_longlong(rows), cols, _ptr(codes, np.uint8),
+                                     _ptr(scales, np.uint8)), "mx_quantize")
+    return codes, scales
+
+
+def mx_dequantize(codes, scales):
+    rows, cols = codes.shape
+    out = np.empty((rows, cols), np.float64)
+    _check(lib().mok_ref_mx_dequantize(_ptr(np.ascontiguousarray(codes), np.uint8),
+                                       _ptr(np.ascontiguousarray(scales), np.uint8), ctypes.c_longlong(rows), cols,
+                                       _ptr(out, np.float64)), "mx_dequantize")
+    return out
+
+
+def mx_roundtrip_bf16(bits):
+    """bf16 bit patterns [..., cols] -> fp32 array of the numbers their MXFP8 quantisation (blocks along the last
+    index) stands for."""
+    b = np.ascontiguousarray(bits, np.uint16)
+    cols = b.shape[-1]
+    rows = b.size // cols
+    out = np.empty(b.shape, np.float32)
+    _check(lib().mok_ref_mx_roundtrip_bf16(_ptr(b, np.uint16), ctypes.c_longlong(rows), cols, _ptr(out, np.float32)),
+           "mx_roundtrip_bf16")
+    return out
+
+
+def ffn_tokens_mx(x, Wgu_q, Wd_q, W_sgu, W_sd, idx, w, tokens):
+    """MoE equation with MXFP8 routed experts and a bf16 shared expert, per token from the definition.
+    Wgu_q / Wd_q: mx_roundtrip_bf16 of W_gate_up / W_down.  out[n,H] fp64."""
+    T, H = x.shape
+    k = idx.shape[1]
+    E, twoI, _ = Wgu_q.shape
+    I = twoI // 2
+    I_s = 0 if W_sgu is None else W_sgu.shape[0] // 2
+    tokens = np.ascontiguousarray(tokens, np.int32)
+    out = np.empty((tokens.size, H), np.float64)
+    rc = lib().mok_ref_ffn_tokens_mx(_ptr(x, np.uint16), _ptr(np.ascontiguousarray(Wgu_q, np.float32), np.float32),
+                                     _ptr(np.ascontiguousarray(Wd_q, np.float32), np.float32),
+                                     _ptr(W_sgu, np.uint16), _ptr(W_sd, np.uint16), H, I, I_s, E, k,
+                                     _ptr(np.ascontiguousarray(idx, np.int32), np.int32),
+                                     _ptr(np.ascontiguousarray(w, np.float64), np.float64),
+                                     _ptr(tokens, np.int32), int(tokens.size), _ptr(out, np.float64))
+    _check(rc, "ffn_tokens_mx")
+    return out
