@@ -53,6 +53,8 @@ enum {
     MOK_IMPL_TCGEN05_TN = 2 /* tcgen05 kernel with the tokens on the MMA's N side (expert padding 16 rows, not 128) */
 };
 
+enum { MOK_PRECISION_BF16 = 0, MOK_PRECISION_MXFP8 = 1 };
+
 #define MOK_MAX_HOST_CHUNKS 8
 #define MOK_DEBUG_STARVE 2
 
@@ -74,6 +76,9 @@ typedef struct mok_config {
                              mok_read_status() == MOK_ERR_TIMEOUT and a usable context (output undefined) */
     int32_t host_chunks;  /* mok_moe_forward_host: token chunks whose copies overlap compute (0 = choose by T,
                              at most MOK_MAX_HOST_CHUNKS) */
+    int32_t precision;    /* MOK_PRECISION_BF16 (0, default) or MOK_PRECISION_MXFP8: routed experts on MXFP8 operands
+                             (Section 3.4 "MXFP8 Support"); needs the pre-quantised weights in mok_args and a workspace
+                             of mok_mx_workspace_bytes(...) */
 } mok_config;
 
 /*
@@ -105,6 +110,12 @@ typedef struct mok_args {
     int32_t* inv_perm;   /* [T*k]   inverse of perm */
     const mok_config* config;       /* NULL = defaults */
     void* stream;
+    /* MXFP8 mode only (config->precision == MOK_PRECISION_MXFP8): the routed weights pre-quantised by
+       mok_mx_quantize_weights; the bf16 W_gate_up / W_down are then not read and may be NULL */
+    const void* W_gate_up_codes;    /* E4M3 [E, 2I, H] */
+    const void* W_gate_up_scales;   /* E8M0 scale atoms of the 2E matrices [I, H] */
+    const void* W_down_codes;       /* E4M3 [E, H, I] */
+    const void* W_down_scales;      /* E8M0 scale atoms of the E matrices [H, I] */
 } mok_args;
 
 /*
@@ -235,6 +246,29 @@ size_t mok_ep_workspace_bytes(int n_ranks, int T_local, int H, int I, int I_shar
 long long mok_ep_y_rows(int n_ranks, int T_local, int E, int k);
 int mok_ep_expert_ffn(const mok_ep_args* args);
 int mok_ep_combine(const mok_ep_combine_args* args);
+
+/*
+ * MXFP8 mode of the routed experts (Section 3.4 "MXFP8 Support"; the shared expert, the router and the combine stay
+ * as in bf16 mode).  Format: the microscaling format the section cites -- along the contraction dimension every 32
+ * consecutive elements share the scale 2^(floor(log2(amax)) - 8), stored as one E8M0 byte (exponent + 127), and hold
+ * v / scale rounded to nearest-even on the FP8 E4M3 grid, magnitudes above 448 clamped; an all-zero block has scale
+ * byte 0.  H and I must be multiples of 32.
+ *   mok_mx_quantize_weights : the weight pre-quantisation kernel.  W is bf16 [groups, rows, K] (W_gate_up: groups = 2E
+ *       matrices of [I, H], i.e. each expert's gate then up projection; W_down: groups = E matrices of [H, I]);
+ *       codes receives groups*rows*K bytes in the same order; scales receives mok_mx_scale_bytes(groups, rows, K)
+ *       bytes in the layout the block-scaled tensor-core instruction loads: for each (group, 128-row block,
+ *       128-element k-group) 512 bytes with the scale of row r, 32-element block j of the k-group at
+ *       (r % 32) * 16 + ((r % 128) / 32) * 4 + j; entries outside the tensor hold 127 (= 1.0).
+ *   mok_mx_quantize_rows    : the activation quantiser as a stage entry point (tests): x bf16 [rows, K] -> codes
+ *       [rows, K] and row-major scales [rows, 4 * ceil(K / 128)] (entries past K / 32 hold 127).
+ *   The forward pass in this mode quantises the token rows once (a pre-pass instead of re-quantising every row k
+ *   times inside the dispatch), the gate/up GEMM pulls codes and scales of its rows, its epilogue quantises the gated
+ *   activation as it is produced, and the down GEMM writes bf16 for the fp32 combine.
+ */
+size_t mok_mx_scale_bytes(int groups, int rows, int K);
+int mok_mx_quantize_weights(const void* W, int groups, int rows, int K, void* codes, void* scales, void* stream);
+int mok_mx_quantize_rows(const void* x, int rows, int K, void* codes, void* scales, void* stream);
+size_t mok_mx_workspace_bytes(int T, int H, int I, int I_shared, int E, int k);
 
 /*
  * Reads the device-side status word of a workspace after synchronising `stream` -- the only call besides

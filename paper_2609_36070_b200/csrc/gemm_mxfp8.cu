@@ -1,0 +1,423 @@
+// Grouped expert GEMMs on MXFP8 operands (Section 3.4 "MXFP8 Support"): E4M3 elements with one E8M0 scale per 32
+// elements along K, multiplied by the block-scaled 5th-generation tensor-core instruction
+// (tcgen05.mma.kind::mxf8f6f4.block_scale, M = 128, N = 256, K = 32, fp32 accumulators in TMEM).
+//
+// Same persistent, warp-specialised shape as the bf16 kernel with 128-row tiles:
+//   warp 0       TMA producer : A tile [128 rows x 128 bytes] and B tile [256 x 128 bytes] (128-byte swizzle) plus
+//                               their scale atoms (512 bytes per 128 rows and 128-element k-group) -> 4-stage ring
+//   warp 1       MMA issuer   : per stage, copies the scale atoms from shared memory into tensor memory
+//                               (tcgen05.cp 32x128b.warpx4: 4 columns per atom, replicated over the four lane
+//                               quadrants), then issues four K = 32 MMAs that pick their scale byte by id 0..3
+//   warps 2..9   epilogue     : two warps per TMEM lane quadrant, each draining half of the tile's columns
+//   warps 10..13 gather       : GATHER only: pull dispatch of the quantised token rows (Section 3.1) with 16-byte
+//                               cp.async, and of their scales (4 bytes per row and stage) into the atom layout
+// Tensor memory holds ONE 256-column accumulator (the scale atoms need columns too, so a second N = 256 accumulator
+// does not fit into the 512 columns); the epilogue therefore hands the accumulator back as soon as its last
+// tcgen05.ld has completed and does its arithmetic and stores afterwards.
+//
+//   EPI_SWIGLU : B tile = 128 gate rows + the matching 128 up rows; the epilogue computes h = silu(g) * u in fp32,
+//                quantises it to MXFP8 along the output columns (the next GEMM's K) -- each thread holds the 32
+//                consecutive columns of one block, so amax, scale and codes need no communication -- and writes the
+//                codes to C [rows, N] and the scales straight into the atom layout the down GEMM loads ("fuses
+//                activation quantization into ... the gated activation computation").
+//   EPI_BF16   : C [rows, N] bf16 = A . B^T (the down projection; its output feeds the fp32 combine).
+// K and N may be ragged: TMA zero-fills bytes past K and rows past the tensor, whose scales are 127 (= 1.0).
+// All mbarrier waits are bounded; on a timeout the CTA records MOK_ERR_TIMEOUT and leaves cleanly.
+#include "mok_internal.cuh"
+#include "tc_ptx.cuh"
+#include "tile_order.cuh"
+#include <cuda_fp8.h>
+
+namespace mok {
+namespace mx {
+
+using namespace tc;
+
+constexpr int BM = 128, BN = 256, BKB = 128;   // BKB: bytes = elements of K per stage (four K = 32 MMAs)
+constexpr int A_BYTES = BM * BKB;              // 16 KB
+constexpr int B_BYTES = BN * BKB;              // 32 KB
+constexpr int SFA_OFF = A_BYTES + B_BYTES;     // 512-byte atom of the A rows
+constexpr int SFB_OFF = SFA_OFF + 512;         // two atoms of the B rows
+constexpr int STAGE_BYTES = 51200;             // 50 KB: keeps every stage 1024-byte aligned for the swizzled tiles
+constexpr int STAGES = 4;
+constexpr int TMEM_COLS = 512, SF_COL0 = BN, SF_COLS = 12;   // per stage: 4 columns for A's atom, 8 for B's two
+constexpr int EPI_WARPS = 8;
+constexpr int THREADS = 64 + 32 * EPI_WARPS;   // + 4 gather warps in the GATHER instantiation
+constexpr int GATHER_THREADS = 128;
+constexpr int SMEM_CTRL = 256;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + SMEM_CTRL + 1024;
+
+struct Ctrl {
+    uint64_t full[STAGES];
+    uint64_t empty[STAGES];
+    uint64_t tfull;
+    uint64_t tempty;
+    uint32_t tmem_base;
+    uint32_t abort;
+};
+static_assert(sizeof(Ctrl) <= SMEM_CTRL, "control block too large");
+
+// Instruction descriptor of the block-scaled MMA: A and B E4M3 (format 0), both K-major, N = 256, scales E8M0,
+// M = 128; the two scale ids (which byte of the 4-byte scale cell a K = 32 step uses) are added per instruction.
+__device__ __forceinline__ constexpr uint32_t make_idesc_mx(uint32_t sf_id) {
+    return (sf_id << 4) | ((uint32_t)(BN >> 3) << 17) | (1u << 23) | ((uint32_t)(BM >> 4) << 24) | (sf_id << 29);
+}
+// Shared-memory descriptor of one scale atom for tcgen05.cp: 32 rows of 16 bytes, no swizzle, 8-row groups 128
+// bytes apart.
+__device__ __forceinline__ uint64_t make_sf_desc(uint32_t addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)(128 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    return d;
+}
+__device__ __forceinline__ void tc_cp_sf(uint32_t taddr, uint64_t sdesc) {
+    asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+}
+__device__ __forceinline__ void tc_mma_mx(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                          uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %6, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::mxf8f6f4.block_scale [%0], %1, %2, %3, [%4], [%5], p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(sfa_tmem), "r"(sfb_tmem), "r"(accumulate) : "memory");
+}
+// Plain (untiled) bulk copy global -> shared, completing on an mbarrier; both addresses 16-byte aligned.
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void cp_async_4(uint32_t dst, const void* src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
+}
+
+// E8M0 code of a block's scale from its amax, and the factor 2^(127 - code) that maps the block onto the E4M3 grid.
+__device__ __forceinline__ int scale_code(float amax) {
+    int code = (int)((__float_as_uint(amax) >> 23) & 0xFFu) - 8;
+    code = code < 0 ? 0 : code;
+    return code > 254 ? 254 : code;
+}
+__device__ __forceinline__ float inv_scale(int code) {
+    const int e = 254 - code;
+    return e > 0 ? __uint_as_float((uint32_t)e << 23) : __uint_as_float(0x00400000u);
+}
+
+template <int EPI, bool GATHER>
+__global__ void __launch_bounds__(THREADS + (GATHER ? GATHER_THREADS : 0), 1)
+gemm_mx_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
+               const __grid_constant__ GemmArgs a, const int n_nt, const int k_blocks) {
+    constexpr bool SWIGLU = (EPI == EPI_SWIGLU);
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t* smem = smem_raw + (base - raw);
+    Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem + STAGES * STAGE_BYTES);
+    volatile uint32_t* abort_flag = &ctrl->abort;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    int n_mt_total = (a.dense_rows > 0) ? (a.dense_rows + BM - 1) / BM : *a.n_mtiles;
+    if (n_mt_total > a.max_mt) n_mt_total = a.max_mt;
+    const int total = n_mt_total * n_nt;
+    const int KG = k_blocks;                                  // 128-element k-groups = scale atoms along K
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(smem_u32(&ctrl->full[s]), 1 + (GATHER ? GATHER_THREADS : 0));
+            mbar_init(smem_u32(&ctrl->empty[s]), 1);
+        }
+        mbar_init(smem_u32(&ctrl->tfull), 1);
+        mbar_init(smem_u32(&ctrl->tempty), EPI_WARPS);
+        ctrl->abort = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&ctrl->tmem_base)), "r"((uint32_t)TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = ctrl->tmem_base;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0 && !a.starve) {
+            int s = 0;
+            uint32_t ph = 0;
+            const int b_rows_per_expert = (SWIGLU ? 2 : 1) * a.N;
+            const int NB = (a.N + 127) / 128;                 // 128-row blocks of one weight matrix (scale atoms)
+            for (int L = blockIdx.x; L < total; L += gridDim.x) {
+                const Tile t = decode_tile(a, L, n_nt, n_mt_total, BM);
+                const int brow0 = t.e * b_rows_per_expert + (SWIGLU ? t.n * (BN / 2) : t.n * BN);
+                const int brow1 = SWIGLU ? brow0 + a.N : brow0 + BN / 2;
+                // scale atoms of the two 128-row halves of the B tile
+                int nb0, nb1;
+                if (SWIGLU) { nb0 = (2 * t.e) * NB + t.n; nb1 = (2 * t.e + 1) * NB + t.n; }
+                else { nb0 = t.e * NB + min(2 * t.n, NB - 1); nb1 = t.e * NB + min(2 * t.n + 1, NB - 1); }
+                const uint8_t* sfb0 = a.sfb + (size_t)nb0 * KG * 512;
+                const uint8_t* sfb1 = a.sfb + (size_t)nb1 * KG * 512;
+                const uint8_t* sfa = GATHER ? nullptr : a.sfa + (size_t)(t.row0 / BM) * KG * 512;
+                bool ok = true;
+                for (int kb = 0; kb < k_blocks; ++kb) {
+                    ok = mbar_wait(smem_u32(&ctrl->empty[s]), ph ^ 1u, abort_flag, a.header, 1);
+                    if (!ok) break;
+                    const uint32_t full = smem_u32(&ctrl->full[s]);
+                    const uint32_t sa = base + s * STAGE_BYTES, sb = sa + A_BYTES;
+                    mbar_expect_tx(full, B_BYTES + 1024 + (GATHER ? 0 : A_BYTES + 512));
+                    if (!GATHER) {
+                        tma_load_2d(sa, &tmapA, full, kb * BKB, t.row0);
+                        bulk_load(sa + SFA_OFF, sfa + (size_t)kb * 512, 512, full);
+                    }
+                    tma_load_2d(sb, &tmapB, full, kb * BKB, brow0);
+                    tma_load_2d(sb + B_BYTES / 2, &tmapB, full, kb * BKB, brow1);
+                    bulk_load(sa + SFB_OFF, sfb0 + (size_t)kb * 512, 512, full);
+                    bulk_load(sa + SFB_OFF + 512, sfb1 + (size_t)kb * 512, 512, full);
+                    if (++s == STAGES) { s = 0; ph ^= 1u; }
+                }
+                if (!ok) break;
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // -------------------------------------------------------------- MMA issuer
+            int s = 0;
+            uint32_t ph = 0, aph = 0;
+            for (int L = blockIdx.x; L < total; L += gridDim.x) {
+                bool ok = mbar_wait(smem_u32(&ctrl->tempty), aph ^ 1u, abort_flag, a.header, 2);
+                if (!ok) break;
+                aph ^= 1u;
+                tc_fence_after();
+                for (int kb = 0; kb < k_blocks; ++kb) {
+                    ok = mbar_wait(smem_u32(&ctrl->full[s]), ph, abort_flag, a.header, 3);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t sa = base + s * STAGE_BYTES, sb = sa + A_BYTES;
+                    const uint32_t sf_tmem = tmem_base + (uint32_t)(SF_COL0 + s * SF_COLS);
+                    tc_cp_sf(sf_tmem, make_sf_desc(sa + SFA_OFF));
+                    tc_cp_sf(sf_tmem + 4, make_sf_desc(sa + SFB_OFF));
+                    tc_cp_sf(sf_tmem + 8, make_sf_desc(sa + SFB_OFF + 512));
+                    const uint64_t adesc = make_smem_desc(sa), bdesc = make_smem_desc(sb);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)               // +32 bytes per K = 32 step inside the 128-byte swizzle row
+                        tc_mma_mx(tmem_base, adesc + (uint64_t)(j * 2), bdesc + (uint64_t)(j * 2), make_idesc_mx((uint32_t)j),
+                                  sf_tmem, sf_tmem + 4, (kb | j) ? 1u : 0u);
+                    tc_commit<1>(smem_u32(&ctrl->empty[s]));
+                    if (++s == STAGES) { s = 0; ph ^= 1u; }
+                }
+                if (!ok) break;
+                tc_commit<1>(smem_u32(&ctrl->tfull));
+            }
+        }
+        __syncwarp();
+    } else if (GATHER && warp >= 2 + EPI_WARPS) {
+        // ------------------------------------------------------------------ gather warps (pull dispatch)
+        // Data: warp gw owns tile rows 32 gw .. 32 gw + 31; lane = (sub-row 0..3, 16-byte chunk 0..7); pass i covers
+        // rows 32 gw + 4 i + sub-row; chunk c of row r lands at r*128 + ((c ^ (r & 7)) * 16).  Scales: thread q of the
+        // 128 copies the 4 scale bytes of row q for this k-group to (q % 32) * 16 + (q / 32) * 4 of the atom.
+        const int gw = warp - (2 + EPI_WARPS), sub = lane >> 3, chunk = lane & 7;
+        const int q = gw * 32 + lane;
+        int s = 0;
+        uint32_t ph = 0;
+        const uint8_t* xq = reinterpret_cast<const uint8_t*>(a.A);
+        for (int L = blockIdx.x; L < total; L += gridDim.x) {
+            const Tile t = decode_tile(a, L, n_nt, n_mt_total, BM);
+            const int valid = __ldg(a.counts + t.e) - t.m * BM;
+            const int tok0 = __ldg(a.row_token + t.row0);
+            const int* rows = a.row_token + t.row0;
+            const uint8_t* src[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int r = gw * 32 + i * 4 + sub;
+                const int tok = (r < valid) ? __ldg(rows + r) : tok0;
+                src[i] = xq + (size_t)tok * a.K + chunk * 16;
+            }
+            const int tokq = (q < valid) ? __ldg(rows + q) : tok0;
+            const uint8_t* sfsrc = a.sfa + (size_t)tokq * a.sfa_stride;
+            const uint32_t sfdst = SFA_OFF + (q & 31) * 16 + (q >> 5) * 4;
+            bool ok = true;
+            for (int kb = 0; kb < k_blocks; ++kb) {
+                ok = mbar_wait(smem_u32(&ctrl->empty[s]), ph ^ 1u, abort_flag, a.header, 5);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                const uint32_t sa = base + s * STAGE_BYTES;
+                const bool in_k = (kb * BKB + chunk * 16) < a.K;          // K tail: zero-fill
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int r = gw * 32 + i * 4 + sub;
+                    const uint32_t dst = sa + r * 128 + ((chunk ^ (r & 7)) << 4);
+                    cp_async_16(dst, in_k ? (const void*)(src[i] + kb * BKB) : (const void*)xq, in_k ? 16u : 0u);
+                }
+                cp_async_4(sa + sfdst, sfsrc + kb * 4);
+                cp_async_mbar_arrive(smem_u32(&ctrl->full[s]));
+                if (++s == STAGES) { s = 0; ph ^= 1u; }
+            }
+            if (!ok) break;
+        }
+        asm volatile("cp.async.wait_all;" ::: "memory");
+    } else {
+        // ------------------------------------------------------------------ epilogue (warps 2..9)
+        // Warp w drains TMEM lane quadrant w % 4 (its 32 rows) and column half (w - 2) / 4 of the tile.
+        const int quad = warp & 3, hh = (warp - 2) >> 2;
+        uint32_t aph = 0;
+        for (int L = blockIdx.x; L < total; L += gridDim.x) {
+            const Tile t = decode_tile(a, L, n_nt, n_mt_total, BM);
+            bool ok = mbar_wait(smem_u32(&ctrl->tfull), aph, abort_flag, a.header, 4);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            aph ^= 1u;
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16);
+            const int row = t.row0 + quad * 32 + lane;
+            if (SWIGLU) {
+                // output columns [64 hh, 64 hh + 64) of the tile's 128: two 32-column MX blocks per thread.  Block 0 is
+                // quantised while block 1's loads are in flight; the accumulator goes back to the MMA issuer as soon
+                // as the last tcgen05.ld has completed.
+                uint32_t o[2][8];
+                int code[2];
+#pragma unroll
+                for (int b = 0; b < 2; ++b) {
+                    uint32_t g[32], u[32];
+                    tc_ld32(taddr + hh * 64 + b * 32, g);
+                    tc_ld32(taddr + BN / 2 + hh * 64 + b * 32, u);
+                    tc_wait_ld();
+                    if (b == 1) {
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(smem_u32(&ctrl->tempty));
+                    }
+                    float amax = 0.f;
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        const float hv = swiglu(__uint_as_float(g[i]), __uint_as_float(u[i]));
+                        g[i] = __float_as_uint(hv);
+                        amax = fmaxf(amax, fabsf(hv));
+                    }
+                    code[b] = scale_code(amax);
+                    const float inv = inv_scale(code[b]);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const uint32_t lo = __nv_cvt_float2_to_fp8x2(make_float2(__uint_as_float(g[4 * i]) * inv, __uint_as_float(g[4 * i + 1]) * inv), __NV_SATFINITE, __NV_E4M3);
+                        const uint32_t hi = __nv_cvt_float2_to_fp8x2(make_float2(__uint_as_float(g[4 * i + 2]) * inv, __uint_as_float(g[4 * i + 3]) * inv), __NV_SATFINITE, __NV_E4M3);
+                        o[b][i] = lo | (hi << 16);
+                    }
+                }
+                uint8_t* crow = reinterpret_cast<uint8_t*>(a.C) + (size_t)row * a.ldc;
+                uint8_t* atom = a.sfc + ((size_t)(t.row0 / BM) * ((a.N + 127) / 128) + t.n) * 512 + lane * 16 + quad * 4;
+#pragma unroll
+                for (int b = 0; b < 2; ++b) {
+                    const int col = t.n * (BN / 2) + hh * 64 + b * 32;
+                    if (col >= a.N) continue;
+                    *reinterpret_cast<uint4*>(crow + col) = make_uint4(o[b][0], o[b][1], o[b][2], o[b][3]);
+                    *reinterpret_cast<uint4*>(crow + col + 16) = make_uint4(o[b][4], o[b][5], o[b][6], o[b][7]);
+                    atom[hh * 2 + b] = (uint8_t)code[b];
+                }
+            } else {
+                // output columns [128 hh, 128 hh + 128) of the tile's 256, as bf16
+                uint32_t o[4][16];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t r[32];
+                    tc_ld32(taddr + hh * 128 + c * 32, r);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) o[c][i] = pack_bf16(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&ctrl->tempty));
+                __nv_bfloat16* crow = reinterpret_cast<__nv_bfloat16*>(a.C) + (size_t)row * a.ldc;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const int col = t.n * BN + hh * 128 + c * 32;
+#pragma unroll
+                    for (int v = 0; v < 4; ++v)
+                        if (col + v * 8 < a.N)
+                            *reinterpret_cast<uint4*>(crow + col + v * 8) = make_uint4(o[c][4 * v], o[c][4 * v + 1], o[c][4 * v + 2], o[c][4 * v + 3]);
+                }
+            }
+        }
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    if (*abort_flag) {   // failure path only: give copies and MMAs already in flight time to land before leaving
+        const unsigned long long t0 = globaltimer();
+        while (globaltimer() - t0 < 200000ull) { }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS) : "memory");
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn get_encode() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// 2D row-major byte tensor [rows, cols] -> tensor map with a [128 rows x 128 bytes] box and 128-byte swizzle.
+static bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols) {
+    EncodeTiledFn enc = get_encode();
+    if (!enc) return false;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols};
+    cuuint32_t box[2] = {(cuuint32_t)BKB, 128};
+    cuuint32_t estr[2] = {1, 1};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace mx
+
+template <int EPI, bool GATHER>
+static cudaError_t launch_one_mx(const CUtensorMap& mA, const CUtensorMap& mB, const GemmArgs& a, int n_nt, int k_blocks,
+                                 int grid, cudaStream_t s) {
+    using namespace mx;
+    static int sms = 0;
+    auto kernel = gemm_mx_kernel<EPI, GATHER>;
+    if (!sms) {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    }
+    int blocks = (grid <= 0 || grid > sms) ? sms : grid;
+    kernel<<<blocks, THREADS + (GATHER ? GATHER_THREADS : 0), SMEM_BYTES, s>>>(mA, mB, a, n_nt, k_blocks);
+    return cudaGetLastError();
+}
+
+// a.A / a.B: E4M3 codes; a.K a multiple of 32 (16 for the TMA row pitch) and, for EPI_SWIGLU, a.N a multiple of 32.
+cudaError_t launch_gemm_mx(const GemmArgs& a, int epi, int grid, cudaStream_t s) {
+    using namespace mx;
+    const bool swiglu = (epi == EPI_SWIGLU), gather = (a.row_token != nullptr);
+    if (a.tile_m != BM || (a.K % 32) || !a.sfa || !a.sfb || (swiglu && (!a.sfc || (a.N % 32)))) return cudaErrorInvalidValue;
+    CUtensorMap mA, mB;
+    const uint64_t b_rows = (uint64_t)a.E * (swiglu ? 2 : 1) * a.N;
+    if (!make_map(&mA, a.A, (uint64_t)a.a_rows, (uint64_t)a.K)) return cudaErrorInvalidValue;
+    if (!make_map(&mB, a.B, b_rows, (uint64_t)a.K)) return cudaErrorInvalidValue;
+    const int n_nt = swiglu ? (a.N + BN / 2 - 1) / (BN / 2) : (a.N + BN - 1) / BN;
+    const int k_blocks = (a.K + BKB - 1) / BKB;
+    if (swiglu && gather) return launch_one_mx<EPI_SWIGLU, true>(mA, mB, a, n_nt, k_blocks, grid, s);
+    if (swiglu) return launch_one_mx<EPI_SWIGLU, false>(mA, mB, a, n_nt, k_blocks, grid, s);
+    if (epi == EPI_BF16 && !gather) return launch_one_mx<EPI_BF16, false>(mA, mB, a, n_nt, k_blocks, grid, s);
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace mok

@@ -34,6 +34,7 @@
 // All mbarrier waits are bounded: on a timeout the CTA records MOK_ERR_TIMEOUT and leaves cleanly.
 #include "mok_internal.cuh"
 #include "tc_ptx.cuh"
+#include "tile_order.cuh"
 
 namespace mok {
 namespace tc {
@@ -45,7 +46,6 @@ constexpr int MAX_STAGES = 6;
 constexpr int ACC_STAGES = 2, TMEM_COLS = 512;
 constexpr int THREADS = 192;                   // + 4 gather warps in the GATHER instantiation
 constexpr int GATHER_THREADS = 128;
-constexpr int GROUP_ROWS = 2048;               // rows of one rasterisation group (16 tiles of 128 rows)
 constexpr int SMEM_CTRL = 256;
 constexpr int OUT_STAGE_BYTES = 4 * 8192;      // per epilogue warp: 32 rows x 128 bf16 columns, as two swizzled boxes
 constexpr int RING_BYTES = 196608;             // 4 x 48 KB or 6 x 32 KB
@@ -66,33 +66,6 @@ static_assert(sizeof(Ctrl) <= SMEM_CTRL, "control block too large");
 template <int CTAS>
 __device__ __forceinline__ constexpr uint32_t make_idesc() {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((BM * CTAS) >> 4) << 24);
-}
-
-struct Tile { int row0, n, e, m; };   // row0: first row of the (pair) tile in the padded row space
-
-// Tile L of the static schedule.  `tm` = rows per tile (128 x CTAS).  Inside an expert, M tiles are taken in groups
-// of GROUP_ROWS rows: all N tiles of a group before the next group, M fastest, so the group's activations stay in
-// L2 while the expert's weight tiles stream.
-__device__ __forceinline__ Tile decode_tile(const GemmArgs& a, int L, int n_nt, int n_mt_total, int tm) {
-    Tile t;
-    int mt0, m_cnt;
-    if (a.dense_rows > 0) {
-        t.e = 0; mt0 = 0; m_cnt = n_mt_total;
-    } else {
-        t.e = __ldg(a.tile_expert + L / n_nt);
-        mt0 = __ldg(a.mt_start + t.e);
-        m_cnt = __ldg(a.mt_start + t.e + 1) - mt0;
-    }
-    const int group_m = GROUP_ROWS / tm;
-    const int r = L - n_nt * mt0;
-    const int per_group = group_m * n_nt;
-    const int g = r / per_group;
-    const int rem = r - g * per_group;
-    const int in_group = min(group_m, m_cnt - g * group_m);
-    t.n = rem / in_group;
-    t.m = g * group_m + (rem - t.n * in_group);
-    t.row0 = (mt0 + t.m) * tm;
-    return t;
 }
 
 template <int EPI, bool GATHER, int CTAS>

@@ -35,8 +35,9 @@ static bool sizes_ok(int T, int H, int I, int Is, int E, int k) {
     return true;
 }
 
-bool ws_layout(int T, int H, int I, int Is, int E, int k, WsLayout* L) {
+bool ws_layout(int T, int H, int I, int Is, int E, int k, WsLayout* L, bool mx) {
     if (!sizes_ok(T, H, I, Is, E, k)) return false;
+    if (mx && ((H % 32) || (I % 32))) return false;
     memset(L, 0, sizeof(*L));
     const long long R = (long long)T * k;
     const long long nonempty_max = R < E ? R : E;
@@ -74,19 +75,38 @@ bool ws_layout(int T, int H, int I, int Is, int E, int k, WsLayout* L) {
     L->y = take(2 * (size_t)Rpad * H);
     L->hs = take(Is > 0 ? 2 * (size_t)L->Tpad * Is : 0);
     L->ysh = take(Is > 0 ? 2 * (size_t)L->Tpad * H : 0);
+    if (mx) {
+        L->x8 = take((size_t)(T > 0 ? T : 1) * H);
+        L->sx = take((size_t)(T > 0 ? T : 1) * ((H + 127) / 128 * 4));
+        L->h8 = take((size_t)Rpad * I);
+        L->sh = take((size_t)(Rpad / TILE_M) * ((I + 127) / 128) * 512);
+    }
     L->total = off;
     return true;
 }
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+static bool use_mx(const mok_config* cfg) { return cfg && cfg->precision == MOK_PRECISION_MXFP8; }
+
 static int validate(const mok_args* a, WsLayout* L, size_t extra_ws) {
     if (!a) return MOK_ERR_NULL;
-    if (!ws_layout(a->T, a->H, a->I, a->I_shared, a->E, a->k, L)) return MOK_ERR_SHAPE;
+    if (a->config && (a->config->precision < 0 || a->config->precision > 1)) return MOK_ERR_SHAPE;
+    const bool mx = use_mx(a->config);
+    if (mx && a->config->impl != MOK_IMPL_TCGEN05) return MOK_ERR_SHAPE;
+    if (!ws_layout(a->T, a->H, a->I, a->I_shared, a->E, a->k, L, mx)) return MOK_ERR_SHAPE;
     if ((a->I_shared > 0) != (a->W_shared_gate_up != nullptr) || (a->I_shared > 0) != (a->W_shared_down != nullptr))
         return MOK_ERR_SHAPE;
     if (a->T == 0) return MOK_OK;
-    if (!a->W_router || !a->W_gate_up || !a->W_down) return MOK_ERR_NULL;
+    if (!a->W_router) return MOK_ERR_NULL;
+    if (mx) {
+        if (!a->W_gate_up_codes || !a->W_gate_up_scales || !a->W_down_codes || !a->W_down_scales) return MOK_ERR_NULL;
+        if (!aligned16(a->W_gate_up_codes) || !aligned16(a->W_gate_up_scales) || !aligned16(a->W_down_codes) ||
+            !aligned16(a->W_down_scales))
+            return MOK_ERR_ALIGN;
+    } else if (!a->W_gate_up || !a->W_down) {
+        return MOK_ERR_NULL;
+    }
     if (!aligned16(a->W_router) || !aligned16(a->W_gate_up) || !aligned16(a->W_down) ||
         !aligned16(a->W_shared_gate_up) || !aligned16(a->W_shared_down))
         return MOK_ERR_ALIGN;
@@ -197,15 +217,24 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
     int rc = route_stage(a, L, ws, x, s);
     if (rc) return rc;
     MOK_MARK(MOK_STAGE_ROUTER + 1);
-    const int tile_m = tile_rows(a->config, a->I);
+    const int tile_m = use_mx(a->config) ? TILE_M : tile_rows(a->config, a->I);
     const int pad_m = use_tn(a->config) ? 16 : tile_m;   // tokens on the MMA's N side need 16-row granularity only
     e = launch_schedule(reinterpret_cast<const int32_t*>(ws + L.idx), a->T, a->E, a->k, tile_m, pad_m, L, ws,
                         a->counts, a->offsets, a->perm, a->inv_perm, s);
     if (e != cudaSuccess) return cuda_fail(e);
     MOK_MARK(MOK_STAGE_SCHEDULE + 1);
-    const bool simt = !fused_gather(a->config, a->I);
+    const bool mx = use_mx(a->config);
+    const bool simt = !mx && !fused_gather(a->config, a->I);
     if (simt) {   // materialise the expert-sorted copy of x
         e = launch_gather(x, a->H, a->k, tile_m, L, ws, s);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    if (mx) {     // quantise the token rows once; the gate/up GEMM pulls codes and scales of the rows it needs
+        e = launch_mx_quantize_rows(x, a->T, a->H, reinterpret_cast<uint8_t*>(ws + L.x8),
+                                    reinterpret_cast<uint8_t*>(ws + L.sx), s);
+        if (e != cudaSuccess) return cuda_fail(e);
+        // scale atoms of the gated activation: blocks past I keep 127 (= 1.0)
+        e = cudaMemsetAsync(ws + L.sh, 127, (size_t)(L.Rpad / TILE_M) * ((a->I + 127) / 128) * 512, s);
         if (e != cudaSuccess) return cuda_fail(e);
     }
     MOK_MARK(MOK_STAGE_GATHER + 1);
@@ -229,31 +258,63 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
         if (e != cudaSuccess) return cuda_fail(e);
         g.starve = 1;
     }
-    // routed experts: h = silu(Xg Wg^T) * (Xg Wu^T);  y = h Wd^T
-    if (simt) {
-        g.A = reinterpret_cast<const __nv_bfloat16*>(ws + L.xg);
-        g.a_rows = L.Rpad;
-    } else {
-        g.A = x;
+    if (mx) {
+        // routed experts on MXFP8 operands (Section 3.4): h = Q(silu(Q(x) Wg_q^T) * (Q(x) Wu_q^T));  y = h Wd_q^T
+        const int grid = a->config->grid;
+        g.A = reinterpret_cast<const __nv_bfloat16*>(ws + L.x8);
         g.a_rows = a->T;
         g.row_token = reinterpret_cast<const int32_t*>(ws + L.row_token);
-        g.counts = reinterpret_cast<const int32_t*>(ws + L.counts);
+        g.sfa = reinterpret_cast<const uint8_t*>(ws + L.sx);
+        g.sfa_stride = (a->H + 127) / 128 * 4;
+        g.B = reinterpret_cast<const __nv_bfloat16*>(a->W_gate_up_codes);
+        g.sfb = reinterpret_cast<const uint8_t*>(a->W_gate_up_scales);
+        g.C = ws + L.h8;
+        g.sfc = reinterpret_cast<uint8_t*>(ws + L.sh);
+        g.K = a->H; g.N = a->I; g.ldc = a->I; g.E = a->E; g.rows_pad = L.Rpad; g.dense_rows = 0;
+        g.total_rows = L.R;
+        e = launch_gemm_mx(g, EPI_SWIGLU, grid, s);
+        if (e != cudaSuccess) return cuda_fail(e);
+        MOK_MARK(MOK_STAGE_GEMM1 + 1);
+        g.row_token = nullptr;
+        g.starve = 0;
+        g.A = reinterpret_cast<const __nv_bfloat16*>(ws + L.h8);
+        g.a_rows = L.Rpad;
+        g.sfa = reinterpret_cast<const uint8_t*>(ws + L.sh);
+        g.B = reinterpret_cast<const __nv_bfloat16*>(a->W_down_codes);
+        g.sfb = reinterpret_cast<const uint8_t*>(a->W_down_scales);
+        g.C = ws + L.y;
+        g.sfc = nullptr;
+        g.K = a->I; g.N = a->H; g.ldc = a->H;
+        e = launch_gemm_mx(g, EPI_BF16, grid, s);
+        if (e != cudaSuccess) return cuda_fail(e);
+        g.sfa = g.sfb = nullptr;
+    } else {
+        // routed experts: h = silu(Xg Wg^T) * (Xg Wu^T);  y = h Wd^T
+        if (simt) {
+            g.A = reinterpret_cast<const __nv_bfloat16*>(ws + L.xg);
+            g.a_rows = L.Rpad;
+        } else {
+            g.A = x;
+            g.a_rows = a->T;
+            g.row_token = reinterpret_cast<const int32_t*>(ws + L.row_token);
+            g.counts = reinterpret_cast<const int32_t*>(ws + L.counts);
+        }
+        g.B = reinterpret_cast<const __nv_bfloat16*>(a->W_gate_up);
+        g.C = ws + L.h;
+        g.K = a->H; g.N = a->I; g.ldc = a->I; g.E = a->E; g.rows_pad = L.Rpad; g.dense_rows = 0;
+        g.total_rows = L.R;
+        if ((rc = run_gemm(g, true, a->config, L, ws, s))) return rc;
+        g.row_token = nullptr;
+        g.starve = 0;
+        g.a_rows = L.Rpad;
+        g.dbg_slot = dbg ? 2 : -1;
+        MOK_MARK(MOK_STAGE_GEMM1 + 1);
+        g.A = reinterpret_cast<const __nv_bfloat16*>(ws + L.h);
+        g.B = reinterpret_cast<const __nv_bfloat16*>(a->W_down);
+        g.C = ws + L.y;
+        g.K = a->I; g.N = a->H; g.ldc = a->H;
+        if ((rc = run_gemm(g, false, a->config, L, ws, s))) return rc;
     }
-    g.B = reinterpret_cast<const __nv_bfloat16*>(a->W_gate_up);
-    g.C = ws + L.h;
-    g.K = a->H; g.N = a->I; g.ldc = a->I; g.E = a->E; g.rows_pad = L.Rpad; g.dense_rows = 0;
-    g.total_rows = L.R;
-    if ((rc = run_gemm(g, true, a->config, L, ws, s))) return rc;
-    g.row_token = nullptr;
-    g.starve = 0;
-    g.a_rows = L.Rpad;
-    g.dbg_slot = dbg ? 2 : -1;
-    MOK_MARK(MOK_STAGE_GEMM1 + 1);
-    g.A = reinterpret_cast<const __nv_bfloat16*>(ws + L.h);
-    g.B = reinterpret_cast<const __nv_bfloat16*>(a->W_down);
-    g.C = ws + L.y;
-    g.K = a->I; g.N = a->H; g.ldc = a->H;
-    if ((rc = run_gemm(g, false, a->config, L, ws, s))) return rc;
     MOK_MARK(MOK_STAGE_GEMM2 + 1);
     g.dbg_slot = dbg ? 3 : -1;
     if (a->I_shared > 0) {   // shared expert: every token in natural order, no gather
@@ -289,6 +350,37 @@ static OwnedWs g_owned[64];
 using namespace mok;
 
 extern "C" {
+
+size_t mok_mx_workspace_bytes(int T, int H, int I, int I_shared, int E, int k) {
+    WsLayout L;
+    return ws_layout(T, H, I, I_shared, E, k, &L, true) ? L.total : 0;
+}
+
+size_t mok_mx_scale_bytes(int groups, int rows, int K) {
+    if (groups < 1 || rows < 1 || K < 32 || (K % 32)) return 0;
+    return (size_t)groups * ((rows + 127) / 128) * ((K + 127) / 128) * 512;
+}
+
+int mok_mx_quantize_weights(const void* W, int groups, int rows, int K, void* codes, void* scales, void* stream) {
+    if (!W || !codes || !scales) return MOK_ERR_NULL;
+    if (mok_mx_scale_bytes(groups, rows, K) == 0) return MOK_ERR_SHAPE;
+    if (!aligned16(W) || !aligned16(codes) || !aligned16(scales)) return MOK_ERR_ALIGN;
+    cudaError_t e = launch_mx_quantize_atoms(reinterpret_cast<const __nv_bfloat16*>(W), groups, rows, K,
+                                             reinterpret_cast<uint8_t*>(codes), reinterpret_cast<uint8_t*>(scales),
+                                             reinterpret_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? MOK_OK : cuda_fail(e);
+}
+
+int mok_mx_quantize_rows(const void* x, int rows, int K, void* codes, void* scales, void* stream) {
+    if (!x || !codes || !scales) return MOK_ERR_NULL;
+    if (rows < 0 || K < 32 || (K % 32)) return MOK_ERR_SHAPE;
+    if (rows == 0) return MOK_OK;
+    if (!aligned16(x) || !aligned16(codes) || !aligned16(scales)) return MOK_ERR_ALIGN;
+    cudaError_t e = launch_mx_quantize_rows(reinterpret_cast<const __nv_bfloat16*>(x), rows, K,
+                                            reinterpret_cast<uint8_t*>(codes), reinterpret_cast<uint8_t*>(scales),
+                                            reinterpret_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? MOK_OK : cuda_fail(e);
+}
 
 size_t mok_workspace_bytes(int T, int H, int I, int I_shared, int E, int k) {
     WsLayout L;
@@ -390,7 +482,7 @@ int mok_moe_forward_host(const mok_args* a, const void* x_host, void* out_host) 
         mok_args ac = *a;
         ac.T = tc;
         WsLayout Lc;
-        if (!ws_layout(tc, a->H, a->I, a->I_shared, a->E, a->k, &Lc)) return MOK_ERR_SHAPE;
+        if (!ws_layout(tc, a->H, a->I, a->I_shared, a->E, a->k, &Lc, use_mx(a->config))) return MOK_ERR_SHAPE;
         if ((e = cudaStreamWaitEvent(s, p->in_done[c], 0)) != cudaSuccess) return cuda_fail(e);
         rc = forward_device(&ac, Lc, xd + (size_t)t0 * a->H, od + (size_t)t0 * a->H);
         if (rc) return rc;
@@ -495,7 +587,9 @@ int mok_launch_count(int T, int H, int I, int I_shared, int E, int k, const mok_
     if (!ws_layout(T, H, I, I_shared, E, k, &L) || T == 0) return 0;
     // router (1 fp32-FMA kernel, or split + GEMM + top-k), 3 schedule kernels, (gather on the SIMT path),
     // 2 routed GEMMs, (2 shared GEMMs), combine
-    return (use_simt_router(config, k) ? 1 : 3) + 3 + (fused_gather(config, I) ? 0 : 1) + 2 + (I_shared > 0 ? 2 : 0) + 1;
+    // (MXFP8 mode: the token-row quantiser instead of the gather kernel; its two memsets are not counted)
+    const int pre = use_mx(config) ? 1 : (fused_gather(config, I) ? 0 : 1);
+    return (use_simt_router(config, k) ? 1 : 3) + 3 + pre + 2 + (I_shared > 0 ? 2 : 0) + 1;
 }
 
 int mok_profile_begin(int max_calls) {

@@ -37,6 +37,7 @@ struct WsLayout {
     size_t wr_split;      // bf16 [3E, H]: W_r split into hi/mid/lo parts for the tensor-core router
     size_t logits;        // fp32 [Tpad, ldl] partial logits of the tensor-core router (ldl = 3E rounded up to 8)
     size_t xg, h, y, hs, ysh;
+    size_t x8, sx, h8, sh;   // MXFP8 mode: quantised token rows + row-major scales, quantised gated activation + scale atoms
     size_t total;
     int32_t R;            // T*k
     int32_t Rpad;         // upper bound on padded rows for either tile_m (multiple of 256)
@@ -45,7 +46,7 @@ struct WsLayout {
     int32_t n_blk;        // schedule blocks
 };
 
-bool ws_layout(int T, int H, int I, int Is, int E, int k, WsLayout* L);
+bool ws_layout(int T, int H, int I, int Is, int E, int k, WsLayout* L, bool mx = false);
 
 // Arguments of the grouped GEMM (both implementations).  Rows live in a padded space: expert e owns rows
 // [128*mt_start[e], 128*mt_start[e+1]); tile q belongs to expert tile_expert[q].  In dense mode (shared
@@ -76,6 +77,11 @@ struct GemmArgs {
     // or a peer's, mapped into this process) with plain 16-byte asynchronous copies -- never a multicast load.
     int32_t peer_tokens;
     const __nv_bfloat16* peer_x[MOK_MAX_RANKS];
+    // MXFP8 mode (Section 3.4): A and B hold E4M3 codes (one byte per element) and these are the E8M0 block scales.
+    const uint8_t* sfa;          // GATHER: row-major [tokens, sfa_stride] of x; else 512-byte atoms [rows_pad/128][KG]
+    const uint8_t* sfb;          // 512-byte atoms [E (x2 for gate, up)][ceil(N/128)][KG] of the weights
+    uint8_t* sfc;                // SWIGLU epilogue: scale atoms of the quantised gated activation [rows_pad/128][ceil(N/128)]
+    int32_t sfa_stride;          // bytes between the scale rows of consecutive tokens (GATHER)
 };
 
 // Source row of the fused gather: row `tok` of A, or of the owning rank's token buffer in expert-parallel mode.
@@ -108,6 +114,11 @@ enum { EPI_BF16 = 0, EPI_SWIGLU = 1, EPI_F32 = 2 };
 cudaError_t launch_gemm_tc(const GemmArgs& a, int epi, int grid, cudaStream_t s);
 cudaError_t launch_gemm_tn(const GemmArgs& a, int epi, int grid, cudaStream_t s);   // tokens on the MMA's N side
 cudaError_t launch_gemm_m2(const GemmArgs& a, int epi, int grid, cudaStream_t s);   // 256-row tiles, two accumulators
+cudaError_t launch_gemm_mx(const GemmArgs& a, int epi, int grid, cudaStream_t s);   // MXFP8 operands, block-scaled MMA
+cudaError_t launch_mx_quantize_rows(const __nv_bfloat16* in, long long rows, int K, uint8_t* codes, uint8_t* scales,
+                                    cudaStream_t s);
+cudaError_t launch_mx_quantize_atoms(const __nv_bfloat16* in, int groups, int rows_per_group, int K, uint8_t* codes,
+                                     uint8_t* scales, cudaStream_t s);
 cudaError_t launch_router_tc(const __nv_bfloat16* x, const float* Wr, const float* bias, int T, int H, int E, int k,
                              const WsLayout& L, char* ws, WsHeader* hdr, int grid, int tile_m, int variant, int32_t* idx,
                              float* w,

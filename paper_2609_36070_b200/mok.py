@@ -22,7 +22,9 @@ MOK_IMPL_TCGEN05, MOK_IMPL_SIMT, MOK_IMPL_TCGEN05_TN = 0, 1, 2
 EXPORTS = ["mok_moe_forward", "mok_workspace_bytes", "mok_moe_forward_ex", "mok_moe_forward_host", "mok_route",
            "mok_schedule", "mok_read_status", "mok_launch_count", "mok_last_cuda_error", "mok_status_string",
            "mok_version", "mok_profile_begin", "mok_profile_end", "mok_schedule_noalloc", "mok_debug_counters",
-           "mok_ep_workspace_bytes", "mok_ep_y_rows", "mok_ep_expert_ffn", "mok_ep_combine"]
+           "mok_ep_workspace_bytes", "mok_ep_y_rows", "mok_ep_expert_ffn", "mok_ep_combine",
+           "mok_mx_scale_bytes", "mok_mx_quantize_weights", "mok_mx_quantize_rows", "mok_mx_workspace_bytes"]
+MOK_PRECISION_BF16, MOK_PRECISION_MXFP8 = 0, 1
 MOK_MAX_RANKS = 16
 MOK_NOALLOC_MAX_ROUTES = 32768
 MOK_DEBUG_STARVE = 2
@@ -32,7 +34,7 @@ STAGES = ["router", "schedule", "gather", "gemm1", "gemm2", "shared_gemm1", "sha
 class mok_config(ctypes.Structure):
     _fields_ = [("impl", ctypes.c_int32), ("grid", ctypes.c_int32), ("router_impl", ctypes.c_int32),
                 ("profile", ctypes.c_int32), ("gather_mode", ctypes.c_int32), ("cta_group", ctypes.c_int32),
-                ("debug", ctypes.c_int32), ("host_chunks", ctypes.c_int32)]
+                ("debug", ctypes.c_int32), ("host_chunks", ctypes.c_int32), ("precision", ctypes.c_int32)]
 
 
 class mok_args(ctypes.Structure):
@@ -44,7 +46,9 @@ class mok_args(ctypes.Structure):
                 ("out", ctypes.c_void_p), ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
                 ("topk_idx", ctypes.c_void_p), ("topk_w", ctypes.c_void_p), ("counts", ctypes.c_void_p),
                 ("offsets", ctypes.c_void_p), ("perm", ctypes.c_void_p), ("inv_perm", ctypes.c_void_p),
-                ("config", ctypes.POINTER(mok_config)), ("stream", ctypes.c_void_p)]
+                ("config", ctypes.POINTER(mok_config)), ("stream", ctypes.c_void_p),
+                ("W_gate_up_codes", ctypes.c_void_p), ("W_gate_up_scales", ctypes.c_void_p),
+                ("W_down_codes", ctypes.c_void_p), ("W_down_scales", ctypes.c_void_p)]
 
 
 class mok_ep_args(ctypes.Structure):
@@ -80,6 +84,14 @@ _lib.mok_ep_combine.restype = ctypes.c_int
 _lib.mok_ep_combine.argtypes = [ctypes.POINTER(mok_ep_combine_args)]
 _lib.mok_workspace_bytes.restype = ctypes.c_size_t
 _lib.mok_workspace_bytes.argtypes = [ctypes.c_int] * 6
+_lib.mok_mx_workspace_bytes.restype = ctypes.c_size_t
+_lib.mok_mx_workspace_bytes.argtypes = [ctypes.c_int] * 6
+_lib.mok_mx_scale_bytes.restype = ctypes.c_size_t
+_lib.mok_mx_scale_bytes.argtypes = [ctypes.c_int] * 3
+_lib.mok_mx_quantize_weights.restype = ctypes.c_int
+_lib.mok_mx_quantize_weights.argtypes = [ctypes.c_void_p] + [ctypes.c_int] * 3 + [ctypes.c_void_p] * 3
+_lib.mok_mx_quantize_rows.restype = ctypes.c_int
+_lib.mok_mx_quantize_rows.argtypes = [ctypes.c_void_p] + [ctypes.c_int] * 2 + [ctypes.c_void_p] * 3
 _lib.mok_moe_forward.restype = ctypes.c_int
 _lib.mok_moe_forward.argtypes = [ctypes.c_void_p] * 6 + [ctypes.c_int] * 6 + [ctypes.c_void_p] * 2
 _lib.mok_moe_forward_ex.restype = ctypes.c_int
@@ -134,8 +146,10 @@ def _stream(stream):
     return ctypes.c_void_p(stream.cuda_stream)
 
 
-def _config(impl=0, grid=0, router_impl=0, profile=0, gather_mode=0, cta_group=0, debug=0, host_chunks=0):
+def _config(impl=0, grid=0, router_impl=0, profile=0, gather_mode=0, cta_group=0, debug=0, host_chunks=0,
+            precision=0):
     c = mok_config()
+    c.precision = precision
     c.impl, c.grid, c.router_impl, c.profile, c.gather_mode = impl, grid, router_impl, profile, gather_mode
     c.cta_group = cta_group
     c.debug = debug
@@ -171,9 +185,45 @@ def mok_launch_count(T, H, I, I_shared, E, k):
     return int(_lib.mok_launch_count(T, H, I, I_shared, E, k, None))
 
 
-def alloc_workspace(T, H, I, I_shared, E, k, device="cuda", host_staging=False):
-    """A torch uint8 buffer large enough for mok_moe_forward_ex (plus the x/out staging copies of the host variant)."""
-    n = mok_workspace_bytes(T, H, I, I_shared, E, k)
+def mok_mx_workspace_bytes(T, H, I, I_shared, E, k):
+    return int(_lib.mok_mx_workspace_bytes(T, H, I, I_shared, E, k))
+
+
+class MxWeights:
+    """The routed weights pre-quantised to MXFP8 by the library's quantisation kernel (Section 3.4)."""
+
+    def __init__(self, W_gate_up, W_down, stream=None):
+        E, twoI, H = W_gate_up.shape
+        I = twoI // 2
+        self.gate_up_codes, self.gate_up_scales = mok_mx_quantize_weights(W_gate_up.view(2 * E, I, H), stream)
+        self.down_codes, self.down_scales = mok_mx_quantize_weights(W_down, stream)
+
+
+def mok_mx_quantize_weights(W, stream=None):
+    """W bf16 [groups, rows, K] -> (codes uint8 [groups, rows, K], scales uint8 in the MMA's atom layout)."""
+    groups, rows, K = W.shape
+    n = int(_lib.mok_mx_scale_bytes(groups, rows, K))
+    if n == 0:
+        raise MokError(MOK_ERR_SHAPE)
+    codes = torch.empty((groups, rows, K), dtype=torch.uint8, device=W.device)
+    scales = torch.empty((n,), dtype=torch.uint8, device=W.device)
+    _check(_lib.mok_mx_quantize_weights(_p(W), groups, rows, K, _p(codes), _p(scales), _stream(stream)))
+    return codes, scales
+
+
+def mok_mx_quantize_rows(x, stream=None):
+    """x bf16 [rows, K] -> (codes uint8 [rows, K], scales uint8 [rows, 4 * ceil(K / 128)])."""
+    rows, K = x.shape
+    codes = torch.empty((rows, K), dtype=torch.uint8, device=x.device)
+    scales = torch.empty((rows, (K + 127) // 128 * 4), dtype=torch.uint8, device=x.device)
+    _check(_lib.mok_mx_quantize_rows(_p(x), rows, K, _p(codes), _p(scales), _stream(stream)))
+    return codes, scales
+
+
+def alloc_workspace(T, H, I, I_shared, E, k, device="cuda", host_staging=False, mx=False):
+    """A torch uint8 buffer large enough for mok_moe_forward_ex (plus the x/out staging copies of the host variant;
+    mx=True: plus the MXFP8 mode's quantised activations)."""
+    n = (mok_mx_workspace_bytes if mx else mok_workspace_bytes)(T, H, I, I_shared, E, k)
     if n == 0:
         raise MokError(MOK_ERR_SHAPE)
     if host_staging:
@@ -233,7 +283,7 @@ def _fill_args(x_shape, W_router, router_bias, W_gate_up, W_down, W_shared_gate_
 
 
 def mok_moe_forward_ex(x, W_router, router_bias, W_gate_up, W_down, W_shared_gate_up, W_shared_down, k, workspace,
-                       out=None, stages=False, config=None, stream=None):
+                       out=None, stages=False, config=None, stream=None, mx_weights=None):
     """The layer with router bias, caller-owned workspace, optional stage outputs and knobs.
 
     Returns out, or (out, dict of stage tensors) when stages=True.
@@ -243,6 +293,9 @@ def mok_moe_forward_ex(x, W_router, router_bias, W_gate_up, W_down, W_shared_gat
     a, res = _fill_args(x.shape, W_router, router_bias, W_gate_up, W_down, W_shared_gate_up, W_shared_down, k,
                         workspace, stages, config, stream, x.device)
     a.x, a.out = x.data_ptr(), out.data_ptr()
+    if mx_weights is not None:
+        a.W_gate_up_codes, a.W_gate_up_scales = mx_weights.gate_up_codes.data_ptr(), mx_weights.gate_up_scales.data_ptr()
+        a.W_down_codes, a.W_down_scales = mx_weights.down_codes.data_ptr(), mx_weights.down_scales.data_ptr()
     _check(_lib.mok_moe_forward_ex(ctypes.byref(a)))
     return (out, res) if stages else out
 
