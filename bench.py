@@ -43,6 +43,8 @@ def parse():
     p.add_argument("--cta-group", type=int, default=0, help="0 default, 1 single CTAs, 2 CTA pairs")
     p.add_argument("--gemm", type=int, default=0, help="0 tcgen05 (tokens on M), 2 tcgen05 (tokens on N), 1 SIMT")
     p.add_argument("--host-chunks", type=int, default=0, help="token chunks of the host-buffer call (0 = auto)")
+    p.add_argument("--precision", default="bf16", choices=["bf16", "mxfp8"],
+                   help="routed experts in bf16 (the headline workload) or MXFP8 with pre-quantised weights")
     return p.parse_args()
 
 
@@ -196,13 +198,16 @@ def main():
     g = {k: (None if d[k] is None else mok.to_device_bf16(d[k], dev)) for k in ("x", "W_gate_up", "W_down", "W_sgu", "W_sd")}
     W_r = torch.from_numpy(d["W_r"]).to(dev)
     bias = None if d["bias"] is None else torch.from_numpy(d["bias"]).to(dev)
-    ws = mok.alloc_workspace(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k, device=dev, host_staging=True)
+    mx = args.precision == "mxfp8"
+    prec = mok.MOK_PRECISION_MXFP8 if mx else mok.MOK_PRECISION_BF16
+    mxw = mok.MxWeights(g["W_gate_up"], g["W_down"]) if mx else None    # weights are quantised ahead of time
+    ws = mok.alloc_workspace(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k, device=dev, host_staging=True, mx=mx)
     out = torch.empty_like(g["x"])
-    conf = mok._config(impl=args.gemm, profile=1, gather_mode=args.gather_mode, cta_group=args.cta_group)
+    conf = mok._config(impl=args.gemm, profile=1, gather_mode=args.gather_mode, cta_group=args.cta_group, precision=prec)
 
     def step():
         mok.mok_moe_forward_ex(g["x"], W_r, bias, g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], cfg.k, ws,
-                               out=out, config=conf)
+                               out=out, config=conf, mx_weights=mxw)
 
     def barrier():
         if dist is not None:
@@ -241,11 +246,12 @@ def main():
     # end to end through the host-buffer entry point: pinned host x -> device, layer, result -> pinned host
     xh = g["x"].cpu().pin_memory()
     oh = torch.empty_like(xh).pin_memory()
-    conf0 = mok._config(impl=args.gemm, gather_mode=args.gather_mode, cta_group=args.cta_group, host_chunks=args.host_chunks)
+    conf0 = mok._config(impl=args.gemm, gather_mode=args.gather_mode, cta_group=args.cta_group, host_chunks=args.host_chunks,
+                        precision=prec)
 
     def e2e_step():
         mok.mok_moe_forward_host(xh, oh, W_r, bias, g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], cfg.k, ws,
-                                 config=conf0)
+                                 config=conf0, mx_weights=mxw)
 
     e2e_steps = max(5, min(args.steps, 50))
     for _ in range(3):
@@ -271,12 +277,14 @@ def main():
     g1_flops = 4.0 * cfg.T * cfg.k * cfg.H * cfg.I
     g1_tflops = g1_flops / (mean["gemm1"] * 1e-3) / 1e12
     peak_tf = pk.get("bf16_tflops_sustained", pk["bf16_tflops"])
+    if mx:   # fp8 tensor peak = the measured bf16 peak x the nominal 2:1 ratio (4.5 vs 2.25 PFLOP/s dense)
+        peak_tf *= 2.0
     per_step = sorted(sum(c[s] for s in mok.STAGES) for c in stage)
     ffn_ms = mean["gemm1"] + mean["gemm2"] + mean["shared_gemm1"] + mean["shared_gemm2"]
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16", "data": "synthetic",
+        "dtype": "mxfp8 routed experts (fp32 accumulate), bf16 elsewhere" if mx else "bf16", "data": "synthetic",
         "config": {"workload": cfg.name, "T": cfg.T, "H": cfg.H, "E": cfg.E, "k": cfg.k, "I": cfg.I,
                    "I_shared": cfg.I_s, "routing": cfg.bias, "parallelism": f"token-sharded replicas x{world}",
                    "l2": "inputs larger than L2 (weights + activations >> 126 MB), no explicit flush"},
@@ -288,14 +296,16 @@ def main():
         "stage_ms": mean,
         "median_step_ms_from_stage_events": per_step[len(per_step) // 2],
         "inputs": fingerprints(d),
-        "roofline": {"kernel": "routed gate/up grouped GEMM + SwiGLU, token gather fused (gemm_m2_kernel<EPI_SWIGLU, GATHER>)",
+        "roofline": {"kernel": ("routed gate/up grouped GEMM on MXFP8 operands + SwiGLU + activation quantisation, token gather fused "
+                                "(gemm_mx_kernel<EPI_SWIGLU, GATHER>)") if mx else
+                               "routed gate/up grouped GEMM + SwiGLU, token gather fused (gemm_m2_kernel<EPI_SWIGLU, GATHER>)",
                      "bound": "tensor",
                      "achieved": g1_tflops, "peak": peak_tf, "unit": "TFLOP/s", "frac": g1_tflops / peak_tf,
-                     "peak_source": f"{pk['source']} bf16_tflops_sustained",
-                     "traffic": NCU_TRAFFIC_BYTES.get(cfg.name)},
+                     "peak_source": f"{pk['source']} bf16_tflops_sustained" + (" x 2 (nominal fp8 : bf16 ratio)" if mx else ""),
+                     "traffic": None if mx else NCU_TRAFFIC_BYTES.get(cfg.name)},
         "e2e": {"value": world * cfg.T / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": act_bytes, "d2h_bytes_per_step": act_bytes},
-        "gpu_launches": args.steps * mok.mok_launch_count(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k),
+        "gpu_launches": args.steps * mok.mok_launch_count(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k, conf),
         "clocks": clocks,
     }
     if not args.no_cpu_baseline:

@@ -36,16 +36,18 @@ using namespace tc;
 constexpr int BM = 128, BN = 256, BKB = 128;   // BKB: bytes = elements of K per stage (four K = 32 MMAs)
 constexpr int A_BYTES = BM * BKB;              // 16 KB
 constexpr int B_BYTES = BN * BKB;              // 32 KB
-constexpr int SFA_OFF = A_BYTES + B_BYTES;     // 512-byte atom of the A rows
-constexpr int SFB_OFF = SFA_OFF + 512;         // two atoms of the B rows
-constexpr int STAGE_BYTES = 51200;             // 50 KB: keeps every stage 1024-byte aligned for the swizzled tiles
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES; // 48 KB of swizzled operand tiles (1024-byte aligned)
 constexpr int STAGES = 4;
+constexpr int SF_BYTES = 1536;                 // per stage: the A rows' scale atom (512 bytes) + the B rows' two
+constexpr int SF_REGION = STAGES * STAGE_BYTES;
+constexpr int SLAB_BYTES = 2048;               // per epilogue warp: 32 rows x 32 bf16 columns, for coalesced stores
+constexpr int SLAB_REGION = SF_REGION + STAGES * SF_BYTES;
 constexpr int TMEM_COLS = 512, SF_COL0 = BN, SF_COLS = 12;   // per stage: 4 columns for A's atom, 8 for B's two
 constexpr int EPI_WARPS = 8;
 constexpr int THREADS = 64 + 32 * EPI_WARPS;   // + 4 gather warps in the GATHER instantiation
 constexpr int GATHER_THREADS = 128;
 constexpr int SMEM_CTRL = 256;
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + SMEM_CTRL + 1024;
+constexpr int SMEM_BYTES = SLAB_REGION + EPI_WARPS * SLAB_BYTES + SMEM_CTRL + 1024;
 
 struct Ctrl {
     uint64_t full[STAGES];
@@ -111,7 +113,7 @@ gemm_mx_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t* smem = smem_raw + (base - raw);
-    Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem + STAGES * STAGE_BYTES);
+    Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem + SLAB_REGION + EPI_WARPS * SLAB_BYTES);
     volatile uint32_t* abort_flag = &ctrl->abort;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -165,15 +167,16 @@ gemm_mx_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
                     if (!ok) break;
                     const uint32_t full = smem_u32(&ctrl->full[s]);
                     const uint32_t sa = base + s * STAGE_BYTES, sb = sa + A_BYTES;
+                    const uint32_t sf = base + SF_REGION + s * SF_BYTES;
                     mbar_expect_tx(full, B_BYTES + 1024 + (GATHER ? 0 : A_BYTES + 512));
                     if (!GATHER) {
                         tma_load_2d(sa, &tmapA, full, kb * BKB, t.row0);
-                        bulk_load(sa + SFA_OFF, sfa + (size_t)kb * 512, 512, full);
+                        bulk_load(sf, sfa + (size_t)kb * 512, 512, full);
                     }
                     tma_load_2d(sb, &tmapB, full, kb * BKB, brow0);
                     tma_load_2d(sb + B_BYTES / 2, &tmapB, full, kb * BKB, brow1);
-                    bulk_load(sa + SFB_OFF, sfb0 + (size_t)kb * 512, 512, full);
-                    bulk_load(sa + SFB_OFF + 512, sfb1 + (size_t)kb * 512, 512, full);
+                    bulk_load(sf + 512, sfb0 + (size_t)kb * 512, 512, full);
+                    bulk_load(sf + 1024, sfb1 + (size_t)kb * 512, 512, full);
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
                 if (!ok) break;
@@ -196,9 +199,10 @@ gemm_mx_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
                     tc_fence_after();
                     const uint32_t sa = base + s * STAGE_BYTES, sb = sa + A_BYTES;
                     const uint32_t sf_tmem = tmem_base + (uint32_t)(SF_COL0 + s * SF_COLS);
-                    tc_cp_sf(sf_tmem, make_sf_desc(sa + SFA_OFF));
-                    tc_cp_sf(sf_tmem + 4, make_sf_desc(sa + SFB_OFF));
-                    tc_cp_sf(sf_tmem + 8, make_sf_desc(sa + SFB_OFF + 512));
+                    const uint32_t sf = base + SF_REGION + s * SF_BYTES;
+                    tc_cp_sf(sf_tmem, make_sf_desc(sf));
+                    tc_cp_sf(sf_tmem + 4, make_sf_desc(sf + 512));
+                    tc_cp_sf(sf_tmem + 8, make_sf_desc(sf + 1024));
                     const uint64_t adesc = make_smem_desc(sa), bdesc = make_smem_desc(sb);
 #pragma unroll
                     for (int j = 0; j < 4; ++j)               // +32 bytes per K = 32 step inside the 128-byte swizzle row
@@ -236,7 +240,7 @@ gemm_mx_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
             }
             const int tokq = (q < valid) ? __ldg(rows + q) : tok0;
             const uint8_t* sfsrc = a.sfa + (size_t)tokq * a.sfa_stride;
-            const uint32_t sfdst = SFA_OFF + (q & 31) * 16 + (q >> 5) * 4;
+            const uint32_t sfdst = base + SF_REGION + (q & 31) * 16 + (q >> 5) * 4;
             bool ok = true;
             for (int kb = 0; kb < k_blocks; ++kb) {
                 ok = mbar_wait(smem_u32(&ctrl->empty[s]), ph ^ 1u, abort_flag, a.header, 5);
@@ -250,7 +254,7 @@ gemm_mx_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
                     const uint32_t dst = sa + r * 128 + ((chunk ^ (r & 7)) << 4);
                     cp_async_16(dst, in_k ? (const void*)(src[i] + kb * BKB) : (const void*)xq, in_k ? 16u : 0u);
                 }
-                cp_async_4(sa + sfdst, sfsrc + kb * 4);
+                cp_async_4(sfdst + s * SF_BYTES, sfsrc + kb * 4);
                 cp_async_mbar_arrive(smem_u32(&ctrl->full[s]));
                 if (++s == STAGES) { s = 0; ph ^= 1u; }
             }
@@ -328,14 +332,30 @@ gemm_mx_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&ctrl->tempty));
-                __nv_bfloat16* crow = reinterpret_cast<__nv_bfloat16*>(a.C) + (size_t)row * a.ldc;
+                // Transpose through this warp's slab so that each store instruction writes whole 64-byte row segments
+                // of 8 rows (full 32-byte sectors) instead of 16 bytes in each of 32 different rows.
+                const uint32_t slab = base + SLAB_REGION + (warp - 2) * SLAB_BYTES;
+                const int rr = lane >> 2, seg = lane & 3;            // read side: row within a group of 8, 16-byte segment
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                     const int col = t.n * BN + hh * 128 + c * 32;
+                    __syncwarp();
 #pragma unroll
                     for (int v = 0; v < 4; ++v)
-                        if (col + v * 8 < a.N)
-                            *reinterpret_cast<uint4*>(crow + col + v * 8) = make_uint4(o[c][4 * v], o[c][4 * v + 1], o[c][4 * v + 2], o[c][4 * v + 3]);
+                        st_shared_v4(slab + lane * 64 + ((v ^ ((lane >> 1) & 3)) << 4), o[c][4 * v], o[c][4 * v + 1], o[c][4 * v + 2], o[c][4 * v + 3]);
+                    __syncwarp();
+                    if (col + seg * 8 < a.N) {
+#pragma unroll
+                        for (int it = 0; it < 4; ++it) {
+                            const int r = it * 8 + rr;
+                            uint4 val;
+                            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                                         : "=r"(val.x), "=r"(val.y), "=r"(val.z), "=r"(val.w)
+                                         : "r"(slab + r * 64 + ((seg ^ ((r >> 1) & 3)) << 4)));
+                            __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(a.C) + (size_t)(t.row0 + quad * 32 + r) * a.ldc + col + seg * 8;
+                            *reinterpret_cast<uint4*>(dst) = val;
+                        }
+                    }
                 }
             }
         }

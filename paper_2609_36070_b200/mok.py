@@ -181,8 +181,8 @@ def mok_workspace_bytes(T, H, I, I_shared, E, k):
     return int(_lib.mok_workspace_bytes(T, H, I, I_shared, E, k))
 
 
-def mok_launch_count(T, H, I, I_shared, E, k):
-    return int(_lib.mok_launch_count(T, H, I, I_shared, E, k, None))
+def mok_launch_count(T, H, I, I_shared, E, k, config=None):
+    return int(_lib.mok_launch_count(T, H, I, I_shared, E, k, None if config is None else ctypes.pointer(config)))
 
 
 def mok_mx_workspace_bytes(T, H, I, I_shared, E, k):
@@ -301,11 +301,14 @@ def mok_moe_forward_ex(x, W_router, router_bias, W_gate_up, W_down, W_shared_gat
 
 
 def mok_moe_forward_host(x_host, out_host, W_router, router_bias, W_gate_up, W_down, W_shared_gate_up, W_shared_down,
-                         k, workspace, config=None, stream=None):
+                         k, workspace, config=None, stream=None, mx_weights=None):
     """Host-buffer variant: x_host / out_host are CPU (ideally pinned) bf16 tensors; blocks until out_host is filled."""
     assert not x_host.is_cuda and not out_host.is_cuda
     a, _ = _fill_args(x_host.shape, W_router, router_bias, W_gate_up, W_down, W_shared_gate_up, W_shared_down, k,
                       workspace, False, config, stream, W_router.device)
+    if mx_weights is not None:
+        a.W_gate_up_codes, a.W_gate_up_scales = mx_weights.gate_up_codes.data_ptr(), mx_weights.gate_up_scales.data_ptr()
+        a.W_down_codes, a.W_down_scales = mx_weights.down_codes.data_ptr(), mx_weights.down_scales.data_ptr()
     _check(_lib.mok_moe_forward_host(ctypes.byref(a), ctypes.c_void_p(x_host.data_ptr()),
                                      ctypes.c_void_p(out_host.data_ptr())))
     return out_host

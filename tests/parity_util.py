@@ -99,3 +99,33 @@ def full_parity(cfg, d=None, g=None, n_sample=None, config=None):
     tokens = np.arange(cfg.T, dtype=np.int32) if n_sample is None else inputs.sample_tokens(cfg, idx, n_sample)
     rep.update(check_output(cfg, d, out, idx, w, tokens))
     return out, st, rep
+
+
+def mx_parity(cfg, d=None, g=None, n_sample=None, config_kw=None):
+    """Parity of the MXFP8 mode (routed experts quantised, Section 3.4) against the oracle's fp64 evaluation of the
+    same quantised definition.  Routing and schedule as in bf16 mode; outputs within the layer's tolerances."""
+    from paper_2609_36070_b200 import mok as m
+    d = d if d is not None else inputs.make_inputs(cfg)
+    g = g if g is not None else upload(d)
+    mxw = m.MxWeights(g["W_gate_up"], g["W_down"])
+    ws = m.alloc_workspace(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k, mx=True)
+    conf = m._config(precision=m.MOK_PRECISION_MXFP8, **(config_kw or {}))
+    out, st = m.mok_moe_forward_ex(g["x"], g["W_r"], g["bias"], g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"],
+                                   cfg.k, ws, stages=True, config=conf, mx_weights=mxw)
+    status = m.mok_read_status(ws)
+    assert status == 0, m.mok_status_string(status)
+    idx, w, rep = check_routing_and_schedule(cfg, d, st)
+    Wgu_q, Wd_q = mok_ref.mx_roundtrip_bf16(d["W_gate_up"]), mok_ref.mx_roundtrip_bf16(d["W_down"])
+    tokens = np.arange(cfg.T, dtype=np.int32) if n_sample is None else inputs.sample_tokens(cfg, idx, n_sample)
+    ref = mok_ref.ffn_tokens_mx(d["x"], Wgu_q, Wd_q, d["W_sgu"], d["W_sd"], idx, w, tokens)
+    got = bf16_to_f64(out[torch.from_numpy(np.asarray(tokens, np.int64)).to(out.device)])
+    diff = np.abs(got - ref)
+    rep["max_rel"] = float(diff.max() / np.abs(ref).max())
+    rep["mean_rel"] = float(diff.mean() / np.abs(ref).mean())
+    # distance to the unquantised layer, for the record: MXFP8 is expected to sit a few per cent away from it
+    plain = mok_ref.ffn_tokens(d["x"], d["W_gate_up"], d["W_down"], d["W_sgu"], d["W_sd"], idx, w, tokens)
+    rep["mean_rel_to_bf16_definition"] = float(np.abs(got - plain).mean() / np.abs(plain).mean())
+    rep["tokens_checked"] = int(len(tokens))
+    assert np.isfinite(got).all()
+    assert rep["max_rel"] <= MAX_REL and rep["mean_rel"] <= MEAN_REL, rep
+    return out, rep

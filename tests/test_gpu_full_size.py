@@ -30,6 +30,18 @@ def test_full_size_sampled(name):
     torch.cuda.empty_cache()
 
 
+def test_full_size_mxfp8_sampled():
+    """The benchmark workload with the routed experts in MXFP8 (Section 3.4), against the oracle's quantised layer."""
+    cfg = inputs.CONFIGS["qwen3_30b_a3b"]
+    d = inputs.make_inputs(cfg)
+    g = pu.upload(d)
+    out, rep = pu.mx_parity(cfg, d=d, g=g, n_sample=256)
+    print(cfg.name, "mxfp8", rep)
+    del d, g, out
+    gc.collect()
+    torch.cuda.empty_cache()
+
+
 def test_deepseek_v3_full_and_small_token_sweep():
     """The largest workload (about 23 GB of expert weights resident) and its small-T sweep with the same weights."""
     cfg = inputs.CONFIGS["deepseek_v3"]

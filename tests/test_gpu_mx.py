@@ -62,30 +62,7 @@ def test_row_quantiser_matches_oracle(rows, K):
 
 
 def mx_case(cfg, config_kw=None):
-    m = mok()
-    d = inputs.make_inputs(cfg)
-    g = pu.upload(d)
-    mxw = m.MxWeights(g["W_gate_up"], g["W_down"])
-    ws = m.alloc_workspace(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k, mx=True)
-    conf = m._config(precision=m.MOK_PRECISION_MXFP8, **(config_kw or {}))
-    out, st = m.mok_moe_forward_ex(g["x"], g["W_r"], g["bias"], g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"],
-                                   cfg.k, ws, stages=True, config=conf, mx_weights=mxw)
-    status = m.mok_read_status(ws)
-    assert status == 0, m.mok_status_string(status)
-    idx, w, rep = pu.check_routing_and_schedule(cfg, d, st)
-    Wgu_q, Wd_q = mok_ref.mx_roundtrip_bf16(d["W_gate_up"]), mok_ref.mx_roundtrip_bf16(d["W_down"])
-    tokens = np.arange(cfg.T, dtype=np.int32)
-    ref = mok_ref.ffn_tokens_mx(d["x"], Wgu_q, Wd_q, d["W_sgu"], d["W_sd"], idx, w, tokens)
-    got = pu.bf16_to_f64(out)
-    diff = np.abs(got - ref)
-    rep["max_rel"] = float(diff.max() / np.abs(ref).max())
-    rep["mean_rel"] = float(diff.mean() / np.abs(ref).mean())
-    # distance to the unquantised layer, for the record: MXFP8 is expected to sit a few per cent away
-    plain = mok_ref.ffn_tokens(d["x"], d["W_gate_up"], d["W_down"], d["W_sgu"], d["W_sd"], idx, w, tokens)
-    rep["mean_rel_to_bf16_definition"] = float(np.abs(got - plain).mean() / np.abs(plain).mean())
-    assert np.isfinite(got).all()
-    assert rep["max_rel"] <= pu.MAX_REL and rep["mean_rel"] <= pu.MEAN_REL, rep
-    return out, rep
+    return pu.mx_parity(cfg, config_kw=config_kw)
 
 
 MX_SHAPES = [
