@@ -88,6 +88,8 @@ bool ws_layout(int T, int H, int I, int Is, int E, int k, WsLayout* L, bool mx) 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 static bool use_mx(const mok_config* cfg) { return cfg && cfg->precision == MOK_PRECISION_MXFP8; }
+// MXFP8 GEMMs on CTA pairs (each CTA stages half of the weight tile): cta_group = 2 asks for them, 1 for single CTAs.
+static bool mx_pairs(const mok_config* cfg) { return cfg && cfg->cta_group == 2; }
 
 static int validate(const mok_args* a, WsLayout* L, size_t extra_ws) {
     if (!a) return MOK_ERR_NULL;
@@ -261,6 +263,12 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
     if (mx) {
         // routed experts on MXFP8 operands (Section 3.4): h = Q(silu(Q(x) Wg_q^T) * (Q(x) Wu_q^T));  y = h Wd_q^T
         const int grid = a->config->grid;
+        if (mx_pairs(a->config)) {   // CTA pairs on the 256-row tile table (over the same 128-row-padded row space)
+            g.tile_m = 2 * TILE_M;
+            g.n_mtiles = &hdr->n_mtiles2;
+            g.mt_start = reinterpret_cast<const int32_t*>(ws + L.mt_start2);
+            g.tile_expert = reinterpret_cast<const int32_t*>(ws + L.tile_expert2);
+        }
         g.A = reinterpret_cast<const __nv_bfloat16*>(ws + L.x8);
         g.a_rows = a->T;
         g.row_token = reinterpret_cast<const int32_t*>(ws + L.row_token);
@@ -277,6 +285,7 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
         MOK_MARK(MOK_STAGE_GEMM1 + 1);
         g.row_token = nullptr;
         g.starve = 0;
+        g.dbg_slot = dbg ? 2 : -1;
         g.A = reinterpret_cast<const __nv_bfloat16*>(ws + L.h8);
         g.a_rows = L.Rpad;
         g.sfa = reinterpret_cast<const uint8_t*>(ws + L.sh);
@@ -288,6 +297,10 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
         e = launch_gemm_mx(g, EPI_BF16, grid, s);
         if (e != cudaSuccess) return cuda_fail(e);
         g.sfa = g.sfb = nullptr;
+        g.tile_m = tile_m;
+        g.n_mtiles = &hdr->n_mtiles;
+        g.mt_start = reinterpret_cast<const int32_t*>(ws + L.mt_start);
+        g.tile_expert = reinterpret_cast<const int32_t*>(ws + L.tile_expert);
     } else {
         // routed experts: h = silu(Xg Wg^T) * (Xg Wu^T);  y = h Wd^T
         if (simt) {

@@ -14,13 +14,14 @@ struct Tile { int row0, n, e, m; };   // row0: first row of the (pair) tile in t
 // L2 while the expert's weight tiles stream.
 __device__ __forceinline__ Tile decode_tile(const GemmArgs& a, int L, int n_nt, int n_mt_total, int tm) {
     Tile t;
-    int mt0, m_cnt;
+    int mt0, m_cnt, pad0;
     if (a.dense_rows > 0) {
-        t.e = 0; mt0 = 0; m_cnt = n_mt_total;
+        t.e = 0; mt0 = 0; m_cnt = n_mt_total; pad0 = 0;
     } else {
         t.e = __ldg(a.tile_expert + L / n_nt);
         mt0 = __ldg(a.mt_start + t.e);
         m_cnt = __ldg(a.mt_start + t.e + 1) - mt0;
+        pad0 = __ldg(a.pad_offsets + t.e);
     }
     const int group_m = GROUP_ROWS / tm;
     const int r = L - n_nt * mt0;
@@ -30,7 +31,9 @@ __device__ __forceinline__ Tile decode_tile(const GemmArgs& a, int L, int n_nt, 
     const int in_group = min(group_m, m_cnt - g * group_m);
     t.n = rem / in_group;
     t.m = g * group_m + (rem - t.n * in_group);
-    t.row0 = (mt0 + t.m) * tm;
+    // first row in the padded row space: the expert's segment start (a multiple of the padding granularity, which
+    // may be finer than the tile: 256-row pair tiles over 128-row padding) plus whole tiles
+    t.row0 = pad0 + t.m * tm;
     return t;
 }
 

@@ -76,16 +76,18 @@ MX_SHAPES = [
 ]
 
 
+@pytest.mark.parametrize("cta_group", [1, 2], ids=["single_cta", "cta_pairs"])
 @pytest.mark.parametrize("name,T,H,E,k,I,I_s,bias", MX_SHAPES)
-def test_mx_layer_parity(name, T, H, E, k, I, I_s, bias):
+def test_mx_layer_parity(name, T, H, E, k, I, I_s, bias, cta_group):
     cfg = inputs.MoEConfig("mx_" + name, T, H, E, k, I, I_s, bias=bias, seed=31)
-    out, rep = mx_case(cfg)
-    print(name, rep)
+    out, rep = mx_case(cfg, {"cta_group": cta_group})
+    print(name, cta_group, rep)
 
 
 def test_mx_layer_is_reproducible_and_grid_independent():
     cfg = inputs.MoEConfig("mx_repro", 768, 256, 16, 4, 256, 0, bias="zipf", seed=32)
-    runs = [mx_case(cfg, kw)[0].view(torch.int16).clone() for kw in (None, None, {"grid": 1}, {"grid": 7})]
+    runs = [mx_case(cfg, kw)[0].view(torch.int16).clone()
+            for kw in (None, None, {"grid": 1}, {"grid": 7}, {"cta_group": 2}, {"cta_group": 2, "grid": 6})]
     for r in runs[1:]:
         assert torch.equal(r, runs[0])
 
