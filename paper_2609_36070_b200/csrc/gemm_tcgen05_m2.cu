@@ -158,8 +158,10 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
                 const Tile t = decode_tile(a, L, n_nt, n_mt_total);
                 const bool two = t.valid > BM;
                 long long w0 = dbg ? clock64() : 0;
+                // Accumulator 0 is needed now, accumulator 1 only after the first k-block's MMAs into accumulator 0; and
+                // accumulator 0 is published before the last k-block's MMAs into accumulator 1 are issued.  Each
+                // accumulator's epilogue thus gets one k-block (512 tensor-pipe cycles) more to drain.
                 bool ok = mbar_wait(smem_u32(&ctrl->tempty[0]), ap0 ^ 1u, abort_flag, a.header, 2);
-                if (ok && two) ok = mbar_wait(smem_u32(&ctrl->tempty[1]), ap1 ^ 1u, abort_flag, a.header, 8);
                 if (dbg) d_tempty += clock64() - w0;
                 if (!ok) break;
                 tc_fence_after();
@@ -176,7 +178,15 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
 #pragma unroll
                     for (int j = 0; j < BK / UMMA_K; ++j)
                         tc_mma<1>(d0, a0 + (uint64_t)(j * 2), bd + (uint64_t)(j * 2), IDESC, (kb | j) ? 1u : 0u);
+                    if (kb == k_blocks - 1) { tc_commit<1>(smem_u32(&ctrl->tfull[0])); ap0 ^= 1u; }
                     if (two) {
+                        if (kb == 0) {
+                            if (dbg) w0 = clock64();
+                            ok = mbar_wait(smem_u32(&ctrl->tempty[1]), ap1 ^ 1u, abort_flag, a.header, 8);
+                            if (dbg) d_tempty += clock64() - w0;
+                            if (!ok) break;
+                            tc_fence_after();
+                        }
 #pragma unroll
                         for (int j = 0; j < BK / UMMA_K; ++j)
                             tc_mma<1>(d1, a1 + (uint64_t)(j * 2), bd + (uint64_t)(j * 2), IDESC, (kb | j) ? 1u : 0u);
@@ -185,8 +195,6 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
                 if (!ok) break;
-                tc_commit<1>(smem_u32(&ctrl->tfull[0]));
-                ap0 ^= 1u;
                 if (two) { tc_commit<1>(smem_u32(&ctrl->tfull[1])); ap1 ^= 1u; }
             }
             if (dbg) {   // k_blocks counted in 128-row units so that the figures compare with the 128-row kernel

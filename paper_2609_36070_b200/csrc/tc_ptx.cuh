@@ -163,11 +163,18 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr) {
     d |= (uint64_t)2 << 61;                           // 128-byte swizzle
     return d;
 }
-// silu(g) * u = g * u / (1 + exp(-g)) with two special-function instructions (ex2, rcp) and no IEEE division: the
-// epilogue warps share issue slots with the MMA issuer and the gather warps, and the result is rounded to bf16 anyway
-// (relative error of this form ~1e-6).  exp(-g) overflows to +inf for g < -88 and the quotient becomes -0: correct limit.
+// silu(g) * u = g * u * sigmoid(g) = (g/2) * u * (1 + tanh(g/2)): ONE special-function instruction (tanh.approx.f32,
+// relative error 2^-11) and three fp32 operations per output.  The special-function unit retires a warp instruction
+// every 8 cycles per SM quarter, and the epilogue's 128 outputs per thread sit between "accumulator complete" and
+// "accumulator free": with exp + reciprocal (two such instructions per output) draining one accumulator took ~2000
+// cycles.  Error: |dh| <= 2^-11 * |g u / 2|, below the bf16 rounding of h that follows for the value ranges of the
+// layer (and a relative 2^-11 where g > 0).  Large |g| saturate tanh to +-1: h -> g u or -0, the correct limits.
 __device__ __forceinline__ float swiglu(float g, float u) {
-    return __fdividef(g * u, 1.f + __expf(-g));
+    const float hg = 0.5f * g;
+    float t;
+    asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(hg));
+    const float p = hg * u;
+    return fmaf(p, t, p);
 }
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
