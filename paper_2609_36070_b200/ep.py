@@ -74,43 +74,76 @@ def forward_emulated(xs, W_router, router_bias, W_gate_up, W_down, W_shared_gate
 
 
 class DistributedLayer:
-    """One process per GPU under torch.distributed.  Buffers that peers read (x, y, pos) are allocated in symmetric
-    memory once and exchanged by a rendezvous; `forward` then makes no allocation a peer depends on."""
+    """One process per rank under torch.distributed.  Buffers that peers read (x, y, pos) are allocated once and
+    exchanged once; `forward` then makes no allocation a peer depends on.
 
-    def __init__(self, T_local, H, I, I_shared, E, k, device, group=None):
+    exchange = None: the buffers live in symmetric memory and the peers' addresses come from its rendezvous (one
+    process per GPU, NCCL for the route all-gather and the barriers).
+    exchange = callable(name, tensor) -> list of one tensor per rank (this rank's own included) that map the peers'
+    buffers into this process, e.g. CUDA IPC handles passed through torch.multiprocessing queues.  The collectives
+    then go through whatever backend the group has; with a CPU backend (gloo) the routes are staged through the host
+    and every barrier synchronises the device first.  That form also runs with several processes on ONE GPU, since no
+    kernel ever waits for another rank's kernel."""
+
+    def __init__(self, T_local, H, I, I_shared, E, k, device, group=None, exchange=None):
         import torch.distributed as dist
-        import torch.distributed._symmetric_memory as symm
         self.dist = dist
         self.group = group or dist.group.WORLD
         self.R, self.rank = dist.get_world_size(self.group), dist.get_rank(self.group)
         self.E, self.k, self.H = E, k, H
-        handles = []
+        self.host_collectives = dist.get_backend(self.group) != "nccl"
+        self._keep = []
+        if exchange is None:
+            import torch.distributed._symmetric_memory as symm
+            handles = []
 
-        def symm_alloc(shape, dtype):
-            t = symm.empty(shape, dtype=dtype, device=device)
-            handles.append(symm.rendezvous(t, self.group))
-            return t
+            def symm_alloc(shape, dtype):
+                t = symm.empty(shape, dtype=dtype, device=device)
+                handles.append(symm.rendezvous(t, self.group))
+                return t
 
-        self.st = RankState(self.R, T_local, H, I, I_shared, E, k, device, alloc=symm_alloc)   # y, pos: symmetric
-        self.x = symm_alloc((T_local, H), torch.bfloat16)
-        h_y, h_pos, h_x = handles
-        self.y_ptrs = [int(p) for p in h_y.buffer_ptrs]
-        self.pos_ptrs = [int(p) for p in h_pos.buffer_ptrs]
-        self.x_ptrs = [int(p) for p in h_x.buffer_ptrs]
+            self.st = RankState(self.R, T_local, H, I, I_shared, E, k, device, alloc=symm_alloc)   # y, pos: symmetric
+            self.x = symm_alloc((T_local, H), torch.bfloat16)
+            h_y, h_pos, h_x = handles
+            self.y_ptrs = [int(p) for p in h_y.buffer_ptrs]
+            self.pos_ptrs = [int(p) for p in h_pos.buffer_ptrs]
+            self.x_ptrs = [int(p) for p in h_x.buffer_ptrs]
+            self._keep = handles
+        else:
+            self.st = RankState(self.R, T_local, H, I, I_shared, E, k, device)
+            self.x = torch.empty((T_local, H), dtype=torch.bfloat16, device=device)
+            for name, t in (("y", self.st.y), ("pos", self.st.pos), ("x", self.x)):
+                peers = exchange(name, t)
+                assert len(peers) == self.R
+                self._keep.append(peers)                    # the mappings must outlive every kernel that reads them
+                setattr(self, name + "_ptrs", [int(q.data_ptr()) for q in peers])
         self.idx_all = torch.empty((self.R, T_local * k), dtype=torch.int32, device=device)
-        self._handles = handles
+
+    def _barrier(self):
+        if self.host_collectives:
+            torch.cuda.synchronize()
+        self.dist.barrier(group=self.group)
+
+    def _gather_routes(self, idx):
+        if not self.host_collectives:
+            self.dist.all_gather_into_tensor(self.idx_all, idx.reshape(-1), group=self.group)
+            return
+        mine = idx.reshape(-1).cpu()                          # synchronises this rank's stream: its x is final too
+        parts = [torch.empty_like(mine) for _ in range(self.R)]
+        self.dist.all_gather(parts, mine, group=self.group)
+        self.idx_all.copy_(torch.stack(parts))
 
     def forward(self, x_local, W_router, router_bias, W_gate_up_local, W_down_local, W_shared_gate_up, W_shared_down,
                 out=None, config=None):
-        st, dist = self.st, self.dist
-        dist.barrier(group=self.group)          # peers have finished reading the previous layer's x / y / pos
+        st = self.st
+        self._barrier()                         # peers have finished reading the previous layer's x / y / pos
         self.x.copy_(x_local)
         st.idx, st.w = mok.mok_route(self.x, W_router, router_bias, self.k, st.route_ws)
         # the all-gather of the routes also orders every rank's x before any rank's pulls
-        dist.all_gather_into_tensor(self.idx_all, st.idx.reshape(-1), group=self.group)
+        self._gather_routes(st.idx)
         mok.mok_ep_expert_ffn(self.rank, self.x_ptrs, self.idx_all, W_gate_up_local, W_down_local, W_shared_gate_up,
                               W_shared_down, self.E, self.k, st.y, st.pos, st.y_shared, st.ws, self.H, config=config)
-        dist.barrier(group=self.group)          # every rank's y and pos are complete
+        self._barrier()                         # every rank's y and pos are complete
         if out is None:
             out = torch.empty_like(x_local)
         mok.mok_ep_combine(self.rank, self.R, st.idx, st.w, self.y_ptrs, self.pos_ptrs, st.y_shared, self.E, out)
@@ -130,11 +163,78 @@ def forward_distributed(x_local, W_router, router_bias, W_gate_up_local, W_down_
     layer = DistributedLayer(T_local, H, I, I_s, E, k, x_local.device, group)
     out = layer.forward(x_local, W_router, router_bias, W_gate_up_local, W_down_local, W_shared_gate_up, W_shared_down,
                         config=config)
-    layer.dist.barrier(group=layer.group)       # nobody frees y while a peer still reads it
+    layer._barrier()                            # nobody frees y while a peer still reads it
     status = layer.status()
     if status != 0:
         raise mok.MokError(status)
     return out
+
+
+def _ipc_rank(rank, world, queues, config_name, port, results):
+    """One rank of the several-processes-on-one-GPU self-check: gloo collectives, peer buffers through CUDA IPC."""
+    import os
+    import torch.distributed as dist
+    from . import inputs
+    os.environ["MASTER_ADDR"], os.environ["MASTER_PORT"] = "127.0.0.1", str(port)
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    cfg = inputs.CONFIGS[config_name]
+    T_local, L = cfg.T // world, cfg.E // world
+
+    def exchange(name, t):
+        # every rank puts its tensor on every other rank's queue (torch.multiprocessing ships a CUDA IPC handle) and
+        # takes world - 1 tensors off its own; tags keep the three rounds apart
+        for r in range(world):
+            if r != rank:
+                queues[r].put((name, rank, t))
+        got = {rank: t}
+        while len(got) < world:
+            tag, src, peer = queues[rank].get()
+            assert tag == name, (tag, name)
+            got[src] = peer
+        dist.barrier()
+        return [got[r] for r in range(world)]
+
+    d = inputs.make_inputs(cfg)
+    g = {k: (None if d[k] is None else mok.to_device_bf16(d[k], dev)) for k in ("x", "W_gate_up", "W_down", "W_sgu", "W_sd")}
+    W_r = torch.from_numpy(d["W_r"]).to(dev)
+    bias = None if d["bias"] is None else torch.from_numpy(d["bias"]).to(dev)
+    x_local = g["x"][rank * T_local:(rank + 1) * T_local].contiguous()
+    layer = DistributedLayer(T_local, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k, dev, exchange=exchange)
+    out = None
+    for _ in range(2):                                         # twice: buffers are reused across layers
+        out = layer.forward(x_local, W_r, bias, g["W_gate_up"][rank * L:(rank + 1) * L].contiguous(),
+                            g["W_down"][rank * L:(rank + 1) * L].contiguous(), g["W_sgu"], g["W_sd"])
+    layer._barrier()
+    ws = mok.alloc_workspace(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k, device=dev)
+    one = mok.mok_moe_forward_ex(g["x"], W_r, bias, g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], cfg.k, ws)
+    same = torch.equal(out.view(torch.int16), one[rank * T_local:(rank + 1) * T_local].view(torch.int16))
+    results.put((rank, bool(same) and layer.status() == 0))
+    layer._barrier()                                           # peers may still read this rank's buffers until here
+    dist.destroy_process_group()
+
+
+def check_processes_on_one_gpu(world=2, config_name="tiny", port=29561):
+    """Runs `world` ranks as separate processes on GPU 0 (each maps the others' x / y / pos through CUDA IPC) and
+    returns True if every rank's output equals its slice of the one-rank layer bit for bit."""
+    import torch.multiprocessing as mp
+    ctx = mp.get_context("spawn")
+    queues = [ctx.Queue() for _ in range(world)]
+    results = ctx.Queue()
+    procs = [ctx.Process(target=_ipc_rank, args=(r, world, queues, config_name, port, results)) for r in range(world)]
+    for p in procs:
+        p.start()
+    ok = []
+    try:
+        for _ in range(world):
+            ok.append(results.get(timeout=240)[1])
+    finally:
+        for p in procs:
+            p.join(timeout=60)
+            if p.is_alive():
+                p.kill()
+    return len(ok) == world and all(ok) and all(p.exitcode == 0 for p in procs)
 
 
 def main():

@@ -160,3 +160,13 @@ def test_distributed_driver_with_a_world_of_one_rank():
     assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
     line = json.loads([l for l in r.stdout.splitlines() if l.startswith("{")][-1])
     assert line["bitwise_equal_to_one_rank_layer"] and line["n_ranks"] == 1
+
+
+@pytest.mark.parametrize("world", [2, 4])
+def test_ranks_as_separate_processes_on_one_gpu(world):
+    """Real cross-process peer pointers: every rank is its own process on GPU 0, maps the other ranks' x / y / pos
+    buffers through CUDA IPC, and runs the expert-parallel layer with gloo collectives (routes staged through the
+    host).  No kernel waits on another rank's kernel, so sharing one GPU is safe; each rank checks its output bit for
+    bit against the one-rank layer."""
+    from paper_2609_36070_b200 import ep
+    assert ep.check_processes_on_one_gpu(world=world, config_name="tiny", port=29561 + world)
