@@ -226,8 +226,18 @@ typedef struct mok_ep_args {
     int32_t* phi_rank;                   /* int32 [n_ranks*T_local*k]: source rank of schedule row p < S[L] */
     int32_t* phi_index;                  /* int32 [n_ranks*T_local*k]: source route index (token*k + slot) of row p */
     int32_t schedule_only;               /* non-zero: stop after Algorithm 1 (y untouched; pos and the outputs written) */
-    const mok_config* config;            /* grid, cta_group 0/1/3, debug; impl must be MOK_IMPL_TCGEN05 */
+    const mok_config* config;            /* grid, cta_group 0/1/3, precision; impl must be MOK_IMPL_TCGEN05 */
     void* stream;
+    /* MXFP8 mode only (config->precision == MOK_PRECISION_MXFP8, Section 3.4; workspace of
+       mok_ep_mx_workspace_bytes): every rank quantises its own token rows with mok_mx_quantize_rows into buffers the
+       peers can read, and this rank's routed weights come pre-quantised; x_peers is then only used for the shared
+       expert (x_peers[rank]) and W_gate_up / W_down may be NULL */
+    const void* x_codes_peers[MOK_MAX_RANKS];   /* E4M3 [T_local, H] of every rank */
+    const void* x_scales_peers[MOK_MAX_RANKS];  /* E8M0 [T_local, 4 * ceil(H / 128)] of every rank */
+    const void* W_gate_up_codes;         /* E4M3 [L, 2I, H] */
+    const void* W_gate_up_scales;        /* scale atoms of the 2L matrices [I, H] (mok_mx_quantize_weights) */
+    const void* W_down_codes;            /* E4M3 [L, H, I] */
+    const void* W_down_scales;           /* scale atoms of the L matrices [H, I] */
 } mok_ep_args;
 
 typedef struct mok_ep_combine_args {
@@ -243,6 +253,7 @@ typedef struct mok_ep_combine_args {
 } mok_ep_combine_args;
 
 size_t mok_ep_workspace_bytes(int n_ranks, int T_local, int H, int I, int I_shared, int E, int k);
+size_t mok_ep_mx_workspace_bytes(int n_ranks, int T_local, int H, int I, int I_shared, int E, int k);
 long long mok_ep_y_rows(int n_ranks, int T_local, int E, int k);
 int mok_ep_expert_ffn(const mok_ep_args* args);
 int mok_ep_combine(const mok_ep_combine_args* args);

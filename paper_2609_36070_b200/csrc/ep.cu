@@ -224,7 +224,7 @@ ep_combine_kernel(const __grid_constant__ EpCombineArgs a) {
 
 // Workspace of one rank: the one-rank layout for n_ranks*T_local "tokens" and L experts without the router and
 // gathered-copy regions, with room for the per-(rank, block) histograms and M.
-static bool ep_layout(int n_ranks, int T_local, int H, int I, int Is, int E, int k, WsLayout* L) {
+static bool ep_layout(int n_ranks, int T_local, int H, int I, int Is, int E, int k, WsLayout* L, bool mx = false) {
     if (n_ranks < 1 || n_ranks > MOK_MAX_RANKS || T_local < 0 || E < 1 || E % n_ranks) return false;
     if (H <= 0 || I <= 0 || Is < 0 || (H % 8) || (I % 8) || (Is % 8) || k < 1 || k > MAX_K || k > E || E > MAX_E) return false;
     const int Lx = E / n_ranks;
@@ -259,7 +259,11 @@ static bool ep_layout(int n_ranks, int T_local, int H, int I, int Is, int E, int
     L->row_token = take(sizeof(int32_t) * (size_t)Rpad);
     L->h = take(2 * (size_t)Rpad * I);
     L->hs = take(Is > 0 ? 2 * (size_t)L->Tpad * Is : 0);
-    (void)H;
+    if (mx) {
+        if ((H % 32) || (I % 32)) return false;
+        L->h8 = take((size_t)Rpad * I);
+        L->sh = take((size_t)(Rpad / TILE_M) * ((I + 127) / 128) * 512);
+    }
     L->total = off;
     return true;
 }
@@ -277,6 +281,11 @@ size_t mok_ep_workspace_bytes(int n_ranks, int T_local, int H, int I, int I_shar
     return ep_layout(n_ranks, T_local, H, I, I_shared, E, k, &L) ? L.total : 0;
 }
 
+size_t mok_ep_mx_workspace_bytes(int n_ranks, int T_local, int H, int I, int I_shared, int E, int k) {
+    WsLayout L;
+    return ep_layout(n_ranks, T_local, H, I, I_shared, E, k, &L, true) ? L.total : 0;
+}
+
 long long mok_ep_y_rows(int n_ranks, int T_local, int E, int k) {
     WsLayout L;
     return ep_layout(n_ranks, T_local, 8, 8, 0, E, k, &L) ? (long long)L.Rpad : 0;
@@ -285,7 +294,9 @@ long long mok_ep_y_rows(int n_ranks, int T_local, int E, int k) {
 int mok_ep_expert_ffn(const mok_ep_args* a) {
     if (!a) return MOK_ERR_NULL;
     WsLayout L;
-    if (!ep_layout(a->n_ranks, a->T_local, a->H, a->I, a->I_shared, a->E, a->k, &L)) return MOK_ERR_SHAPE;
+    if (a->config && (a->config->precision < 0 || a->config->precision > 1)) return MOK_ERR_SHAPE;
+    const bool mx = a->config && a->config->precision == MOK_PRECISION_MXFP8;
+    if (!ep_layout(a->n_ranks, a->T_local, a->H, a->I, a->I_shared, a->E, a->k, &L, mx)) return MOK_ERR_SHAPE;
     if (a->rank < 0 || a->rank >= a->n_ranks) return MOK_ERR_SHAPE;
     if ((a->I_shared > 0) != (a->W_shared_gate_up != nullptr) || (a->I_shared > 0) != (a->W_shared_down != nullptr))
         return MOK_ERR_SHAPE;
@@ -295,10 +306,24 @@ int mok_ep_expert_ffn(const mok_ep_args* a) {
     if (a->T_local == 0) return MOK_OK;
     if (!a->idx_all || !a->pos) return MOK_ERR_NULL;
     if (!a->schedule_only) {
-        if (!a->W_gate_up || !a->W_down || !a->y || (a->I_shared > 0 && !a->y_shared)) return MOK_ERR_NULL;
+        if (!a->y || (a->I_shared > 0 && !a->y_shared)) return MOK_ERR_NULL;
+        if (mx) {
+            if (!a->W_gate_up_codes || !a->W_gate_up_scales || !a->W_down_codes || !a->W_down_scales) return MOK_ERR_NULL;
+            if (!aligned16(a->W_gate_up_codes) || !aligned16(a->W_gate_up_scales) || !aligned16(a->W_down_codes) ||
+                !aligned16(a->W_down_scales))
+                return MOK_ERR_ALIGN;
+            if (a->I_shared > 0 && !a->x_peers[a->rank]) return MOK_ERR_NULL;
+        } else if (!a->W_gate_up || !a->W_down) {
+            return MOK_ERR_NULL;
+        }
         for (int r = 0; r < a->n_ranks; ++r) {
-            if (!a->x_peers[r]) return MOK_ERR_NULL;
-            if (!aligned16(a->x_peers[r])) return MOK_ERR_ALIGN;
+            if (mx) {
+                if (!a->x_codes_peers[r] || !a->x_scales_peers[r]) return MOK_ERR_NULL;
+                if (!aligned16(a->x_codes_peers[r]) || (reinterpret_cast<uintptr_t>(a->x_scales_peers[r]) & 3u)) return MOK_ERR_ALIGN;
+            } else {
+                if (!a->x_peers[r]) return MOK_ERR_NULL;
+                if (!aligned16(a->x_peers[r])) return MOK_ERR_ALIGN;
+            }
         }
         if (!aligned16(a->W_gate_up) || !aligned16(a->W_down) || !aligned16(a->W_shared_gate_up) ||
             !aligned16(a->W_shared_down) || !aligned16(a->y) || !aligned16(a->y_shared))
@@ -322,7 +347,7 @@ int mok_ep_expert_ffn(const mok_ep_args* a) {
     mok_config cfg;
     memset(&cfg, 0, sizeof(cfg));
     if (a->config) { cfg.grid = a->config->grid; cfg.cta_group = a->config->cta_group; }
-    const __nv_bfloat16* x_own = reinterpret_cast<const __nv_bfloat16*>(a->x_peers[a->rank]);
+    const __nv_bfloat16* x_own = reinterpret_cast<const __nv_bfloat16*>(a->x_peers[a->rank]);   // (may be NULL in MXFP8 mode without a shared expert)
     GemmArgs g;
     memset(&g, 0, sizeof(g));
     g.header = hdr;
@@ -334,26 +359,64 @@ int mok_ep_expert_ffn(const mok_ep_args* a) {
     g.pad_offsets = reinterpret_cast<const int32_t*>(ws + L.pad_offsets);
     g.counts = reinterpret_cast<const int32_t*>(ws + L.counts);
     g.dbg_slot = -1;
-    // routed experts of this rank: the gather warps pull row (src_rank, token) of the schedule from x_peers[src_rank]
-    g.A = x_own;
-    g.a_rows = a->T_local;
-    g.row_token = reinterpret_cast<const int32_t*>(ws + L.row_token);
-    g.peer_tokens = a->T_local;
-    for (int r = 0; r < a->n_ranks; ++r) g.peer_x[r] = reinterpret_cast<const __nv_bfloat16*>(a->x_peers[r]);
-    g.B = reinterpret_cast<const __nv_bfloat16*>(a->W_gate_up);
-    g.C = ws + L.h;
-    g.K = a->H; g.N = a->I; g.ldc = a->I; g.E = Lx; g.rows_pad = L.Rpad; g.dense_rows = 0;
-    g.total_rows = n;   // expected share of this rank, for the kernel choice
     int rc;
-    if ((rc = run_gemm(g, true, &cfg, L, ws, s))) return rc;
-    g.row_token = nullptr;
-    g.peer_tokens = 0;
-    g.a_rows = L.Rpad;
-    g.A = reinterpret_cast<const __nv_bfloat16*>(ws + L.h);
-    g.B = reinterpret_cast<const __nv_bfloat16*>(a->W_down);
-    g.C = a->y;
-    g.K = a->I; g.N = a->H; g.ldc = a->H;
-    if ((rc = run_gemm(g, false, &cfg, L, ws, s))) return rc;
+    if (mx) {
+        // routed experts on MXFP8 operands (Section 3.4): codes and scales of row (src_rank, token) are pulled from that
+        // rank's quantised buffers; the gated activation is quantised in the gate/up epilogue
+        e = cudaMemsetAsync(ws + L.sh, 127, (size_t)(L.Rpad / TILE_M) * ((a->I + 127) / 128) * 512, s);
+        if (e != cudaSuccess) return cuda_fail(e);
+        g.A = reinterpret_cast<const __nv_bfloat16*>(a->x_codes_peers[a->rank]);
+        g.a_rows = a->T_local;
+        g.row_token = reinterpret_cast<const int32_t*>(ws + L.row_token);
+        g.peer_tokens = a->T_local;
+        for (int r = 0; r < a->n_ranks; ++r) {
+            g.peer_x[r] = reinterpret_cast<const __nv_bfloat16*>(a->x_codes_peers[r]);
+            g.peer_sfa[r] = reinterpret_cast<const uint8_t*>(a->x_scales_peers[r]);
+        }
+        g.sfa = g.peer_sfa[a->rank];
+        g.sfa_stride = (a->H + 127) / 128 * 4;
+        g.B = reinterpret_cast<const __nv_bfloat16*>(a->W_gate_up_codes);
+        g.sfb = reinterpret_cast<const uint8_t*>(a->W_gate_up_scales);
+        g.C = ws + L.h8;
+        g.sfc = reinterpret_cast<uint8_t*>(ws + L.sh);
+        g.K = a->H; g.N = a->I; g.ldc = a->I; g.E = Lx; g.rows_pad = L.Rpad; g.dense_rows = 0;
+        g.total_rows = n;
+        e = launch_gemm_mx(g, EPI_SWIGLU, cfg.grid, s);
+        if (e != cudaSuccess) return cuda_fail(e);
+        g.row_token = nullptr;
+        g.peer_tokens = 0;
+        g.A = reinterpret_cast<const __nv_bfloat16*>(ws + L.h8);
+        g.a_rows = L.Rpad;
+        g.sfa = reinterpret_cast<const uint8_t*>(ws + L.sh);
+        g.B = reinterpret_cast<const __nv_bfloat16*>(a->W_down_codes);
+        g.sfb = reinterpret_cast<const uint8_t*>(a->W_down_scales);
+        g.C = a->y;
+        g.sfc = nullptr;
+        g.K = a->I; g.N = a->H; g.ldc = a->H;
+        e = launch_gemm_mx(g, EPI_BF16, cfg.grid, s);
+        if (e != cudaSuccess) return cuda_fail(e);
+        g.sfa = g.sfb = nullptr;
+    } else {
+        // routed experts of this rank: the gather warps pull row (src_rank, token) of the schedule from x_peers[src_rank]
+        g.A = x_own;
+        g.a_rows = a->T_local;
+        g.row_token = reinterpret_cast<const int32_t*>(ws + L.row_token);
+        g.peer_tokens = a->T_local;
+        for (int r = 0; r < a->n_ranks; ++r) g.peer_x[r] = reinterpret_cast<const __nv_bfloat16*>(a->x_peers[r]);
+        g.B = reinterpret_cast<const __nv_bfloat16*>(a->W_gate_up);
+        g.C = ws + L.h;
+        g.K = a->H; g.N = a->I; g.ldc = a->I; g.E = Lx; g.rows_pad = L.Rpad; g.dense_rows = 0;
+        g.total_rows = n;   // expected share of this rank, for the kernel choice
+        if ((rc = run_gemm(g, true, &cfg, L, ws, s))) return rc;
+        g.row_token = nullptr;
+        g.peer_tokens = 0;
+        g.a_rows = L.Rpad;
+        g.A = reinterpret_cast<const __nv_bfloat16*>(ws + L.h);
+        g.B = reinterpret_cast<const __nv_bfloat16*>(a->W_down);
+        g.C = a->y;
+        g.K = a->I; g.N = a->H; g.ldc = a->H;
+        if ((rc = run_gemm(g, false, &cfg, L, ws, s))) return rc;
+    }
     if (a->I_shared > 0) {   // shared expert on the rank's own tokens, natural order
         g.A = x_own;
         g.B = reinterpret_cast<const __nv_bfloat16*>(a->W_shared_gate_up);

@@ -69,6 +69,23 @@ struct Ctrl {
 };
 static_assert(sizeof(Ctrl) <= SMEM_CTRL, "control block too large");
 
+// Source of a gathered token row (E4M3 codes) and of its scale bytes: this GPU's own buffers, or in expert-parallel
+// mode (global token id = source_rank * peer_tokens + token) the owning rank's, read with plain peer loads.
+__device__ __forceinline__ const uint8_t* mx_row(const GemmArgs& a, const uint8_t* xq, int tok) {
+    if (a.peer_tokens > 0) {
+        const int r = tok / a.peer_tokens;
+        return reinterpret_cast<const uint8_t*>(a.peer_x[r]) + (size_t)(tok - r * a.peer_tokens) * a.K;
+    }
+    return xq + (size_t)tok * a.K;
+}
+__device__ __forceinline__ const uint8_t* mx_row_scales(const GemmArgs& a, int tok) {
+    if (a.peer_tokens > 0) {
+        const int r = tok / a.peer_tokens;
+        return a.peer_sfa[r] + (size_t)(tok - r * a.peer_tokens) * a.sfa_stride;
+    }
+    return a.sfa + (size_t)tok * a.sfa_stride;
+}
+
 template <int EPI, bool GATHER, int CTAS>
 __global__ void __launch_bounds__(THREADS + (GATHER ? GATHER_THREADS : 0), 1)
 gemm_mx_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
@@ -272,10 +289,10 @@ gemm_mx_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
             for (int i = 0; i < 8; ++i) {
                 const int r = gw * 32 + i * 4 + sub;
                 const int tok = (r < valid) ? __ldg(rows + r) : tok0;
-                src[i] = xq + (size_t)tok * a.K + chunk * 16;
+                src[i] = mx_row(a, xq, tok) + chunk * 16;
             }
             const int tokq = (q < valid) ? __ldg(rows + q) : tok0;
-            const uint8_t* sfsrc = a.sfa + (size_t)tokq * a.sfa_stride;
+            const uint8_t* sfsrc = mx_row_scales(a, tokq);
             const uint32_t sfdst = base + SF_REGION + (q & 31) * 16 + (q >> 5) * 4;
             bool ok = true;
             for (int kb = 0; kb < k_blocks; ++kb) {

@@ -82,6 +82,8 @@ struct GemmArgs {
     const uint8_t* sfb;          // 512-byte atoms [E (x2 for gate, up)][ceil(N/128)][KG] of the weights
     uint8_t* sfc;                // SWIGLU epilogue: scale atoms of the quantised gated activation [rows_pad/128][ceil(N/128)]
     int32_t sfa_stride;          // bytes between the scale rows of consecutive tokens (GATHER)
+    const uint8_t* peer_sfa[MOK_MAX_RANKS];   // expert-parallel MXFP8: every rank's row-major token scales (with peer_x
+                                              // holding every rank's E4M3 token rows)
 };
 
 // Source row of the fused gather: row `tok` of A, or of the owning rank's token buffer in expert-parallel mode.

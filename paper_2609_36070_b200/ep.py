@@ -21,10 +21,10 @@ from . import mok
 class RankState:
     """Buffers of one rank for fixed sizes: workspace, y / pos / y_shared, and (local) routing results."""
 
-    def __init__(self, n_ranks, T_local, H, I, I_shared, E, k, device, alloc=None):
+    def __init__(self, n_ranks, T_local, H, I, I_shared, E, k, device, alloc=None, mx=False):
         alloc = alloc or (lambda shape, dtype: torch.empty(shape, dtype=dtype, device=device))
         self.n_ranks, self.T_local, self.H, self.I, self.I_shared, self.E, self.k = n_ranks, T_local, H, I, I_shared, E, k
-        n = mok.mok_ep_workspace_bytes(n_ranks, T_local, H, I, I_shared, E, k)
+        n = (mok.mok_ep_mx_workspace_bytes if mx else mok.mok_ep_workspace_bytes)(n_ranks, T_local, H, I, I_shared, E, k)
         if n == 0:
             raise mok.MokError(mok.MOK_ERR_SHAPE)
         self.ws = torch.empty(n + 256, dtype=torch.uint8, device=device)
@@ -33,11 +33,14 @@ class RankState:
         self.pos = alloc((n_ranks * T_local * k,), torch.int32)
         tpad = (T_local + 255) // 256 * 256
         self.y_shared = torch.empty((max(tpad, 256), H), dtype=torch.bfloat16, device=device) if I_shared else None
+        # MXFP8 mode: this rank's quantised token rows and their scales, read by the peers' gather warps
+        self.x_codes = alloc((T_local, H), torch.uint8) if mx else None
+        self.x_scales = alloc((T_local, (H + 127) // 128 * 4), torch.uint8) if mx else None
         self.idx = self.w = None
 
 
 def forward_emulated(xs, W_router, router_bias, W_gate_up, W_down, W_shared_gate_up, W_shared_down, k, config=None,
-                     return_tables=False):
+                     return_tables=False, mx=False):
     """All ranks on the current GPU.  xs: list of bf16 [T_local, H] (one per rank); W_gate_up [E, 2I, H] and
     W_down [E, H, I] hold ALL experts and are cut into per-rank shards here.  Returns the list of per-rank outputs
     (and, with return_tables, each rank's Algorithm 1 tables)."""
@@ -48,16 +51,28 @@ def forward_emulated(xs, W_router, router_bias, W_gate_up, W_down, W_shared_gate
     I = W_gate_up.shape[1] // 2
     I_s = 0 if W_shared_gate_up is None else W_shared_gate_up.shape[0] // 2
     dev = xs[0].device
-    st = [RankState(R, T_local, H, I, I_s, E, k, dev) for _ in range(R)]
-    for r in range(R):                                                  # 1. local routing
+    st = [RankState(R, T_local, H, I, I_s, E, k, dev, mx=mx) for _ in range(R)]
+    if mx:
+        config = config or mok._config()
+        config.precision = mok.MOK_PRECISION_MXFP8
+    mxw = [None] * R
+    for r in range(R):                                                  # 1. local routing (+ quantised rows for the peers)
         st[r].idx, st[r].w = mok.mok_route(xs[r], W_router, router_bias, k, st[r].route_ws)
+        if mx:
+            codes, scales = mok.mok_mx_quantize_rows(xs[r])
+            st[r].x_codes.copy_(codes)
+            st[r].x_scales.copy_(scales)
+            mxw[r] = mok.MxWeights(W_gate_up[r * L:(r + 1) * L].contiguous(), W_down[r * L:(r + 1) * L].contiguous())
     idx_all = torch.stack([s.idx.reshape(-1) for s in st]).contiguous()  # 2. the all-gather of the routes
     x_ptrs = [x.data_ptr() for x in xs]
+    xc_ptrs = [s.x_codes.data_ptr() for s in st] if mx else None
+    xs_ptrs = [s.x_scales.data_ptr() for s in st] if mx else None
     tables = []
     for c in range(R):                                                  # 3. schedule + expert FFNs of rank c
         tables.append(mok.mok_ep_expert_ffn(c, x_ptrs, idx_all, W_gate_up[c * L:(c + 1) * L], W_down[c * L:(c + 1) * L],
                                             W_shared_gate_up, W_shared_down, E, k, st[c].y, st[c].pos, st[c].y_shared,
-                                            st[c].ws, H, outputs=return_tables, config=config))
+                                            st[c].ws, H, outputs=return_tables, config=config, mx_weights=mxw[c],
+                                            x_codes_ptrs=xc_ptrs, x_scales_ptrs=xs_ptrs))
     # 4. the barrier: one stream, so every rank's y and pos are complete before the combines below start
     outs = []
     y_ptrs = [s.y.data_ptr() for s in st]
@@ -85,38 +100,40 @@ class DistributedLayer:
     and every barrier synchronises the device first.  That form also runs with several processes on ONE GPU, since no
     kernel ever waits for another rank's kernel."""
 
-    def __init__(self, T_local, H, I, I_shared, E, k, device, group=None, exchange=None):
+    def __init__(self, T_local, H, I, I_shared, E, k, device, group=None, exchange=None, mx=False):
         import torch.distributed as dist
         self.dist = dist
         self.group = group or dist.group.WORLD
         self.R, self.rank = dist.get_world_size(self.group), dist.get_rank(self.group)
-        self.E, self.k, self.H = E, k, H
+        self.E, self.k, self.H, self.mx = E, k, H, mx
         self.host_collectives = dist.get_backend(self.group) != "nccl"
         self._keep = []
         if exchange is None:
             import torch.distributed._symmetric_memory as symm
-            handles = []
 
-            def symm_alloc(shape, dtype):
-                t = symm.empty(shape, dtype=dtype, device=device)
-                handles.append(symm.rendezvous(t, self.group))
-                return t
+            def alloc(shape, dtype):
+                return symm.empty(shape, dtype=dtype, device=device)
 
-            self.st = RankState(self.R, T_local, H, I, I_shared, E, k, device, alloc=symm_alloc)   # y, pos: symmetric
-            self.x = symm_alloc((T_local, H), torch.bfloat16)
-            h_y, h_pos, h_x = handles
-            self.y_ptrs = [int(p) for p in h_y.buffer_ptrs]
-            self.pos_ptrs = [int(p) for p in h_pos.buffer_ptrs]
-            self.x_ptrs = [int(p) for p in h_x.buffer_ptrs]
-            self._keep = handles
+            def peers_of(name, t):
+                h = symm.rendezvous(t, self.group)
+                self._keep.append(h)
+                return [int(p) for p in h.buffer_ptrs]
         else:
-            self.st = RankState(self.R, T_local, H, I, I_shared, E, k, device)
-            self.x = torch.empty((T_local, H), dtype=torch.bfloat16, device=device)
-            for name, t in (("y", self.st.y), ("pos", self.st.pos), ("x", self.x)):
+            def alloc(shape, dtype):
+                return torch.empty(shape, dtype=dtype, device=device)
+
+            def peers_of(name, t):
                 peers = exchange(name, t)
                 assert len(peers) == self.R
                 self._keep.append(peers)                    # the mappings must outlive every kernel that reads them
-                setattr(self, name + "_ptrs", [int(q.data_ptr()) for q in peers])
+                return [int(q.data_ptr()) for q in peers]
+        self.st = RankState(self.R, T_local, H, I, I_shared, E, k, device, alloc=alloc, mx=mx)
+        self.x = alloc((T_local, H), torch.bfloat16)
+        self.y_ptrs = peers_of("y", self.st.y)
+        self.pos_ptrs = peers_of("pos", self.st.pos)
+        self.x_ptrs = peers_of("x", self.x)
+        self.xc_ptrs = peers_of("x_codes", self.st.x_codes) if mx else None
+        self.xs_ptrs = peers_of("x_scales", self.st.x_scales) if mx else None
         self.idx_all = torch.empty((self.R, T_local * k), dtype=torch.int32, device=device)
 
     def _barrier(self):
@@ -134,15 +151,23 @@ class DistributedLayer:
         self.idx_all.copy_(torch.stack(parts))
 
     def forward(self, x_local, W_router, router_bias, W_gate_up_local, W_down_local, W_shared_gate_up, W_shared_down,
-                out=None, config=None):
+                out=None, config=None, mx_weights=None):
+        """mx_weights: this rank's experts pre-quantised (mok.MxWeights) when the layer was built with mx=True."""
         st = self.st
         self._barrier()                         # peers have finished reading the previous layer's x / y / pos
         self.x.copy_(x_local)
+        if self.mx:                             # this rank's token rows as the peers' gather warps will pull them
+            codes, scales = mok.mok_mx_quantize_rows(self.x)
+            st.x_codes.copy_(codes)
+            st.x_scales.copy_(scales)
+            config = config or mok._config()
+            config.precision = mok.MOK_PRECISION_MXFP8
         st.idx, st.w = mok.mok_route(self.x, W_router, router_bias, self.k, st.route_ws)
         # the all-gather of the routes also orders every rank's x before any rank's pulls
         self._gather_routes(st.idx)
         mok.mok_ep_expert_ffn(self.rank, self.x_ptrs, self.idx_all, W_gate_up_local, W_down_local, W_shared_gate_up,
-                              W_shared_down, self.E, self.k, st.y, st.pos, st.y_shared, st.ws, self.H, config=config)
+                              W_shared_down, self.E, self.k, st.y, st.pos, st.y_shared, st.ws, self.H, config=config,
+                              mx_weights=mx_weights, x_codes_ptrs=self.xc_ptrs, x_scales_ptrs=self.xs_ptrs)
         self._barrier()                         # every rank's y and pos are complete
         if out is None:
             out = torch.empty_like(x_local)
@@ -170,7 +195,7 @@ def forward_distributed(x_local, W_router, router_bias, W_gate_up_local, W_down_
     return out
 
 
-def _ipc_rank(rank, world, queues, config_name, port, results):
+def _ipc_rank(rank, world, queues, config_name, port, results, mx=False):
     """One rank of the several-processes-on-one-GPU self-check: gloo collectives, peer buffers through CUDA IPC."""
     import os
     import torch.distributed as dist
@@ -201,28 +226,31 @@ def _ipc_rank(rank, world, queues, config_name, port, results):
     W_r = torch.from_numpy(d["W_r"]).to(dev)
     bias = None if d["bias"] is None else torch.from_numpy(d["bias"]).to(dev)
     x_local = g["x"][rank * T_local:(rank + 1) * T_local].contiguous()
-    layer = DistributedLayer(T_local, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k, dev, exchange=exchange)
+    layer = DistributedLayer(T_local, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k, dev, exchange=exchange, mx=mx)
+    Wgu, Wd = g["W_gate_up"][rank * L:(rank + 1) * L].contiguous(), g["W_down"][rank * L:(rank + 1) * L].contiguous()
+    mxw = mok.MxWeights(Wgu, Wd) if mx else None
     out = None
     for _ in range(2):                                         # twice: buffers are reused across layers
-        out = layer.forward(x_local, W_r, bias, g["W_gate_up"][rank * L:(rank + 1) * L].contiguous(),
-                            g["W_down"][rank * L:(rank + 1) * L].contiguous(), g["W_sgu"], g["W_sd"])
+        out = layer.forward(x_local, W_r, bias, Wgu, Wd, g["W_sgu"], g["W_sd"], mx_weights=mxw)
     layer._barrier()
-    ws = mok.alloc_workspace(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k, device=dev)
-    one = mok.mok_moe_forward_ex(g["x"], W_r, bias, g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], cfg.k, ws)
+    ws = mok.alloc_workspace(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k, device=dev, mx=mx)
+    one = mok.mok_moe_forward_ex(g["x"], W_r, bias, g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], cfg.k, ws,
+                                 config=mok._config(precision=int(mx)),
+                                 mx_weights=mok.MxWeights(g["W_gate_up"], g["W_down"]) if mx else None)
     same = torch.equal(out.view(torch.int16), one[rank * T_local:(rank + 1) * T_local].view(torch.int16))
     results.put((rank, bool(same) and layer.status() == 0))
     layer._barrier()                                           # peers may still read this rank's buffers until here
     dist.destroy_process_group()
 
 
-def check_processes_on_one_gpu(world=2, config_name="tiny", port=29561):
+def check_processes_on_one_gpu(world=2, config_name="tiny", port=29561, mx=False):
     """Runs `world` ranks as separate processes on GPU 0 (each maps the others' x / y / pos through CUDA IPC) and
     returns True if every rank's output equals its slice of the one-rank layer bit for bit."""
     import torch.multiprocessing as mp
     ctx = mp.get_context("spawn")
     queues = [ctx.Queue() for _ in range(world)]
     results = ctx.Queue()
-    procs = [ctx.Process(target=_ipc_rank, args=(r, world, queues, config_name, port, results)) for r in range(world)]
+    procs = [ctx.Process(target=_ipc_rank, args=(r, world, queues, config_name, port, results, mx)) for r in range(world)]
     for p in procs:
         p.start()
     ok = []

@@ -23,7 +23,8 @@ EXPORTS = ["mok_moe_forward", "mok_workspace_bytes", "mok_moe_forward_ex", "mok_
            "mok_schedule", "mok_read_status", "mok_launch_count", "mok_last_cuda_error", "mok_status_string",
            "mok_version", "mok_profile_begin", "mok_profile_end", "mok_schedule_noalloc", "mok_debug_counters",
            "mok_ep_workspace_bytes", "mok_ep_y_rows", "mok_ep_expert_ffn", "mok_ep_combine",
-           "mok_mx_scale_bytes", "mok_mx_quantize_weights", "mok_mx_quantize_rows", "mok_mx_workspace_bytes"]
+           "mok_mx_scale_bytes", "mok_mx_quantize_weights", "mok_mx_quantize_rows", "mok_mx_workspace_bytes",
+           "mok_ep_mx_workspace_bytes"]
 MOK_PRECISION_BF16, MOK_PRECISION_MXFP8 = 0, 1
 MOK_MAX_RANKS = 16
 MOK_NOALLOC_MAX_ROUTES = 32768
@@ -63,7 +64,10 @@ class mok_ep_args(ctypes.Structure):
                 ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
                 ("M", ctypes.c_void_p), ("S", ctypes.c_void_p), ("phi_rank", ctypes.c_void_p),
                 ("phi_index", ctypes.c_void_p), ("schedule_only", ctypes.c_int32),
-                ("config", ctypes.POINTER(mok_config)), ("stream", ctypes.c_void_p)]
+                ("config", ctypes.POINTER(mok_config)), ("stream", ctypes.c_void_p),
+                ("x_codes_peers", ctypes.c_void_p * MOK_MAX_RANKS), ("x_scales_peers", ctypes.c_void_p * MOK_MAX_RANKS),
+                ("W_gate_up_codes", ctypes.c_void_p), ("W_gate_up_scales", ctypes.c_void_p),
+                ("W_down_codes", ctypes.c_void_p), ("W_down_scales", ctypes.c_void_p)]
 
 
 class mok_ep_combine_args(ctypes.Structure):
@@ -76,6 +80,8 @@ class mok_ep_combine_args(ctypes.Structure):
 
 _lib.mok_ep_workspace_bytes.restype = ctypes.c_size_t
 _lib.mok_ep_workspace_bytes.argtypes = [ctypes.c_int] * 7
+_lib.mok_ep_mx_workspace_bytes.restype = ctypes.c_size_t
+_lib.mok_ep_mx_workspace_bytes.argtypes = [ctypes.c_int] * 7
 _lib.mok_ep_y_rows.restype = ctypes.c_longlong
 _lib.mok_ep_y_rows.argtypes = [ctypes.c_int] * 4
 _lib.mok_ep_expert_ffn.restype = ctypes.c_int
@@ -357,12 +363,17 @@ def mok_ep_workspace_bytes(n_ranks, T_local, H, I, I_shared, E, k):
     return int(_lib.mok_ep_workspace_bytes(n_ranks, T_local, H, I, I_shared, E, k))
 
 
+def mok_ep_mx_workspace_bytes(n_ranks, T_local, H, I, I_shared, E, k):
+    return int(_lib.mok_ep_mx_workspace_bytes(n_ranks, T_local, H, I, I_shared, E, k))
+
+
 def mok_ep_y_rows(n_ranks, T_local, E, k):
     return int(_lib.mok_ep_y_rows(n_ranks, T_local, E, k))
 
 
 def mok_ep_expert_ffn(rank, x_peer_ptrs, idx_all, W_gate_up, W_down, W_shared_gate_up, W_shared_down, E, k, y, pos,
-                      y_shared, workspace, H, schedule_only=False, outputs=False, config=None, stream=None):
+                      y_shared, workspace, H, schedule_only=False, outputs=False, config=None, stream=None,
+                      mx_weights=None, x_codes_ptrs=None, x_scales_ptrs=None):
     """Algorithm 1 for `rank` from the gathered routes idx_all [n_ranks, T_local*k], then this rank's expert FFNs with
     the rows pulled from x_peer_ptrs (device addresses, one per rank).  Fills y, pos (and y_shared).  With
     outputs=True also returns Algorithm 1's tables {M, S, phi_rank, phi_index}."""
@@ -393,6 +404,13 @@ def mok_ep_expert_ffn(rank, x_peer_ptrs, idx_all, W_gate_up, W_down, W_shared_ga
     a.schedule_only = int(schedule_only)
     if config is not None:
         a.config = ctypes.pointer(config)
+    if mx_weights is not None:      # MXFP8 mode: this rank's pre-quantised experts and every rank's quantised token rows
+        a.I = mx_weights.gate_up_codes.shape[1]
+        a.W_gate_up_codes, a.W_gate_up_scales = mx_weights.gate_up_codes.data_ptr(), mx_weights.gate_up_scales.data_ptr()
+        a.W_down_codes, a.W_down_scales = mx_weights.down_codes.data_ptr(), mx_weights.down_scales.data_ptr()
+        for r in range(n_ranks):
+            a.x_codes_peers[r] = x_codes_ptrs[r]
+            a.x_scales_peers[r] = x_scales_ptrs[r]
     a.stream = _stream(stream).value
     _check(_lib.mok_ep_expert_ffn(ctypes.byref(a)))
     return res

@@ -162,11 +162,29 @@ def test_distributed_driver_with_a_world_of_one_rank():
     assert line["bitwise_equal_to_one_rank_layer"] and line["n_ranks"] == 1
 
 
-@pytest.mark.parametrize("world", [2, 4])
-def test_ranks_as_separate_processes_on_one_gpu(world):
+@pytest.mark.parametrize("world,mx", [(2, False), (4, False), (2, True)], ids=["2_ranks", "4_ranks", "2_ranks_mxfp8"])
+def test_ranks_as_separate_processes_on_one_gpu(world, mx):
     """Real cross-process peer pointers: every rank is its own process on GPU 0, maps the other ranks' x / y / pos
     buffers through CUDA IPC, and runs the expert-parallel layer with gloo collectives (routes staged through the
     host).  No kernel waits on another rank's kernel, so sharing one GPU is safe; each rank checks its output bit for
     bit against the one-rank layer."""
     from paper_2609_36070_b200 import ep
-    assert ep.check_processes_on_one_gpu(world=world, config_name="tiny", port=29561 + world)
+    assert ep.check_processes_on_one_gpu(world=world, config_name="tiny", port=29561 + world + 10 * int(mx), mx=mx)
+
+
+@pytest.mark.parametrize("R", [1, 2, 4])
+def test_expert_parallel_mxfp8_equals_the_one_rank_mxfp8_layer(R):
+    """The paper's main configuration: expert parallelism with MXFP8 routed experts (Section 3.4).  Every rank quantises
+    its own token rows; the serving rank's gather warps pull codes and scales from the owner; the result is bitwise the
+    one-rank MXFP8 layer on the concatenated batch (which the MXFP8 tests check against the oracle)."""
+    m = mok()
+    from paper_2609_36070_b200 import ep
+    cfg = inputs.MoEConfig("ep_mx", 1024, 512, 16, 4, 384, 256, bias="zipf", seed=6)
+    d = inputs.make_inputs(cfg)
+    g = pu.upload(d)
+    T_local = cfg.T // R
+    xs = [g["x"][r * T_local:(r + 1) * T_local].contiguous() for r in range(R)]
+    out = torch.cat(ep.forward_emulated(xs, g["W_r"], g["bias"], g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"],
+                                        cfg.k, mx=True))
+    one, rep = pu.mx_parity(cfg, d=d, g=g)
+    assert torch.equal(out.view(torch.int16), one.view(torch.int16)), rep
