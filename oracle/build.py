@@ -1,4 +1,4 @@
-"""Compile the CPU oracle (oracle/mok_ref.c, oracle/mok_ref_mx.c) into oracle/libmok_ref.so with gcc.
+"""Compile the CPU oracle (oracle/mok_ref.c, oracle/mok_ref_mx.c, oracle/mok_ref_bwd.c) into oracle/libmok_ref.so with gcc.
 
 Test infrastructure only.  Building the checker is not using it: the product never loads this
 library.  Run `python oracle/build.py` or call `build()`.
@@ -9,7 +9,7 @@ import sys
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 SRC = os.path.join(HERE, "mok_ref.c")
-SRCS = [SRC, os.path.join(HERE, "mok_ref_mx.c")]
+SRCS = [SRC, os.path.join(HERE, "mok_ref_mx.c"), os.path.join(HERE, "mok_ref_bwd.c")]
 LIB = os.path.join(HERE, "libmok_ref.so")
 
 

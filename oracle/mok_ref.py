@@ -214,3 +214,31 @@ def ffn_tokens_mx(x, Wgu_q, Wd_q, W_sgu, W_sd, idx, w, tokens):
                                      _ptr(tokens, np.int32), int(tokens.size), _ptr(out, np.float64))
     _check(rc, "ffn_tokens_mx")
     return out
+
+
+# ---- backward pass (oracle/mok_ref_bwd.c): the derivative of the Section 2.1 definition ----
+
+def backward(x, W_gate_up, W_down, W_sgu, W_sd, idx, w, dout, weights=True):
+    """dout fp64 [T,H] -> dict(dx [T,H], dw [T,k], and with weights=True dW_gate_up [E,2I,H], dW_down [E,H,I],
+    dW_sgu, dW_sd), all fp64.  The router weights w are inputs of the layer; dw is their gradient."""
+    T, H = x.shape
+    k = idx.shape[1]
+    E, twoI, _ = W_gate_up.shape
+    I = twoI // 2
+    I_s = 0 if W_sgu is None else W_sgu.shape[0] // 2
+    out = {"dx": np.empty((T, H), np.float64), "dw": np.empty((T, k), np.float64)}
+    if weights:
+        out["dW_gate_up"] = np.empty((E, 2 * I, H), np.float64)
+        out["dW_down"] = np.empty((E, H, I), np.float64)
+        if I_s:
+            out["dW_sgu"] = np.empty((2 * I_s, H), np.float64)
+            out["dW_sd"] = np.empty((H, I_s), np.float64)
+    g = lambda name: _ptr(out[name], np.float64) if name in out else None
+    rc = lib().mok_ref_backward(_ptr(x, np.uint16), _ptr(W_gate_up, np.uint16), _ptr(W_down, np.uint16),
+                                _ptr(W_sgu, np.uint16), _ptr(W_sd, np.uint16), T, H, I, I_s, E, k,
+                                _ptr(np.ascontiguousarray(idx, np.int32), np.int32),
+                                _ptr(np.ascontiguousarray(w, np.float64), np.float64),
+                                _ptr(np.ascontiguousarray(dout, np.float64), np.float64),
+                                g("dx"), g("dw"), g("dW_gate_up"), g("dW_down"), g("dW_sgu"), g("dW_sd"))
+    _check(rc, "backward")
+    return out
