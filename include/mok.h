@@ -282,6 +282,41 @@ int mok_mx_quantize_rows(const void* x, int rows, int K, void* codes, void* scal
 size_t mok_mx_workspace_bytes(int T, int H, int I, int I_shared, int E, int k);
 
 /*
+ * Backward pass of the layer (Section 3.4 "fused router weight gradient computation", "activation recomputation";
+ * Section 4.1: dgrad + wgrad).  The paper prints no formulas: this is the chain rule of the Section 2.1 definition.
+ * Inputs: the forward pass's inputs, its routing (topk_idx, topk_w as returned by mok_moe_forward_ex -- the only
+ * thing that has to be kept from the forward pass; every activation is recomputed) and dout = dL/dout.
+ * Outputs: dx = dL/dx through the experts (bf16 [T, H]; the router's own path from x to the logits is not part of
+ * the layer's backward), dw = dL/dtopk_w (fp32 [T, k], the router-weight gradient, or NULL), and the weight
+ * gradients in bf16 with the shapes of the weights (all four NULL = activation gradients only; otherwise all that
+ * belong to present experts must be given).  bf16 mode only; H, I and I_shared must be multiples of 32.
+ * Deterministic like the forward pass: no float atomics, fixed reduction orders.
+ */
+typedef struct mok_bwd_args {
+    const void* x;                  /* bf16 [T, H] */
+    const void* W_gate_up;          /* bf16 [E, 2I, H] */
+    const void* W_down;             /* bf16 [E, H, I] */
+    const void* W_shared_gate_up;   /* bf16 [2*I_shared, H] or NULL */
+    const void* W_shared_down;      /* bf16 [H, I_shared]   or NULL */
+    int32_t T, H, I, I_shared, E, k;
+    const int32_t* topk_idx;        /* int32 [T, k] from the forward pass */
+    const float* topk_w;            /* fp32 [T, k]  from the forward pass */
+    const void* dout;               /* bf16 [T, H] */
+    void* dx;                       /* out: bf16 [T, H] */
+    float* dw;                      /* out: fp32 [T, k] or NULL */
+    void* dW_gate_up;               /* out: bf16 [E, 2I, H] or NULL */
+    void* dW_down;                  /* out: bf16 [E, H, I] or NULL */
+    void* dW_shared_gate_up;        /* out: bf16 [2*I_shared, H] or NULL */
+    void* dW_shared_down;           /* out: bf16 [H, I_shared] or NULL */
+    void* workspace;                /* mok_bwd_workspace_bytes(...) bytes, 256-byte aligned */
+    size_t workspace_bytes;
+    const mok_config* config;       /* grid, cta_group 0/1/3 */
+    void* stream;
+} mok_bwd_args;
+size_t mok_bwd_workspace_bytes(int T, int H, int I, int I_shared, int E, int k);
+int mok_moe_backward(const mok_bwd_args* args);
+
+/*
  * Reads the device-side status word of a workspace after synchronising `stream` -- the only call besides
  * mok_moe_forward_host that blocks the host.  Returns MOK_OK, MOK_ERR_TIMEOUT or MOK_ERR_SCHEDULE
  * (or MOK_ERR_CUDA if the stream itself is in error).

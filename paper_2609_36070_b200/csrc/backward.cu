@@ -1,0 +1,272 @@
+// Backward pass of the MoE layer (paper, Section 3.4 "fused router weight gradient", "activation recomputation";
+// Section 4.1: backward = dgrad + wgrad, twice the forward FLOPs).  The paper prints no formulas; this is the chain
+// rule of the Section 2.1 definition, arranged so that every contraction runs on the forward pass's grouped tcgen05
+// GEMM kernels:
+//
+//   saved from the forward pass: only the routing (top-k ids and weights).  Everything else is recomputed from x
+//   ("activation recomputation"): the dispatch schedule from the ids, the pre-activations gu = [g | u] = Xg Wgu^T.
+//
+//   activation gradients (dgrad)
+//     dhu  = gather(dout) Wd            grouped GEMM, rows pulled from dout through the schedule (K = H, N = I)
+//     per row p (route j = (t, s), weight w):                                       [swiglu_bwd_kernel]
+//         h = silu(g) u,   dw[t,s] = <dhu, h>   (the router-weight gradient, fused: y is never rebuilt)
+//         dh = w dhu,  dg = dh u sig (1 + g (1 - sig)),  du = dh silu(g),  hw = w h
+//     dXg  = [dg | du] Wgu              grouped GEMM (K = 2I, N = H)
+//     dx[t] = dx_shared[t] + sum_s dXg[pos[t,s]]      the forward combine kernel with unit weights (fixed order)
+//   weight gradients (wgrad), per expert e over its rows (a contraction over the ROW index):
+//     dWd_e  = gather(dout)_e^T hw_e    [H, I]        dWgu_e = [dg | du]_e^T Xg_e    [2I, H]
+//   Both operands of these products are activations whose contraction index is the row, so they are transposed once
+//   ([rows, C] -> [C, rows], pad rows zero) and fed to the same kernel in its "K range per expert" mode.
+//   The shared expert is the same computation on every token with w = 1 and no dw.
+//   The weights enter dgrad transposed (Wd^T, Wgu^T as K-contiguous operands): they are transposed into the workspace
+//   at the start of every call (they change between training steps).
+// Intermediates (gu, dhu, dg|du, hw, dXg) are bf16 like the forward pass's h and y; accumulation is fp32 in TMEM;
+// dw is accumulated in fp32.  Deterministic: fixed tile order, fixed k order, fixed combine order, no float atomics.
+#include "mok_internal.cuh"
+#include <string.h>
+
+namespace mok {
+
+// [B, R, C] -> [B, C, R] for bf16, 64 x 64 tiles through shared memory.  Zero-fills nothing: R and C are exact.
+__global__ void __launch_bounds__(256)
+transpose_kernel(const __nv_bfloat16* __restrict__ in, __nv_bfloat16* __restrict__ out, int R, int C, long long in_batch,
+                 long long out_batch, int out_ld) {
+    __shared__ __nv_bfloat16 tile[64][66];
+    const __nv_bfloat16* src = in + (size_t)blockIdx.z * in_batch;
+    __nv_bfloat16* dst = out + (size_t)blockIdx.z * out_batch;
+    const int r0 = blockIdx.y * 64, c0 = blockIdx.x * 64;
+    for (int i = threadIdx.x; i < 64 * 64; i += 256) {
+        const int r = i >> 6, c = i & 63;
+        tile[r][c] = (r0 + r < R && c0 + c < C) ? src[(size_t)(r0 + r) * C + c0 + c] : __float2bfloat16(0.f);
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < 64 * 64; i += 256) {
+        const int c = i >> 6, r = i & 63;
+        if (c0 + c < C && r0 + r < R) dst[(size_t)(c0 + c) * out_ld + r0 + r] = tile[r][c];
+    }
+}
+
+static cudaError_t launch_transpose(const __nv_bfloat16* in, __nv_bfloat16* out, int batch, int R, int C, int out_ld,
+                                    cudaStream_t s) {
+    if (batch <= 0 || R <= 0 || C <= 0) return cudaSuccess;
+    dim3 grid((C + 63) / 64, (R + 63) / 64, batch);
+    transpose_kernel<<<grid, 256, 0, s>>>(in, out, R, C, (long long)R * C, (long long)C * out_ld, out_ld);
+    return cudaGetLastError();
+}
+
+// SwiGLU backward, one warp per row of the (padded) dispatch space, or per token for the shared expert.
+//   gu [rows, 2I] = [g | u] (bf16), dhu [rows, I] = dL/dh before the router weight (bf16)
+//   -> dgu [rows, 2I] = [dg | du], hw [rows, I] = w h, dw[route] = <dhu, h>.
+// Routed mode: row p belongs to expert tile_expert[p / 128]; rows past the expert's count are padding and get zeros
+// (the weight-gradient products run over whole padded segments).  Dense mode (row_route == NULL): w = 1, no dw.
+__global__ void __launch_bounds__(256)
+swiglu_bwd_kernel(const __nv_bfloat16* __restrict__ gu, const __nv_bfloat16* __restrict__ dhu, int I, int rows_dense,
+                  const WsHeader* __restrict__ hdr, const int32_t* __restrict__ tile_expert,
+                  const int32_t* __restrict__ pad_offsets, const int32_t* __restrict__ counts,
+                  const int32_t* __restrict__ row_route, const float* __restrict__ w,
+                  __nv_bfloat16* __restrict__ dgu, __nv_bfloat16* __restrict__ hw, float* __restrict__ dw) {
+    const int lane = threadIdx.x & 31;
+    const int rows = row_route ? hdr->n_mtiles * TILE_M : rows_dense;
+    const int chunks = I >> 3;
+    for (int p = blockIdx.x * 8 + (threadIdx.x >> 5); p < rows; p += gridDim.x * 8) {
+        float wt = 1.f;
+        int route = -1;
+        bool valid = true;
+        if (row_route) {
+            const int e = tile_expert[p / TILE_M];
+            valid = (p - pad_offsets[e]) < counts[e];
+            if (valid) { route = row_route[p]; wt = w[route]; }
+        }
+        const uint4* g4 = reinterpret_cast<const uint4*>(gu + (size_t)p * 2 * I);
+        const uint4* u4 = reinterpret_cast<const uint4*>(gu + (size_t)p * 2 * I + I);
+        const uint4* d4 = reinterpret_cast<const uint4*>(dhu + (size_t)p * I);
+        uint4* dg4 = reinterpret_cast<uint4*>(dgu + (size_t)p * 2 * I);
+        uint4* du4 = reinterpret_cast<uint4*>(dgu + (size_t)p * 2 * I + I);
+        uint4* hw4 = reinterpret_cast<uint4*>(hw + (size_t)p * I);
+        float dot = 0.f;
+        for (int c = lane; c < chunks; c += 32) {
+            uint4 og = make_uint4(0u, 0u, 0u, 0u), ou = og, oh = og;
+            if (valid) {
+                const uint4 rg = g4[c], ru = u4[c], rd = d4[c];
+                const __nv_bfloat162* pg = reinterpret_cast<const __nv_bfloat162*>(&rg);
+                const __nv_bfloat162* pu = reinterpret_cast<const __nv_bfloat162*>(&ru);
+                const __nv_bfloat162* pd = reinterpret_cast<const __nv_bfloat162*>(&rd);
+                __nv_bfloat162* qg = reinterpret_cast<__nv_bfloat162*>(&og);
+                __nv_bfloat162* qu = reinterpret_cast<__nv_bfloat162*>(&ou);
+                __nv_bfloat162* qh = reinterpret_cast<__nv_bfloat162*>(&oh);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const float2 g = __bfloat1622float2(pg[q]), u = __bfloat1622float2(pu[q]), d = __bfloat1622float2(pd[q]);
+                    float r0[3], r1[3];
+                    {
+                        const float sig = 1.f / (1.f + __expf(-g.x)), a = g.x * sig, h = a * u.x, dh = wt * d.x;
+                        dot = fmaf(d.x, h, dot);
+                        r0[0] = dh * u.x * sig * (1.f + g.x * (1.f - sig)); r0[1] = dh * a; r0[2] = wt * h;
+                    }
+                    {
+                        const float sig = 1.f / (1.f + __expf(-g.y)), a = g.y * sig, h = a * u.y, dh = wt * d.y;
+                        dot = fmaf(d.y, h, dot);
+                        r1[0] = dh * u.y * sig * (1.f + g.y * (1.f - sig)); r1[1] = dh * a; r1[2] = wt * h;
+                    }
+                    qg[q] = __floats2bfloat162_rn(r0[0], r1[0]);
+                    qu[q] = __floats2bfloat162_rn(r0[1], r1[1]);
+                    qh[q] = __floats2bfloat162_rn(r0[2], r1[2]);
+                }
+            }
+            dg4[c] = og;
+            du4[c] = ou;
+            hw4[c] = oh;
+        }
+        if (dw && row_route) {
+            // fixed-order reduction over the warp (every lane takes part; `valid` is the same for the whole warp)
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+            if (lane == 0 && valid) dw[route] = dot;
+        }
+    }
+}
+
+// Workspace of the backward pass: the forward layout (schedule tables; its h / y / hs / ysh regions hold hw, dXg, the
+// shared expert's h and dx) followed by the regions only the backward pass needs.
+struct BwdLayout {
+    WsLayout F;
+    size_t row_route, gu, dhu, dgu, WdT, WguT, WsdT, WsguT, gus, dhus, dgus;
+    size_t doutT, hwT, dguT, xgT;      // transposed activations of the weight-gradient products
+    size_t total;
+};
+
+static bool bwd_layout(int T, int H, int I, int Is, int E, int k, BwdLayout* B) {
+    if ((H % 32) || (I % 32) || (Is % 32)) return false;
+    if (!ws_layout(T, H, I, Is, E, k, &B->F)) return false;
+    const WsLayout& F = B->F;
+    size_t off = F.total;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    const size_t Rp = (size_t)F.Rpad, Tp = (size_t)F.Tpad;
+    B->row_route = take(sizeof(int32_t) * Rp);
+    B->gu = take(2 * Rp * 2 * I);
+    B->dhu = take(2 * Rp * I);
+    B->dgu = take(2 * Rp * 2 * I);
+    B->WdT = take(2 * (size_t)E * I * H);
+    B->WguT = take(2 * (size_t)E * H * 2 * I);
+    B->WsdT = take(2 * (size_t)Is * H);
+    B->WsguT = take(2 * (size_t)H * 2 * Is);
+    B->gus = take(2 * Tp * 2 * Is);
+    B->dhus = take(2 * Tp * Is);
+    B->dgus = take(2 * Tp * 2 * Is);
+    const size_t Rm = Rp > Tp ? Rp : Tp;
+    B->doutT = take(2 * (size_t)H * Rm);
+    B->hwT = take(2 * (size_t)(I > Is ? I : Is) * Rm);
+    B->dguT = take(2 * (size_t)2 * (I > Is ? I : Is) * Rm);
+    B->xgT = take(2 * (size_t)H * Rm);
+    B->total = off;
+    return true;
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace mok
+
+using namespace mok;
+
+extern "C" {
+
+size_t mok_bwd_workspace_bytes(int T, int H, int I, int I_shared, int E, int k) {
+    BwdLayout B;
+    return bwd_layout(T, H, I, I_shared, E, k, &B) ? B.total : 0;
+}
+
+int mok_moe_backward(const mok_bwd_args* a) {
+    if (!a) return MOK_ERR_NULL;
+    BwdLayout B;
+    if (!bwd_layout(a->T, a->H, a->I, a->I_shared, a->E, a->k, &B)) return MOK_ERR_SHAPE;
+    if ((a->I_shared > 0) != (a->W_shared_gate_up != nullptr) || (a->I_shared > 0) != (a->W_shared_down != nullptr))
+        return MOK_ERR_SHAPE;
+    if (a->T == 0) return MOK_OK;
+    if (!a->x || !a->W_gate_up || !a->W_down || !a->topk_idx || !a->topk_w || !a->dout || !a->dx) return MOK_ERR_NULL;
+    if (!aligned16(a->x) || !aligned16(a->W_gate_up) || !aligned16(a->W_down) || !aligned16(a->W_shared_gate_up) ||
+        !aligned16(a->W_shared_down) || !aligned16(a->dout) || !aligned16(a->dx) || !aligned16(a->dW_gate_up) ||
+        !aligned16(a->dW_down) || !aligned16(a->dW_shared_gate_up) || !aligned16(a->dW_shared_down))
+        return MOK_ERR_ALIGN;
+    if (!a->workspace || (reinterpret_cast<uintptr_t>(a->workspace) & 255u) || a->workspace_bytes < B.total)
+        return MOK_ERR_WORKSPACE;
+    if (a->config && (a->config->impl != MOK_IMPL_TCGEN05 || a->config->grid < 0 || a->config->precision != MOK_PRECISION_BF16 ||
+                      (a->config->cta_group != 0 && a->config->cta_group != 1 && a->config->cta_group != 3)))
+        return MOK_ERR_SHAPE;
+    const WsLayout& L = B.F;
+    const int T = a->T, H = a->H, I = a->I, Is = a->I_shared, E = a->E, k = a->k;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(a->stream);
+    char* ws = reinterpret_cast<char*>(a->workspace);
+    WsHeader* hdr = reinterpret_cast<WsHeader*>(ws + L.header);
+    const __nv_bfloat16* x = reinterpret_cast<const __nv_bfloat16*>(a->x);
+    const __nv_bfloat16* dout = reinterpret_cast<const __nv_bfloat16*>(a->dout);
+    auto bf = [&](size_t off) { return reinterpret_cast<__nv_bfloat16*>(ws + off); };
+    mok_config cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    if (a->config) { cfg.grid = a->config->grid; cfg.cta_group = a->config->cta_group; }
+    cudaError_t e = cudaMemsetAsync(hdr, 0, sizeof(WsHeader), s);
+    if (e != cudaSuccess) return cuda_fail(e);
+    // the dispatch schedule again, from the saved routing (no host readback)
+    e = launch_schedule(a->topk_idx, T, E, k, TILE_M, TILE_M, L, ws, nullptr, nullptr, nullptr, nullptr, s,
+                        reinterpret_cast<int32_t*>(ws + B.row_route));
+    if (e != cudaSuccess) return cuda_fail(e);
+    // K-contiguous copies of the transposed weights
+    if ((e = launch_transpose(reinterpret_cast<const __nv_bfloat16*>(a->W_down), bf(B.WdT), E, H, I, H, s)) != cudaSuccess) return cuda_fail(e);
+    if ((e = launch_transpose(reinterpret_cast<const __nv_bfloat16*>(a->W_gate_up), bf(B.WguT), E, 2 * I, H, 2 * I, s)) != cudaSuccess) return cuda_fail(e);
+
+    GemmArgs g;
+    memset(&g, 0, sizeof(g));
+    g.header = hdr;
+    g.n_mtiles = &hdr->n_mtiles;
+    g.tile_expert = reinterpret_cast<const int32_t*>(ws + L.tile_expert);
+    g.mt_start = reinterpret_cast<const int32_t*>(ws + L.mt_start);
+    g.max_mt = L.max_mt;
+    g.tile_m = TILE_M;
+    g.pad_offsets = reinterpret_cast<const int32_t*>(ws + L.pad_offsets);
+    g.counts = reinterpret_cast<const int32_t*>(ws + L.counts);
+    g.dbg_slot = -1;
+    g.E = E; g.rows_pad = L.Rpad; g.dense_rows = 0; g.total_rows = L.R;
+    int rc;
+    // gu = gather(x) Wgu^T  (activation recomputation)
+    g.A = x; g.a_rows = T; g.row_token = reinterpret_cast<const int32_t*>(ws + L.row_token);
+    g.B = reinterpret_cast<const __nv_bfloat16*>(a->W_gate_up);
+    g.C = ws + B.gu; g.K = H; g.N = 2 * I; g.ldc = 2 * I;
+    if ((rc = run_gemm(g, false, &cfg, L, ws, s))) return rc;
+    // dhu = gather(dout) Wd
+    g.A = dout; g.B = bf(B.WdT); g.C = ws + B.dhu; g.K = H; g.N = I; g.ldc = I;
+    if ((rc = run_gemm(g, false, &cfg, L, ws, s))) return rc;
+    // SwiGLU backward + router-weight gradient
+    {
+        int blocks = (L.Rpad + 7) / 8;
+        if (blocks > 148 * 16) blocks = 148 * 16;
+        swiglu_bwd_kernel<<<blocks, 256, 0, s>>>(bf(B.gu), bf(B.dhu), I, 0, hdr, g.tile_expert, g.pad_offsets, g.counts,
+                                                 reinterpret_cast<const int32_t*>(ws + B.row_route), a->topk_w, bf(B.dgu),
+                                                 bf(L.h), a->dw);
+        if ((e = cudaGetLastError()) != cudaSuccess) return cuda_fail(e);
+    }
+    // dXg = [dg | du] Wgu
+    g.row_token = nullptr;
+    g.A = bf(B.dgu); g.a_rows = L.Rpad; g.B = bf(B.WguT); g.C = ws + L.y; g.K = 2 * I; g.N = H; g.ldc = H;
+    if ((rc = run_gemm(g, false, &cfg, L, ws, s))) return rc;
+    if (Is > 0) {   // shared expert: the same chain on every token, w = 1
+        if ((e = launch_transpose(reinterpret_cast<const __nv_bfloat16*>(a->W_shared_down), bf(B.WsdT), 1, H, Is, H, s)) != cudaSuccess) return cuda_fail(e);
+        if ((e = launch_transpose(reinterpret_cast<const __nv_bfloat16*>(a->W_shared_gate_up), bf(B.WsguT), 1, 2 * Is, H, 2 * Is, s)) != cudaSuccess) return cuda_fail(e);
+        g.E = 1; g.rows_pad = L.Tpad; g.dense_rows = T; g.a_rows = T;
+        g.A = x; g.B = reinterpret_cast<const __nv_bfloat16*>(a->W_shared_gate_up); g.C = ws + B.gus; g.K = H; g.N = 2 * Is; g.ldc = 2 * Is;
+        if ((rc = run_gemm(g, false, &cfg, L, ws, s))) return rc;
+        g.A = dout; g.B = bf(B.WsdT); g.C = ws + B.dhus; g.K = H; g.N = Is; g.ldc = Is;
+        if ((rc = run_gemm(g, false, &cfg, L, ws, s))) return rc;
+        int blocks = (T + 7) / 8;
+        if (blocks > 148 * 16) blocks = 148 * 16;
+        swiglu_bwd_kernel<<<blocks, 256, 0, s>>>(bf(B.gus), bf(B.dhus), Is, T, hdr, nullptr, nullptr, nullptr, nullptr,
+                                                 nullptr, bf(B.dgus), bf(L.hs), nullptr);
+        if ((e = cudaGetLastError()) != cudaSuccess) return cuda_fail(e);
+        g.A = bf(B.dgus); g.a_rows = L.Tpad; g.B = bf(B.WsguT); g.C = ws + L.ysh; g.K = 2 * Is; g.N = H; g.ldc = H;
+        if ((rc = run_gemm(g, false, &cfg, L, ws, s))) return rc;
+    }
+    // dx[t] = dx_shared[t] + sum_s dXg[pos[t,s]]: the forward combine with unit weights, same fixed order
+    e = launch_combine(L, ws, T, H, k, Is > 0, reinterpret_cast<__nv_bfloat16*>(a->dx), s, /*unit_weights=*/true);
+    if (e != cudaSuccess) return cuda_fail(e);
+    return MOK_OK;
+}
+
+}  // extern "C"

@@ -42,7 +42,7 @@ combine_kernel(const __nv_bfloat16* __restrict__ y, const __nv_bfloat16* __restr
     const int t = blockIdx.x;
     if (threadIdx.x < k) {
         s_pos[threadIdx.x] = pos[(size_t)t * k + threadIdx.x];
-        s_w[threadIdx.x] = w[(size_t)t * k + threadIdx.x];
+        s_w[threadIdx.x] = w ? w[(size_t)t * k + threadIdx.x] : 1.f;   // w == NULL: plain sum (backward pass)
     }
     __syncthreads();
     const int chunks = H >> 3;
@@ -95,11 +95,11 @@ cudaError_t launch_gather(const __nv_bfloat16* x, int H, int k, int tile_m, cons
 }
 
 cudaError_t launch_combine(const WsLayout& L, char* ws, int T, int H, int k, bool shared, __nv_bfloat16* out,
-                           cudaStream_t s) {
+                           cudaStream_t s, bool unit_weights) {
     combine_kernel<<<T, 128, 0, s>>>(reinterpret_cast<const __nv_bfloat16*>(ws + L.y),
                                      shared ? reinterpret_cast<const __nv_bfloat16*>(ws + L.ysh) : nullptr,
                                      reinterpret_cast<const int32_t*>(ws + L.pos),
-                                     reinterpret_cast<const float*>(ws + L.w), T, H, k, out);
+                                     unit_weights ? nullptr : reinterpret_cast<const float*>(ws + L.w), T, H, k, out);
     return cudaGetLastError();
 }
 

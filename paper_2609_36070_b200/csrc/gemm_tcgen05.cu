@@ -485,6 +485,7 @@ cudaError_t launch_gemm_tc(const GemmArgs& a, int epi, int grid, cudaStream_t s)
         if (epi == EPI_SWIGLU && gather) return launch_one<EPI_SWIGLU, true, 1>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
         if (epi == EPI_SWIGLU) return launch_one<EPI_SWIGLU, false, 1>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
         if (epi == EPI_BF16 && !gather) return launch_one<EPI_BF16, false, 1>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
+        if (epi == EPI_BF16) return launch_one<EPI_BF16, true, 1>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
         if (epi == EPI_F32 && !gather) return launch_one<EPI_F32, false, 1>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
     }
     return cudaErrorInvalidValue;

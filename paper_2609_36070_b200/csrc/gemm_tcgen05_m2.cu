@@ -419,6 +419,7 @@ cudaError_t launch_gemm_m2(const GemmArgs& a, int epi, int grid, cudaStream_t s)
     if (epi == EPI_SWIGLU && gather) return launch_one<EPI_SWIGLU, true>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
     if (epi == EPI_SWIGLU) return launch_one<EPI_SWIGLU, false>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
     if (epi == EPI_BF16 && !gather) return launch_one<EPI_BF16, false>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
+    if (epi == EPI_BF16) return launch_one<EPI_BF16, true>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
     if (epi == EPI_F32 && !gather) return launch_one<EPI_F32, false>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
     return cudaErrorInvalidValue;
 }

@@ -66,7 +66,7 @@ sched_scatter_kernel(const int32_t* __restrict__ a, int n, int E,
                      const int32_t* __restrict__ pad_offsets,
                      int32_t* __restrict__ perm, int32_t* __restrict__ inv, int32_t* __restrict__ pos,
                      int32_t* __restrict__ row_token, int k,
-                     int32_t* __restrict__ perm_out, int32_t* __restrict__ inv_out) {
+                     int32_t* __restrict__ perm_out, int32_t* __restrict__ inv_out, int32_t* __restrict__ row_route) {
     extern __shared__ int32_t ssm[];                 // [SCHED_WARPS][E] running counters per warp
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     int32_t* mine = ssm + warp * E;
@@ -114,6 +114,7 @@ sched_scatter_kernel(const int32_t* __restrict__ a, int n, int E,
             const int32_t prow = pad_offsets[e] + rank;   // row in the padded GEMM space
             pos[j] = prow;
             row_token[prow] = j / k;                 // the schedule table's src_index column, as a token id
+            if (row_route) row_route[prow] = j;      // ... and as the route itself (the backward pass needs the slot)
             if (perm_out) perm_out[p] = j;
             if (inv_out) inv_out[j] = p;
         }
@@ -122,7 +123,7 @@ sched_scatter_kernel(const int32_t* __restrict__ a, int n, int E,
 
 cudaError_t launch_schedule(const int32_t* idx, int T, int E, int k, int tile_m, int pad_m, const WsLayout& L, char* ws,
                             int32_t* counts_out, int32_t* offsets_out, int32_t* perm_out, int32_t* inv_out,
-                            cudaStream_t s) {
+                            cudaStream_t s, int32_t* row_route) {
     const int n = T * k;
     int32_t* blk_hist = reinterpret_cast<int32_t*>(ws + L.blk_hist);
     int32_t* counts = reinterpret_cast<int32_t*>(ws + L.counts);
@@ -138,7 +139,7 @@ cudaError_t launch_schedule(const int32_t* idx, int T, int E, int k, int tile_m,
     sched_scatter_kernel<<<L.n_blk, SCHED_THREADS, sizeof(int32_t) * SCHED_WARPS * E, s>>>(
         idx, n, E, blk_hist, offsets, pad_offsets,
         reinterpret_cast<int32_t*>(ws + L.perm), reinterpret_cast<int32_t*>(ws + L.inv),
-        reinterpret_cast<int32_t*>(ws + L.pos), reinterpret_cast<int32_t*>(ws + L.row_token), k, perm_out, inv_out);
+        reinterpret_cast<int32_t*>(ws + L.pos), reinterpret_cast<int32_t*>(ws + L.row_token), k, perm_out, inv_out, row_route);
     return cudaGetLastError();
 }
 

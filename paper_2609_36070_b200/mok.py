@@ -24,7 +24,7 @@ EXPORTS = ["mok_moe_forward", "mok_workspace_bytes", "mok_moe_forward_ex", "mok_
            "mok_version", "mok_profile_begin", "mok_profile_end", "mok_schedule_noalloc", "mok_debug_counters",
            "mok_ep_workspace_bytes", "mok_ep_y_rows", "mok_ep_expert_ffn", "mok_ep_combine",
            "mok_mx_scale_bytes", "mok_mx_quantize_weights", "mok_mx_quantize_rows", "mok_mx_workspace_bytes",
-           "mok_ep_mx_workspace_bytes"]
+           "mok_ep_mx_workspace_bytes", "mok_bwd_workspace_bytes", "mok_moe_backward"]
 MOK_PRECISION_BF16, MOK_PRECISION_MXFP8 = 0, 1
 MOK_MAX_RANKS = 16
 MOK_NOALLOC_MAX_ROUTES = 32768
@@ -78,6 +78,22 @@ class mok_ep_combine_args(ctypes.Structure):
                 ("y_shared", ctypes.c_void_p), ("out", ctypes.c_void_p), ("stream", ctypes.c_void_p)]
 
 
+class mok_bwd_args(ctypes.Structure):
+    _fields_ = [("x", ctypes.c_void_p), ("W_gate_up", ctypes.c_void_p), ("W_down", ctypes.c_void_p),
+                ("W_shared_gate_up", ctypes.c_void_p), ("W_shared_down", ctypes.c_void_p),
+                ("T", ctypes.c_int32), ("H", ctypes.c_int32), ("I", ctypes.c_int32), ("I_shared", ctypes.c_int32),
+                ("E", ctypes.c_int32), ("k", ctypes.c_int32),
+                ("topk_idx", ctypes.c_void_p), ("topk_w", ctypes.c_void_p), ("dout", ctypes.c_void_p),
+                ("dx", ctypes.c_void_p), ("dw", ctypes.c_void_p), ("dW_gate_up", ctypes.c_void_p),
+                ("dW_down", ctypes.c_void_p), ("dW_shared_gate_up", ctypes.c_void_p), ("dW_shared_down", ctypes.c_void_p),
+                ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
+                ("config", ctypes.POINTER(mok_config)), ("stream", ctypes.c_void_p)]
+
+
+_lib.mok_bwd_workspace_bytes.restype = ctypes.c_size_t
+_lib.mok_bwd_workspace_bytes.argtypes = [ctypes.c_int] * 6
+_lib.mok_moe_backward.restype = ctypes.c_int
+_lib.mok_moe_backward.argtypes = [ctypes.POINTER(mok_bwd_args)]
 _lib.mok_ep_workspace_bytes.restype = ctypes.c_size_t
 _lib.mok_ep_workspace_bytes.argtypes = [ctypes.c_int] * 7
 _lib.mok_ep_mx_workspace_bytes.restype = ctypes.c_size_t
@@ -431,6 +447,48 @@ def mok_ep_combine(rank, n_ranks, topk_idx, topk_w, y_peer_ptrs, pos_peer_ptrs, 
     a.stream = _stream(stream).value
     _check(_lib.mok_ep_combine(ctypes.byref(a)))
     return out
+
+
+def mok_bwd_workspace_bytes(T, H, I, I_shared, E, k):
+    return int(_lib.mok_bwd_workspace_bytes(T, H, I, I_shared, E, k))
+
+
+def mok_moe_backward(x, W_gate_up, W_down, W_shared_gate_up, W_shared_down, topk_idx, topk_w, dout, workspace=None,
+                     weight_grads=True, config=None, stream=None):
+    """Backward pass from the forward inputs, its routing and dout.  Returns a dict: dx (bf16 [T,H]), dw (fp32 [T,k])
+    and, with weight_grads, dW_gate_up, dW_down (and dW_shared_gate_up, dW_shared_down) in bf16."""
+    T, H = x.shape
+    E, twoI, _ = W_gate_up.shape
+    I = twoI // 2
+    I_s = 0 if W_shared_gate_up is None else W_shared_gate_up.shape[0] // 2
+    k = topk_idx.shape[1]
+    if workspace is None:
+        n = mok_bwd_workspace_bytes(T, H, I, I_s, E, k)
+        if n == 0:
+            raise MokError(MOK_ERR_SHAPE)
+        workspace = torch.empty(n + 256, dtype=torch.uint8, device=x.device)
+    a = mok_bwd_args()
+    a.x, a.W_gate_up, a.W_down = x.data_ptr(), W_gate_up.data_ptr(), W_down.data_ptr()
+    a.W_shared_gate_up = None if W_shared_gate_up is None else W_shared_gate_up.data_ptr()
+    a.W_shared_down = None if W_shared_down is None else W_shared_down.data_ptr()
+    a.T, a.H, a.I, a.I_shared, a.E, a.k = T, H, I, I_s, E, k
+    a.topk_idx, a.topk_w, a.dout = topk_idx.data_ptr(), topk_w.data_ptr(), dout.data_ptr()
+    res = {"dx": torch.empty_like(x), "dw": torch.empty((T, k), dtype=torch.float32, device=x.device)}
+    if weight_grads:
+        res["dW_gate_up"] = torch.empty_like(W_gate_up)
+        res["dW_down"] = torch.empty_like(W_down)
+        if I_s:
+            res["dW_shared_gate_up"] = torch.empty_like(W_shared_gate_up)
+            res["dW_shared_down"] = torch.empty_like(W_shared_down)
+    for name, t in res.items():
+        setattr(a, name, t.data_ptr())
+    a.workspace, a.workspace_bytes = _aligned_ws(workspace)
+    if config is not None:
+        a.config = ctypes.pointer(config)
+    a.stream = _stream(stream).value
+    _check(_lib.mok_moe_backward(ctypes.byref(a)))
+    res["workspace"] = workspace
+    return res
 
 
 DEBUG_COUNTERS = ["mma_wait_operands", "mma_wait_peer_operands", "mma_wait_accumulator", "mma_total", "k_blocks",

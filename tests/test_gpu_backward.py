@@ -1,0 +1,93 @@
+"""Backward pass on the GPU against the CPU oracle (the chain rule of the layer definition in fp64) on the same seeded
+inputs: activation gradient dx, router-weight gradient dw and the weight gradients, every element, on shapes that span
+several tiles, ragged expert segments, empty experts and a shared expert.  Tolerances: the backward chain rounds five
+intermediates to bf16 (pre-activations, dL/dh, dg|du, dXg or the transposed operands, the result) where the forward
+rounds three, so the bounds are twice the forward pass's: max|gpu - ref| <= 2e-2 max|ref| and
+mean|gpu - ref| <= 1e-2 mean|ref| per tensor."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import mok_ref
+from paper_2609_36070_b200 import inputs
+from tests import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+MAX_REL_BWD, MEAN_REL_BWD = 2e-2, 1e-2
+
+
+def mok():
+    from paper_2609_36070_b200 import mok as m
+    return m
+
+
+def run_case(cfg, weight_grads=True, config=None, wscale=None):
+    m = mok()
+    d = inputs.make_inputs(cfg)
+    if wscale:                                                   # larger weights: silu' away from its linear range
+        rng = np.random.default_rng(cfg.seed + 100)
+        for name in ("W_gate_up", "W_down", "W_sgu", "W_sd"):
+            if d[name] is not None:
+                d[name] = inputs.f32_to_bf16_bits(rng.normal(0, wscale, d[name].shape).astype(np.float32))
+    g = pu.upload(d)
+    out, st = pu.run_gpu(cfg, g)
+    idx = st["topk_idx"]
+    w = st["topk_w"]
+    rng = np.random.default_rng(cfg.seed + 7)
+    dout_bits = inputs.f32_to_bf16_bits(rng.normal(0, 1, (cfg.T, cfg.H)).astype(np.float32))
+    dout = m.to_device_bf16(dout_bits)
+    res = m.mok_moe_backward(g["x"], g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], idx, w, dout,
+                             weight_grads=weight_grads, config=config)
+    torch.cuda.synchronize()
+    assert m.mok_read_status(res["workspace"]) == 0
+    ref = mok_ref.backward(d["x"], d["W_gate_up"], d["W_down"], d["W_sgu"], d["W_sd"], idx.cpu().numpy(),
+                           w.cpu().numpy().astype(np.float64), inputs.bf16_bits_to_f32(dout_bits).astype(np.float64),
+                           weights=weight_grads)
+    rep = {}
+    names = {"dx": "dx", "dw": "dw", "dW_gate_up": "dW_gate_up", "dW_down": "dW_down", "dW_shared_gate_up": "dW_sgu",
+             "dW_shared_down": "dW_sd"}
+    for gname, rname in names.items():
+        if gname not in res or rname not in ref:
+            continue
+        got = res[gname].float().cpu().numpy().astype(np.float64)
+        want = ref[rname]
+        assert np.isfinite(got).all(), gname
+        diff = np.abs(got - want)
+        rep[gname] = (float(diff.max() / np.abs(want).max()), float(diff.mean() / np.abs(want).mean()))
+        assert rep[gname][0] <= MAX_REL_BWD and rep[gname][1] <= MEAN_REL_BWD, (gname, rep[gname])
+    return res, rep
+
+
+SHAPES = [
+    # name, T, H, E, k, I, I_s, bias
+    ("tiny", 256, 256, 8, 2, 512, 512, "none"),
+    ("ragged", 300, 288, 4, 2, 160, 0, "normal"),
+    ("skewed_empty_experts", 1024, 512, 32, 4, 384, 0, "zipf"),
+    ("shared_wider_than_routed", 200, 128, 4, 2, 64, 256, "none"),
+    ("one_route", 130, 64, 2, 1, 32, 0, "none"),
+]
+
+
+@pytest.mark.parametrize("name,T,H,E,k,I,I_s,bias", SHAPES)
+def test_activation_and_router_weight_gradients(name, T, H, E, k, I, I_s, bias):
+    cfg = inputs.MoEConfig("bwd_" + name, T, H, E, k, I, I_s, bias=bias, seed=51)
+    res, rep = run_case(cfg, weight_grads=False)
+    print(name, rep)
+
+
+def test_gradients_with_large_weights():
+    cfg = inputs.MoEConfig("bwd_large_w", 384, 128, 4, 2, 128, 64, seed=52)
+    res, rep = run_case(cfg, weight_grads=False, wscale=0.15)
+    print(rep)
+
+
+def test_backward_is_reproducible_and_grid_independent():
+    m = mok()
+    cfg = inputs.MoEConfig("bwd_repro", 512, 256, 16, 4, 256, 128, bias="zipf", seed=53)
+    runs = []
+    for conf in (None, None, m._config(grid=3), m._config(cta_group=1)):
+        res, _ = run_case(cfg, weight_grads=False, config=conf)
+        runs.append((res["dx"].view(torch.int16).clone(), res["dw"].view(torch.int32).clone()))
+    for dx, dw in runs[1:]:
+        assert torch.equal(dx, runs[0][0]) and torch.equal(dw, runs[0][1])
