@@ -192,6 +192,9 @@ int mok_moe_backward(const mok_bwd_args* a) {
     if (a->config && (a->config->impl != MOK_IMPL_TCGEN05 || a->config->grid < 0 || a->config->precision != MOK_PRECISION_BF16 ||
                       (a->config->cta_group != 0 && a->config->cta_group != 1 && a->config->cta_group != 3)))
         return MOK_ERR_SHAPE;
+    const bool want_w = a->dW_gate_up || a->dW_down || a->dW_shared_gate_up || a->dW_shared_down;
+    if (want_w && (!a->dW_gate_up || !a->dW_down || (a->I_shared > 0 && (!a->dW_shared_gate_up || !a->dW_shared_down))))
+        return MOK_ERR_NULL;
     const WsLayout& L = B.F;
     const int T = a->T, H = a->H, I = a->I, Is = a->I_shared, E = a->E, k = a->k;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(a->stream);
@@ -266,6 +269,47 @@ int mok_moe_backward(const mok_bwd_args* a) {
     // dx[t] = dx_shared[t] + sum_s dXg[pos[t,s]]: the forward combine with unit weights, same fixed order
     e = launch_combine(L, ws, T, H, k, Is > 0, reinterpret_cast<__nv_bfloat16*>(a->dx), s, /*unit_weights=*/true);
     if (e != cudaSuccess) return cuda_fail(e);
+    if (!want_w) return MOK_OK;
+
+    // ------------------------------------------------------------------ weight gradients
+    // Experts without rows keep the zeros written here; every other output element is written by exactly one tile.
+    if ((e = cudaMemsetAsync(a->dW_down, 0, 2 * (size_t)E * H * I, s)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaMemsetAsync(a->dW_gate_up, 0, 2 * (size_t)E * 2 * I * H, s)) != cudaSuccess) return cuda_fail(e);
+    GemmArgs q;
+    memset(&q, 0, sizeof(q));
+    q.header = hdr;
+    q.n_mtiles = &hdr->n_mtiles;
+    q.tile_expert = g.tile_expert; q.mt_start = g.mt_start; q.max_mt = L.max_mt; q.tile_m = TILE_M;
+    q.pad_offsets = g.pad_offsets; q.counts = g.counts;
+    q.dbg_slot = -1;
+    const int Rp = L.Rpad, Tp = L.Tpad;
+    // dWd_e = gather(dout)_e^T (w h)_e: both operands transposed so that the row index is the contiguous (K) one
+    if ((e = launch_gather(dout, H, k, TILE_M, L, ws, s)) != cudaSuccess) return cuda_fail(e);
+    if ((e = launch_transpose(bf(L.xg), bf(B.doutT), 1, Rp, H, Rp, s)) != cudaSuccess) return cuda_fail(e);
+    if ((e = launch_transpose(bf(L.h), bf(B.hwT), 1, Rp, I, Rp, s)) != cudaSuccess) return cuda_fail(e);
+    q.E = E; q.kgroup_rows = H; q.A = bf(B.doutT); q.a_rows = H; q.K = Rp; q.lda = Rp;
+    q.B = bf(B.hwT); q.N = I; q.ldb = Rp; q.C = a->dW_down; q.rows_pad = E * H; q.ldc = I; q.dense_rows = 0;
+    if ((e = launch_gemm_m2(q, EPI_BF16, cfg.grid, s)) != cudaSuccess) return cuda_fail(e);
+    // dWgu_e = [dg | du]_e^T Xg_e
+    if ((e = launch_gather(x, H, k, TILE_M, L, ws, s)) != cudaSuccess) return cuda_fail(e);
+    if ((e = launch_transpose(bf(L.xg), bf(B.xgT), 1, Rp, H, Rp, s)) != cudaSuccess) return cuda_fail(e);
+    if ((e = launch_transpose(bf(B.dgu), bf(B.dguT), 1, Rp, 2 * I, Rp, s)) != cudaSuccess) return cuda_fail(e);
+    q.kgroup_rows = 2 * I; q.A = bf(B.dguT); q.a_rows = 2 * I; q.B = bf(B.xgT); q.N = H; q.C = a->dW_gate_up;
+    q.rows_pad = E * 2 * I; q.ldc = H;
+    if ((e = launch_gemm_m2(q, EPI_BF16, cfg.grid, s)) != cudaSuccess) return cuda_fail(e);
+    if (Is > 0) {   // shared expert: one group over all T tokens (K tail past T is zero-filled by the tensor map)
+        if ((e = launch_transpose(dout, bf(B.doutT), 1, T, H, Tp, s)) != cudaSuccess) return cuda_fail(e);
+        if ((e = launch_transpose(bf(L.hs), bf(B.hwT), 1, T, Is, Tp, s)) != cudaSuccess) return cuda_fail(e);
+        q.E = 1; q.dense_rows = T; q.K = T; q.lda = Tp; q.ldb = Tp;
+        q.kgroup_rows = H; q.A = bf(B.doutT); q.a_rows = H; q.B = bf(B.hwT); q.N = Is; q.C = a->dW_shared_down;
+        q.rows_pad = H; q.ldc = Is;
+        if ((e = launch_gemm_m2(q, EPI_BF16, cfg.grid, s)) != cudaSuccess) return cuda_fail(e);
+        if ((e = launch_transpose(x, bf(B.xgT), 1, T, H, Tp, s)) != cudaSuccess) return cuda_fail(e);
+        if ((e = launch_transpose(bf(B.dgus), bf(B.dguT), 1, T, 2 * Is, Tp, s)) != cudaSuccess) return cuda_fail(e);
+        q.kgroup_rows = 2 * Is; q.A = bf(B.dguT); q.a_rows = 2 * Is; q.B = bf(B.xgT); q.N = H; q.C = a->dW_shared_gate_up;
+        q.rows_pad = 2 * Is; q.ldc = H;
+        if ((e = launch_gemm_m2(q, EPI_BF16, cfg.grid, s)) != cudaSuccess) return cuda_fail(e);
+    }
     return MOK_OK;
 }
 

@@ -50,10 +50,33 @@ static_assert(sizeof(Ctrl) <= SMEM_CTRL, "control block too large");
 
 constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 
-struct Tile { int e, n, row0, valid; };        // valid: real rows of this tile (1..256); > 128 => both halves
+// valid: real rows of this tile (1..256); > 128 => both halves.  row0: first A row and first C row.  In the
+// K-range mode (weight gradients, see GemmArgs::kgroup_rows) the A rows and the C rows differ and the contraction
+// runs over kcol0 .. kcol0 + 64 kblocks of the operands' column space.
+struct Tile { int e, n, row0, valid, crow0, kcol0, kblocks; };
 
-__device__ __forceinline__ Tile decode_tile(const GemmArgs& a, int L, int n_nt, int n_mt_total) {
+__device__ __forceinline__ Tile decode_tile(const GemmArgs& a, int L, int n_nt, int n_mt_total, int k_blocks) {
     Tile t;
+    if (a.kgroup_rows > 0) {
+        // one output matrix [kgroup_rows, N] per expert; tiles in the order expert, N tile, M tile
+        const int m_tiles = (a.kgroup_rows + TM - 1) / TM;
+        const int per_e = m_tiles * n_nt;
+        t.e = L / per_e;
+        const int rem = L - t.e * per_e;
+        t.n = rem / m_tiles;
+        const int m = rem - t.n * m_tiles;
+        t.row0 = m * TM;
+        t.crow0 = t.e * a.kgroup_rows + m * TM;
+        t.valid = min(TM, a.kgroup_rows - m * TM);
+        if (a.dense_rows > 0) {            // one group over all rows (shared expert)
+            t.kcol0 = 0;
+            t.kblocks = (a.dense_rows + 63) / 64;
+        } else {                           // the expert's padded segment of the dispatch space
+            t.kcol0 = __ldg(a.pad_offsets + t.e);
+            t.kblocks = (__ldg(a.pad_offsets + t.e + 1) - t.kcol0) / 64;
+        }
+        return t;
+    }
     int mt0, m_cnt, pad0, cnt;
     if (a.dense_rows > 0) {
         t.e = 0; mt0 = 0; m_cnt = n_mt_total; pad0 = 0; cnt = a.dense_rows;
@@ -72,7 +95,10 @@ __device__ __forceinline__ Tile decode_tile(const GemmArgs& a, int L, int n_nt, 
     t.n = rem / in_group;
     const int m = g * GROUP_TILES + (rem - t.n * in_group);
     t.row0 = pad0 + m * TM;
+    t.crow0 = t.row0;
     t.valid = min(TM, cnt - m * TM);
+    t.kcol0 = 0;
+    t.kblocks = k_blocks;
     return t;
 }
 
@@ -91,7 +117,7 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
 
     int n_mt_total = (a.dense_rows > 0) ? (a.dense_rows + TM - 1) / TM : *a.n_mtiles;
     if (n_mt_total > a.max_mt) n_mt_total = a.max_mt;
-    const int total = n_mt_total * n_nt;
+    const int total = (a.kgroup_rows > 0) ? a.E * ((a.kgroup_rows + TM - 1) / TM) * n_nt : n_mt_total * n_nt;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -123,23 +149,25 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
             uint32_t ph = 0;
             const int b_rows_per_expert = (SWIGLU ? 2 : 1) * a.N;
             for (int L = blockIdx.x; L < total; L += gridDim.x) {
-                const Tile t = decode_tile(a, L, n_nt, n_mt_total);
+                const Tile t = decode_tile(a, L, n_nt, n_mt_total, k_blocks);
                 const bool two = t.valid > BM;
-                const int brow0 = t.e * b_rows_per_expert + (SWIGLU ? t.n * (BN / 2) : t.n * BN);
+                // weight rows of this tile; in the K-range mode B is an activation matrix shared by all experts
+                const int brow0 = (a.kgroup_rows > 0) ? t.n * BN
+                                                      : t.e * b_rows_per_expert + (SWIGLU ? t.n * (BN / 2) : t.n * BN);
                 const int brow1 = SWIGLU ? brow0 + a.N : brow0 + BN / 2;
                 bool ok = true;
-                for (int kb = 0; kb < k_blocks; ++kb) {
+                for (int kb = 0; kb < t.kblocks; ++kb) {
                     ok = mbar_wait(smem_u32(&ctrl->empty[s]), ph ^ 1u, abort_flag, a.header, 1);
                     if (!ok) break;
                     const uint32_t full = smem_u32(&ctrl->full[s]);
                     const uint32_t sa = base + s * STAGE_BYTES, sb = sa + 2 * A_BYTES;
                     mbar_expect_tx(full, B_BYTES + (GATHER ? 0 : (two ? 2 : 1) * A_BYTES));
                     if (!GATHER) {
-                        tma_load_2d(sa, &tmapA, full, kb * BK, t.row0);
-                        if (two) tma_load_2d(sa + A_BYTES, &tmapA, full, kb * BK, t.row0 + BM);
+                        tma_load_2d(sa, &tmapA, full, t.kcol0 + kb * BK, t.row0);
+                        if (two) tma_load_2d(sa + A_BYTES, &tmapA, full, t.kcol0 + kb * BK, t.row0 + BM);
                     }
-                    tma_load_2d(sb, &tmapB, full, kb * BK, brow0);
-                    tma_load_2d(sb + B_BYTES / 2, &tmapB, full, kb * BK, brow1);
+                    tma_load_2d(sb, &tmapB, full, t.kcol0 + kb * BK, brow0);
+                    tma_load_2d(sb + B_BYTES / 2, &tmapB, full, t.kcol0 + kb * BK, brow1);
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
                 if (!ok) break;
@@ -155,7 +183,8 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
             long long d_full = 0, d_tempty = 0, d_kb = 0;
             const long long d_t0 = dbg ? clock64() : 0;
             for (int L = blockIdx.x; L < total; L += gridDim.x) {
-                const Tile t = decode_tile(a, L, n_nt, n_mt_total);
+                const Tile t = decode_tile(a, L, n_nt, n_mt_total, k_blocks);
+                if (t.kblocks == 0) continue;                 // K-range mode: an expert without rows (output pre-zeroed)
                 const bool two = t.valid > BM;
                 long long w0 = dbg ? clock64() : 0;
                 // Accumulator 0 is needed now, accumulator 1 only after the first k-block's MMAs into accumulator 0; and
@@ -166,7 +195,7 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t d0 = tmem_base, d1 = tmem_base + BN;
-                for (int kb = 0; kb < k_blocks; ++kb) {
+                for (int kb = 0; kb < t.kblocks; ++kb) {
                     if (dbg) w0 = clock64();
                     ok = mbar_wait(smem_u32(&ctrl->full[s]), ph, abort_flag, a.header, 3);
                     if (dbg) { d_full += clock64() - w0; d_kb += two ? 2 : 1; }
@@ -178,7 +207,7 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
 #pragma unroll
                     for (int j = 0; j < BK / UMMA_K; ++j)
                         tc_mma<1>(d0, a0 + (uint64_t)(j * 2), bd + (uint64_t)(j * 2), IDESC, (kb | j) ? 1u : 0u);
-                    if (kb == k_blocks - 1) { tc_commit<1>(smem_u32(&ctrl->tfull[0])); ap0 ^= 1u; }
+                    if (kb == t.kblocks - 1) { tc_commit<1>(smem_u32(&ctrl->tfull[0])); ap0 ^= 1u; }
                     if (two) {
                         if (kb == 0) {
                             if (dbg) w0 = clock64();
@@ -215,7 +244,7 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
         int s = 0;
         uint32_t ph = 0;
         for (int L = blockIdx.x; L < total; L += gridDim.x) {
-            const Tile t = decode_tile(a, L, n_nt, n_mt_total);
+            const Tile t = decode_tile(a, L, n_nt, n_mt_total, k_blocks);
             const bool two = t.valid > BM;
             const int tok0 = __ldg(a.row_token + t.row0);
             const __nv_bfloat16* src[16];
@@ -255,15 +284,17 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
         const uint32_t slab = base + STAGES * STAGE_BYTES + (warp - 2) * SLAB_BYTES;
         uint32_t aph = 0;
         for (int L = blockIdx.x; L < total; L += gridDim.x) {
-            const Tile t = decode_tile(a, L, n_nt, n_mt_total);
-            if (acc == 1 && t.valid <= BM) continue;          // this tile has no second half
+            const Tile t = decode_tile(a, L, n_nt, n_mt_total, k_blocks);
+            if (t.kblocks == 0 || (acc == 1 && t.valid <= BM)) continue;   // no rows to contract / no second half
             bool ok = mbar_wait(smem_u32(&ctrl->tfull[acc]), aph, abort_flag, a.header, 4);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             aph ^= 1u;
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * BN);
-            const int row = t.row0 + acc * BM + quad * 32;
+            const int row = t.crow0 + acc * BM + quad * 32;
+            // K-range mode: 32-row boxes past the expert's output matrix belong to the next expert
+            const bool store_ok = a.kgroup_rows <= 0 || (row - t.e * a.kgroup_rows) < a.kgroup_rows;
             if (EPI == EPI_F32) {
                 float* frow = reinterpret_cast<float*>(a.C) + (size_t)(row + lane) * a.ldc;
                 const int c0 = t.n * BN;
@@ -334,7 +365,7 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
                     __syncwarp();
                     if (lane == 0) {
                         const int col = c0 + pass * 64;
-                        if (col < a.N) tma_store_2d(&tmapC, slab, col, row);
+                        if (col < a.N && store_ok) tma_store_2d(&tmapC, slab, col, row);
                         tma_store_commit();
                     }
                 }
@@ -410,8 +441,10 @@ cudaError_t launch_gemm_m2(const GemmArgs& a, int epi, int grid, cudaStream_t s)
     const bool swiglu = (epi == EPI_SWIGLU), gather = (a.row_token != nullptr);
     CUtensorMap mA, mB, mC;
     const uint64_t b_rows = (uint64_t)a.E * (swiglu ? 2 : 1) * a.N;
-    if (!make_map(&mA, a.A, (uint64_t)a.a_rows, (uint64_t)a.K, BM, (uint64_t)a.K)) return cudaErrorInvalidValue;
-    if (!make_map(&mB, a.B, b_rows, (uint64_t)a.K, BN / 2, (uint64_t)a.K)) return cudaErrorInvalidValue;
+    if (a.kgroup_rows > 0 && (epi != EPI_BF16 || gather || (a.kgroup_rows % 32))) return cudaErrorInvalidValue;
+    const uint64_t lda = a.lda ? (uint64_t)a.lda : (uint64_t)a.K, ldb = a.ldb ? (uint64_t)a.ldb : (uint64_t)a.K;
+    if (!make_map(&mA, a.A, (uint64_t)a.a_rows, (uint64_t)a.K, BM, lda)) return cudaErrorInvalidValue;
+    if (!make_map(&mB, a.B, a.kgroup_rows > 0 ? (uint64_t)a.N : b_rows, (uint64_t)a.K, BN / 2, ldb)) return cudaErrorInvalidValue;
     if (epi == EPI_F32) mC = mB;      // the fp32 epilogue stores directly
     else if (!make_map(&mC, a.C, (uint64_t)a.rows_pad, (uint64_t)a.N, 32, (uint64_t)a.ldc)) return cudaErrorInvalidValue;
     const int n_nt = swiglu ? (a.N + BN / 2 - 1) / (BN / 2) : (a.N + BN - 1) / BN;

@@ -71,6 +71,12 @@ struct GemmArgs {
     int32_t tile_m;              // rows of one tile of the padded row space: 128, or 256 for CTA pairs
     int32_t dbg_slot;            // >= 0: accumulate wait-time counters into header->dbg[dbg_slot]
     int32_t starve;              // test hook: the TMA producer issues nothing, so the kernel's waits run out
+    // K-range mode of the 256-row kernel (weight gradients): C holds E matrices [kgroup_rows, N]; A is ONE matrix
+    // [kgroup_rows, K extent] and B ONE matrix [N, K extent] whose columns are the rows of the dispatch space; expert e
+    // contracts over its padded segment [pad_offsets[e], pad_offsets[e+1]) (dense_rows > 0: one group over columns
+    // 0 .. dense_rows).  lda / ldb: elements between consecutive rows of A / B (0 = K).
+    int32_t kgroup_rows;
+    int32_t lda, ldb;
     WsHeader* header;
     // Expert-parallel pull dispatch (Section 3.1): with peer_tokens > 0 the ids in row_token are global,
     // id = source_rank * peer_tokens + token, and row `id` is read from peer_x[source_rank] (this GPU's own tokens

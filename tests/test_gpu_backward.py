@@ -76,9 +76,16 @@ def test_activation_and_router_weight_gradients(name, T, H, E, k, I, I_s, bias):
     print(name, rep)
 
 
+@pytest.mark.parametrize("name,T,H,E,k,I,I_s,bias", SHAPES)
+def test_weight_gradients(name, T, H, E, k, I, I_s, bias):
+    cfg = inputs.MoEConfig("bwd_" + name, T, H, E, k, I, I_s, bias=bias, seed=51)
+    res, rep = run_case(cfg, weight_grads=True)
+    print(name, rep)
+
+
 def test_gradients_with_large_weights():
     cfg = inputs.MoEConfig("bwd_large_w", 384, 128, 4, 2, 128, 64, seed=52)
-    res, rep = run_case(cfg, weight_grads=False, wscale=0.15)
+    res, rep = run_case(cfg, weight_grads=True, wscale=0.15)
     print(rep)
 
 
