@@ -242,3 +242,23 @@ def backward(x, W_gate_up, W_down, W_sgu, W_sd, idx, w, dout, weights=True):
                                 g("dx"), g("dw"), g("dW_gate_up"), g("dW_down"), g("dW_sgu"), g("dW_sd"))
     _check(rc, "backward")
     return out
+
+
+def backward_tokens(x, W_gate_up, W_down, W_sgu, W_sd, idx, w, dout, tokens):
+    """dx [n,H] and dw [n,k] of the listed tokens only (full-size checks); same chain rule as backward()."""
+    T, H = x.shape
+    k = idx.shape[1]
+    E, twoI, _ = W_gate_up.shape
+    I = twoI // 2
+    I_s = 0 if W_sgu is None else W_sgu.shape[0] // 2
+    tokens = np.ascontiguousarray(tokens, np.int32)
+    dx = np.empty((tokens.size, H), np.float64)
+    dw = np.empty((tokens.size, k), np.float64)
+    rc = lib().mok_ref_backward_tokens(_ptr(x, np.uint16), _ptr(W_gate_up, np.uint16), _ptr(W_down, np.uint16),
+                                       _ptr(W_sgu, np.uint16), _ptr(W_sd, np.uint16), H, I, I_s, E, k,
+                                       _ptr(np.ascontiguousarray(idx, np.int32), np.int32),
+                                       _ptr(np.ascontiguousarray(w, np.float64), np.float64),
+                                       _ptr(np.ascontiguousarray(dout, np.float64), np.float64),
+                                       _ptr(tokens, np.int32), int(tokens.size), _ptr(dx, np.float64), _ptr(dw, np.float64))
+    _check(rc, "backward_tokens")
+    return dx, dw

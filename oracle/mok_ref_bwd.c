@@ -153,3 +153,41 @@ int mok_ref_backward(const uint16_t* x, const uint16_t* W_gate_up, const uint16_
     }
     return 0;
 }
+
+/*
+ * Token side of the backward pass for a list of tokens only (full-size checks): dx[n_tok, H] and dw[n_tok, k] of the
+ * listed tokens, from the same chain rule.  idx, w and dout are indexed by token id.
+ */
+int mok_ref_backward_tokens(const uint16_t* x, const uint16_t* W_gate_up, const uint16_t* W_down,
+                            const uint16_t* W_sgu, const uint16_t* W_sd,
+                            int H, int I, int I_s, int E, int k, const int32_t* idx, const double* w,
+                            const double* dout, const int32_t* tokens, int n_tok, double* dx, double* dw) {
+    if (!x || !dout || !tokens || !dx || n_tok < 0 || H <= 0 || I <= 0 || E <= 0 || k < 1 || !W_gate_up || !W_down || !idx || !w)
+        return -1;
+    if ((I_s > 0) != (W_sgu != NULL) || (I_s > 0) != (W_sd != NULL)) return -1;
+    const int Imax = I > I_s ? I : I_s;
+    memset(dx, 0, sizeof(double) * (size_t)n_tok * H);
+    int bad = 0;
+#pragma omp parallel
+    {
+        double* v = (double*)malloc(sizeof(double) * (size_t)H);
+        double* scratch = (double*)malloc(sizeof(double) * (size_t)(5 * Imax + H));
+#pragma omp for schedule(dynamic, 1)
+        for (int n = 0; n < n_tok; ++n) {
+            const int t = tokens[n];
+            for (int c = 0; c < H; ++c) v[c] = bf16_f64(x[(size_t)t * H + c]);
+            const double* dr = dout + (size_t)t * H;
+            if (I_s > 0) expert_backward(v, W_sgu, W_sd, H, I_s, 1.0, dr, dx + (size_t)n * H, NULL, NULL, NULL, scratch);
+            for (int s = 0; s < k; ++s) {
+                const int e = idx[(size_t)t * k + s];
+                if (e < 0 || e >= E) { bad = 1; continue; }
+                double d = 0.0;
+                expert_backward(v, W_gate_up + (size_t)e * 2 * I * H, W_down + (size_t)e * H * I, H, I,
+                                w[(size_t)t * k + s], dr, dx + (size_t)n * H, NULL, NULL, &d, scratch);
+                if (dw) dw[(size_t)n * k + s] = d;
+            }
+        }
+        free(v); free(scratch);
+    }
+    return bad ? -2 : 0;
+}

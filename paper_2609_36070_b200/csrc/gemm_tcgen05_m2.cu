@@ -55,9 +55,10 @@ constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >
 // runs over kcol0 .. kcol0 + 64 kblocks of the operands' column space.
 struct Tile { int e, n, row0, valid, crow0, kcol0, kblocks; };
 
+template <bool KGROUP>
 __device__ __forceinline__ Tile decode_tile(const GemmArgs& a, int L, int n_nt, int n_mt_total, int k_blocks) {
     Tile t;
-    if (a.kgroup_rows > 0) {
+    if (KGROUP) {
         // one output matrix [kgroup_rows, N] per expert; tiles in the order expert, N tile, M tile
         const int m_tiles = (a.kgroup_rows + TM - 1) / TM;
         const int per_e = m_tiles * n_nt;
@@ -102,7 +103,8 @@ __device__ __forceinline__ Tile decode_tile(const GemmArgs& a, int L, int n_nt, 
     return t;
 }
 
-template <int EPI, bool GATHER>
+// KGROUP: the K-range mode (weight gradients), compiled separately so that the forward kernels carry none of it.
+template <int EPI, bool GATHER, bool KGROUP>
 __global__ void __launch_bounds__(THREADS + (GATHER ? GATHER_THREADS : 0), 1)
 gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
                const __grid_constant__ CUtensorMap tmapC, const __grid_constant__ GemmArgs a, const int n_nt, const int k_blocks) {
@@ -117,7 +119,7 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
 
     int n_mt_total = (a.dense_rows > 0) ? (a.dense_rows + TM - 1) / TM : *a.n_mtiles;
     if (n_mt_total > a.max_mt) n_mt_total = a.max_mt;
-    const int total = (a.kgroup_rows > 0) ? a.E * ((a.kgroup_rows + TM - 1) / TM) * n_nt : n_mt_total * n_nt;
+    const int total = KGROUP ? a.E * ((a.kgroup_rows + TM - 1) / TM) * n_nt : n_mt_total * n_nt;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -149,10 +151,10 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
             uint32_t ph = 0;
             const int b_rows_per_expert = (SWIGLU ? 2 : 1) * a.N;
             for (int L = blockIdx.x; L < total; L += gridDim.x) {
-                const Tile t = decode_tile(a, L, n_nt, n_mt_total, k_blocks);
+                const Tile t = decode_tile<KGROUP>(a, L, n_nt, n_mt_total, k_blocks);
                 const bool two = t.valid > BM;
                 // weight rows of this tile; in the K-range mode B is an activation matrix shared by all experts
-                const int brow0 = (a.kgroup_rows > 0) ? t.n * BN
+                const int brow0 = KGROUP ? t.n * BN
                                                       : t.e * b_rows_per_expert + (SWIGLU ? t.n * (BN / 2) : t.n * BN);
                 const int brow1 = SWIGLU ? brow0 + a.N : brow0 + BN / 2;
                 bool ok = true;
@@ -183,8 +185,8 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
             long long d_full = 0, d_tempty = 0, d_kb = 0;
             const long long d_t0 = dbg ? clock64() : 0;
             for (int L = blockIdx.x; L < total; L += gridDim.x) {
-                const Tile t = decode_tile(a, L, n_nt, n_mt_total, k_blocks);
-                if (t.kblocks == 0) continue;                 // K-range mode: an expert without rows (output pre-zeroed)
+                const Tile t = decode_tile<KGROUP>(a, L, n_nt, n_mt_total, k_blocks);
+                if (KGROUP && t.kblocks == 0) continue;       // K-range mode: an expert without rows (output pre-zeroed)
                 const bool two = t.valid > BM;
                 long long w0 = dbg ? clock64() : 0;
                 // Accumulator 0 is needed now, accumulator 1 only after the first k-block's MMAs into accumulator 0; and
@@ -244,7 +246,7 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
         int s = 0;
         uint32_t ph = 0;
         for (int L = blockIdx.x; L < total; L += gridDim.x) {
-            const Tile t = decode_tile(a, L, n_nt, n_mt_total, k_blocks);
+            const Tile t = decode_tile<KGROUP>(a, L, n_nt, n_mt_total, k_blocks);
             const bool two = t.valid > BM;
             const int tok0 = __ldg(a.row_token + t.row0);
             const __nv_bfloat16* src[16];
@@ -284,8 +286,8 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
         const uint32_t slab = base + STAGES * STAGE_BYTES + (warp - 2) * SLAB_BYTES;
         uint32_t aph = 0;
         for (int L = blockIdx.x; L < total; L += gridDim.x) {
-            const Tile t = decode_tile(a, L, n_nt, n_mt_total, k_blocks);
-            if (t.kblocks == 0 || (acc == 1 && t.valid <= BM)) continue;   // no rows to contract / no second half
+            const Tile t = decode_tile<KGROUP>(a, L, n_nt, n_mt_total, k_blocks);
+            if ((KGROUP && t.kblocks == 0) || (acc == 1 && t.valid <= BM)) continue;   // no rows to contract / no second half
             bool ok = mbar_wait(smem_u32(&ctrl->tfull[acc]), aph, abort_flag, a.header, 4);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
@@ -294,7 +296,7 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
             const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * BN);
             const int row = t.crow0 + acc * BM + quad * 32;
             // K-range mode: 32-row boxes past the expert's output matrix belong to the next expert
-            const bool store_ok = a.kgroup_rows <= 0 || (row - t.e * a.kgroup_rows) < a.kgroup_rows;
+            const bool store_ok = !KGROUP || (row - t.e * a.kgroup_rows) < a.kgroup_rows;
             if (EPI == EPI_F32) {
                 float* frow = reinterpret_cast<float*>(a.C) + (size_t)(row + lane) * a.ldc;
                 const int c0 = t.n * BN;
@@ -416,12 +418,12 @@ static bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t co
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int EPI, bool GATHER>
+template <int EPI, bool GATHER, bool KGROUP = false>
 static cudaError_t launch_one(const CUtensorMap& mA, const CUtensorMap& mB, const CUtensorMap& mC, const GemmArgs& a,
                               int n_nt, int k_blocks, int grid, cudaStream_t s) {
     static int sm_count = 0;
     if (!sm_count) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_m2_kernel<EPI, GATHER>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(gemm_m2_kernel<EPI, GATHER, KGROUP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              SMEM_BYTES);
         if (e != cudaSuccess) return e;
         int dev = 0;
@@ -429,7 +431,7 @@ static cudaError_t launch_one(const CUtensorMap& mA, const CUtensorMap& mB, cons
         cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
     }
     if (grid <= 0 || grid > sm_count) grid = sm_count;
-    gemm_m2_kernel<EPI, GATHER><<<grid, THREADS + (GATHER ? GATHER_THREADS : 0), SMEM_BYTES, s>>>(mA, mB, mC, a, n_nt,
+    gemm_m2_kernel<EPI, GATHER, KGROUP><<<grid, THREADS + (GATHER ? GATHER_THREADS : 0), SMEM_BYTES, s>>>(mA, mB, mC, a, n_nt,
                                                                                                  k_blocks);
     return cudaGetLastError();
 }
@@ -449,6 +451,7 @@ cudaError_t launch_gemm_m2(const GemmArgs& a, int epi, int grid, cudaStream_t s)
     else if (!make_map(&mC, a.C, (uint64_t)a.rows_pad, (uint64_t)a.N, 32, (uint64_t)a.ldc)) return cudaErrorInvalidValue;
     const int n_nt = swiglu ? (a.N + BN / 2 - 1) / (BN / 2) : (a.N + BN - 1) / BN;
     const int k_blocks = (a.K + BK - 1) / BK;
+    if (a.kgroup_rows > 0) return launch_one<EPI_BF16, false, true>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
     if (epi == EPI_SWIGLU && gather) return launch_one<EPI_SWIGLU, true>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
     if (epi == EPI_SWIGLU) return launch_one<EPI_SWIGLU, false>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
     if (epi == EPI_BF16 && !gather) return launch_one<EPI_BF16, false>(mA, mB, mC, a, n_nt, k_blocks, grid, s);

@@ -98,3 +98,43 @@ def test_backward_is_reproducible_and_grid_independent():
         runs.append((res["dx"].view(torch.int16).clone(), res["dw"].view(torch.int32).clone()))
     for dx, dw in runs[1:]:
         assert torch.equal(dx, runs[0][0]) and torch.equal(dw, runs[0][1])
+
+
+def test_bench_shape_with_fewer_tokens_all_gradients():
+    """The benchmark layer (H = 2048, E = 128, k = 8, I = 768, Zipf routing: hot and empty experts) at T = 2048, where
+    the oracle can still evaluate every weight gradient."""
+    cfg = inputs.CONFIGS["qwen3_30b_a3b"].with_tokens(2048)
+    res, rep = run_case(cfg, weight_grads=True)
+    print(rep)
+
+
+def test_bench_shape_full_size_sampled():
+    """Full benchmark workload: dx and dw of a token sample against the oracle, everything finite, run-to-run bitwise."""
+    m = mok()
+    cfg = inputs.CONFIGS["qwen3_30b_a3b"]
+    d = inputs.make_inputs(cfg)
+    g = pu.upload(d)
+    out, st = pu.run_gpu(cfg, g)
+    idx, w = st["topk_idx"], st["topk_w"]
+    rng = np.random.default_rng(77)
+    dout_bits = inputs.f32_to_bf16_bits(rng.normal(0, 1, (cfg.T, cfg.H)).astype(np.float32))
+    dout = m.to_device_bf16(dout_bits)
+    res = m.mok_moe_backward(g["x"], g["W_gate_up"], g["W_down"], None, None, idx, w, dout)
+    torch.cuda.synchronize()
+    assert m.mok_read_status(res["workspace"]) == 0
+    tokens = inputs.sample_tokens(cfg, idx.cpu().numpy(), 256)
+    dx_ref, dw_ref = mok_ref.backward_tokens(d["x"], d["W_gate_up"], d["W_down"], None, None, idx.cpu().numpy(),
+                                             w.cpu().numpy().astype(np.float64),
+                                             inputs.bf16_bits_to_f32(dout_bits).astype(np.float64), tokens)
+    sel = torch.from_numpy(np.asarray(tokens, np.int64)).cuda()
+    for got, want, name in ((res["dx"][sel], dx_ref, "dx"), (res["dw"][sel], dw_ref, "dw")):
+        got = got.float().cpu().numpy().astype(np.float64)
+        diff = np.abs(got - want)
+        assert diff.max() <= MAX_REL_BWD * np.abs(want).max() and diff.mean() <= MEAN_REL_BWD * np.abs(want).mean(), name
+    for name in ("dW_gate_up", "dW_down"):
+        assert torch.isfinite(res[name].float()).all()
+    again = m.mok_moe_backward(g["x"], g["W_gate_up"], g["W_down"], None, None, idx, w, dout, workspace=res["workspace"])
+    torch.cuda.synchronize()
+    for name in ("dx", "dW_gate_up", "dW_down"):
+        assert torch.equal(again[name].view(torch.int16), res[name].view(torch.int16)), name
+    assert torch.equal(again["dw"].view(torch.int32), res["dw"].view(torch.int32))

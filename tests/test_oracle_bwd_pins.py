@@ -112,3 +112,11 @@ def test_special_cases():
             gu = f64(d["W_gate_up"])[e] @ x[t]
             acc[e] += np.outer(w[t, s] * dout[t], silu(gu[:cfg.I]) * gu[cfg.I:])
     assert np.abs(acc - base["dW_down"]).max() <= 1e-12 * np.abs(acc).max()
+
+
+def test_token_subset_equals_the_full_backward():
+    cfg, d, idx, w, dout = case(6, T=9)
+    full = mok_ref.backward(d["x"], d["W_gate_up"], d["W_down"], d["W_sgu"], d["W_sd"], idx, w, dout, weights=False)
+    tok = np.array([7, 0, 3], np.int32)
+    dx, dw = mok_ref.backward_tokens(d["x"], d["W_gate_up"], d["W_down"], d["W_sgu"], d["W_sd"], idx, w, dout, tok)
+    assert np.array_equal(dx, full["dx"][tok]) and np.array_equal(dw, full["dw"][tok])
