@@ -45,6 +45,8 @@ def parse():
     p.add_argument("--host-chunks", type=int, default=0, help="token chunks of the host-buffer call (0 = auto)")
     p.add_argument("--precision", default="bf16", choices=["bf16", "mxfp8"],
                    help="routed experts in bf16 (the headline workload) or MXFP8 with pre-quantised weights")
+    p.add_argument("--pass", dest="which", default="forward", choices=["forward", "backward"],
+                   help="forward (the headline metric) or the backward pass of the same workload (bf16)")
     return p.parse_args()
 
 
@@ -166,6 +168,56 @@ def run_reference(args, cfg, rank):
     print(json.dumps(line), flush=True)
 
 
+def run_backward(args, cfg):
+    """Times mok_moe_backward (activation recomputation, dx, router-weight and weight gradients) on one GPU.  FLOPs
+    are counted as twice the forward pass's (dgrad + wgrad), as in the paper's Section 4.1; the recomputed gate/up
+    product and the transposes are extra work that is not counted."""
+    import numpy as np
+    import torch
+    from paper_2609_36070_b200 import inputs, mok
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    d = inputs.make_inputs(cfg)
+    g = {k: (None if d[k] is None else mok.to_device_bf16(d[k], dev)) for k in ("x", "W_gate_up", "W_down", "W_sgu", "W_sd")}
+    W_r = torch.from_numpy(d["W_r"]).to(dev)
+    bias = None if d["bias"] is None else torch.from_numpy(d["bias"]).to(dev)
+    ws = mok.alloc_workspace(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k, device=dev)
+    out, st = mok.mok_moe_forward_ex(g["x"], W_r, bias, g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], cfg.k, ws,
+                                     stages=True)
+    idx, w = st["topk_idx"], st["topk_w"]
+    rng = np.random.default_rng(1)
+    dout = mok.to_device_bf16(inputs.f32_to_bf16_bits(rng.standard_normal((cfg.T, cfg.H), dtype=np.float32)), dev)
+    res = mok.mok_moe_backward(g["x"], g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], idx, w, dout)
+    bws = res["workspace"]
+    conf = mok._config(cta_group=args.cta_group)
+
+    def step():
+        mok.mok_moe_backward(g["x"], g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], idx, w, dout, workspace=bws,
+                             config=conf)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0)
+    sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for _ in range(args.steps):
+        step()
+    ev1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = ev0.elapsed_time(ev1) / args.steps
+    assert mok.mok_read_status(bws) == 0
+    flops = 2.0 * cfg.ffn_flops()
+    print(json.dumps({"metric": "moe_layer_bwd_tokens_per_s", "value": cfg.T / (ms * 1e-3), "unit": UNIT, "n_gpus": 1,
+                      "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True,
+                      "dtype": "bf16", "data": "synthetic", "tflops": flops / (ms * 1e-3) / 1e12,
+                      "config": {"workload": cfg.name, "T": cfg.T, "H": cfg.H, "E": cfg.E, "k": cfg.k, "I": cfg.I,
+                                 "I_shared": cfg.I_s, "pass": "backward (recompute + dgrad + wgrad)"},
+                      "clocks": clocks}), flush=True)
+
+
 def main():
     args = parse()
     rank = int(os.environ.get("RANK", "0"))
@@ -177,6 +229,10 @@ def main():
         cfg = cfg.with_tokens(args.tokens)
     if args.impl == "reference":
         run_reference(args, cfg, rank)
+        return
+    if args.which == "backward":
+        if rank == 0:
+            run_backward(args, cfg)
         return
 
     import numpy as np

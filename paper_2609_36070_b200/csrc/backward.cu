@@ -27,30 +27,61 @@
 
 namespace mok {
 
-// [B, R, C] -> [B, C, R] for bf16, 64 x 64 tiles through shared memory.  Zero-fills nothing: R and C are exact.
+// [B, R, C] -> [B, C, R] for bf16 (C a multiple of 8), 64 x 64 tiles through shared memory with 16-byte global
+// accesses on both sides: a block reads 64 row segments of 128 bytes and writes 64 column segments of 128 bytes.
+// With `route_of_row` the source rows are gathered on the fly: row p of the (padded) dispatch space is token
+// route_of_row[p] / k of `in` when p is a real row of its expert, and zero when it is padding -- the gather and the
+// transpose of the weight-gradient operands in one pass.  Rows >= R of the last tile are not written (out_ld >= R).
 __global__ void __launch_bounds__(256)
 transpose_kernel(const __nv_bfloat16* __restrict__ in, __nv_bfloat16* __restrict__ out, int R, int C, long long in_batch,
-                 long long out_batch, int out_ld) {
-    __shared__ __nv_bfloat16 tile[64][66];
+                 long long out_batch, int out_ld, const int32_t* __restrict__ route_of_row, int k,
+                 const int32_t* __restrict__ tile_expert, const int32_t* __restrict__ pad_offsets,
+                 const int32_t* __restrict__ counts, const WsHeader* __restrict__ hdr) {
+    __shared__ __align__(16) __nv_bfloat16 tile[64][72];      // row pitch 144 bytes: 16-byte aligned, conflicts <= 2-way
     const __nv_bfloat16* src = in + (size_t)blockIdx.z * in_batch;
     __nv_bfloat16* dst = out + (size_t)blockIdx.z * out_batch;
     const int r0 = blockIdx.y * 64, c0 = blockIdx.x * 64;
-    for (int i = threadIdx.x; i < 64 * 64; i += 256) {
-        const int r = i >> 6, c = i & 63;
-        tile[r][c] = (r0 + r < R && c0 + c < C) ? src[(size_t)(r0 + r) * C + c0 + c] : __float2bfloat16(0.f);
+    const int rows_live = route_of_row ? hdr->n_mtiles * TILE_M : R;   // gather mode: rows beyond the schedule are zero
+#pragma unroll
+    for (int pass = 0; pass < 2; ++pass) {
+        const int r = (threadIdx.x >> 3) + pass * 32, ch = threadIdx.x & 7;
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        const int p = r0 + r;
+        if (p < R && c0 + ch * 8 < C) {
+            long long srow = p;
+            if (route_of_row) {
+                srow = -1;
+                if (p < rows_live) {
+                    const int e = tile_expert[p / TILE_M];
+                    if (p - pad_offsets[e] < counts[e]) srow = route_of_row[p] / k;
+                }
+            }
+            if (srow >= 0) v = __ldg(reinterpret_cast<const uint4*>(src + (size_t)srow * C + c0 + ch * 8));
+        }
+        *reinterpret_cast<uint4*>(&tile[r][ch * 8]) = v;
     }
     __syncthreads();
-    for (int i = threadIdx.x; i < 64 * 64; i += 256) {
-        const int c = i >> 6, r = i & 63;
-        if (c0 + c < C && r0 + r < R) dst[(size_t)(c0 + c) * out_ld + r0 + r] = tile[r][c];
+#pragma unroll
+    for (int pass = 0; pass < 2; ++pass) {
+        const int c = (threadIdx.x >> 3) + pass * 32, rc = threadIdx.x & 7;
+        if (c0 + c >= C || r0 + rc * 8 >= R) continue;
+        __nv_bfloat16 v[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) v[j] = tile[rc * 8 + j][c];
+        *reinterpret_cast<uint4*>(dst + (size_t)(c0 + c) * out_ld + r0 + rc * 8) = *reinterpret_cast<const uint4*>(v);
     }
 }
 
+// R must be a multiple of 8 wherever the output rows are written 16 bytes at a time: here R is Rpad, Tpad-padded T (the
+// tail chunk past R is written with the zeros read for p >= R; out_ld covers it) or a weight dimension (multiple of 32).
 static cudaError_t launch_transpose(const __nv_bfloat16* in, __nv_bfloat16* out, int batch, int R, int C, int out_ld,
-                                    cudaStream_t s) {
+                                    cudaStream_t s, const int32_t* route_of_row = nullptr, int k = 1,
+                                    const int32_t* tile_expert = nullptr, const int32_t* pad_offsets = nullptr,
+                                    const int32_t* counts = nullptr, const WsHeader* hdr = nullptr) {
     if (batch <= 0 || R <= 0 || C <= 0) return cudaSuccess;
     dim3 grid((C + 63) / 64, (R + 63) / 64, batch);
-    transpose_kernel<<<grid, 256, 0, s>>>(in, out, R, C, (long long)R * C, (long long)C * out_ld, out_ld);
+    transpose_kernel<<<grid, 256, 0, s>>>(in, out, R, C, (long long)R * C, (long long)C * out_ld, out_ld, route_of_row, k,
+                                          tile_expert, pad_offsets, counts, hdr);
     return cudaGetLastError();
 }
 
@@ -284,15 +315,16 @@ int mok_moe_backward(const mok_bwd_args* a) {
     q.dbg_slot = -1;
     const int Rp = L.Rpad, Tp = L.Tpad;
     // dWd_e = gather(dout)_e^T (w h)_e: both operands transposed so that the row index is the contiguous (K) one
-    if ((e = launch_gather(dout, H, k, TILE_M, L, ws, s)) != cudaSuccess) return cuda_fail(e);
-    if ((e = launch_transpose(bf(L.xg), bf(B.doutT), 1, Rp, H, Rp, s)) != cudaSuccess) return cuda_fail(e);
+    const int32_t* rr = reinterpret_cast<const int32_t*>(ws + B.row_route);
+    if ((e = launch_transpose(dout, bf(B.doutT), 1, Rp, H, Rp, s, rr, k, g.tile_expert, g.pad_offsets, g.counts, hdr)) != cudaSuccess)
+        return cuda_fail(e);
     if ((e = launch_transpose(bf(L.h), bf(B.hwT), 1, Rp, I, Rp, s)) != cudaSuccess) return cuda_fail(e);
     q.E = E; q.kgroup_rows = H; q.A = bf(B.doutT); q.a_rows = H; q.K = Rp; q.lda = Rp;
     q.B = bf(B.hwT); q.N = I; q.ldb = Rp; q.C = a->dW_down; q.rows_pad = E * H; q.ldc = I; q.dense_rows = 0;
     if ((e = launch_gemm_m2(q, EPI_BF16, cfg.grid, s)) != cudaSuccess) return cuda_fail(e);
     // dWgu_e = [dg | du]_e^T Xg_e
-    if ((e = launch_gather(x, H, k, TILE_M, L, ws, s)) != cudaSuccess) return cuda_fail(e);
-    if ((e = launch_transpose(bf(L.xg), bf(B.xgT), 1, Rp, H, Rp, s)) != cudaSuccess) return cuda_fail(e);
+    if ((e = launch_transpose(x, bf(B.xgT), 1, Rp, H, Rp, s, rr, k, g.tile_expert, g.pad_offsets, g.counts, hdr)) != cudaSuccess)
+        return cuda_fail(e);
     if ((e = launch_transpose(bf(B.dgu), bf(B.dguT), 1, Rp, 2 * I, Rp, s)) != cudaSuccess) return cuda_fail(e);
     q.kgroup_rows = 2 * I; q.A = bf(B.dguT); q.a_rows = 2 * I; q.B = bf(B.xgT); q.N = H; q.C = a->dW_gate_up;
     q.rows_pad = E * 2 * I; q.ldc = H;
