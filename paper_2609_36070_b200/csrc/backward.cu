@@ -27,25 +27,30 @@
 
 namespace mok {
 
-// [B, R, C] -> [B, C, R] for bf16 (C a multiple of 8), 64 x 64 tiles through shared memory with 16-byte global
-// accesses on both sides: a block reads 64 row segments of 128 bytes and writes 64 column segments of 128 bytes.
+// [B, R, C] -> [B, C, R] for bf16 (C a multiple of 8), 128 x 128 tiles through shared memory with 16-byte global
+// accesses on both sides: a block reads 128 row segments of 256 bytes and writes 128 column segments of 256 bytes.
 // With `route_of_row` the source rows are gathered on the fly: row p of the (padded) dispatch space is token
 // route_of_row[p] / k of `in` when p is a real row of its expert, and zero when it is padding -- the gather and the
 // transpose of the weight-gradient operands in one pass.  Rows >= R of the last tile are not written (out_ld >= R).
+constexpr int TT = 128;                                       // transpose tile: 128 x 128 elements
 __global__ void __launch_bounds__(256)
 transpose_kernel(const __nv_bfloat16* __restrict__ in, __nv_bfloat16* __restrict__ out, int R, int C, long long in_batch,
                  long long out_batch, int out_ld, const int32_t* __restrict__ route_of_row, int k,
                  const int32_t* __restrict__ tile_expert, const int32_t* __restrict__ pad_offsets,
                  const int32_t* __restrict__ counts, const WsHeader* __restrict__ hdr) {
-    __shared__ __align__(16) __nv_bfloat16 tile[64][72];      // row pitch 144 bytes: 16-byte aligned, conflicts <= 2-way
+    // 32-bit words, row r at word r * PW + (r >> 3): the skew of one word per 8 rows keeps the column reads of the
+    // write phase (rows 8 apart across the lanes) on different banks
+    extern __shared__ __align__(16) uint32_t tile[];
+    constexpr int PW = TT / 2 + 4;
     const __nv_bfloat16* src = in + (size_t)blockIdx.z * in_batch;
     __nv_bfloat16* dst = out + (size_t)blockIdx.z * out_batch;
-    const int r0 = blockIdx.y * 64, c0 = blockIdx.x * 64;
+    const int r0 = blockIdx.y * TT, c0 = blockIdx.x * TT;
     const int rows_live = route_of_row ? hdr->n_mtiles * TILE_M : R;   // gather mode: rows beyond the schedule are zero
+    uint4 v[8];
 #pragma unroll
-    for (int pass = 0; pass < 2; ++pass) {
-        const int r = (threadIdx.x >> 3) + pass * 32, ch = threadIdx.x & 7;
-        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    for (int pass = 0; pass < 8; ++pass) {                     // 8 independent 16-byte loads per thread in flight
+        const int r = (threadIdx.x >> 4) + pass * 16, ch = threadIdx.x & 15;
+        v[pass] = make_uint4(0u, 0u, 0u, 0u);
         const int p = r0 + r;
         if (p < R && c0 + ch * 8 < C) {
             long long srow = p;
@@ -56,19 +61,31 @@ transpose_kernel(const __nv_bfloat16* __restrict__ in, __nv_bfloat16* __restrict
                     if (p - pad_offsets[e] < counts[e]) srow = route_of_row[p] / k;
                 }
             }
-            if (srow >= 0) v = __ldg(reinterpret_cast<const uint4*>(src + (size_t)srow * C + c0 + ch * 8));
+            if (srow >= 0) v[pass] = __ldg(reinterpret_cast<const uint4*>(src + (size_t)srow * C + c0 + ch * 8));
         }
-        *reinterpret_cast<uint4*>(&tile[r][ch * 8]) = v;
+    }
+#pragma unroll
+    for (int pass = 0; pass < 8; ++pass) {
+        const int r = (threadIdx.x >> 4) + pass * 16, ch = threadIdx.x & 15;
+        uint32_t* row = tile + r * PW + (r >> 3) + ch * 4;
+        row[0] = v[pass].x; row[1] = v[pass].y; row[2] = v[pass].z; row[3] = v[pass].w;
     }
     __syncthreads();
 #pragma unroll
-    for (int pass = 0; pass < 2; ++pass) {
-        const int c = (threadIdx.x >> 3) + pass * 32, rc = threadIdx.x & 7;
+    for (int pass = 0; pass < 8; ++pass) {
+        const int c = (threadIdx.x >> 4) + pass * 16, rc = threadIdx.x & 15;
         if (c0 + c >= C || r0 + rc * 8 >= R) continue;
-        __nv_bfloat16 v[8];
+        uint32_t wv[8];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) v[j] = tile[rc * 8 + j][c];
-        *reinterpret_cast<uint4*>(dst + (size_t)(c0 + c) * out_ld + r0 + rc * 8) = *reinterpret_cast<const uint4*>(v);
+        for (int j = 0; j < 8; ++j) {
+            const int r = rc * 8 + j;
+            wv[j] = tile[r * PW + (r >> 3) + (c >> 1)];
+        }
+        const uint32_t sel = (c & 1) ? 0x7632u : 0x5410u;          // high or low halves of two words
+        uint4 o;
+        o.x = __byte_perm(wv[0], wv[1], sel); o.y = __byte_perm(wv[2], wv[3], sel);
+        o.z = __byte_perm(wv[4], wv[5], sel); o.w = __byte_perm(wv[6], wv[7], sel);
+        *reinterpret_cast<uint4*>(dst + (size_t)(c0 + c) * out_ld + r0 + rc * 8) = o;
     }
 }
 
@@ -79,8 +96,15 @@ static cudaError_t launch_transpose(const __nv_bfloat16* in, __nv_bfloat16* out,
                                     const int32_t* tile_expert = nullptr, const int32_t* pad_offsets = nullptr,
                                     const int32_t* counts = nullptr, const WsHeader* hdr = nullptr) {
     if (batch <= 0 || R <= 0 || C <= 0) return cudaSuccess;
-    dim3 grid((C + 63) / 64, (R + 63) / 64, batch);
-    transpose_kernel<<<grid, 256, 0, s>>>(in, out, R, C, (long long)R * C, (long long)C * out_ld, out_ld, route_of_row, k,
+    static bool attr_set = false;
+    constexpr int smem = (TT * (TT / 2 + 4) + TT / 8) * 4;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(transpose_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    dim3 grid((C + TT - 1) / TT, (R + TT - 1) / TT, batch);
+    transpose_kernel<<<grid, 256, smem, s>>>(in, out, R, C, (long long)R * C, (long long)C * out_ld, out_ld, route_of_row, k,
                                           tile_expert, pad_offsets, counts, hdr);
     return cudaGetLastError();
 }
