@@ -245,6 +245,7 @@ int mok_moe_backward(const mok_bwd_args* a) {
     if (!a->workspace || (reinterpret_cast<uintptr_t>(a->workspace) & 255u) || a->workspace_bytes < B.total)
         return MOK_ERR_WORKSPACE;
     if (a->config && (a->config->impl != MOK_IMPL_TCGEN05 || a->config->grid < 0 || a->config->precision != MOK_PRECISION_BF16 ||
+                      a->config->gather_mode < 0 || a->config->gather_mode > 2 ||
                       (a->config->cta_group != 0 && a->config->cta_group != 1 && a->config->cta_group != 3)))
         return MOK_ERR_SHAPE;
     const bool want_w = a->dW_gate_up || a->dW_down || a->dW_shared_gate_up || a->dW_shared_down;
@@ -267,9 +268,27 @@ int mok_moe_backward(const mok_bwd_args* a) {
     e = launch_schedule(a->topk_idx, T, E, k, TILE_M, TILE_M, L, ws, nullptr, nullptr, nullptr, nullptr, s,
                         reinterpret_cast<int32_t*>(ws + B.row_route));
     if (e != cudaSuccess) return cuda_fail(e);
-    // K-contiguous copies of the transposed weights
-    if ((e = launch_transpose(reinterpret_cast<const __nv_bfloat16*>(a->W_down), bf(B.WdT), E, H, I, H, s)) != cudaSuccess) return cuda_fail(e);
-    if ((e = launch_transpose(reinterpret_cast<const __nv_bfloat16*>(a->W_gate_up), bf(B.WguT), E, 2 * I, H, 2 * I, s)) != cudaSuccess) return cuda_fail(e);
+    // The transposed products of dgrad read the weights MN-major, as they sit in memory (W[e] = [K, N], N contiguous).
+    // config.gather_mode = 2 selects the older path instead: K-contiguous transposed copies made at every call.
+    const bool wT = a->config && a->config->gather_mode == 2;
+    if (wT) {
+        if ((e = launch_transpose(reinterpret_cast<const __nv_bfloat16*>(a->W_down), bf(B.WdT), E, H, I, H, s)) != cudaSuccess) return cuda_fail(e);
+        if ((e = launch_transpose(reinterpret_cast<const __nv_bfloat16*>(a->W_gate_up), bf(B.WguT), E, 2 * I, H, 2 * I, s)) != cudaSuccess) return cuda_fail(e);
+    }
+    auto dgrad_gemm = [&](GemmArgs& q, const void* W, size_t WT_off) -> int {
+        if (wT) { q.B = bf(WT_off); q.b_mn = 0; return run_gemm(q, false, &cfg, L, ws, s); }
+        q.B = reinterpret_cast<const __nv_bfloat16*>(W); q.b_mn = 1;
+        WsHeader* h2 = hdr;
+        q.n_mtiles = q.dense_rows > 0 ? q.n_mtiles : &h2->n_mtiles2;        // the 256-row kernel's tile table
+        const int32_t* mt = q.mt_start; const int32_t* te = q.tile_expert;
+        if (q.dense_rows == 0) {
+            q.mt_start = reinterpret_cast<const int32_t*>(ws + L.mt_start2);
+            q.tile_expert = reinterpret_cast<const int32_t*>(ws + L.tile_expert2);
+        }
+        cudaError_t ee = launch_gemm_m2(q, EPI_BF16, cfg.grid, s);
+        q.n_mtiles = &h2->n_mtiles; q.mt_start = mt; q.tile_expert = te; q.b_mn = 0;
+        return ee == cudaSuccess ? MOK_OK : cuda_fail(ee);
+    };
 
     GemmArgs g;
     memset(&g, 0, sizeof(g));
@@ -290,8 +309,8 @@ int mok_moe_backward(const mok_bwd_args* a) {
     g.C = ws + B.gu; g.K = H; g.N = 2 * I; g.ldc = 2 * I;
     if ((rc = run_gemm(g, false, &cfg, L, ws, s))) return rc;
     // dhu = gather(dout) Wd
-    g.A = dout; g.B = bf(B.WdT); g.C = ws + B.dhu; g.K = H; g.N = I; g.ldc = I;
-    if ((rc = run_gemm(g, false, &cfg, L, ws, s))) return rc;
+    g.A = dout; g.C = ws + B.dhu; g.K = H; g.N = I; g.ldc = I;
+    if ((rc = dgrad_gemm(g, a->W_down, B.WdT))) return rc;
     // SwiGLU backward + router-weight gradient
     {
         int blocks = (L.Rpad + 7) / 8;
@@ -303,23 +322,25 @@ int mok_moe_backward(const mok_bwd_args* a) {
     }
     // dXg = [dg | du] Wgu
     g.row_token = nullptr;
-    g.A = bf(B.dgu); g.a_rows = L.Rpad; g.B = bf(B.WguT); g.C = ws + L.y; g.K = 2 * I; g.N = H; g.ldc = H;
-    if ((rc = run_gemm(g, false, &cfg, L, ws, s))) return rc;
+    g.A = bf(B.dgu); g.a_rows = L.Rpad; g.C = ws + L.y; g.K = 2 * I; g.N = H; g.ldc = H;
+    if ((rc = dgrad_gemm(g, a->W_gate_up, B.WguT))) return rc;
     if (Is > 0) {   // shared expert: the same chain on every token, w = 1
-        if ((e = launch_transpose(reinterpret_cast<const __nv_bfloat16*>(a->W_shared_down), bf(B.WsdT), 1, H, Is, H, s)) != cudaSuccess) return cuda_fail(e);
-        if ((e = launch_transpose(reinterpret_cast<const __nv_bfloat16*>(a->W_shared_gate_up), bf(B.WsguT), 1, 2 * Is, H, 2 * Is, s)) != cudaSuccess) return cuda_fail(e);
+        if (wT) {
+            if ((e = launch_transpose(reinterpret_cast<const __nv_bfloat16*>(a->W_shared_down), bf(B.WsdT), 1, H, Is, H, s)) != cudaSuccess) return cuda_fail(e);
+            if ((e = launch_transpose(reinterpret_cast<const __nv_bfloat16*>(a->W_shared_gate_up), bf(B.WsguT), 1, 2 * Is, H, 2 * Is, s)) != cudaSuccess) return cuda_fail(e);
+        }
         g.E = 1; g.rows_pad = L.Tpad; g.dense_rows = T; g.a_rows = T;
         g.A = x; g.B = reinterpret_cast<const __nv_bfloat16*>(a->W_shared_gate_up); g.C = ws + B.gus; g.K = H; g.N = 2 * Is; g.ldc = 2 * Is;
         if ((rc = run_gemm(g, false, &cfg, L, ws, s))) return rc;
-        g.A = dout; g.B = bf(B.WsdT); g.C = ws + B.dhus; g.K = H; g.N = Is; g.ldc = Is;
-        if ((rc = run_gemm(g, false, &cfg, L, ws, s))) return rc;
+        g.A = dout; g.C = ws + B.dhus; g.K = H; g.N = Is; g.ldc = Is;
+        if ((rc = dgrad_gemm(g, a->W_shared_down, B.WsdT))) return rc;
         int blocks = (T + 7) / 8;
         if (blocks > 148 * 16) blocks = 148 * 16;
         swiglu_bwd_kernel<<<blocks, 256, 0, s>>>(bf(B.gus), bf(B.dhus), Is, T, hdr, nullptr, nullptr, nullptr, nullptr,
                                                  nullptr, bf(B.dgus), bf(L.hs), nullptr);
         if ((e = cudaGetLastError()) != cudaSuccess) return cuda_fail(e);
-        g.A = bf(B.dgus); g.a_rows = L.Tpad; g.B = bf(B.WsguT); g.C = ws + L.ysh; g.K = 2 * Is; g.N = H; g.ldc = H;
-        if ((rc = run_gemm(g, false, &cfg, L, ws, s))) return rc;
+        g.A = bf(B.dgus); g.a_rows = L.Tpad; g.C = ws + L.ysh; g.K = 2 * Is; g.N = H; g.ldc = H;
+        if ((rc = dgrad_gemm(g, a->W_shared_gate_up, B.WsguT))) return rc;
     }
     // dx[t] = dx_shared[t] + sum_s dXg[pos[t,s]]: the forward combine with unit weights, same fixed order
     e = launch_combine(L, ws, T, H, k, Is > 0, reinterpret_cast<__nv_bfloat16*>(a->dx), s, /*unit_weights=*/true);
@@ -338,6 +359,29 @@ int mok_moe_backward(const mok_bwd_args* a) {
     q.pad_offsets = g.pad_offsets; q.counts = g.counts;
     q.dbg_slot = -1;
     const int Rp = L.Rpad, Tp = L.Tpad;
+    if (!wT) {
+        // Both operands of a weight-gradient product are read MN-major, exactly as the chain above left them:
+        // A = [rows, M] and B = [rows, N] with the row index as K.  Only the row gather of dout / x is materialised.
+        q.b_mn = 1; q.E = E; q.dense_rows = 0; q.K = Rp;
+        if ((e = launch_gather(dout, H, k, TILE_M, L, ws, s)) != cudaSuccess) return cuda_fail(e);
+        q.kgroup_rows = H; q.A = bf(L.xg); q.lda = H; q.B = bf(L.h); q.N = I; q.ldb = I;
+        q.C = a->dW_down; q.rows_pad = E * H; q.ldc = I;
+        if ((e = launch_gemm_m2(q, EPI_BF16, cfg.grid, s)) != cudaSuccess) return cuda_fail(e);
+        if ((e = launch_gather(x, H, k, TILE_M, L, ws, s)) != cudaSuccess) return cuda_fail(e);
+        q.kgroup_rows = 2 * I; q.A = bf(B.dgu); q.lda = 2 * I; q.B = bf(L.xg); q.N = H; q.ldb = H;
+        q.C = a->dW_gate_up; q.rows_pad = E * 2 * I; q.ldc = H;
+        if ((e = launch_gemm_m2(q, EPI_BF16, cfg.grid, s)) != cudaSuccess) return cuda_fail(e);
+        if (Is > 0) {   // shared expert: one K range over the T tokens (rows past T are zero-filled by the tensor maps)
+            q.E = 1; q.dense_rows = T; q.K = T;
+            q.kgroup_rows = H; q.A = dout; q.lda = H; q.B = bf(L.hs); q.N = Is; q.ldb = Is;
+            q.C = a->dW_shared_down; q.rows_pad = H; q.ldc = Is;
+            if ((e = launch_gemm_m2(q, EPI_BF16, cfg.grid, s)) != cudaSuccess) return cuda_fail(e);
+            q.kgroup_rows = 2 * Is; q.A = bf(B.dgus); q.lda = 2 * Is; q.B = x; q.N = H; q.ldb = H;
+            q.C = a->dW_shared_gate_up; q.rows_pad = 2 * Is; q.ldc = H;
+            if ((e = launch_gemm_m2(q, EPI_BF16, cfg.grid, s)) != cudaSuccess) return cuda_fail(e);
+        }
+        return MOK_OK;
+    }
     // dWd_e = gather(dout)_e^T (w h)_e: both operands transposed so that the row index is the contiguous (K) one
     const int32_t* rr = reinterpret_cast<const int32_t*>(ws + B.row_route);
     if ((e = launch_transpose(dout, bf(B.doutT), 1, Rp, H, Rp, s, rr, k, g.tile_expert, g.pad_offsets, g.counts, hdr)) != cudaSuccess)

@@ -103,12 +103,31 @@ __device__ __forceinline__ Tile decode_tile(const GemmArgs& a, int L, int n_nt, 
     return t;
 }
 
-// KGROUP: the K-range mode (weight gradients), compiled separately so that the forward kernels carry none of it.
-template <int EPI, bool GATHER, bool KGROUP>
+// Shared-memory matrix descriptor of an MN-major bf16 operand tile (the N index contiguous in global memory): groups of
+// 64 N-elements x 64 K-rows, each a [K row][128 bytes] block with the 128-byte swizzle; consecutive N groups are
+// `group_bytes` apart (leading byte offset), consecutive groups of 8 K-rows 1024 bytes (stride byte offset).
+__device__ __forceinline__ uint64_t make_smem_desc_mn(uint32_t addr, uint32_t group_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)(group_bytes >> 4) << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+
+// MODE 0: forward layout.  MODE 1 (KGROUP): the K-range mode (weight gradients).  MODE 2 (BMN): B is read MN-major,
+// i.e. W[e] is [K, N] with N contiguous -- the weights as they sit in memory serve the transposed products of the
+// backward pass (dL/dh = dy Wd, dXg = [dg|du] Wgu) without a transposed copy.  Compiled separately so that the
+// forward kernels carry none of it.
+template <int EPI, bool GATHER, int MODE>
 __global__ void __launch_bounds__(THREADS + (GATHER ? GATHER_THREADS : 0), 1)
 gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
                const __grid_constant__ CUtensorMap tmapC, const __grid_constant__ GemmArgs a, const int n_nt, const int k_blocks) {
     constexpr bool SWIGLU = (EPI == EPI_SWIGLU);
+    // MODE 3: the K-range mode with BOTH operands read MN-major: A = [rows of the dispatch space, M] and
+    // B = [rows, N] as the backward pass produces them, no transposed copies
+    constexpr bool KGROUP = (MODE == 1 || MODE == 3), BMN = (MODE == 2 || MODE == 3), AMN = (MODE == 3);
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -164,12 +183,26 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
                     const uint32_t full = smem_u32(&ctrl->full[s]);
                     const uint32_t sa = base + s * STAGE_BYTES, sb = sa + 2 * A_BYTES;
                     mbar_expect_tx(full, B_BYTES + (GATHER ? 0 : (two ? 2 : 1) * A_BYTES));
-                    if (!GATHER) {
+                    if (AMN) {   // per half two boxes of 64 M-columns x 64 K-rows (K = rows of the dispatch space)
+                        tma_load_2d(sa, &tmapA, full, t.row0, t.kcol0 + kb * BK);
+                        tma_load_2d(sa + A_BYTES / 2, &tmapA, full, t.row0 + 64, t.kcol0 + kb * BK);
+                        if (two) {
+                            tma_load_2d(sa + A_BYTES, &tmapA, full, t.row0 + BM, t.kcol0 + kb * BK);
+                            tma_load_2d(sa + A_BYTES + A_BYTES / 2, &tmapA, full, t.row0 + BM + 64, t.kcol0 + kb * BK);
+                        }
+                    } else if (!GATHER) {
                         tma_load_2d(sa, &tmapA, full, t.kcol0 + kb * BK, t.row0);
                         if (two) tma_load_2d(sa + A_BYTES, &tmapA, full, t.kcol0 + kb * BK, t.row0 + BM);
                     }
-                    tma_load_2d(sb, &tmapB, full, t.kcol0 + kb * BK, brow0);
-                    tma_load_2d(sb + B_BYTES / 2, &tmapB, full, t.kcol0 + kb * BK, brow1);
+                    if (BMN) {   // four boxes of 64 N-columns x 64 K-rows: W[e] viewed as [E * K, N], or the shared B rows
+                        const int krow = AMN ? t.kcol0 + kb * BK : t.e * a.K + kb * BK;
+#pragma unroll
+                        for (int q = 0; q < 4; ++q)
+                            tma_load_2d(sb + q * (B_BYTES / 4), &tmapB, full, t.n * BN + q * 64, krow);
+                    } else {
+                        tma_load_2d(sb, &tmapB, full, t.kcol0 + kb * BK, brow0);
+                        tma_load_2d(sb + B_BYTES / 2, &tmapB, full, t.kcol0 + kb * BK, brow1);
+                    }
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
                 if (!ok) break;
@@ -204,11 +237,16 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t sa = base + s * STAGE_BYTES;
-                    const uint64_t a0 = make_smem_desc(sa), a1 = make_smem_desc(sa + A_BYTES);
-                    const uint64_t bd = make_smem_desc(sa + 2 * A_BYTES);
+                    const uint64_t a0 = AMN ? make_smem_desc_mn(sa, A_BYTES / 2) : make_smem_desc(sa);
+                    const uint64_t a1 = AMN ? make_smem_desc_mn(sa + A_BYTES, A_BYTES / 2) : make_smem_desc(sa + A_BYTES);
+                    constexpr uint32_t ASTEP = AMN ? (2048 >> 4) : 2;
+                    // K-major B: +32 bytes per K = 16 step inside the swizzled row; MN-major B: +2 groups of 8 K-rows
+                    const uint64_t bd = BMN ? make_smem_desc_mn(sa + 2 * A_BYTES, B_BYTES / 4) : make_smem_desc(sa + 2 * A_BYTES);
+                    constexpr uint32_t BSTEP = BMN ? (2048 >> 4) : 2;
+                    constexpr uint32_t IDESC_K = IDESC | (BMN ? (1u << 16) : 0u) | (AMN ? (1u << 15) : 0u);
 #pragma unroll
                     for (int j = 0; j < BK / UMMA_K; ++j)
-                        tc_mma<1>(d0, a0 + (uint64_t)(j * 2), bd + (uint64_t)(j * 2), IDESC, (kb | j) ? 1u : 0u);
+                        tc_mma<1>(d0, a0 + (uint64_t)(j * ASTEP), bd + (uint64_t)(j * BSTEP), IDESC_K, (kb | j) ? 1u : 0u);
                     if (kb == t.kblocks - 1) { tc_commit<1>(smem_u32(&ctrl->tfull[0])); ap0 ^= 1u; }
                     if (two) {
                         if (kb == 0) {
@@ -220,7 +258,7 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
                         }
 #pragma unroll
                         for (int j = 0; j < BK / UMMA_K; ++j)
-                            tc_mma<1>(d1, a1 + (uint64_t)(j * 2), bd + (uint64_t)(j * 2), IDESC, (kb | j) ? 1u : 0u);
+                            tc_mma<1>(d1, a1 + (uint64_t)(j * ASTEP), bd + (uint64_t)(j * BSTEP), IDESC_K, (kb | j) ? 1u : 0u);
                     }
                     tc_commit<1>(smem_u32(&ctrl->empty[s]));
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
@@ -418,12 +456,12 @@ static bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t co
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int EPI, bool GATHER, bool KGROUP = false>
+template <int EPI, bool GATHER, int MODE = 0>
 static cudaError_t launch_one(const CUtensorMap& mA, const CUtensorMap& mB, const CUtensorMap& mC, const GemmArgs& a,
                               int n_nt, int k_blocks, int grid, cudaStream_t s) {
     static int sm_count = 0;
     if (!sm_count) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_m2_kernel<EPI, GATHER, KGROUP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(gemm_m2_kernel<EPI, GATHER, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              SMEM_BYTES);
         if (e != cudaSuccess) return e;
         int dev = 0;
@@ -431,7 +469,7 @@ static cudaError_t launch_one(const CUtensorMap& mA, const CUtensorMap& mB, cons
         cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
     }
     if (grid <= 0 || grid > sm_count) grid = sm_count;
-    gemm_m2_kernel<EPI, GATHER, KGROUP><<<grid, THREADS + (GATHER ? GATHER_THREADS : 0), SMEM_BYTES, s>>>(mA, mB, mC, a, n_nt,
+    gemm_m2_kernel<EPI, GATHER, MODE><<<grid, THREADS + (GATHER ? GATHER_THREADS : 0), SMEM_BYTES, s>>>(mA, mB, mC, a, n_nt,
                                                                                                  k_blocks);
     return cudaGetLastError();
 }
@@ -445,13 +483,25 @@ cudaError_t launch_gemm_m2(const GemmArgs& a, int epi, int grid, cudaStream_t s)
     const uint64_t b_rows = (uint64_t)a.E * (swiglu ? 2 : 1) * a.N;
     if (a.kgroup_rows > 0 && (epi != EPI_BF16 || gather || (a.kgroup_rows % 32))) return cudaErrorInvalidValue;
     const uint64_t lda = a.lda ? (uint64_t)a.lda : (uint64_t)a.K, ldb = a.ldb ? (uint64_t)a.ldb : (uint64_t)a.K;
-    if (!make_map(&mA, a.A, (uint64_t)a.a_rows, (uint64_t)a.K, BM, lda)) return cudaErrorInvalidValue;
-    if (!make_map(&mB, a.B, a.kgroup_rows > 0 ? (uint64_t)a.N : b_rows, (uint64_t)a.K, BN / 2, ldb)) return cudaErrorInvalidValue;
+    if (a.kgroup_rows > 0 && a.b_mn) {
+        // both operands as produced: A = [K rows, kgroup_rows columns], B = [K rows, N columns]; a.K = rows that exist
+        if (!make_map(&mA, a.A, (uint64_t)a.K, (uint64_t)a.kgroup_rows, 64, lda)) return cudaErrorInvalidValue;
+        if (!make_map(&mB, a.B, (uint64_t)a.K, (uint64_t)a.N, 64, ldb)) return cudaErrorInvalidValue;
+    } else if (!make_map(&mA, a.A, (uint64_t)a.a_rows, (uint64_t)a.K, BM, lda)) return cudaErrorInvalidValue;
+    else if (a.b_mn) {   // W viewed as [E * K, N], N contiguous: boxes of 64 columns x 64 rows
+        if (!make_map(&mB, a.B, (uint64_t)a.E * a.K, (uint64_t)a.N, 64, (uint64_t)a.N)) return cudaErrorInvalidValue;
+    } else if (!make_map(&mB, a.B, a.kgroup_rows > 0 ? (uint64_t)a.N : b_rows, (uint64_t)a.K, BN / 2, ldb)) return cudaErrorInvalidValue;
     if (epi == EPI_F32) mC = mB;      // the fp32 epilogue stores directly
     else if (!make_map(&mC, a.C, (uint64_t)a.rows_pad, (uint64_t)a.N, 32, (uint64_t)a.ldc)) return cudaErrorInvalidValue;
     const int n_nt = swiglu ? (a.N + BN / 2 - 1) / (BN / 2) : (a.N + BN - 1) / BN;
     const int k_blocks = (a.K + BK - 1) / BK;
-    if (a.kgroup_rows > 0) return launch_one<EPI_BF16, false, true>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
+    if (a.kgroup_rows > 0 && a.b_mn) return launch_one<EPI_BF16, false, 3>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
+    if (a.kgroup_rows > 0) return launch_one<EPI_BF16, false, 1>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
+    if (a.b_mn) {
+        if (epi != EPI_BF16) return cudaErrorInvalidValue;
+        return gather ? launch_one<EPI_BF16, true, 2>(mA, mB, mC, a, n_nt, k_blocks, grid, s)
+                      : launch_one<EPI_BF16, false, 2>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
+    }
     if (epi == EPI_SWIGLU && gather) return launch_one<EPI_SWIGLU, true>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
     if (epi == EPI_SWIGLU) return launch_one<EPI_SWIGLU, false>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
     if (epi == EPI_BF16 && !gather) return launch_one<EPI_BF16, false>(mA, mB, mC, a, n_nt, k_blocks, grid, s);

@@ -77,6 +77,7 @@ struct GemmArgs {
     // 0 .. dense_rows).  lda / ldb: elements between consecutive rows of A / B (0 = K).
     int32_t kgroup_rows;
     int32_t lda, ldb;
+    int32_t b_mn;                // 256-row kernel: B is W[e] = [K, N] with N contiguous (read MN-major), EPI_BF16 only
     WsHeader* header;
     // Expert-parallel pull dispatch (Section 3.1): with peer_tokens > 0 the ids in row_token are global,
     // id = source_rank * peer_tokens + token, and row `id` is read from peer_x[source_rank] (this GPU's own tokens

@@ -93,7 +93,7 @@ def test_backward_is_reproducible_and_grid_independent():
     m = mok()
     cfg = inputs.MoEConfig("bwd_repro", 512, 256, 16, 4, 256, 128, bias="zipf", seed=53)
     runs = []
-    for conf in (None, None, m._config(grid=3), m._config(cta_group=1)):
+    for conf in (None, None, m._config(grid=3), m._config(cta_group=1), m._config(gather_mode=2)):
         res, _ = run_case(cfg, weight_grads=False, config=conf)
         runs.append((res["dx"].view(torch.int16).clone(), res["dw"].view(torch.int32).clone()))
     for dx, dw in runs[1:]:
