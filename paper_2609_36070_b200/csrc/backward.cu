@@ -303,13 +303,22 @@ int mok_moe_backward(const mok_bwd_args* a) {
     g.dbg_slot = -1;
     g.E = E; g.rows_pad = L.Rpad; g.dense_rows = 0; g.total_rows = L.R;
     int rc;
-    // gu = gather(x) Wgu^T  (activation recomputation)
-    g.A = x; g.a_rows = T; g.row_token = reinterpret_cast<const int32_t*>(ws + L.row_token);
+    // The expert-sorted copies of x and dout (padding rows zero) serve four products each way: made once.  (Pulling the
+    // rows inside the GEMMs, as the forward pass does, would re-gather them once per N tile of 2I and I columns.)
+    __nv_bfloat16* XG = bf(L.xg);
+    __nv_bfloat16* DG = bf(B.doutT);
+    if (!wT) {
+        if ((e = launch_gather(x, H, k, TILE_M, L, ws, s, XG)) != cudaSuccess) return cuda_fail(e);
+        if ((e = launch_gather(dout, H, k, TILE_M, L, ws, s, DG)) != cudaSuccess) return cuda_fail(e);
+    }
+    // gu = Xg Wgu^T  (activation recomputation)
+    if (wT) { g.A = x; g.a_rows = T; g.row_token = reinterpret_cast<const int32_t*>(ws + L.row_token); }
+    else { g.A = XG; g.a_rows = L.Rpad; g.row_token = nullptr; }
     g.B = reinterpret_cast<const __nv_bfloat16*>(a->W_gate_up);
     g.C = ws + B.gu; g.K = H; g.N = 2 * I; g.ldc = 2 * I;
     if ((rc = run_gemm(g, false, &cfg, L, ws, s))) return rc;
     // dhu = gather(dout) Wd
-    g.A = dout; g.C = ws + B.dhu; g.K = H; g.N = I; g.ldc = I;
+    g.A = wT ? dout : DG; g.C = ws + B.dhu; g.K = H; g.N = I; g.ldc = I;
     if ((rc = dgrad_gemm(g, a->W_down, B.WdT))) return rc;
     // SwiGLU backward + router-weight gradient
     {
@@ -361,14 +370,12 @@ int mok_moe_backward(const mok_bwd_args* a) {
     const int Rp = L.Rpad, Tp = L.Tpad;
     if (!wT) {
         // Both operands of a weight-gradient product are read MN-major, exactly as the chain above left them:
-        // A = [rows, M] and B = [rows, N] with the row index as K.  Only the row gather of dout / x is materialised.
+        // A = [rows, M] and B = [rows, N] with the row index as K (Xg and gather(dout) were made at the start).
         q.b_mn = 1; q.E = E; q.dense_rows = 0; q.K = Rp;
-        if ((e = launch_gather(dout, H, k, TILE_M, L, ws, s)) != cudaSuccess) return cuda_fail(e);
-        q.kgroup_rows = H; q.A = bf(L.xg); q.lda = H; q.B = bf(L.h); q.N = I; q.ldb = I;
+        q.kgroup_rows = H; q.A = DG; q.lda = H; q.B = bf(L.h); q.N = I; q.ldb = I;
         q.C = a->dW_down; q.rows_pad = E * H; q.ldc = I;
         if ((e = launch_gemm_m2(q, EPI_BF16, cfg.grid, s)) != cudaSuccess) return cuda_fail(e);
-        if ((e = launch_gather(x, H, k, TILE_M, L, ws, s)) != cudaSuccess) return cuda_fail(e);
-        q.kgroup_rows = 2 * I; q.A = bf(B.dgu); q.lda = 2 * I; q.B = bf(L.xg); q.N = H; q.ldb = H;
+        q.kgroup_rows = 2 * I; q.A = bf(B.dgu); q.lda = 2 * I; q.B = XG; q.N = H; q.ldb = H;
         q.C = a->dW_gate_up; q.rows_pad = E * 2 * I; q.ldc = H;
         if ((e = launch_gemm_m2(q, EPI_BF16, cfg.grid, s)) != cudaSuccess) return cuda_fail(e);
         if (Is > 0) {   // shared expert: one K range over the T tokens (rows past T are zero-filled by the tensor maps)

@@ -81,7 +81,8 @@ combine_kernel(const __nv_bfloat16* __restrict__ y, const __nv_bfloat16* __restr
     }
 }
 
-cudaError_t launch_gather(const __nv_bfloat16* x, int H, int k, int tile_m, const WsLayout& L, char* ws, cudaStream_t s) {
+cudaError_t launch_gather(const __nv_bfloat16* x, int H, int k, int tile_m, const WsLayout& L, char* ws, cudaStream_t s,
+                          __nv_bfloat16* dst) {
     int blocks = (L.Rpad + 7) / 8;
     if (blocks > 148 * 64) blocks = 148 * 64;
     gather_kernel<<<blocks, 256, 0, s>>>(x, H, k, tile_m, reinterpret_cast<const WsHeader*>(ws + L.header),
@@ -90,7 +91,7 @@ cudaError_t launch_gather(const __nv_bfloat16* x, int H, int k, int tile_m, cons
                                          reinterpret_cast<const int32_t*>(ws + L.offsets),
                                          reinterpret_cast<const int32_t*>(ws + L.counts),
                                          reinterpret_cast<const int32_t*>(ws + L.perm),
-                                         reinterpret_cast<__nv_bfloat16*>(ws + L.xg));
+                                         dst ? dst : reinterpret_cast<__nv_bfloat16*>(ws + L.xg));
     return cudaGetLastError();
 }
 

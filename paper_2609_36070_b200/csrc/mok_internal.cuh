@@ -108,7 +108,8 @@ cudaError_t launch_router_simt(const __nv_bfloat16* x, const float* Wr, const fl
 cudaError_t launch_schedule(const int32_t* idx, int T, int E, int k, int tile_m, int pad_m, const WsLayout& L, char* ws,
                             int32_t* counts_out, int32_t* offsets_out, int32_t* perm_out, int32_t* inv_out,
                             cudaStream_t s, int32_t* row_route = nullptr);
-cudaError_t launch_gather(const __nv_bfloat16* x, int H, int k, int tile_m, const WsLayout& L, char* ws, cudaStream_t s);
+cudaError_t launch_gather(const __nv_bfloat16* x, int H, int k, int tile_m, const WsLayout& L, char* ws, cudaStream_t s,
+                          __nv_bfloat16* dst = nullptr);   // dst = NULL: the workspace's own expert-sorted buffer
 cudaError_t launch_combine(const WsLayout& L, char* ws, int T, int H, int k, bool shared, __nv_bfloat16* out,
                            cudaStream_t s, bool unit_weights = false);
 cudaError_t launch_ep_schedule(const int32_t* idx_all, int n_ranks, int rank, int routes_per_rank, int k, int tokens_per_rank,
