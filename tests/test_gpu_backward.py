@@ -138,3 +138,34 @@ def test_bench_shape_full_size_sampled():
     for name in ("dx", "dW_gate_up", "dW_down"):
         assert torch.equal(again[name].view(torch.int16), res[name].view(torch.int16)), name
     assert torch.equal(again["dw"].view(torch.int32), res["dw"].view(torch.int32))
+
+
+def test_backward_argument_errors():
+    m = mok()
+    assert m._lib.mok_moe_backward(None) == m.MOK_ERR_NULL
+    assert m.mok_bwd_workspace_bytes(64, 72, 64, 0, 4, 2) == 0                 # H not a multiple of 32
+    assert m.mok_bwd_workspace_bytes(64, 64, 64, 0, 4, 2) > m.mok_workspace_bytes(64, 64, 64, 0, 4, 2)
+    a = m.mok_bwd_args()
+    a.T, a.H, a.I, a.I_shared, a.E, a.k = 64, 64, 40, 0, 4, 2                  # I not a multiple of 32
+    assert m._lib.mok_moe_backward(a) == m.MOK_ERR_SHAPE
+    a.I = 64
+    assert m._lib.mok_moe_backward(a) == m.MOK_ERR_NULL                        # nothing given
+    a.T = 0
+    assert m._lib.mok_moe_backward(a) == m.MOK_OK                              # nothing to do
+    cfg = inputs.MoEConfig("bwd_err", 64, 64, 4, 2, 64, 0, seed=9)
+    d = inputs.make_inputs(cfg)
+    g = pu.upload(d)
+    out, st = pu.run_gpu(cfg, g)
+    dout = torch.zeros_like(g["x"])
+    small = torch.empty(1024, dtype=torch.uint8, device="cuda")
+    with pytest.raises(m.MokError) as ei:
+        m.mok_moe_backward(g["x"], g["W_gate_up"], g["W_down"], None, None, st["topk_idx"], st["topk_w"], dout,
+                           workspace=small)
+    assert ei.value.status == m.MOK_ERR_WORKSPACE
+    with pytest.raises(m.MokError) as ei:                                      # MXFP8 backward is not built
+        m.mok_moe_backward(g["x"], g["W_gate_up"], g["W_down"], None, None, st["topk_idx"], st["topk_w"], dout,
+                           config=m._config(precision=m.MOK_PRECISION_MXFP8))
+    assert ei.value.status == m.MOK_ERR_SHAPE
+    res = m.mok_moe_backward(g["x"], g["W_gate_up"], g["W_down"], None, None, st["topk_idx"], st["topk_w"], dout)
+    torch.cuda.synchronize()
+    assert all(float(res[n].float().abs().max()) == 0.0 for n in ("dx", "dw", "dW_gate_up", "dW_down"))   # dout = 0
