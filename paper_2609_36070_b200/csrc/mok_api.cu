@@ -598,11 +598,11 @@ int mok_debug_counters(const void* workspace, void* stream, unsigned long long* 
 int mok_launch_count(int T, int H, int I, int I_shared, int E, int k, const mok_config* config) {
     WsLayout L;
     if (!ws_layout(T, H, I, I_shared, E, k, &L) || T == 0) return 0;
-    // router (1 fp32-FMA kernel, or split + GEMM + top-k), 3 schedule kernels, (gather on the SIMT path),
+    // router (1 fp32-FMA kernel, or split + GEMM + top-k + near-tie fix-up), 3 schedule kernels, (gather on the SIMT path),
     // 2 routed GEMMs, (2 shared GEMMs), combine
     // (MXFP8 mode: the token-row quantiser instead of the gather kernel; its two memsets are not counted)
     const int pre = use_mx(config) ? 1 : (fused_gather(config, I) ? 0 : 1);
-    return (use_simt_router(config, k) ? 1 : 3) + 3 + pre + 2 + (I_shared > 0 ? 2 : 0) + 1;
+    return (use_simt_router(config, k) ? 1 : 4) + 3 + pre + 2 + (I_shared > 0 ? 2 : 0) + 1;
 }
 
 int mok_profile_begin(int max_calls) {

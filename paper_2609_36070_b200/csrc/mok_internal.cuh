@@ -22,7 +22,8 @@ struct WsHeader {
     int32_t n_mtiles2;     // number of 2*tile_m-row tiles of the same buffer (second tile table)
     int32_t where;         // diagnostic: which wait gave up (site number inside the kernel)
     uint32_t wait_limit_us; // 0 = default (2 s): bound of every mbarrier wait, in microseconds
-    int32_t pad[59];
+    int32_t n_flag;        // tensor-core router: tokens on the near-tie list of the current call
+    int32_t pad[58];
     // optional wait-time counters of the tcgen05 GEMMs (config.debug): [slot][counter], SM cycles summed over CTAs
     unsigned long long dbg[4][8];
 };

@@ -9,14 +9,18 @@
 //   1. router_split_kernel  W_r [E,H] fp32 -> [ldl, H] bf16 rows: hi (0..E-1), mid (E..2E-1), lo (2E..3E-1), zero pad
 //   2. the tcgen05 GEMM     x [T,H] . split^T -> partial logits fp32 [T, ldl]
 //   3. router_topk_kernel   logit = (lo + mid) + hi + bias, warp-shuffle top-k and softmax weights; tokens with a
-//                           pair of candidates closer than the accumulation error are re-decided with exact FMAs
+//                           pair of candidates closer than the accumulation error are put on a list
+//   4. router_fixup_kernel  the listed tokens (about 1 % of them) are re-decided with exact FMAs.  A kernel of its own,
+//                           because one such token costs a warp ~10 us of dependent L2 round trips: inside kernel 3
+//                           that latency was the kernel's duration
 #include "mok_internal.cuh"
 #include "router_common.cuh"
 
 namespace mok {
 
 __global__ void __launch_bounds__(256)
-router_split_kernel(const float* __restrict__ Wr, int E, int H, int ldl, __nv_bfloat16* __restrict__ out) {
+router_split_kernel(const float* __restrict__ Wr, int E, int H, int ldl, __nv_bfloat16* __restrict__ out, WsHeader* hdr) {
+    if (blockIdx.x == 0 && threadIdx.x == 0) hdr->n_flag = 0;   // the near-tie list of this call starts empty
     const size_t n = (size_t)ldl * H;
     for (size_t i = (size_t)blockIdx.x * 256 + threadIdx.x; i < n; i += (size_t)gridDim.x * 256) {
         const int row = (int)(i / H), h = (int)(i - (size_t)row * H);
@@ -44,6 +48,7 @@ __device__ __forceinline__ void warp_exact_logits4(const __nv_bfloat16* __restri
     const float* wrow[4];
 #pragma unroll
     for (int c = 0; c < 4; ++c) wrow[c] = Wr + (size_t)e[c < n ? c : 0] * H;
+#pragma unroll 4
     for (int h = lane * 8; h < H; h += 256) {
         const uint4 raw = *reinterpret_cast<const uint4*>(xrow + h);
         const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&raw);
@@ -111,29 +116,30 @@ __device__ __forceinline__ void reg_select(float (&v)[VPL], int lane, int s_begi
 //     guard = H * 2^-26 * (1 + max|logit|)      (four times the modelled bound (H/16) * 2^-24 * |acc|)
 // get the logits of their top-(k+4) candidates recomputed with plain fp32 FMAs and are selected again.
 template <int VPL>
+__device__ __forceinline__ void load_logits(const float* __restrict__ row, const float* __restrict__ bias, int E, int lane,
+                                            float (&v)[VPL]) {
+#pragma unroll
+    for (int j = 0; j < VPL; ++j) {
+        const int e = lane + 32 * j;
+        float val = -FLT_MAX;
+        if (e < E) {
+            val = (row[2 * E + e] + row[E + e]) + row[e];      // smallest terms first
+            if (bias) val += bias[e];
+        }
+        v[j] = val;
+    }
+}
+
+template <int VPL>
 __global__ void __launch_bounds__(256)
-router_topk_kernel(const float* __restrict__ part, const float* __restrict__ bias,
-                   const __nv_bfloat16* __restrict__ x, const float* __restrict__ Wr,
-                   int T, int H, int E, int k, int ldl, int32_t* __restrict__ idx, float* __restrict__ w) {
+router_topk_kernel(const float* __restrict__ part, const float* __restrict__ bias, int T, int H, int E, int k, int ldl,
+                   int32_t* __restrict__ idx, float* __restrict__ w, WsHeader* hdr, int32_t* __restrict__ flagged) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_check = (k + 1 < E) ? k + 1 : E;        // slots compared pairwise
-    int n_cand = (k + 4 < E) ? k + 4 : E;               // candidates recomputed when a pair is too close
-    if (n_cand > 32) n_cand = 32;
     const float guard_scale = (float)H * 1.4901161e-8f; // H * 2^-26
     for (int t = blockIdx.x * 8 + warp; t < T; t += gridDim.x * 8) {
-        const float* row = part + (size_t)t * ldl;
-        float orig[VPL], v[VPL];
-#pragma unroll
-        for (int j = 0; j < VPL; ++j) {
-            const int e = lane + 32 * j;
-            float val = -FLT_MAX;
-            if (e < E) {
-                val = (row[2 * E + e] + row[E + e]) + row[e];      // smallest terms first
-                if (bias) val += bias[e];
-            }
-            orig[j] = val;
-            v[j] = val;
-        }
+        float v[VPL];
+        load_logits<VPL>(part + (size_t)t * ldl, bias, E, lane, v);
         TopkState st = {0u, 0.f, 0};
         reg_select<VPL>(v, lane, 0, n_check, st.v, st.e);
         const float next_v = __shfl_down_sync(0xffffffffu, st.v, 1);
@@ -141,31 +147,89 @@ router_topk_kernel(const float* __restrict__ part, const float* __restrict__ bia
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, off));
         const bool close = (lane + 1 < n_check) && (st.v - next_v < guard_scale * (1.f + amax));
-        if (__any_sync(0xffffffffu, close)) {
-            reg_select<VPL>(v, lane, n_check, n_cand, st.v, st.e);
-            for (int c0 = 0; c0 < n_cand; c0 += 4) {
-                int e[4];
-                float ex[4];
+        if (__any_sync(0xffffffffu, close) && lane == 0) flagged[atomicAdd(&hdr->n_flag, 1)] = t;
+        warp_write_topk(st, k, lane, idx + (size_t)t * k, w + (size_t)t * k);   // provisional for a listed token
+    }
+}
+
+// One block per listed token: the logits of its top-(k+4) candidates are recomputed with plain fp32 FMAs, then the
+// top-k is selected again from all E logits and overwrites the provisional result.  There are few such tokens, so the
+// kernel's duration is the latency of one of them: warp 0 selects, all eight warps share the candidates' dot products
+// (each lane keeps many independent loads in flight), warp 0 selects again.  The list's order (atomic appends) does
+// not matter: every token is decided on its own.
+template <int VPL>
+__global__ void __launch_bounds__(256)
+router_fixup_kernel(const float* __restrict__ part, const float* __restrict__ bias,
+                    const __nv_bfloat16* __restrict__ x, const float* __restrict__ Wr, int H, int E, int k, int ldl,
+                    int32_t* __restrict__ idx, float* __restrict__ w, const WsHeader* hdr,
+                    const int32_t* __restrict__ flagged) {
+    __shared__ int s_e[32];
+    __shared__ float s_ex[32];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    int n_cand = (k + 4 < E) ? k + 4 : E;               // candidates recomputed
+    if (n_cand > 32) n_cand = 32;
+    const int n_flag = hdr->n_flag;
+    for (int i = blockIdx.x; i < n_flag; i += gridDim.x) {
+        const int t = flagged[i];
+        float orig[VPL], v[VPL];
+        TopkState st = {0u, 0.f, 0};
+        if (warp == 0) {
+            load_logits<VPL>(part + (size_t)t * ldl, bias, E, lane, orig);
 #pragma unroll
-                for (int c = 0; c < 4; ++c) e[c] = __shfl_sync(0xffffffffu, st.e, (c0 + c < n_cand) ? c0 + c : c0);
-                const int n = (n_cand - c0 < 4) ? n_cand - c0 : 4;
+            for (int j = 0; j < VPL; ++j) v[j] = orig[j];
+            reg_select<VPL>(v, lane, 0, n_cand, st.v, st.e);
+            if (lane < n_cand) s_e[lane] = st.e;
+        }
+        __syncthreads();
+        {   // warp w recomputes candidates w, w + 8, w + 16, w + 24
+            int e[4], n = 0;
+            float ex[4];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const int ci = warp + 8 * c;
+                e[c] = s_e[ci < n_cand ? ci : 0];
+                if (ci < n_cand) n = c + 1;
+            }
+            if (n > 0) {
                 warp_exact_logits4(x + (size_t)t * H, Wr, e, n, H, lane, ex);
+                if (lane == 0) {
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    if (c < n && (e[c] & 31) == lane) {
-                        const float val = ex[c] + (bias ? bias[e[c]] : 0.f);
+                    for (int c = 0; c < 4; ++c)
+                        if (c < n) s_ex[warp + 8 * c] = ex[c];
+                }
+            }
+        }
+        __syncthreads();
+        if (warp == 0) {
+            for (int c = 0; c < n_cand; ++c) {
+                const int ec = s_e[c];
+                if ((ec & 31) == lane) {
+                    const float val = s_ex[c] + (bias ? bias[ec] : 0.f);
 #pragma unroll
-                        for (int j = 0; j < VPL; ++j)
-                            if (j == (e[c] >> 5)) orig[j] = val;
-                    }
+                    for (int j = 0; j < VPL; ++j)
+                        if (j == (ec >> 5)) orig[j] = val;
                 }
             }
 #pragma unroll
             for (int j = 0; j < VPL; ++j) v[j] = orig[j];
             reg_select<VPL>(v, lane, 0, k, st.v, st.e);
+            warp_write_topk(st, k, lane, idx + (size_t)t * k, w + (size_t)t * k);
         }
-        warp_write_topk(st, k, lane, idx + (size_t)t * k, w + (size_t)t * k);
+        __syncthreads();                                // s_e / s_ex are reused by the next token
     }
+}
+
+template <int VPL>
+static cudaError_t launch_topk(const float* part, const float* bias, const __nv_bfloat16* x, const float* Wr, int T, int H,
+                               int E, int k, int ldl, int32_t* idx, float* w, WsHeader* hdr, int32_t* flagged,
+                               cudaStream_t s) {
+    int tblocks = (T + 7) / 8;
+    if (tblocks > 148 * 16) tblocks = 148 * 16;
+    router_topk_kernel<VPL><<<tblocks, 256, 0, s>>>(part, bias, T, H, E, k, ldl, idx, w, hdr, flagged);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    router_fixup_kernel<VPL><<<296, 256, 0, s>>>(part, bias, x, Wr, H, E, k, ldl, idx, w, hdr, flagged);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_router_tc(const __nv_bfloat16* x, const float* Wr, const float* bias, int T, int H, int E, int k,
@@ -177,7 +241,7 @@ cudaError_t launch_router_tc(const __nv_bfloat16* x, const float* Wr, const floa
     size_t n = (size_t)ldl * H;
     int blocks = (int)((n + 255) / 256);
     if (blocks > 148 * 8) blocks = 148 * 8;
-    router_split_kernel<<<blocks, 256, 0, s>>>(Wr, E, H, ldl, split);
+    router_split_kernel<<<blocks, 256, 0, s>>>(Wr, E, H, ldl, split, hdr);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     GemmArgs g = {};
@@ -193,15 +257,14 @@ cudaError_t launch_router_tc(const __nv_bfloat16* x, const float* Wr, const floa
     e = variant == 2 ? launch_gemm_tn(g, EPI_F32, grid, s)
         : variant == 3 ? launch_gemm_m2(g, EPI_F32, grid, s) : launch_gemm_tc(g, EPI_F32, grid, s);
     if (e != cudaSuccess) return e;
-    int tblocks = (T + 7) / 8;
-    if (tblocks > 148 * 16) tblocks = 148 * 16;
+    // the near-tie list lives in the schedule's `perm` region (T*k entries), which is not written before the schedule runs
+    int32_t* flagged = reinterpret_cast<int32_t*>(ws + L.perm);
     const int vpl = (E + 31) / 32;
-    if (vpl <= 1) router_topk_kernel<1><<<tblocks, 256, 0, s>>>(part, bias, x, Wr, T, H, E, k, ldl, idx, w);
-    else if (vpl <= 2) router_topk_kernel<2><<<tblocks, 256, 0, s>>>(part, bias, x, Wr, T, H, E, k, ldl, idx, w);
-    else if (vpl <= 4) router_topk_kernel<4><<<tblocks, 256, 0, s>>>(part, bias, x, Wr, T, H, E, k, ldl, idx, w);
-    else if (vpl <= 8) router_topk_kernel<8><<<tblocks, 256, 0, s>>>(part, bias, x, Wr, T, H, E, k, ldl, idx, w);
-    else router_topk_kernel<16><<<tblocks, 256, 0, s>>>(part, bias, x, Wr, T, H, E, k, ldl, idx, w);
-    return cudaGetLastError();
+    if (vpl <= 1) return launch_topk<1>(part, bias, x, Wr, T, H, E, k, ldl, idx, w, hdr, flagged, s);
+    if (vpl <= 2) return launch_topk<2>(part, bias, x, Wr, T, H, E, k, ldl, idx, w, hdr, flagged, s);
+    if (vpl <= 4) return launch_topk<4>(part, bias, x, Wr, T, H, E, k, ldl, idx, w, hdr, flagged, s);
+    if (vpl <= 8) return launch_topk<8>(part, bias, x, Wr, T, H, E, k, ldl, idx, w, hdr, flagged, s);
+    return launch_topk<16>(part, bias, x, Wr, T, H, E, k, ldl, idx, w, hdr, flagged, s);
 }
 
 }  // namespace mok
