@@ -63,7 +63,9 @@ typedef struct mok_config {
     int32_t impl;         /* MOK_IMPL_* */
     int32_t grid;         /* persistent grid size override for the tcgen05 kernels (0 = number of SMs).  The
                              output bits do not depend on it (Section 3.4 "Determinism"). */
-    int32_t router_impl;  /* 0 = default, 1 = fp32 FMA router, 2 = split-bf16 tensor-core router */
+    int32_t router_impl;  /* 0 = default (split-bf16 tensor-core router; projection and top-k in one kernel for up to
+                             160 experts), 1 = fp32 FMA router, 2 = split-bf16 tensor-core router as three kernels
+                             (split, GEMM, top-k); 0 and 2 give the same bits */
     int32_t profile;      /* != 0: record CUDA events around every stage of this call (see mok_profile_begin) */
     int32_t gather_mode;  /* token gather of the routed gate/up GEMM: 0 = choose by shape, 1 = fused into the GEMM's
                              operand loads (no expert-sorted copy of x), 2 = separate gather kernel + TMA loads */

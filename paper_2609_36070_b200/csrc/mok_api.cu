@@ -67,7 +67,8 @@ bool ws_layout(int T, int H, int I, int Is, int E, int k, WsLayout* L, bool mx) 
     L->pos = take(sizeof(int32_t) * (size_t)(R > 0 ? R : 1));
     L->blk_hist = take(sizeof(int32_t) * (size_t)L->n_blk * E);
     L->row_token = take(sizeof(int32_t) * (size_t)Rpad);
-    const size_t ldl = (size_t)(3 * E + 7) / 8 * 8;
+    size_t ldl = (size_t)(3 * E + 7) / 8 * 8;
+    if (ldl < 3 * (size_t)((E + 31) / 32 * 32)) ldl = 3 * (size_t)((E + 31) / 32 * 32);
     L->wr_split = take(2 * ldl * H);
     L->logits = take(sizeof(float) * (size_t)L->Tpad * ldl);
     L->xg = take(2 * (size_t)Rpad * H);
@@ -128,6 +129,13 @@ static bool use_tn(const mok_config* cfg) { return cfg && cfg->impl == MOK_IMPL_
 static bool use_simt_router(const mok_config* cfg, int k) {
     if (k > 28) return true;   // the tensor-core router keeps k + 4 candidates in one warp's 32 lanes
     return cfg && (cfg->router_impl == 1 || (cfg->router_impl == 0 && cfg->impl == MOK_IMPL_SIMT));
+}
+
+// Projection + top-k in one kernel (router_fused.cu) whenever the shape allows it; router_impl = 2 keeps the
+// three-kernel tensor-core path (split, GEMM, top-k), which also serves more than 160 experts.
+static bool use_fused_router(const mok_config* cfg, int E, int k) {
+    if (use_simt_router(cfg, k) || (cfg && cfg->router_impl == 2)) return false;
+    return router_fused_ok(E, k);
 }
 
 // Whether the routed gate/up GEMM gathers its rows itself.  The fused path re-gathers the rows once per N tile
@@ -193,7 +201,7 @@ static int route_stage(const mok_args* a, const WsLayout& L, char* ws, const __n
                              reinterpret_cast<WsHeader*>(ws + L.header), a->config ? a->config->grid : 0,
                              tile_rows(a->config, a->I > 0 ? a->I : 8),
                              use_tn(a->config) ? 2 : use_m2(a->config, a->H, tile_rows(a->config, a->I > 0 ? a->I : 8), a->T, 1) ? 3 : 0,
-                             idx, w, s);
+                             use_fused_router(a->config, a->E, a->k), idx, w, s);
     if (e != cudaSuccess) return cuda_fail(e);
     if (a->topk_idx) {
         e = cudaMemcpyAsync(a->topk_idx, idx, sizeof(int32_t) * (size_t)L.R, cudaMemcpyDeviceToDevice, s);
@@ -602,7 +610,7 @@ int mok_launch_count(int T, int H, int I, int I_shared, int E, int k, const mok_
     // 2 routed GEMMs, (2 shared GEMMs), combine
     // (MXFP8 mode: the token-row quantiser instead of the gather kernel; its two memsets are not counted)
     const int pre = use_mx(config) ? 1 : (fused_gather(config, I) ? 0 : 1);
-    return (use_simt_router(config, k) ? 1 : 4) + 3 + pre + 2 + (I_shared > 0 ? 2 : 0) + 1;
+    return (use_simt_router(config, k) ? 1 : use_fused_router(config, E, k) ? 3 : 4) + 3 + pre + 2 + (I_shared > 0 ? 2 : 0) + 1;
 }
 
 int mok_profile_begin(int max_calls) {

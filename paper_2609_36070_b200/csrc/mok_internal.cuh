@@ -35,8 +35,9 @@ struct WsLayout {
     size_t header, idx, w, counts, offsets, pad_offsets, mt_start, tile_expert, perm, inv, pos, blk_hist;
     size_t mt_start2, tile_expert2;   // the same segments cut into tiles of 2*tile_m rows
     size_t row_token;     // int32 [Rpad]: source token of every row of the padded dispatch space (pad rows undefined)
-    size_t wr_split;      // bf16 [3E, H]: W_r split into hi/mid/lo parts for the tensor-core router
-    size_t logits;        // fp32 [Tpad, ldl] partial logits of the tensor-core router (ldl = 3E rounded up to 8)
+    size_t wr_split;      // bf16 [ldl, H]: W_r split into hi/mid/lo parts for the tensor-core router
+    size_t logits;        // fp32 [Tpad, ldl] partial logits of the tensor-core router (ldl = 3E rounded up to 8, or
+                          // 3 * (E rounded up to 32) if larger: the one-kernel router pads each part to 32 rows)
     size_t xg, h, y, hs, ysh;
     size_t x8, sx, h8, sh;   // MXFP8 mode: quantised token rows + row-major scales, quantised gated activation + scale atoms
     size_t total;
@@ -131,9 +132,12 @@ cudaError_t launch_mx_quantize_rows(const __nv_bfloat16* in, long long rows, int
 cudaError_t launch_mx_quantize_atoms(const __nv_bfloat16* in, int groups, int rows_per_group, int K, uint8_t* codes,
                                      uint8_t* scales, cudaStream_t s);
 cudaError_t launch_router_tc(const __nv_bfloat16* x, const float* Wr, const float* bias, int T, int H, int E, int k,
-                             const WsLayout& L, char* ws, WsHeader* hdr, int grid, int tile_m, int variant, int32_t* idx,
-                             float* w,
-                             cudaStream_t s);
+                             const WsLayout& L, char* ws, WsHeader* hdr, int grid, int tile_m, int variant, bool fused,
+                             int32_t* idx, float* w, cudaStream_t s);
+bool router_fused_ok(int E, int k);     // the one-kernel projection + top-k serves this shape
+cudaError_t launch_router_fused(const __nv_bfloat16* x, const __nv_bfloat16* split, const float* bias, int T, int H, int E,
+                                int k, float* rows, int32_t* flagged, WsHeader* hdr, int grid, int32_t* idx, float* w,
+                                cudaStream_t s);
 
 inline __host__ __device__ size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 

@@ -18,15 +18,17 @@
 
 namespace mok {
 
+// rows of `out`: part * estride + e for part = hi, mid, lo (estride >= E); every other row is zero
 __global__ void __launch_bounds__(256)
-router_split_kernel(const float* __restrict__ Wr, int E, int H, int ldl, __nv_bfloat16* __restrict__ out, WsHeader* hdr) {
+router_split_kernel(const float* __restrict__ Wr, int E, int estride, int H, int rows, __nv_bfloat16* __restrict__ out,
+                    WsHeader* hdr) {
     if (blockIdx.x == 0 && threadIdx.x == 0) hdr->n_flag = 0;   // the near-tie list of this call starts empty
-    const size_t n = (size_t)ldl * H;
+    const size_t n = (size_t)rows * H;
     for (size_t i = (size_t)blockIdx.x * 256 + threadIdx.x; i < n; i += (size_t)gridDim.x * 256) {
         const int row = (int)(i / H), h = (int)(i - (size_t)row * H);
+        const int part = row / estride, e = row - part * estride;
         float v = 0.f;
-        if (row < 3 * E) {
-            const int part = row / E, e = row - part * E;
+        if (part < 3 && e < E) {
             const float wv = Wr[(size_t)e * H + h];
             const float hi = __bfloat162float(__float2bfloat16_rn(wv));
             const float r1 = wv - hi;                                   // exact
@@ -117,14 +119,18 @@ __device__ __forceinline__ void reg_select(float (&v)[VPL], int lane, int s_begi
 // get the logits of their top-(k+4) candidates recomputed with plain fp32 FMAs and are selected again.
 template <int VPL>
 __device__ __forceinline__ void load_logits(const float* __restrict__ row, const float* __restrict__ bias, int E, int lane,
-                                            float (&v)[VPL]) {
+                                            float (&v)[VPL], bool summed = false) {
 #pragma unroll
     for (int j = 0; j < VPL; ++j) {
         const int e = lane + 32 * j;
         float val = -FLT_MAX;
         if (e < E) {
-            val = (row[2 * E + e] + row[E + e]) + row[e];      // smallest terms first
-            if (bias) val += bias[e];
+            if (summed) {
+                val = row[e];                                  // written by the fused kernel, bias included
+            } else {
+                val = (row[2 * E + e] + row[E + e]) + row[e];  // smallest terms first
+                if (bias) val += bias[e];
+            }
         }
         v[j] = val;
     }
@@ -161,7 +167,7 @@ template <int VPL>
 __global__ void __launch_bounds__(256)
 router_fixup_kernel(const float* __restrict__ part, const float* __restrict__ bias,
                     const __nv_bfloat16* __restrict__ x, const float* __restrict__ Wr, int H, int E, int k, int ldl,
-                    int32_t* __restrict__ idx, float* __restrict__ w, const WsHeader* hdr,
+                    bool summed, int32_t* __restrict__ idx, float* __restrict__ w, const WsHeader* hdr,
                     const int32_t* __restrict__ flagged) {
     __shared__ int s_e[32];
     __shared__ float s_ex[32];
@@ -174,7 +180,7 @@ router_fixup_kernel(const float* __restrict__ part, const float* __restrict__ bi
         float orig[VPL], v[VPL];
         TopkState st = {0u, 0.f, 0};
         if (warp == 0) {
-            load_logits<VPL>(part + (size_t)t * ldl, bias, E, lane, orig);
+            load_logits<VPL>(part + (size_t)t * ldl, bias, E, lane, orig, summed);
 #pragma unroll
             for (int j = 0; j < VPL; ++j) v[j] = orig[j];
             reg_select<VPL>(v, lane, 0, n_cand, st.v, st.e);
@@ -221,50 +227,59 @@ router_fixup_kernel(const float* __restrict__ part, const float* __restrict__ bi
 
 template <int VPL>
 static cudaError_t launch_topk(const float* part, const float* bias, const __nv_bfloat16* x, const float* Wr, int T, int H,
-                               int E, int k, int ldl, int32_t* idx, float* w, WsHeader* hdr, int32_t* flagged,
+                               int E, int k, int ldl, bool fused, int32_t* idx, float* w, WsHeader* hdr, int32_t* flagged,
                                cudaStream_t s) {
-    int tblocks = (T + 7) / 8;
-    if (tblocks > 148 * 16) tblocks = 148 * 16;
-    router_topk_kernel<VPL><<<tblocks, 256, 0, s>>>(part, bias, T, H, E, k, ldl, idx, w, hdr, flagged);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
-    router_fixup_kernel<VPL><<<296, 256, 0, s>>>(part, bias, x, Wr, H, E, k, ldl, idx, w, hdr, flagged);
+    if (!fused) {
+        int tblocks = (T + 7) / 8;
+        if (tblocks > 148 * 16) tblocks = 148 * 16;
+        router_topk_kernel<VPL><<<tblocks, 256, 0, s>>>(part, bias, T, H, E, k, ldl, idx, w, hdr, flagged);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
+    router_fixup_kernel<VPL><<<296, 256, 0, s>>>(part, bias, x, Wr, H, E, k, ldl, fused, idx, w, hdr, flagged);
     return cudaGetLastError();
 }
 
 cudaError_t launch_router_tc(const __nv_bfloat16* x, const float* Wr, const float* bias, int T, int H, int E, int k,
-                             const WsLayout& L, char* ws, WsHeader* hdr, int grid, int tile_m, int variant, int32_t* idx,
-                             float* w, cudaStream_t s) {
-    const int ldl = (3 * E + 7) / 8 * 8;
+                             const WsLayout& L, char* ws, WsHeader* hdr, int grid, int tile_m, int variant, bool fused,
+                             int32_t* idx, float* w, cudaStream_t s) {
+    fused = fused && router_fused_ok(E, k);
+    const int ep = (E + 31) / 32 * 32;
+    const int ldl = fused ? ep : (3 * E + 7) / 8 * 8;       // row stride of the logits buffer
+    const int split_rows = fused ? 3 * ep : ldl;
     __nv_bfloat16* split = reinterpret_cast<__nv_bfloat16*>(ws + L.wr_split);
     float* part = reinterpret_cast<float*>(ws + L.logits);
-    size_t n = (size_t)ldl * H;
-    int blocks = (int)((n + 255) / 256);
-    if (blocks > 148 * 8) blocks = 148 * 8;
-    router_split_kernel<<<blocks, 256, 0, s>>>(Wr, E, H, ldl, split, hdr);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
-    GemmArgs g = {};
-    g.A = x;
-    g.B = split;
-    g.C = part;
-    g.K = H; g.N = ldl; g.E = 1; g.ldc = ldl;
-    g.rows_pad = L.Tpad; g.a_rows = T; g.dense_rows = T;
-    g.max_mt = L.Tpad / TILE_M;
-    g.tile_m = tile_m;
-    g.dbg_slot = -1;
-    g.header = hdr;
-    e = variant == 2 ? launch_gemm_tn(g, EPI_F32, grid, s)
-        : variant == 3 ? launch_gemm_m2(g, EPI_F32, grid, s) : launch_gemm_tc(g, EPI_F32, grid, s);
-    if (e != cudaSuccess) return e;
     // the near-tie list lives in the schedule's `perm` region (T*k entries), which is not written before the schedule runs
     int32_t* flagged = reinterpret_cast<int32_t*>(ws + L.perm);
+    size_t n = (size_t)split_rows * H;
+    int blocks = (int)((n + 255) / 256);
+    if (blocks > 148 * 8) blocks = 148 * 8;
+    router_split_kernel<<<blocks, 256, 0, s>>>(Wr, E, fused ? ep : E, H, split_rows, split, hdr);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    if (fused) {
+        e = launch_router_fused(x, split, bias, T, H, E, k, part, flagged, hdr, grid, idx, w, s);
+    } else {
+        GemmArgs g = {};
+        g.A = x;
+        g.B = split;
+        g.C = part;
+        g.K = H; g.N = ldl; g.E = 1; g.ldc = ldl;
+        g.rows_pad = L.Tpad; g.a_rows = T; g.dense_rows = T;
+        g.max_mt = L.Tpad / TILE_M;
+        g.tile_m = tile_m;
+        g.dbg_slot = -1;
+        g.header = hdr;
+        e = variant == 2 ? launch_gemm_tn(g, EPI_F32, grid, s)
+            : variant == 3 ? launch_gemm_m2(g, EPI_F32, grid, s) : launch_gemm_tc(g, EPI_F32, grid, s);
+    }
+    if (e != cudaSuccess) return e;
     const int vpl = (E + 31) / 32;
-    if (vpl <= 1) return launch_topk<1>(part, bias, x, Wr, T, H, E, k, ldl, idx, w, hdr, flagged, s);
-    if (vpl <= 2) return launch_topk<2>(part, bias, x, Wr, T, H, E, k, ldl, idx, w, hdr, flagged, s);
-    if (vpl <= 4) return launch_topk<4>(part, bias, x, Wr, T, H, E, k, ldl, idx, w, hdr, flagged, s);
-    if (vpl <= 8) return launch_topk<8>(part, bias, x, Wr, T, H, E, k, ldl, idx, w, hdr, flagged, s);
-    return launch_topk<16>(part, bias, x, Wr, T, H, E, k, ldl, idx, w, hdr, flagged, s);
+    if (vpl <= 1) return launch_topk<1>(part, bias, x, Wr, T, H, E, k, ldl, fused, idx, w, hdr, flagged, s);
+    if (vpl <= 2) return launch_topk<2>(part, bias, x, Wr, T, H, E, k, ldl, fused, idx, w, hdr, flagged, s);
+    if (vpl <= 4) return launch_topk<4>(part, bias, x, Wr, T, H, E, k, ldl, fused, idx, w, hdr, flagged, s);
+    if (vpl <= 8) return launch_topk<8>(part, bias, x, Wr, T, H, E, k, ldl, fused, idx, w, hdr, flagged, s);
+    return launch_topk<16>(part, bias, x, Wr, T, H, E, k, ldl, fused, idx, w, hdr, flagged, s);
 }
 
 }  // namespace mok

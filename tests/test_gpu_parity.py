@@ -71,6 +71,60 @@ def test_all_routes_to_one_expert():
     assert st["counts"].cpu().numpy()[3] == cfg.T
 
 
+ROUTER_SHAPES = [
+    # the one-kernel router pads the experts to 32, 64, 96, 128 and 160; ragged token tiles; k up to its limit of 28
+    MoEConfig("r_e6", T=333, H=200, E=6, k=2, I=64, I_s=0, seed=71),
+    MoEConfig("r_e40", T=129, H=264, E=40, k=28, I=64, I_s=0, bias="normal", seed=72),
+    MoEConfig("r_e64", T=700, H=256, E=64, k=4, I=64, I_s=0, bias="zipf", seed=73),
+    MoEConfig("r_e96", T=1000, H=512, E=96, k=6, I=64, I_s=0, seed=74),
+    MoEConfig("r_e128", T=2100, H=1024, E=128, k=8, I=64, I_s=0, bias="zipf", seed=75),
+    MoEConfig("r_e150", T=515, H=320, E=150, k=5, I=64, I_s=0, bias="normal", seed=76),
+    MoEConfig("r_e160", T=260, H=2048, E=160, k=8, I=64, I_s=0, seed=77),
+    MoEConfig("r_k_eq_e", T=70, H=64, E=4, k=4, I=64, I_s=0, seed=78),
+]
+
+
+@pytest.mark.parametrize("cfg", ROUTER_SHAPES, ids=[c.name for c in ROUTER_SHAPES])
+def test_one_kernel_router_against_oracle_and_three_kernel_router(cfg):
+    """Projection + top-k in one kernel (the default up to 160 experts): every token against the oracle, and the
+    same bits (indices, weights, output) as the three-kernel tensor-core router; grid-size independent."""
+    m = mok()
+    d = inputs.make_inputs(cfg)
+    g = pu.upload(d)
+    out, st, rep = pu.full_parity(cfg, d=d, g=g)
+    print(cfg.name, rep)
+    out3, st3 = pu.run_gpu(cfg, g, config=m._config(router_impl=2))
+    assert torch.equal(st["topk_idx"], st3["topk_idx"])
+    assert torch.equal(st["topk_w"].view(torch.int32), st3["topk_w"].view(torch.int32))
+    assert torch.equal(out.view(torch.int16), out3.view(torch.int16))
+    outg, stg = pu.run_gpu(cfg, g, config=m._config(grid=3))
+    assert torch.equal(st["topk_idx"], stg["topk_idx"])
+    assert torch.equal(st["topk_w"].view(torch.int32), stg["topk_w"].view(torch.int32))
+
+
+def test_one_kernel_router_lists_near_ties_for_the_exact_fix_up():
+    """Duplicate expert rows give exact ties and rows that differ in the last bit give logits closer than the tensor
+    cores' accumulation error: both must come out as the oracle decides them (lowest id first on exact ties)."""
+    m = mok()
+    cfg = MoEConfig("r_ties", T=300, H=512, E=32, k=4, I=64, I_s=0, seed=79)
+    d = inputs.make_inputs(cfg)
+    W = d["W_r"].copy()
+    W[5] = W[2]                                   # exact tie between experts 2 and 5 for every token
+    W[9] = W[7] * np.float32(1 + 2.0 ** -20)      # near-tie between 7 and 9
+    d["W_r"] = W
+    g = pu.upload(d)
+    out, st, rep = pu.full_parity(cfg, d=d, g=g)
+    print(rep)
+    idx = st["topk_idx"].cpu().numpy()
+    both = (idx == 2).any(axis=1) & (idx == 5).any(axis=1)
+    assert both.any()
+    for t in np.flatnonzero(both):
+        assert list(idx[t]).index(2) < list(idx[t]).index(5)
+    out3, st3 = pu.run_gpu(cfg, g, config=m._config(router_impl=2))
+    assert torch.equal(st["topk_idx"], st3["topk_idx"])
+    assert torch.equal(st["topk_w"].view(torch.int32), st3["topk_w"].view(torch.int32))
+
+
 def test_tiny_config_every_token_and_determinism():
     cfg = inputs.CONFIGS["tiny"]
     d = inputs.make_inputs(cfg)
