@@ -43,12 +43,12 @@ sched_scan_kernel(int32_t* __restrict__ blk_hist, int n_blk, int E, int max_mt, 
     const int e = threadIdx.x;
     int32_t total = 0;
     if (e < E) {
-        for (int b0 = 0; b0 < n_blk; b0 += 8) {          // 8 independent loads in flight, then the serial prefix
-            int32_t c[8];
+        for (int b0 = 0; b0 < n_blk; b0 += 16) {         // 16 independent loads in flight, then the serial prefix
+            int32_t c[16];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) c[i] = (b0 + i < n_blk) ? blk_hist[(size_t)(b0 + i) * E + e] : 0;
+            for (int i = 0; i < 16; ++i) c[i] = (b0 + i < n_blk) ? blk_hist[(size_t)(b0 + i) * E + e] : 0;
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
+            for (int i = 0; i < 16; ++i) {
                 if (b0 + i < n_blk) blk_hist[(size_t)(b0 + i) * E + e] = total;
                 total += c[i];
             }
