@@ -153,6 +153,25 @@ int mok_moe_forward_ex(const mok_args* args);
 int mok_moe_forward_host(const mok_args* args, const void* x_host, void* out_host);
 
 /*
+ * The host-buffer call without the wait at its end, for a stream of batches (this entry point and the wait below are
+ * this library's own; the paper measures device-side latency only, Section 4.1).  It enqueues: upload of x_host on the
+ * library's input copy stream, the layer on args->stream, download into out_host on the library's output copy stream,
+ * chained by events, and returns at once.  Two staging slots at the end of the workspace are used in turn, so
+ * consecutive submissions overlap: while batch i computes, batch i+1 uploads and batch i-1 downloads (PCIe is full
+ * duplex).  A slot's copy of x is reused once the layer that read it has run, its copy of out once that result has left
+ * the device (event waits on the device, not on the host).  The result bits equal those of mok_moe_forward_ex.
+ *   - x_host must stay unchanged, and out_host must not be read, until mok_host_wait() has returned; use a
+ *     different out_host for submissions that are in flight together.  Pinned buffers are needed for the overlap.
+ *   - The workspace must have mok_workspace_bytes(...) + 4 * T*H*2 bytes (each slot: x and out, 256-byte aligned)
+ *     and must serve these submissions only while any is in flight; all submissions in flight use the same T and H.
+ *   - Stage outputs are not supported here (MOK_ERR_UNSUPPORTED); the other errors are those of mok_moe_forward_ex,
+ *     reported before anything is enqueued.  Device-side failures show in mok_read_status after the wait.
+ * mok_host_wait blocks until every submission made so far on the current device has delivered its result.
+ */
+int mok_moe_forward_host_async(const mok_args* args, const void* x_host, void* out_host);
+int mok_host_wait(void);
+
+/*
  * Stage entry points (used by tests and profiling; each is the corresponding step of mok_moe_forward_ex).
  *   mok_route    : router projection + top-k + weights (Section 2.1)          -> topk_idx [T,k], topk_w [T,k]
  *   mok_schedule : Algorithm 1 for one rank from topk_idx [T*k]               -> counts, offsets, perm, inv_perm

@@ -421,6 +421,10 @@ int mok_moe_forward_ex(const mok_args* a) {
 struct HostPipe {
     cudaStream_t s_in = nullptr, s_out = nullptr;
     cudaEvent_t start = nullptr, out_done = nullptr, in_done[MOK_MAX_HOST_CHUNKS] = {}, fwd_done[MOK_MAX_HOST_CHUNKS] = {};
+    // asynchronous submissions: two staging slots used in turn; slot_free[i] fires when slot i's result has left the device
+    cudaEvent_t a_in[2] = {}, a_fwd[2] = {}, slot_free[2] = {};
+    bool slot_used[2] = {false, false};
+    unsigned long long n_async = 0;
     bool ready = false;
 };
 static HostPipe g_pipe[64];
@@ -439,6 +443,11 @@ static int host_pipe(HostPipe** out) {
         for (int c = 0; c < MOK_MAX_HOST_CHUNKS; ++c) {
             if ((e = cudaEventCreateWithFlags(&p.in_done[c], cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
             if ((e = cudaEventCreateWithFlags(&p.fwd_done[c], cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
+        }
+        for (int c = 0; c < 2; ++c) {
+            if ((e = cudaEventCreateWithFlags(&p.a_in[c], cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
+            if ((e = cudaEventCreateWithFlags(&p.a_fwd[c], cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
+            if ((e = cudaEventCreateWithFlags(&p.slot_free[c], cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
         }
         p.ready = true;
     }
@@ -515,6 +524,55 @@ int mok_moe_forward_host(const mok_args* a, const void* x_host, void* out_host) 
     if ((e = cudaEventRecord(p->out_done, p->s_out)) != cudaSuccess) return cuda_fail(e);
     if ((e = cudaStreamWaitEvent(s, p->out_done, 0)) != cudaSuccess) return cuda_fail(e);
     e = cudaStreamSynchronize(s);
+    return e == cudaSuccess ? MOK_OK : cuda_fail(e);
+}
+
+// Submission without waiting: upload on the input copy stream, layer on the caller's stream, download on the output copy
+// stream, chained by events; two staging slots at the end of the workspace alternate, so the upload of submission
+// i+1 and the download of submission i-1 overlap the layer of submission i.  Nothing here blocks the host.
+int mok_moe_forward_host_async(const mok_args* a, const void* x_host, void* out_host) {
+    WsLayout L;
+    if (!a) return MOK_ERR_NULL;
+    const size_t act = 2 * (size_t)(a->T > 0 ? a->T : 0) * (size_t)(a->H > 0 ? a->H : 0);
+    const size_t act_al = align_up(act, 256);
+    int rc = validate(a, &L, 4 * act_al);
+    if (rc || a->T == 0) return rc;
+    if (!x_host || !out_host) return MOK_ERR_NULL;
+    if (a->topk_idx || a->topk_w || a->counts || a->offsets || a->perm || a->inv_perm) return MOK_ERR_UNSUPPORTED;
+    HostPipe* p = nullptr;
+    if ((rc = host_pipe(&p))) return rc;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(a->stream);
+    char* ws = reinterpret_cast<char*>(a->workspace);
+    const int slot = (int)(p->n_async & 1ull);
+    __nv_bfloat16* xd = reinterpret_cast<__nv_bfloat16*>(ws + L.total + (size_t)slot * 2 * act_al);
+    __nv_bfloat16* od = reinterpret_cast<__nv_bfloat16*>(ws + L.total + (size_t)slot * 2 * act_al + act_al);
+    cudaError_t e;
+    // the slot's x copy is free once the layer that read it has run; its out copy once that result has been downloaded.
+    // Three stages of about equal length (upload, layer, download) thus stay busy with two slots.
+    if (p->slot_used[slot] && (e = cudaStreamWaitEvent(p->s_in, p->a_fwd[slot], 0)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaMemcpyAsync(xd, x_host, act, cudaMemcpyHostToDevice, p->s_in)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaEventRecord(p->a_in[slot], p->s_in)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaStreamWaitEvent(s, p->a_in[slot], 0)) != cudaSuccess) return cuda_fail(e);
+    if (p->slot_used[slot] && (e = cudaStreamWaitEvent(s, p->slot_free[slot], 0)) != cudaSuccess) return cuda_fail(e);
+    if ((rc = forward_device(a, L, xd, od))) return rc;
+    if ((e = cudaEventRecord(p->a_fwd[slot], s)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaStreamWaitEvent(p->s_out, p->a_fwd[slot], 0)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaMemcpyAsync(out_host, od, act, cudaMemcpyDeviceToHost, p->s_out)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaEventRecord(p->slot_free[slot], p->s_out)) != cudaSuccess) return cuda_fail(e);
+    p->slot_used[slot] = true;
+    ++p->n_async;
+    return MOK_OK;
+}
+
+int mok_host_wait(void) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (dev < 0 || dev >= 64) return MOK_ERR_UNSUPPORTED;
+    HostPipe& p = g_pipe[dev];
+    if (!p.ready) return MOK_OK;
+    // every download is ordered after its layer and its upload, and the output stream runs in order
+    e = cudaStreamSynchronize(p.s_out);
     return e == cudaSuccess ? MOK_OK : cuda_fail(e);
 }
 

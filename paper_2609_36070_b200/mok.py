@@ -19,7 +19,8 @@ MOK_ERR_NULL, MOK_ERR_SHAPE, MOK_ERR_ALIGN, MOK_ERR_WORKSPACE = -1, -2, -3, -4
 MOK_ERR_CUDA, MOK_ERR_TIMEOUT, MOK_ERR_SCHEDULE, MOK_ERR_UNSUPPORTED = -5, -6, -7, -8
 MOK_IMPL_TCGEN05, MOK_IMPL_SIMT, MOK_IMPL_TCGEN05_TN = 0, 1, 2
 
-EXPORTS = ["mok_moe_forward", "mok_workspace_bytes", "mok_moe_forward_ex", "mok_moe_forward_host", "mok_route",
+EXPORTS = ["mok_moe_forward", "mok_workspace_bytes", "mok_moe_forward_ex", "mok_moe_forward_host",
+           "mok_moe_forward_host_async", "mok_host_wait", "mok_route",
            "mok_schedule", "mok_read_status", "mok_launch_count", "mok_last_cuda_error", "mok_status_string",
            "mok_version", "mok_profile_begin", "mok_profile_end", "mok_schedule_noalloc", "mok_debug_counters",
            "mok_ep_workspace_bytes", "mok_ep_y_rows", "mok_ep_expert_ffn", "mok_ep_combine",
@@ -120,6 +121,10 @@ _lib.mok_moe_forward_ex.restype = ctypes.c_int
 _lib.mok_moe_forward_ex.argtypes = [ctypes.POINTER(mok_args)]
 _lib.mok_moe_forward_host.restype = ctypes.c_int
 _lib.mok_moe_forward_host.argtypes = [ctypes.POINTER(mok_args), ctypes.c_void_p, ctypes.c_void_p]
+_lib.mok_moe_forward_host_async.restype = ctypes.c_int
+_lib.mok_moe_forward_host_async.argtypes = [ctypes.POINTER(mok_args), ctypes.c_void_p, ctypes.c_void_p]
+_lib.mok_host_wait.restype = ctypes.c_int
+_lib.mok_host_wait.argtypes = []
 _lib.mok_route.restype = ctypes.c_int
 _lib.mok_route.argtypes = ([ctypes.c_void_p] * 3 + [ctypes.c_int] * 4 + [ctypes.c_void_p] * 3 +
                            [ctypes.c_size_t, ctypes.POINTER(mok_config), ctypes.c_void_p])
@@ -248,8 +253,8 @@ def alloc_workspace(T, H, I, I_shared, E, k, device="cuda", host_staging=False, 
     n = (mok_mx_workspace_bytes if mx else mok_workspace_bytes)(T, H, I, I_shared, E, k)
     if n == 0:
         raise MokError(MOK_ERR_SHAPE)
-    if host_staging:
-        n += 2 * ((2 * T * H + 255) // 256 * 256)
+    if host_staging:    # True / 1: the blocking host call; 2: the two slots of the asynchronous one
+        n += (4 if host_staging == 2 else 2) * ((2 * T * H + 255) // 256 * 256)
     return torch.empty(n + 256, dtype=torch.uint8, device=device)
 
 
@@ -334,6 +339,24 @@ def mok_moe_forward_host(x_host, out_host, W_router, router_bias, W_gate_up, W_d
     _check(_lib.mok_moe_forward_host(ctypes.byref(a), ctypes.c_void_p(x_host.data_ptr()),
                                      ctypes.c_void_p(out_host.data_ptr())))
     return out_host
+
+
+def mok_moe_forward_host_async(x_host, out_host, W_router, router_bias, W_gate_up, W_down, W_shared_gate_up,
+                               W_shared_down, k, workspace, config=None, stream=None, mx_weights=None):
+    """Submission without waiting (workspace from alloc_workspace(..., host_staging=2)); out_host is valid after
+    mok_host_wait()."""
+    assert not x_host.is_cuda and not out_host.is_cuda
+    a, _ = _fill_args(x_host.shape, W_router, router_bias, W_gate_up, W_down, W_shared_gate_up, W_shared_down, k,
+                      workspace, False, config, stream, W_router.device)
+    if mx_weights is not None:
+        a.W_gate_up_codes, a.W_gate_up_scales = mx_weights.gate_up_codes.data_ptr(), mx_weights.gate_up_scales.data_ptr()
+        a.W_down_codes, a.W_down_scales = mx_weights.down_codes.data_ptr(), mx_weights.down_scales.data_ptr()
+    _check(_lib.mok_moe_forward_host_async(ctypes.byref(a), ctypes.c_void_p(x_host.data_ptr()),
+                                           ctypes.c_void_p(out_host.data_ptr())))
+
+
+def mok_host_wait():
+    _check(_lib.mok_host_wait())
 
 
 def mok_route(x, W_router, router_bias, k, workspace, config=None, stream=None):

@@ -189,6 +189,42 @@ def test_host_buffer_entry_point_chunked_copies_give_the_same_bits():
         assert torch.equal(oh.view(torch.int16), ref.view(torch.int16)), chunks
 
 
+def test_asynchronous_host_submissions_overlap_and_match_the_device_call():
+    """A stream of batches through mok_moe_forward_host_async: different inputs in flight together (the two staging
+    slots alternate), results after mok_host_wait bitwise equal to mok_moe_forward_ex on the same inputs."""
+    m = mok()
+    cfg = SMALL[-1]
+    d = inputs.make_inputs(cfg)
+    g = pu.upload(d)
+    ws = m.alloc_workspace(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k, host_staging=2)
+    xs = [g["x"], (g["x"].float() * 0.5).to(torch.bfloat16), (g["x"].float() * -1.25).to(torch.bfloat16)]
+    want = []
+    for x in xs:
+        want.append(m.mok_moe_forward_ex(x, g["W_r"], g["bias"], g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"],
+                                         cfg.k, ws).clone())
+    torch.cuda.synchronize()
+    xh = [x.cpu().pin_memory() for x in xs]
+    n_sub = 7
+    oh = [torch.zeros_like(xh[0]).pin_memory() for _ in range(n_sub)]
+    for i in range(n_sub):
+        m.mok_moe_forward_host_async(xh[i % 3], oh[i], g["W_r"], g["bias"], g["W_gate_up"], g["W_down"], g["W_sgu"],
+                                     g["W_sd"], cfg.k, ws)
+    m.mok_host_wait()
+    assert m.mok_read_status(ws) == 0
+    for i in range(n_sub):
+        assert torch.equal(oh[i].view(torch.int16), want[i % 3].cpu().view(torch.int16)), i
+    # the blocking call still works on the same workspace afterwards, and a workspace without the second slot is refused
+    out1 = torch.zeros_like(xh[0]).pin_memory()
+    m.mok_moe_forward_host(xh[1], out1, g["W_r"], g["bias"], g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], cfg.k, ws)
+    assert torch.equal(out1.view(torch.int16), want[1].cpu().view(torch.int16))
+    small = m.alloc_workspace(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k, host_staging=True)
+    small = small[:small.numel() - 256]
+    with pytest.raises(m.MokError):
+        m.mok_moe_forward_host_async(xh[0], oh[0], g["W_r"], g["bias"], g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"],
+                                     cfg.k, small)
+    m.mok_host_wait()
+
+
 def test_stage_entry_points():
     m = mok()
     cfg = SMALL[-1]
