@@ -36,6 +36,7 @@
 #include "tc_ptx.cuh"
 #include "tile_order.cuh"
 #include "mx_ptx.cuh"
+#include "tensor_map.cuh"
 
 namespace mok {
 namespace mx {
@@ -443,46 +444,14 @@ gemm_mx_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
     }
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static EncodeTiledFn get_encode() {
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-            q == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(p);
-    }
-    return fn;
-}
-
 // 2D row-major byte tensor [rows, cols] -> tensor map with a [128 rows x 128 bytes] box and 128-byte swizzle.
 static bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols) {
-    EncodeTiledFn enc = get_encode();
-    if (!enc) return false;
-    cuuint64_t dims[2] = {cols, rows};
-    cuuint64_t strides[1] = {cols};
-    cuuint32_t box[2] = {(cuuint32_t)BKB, 128};
-    cuuint32_t estr[2] = {1, 1};
-    return enc(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(ptr), dims, strides, box, estr,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    return tmap::encode_2d(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, ptr, rows, cols, cols, (uint32_t)BKB, 128, CU_TENSOR_MAP_SWIZZLE_128B);
 }
 
 // Scale atoms as a 2D tensor [atoms, 128 words]: one box = one 512-byte atom, no swizzle.
 static bool make_sf_map(CUtensorMap* m, const void* ptr, uint64_t atoms) {
-    EncodeTiledFn enc = get_encode();
-    if (!enc) return false;
-    cuuint64_t dims[2] = {128, atoms};
-    cuuint64_t strides[1] = {512};
-    cuuint32_t box[2] = {128, 1};
-    cuuint32_t estr[2] = {1, 1};
-    return enc(m, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void*>(ptr), dims, strides, box, estr,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    return tmap::encode_2d(m, CU_TENSOR_MAP_DATA_TYPE_UINT32, ptr, atoms, 128, 512, 128, 1, CU_TENSOR_MAP_SWIZZLE_NONE);
 }
 
 }  // namespace mx
