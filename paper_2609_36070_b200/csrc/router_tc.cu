@@ -236,7 +236,8 @@ static cudaError_t launch_topk(const float* part, const float* bias, const __nv_
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }
-    router_fixup_kernel<VPL><<<296, 256, 0, s>>>(part, bias, x, Wr, H, E, k, ldl, fused, idx, w, hdr, flagged);
+    // one block per listed token; 8 blocks fit on an SM at once, and blocks beyond the list's length leave at once
+    router_fixup_kernel<VPL><<<148 * 8, 256, 0, s>>>(part, bias, x, Wr, H, E, k, ldl, fused, idx, w, hdr, flagged);
     return cudaGetLastError();
 }
 
