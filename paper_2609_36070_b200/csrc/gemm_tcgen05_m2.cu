@@ -354,6 +354,41 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&ctrl->tempty[acc]));
+            } else if (EPI == EPI_BF16 && !GATHER) {
+                // Plain bf16 output (this instantiation has registers to spare): the whole accumulator row is read and
+                // packed first, the accumulator goes back to the MMA issuer, and only then do the four 64-column passes
+                // through the slab start -- the hand-over no longer waits behind the first passes' stores.
+                const int c0 = t.n * BN;
+                uint32_t o[128];
+#pragma unroll
+                for (int c = 0; c < BN; c += 32) {
+                    uint32_t r[32];
+                    tc_ld32(taddr + c, r);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 16; ++i)
+                        o[(c >> 1) + i] = pack_bf16(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&ctrl->tempty[acc]));
+#pragma unroll
+                for (int pass = 0; pass < 4; ++pass) {
+                    if (lane == 0) tma_store_wait_read();     // the slab's previous store has been read out
+                    __syncwarp();
+                    const uint32_t line = slab + lane * 128;  // 64 columns = 8 chunks of 16 bytes
+#pragma unroll
+                    for (int v = 0; v < 8; ++v)
+                        st_shared_v4(line + ((v ^ (lane & 7)) << 4), o[pass * 32 + 4 * v], o[pass * 32 + 4 * v + 1],
+                                     o[pass * 32 + 4 * v + 2], o[pass * 32 + 4 * v + 3]);
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) {
+                        const int col = c0 + pass * 64;
+                        if (col < a.N && store_ok) tma_store_2d(&tmapC, slab, col, row);
+                        tma_store_commit();
+                    }
+                }
             } else {
                 // 64 output columns per pass.  The TMEM reads and the arithmetic of pass p+1 are done BEFORE waiting for
                 // the slab that pass p is about to overwrite, so the accumulator goes back to the MMA issuer as soon as
