@@ -26,7 +26,7 @@ UNIT = "tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # dram bytes (read + write) of one launch of the dominant kernel from the committed ncu capture, keyed by config
 # (None until a capture exists for that workload; see profiles/).
-NCU_TRAFFIC_BYTES = {"qwen3_30b_a3b": 1.413e9}   # profiles/gemm_kernels_qwen3_30b_a3b.md: 1.183 GB read + 0.230 GB written
+NCU_TRAFFIC_BYTES = {"qwen3_30b_a3b": 1.420e9}   # profiles/gemm_kernels_qwen3_30b_a3b.md: 1.189 GB read + 0.231 GB written
 
 
 def parse():
