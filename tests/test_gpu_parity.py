@@ -81,6 +81,7 @@ ROUTER_SHAPES = [
     MoEConfig("r_e150", T=515, H=320, E=150, k=5, I=64, I_s=0, bias="normal", seed=76),
     MoEConfig("r_e160", T=260, H=2048, E=160, k=8, I=64, I_s=0, seed=77),
     MoEConfig("r_k_eq_e", T=70, H=64, E=4, k=4, I=64, I_s=0, seed=78),
+    MoEConfig("r_e161", T=200, H=192, E=161, k=7, I=64, I_s=0, bias="normal", seed=80),   # first size of the three-kernel path
 ]
 
 

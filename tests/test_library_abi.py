@@ -78,6 +78,8 @@ def test_argument_validation_needs_no_device(lib):
     lib.mok_launch_count.argtypes = [ctypes.c_int] * 6 + [ctypes.c_void_p]
     assert lib.mok_launch_count(256, 256, 512, 512, 8, 2, None) == lib.mok_launch_count(256, 256, 512, 0, 8, 2, None) + 2
     assert lib.mok_launch_count(0, 256, 512, 0, 8, 2, None) == 0
+    # up to 160 experts the router is one kernel less (projection + top-k fused)
+    assert lib.mok_launch_count(256, 256, 512, 0, 160, 2, None) + 1 == lib.mok_launch_count(256, 256, 512, 0, 161, 2, None)
 
 
 def test_binding_fails_loudly_without_the_library(tmp_path, monkeypatch):
