@@ -5,7 +5,7 @@
 // that are nowhere near a tie.  Instead every fp32 weight is split exactly into three bf16 terms,
 //     W_r = hi + mid + lo,   hi = bf16(W_r), mid = bf16(W_r - hi), lo = bf16(W_r - hi - mid),
 // x is bf16 already, so all products are exact in fp32 and the tensor cores only add rounding in the fp32
-// accumulation.  Three kernels:
+// accumulation.  Four kernels (up to 160 experts kernels 2 and 3 are one: router_fused.cu):
 //   1. router_split_kernel  W_r [E,H] fp32 -> [ldl, H] bf16 rows: hi (0..E-1), mid (E..2E-1), lo (2E..3E-1), zero pad
 //   2. the tcgen05 GEMM     x [T,H] . split^T -> partial logits fp32 [T, ldl]
 //   3. router_topk_kernel   logit = (lo + mid) + hi + bias, warp-shuffle top-k and softmax weights; tokens with a
