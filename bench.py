@@ -42,6 +42,7 @@ def parse():
     p.add_argument("--gather-mode", type=int, default=0, help="0 auto, 1 fused into the GEMM, 2 separate kernel")
     p.add_argument("--cta-group", type=int, default=0, help="0 default, 1 single CTAs, 2 CTA pairs")
     p.add_argument("--gemm", type=int, default=0, help="0 tcgen05 (tokens on M), 2 tcgen05 (tokens on N), 1 SIMT")
+    p.add_argument("--tile-sched", type=int, default=0, help="routed GEMMs: 0 persistent grid, 1 tiles stolen through cluster launch control")
     p.add_argument("--host-chunks", type=int, default=0, help="token chunks of the host-buffer call (0 = auto)")
     p.add_argument("--precision", default="bf16", choices=["bf16", "mxfp8"],
                    help="routed experts in bf16 (the headline workload) or MXFP8 with pre-quantised weights")
@@ -259,7 +260,8 @@ def main():
     mxw = mok.MxWeights(g["W_gate_up"], g["W_down"]) if mx else None    # weights are quantised ahead of time
     ws = mok.alloc_workspace(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k, device=dev, host_staging=2, mx=mx)
     out = torch.empty_like(g["x"])
-    conf = mok._config(impl=args.gemm, profile=1, gather_mode=args.gather_mode, cta_group=args.cta_group, precision=prec)
+    conf = mok._config(impl=args.gemm, profile=1, gather_mode=args.gather_mode, cta_group=args.cta_group, precision=prec,
+                       tile_sched=args.tile_sched)
 
     def step():
         mok.mok_moe_forward_ex(g["x"], W_r, bias, g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], cfg.k, ws,

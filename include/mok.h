@@ -81,6 +81,13 @@ typedef struct mok_config {
     int32_t precision;    /* MOK_PRECISION_BF16 (0, default) or MOK_PRECISION_MXFP8: routed experts on MXFP8 operands
                              (Section 3.4 "MXFP8 Support"); needs the pre-quantised weights in mok_args and a workspace
                              of mok_mx_workspace_bytes(...) */
+    int32_t tile_sched;   /* routed expert GEMMs of the forward pass (256-row-tile kernel): 0 = persistent grid, tile L on
+                             CTA L mod grid; 1 = one CTA per tile, running CTAs steal the tiles of CTAs that have not
+                             started through cluster launch control (Section 3.4 "Cluster Launch Control": hardware
+                             work stealing).  The hardware refuses the request while work of a higher stream priority
+                             waits for an SM; the CTA then leaves and the tiles nobody stole start as CTAs of their own
+                             afterwards, so such work gets onto the SMs at the next tile boundary instead of at the end
+                             of the kernel.  Same bits either way. */
 } mok_config;
 
 /*

@@ -39,13 +39,18 @@ constexpr int THREADS = 64 + 32 * EPI_WARPS;   // producer + MMA + epilogue warp
 constexpr int GATHER_THREADS = 128;
 constexpr int GROUP_TILES = 8;                 // 2048 rows per rasterisation group
 constexpr int SLAB_BYTES = 4096;               // per epilogue warp: 32 rows x 64 bf16 columns (one swizzled box)
-constexpr int SMEM_CTRL = 256;
+constexpr int SMEM_CTRL = 512;
+constexpr int QSLOTS = 2;                      // tile ids the hardware scheduler hands out ahead (stolen mode)
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_WARPS * SLAB_BYTES + SMEM_CTRL + 1024;
 
 struct Ctrl {
     uint64_t full[STAGES], empty[STAGES];
     uint64_t tfull[2], tempty[2];              // per accumulator
     uint32_t tmem_base, abort;
+    // stolen mode (cluster launch control): the scheduler warp's queue of tile ids for the roles of this CTA
+    alignas(16) uint8_t clc_response[16];
+    uint64_t clc_done, q_full[QSLOTS], q_empty[QSLOTS];
+    int32_t q_tile[QSLOTS];
 };
 static_assert(sizeof(Ctrl) <= SMEM_CTRL, "control block too large");
 
@@ -117,12 +122,45 @@ __device__ __forceinline__ uint64_t make_smem_desc_mn(uint32_t addr, uint32_t gr
     return d;
 }
 
+// How a role walks over its tiles.  Static mode: tile L -> CTA L mod grid of a persistent grid.  Stolen mode (paper,
+// Section 3.4 "Cluster Launch Control"): the grid has one CTA per tile; a CTA that runs computes its own tile and
+// then cancels CTAs that have not started yet and computes theirs (clusterlaunchcontrol.try_cancel: hardware work
+// stealing) -- CTAs come and go at tile granularity, so other work can get onto the SMs between them.  The scheduler
+// warp steals; the other roles read the stolen ids from a two-entry queue in shared memory (bounded waits; an entry
+// is released once every role has read it).  Ids at or past `total` (the grid is a host-side upper bound) are skipped.
+template <bool CLC>
+struct TileSeq {
+    Ctrl* ctrl;
+    volatile uint32_t* abort_flag;
+    WsHeader* hdr;
+    int total, slot;
+    uint32_t ph;
+    bool warp_role;       // all 32 lanes call next() together (epilogue, gather) / one lane calls it (producer, issuer)
+    __device__ __forceinline__ TileSeq(Ctrl* c, volatile uint32_t* af, WsHeader* h, int tot, bool wr)
+        : ctrl(c), abort_flag(af), hdr(h), total(tot), slot(0), ph(0), warp_role(wr) {}
+    __device__ __forceinline__ int first() {
+        if (!CLC) return blockIdx.x;
+        return (int)blockIdx.x < total ? (int)blockIdx.x : next(0);
+    }
+    __device__ __forceinline__ int next(int L) {
+        if (!CLC) return L + gridDim.x;
+        bool ok = mbar_wait(smem_u32(&ctrl->q_full[slot]), ph, abort_flag, hdr, 30);
+        if (warp_role) ok = __all_sync(0xffffffffu, ok);
+        if (!ok) return total;
+        const int t = *reinterpret_cast<volatile int32_t*>(&ctrl->q_tile[slot]);
+        if (warp_role) __syncwarp();
+        if (!warp_role || (threadIdx.x & 31) == 0) mbar_arrive(smem_u32(&ctrl->q_empty[slot]));
+        if (++slot == QSLOTS) { slot = 0; ph ^= 1u; }
+        return t < 0 ? total : t;
+    }
+};
+
 // MODE 0: forward layout.  MODE 1 (KGROUP): the K-range mode (weight gradients).  MODE 2 (BMN): B is read MN-major,
 // i.e. W[e] is [K, N] with N contiguous -- the weights as they sit in memory serve the transposed products of the
 // backward pass (dL/dh = dy Wd, dXg = [dg|du] Wgu) without a transposed copy.  Compiled separately so that the
 // forward kernels carry none of it.
-template <int EPI, bool GATHER, int MODE>
-__global__ void __launch_bounds__(THREADS + (GATHER ? GATHER_THREADS : 0), 1)
+template <int EPI, bool GATHER, int MODE, bool CLC>
+__global__ void __launch_bounds__(THREADS + (GATHER ? GATHER_THREADS : 0) + (CLC ? 32 : 0), 1)
 gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
                const __grid_constant__ CUtensorMap tmapC, const __grid_constant__ GemmArgs a, const int n_nt, const int k_blocks) {
     constexpr bool SWIGLU = (EPI == EPI_SWIGLU);
@@ -150,6 +188,13 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
             mbar_init(smem_u32(&ctrl->tfull[s]), 1);
             mbar_init(smem_u32(&ctrl->tempty[s]), 4);           // one arrive per epilogue warp of that accumulator
         }
+        if (CLC) {
+            mbar_init(smem_u32(&ctrl->clc_done), 1);
+            for (int q = 0; q < QSLOTS; ++q) {
+                mbar_init(smem_u32(&ctrl->q_full[q]), 1);
+                mbar_init(smem_u32(&ctrl->q_empty[q]), 2 + EPI_WARPS + (GATHER ? GATHER_THREADS / 32 : 0));   // every role
+            }
+        }
         ctrl->abort = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -170,7 +215,8 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
             int s = 0;
             uint32_t ph = 0;
             const int b_rows_per_expert = (SWIGLU ? 2 : 1) * a.N;
-            for (int L = blockIdx.x; L < total; L += gridDim.x) {
+            TileSeq<CLC> seq(ctrl, abort_flag, a.header, total, false);
+            for (int L = seq.first(); L < total; L = seq.next(L)) {
                 const Tile t = decode_tile<KGROUP>(a, L, n_nt, n_mt_total, k_blocks);
                 const bool two = t.valid > BM;
                 // weight rows of this tile; in the K-range mode B is an activation matrix shared by all experts
@@ -218,7 +264,8 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
             const bool dbg = a.dbg_slot >= 0;
             long long d_full = 0, d_tempty = 0, d_kb = 0;
             const long long d_t0 = dbg ? clock64() : 0;
-            for (int L = blockIdx.x; L < total; L += gridDim.x) {
+            TileSeq<CLC> seq(ctrl, abort_flag, a.header, total, false);
+            for (int L = seq.first(); L < total; L = seq.next(L)) {
                 const Tile t = decode_tile<KGROUP>(a, L, n_nt, n_mt_total, k_blocks);
                 if (KGROUP && t.kblocks == 0) continue;       // K-range mode: an expert without rows (output pre-zeroed)
                 const bool two = t.valid > BM;
@@ -276,7 +323,45 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
             }
         }
         __syncwarp();
-    } else if (GATHER && warp >= 2 + EPI_WARPS) {
+    } else if (CLC && warp == (THREADS + (GATHER ? GATHER_THREADS : 0)) / 32) {
+        // ------------------------------------------------------------------ scheduler (stolen mode): steals tile ids
+        if (lane == 0) {
+            int slot = 0;
+            uint32_t qph = 0, cph = 0;
+            bool more = true;
+            while (more) {
+                int tile = -1;
+                bool ok = true;
+                while (ok) {
+                    mbar_expect_tx(smem_u32(&ctrl->clc_done), 16);
+                    asm volatile("clusterlaunchcontrol.try_cancel.async.shared::cta.mbarrier::complete_tx::bytes.b128 [%0], [%1];"
+                                 ::"r"(smem_u32(ctrl->clc_response)), "r"(smem_u32(&ctrl->clc_done)) : "memory");
+                    ok = mbar_wait(smem_u32(&ctrl->clc_done), cph, abort_flag, a.header, 31);
+                    cph ^= 1u;
+                    if (!ok) break;
+                    uint32_t canceled = 0, bx = 0;
+                    asm volatile("{\n\t.reg .b128 r;\n\t.reg .pred p;\n\t"
+                                 "ld.shared.b128 r, [%2];\n\t"
+                                 "clusterlaunchcontrol.query_cancel.is_canceled.pred.b128 p, r;\n\t"
+                                 "selp.u32 %0, 1, 0, p;\n\t"
+                                 "@p clusterlaunchcontrol.query_cancel.get_first_ctaid::x.b32.b128 %1, r;\n\t}"
+                                 : "=r"(canceled), "=r"(bx) : "r"(smem_u32(ctrl->clc_response)) : "memory");
+                    // refused: nothing is left to steal, or work of a higher stream priority is waiting for an SM -- then this
+                    // CTA leaves and the tiles nobody stole start as CTAs of their own afterwards.  (No request may follow a
+                    // refused one.)
+                    if (!canceled) break;
+                    if ((int)bx < total) { tile = (int)bx; break; }
+                }
+                if (!ok) break;
+                if (!mbar_wait(smem_u32(&ctrl->q_empty[slot]), qph ^ 1u, abort_flag, a.header, 32)) break;
+                *reinterpret_cast<volatile int32_t*>(&ctrl->q_tile[slot]) = tile;
+                mbar_arrive(smem_u32(&ctrl->q_full[slot]));   // release semantics order the id before the arrive
+                if (++slot == QSLOTS) { slot = 0; qph ^= 1u; }
+                more = tile >= 0;
+            }
+        }
+        __syncwarp();
+    } else if (GATHER && warp >= 2 + EPI_WARPS && warp < 2 + EPI_WARPS + GATHER_THREADS / 32) {
         // ------------------------------------------------------------------ gather warps (pull dispatch)
         // Warp gw owns rows 32 gw .. 32 gw + 31 of each half; lane = (sub-row 0..3, 16-byte chunk 0..7); pass i of half
         // h covers row 128 h + 32 gw + 4 i + sub-row.  Chunk c of row r lands at r*128 + ((c ^ (r & 7)) * 16) inside
@@ -284,7 +369,8 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
         const int gw = warp - (2 + EPI_WARPS), sub = lane >> 3, chunk = lane & 7;
         int s = 0;
         uint32_t ph = 0;
-        for (int L = blockIdx.x; L < total; L += gridDim.x) {
+        TileSeq<CLC> seq(ctrl, abort_flag, a.header, total, true);
+        for (int L = seq.first(); L < total; L = seq.next(L)) {
             const Tile t = decode_tile<KGROUP>(a, L, n_nt, n_mt_total, k_blocks);
             const bool two = t.valid > BM;
             const int tok0 = __ldg(a.row_token + t.row0);
@@ -324,7 +410,8 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
         const int quad = warp & 3;                            // TMEM lane quadrant this warp may access
         const uint32_t slab = base + STAGES * STAGE_BYTES + (warp - 2) * SLAB_BYTES;
         uint32_t aph = 0;
-        for (int L = blockIdx.x; L < total; L += gridDim.x) {
+        TileSeq<CLC> seq(ctrl, abort_flag, a.header, total, true);
+        for (int L = seq.first(); L < total; L = seq.next(L)) {
             const Tile t = decode_tile<KGROUP>(a, L, n_nt, n_mt_total, k_blocks);
             if ((KGROUP && t.kblocks == 0) || (acc == 1 && t.valid <= BM)) continue;   // no rows to contract / no second half
             bool ok = mbar_wait(smem_u32(&ctrl->tfull[acc]), aph, abort_flag, a.header, 4);
@@ -468,21 +555,29 @@ static bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t co
     return tmap::bf16_sw128(m, ptr, rows, cols, box_rows, stride);
 }
 
-template <int EPI, bool GATHER, int MODE = 0>
+template <int EPI, bool GATHER, int MODE = 0, bool CLC = false>
 static cudaError_t launch_one(const CUtensorMap& mA, const CUtensorMap& mB, const CUtensorMap& mC, const GemmArgs& a,
                               int n_nt, int k_blocks, int grid, cudaStream_t s) {
     static int sm_count = 0;
     if (!sm_count) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_m2_kernel<EPI, GATHER, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             SMEM_BYTES);
+        cudaError_t e = cudaFuncSetAttribute(gemm_m2_kernel<EPI, GATHER, MODE, CLC>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
         if (e != cudaSuccess) return e;
         int dev = 0;
         cudaGetDevice(&dev);
         cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
     }
-    if (grid <= 0 || grid > sm_count) grid = sm_count;
-    gemm_m2_kernel<EPI, GATHER, MODE><<<grid, THREADS + (GATHER ? GATHER_THREADS : 0), SMEM_BYTES, s>>>(mA, mB, mC, a, n_nt,
-                                                                                                 k_blocks);
+    if (CLC) {
+        // one CTA per tile: a host-side upper bound of the tile count (every expert with rows has at most one partial tile)
+        const long long rows = a.total_rows > 0 ? a.total_rows : 0;
+        const long long m_tiles = (rows + TM - 1) / TM + (rows < a.E ? rows : a.E);
+        grid = (int)(m_tiles * n_nt);
+        if (grid < 1) grid = 1;
+    } else if (grid <= 0 || grid > sm_count) {
+        grid = sm_count;
+    }
+    gemm_m2_kernel<EPI, GATHER, MODE, CLC><<<grid, THREADS + (GATHER ? GATHER_THREADS : 0) + (CLC ? 32 : 0), SMEM_BYTES, s>>>(
+        mA, mB, mC, a, n_nt, k_blocks);
     return cudaGetLastError();
 }
 
@@ -514,6 +609,9 @@ cudaError_t launch_gemm_m2(const GemmArgs& a, int epi, int grid, cudaStream_t s)
         return gather ? launch_one<EPI_BF16, true, 2>(mA, mB, mC, a, n_nt, k_blocks, grid, s)
                       : launch_one<EPI_BF16, false, 2>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
     }
+    const bool stolen = a.tile_sched == 1 && a.dense_rows == 0;   // hardware tile stealing: routed forward GEMMs only
+    if (stolen && epi == EPI_SWIGLU && gather) return launch_one<EPI_SWIGLU, true, 0, true>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
+    if (stolen && epi == EPI_BF16 && !gather) return launch_one<EPI_BF16, false, 0, true>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
     if (epi == EPI_SWIGLU && gather) return launch_one<EPI_SWIGLU, true>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
     if (epi == EPI_SWIGLU) return launch_one<EPI_SWIGLU, false>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
     if (epi == EPI_BF16 && !gather) return launch_one<EPI_BF16, false>(mA, mB, mC, a, n_nt, k_blocks, grid, s);

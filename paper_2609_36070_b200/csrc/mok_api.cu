@@ -95,6 +95,7 @@ static bool mx_pairs(const mok_config* cfg) { return cfg && cfg->cta_group == 2;
 static int validate(const mok_args* a, WsLayout* L, size_t extra_ws) {
     if (!a) return MOK_ERR_NULL;
     if (a->config && (a->config->precision < 0 || a->config->precision > 1)) return MOK_ERR_SHAPE;
+    if (a->config && (a->config->tile_sched < 0 || a->config->tile_sched > 1)) return MOK_ERR_SHAPE;
     const bool mx = use_mx(a->config);
     if (mx && a->config->impl != MOK_IMPL_TCGEN05) return MOK_ERR_SHAPE;
     if (!ws_layout(a->T, a->H, a->I, a->I_shared, a->E, a->k, L, mx)) return MOK_ERR_SHAPE;
@@ -324,6 +325,7 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
         g.C = ws + L.h;
         g.K = a->H; g.N = a->I; g.ldc = a->I; g.E = a->E; g.rows_pad = L.Rpad; g.dense_rows = 0;
         g.total_rows = L.R;
+        g.tile_sched = a->config ? a->config->tile_sched : 0;
         if ((rc = run_gemm(g, true, a->config, L, ws, s))) return rc;
         g.row_token = nullptr;
         g.starve = 0;
@@ -335,6 +337,7 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
         g.C = ws + L.y;
         g.K = a->I; g.N = a->H; g.ldc = a->H;
         if ((rc = run_gemm(g, false, a->config, L, ws, s))) return rc;
+        g.tile_sched = 0;
     }
     MOK_MARK(MOK_STAGE_GEMM2 + 1);
     g.dbg_slot = dbg ? 3 : -1;

@@ -139,6 +139,20 @@ def test_tiny_config_every_token_and_determinism():
         for cta_group in (1, 2, 3):                                                # nor on the tile / CTA arrangement
             o = pu.run_gpu(cfg, g, config=m._config(grid=grid, cta_group=cta_group), stages=False)
             assert torch.equal(out.view(torch.int16), o.view(torch.int16)), (grid, cta_group)
+    o = pu.run_gpu(cfg, g, config=m._config(tile_sched=1), stages=False)                # nor on who computes which tile
+    assert torch.equal(out.view(torch.int16), o.view(torch.int16))
+
+
+@pytest.mark.parametrize("cfg", [SMALL[0], SMALL[5], SMALL[6]], ids=lambda c: c.name)
+def test_tiles_stolen_through_cluster_launch_control_give_the_same_bits(cfg):
+    """config.tile_sched = 1: one CTA per tile, running CTAs cancel pending ones and compute their tiles.  Every token
+    against the oracle, and the same bits as the persistent grid."""
+    m = mok()
+    d = inputs.make_inputs(cfg)
+    g = pu.upload(d)
+    out, st, rep = pu.full_parity(cfg, d=d, g=g, config=m._config(tile_sched=1))
+    out0 = pu.run_gpu(cfg, g, stages=False)
+    assert torch.equal(out.view(torch.int16), out0.view(torch.int16))
 
 
 def test_fourteen_argument_entry_point_matches_ex():
