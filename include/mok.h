@@ -88,6 +88,12 @@ typedef struct mok_config {
                              waits for an SM; the CTA then leaves and the tiles nobody stole start as CTAs of their own
                              afterwards, so such work gets onto the SMs at the next tile boundary instead of at the end
                              of the kernel.  Same bits either way. */
+    int32_t macrobatch_tokens; /* mok_moe_forward_ex: > 0 and < T: the tokens pass through the workspace in macrobatches of
+                             this many tokens, one after the other (Section 3.3: a fixed-size buffer through which the
+                             tokens cycle, instead of buffers sized for the whole batch).  The workspace then only needs
+                             mok_workspace_bytes(macrobatch_tokens, ...); every macrobatch streams the expert weights
+                             again.  Same bits as the single pass; counts / offsets / perm / inv_perm (tables of ONE
+                             schedule) cannot be returned: MOK_ERR_UNSUPPORTED. */
 } mok_config;
 
 /*

@@ -216,11 +216,13 @@ static int route_stage(const mok_args* a, const WsLayout& L, char* ws, const __n
 }
 
 // The whole layer on device pointers.  x / out may differ from a->x / a->out (host-buffer variant).
-static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloat16* x, __nv_bfloat16* out) {
+static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloat16* x, __nv_bfloat16* out,
+                          bool reset_header = true) {
     cudaStream_t s = reinterpret_cast<cudaStream_t>(a->stream);
     char* ws = reinterpret_cast<char*>(a->workspace);
     WsHeader* hdr = reinterpret_cast<WsHeader*>(ws + L.header);
-    cudaError_t e = cudaMemsetAsync(hdr, 0, sizeof(WsHeader), s);
+    // (later macrobatches of one call keep the header: its status word is sticky, the tile counts are rewritten anyway)
+    cudaError_t e = reset_header ? cudaMemsetAsync(hdr, 0, sizeof(WsHeader), s) : cudaSuccess;
     if (e != cudaSuccess) return cuda_fail(e);
     cudaEvent_t* pev = profile_slot(a->config);
 #define MOK_MARK(i) do { if (pev) cudaEventRecord(pev[i], s); } while (0)
@@ -413,6 +415,33 @@ size_t mok_workspace_bytes(int T, int H, int I, int I_shared, int E, int k) {
 
 int mok_moe_forward_ex(const mok_args* a) {
     WsLayout L;
+    if (!a) return MOK_ERR_NULL;
+    const int mb = a->config ? a->config->macrobatch_tokens : 0;
+    if (mb < 0) return MOK_ERR_SHAPE;
+    if (mb > 0 && a->T > mb) {
+        // Fixed-size macrobatches (Section 3.3): the tokens pass through a workspace sized for `mb` tokens, one macrobatch
+        // after the other on the same stream.  A token's output depends only on its own row of x, so the bits equal
+        // those of the single pass.  The schedule tables describe one macrobatch each, so only the per-token stage
+        // outputs can be returned.
+        if (a->counts || a->offsets || a->perm || a->inv_perm) return MOK_ERR_UNSUPPORTED;
+        mok_args ac = *a;
+        ac.T = mb;
+        int rc = validate(&ac, &L, 0);
+        if (rc) return rc;
+        if (!a->x || !a->out) return MOK_ERR_NULL;
+        if (!aligned16(a->x) || !aligned16(a->out)) return MOK_ERR_ALIGN;
+        const __nv_bfloat16* x = reinterpret_cast<const __nv_bfloat16*>(a->x);
+        __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(a->out);
+        for (int t0 = 0; t0 < a->T; t0 += mb) {
+            ac.T = a->T - t0 < mb ? a->T - t0 : mb;
+            if (!ws_layout(ac.T, a->H, a->I, a->I_shared, a->E, a->k, &L, use_mx(a->config))) return MOK_ERR_SHAPE;
+            ac.topk_idx = a->topk_idx ? a->topk_idx + (size_t)t0 * a->k : nullptr;
+            ac.topk_w = a->topk_w ? a->topk_w + (size_t)t0 * a->k : nullptr;
+            rc = forward_device(&ac, L, x + (size_t)t0 * a->H, out + (size_t)t0 * a->H, t0 == 0);
+            if (rc) return rc;
+        }
+        return MOK_OK;
+    }
     int rc = validate(a, &L, 0);
     if (rc || a->T == 0) return rc;
     if (!a->x || !a->out) return MOK_ERR_NULL;

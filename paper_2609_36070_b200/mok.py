@@ -37,7 +37,7 @@ class mok_config(ctypes.Structure):
     _fields_ = [("impl", ctypes.c_int32), ("grid", ctypes.c_int32), ("router_impl", ctypes.c_int32),
                 ("profile", ctypes.c_int32), ("gather_mode", ctypes.c_int32), ("cta_group", ctypes.c_int32),
                 ("debug", ctypes.c_int32), ("host_chunks", ctypes.c_int32), ("precision", ctypes.c_int32),
-                ("tile_sched", ctypes.c_int32)]
+                ("tile_sched", ctypes.c_int32), ("macrobatch_tokens", ctypes.c_int32)]
 
 
 class mok_args(ctypes.Structure):
@@ -175,10 +175,11 @@ def _stream(stream):
 
 
 def _config(impl=0, grid=0, router_impl=0, profile=0, gather_mode=0, cta_group=0, debug=0, host_chunks=0,
-            precision=0, tile_sched=0):
+            precision=0, tile_sched=0, macrobatch_tokens=0):
     c = mok_config()
     c.precision = precision
     c.tile_sched = tile_sched
+    c.macrobatch_tokens = macrobatch_tokens
     c.impl, c.grid, c.router_impl, c.profile, c.gather_mode = impl, grid, router_impl, profile, gather_mode
     c.cta_group = cta_group
     c.debug = debug

@@ -155,6 +155,31 @@ def test_tiles_stolen_through_cluster_launch_control_give_the_same_bits(cfg):
     assert torch.equal(out.view(torch.int16), out0.view(torch.int16))
 
 
+def test_fixed_size_macrobatches_need_only_their_own_workspace_and_give_the_same_bits():
+    """config.macrobatch_tokens: the batch passes through a workspace sized for one macrobatch (ragged last one
+    included); bits equal the single pass; schedule tables cannot be returned."""
+    m = mok()
+    cfg = SMALL[6]                                                   # T = 700
+    d = inputs.make_inputs(cfg)
+    g = pu.upload(d)
+    out = pu.run_gpu(cfg, g, stages=False)
+    for mb in (256, 300, 699):
+        ws = m.alloc_workspace(mb, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k)           # NOT large enough for T tokens
+        full = m.alloc_workspace(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k).numel()
+        assert ws.numel() <= full and (mb > 300 or ws.numel() < full)
+        o = m.mok_moe_forward_ex(g["x"], g["W_r"], g["bias"], g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], cfg.k, ws,
+                                 config=m._config(macrobatch_tokens=mb))
+        torch.cuda.synchronize()
+        assert m.mok_read_status(ws) == 0
+        assert torch.equal(out.view(torch.int16), o.view(torch.int16)), mb
+    ws = m.alloc_workspace(256, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k)
+    with pytest.raises(m.MokError):                                   # without the knob the small workspace is refused
+        m.mok_moe_forward_ex(g["x"], g["W_r"], g["bias"], g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], cfg.k, ws)
+    with pytest.raises(m.MokError):                                   # the tables of one schedule do not exist here
+        m.mok_moe_forward_ex(g["x"], g["W_r"], g["bias"], g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], cfg.k, ws,
+                             stages=True, config=m._config(macrobatch_tokens=256))
+
+
 def test_fourteen_argument_entry_point_matches_ex():
     m = mok()
     cfg = inputs.CONFIGS["tiny"]
