@@ -269,6 +269,12 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
                 const Tile t = decode_tile<KGROUP>(a, L, n_nt, n_mt_total, k_blocks);
                 if (KGROUP && t.kblocks == 0) continue;       // K-range mode: an expert without rows (output pre-zeroed)
                 const bool two = t.valid > BM;
+                // the last N tile of a plain output may be narrower than 256 columns: the MMA is told so (its duration is
+                // proportional to N); the columns past it are never stored.  (A SwiGLU tile is [gate 128 | up 128].)
+                constexpr uint32_t IDESC_K = IDESC | (BMN ? (1u << 16) : 0u) | (AMN ? (1u << 15) : 0u);
+                uint32_t idesc = IDESC_K;
+                if (!SWIGLU && a.N - t.n * BN < BN)
+                    idesc = (IDESC_K & ~(0x3Fu << 17)) | ((uint32_t)(((a.N - t.n * BN + 15) & ~15) >> 3) << 17);
                 long long w0 = dbg ? clock64() : 0;
                 // Accumulator 0 is needed now, accumulator 1 only after the first k-block's MMAs into accumulator 0; and
                 // accumulator 0 is published before the last k-block's MMAs into accumulator 1 are issued.  Each
@@ -291,10 +297,9 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
                     // K-major B: +32 bytes per K = 16 step inside the swizzled row; MN-major B: +2 groups of 8 K-rows
                     const uint64_t bd = BMN ? make_smem_desc_mn(sa + 2 * A_BYTES, B_BYTES / 4) : make_smem_desc(sa + 2 * A_BYTES);
                     constexpr uint32_t BSTEP = BMN ? (2048 >> 4) : 2;
-                    constexpr uint32_t IDESC_K = IDESC | (BMN ? (1u << 16) : 0u) | (AMN ? (1u << 15) : 0u);
 #pragma unroll
                     for (int j = 0; j < BK / UMMA_K; ++j)
-                        tc_mma<1>(d0, a0 + (uint64_t)(j * ASTEP), bd + (uint64_t)(j * BSTEP), IDESC_K, (kb | j) ? 1u : 0u);
+                        tc_mma<1>(d0, a0 + (uint64_t)(j * ASTEP), bd + (uint64_t)(j * BSTEP), idesc, (kb | j) ? 1u : 0u);
                     if (kb == t.kblocks - 1) { tc_commit<1>(smem_u32(&ctrl->tfull[0])); ap0 ^= 1u; }
                     if (two) {
                         if (kb == 0) {
@@ -306,7 +311,7 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
                         }
 #pragma unroll
                         for (int j = 0; j < BK / UMMA_K; ++j)
-                            tc_mma<1>(d1, a1 + (uint64_t)(j * ASTEP), bd + (uint64_t)(j * BSTEP), IDESC_K, (kb | j) ? 1u : 0u);
+                            tc_mma<1>(d1, a1 + (uint64_t)(j * ASTEP), bd + (uint64_t)(j * BSTEP), idesc, (kb | j) ? 1u : 0u);
                     }
                     tc_commit<1>(smem_u32(&ctrl->empty[s]));
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
