@@ -303,22 +303,27 @@ int mok_moe_backward(const mok_bwd_args* a) {
     g.dbg_slot = -1;
     g.E = E; g.rows_pad = L.Rpad; g.dense_rows = 0; g.total_rows = L.R;
     int rc;
-    // The expert-sorted copies of x and dout (padding rows zero) serve four products each way: made once.  (Pulling the
-    // rows inside the GEMMs, as the forward pass does, would re-gather them once per N tile of 2I and I columns.)
+    // Four products need the rows of x or dout in dispatch order.  Up to I = 2048 each of them pulls the rows through the
+    // schedule's row_token table inside the GEMM, as the forward pass does (K-major for the recomputation and the dgrad
+    // product, MN-major for the weight gradients): no expert-sorted copies (bench workload 3.47 vs 3.73 ms).  A GEMM
+    // re-gathers its rows once per tile along the other output dimension (2I/256 or I/256 times), so for wide experts
+    // the copies are made once instead (I = 14336: 13.3 vs 13.9 ms, I = 2880: 10.9 vs 11.2 ms), padding rows zero.
+    const int32_t* row_token = reinterpret_cast<const int32_t*>(ws + L.row_token);
+    const bool pull = !wT && I <= 2048;
     __nv_bfloat16* XG = bf(L.xg);
     __nv_bfloat16* DG = bf(B.doutT);
-    if (!wT) {
+    if (!wT && !pull) {
         if ((e = launch_gather(x, H, k, TILE_M, L, ws, s, XG)) != cudaSuccess) return cuda_fail(e);
         if ((e = launch_gather(dout, H, k, TILE_M, L, ws, s, DG)) != cudaSuccess) return cuda_fail(e);
     }
     // gu = Xg Wgu^T  (activation recomputation)
-    if (wT) { g.A = x; g.a_rows = T; g.row_token = reinterpret_cast<const int32_t*>(ws + L.row_token); }
+    if (wT || pull) { g.A = x; g.a_rows = T; g.row_token = row_token; }
     else { g.A = XG; g.a_rows = L.Rpad; g.row_token = nullptr; }
     g.B = reinterpret_cast<const __nv_bfloat16*>(a->W_gate_up);
     g.C = ws + B.gu; g.K = H; g.N = 2 * I; g.ldc = 2 * I;
     if ((rc = run_gemm(g, false, &cfg, L, ws, s))) return rc;
     // dhu = gather(dout) Wd
-    g.A = wT ? dout : DG; g.C = ws + B.dhu; g.K = H; g.N = I; g.ldc = I;
+    g.A = (wT || pull) ? dout : DG; g.C = ws + B.dhu; g.K = H; g.N = I; g.ldc = I;
     if ((rc = dgrad_gemm(g, a->W_down, B.WdT))) return rc;
     // SwiGLU backward + router-weight gradient
     {
@@ -370,14 +375,17 @@ int mok_moe_backward(const mok_bwd_args* a) {
     const int Rp = L.Rpad, Tp = L.Tpad;
     if (!wT) {
         // Both operands of a weight-gradient product are read MN-major, exactly as the chain above left them:
-        // A = [rows, M] and B = [rows, N] with the row index as K (Xg and gather(dout) were made at the start).
+        // A = [rows, M] and B = [rows, N] with the row index as K; the operand that is a gathered x or dout is pulled
+        // through row_token by the kernel's gather warps (rows past an expert's count read as zero).
         q.b_mn = 1; q.E = E; q.dense_rows = 0; q.K = Rp;
-        q.kgroup_rows = H; q.A = DG; q.lda = H; q.B = bf(L.h); q.N = I; q.ldb = I;
+        if (pull) { q.row_token = row_token; q.a_rows = T; }   // dout / x stay in token order: their rows are pulled by the GEMM
+        q.kgroup_rows = H; q.A = pull ? dout : DG; q.lda = H; q.gather_mn = pull ? 1 : 0; q.B = bf(L.h); q.N = I; q.ldb = I;
         q.C = a->dW_down; q.rows_pad = E * H; q.ldc = I;
         if ((e = launch_gemm_m2(q, EPI_BF16, cfg.grid, s)) != cudaSuccess) return cuda_fail(e);
-        q.kgroup_rows = 2 * I; q.A = bf(B.dgu); q.lda = 2 * I; q.B = XG; q.N = H; q.ldb = H;
+        q.kgroup_rows = 2 * I; q.A = bf(B.dgu); q.lda = 2 * I; q.B = pull ? x : XG; q.N = H; q.ldb = H; q.gather_mn = pull ? 2 : 0;
         q.C = a->dW_gate_up; q.rows_pad = E * 2 * I; q.ldc = H;
         if ((e = launch_gemm_m2(q, EPI_BF16, cfg.grid, s)) != cudaSuccess) return cuda_fail(e);
+        q.row_token = nullptr; q.gather_mn = 0;
         if (Is > 0) {   // shared expert: one K range over the T tokens (rows past T are zero-filled by the tensor maps)
             q.E = 1; q.dense_rows = T; q.K = T;
             q.kgroup_rows = H; q.A = dout; q.lda = H; q.B = bf(L.hs); q.N = Is; q.ldb = Is;

@@ -229,19 +229,22 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
                     if (!ok) break;
                     const uint32_t full = smem_u32(&ctrl->full[s]);
                     const uint32_t sa = base + s * STAGE_BYTES, sb = sa + 2 * A_BYTES;
-                    mbar_expect_tx(full, B_BYTES + (GATHER ? 0 : (two ? 2 : 1) * A_BYTES));
-                    if (AMN) {   // per half two boxes of 64 M-columns x 64 K-rows (K = rows of the dispatch space)
+                    // GATHER: the gather warps bring A (forward layout), or in MODE 3 the operand a.gather_mn names
+                    const bool gA = GATHER && (!AMN || a.gather_mn == 1), gB = GATHER && AMN && a.gather_mn == 2;
+                    mbar_expect_tx(full, (gB ? 0 : B_BYTES) + (gA ? 0 : (two ? 2 : 1) * A_BYTES));
+                    if (AMN && !gA) {   // per half two boxes of 64 M-columns x 64 K-rows (K = rows of the dispatch space)
                         tma_load_2d(sa, &tmapA, full, t.row0, t.kcol0 + kb * BK);
                         tma_load_2d(sa + A_BYTES / 2, &tmapA, full, t.row0 + 64, t.kcol0 + kb * BK);
                         if (two) {
                             tma_load_2d(sa + A_BYTES, &tmapA, full, t.row0 + BM, t.kcol0 + kb * BK);
                             tma_load_2d(sa + A_BYTES + A_BYTES / 2, &tmapA, full, t.row0 + BM + 64, t.kcol0 + kb * BK);
                         }
-                    } else if (!GATHER) {
+                    } else if (!AMN && !GATHER) {
                         tma_load_2d(sa, &tmapA, full, t.kcol0 + kb * BK, t.row0);
                         if (two) tma_load_2d(sa + A_BYTES, &tmapA, full, t.kcol0 + kb * BK, t.row0 + BM);
                     }
-                    if (BMN) {   // four boxes of 64 N-columns x 64 K-rows: W[e] viewed as [E * K, N], or the shared B rows
+                    if (gB) {
+                    } else if (BMN) {   // four boxes of 64 N-columns x 64 K-rows: W[e] viewed as [E * K, N], or the shared B rows
                         const int krow = AMN ? t.kcol0 + kb * BK : t.e * a.K + kb * BK;
 #pragma unroll
                         for (int q = 0; q < 4; ++q)
@@ -375,6 +378,67 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
         int s = 0;
         uint32_t ph = 0;
         TileSeq<CLC> seq(ctrl, abort_flag, a.header, total, true);
+        if (AMN) {
+            // MODE 3 (weight gradients): the gathered operand is read MN-major, K = rows of the dispatch space.  One
+            // k-block = 64 dispatch rows x 256 columns of x or dout, laid out as four 64-column groups of [K row][128
+            // bytes] (chunk c of row kr at kr*128 + ((c ^ (kr & 7)) * 16) of its group), as the MMA descriptors expect.
+            // Warp gw owns rows 16 gw .. 16 gw + 15; lane = (sub-row 0..3, 16-byte chunk 0..7), so eight lanes read 128
+            // contiguous bytes of one row; a thread copies 4 rows x 4 column groups per k-block.  Rows past the expert's
+            // count are written as zeros: they must not contribute to the sums over rows.  The row ids of the next two
+            // k-blocks are loaded ahead.
+            const bool gB = a.gather_mn == 2;
+            const __nv_bfloat16* mat = gB ? a.B : a.A;
+            const int ld = gB ? (a.ldb ? a.ldb : a.K) : (a.lda ? a.lda : a.K);
+            const int col_lim = gB ? a.N : a.kgroup_rows;
+            const uint32_t obase = gB ? 2u * A_BYTES : 0u;
+            for (int L = seq.first(); L < total; L = seq.next(L)) {
+                const Tile t = decode_tile<KGROUP>(a, L, n_nt, n_mt_total, k_blocks);
+                if (t.kblocks == 0) continue;
+                const bool second = gB || t.valid > BM;      // column groups 2, 3 are in use
+                const int cnt = __ldg(a.counts + t.e);
+                const int colbase = (gB ? t.n * BN : t.row0) + chunk * 8;
+                const int32_t* rt = a.row_token + t.kcol0 + gw * 16 + sub;
+                int tok_cur[4], tok_nxt[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const int r = gw * 16 + q * 4 + sub;
+                    tok_cur[q] = (r < cnt) ? __ldg(rt + q * 4) : -1;
+                    tok_nxt[q] = (t.kblocks > 1 && 64 + r < cnt) ? __ldg(rt + 64 + q * 4) : -1;
+                }
+                bool ok = true;
+                for (int kb = 0; kb < t.kblocks; ++kb) {
+                    int tok_n2[4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const int r = (kb + 2) * 64 + gw * 16 + q * 4 + sub;
+                        tok_n2[q] = (kb + 2 < t.kblocks && r < cnt) ? __ldg(rt + (kb + 2) * 64 + q * 4) : -1;
+                    }
+                    ok = mbar_wait(smem_u32(&ctrl->empty[s]), ph ^ 1u, abort_flag, a.header, 5);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    const uint32_t stage = base + s * STAGE_BYTES + obase;
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const int kr = gw * 16 + q * 4 + sub;
+                        const __nv_bfloat16* srow = mat + (size_t)(tok_cur[q] >= 0 ? tok_cur[q] : 0) * ld + colbase;
+                        const uint32_t drow = stage + (uint32_t)kr * 128u + (uint32_t)((chunk ^ (kr & 7)) << 4);
+#pragma unroll
+                        for (int g4 = 0; g4 < 4; ++g4) {
+                            if (g4 < 2 || second) {
+                                const bool live = tok_cur[q] >= 0 && colbase + g4 * 64 < col_lim;
+                                cp_async_16(drow + (uint32_t)g4 * 8192u, live ? (const void*)(srow + g4 * 64) : (const void*)a.A,
+                                            live ? 16u : 0u);
+                            }
+                        }
+                    }
+                    cp_async_mbar_arrive(smem_u32(&ctrl->full[s]));
+                    if (++s == STAGES) { s = 0; ph ^= 1u; }
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) { tok_cur[q] = tok_nxt[q]; tok_nxt[q] = tok_n2[q]; }
+                }
+                if (!ok) break;
+            }
+        } else
         for (int L = seq.first(); L < total; L = seq.next(L)) {
             const Tile t = decode_tile<KGROUP>(a, L, n_nt, n_mt_total, k_blocks);
             const bool two = t.valid > BM;
@@ -593,12 +657,16 @@ cudaError_t launch_gemm_m2(const GemmArgs& a, int epi, int grid, cudaStream_t s)
     const bool swiglu = (epi == EPI_SWIGLU), gather = (a.row_token != nullptr);
     CUtensorMap mA, mB, mC;
     const uint64_t b_rows = (uint64_t)a.E * (swiglu ? 2 : 1) * a.N;
-    if (a.kgroup_rows > 0 && (epi != EPI_BF16 || gather || (a.kgroup_rows % 32))) return cudaErrorInvalidValue;
+    if (a.kgroup_rows > 0 && (epi != EPI_BF16 || (gather && !a.b_mn) || (a.kgroup_rows % 32))) return cudaErrorInvalidValue;
+    if (gather && a.kgroup_rows > 0 && (a.gather_mn < 1 || a.gather_mn > 2 || a.dense_rows > 0)) return cudaErrorInvalidValue;
     const uint64_t lda = a.lda ? (uint64_t)a.lda : (uint64_t)a.K, ldb = a.ldb ? (uint64_t)a.ldb : (uint64_t)a.K;
     if (a.kgroup_rows > 0 && a.b_mn) {
         // both operands as produced: A = [K rows, kgroup_rows columns], B = [K rows, N columns]; a.K = rows that exist
-        if (!make_map(&mA, a.A, (uint64_t)a.K, (uint64_t)a.kgroup_rows, 64, lda)) return cudaErrorInvalidValue;
-        if (!make_map(&mB, a.B, (uint64_t)a.K, (uint64_t)a.N, 64, ldb)) return cudaErrorInvalidValue;
+        // (a gathered operand is not read through its map: the map then only has to be a valid one over its a_rows rows)
+        const uint64_t ra = (gather && a.gather_mn == 1) ? (uint64_t)a.a_rows : (uint64_t)a.K;
+        const uint64_t rb = (gather && a.gather_mn == 2) ? (uint64_t)a.a_rows : (uint64_t)a.K;
+        if (!make_map(&mA, a.A, ra, (uint64_t)a.kgroup_rows, 64, lda)) return cudaErrorInvalidValue;
+        if (!make_map(&mB, a.B, rb, (uint64_t)a.N, 64, ldb)) return cudaErrorInvalidValue;
     } else if (!make_map(&mA, a.A, (uint64_t)a.a_rows, (uint64_t)a.K, BM, lda)) return cudaErrorInvalidValue;
     else if (a.b_mn) {   // W viewed as [E * K, N], N contiguous: boxes of 64 columns x 64 rows
         if (!make_map(&mB, a.B, (uint64_t)a.E * a.K, (uint64_t)a.N, 64, (uint64_t)a.N)) return cudaErrorInvalidValue;
@@ -607,6 +675,7 @@ cudaError_t launch_gemm_m2(const GemmArgs& a, int epi, int grid, cudaStream_t s)
     else if (!make_map(&mC, a.C, (uint64_t)a.rows_pad, (uint64_t)a.N, 32, (uint64_t)a.ldc)) return cudaErrorInvalidValue;
     const int n_nt = swiglu ? (a.N + BN / 2 - 1) / (BN / 2) : (a.N + BN - 1) / BN;
     const int k_blocks = (a.K + BK - 1) / BK;
+    if (a.kgroup_rows > 0 && a.b_mn && gather) return launch_one<EPI_BF16, true, 3>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
     if (a.kgroup_rows > 0 && a.b_mn) return launch_one<EPI_BF16, false, 3>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
     if (a.kgroup_rows > 0) return launch_one<EPI_BF16, false, 1>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
     if (a.b_mn) {

@@ -81,6 +81,9 @@ struct GemmArgs {
     int32_t kgroup_rows;
     int32_t lda, ldb;
     int32_t b_mn;                // 256-row kernel: B is W[e] = [K, N] with N contiguous (read MN-major), EPI_BF16 only
+    int32_t gather_mn;           // K-range mode with both operands MN-major and row_token set: 1 = A, 2 = B is x or dout in
+                                 // TOKEN order ([a_rows tokens, columns]) and its rows are pulled through row_token by the
+                                 // gather warps (rows past an expert's count read as zero)
     WsHeader* header;
     // Expert-parallel pull dispatch (Section 3.1): with peer_tokens > 0 the ids in row_token are global,
     // id = source_rank * peer_tokens + token, and row `id` is read from peer_x[source_rank] (this GPU's own tokens

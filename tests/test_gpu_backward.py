@@ -66,6 +66,7 @@ SHAPES = [
     ("skewed_empty_experts", 1024, 512, 32, 4, 384, 0, "zipf"),
     ("shared_wider_than_routed", 200, 128, 4, 2, 64, 256, "none"),
     ("one_route", 130, 64, 2, 1, 32, 0, "none"),
+    ("wide_experts_expert_sorted_copies", 200, 64, 3, 2, 2080, 0, "none"),   # I > 2048: rows of x / dout copied once, not pulled
 ]
 
 
