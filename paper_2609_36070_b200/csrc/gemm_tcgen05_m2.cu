@@ -552,6 +552,11 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
                 constexpr int PASSES = SWIGLU ? 2 : 4;
                 const int c0 = SWIGLU ? t.n * (BN / 2) : t.n * BN;
                 uint32_t cur[32], nxt[32];                    // one pass = 64 columns = 32 packed bf16 pairs per row
+                auto hand_back = [&]() {                       // the accumulator goes back to the MMA issuer
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&ctrl->tempty[acc]));
+                };
                 auto load_pass = [&](int pass, uint32_t (&o)[32]) {
 #pragma unroll
                     for (int c = 0; c < 64; c += 32) {
@@ -560,6 +565,7 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
                             tc_ld32(taddr + pass * 64 + c, g);
                             tc_ld32(taddr + BN / 2 + pass * 64 + c, u);
                             tc_wait_ld();
+                            if (pass == PASSES - 1 && c == 32) hand_back();   // the tile's last TMEM read: arithmetic comes after
 #pragma unroll
                             for (int i = 0; i < 16; ++i)
                                 o[(c >> 1) + i] = pack_bf16(swiglu(__uint_as_float(g[2 * i]), __uint_as_float(u[2 * i])),
@@ -568,6 +574,7 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
                             uint32_t r[32];
                             tc_ld32(taddr + pass * 64 + c, r);
                             tc_wait_ld();
+                            if (pass == PASSES - 1 && c == 32) hand_back();
 #pragma unroll
                             for (int i = 0; i < 16; ++i)
                                 o[(c >> 1) + i] = pack_bf16(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
@@ -581,11 +588,6 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
                     for (int i = 0; i < 32; ++i) cur[i] = nxt[i];
                     if (pass + 1 < PASSES) {
                         load_pass(pass + 1, nxt);
-                    }
-                    if (pass + 1 == PASSES - 1) {                 // the last TMEM read of this tile just happened
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(smem_u32(&ctrl->tempty[acc]));
                     }
                     if (lane == 0) tma_store_wait_read();     // the slab's previous store has been read out
                     __syncwarp();
