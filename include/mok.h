@@ -178,7 +178,8 @@ int mok_moe_forward_host(const mok_args* args, const void* x_host, void* out_hos
  *   - The workspace must have mok_workspace_bytes(...) + 4 * T*H*2 bytes (each slot: x and out, 256-byte aligned)
  *     and must serve these submissions only while any is in flight; all submissions in flight use the same T and H.
  *   - Stage outputs are not supported here (MOK_ERR_UNSUPPORTED); the other errors are those of mok_moe_forward_ex,
- *     reported before anything is enqueued.  Device-side failures show in mok_read_status after the wait.
+ *     reported before anything is enqueued.  Device-side failures show in mok_read_status after the wait: the status
+ *     word is cleared by the first submission after a mok_host_wait only, so it covers every submission since then.
  * mok_host_wait blocks until every submission made so far on the current device has delivered its result.
  */
 int mok_moe_forward_host_async(const mok_args* args, const void* x_host, void* out_host);
@@ -384,6 +385,11 @@ int mok_debug_counters(const void* workspace, void* stream, unsigned long long* 
 /* Number of kernels one mok_moe_forward_ex call enqueues for these arguments (the memset of the workspace header
    is not counted); 0 on bad sizes. */
 int mok_launch_count(int T, int H, int I, int I_shared, int E, int k, const mok_config* config);
+
+/* Host-only self-test of the per-device launch-state cache (the shared-memory opt-in of every kernel and the SM
+   count are remembered per device, not per process, so that one process can drive several GPUs).  Makes no CUDA
+   call; returns MOK_OK or the number of the failed check. */
+int mok_selftest_per_device(void);
 
 int mok_last_cuda_error(void);          /* cudaError_t of the most recent failed CUDA call on this thread */
 const char* mok_status_string(int status);

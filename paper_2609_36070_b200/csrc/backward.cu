@@ -96,13 +96,16 @@ static cudaError_t launch_transpose(const __nv_bfloat16* in, __nv_bfloat16* out,
                                     const int32_t* tile_expert = nullptr, const int32_t* pad_offsets = nullptr,
                                     const int32_t* counts = nullptr, const WsHeader* hdr = nullptr) {
     if (batch <= 0 || R <= 0 || C <= 0) return cudaSuccess;
-    static bool attr_set = false;
+    static PerDevice configured;      // per device: 1 once the kernel has its shared-memory opt-in there
     constexpr int smem = (TT * (TT / 2 + 4) + TT / 8) * 4;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(transpose_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        if (e != cudaSuccess) return e;
-        attr_set = true;
-    }
+    int dev = 0, done = 0;
+    cudaError_t e = current_device(&dev);
+    if (e != cudaSuccess) return e;
+    e = configured.get(dev, &done, [&](int, int* flag) {
+        *flag = 1;
+        return cudaFuncSetAttribute(transpose_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    });
+    if (e != cudaSuccess) return e;
     dim3 grid((C + TT - 1) / TT, (R + TT - 1) / TT, batch);
     transpose_kernel<<<grid, 256, smem, s>>>(in, out, R, C, (long long)R * C, (long long)C * out_ld, out_ld, route_of_row, k,
                                           tile_expert, pad_offsets, counts, hdr);

@@ -401,7 +401,8 @@ template <int EPI, bool GATHER, int CTAS>
 static cudaError_t launch_one(const CUtensorMap& mA, const CUtensorMap& mB, const CUtensorMap& mC, const GemmArgs& a,
                               int n_nt, int k_blocks, int grid, cudaStream_t s) {
     using namespace tc;
-    static int max_units = 0;
+    static PerDevice configured;      // per device: CTAs (or CTA pairs) of the persistent grid, once configured there
+    int max_units = 0;
     const int threads = THREADS + (GATHER ? GATHER_THREADS : 0);
     auto kernel = gemm_tc_kernel<EPI, GATHER, CTAS>;
     cudaLaunchConfig_t cfg = {};
@@ -418,22 +419,28 @@ static cudaError_t launch_one(const CUtensorMap& mA, const CUtensorMap& mB, cons
         cfg.attrs = attr;
         cfg.numAttrs = 1;
     }
-    if (!max_units) {
-        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    {
+        int dev = 0;
+        cudaError_t e = current_device(&dev);
         if (e != cudaSuccess) return e;
-        int dev = 0, sms = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        if (CTAS == 2) {
-            int clusters = 0;
-            cfg.gridDim = dim3(sms / 2 * 2);
-            e = cudaOccupancyMaxActiveClusters(&clusters, kernel, &cfg);
-            if (e != cudaSuccess) return e;
-            if (clusters < 1) return cudaErrorInvalidConfiguration;
-            max_units = clusters < sms / 2 ? clusters : sms / 2;
-        } else {
-            max_units = sms;
-        }
+        e = configured.get(dev, &max_units, [&](int d, int* units) {
+            cudaError_t e2 = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+            if (e2 != cudaSuccess) return e2;
+            int sms = 0;
+            if ((e2 = device_sm_count(d, &sms)) != cudaSuccess) return e2;
+            if (CTAS == 2) {
+                int clusters = 0;
+                cfg.gridDim = dim3(sms / 2 * 2);
+                e2 = cudaOccupancyMaxActiveClusters(&clusters, kernel, &cfg);
+                if (e2 != cudaSuccess) return e2;
+                if (clusters < 1) return cudaErrorInvalidConfiguration;
+                *units = clusters < sms / 2 ? clusters : sms / 2;
+            } else {
+                *units = sms;
+            }
+            return cudaSuccess;
+        });
+        if (e != cudaSuccess) return e;
     }
     int units = (grid <= 0) ? max_units : (grid + CTAS - 1) / CTAS;
     if (units > max_units) units = max_units;

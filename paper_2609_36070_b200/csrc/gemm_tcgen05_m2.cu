@@ -629,15 +629,16 @@ static bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t co
 template <int EPI, bool GATHER, int MODE = 0, bool CLC = false>
 static cudaError_t launch_one(const CUtensorMap& mA, const CUtensorMap& mB, const CUtensorMap& mC, const GemmArgs& a,
                               int n_nt, int k_blocks, int grid, cudaStream_t s) {
-    static int sm_count = 0;
-    if (!sm_count) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_m2_kernel<EPI, GATHER, MODE, CLC>,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
-        if (e != cudaSuccess) return e;
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
-    }
+    static PerDevice configured;      // per device: SM count once this instantiation has its shared-memory opt-in there
+    int dev = 0, sm_count = 0;
+    cudaError_t e = current_device(&dev);
+    if (e != cudaSuccess) return e;
+    e = configured.get(dev, &sm_count, [](int d, int* sms) {
+        cudaError_t e2 = cudaFuncSetAttribute(gemm_m2_kernel<EPI, GATHER, MODE, CLC>,
+                                              cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+        return e2 != cudaSuccess ? e2 : device_sm_count(d, sms);
+    });
+    if (e != cudaSuccess) return e;
     if (CLC) {
         // one CTA per tile: a host-side upper bound of the tile count (every expert with rows has at most one partial tile)
         const long long rows = a.total_rows > 0 ? a.total_rows : 0;

@@ -222,7 +222,8 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
     char* ws = reinterpret_cast<char*>(a->workspace);
     WsHeader* hdr = reinterpret_cast<WsHeader*>(ws + L.header);
     // (later macrobatches of one call keep the header: its status word is sticky, the tile counts are rewritten anyway)
-    cudaError_t e = reset_header ? cudaMemsetAsync(hdr, 0, sizeof(WsHeader), s) : cudaSuccess;
+    cudaError_t e = reset_header ? cudaMemsetAsync(hdr, 0, sizeof(WsHeader), s)
+                                 : cudaMemsetAsync(&hdr->n_flag, 0, sizeof(hdr->n_flag), s);
     if (e != cudaSuccess) return cuda_fail(e);
     cudaEvent_t* pev = profile_slot(a->config);
 #define MOK_MARK(i) do { if (pev) cudaEventRecord(pev[i], s); } while (0)
@@ -457,6 +458,7 @@ struct HostPipe {
     cudaEvent_t a_in[2] = {}, a_fwd[2] = {}, slot_free[2] = {};
     bool slot_used[2] = {false, false};
     unsigned long long n_async = 0;
+    unsigned long long n_since_wait = 0;     // submissions since the last mok_host_wait
     bool ready = false;
 };
 static HostPipe g_pipe[64];
@@ -546,7 +548,8 @@ int mok_moe_forward_host(const mok_args* a, const void* x_host, void* out_host) 
         WsLayout Lc;
         if (!ws_layout(tc, a->H, a->I, a->I_shared, a->E, a->k, &Lc, use_mx(a->config))) return MOK_ERR_SHAPE;
         if ((e = cudaStreamWaitEvent(s, p->in_done[c], 0)) != cudaSuccess) return cuda_fail(e);
-        rc = forward_device(&ac, Lc, xd + (size_t)t0 * a->H, od + (size_t)t0 * a->H);
+        // only the first chunk clears the header: a device-side failure of any chunk stays in the status word
+        rc = forward_device(&ac, Lc, xd + (size_t)t0 * a->H, od + (size_t)t0 * a->H, c == 0);
         if (rc) return rc;
         if ((e = cudaEventRecord(p->fwd_done[c], s)) != cudaSuccess) return cuda_fail(e);
         if ((e = cudaStreamWaitEvent(p->s_out, p->fwd_done[c], 0)) != cudaSuccess) return cuda_fail(e);
@@ -586,7 +589,10 @@ int mok_moe_forward_host_async(const mok_args* a, const void* x_host, void* out_
     if ((e = cudaEventRecord(p->a_in[slot], p->s_in)) != cudaSuccess) return cuda_fail(e);
     if ((e = cudaStreamWaitEvent(s, p->a_in[slot], 0)) != cudaSuccess) return cuda_fail(e);
     if (p->slot_used[slot] && (e = cudaStreamWaitEvent(s, p->slot_free[slot], 0)) != cudaSuccess) return cuda_fail(e);
-    if ((rc = forward_device(a, L, xd, od))) return rc;
+    // The status word is shared by every submission on this workspace: only the first submission after a
+    // mok_host_wait clears it, so a device-side failure of ANY submission is still there when the caller reads it.
+    if ((rc = forward_device(a, L, xd, od, p->n_since_wait == 0))) return rc;
+    ++p->n_since_wait;
     if ((e = cudaEventRecord(p->a_fwd[slot], s)) != cudaSuccess) return cuda_fail(e);
     if ((e = cudaStreamWaitEvent(p->s_out, p->a_fwd[slot], 0)) != cudaSuccess) return cuda_fail(e);
     if ((e = cudaMemcpyAsync(out_host, od, act, cudaMemcpyDeviceToHost, p->s_out)) != cudaSuccess) return cuda_fail(e);
@@ -605,6 +611,7 @@ int mok_host_wait(void) {
     if (!p.ready) return MOK_OK;
     // every download is ordered after its layer and its upload, and the output stream runs in order
     e = cudaStreamSynchronize(p.s_out);
+    p.n_since_wait = 0;
     return e == cudaSuccess ? MOK_OK : cuda_fail(e);
 }
 
@@ -748,6 +755,30 @@ int mok_profile_end(float* ms, int max_calls_out, int* n_calls) {
 }
 
 int mok_last_cuda_error(void) { return g_last_cuda_error; }
+
+int mok_selftest_per_device(void) {
+    // walks the per-device launch-state cache with a stand-in for the configuration step; no CUDA call is made
+    static PerDevice cache;
+    int calls = 0, fail_next = 0, out = 0;
+    auto configure = [&](int dev, int* value) {
+        ++calls;
+        if (fail_next) { fail_next = 0; return cudaErrorInvalidValue; }
+        *value = 100 + dev;
+        return cudaSuccess;
+    };
+    for (int d = 0; d < MAX_DEVICES; ++d) cache.v[d].store(0);
+    if (cache.get(3, &out, configure) != cudaSuccess || out != 103 || calls != 1) return 1;
+    if (cache.get(3, &out, configure) != cudaSuccess || out != 103 || calls != 1) return 2;   // cached
+    if (cache.get(5, &out, configure) != cudaSuccess || out != 105 || calls != 2) return 3;   // a second device configures again
+    if (cache.get(3, &out, configure) != cudaSuccess || out != 103 || calls != 2) return 4;
+    fail_next = 1;                                                                           // a failure is not remembered
+    if (cache.get(7, &out, configure) != cudaErrorInvalidValue || calls != 3) return 5;
+    if (cache.get(7, &out, configure) != cudaSuccess || out != 107 || calls != 4) return 6;
+    if (cache.get(-1, &out, configure) != cudaErrorInvalidDevice || cache.get(MAX_DEVICES, &out, configure) != cudaErrorInvalidDevice)
+        return 7;
+    if (calls != 4) return 8;
+    return MOK_OK;
+}
 
 const char* mok_status_string(int status) {
     switch (status) {

@@ -5,6 +5,7 @@
 #include <cuda.h>
 #include <stdint.h>
 #include <stddef.h>
+#include <atomic>
 #include "mok.h"
 
 namespace mok {
@@ -144,5 +145,34 @@ cudaError_t launch_router_fused(const __nv_bfloat16* x, const __nv_bfloat16* spl
                                 cudaStream_t s);
 
 inline __host__ __device__ size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Launch state that belongs to ONE device.  cudaFuncSetAttribute (the opt-in to more than 48 KB of dynamic shared
+// memory) applies to the device that is current when it is called, and the SM count is a property of that device, so
+// a launcher that remembers "configured" per process would launch unconfigured kernels on a second GPU of the same
+// process.  Each launcher keeps one PerDevice per kernel instantiation: value(dev) is 0 until `configure` has
+// succeeded on that device and then holds what it returned (the SM count, or the number of co-resident CTA pairs).
+// Concurrent first calls may both configure (the calls are idempotent) and store the same value.
+constexpr int MAX_DEVICES = 64;
+struct PerDevice {
+    std::atomic<int> v[MAX_DEVICES];
+    // configure(dev, &value) -> cudaError_t; value must come back > 0
+    template <class F>
+    cudaError_t get(int dev, int* out, F configure) {
+        if (dev < 0 || dev >= MAX_DEVICES) return cudaErrorInvalidDevice;
+        int cur = v[dev].load(std::memory_order_acquire);
+        if (cur == 0) {
+            cudaError_t e = configure(dev, &cur);
+            if (e != cudaSuccess) return e;
+            if (cur <= 0) return cudaErrorInvalidConfiguration;
+            v[dev].store(cur, std::memory_order_release);
+        }
+        *out = cur;
+        return cudaSuccess;
+    }
+};
+inline cudaError_t current_device(int* dev) { return cudaGetDevice(dev); }
+inline cudaError_t device_sm_count(int dev, int* sms) {
+    return cudaDeviceGetAttribute(sms, cudaDevAttrMultiProcessorCount, dev);
+}
 
 }  // namespace mok

@@ -283,16 +283,15 @@ static cudaError_t launch_one(const CUtensorMap& mA, const CUtensorMap& mB, Args
     if (stages > MAX_STAGES) stages = MAX_STAGES;
     if (stages < 2) return cudaErrorInvalidConfiguration;
     const int smem_bytes = stages * STAGE_BYTES + SMEM_CTRL + 1024;
-    static bool configured = false;
-    static int sms = 0;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(router_fused_kernel<NJ>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
-        if (e != cudaSuccess) return e;
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        configured = true;
-    }
+    static PerDevice configured;      // per device: SM count once this instantiation has its shared-memory opt-in there
+    int dev = 0, sms = 0;
+    cudaError_t e = current_device(&dev);
+    if (e != cudaSuccess) return e;
+    e = configured.get(dev, &sms, [&](int d, int* n) {
+        cudaError_t e2 = cudaFuncSetAttribute(router_fused_kernel<NJ>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+        return e2 != cudaSuccess ? e2 : device_sm_count(d, n);
+    });
+    if (e != cudaSuccess) return e;
     a.stages = stages;
     a.tmem_cols = 3 * EP <= 128 ? 128u : 3 * EP <= 256 ? 256u : 512u;
     int blocks = a.n_tiles < sms ? a.n_tiles : sms;

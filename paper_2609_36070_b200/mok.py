@@ -25,7 +25,7 @@ EXPORTS = ["mok_moe_forward", "mok_workspace_bytes", "mok_moe_forward_ex", "mok_
            "mok_version", "mok_profile_begin", "mok_profile_end", "mok_schedule_noalloc", "mok_debug_counters",
            "mok_ep_workspace_bytes", "mok_ep_y_rows", "mok_ep_expert_ffn", "mok_ep_combine",
            "mok_mx_scale_bytes", "mok_mx_quantize_weights", "mok_mx_quantize_rows", "mok_mx_workspace_bytes",
-           "mok_ep_mx_workspace_bytes", "mok_bwd_workspace_bytes", "mok_moe_backward"]
+           "mok_ep_mx_workspace_bytes", "mok_bwd_workspace_bytes", "mok_moe_backward", "mok_selftest_per_device"]
 MOK_PRECISION_BF16, MOK_PRECISION_MXFP8 = 0, 1
 MOK_MAX_RANKS = 16
 MOK_NOALLOC_MAX_ROUTES = 32768
@@ -144,6 +144,8 @@ _lib.mok_last_cuda_error.restype = ctypes.c_int
 _lib.mok_status_string.restype = ctypes.c_char_p
 _lib.mok_status_string.argtypes = [ctypes.c_int]
 _lib.mok_version.restype = ctypes.c_int
+_lib.mok_selftest_per_device.restype = ctypes.c_int
+_lib.mok_selftest_per_device.argtypes = []
 _lib.mok_profile_begin.restype = ctypes.c_int
 _lib.mok_profile_begin.argtypes = [ctypes.c_int]
 _lib.mok_profile_end.restype = ctypes.c_int
@@ -201,6 +203,11 @@ def mok_profile_end(max_calls):
 
 def mok_version():
     return int(_lib.mok_version())
+
+
+def mok_selftest_per_device():
+    """0 if the library's per-device launch-state cache behaves (host-only check, no CUDA call)."""
+    return int(_lib.mok_selftest_per_device())
 
 
 def mok_status_string(status):

@@ -82,6 +82,12 @@ def test_argument_validation_needs_no_device(lib):
     assert lib.mok_launch_count(256, 256, 512, 0, 160, 2, None) + 1 == lib.mok_launch_count(256, 256, 512, 0, 161, 2, None)
 
 
+def test_launch_state_is_kept_per_device(lib):
+    """The shared-memory opt-in and the SM count are cached per device, not per process: a second device configures
+    its kernels again, a failed configuration is retried, device ids out of range are refused."""
+    assert lib.mok_selftest_per_device() == 0
+
+
 def test_binding_fails_loudly_without_the_library(tmp_path, monkeypatch):
     """The product path has no fallback: importing the binding without libmok.so raises."""
     import importlib.util
