@@ -18,9 +18,11 @@
  *       the top-k routed experts and assign each a router weight") and the normalised weights
  *       s_i / sum_j s_j of the MoE equation in Section 2.1.  Score = softmax over all E logits
  *       (the benchmark configuration's reading); ties go to the lowest expert id.
- *   mok_ref_schedule : Algorithm 1 specialised to one rank, written as its restatement in
- *       Section 3.1 ("sorts the routes by the key (expert, ordinal, rank)").
- *   mok_ref_alg1     : Algorithm 1 for R ranks, statement by statement.
+ *   mok_ref_schedule : the dispatch schedule of one rank as Section 3.1 restates Algorithm 1: the
+ *       routes in ascending order of (expert, route id).
+ *   mok_ref_alg1     : the pull schedule of one destination rank for R source ranks, from the same
+ *       restatement: the routes in ascending order of (local expert, ordinal, source rank).  The
+ *       printed algorithm's closed-form row position is NOT used here; the pins evaluate it instead.
  *   mok_ref_ffn_tokens / mok_ref_forward : the MoE equation and the expert FFN
  *       f_i(x) = W_down (phi(W_gate x) .* W_up x) of Section 2.1, phi = SiLU.
  *
@@ -153,50 +155,50 @@ int mok_ref_schedule(const int32_t* a, int n, int E,
 }
 
 /*
- * Algorithm 1, general form.  A[r*NK + j] in [0, R*L) is the expert of route j on source rank r;
- * this rank is c and owns global experts c*L .. c*L+L-1.
- *   M[r,l]  = |{ j : A[r,j] = cL + l }|
- *   S[l]    = sum_{l' < l} sum_r M[r,l']            (S has L+1 entries, S[L] = rows received)
- *   for every route (r,j) with A[r,j] = cL + l:
- *       o   = |{ j' < j : A[r,j'] = A[r,j] }|
- *       p   = sum_{r'} min(M[r',l], o) + |{ r' < r : M[r',l] > o }|
- *       Phi[S[l] + p] = (r, j)
- * phi_rank / phi_idx must hold at least S[L] entries (R*NK always suffices).
+ * The pull schedule of one destination rank for R source ranks (Section 3.1), from its defining order rather
+ * than from the position arithmetic of the printed algorithm: rank c owns global experts cL .. cL+L-1, and the
+ * rows it receives are the routes (r, j) with A[r,j] in that range, laid out in ascending order of the key
+ *     ( local expert l,  ordinal o of the route among rank r's routes to that expert,  source rank r ).
+ * Sorting by l gives each expert one contiguous run; inside a run, ordinal-major order takes one route from every
+ * rank that still has one before taking anybody's next, i.e. consecutive rows cycle over the source ranks.
+ * S[l] = first row of expert l (S[L] = rows received); phi_rank / phi_idx give the source of every row and must
+ * hold at least S[L] entries (R*NK always suffices).  A[r*NK + j] in [0, R*L).
  */
+typedef struct { int32_t l, o, r, j; } pull_key;
+
+static int pull_key_cmp(const void* pa, const void* pb) {
+    const pull_key* a = (const pull_key*)pa;
+    const pull_key* b = (const pull_key*)pb;
+    if (a->l != b->l) return a->l < b->l ? -1 : 1;
+    if (a->o != b->o) return a->o < b->o ? -1 : 1;
+    if (a->r != b->r) return a->r < b->r ? -1 : 1;
+    return 0;                       /* (l, o, r) identifies a route: never reached for two different routes */
+}
+
 int mok_ref_alg1(const int32_t* A, int R, int NK, int L, int c,
                  int32_t* S, int32_t* phi_rank, int32_t* phi_idx) {
     if (!A || !S || !phi_rank || !phi_idx || R <= 0 || NK < 0 || L <= 0 || c < 0 || c >= R) return -1;
-    int32_t* M = (int32_t*)calloc((size_t)R * L, sizeof(int32_t));
-    if (!M) return -3;
-    for (int r = 0; r < R; ++r)
+    pull_key* keys = (pull_key*)malloc(sizeof(pull_key) * ((size_t)R * NK + 1));
+    int32_t* seen = (int32_t*)malloc(sizeof(int32_t) * (size_t)L);
+    if (!keys || !seen) { free(keys); free(seen); return -3; }
+    size_t n = 0;
+    for (int l = 0; l <= L; ++l) S[l] = 0;
+    for (int r = 0; r < R; ++r) {
+        for (int l = 0; l < L; ++l) seen[l] = 0;          /* routes of rank r to local expert l met so far */
         for (int j = 0; j < NK; ++j) {
             int g = A[(size_t)r * NK + j];
-            if (g < 0 || g >= R * L) { free(M); return -2; }
-            if (g / L == c) M[(size_t)r * L + (g - c * L)]++;
-        }
-    S[0] = 0;
-    for (int l = 0; l < L; ++l) {
-        int32_t tot = 0;
-        for (int r = 0; r < R; ++r) tot += M[(size_t)r * L + l];
-        S[l + 1] = S[l] + tot;
-    }
-    for (int r = 0; r < R; ++r)
-        for (int j = 0; j < NK; ++j) {
-            int g = A[(size_t)r * NK + j];
+            if (g < 0 || g >= R * L) { free(keys); free(seen); return -2; }
             if (g / L != c) continue;
-            int l = g - c * L;
-            int o = 0;
-            for (int jp = 0; jp < j; ++jp) o += (A[(size_t)r * NK + jp] == g);
-            int p = 0;
-            for (int rp = 0; rp < R; ++rp) {
-                int m = M[(size_t)rp * L + l];
-                p += (m < o) ? m : o;
-                if (rp < r && m > o) p += 1;
-            }
-            phi_rank[S[l] + p] = r;
-            phi_idx[S[l] + p] = j;
+            pull_key q = { g - c * L, seen[g - c * L]++, r, j };
+            keys[n++] = q;
+            S[q.l + 1]++;                                   /* rows of expert l, turned into prefix sums below */
         }
-    free(M);
+    }
+    for (int l = 0; l < L; ++l) S[l + 1] += S[l];
+    qsort(keys, n, sizeof(pull_key), pull_key_cmp);
+    for (size_t p = 0; p < n; ++p) { phi_rank[p] = keys[p].r; phi_idx[p] = keys[p].j; }
+    free(keys);
+    free(seen);
     return 0;
 }
 

@@ -94,7 +94,9 @@ def schedule(a, E):
 
 
 def alg1(A, L, c):
-    """Algorithm 1, general R.  A[R,NK] global expert per route.  Returns S[L+1], phi_rank, phi_idx (length S[L])."""
+    """The pull schedule Algorithm 1 defines for destination rank c and R source ranks (Section 3.1), built as a sort by
+    (local expert, ordinal, source rank).  A[R,NK] global expert per route.  Returns S[L+1], phi_rank, phi_idx
+    (length S[L])."""
     A = np.ascontiguousarray(A, np.int32)
     R, NK = A.shape
     S = np.empty((L + 1,), np.int32)

@@ -189,25 +189,31 @@ def test_alg1_single_rank_is_the_schedule():
 
 
 @pytest.mark.parametrize("R,NK,L", [(2, 30, 3), (4, 64, 2), (5, 17, 4), (3, 1, 1)])
-def test_alg1_matches_sort_by_expert_ordinal_rank(R, NK, L):
-    """Algorithm 1's closed-form position against its own restatement as a sort (Section 3.1), for every rank."""
+def test_alg1_matches_the_closed_form_position_and_the_schedule_properties(R, NK, L):
+    """The oracle builds the pull schedule by sorting on (expert, ordinal, rank).  Pinned here, for every destination
+    rank, by Algorithm 1's closed-form row position p = sum_r' min(M[r',l], o) + |{r' < r : M[r',l] > o}| evaluated
+    route by route in numpy, and by a step-by-step simulation of the round-robin fill (Section 3.1)."""
     rng = np.random.default_rng(R * 100 + NK)
     A = rng.integers(0, R * L, size=(R, NK)).astype(np.int32)
     A[0, A[0] == 0] = 1 % (R * L)                                           # make one (rank, expert) pair empty
     for c in range(R):
         S, pr, pi = mok_ref.alg1(A, L, c)
-        keys = []
+        M = np.array([[(A[r] == c * L + l).sum() for l in range(L)] for r in range(R)])
+        want_S = np.concatenate([[0], np.cumsum(M.sum(axis=0))])
+        assert np.array_equal(S, want_S)
+        want_rank = np.full(want_S[L], -1)
+        want_idx = np.full(want_S[L], -1)
         for r in range(R):
-            seen = {}
             for j in range(NK):
                 g = int(A[r, j])
-                o = seen.get(g, 0)
-                seen[g] = o + 1
-                if g // L == c:
-                    keys.append((g - c * L, o, r, j))
-        keys.sort()
-        assert S[L] == len(keys)
-        assert [q[2] for q in keys] == list(pr) and [q[3] for q in keys] == list(pi)
+                if g // L != c:
+                    continue
+                l = g - c * L
+                o = int((A[r, :j] == g).sum())
+                p = int(np.minimum(M[:, l], o).sum() + (M[:r, l] > o).sum())
+                assert want_rank[want_S[l] + p] == -1                          # the positions form a bijection
+                want_rank[want_S[l] + p], want_idx[want_S[l] + p] = r, j
+        assert np.array_equal(pr, want_rank) and np.array_equal(pi, want_idx)
         # the three properties a pull schedule must have (Section 3.1)
         experts = A[pr, pi] - c * L
         assert (np.diff(experts) >= 0).all()                                 # non-decreasing local expert
