@@ -2,16 +2,22 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl mok|reference]
 
-Prints ONE JSON line.  Default workload: the Qwen3-30B-A3B-like layer (T=16384, H=2048, E=128, k=8, I=768,
-Zipf-skewed routing), synthetic seeded inputs.  With N > 1 (launched by torch.distributed.run) every rank holds a
-full copy of the weights and its own batch of T tokens (token-sharded replicas: no data-path collective), the step
-time is the max over ranks and `value` is the aggregate tokens/s ("weak" scaling).
+Prints ONE JSON line.  Default workload: the DeepSeek-V3-like layer (T=32768, H=7168, E=256, k=8, I=2048, one shared
+expert of I=2048; about 23 GB of expert weights resident in HBM), synthetic seeded inputs.  The same line carries
+`per_config` (the four smaller workloads, each timed the same way) and `sweep` (the default workload at T = 64, 512,
+4096 against the HBM weight-read roofline); `--per-config none` / `--no-sweep` leave them out.
+
+With N > 1 (launched by torch.distributed.run) every rank holds a full copy of the weights and its own batch of T
+tokens (token-sharded replicas: no data-path collective), the step time is the max over ranks and `value` is the
+aggregate tokens/s ("weak" scaling); the sub-records are only produced at N = 1.
 
 `--impl reference` times the CPU oracle (the fp64 definition of the layer) on the host cores on a bounded token
 sample of the same workload; it is a deliberately slow baseline, not a target.
 """
 import argparse
+import datetime
 import json
+import math
 import os
 import subprocess
 import sys
@@ -23,22 +29,34 @@ if ROOT not in sys.path:
 
 METRIC = "moe_layer_fwd_tokens_per_s"
 UNIT = "tokens/s"
+DEFAULT_WORKLOAD = "deepseek_v3"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# dram bytes (read + write) of one launch of the dominant kernel from the committed ncu capture, keyed by config
-# (None until a capture exists for that workload; see profiles/).
-NCU_TRAFFIC_BYTES = {"qwen3_30b_a3b": 1.420e9}   # profiles/gemm_kernels_qwen3_30b_a3b.md: 1.189 GB read + 0.231 GB written
+# DRAM bytes (read + write) of ONE launch of the dominant kernel (routed gate/up grouped GEMM), from the ncu captures
+# summarised under profiles/.  A workload whose device footprint is too large to capture under the profiler is
+# captured on a scaled case with the same H, I, k and rows per expert and a fraction of the experts and tokens; DRAM
+# traffic of this kernel grows in proportion to both (weights read once per expert, rows gathered and written once
+# per route), so the capture is multiplied by `scale`.
+NCU_TRAFFIC = {
+    "qwen3_30b_a3b": {"bytes": 1.420e9, "scale": 1, "source": "profiles/gemm_kernels_qwen3_30b_a3b.md"},
+}
 
 
 def parse():
     p = argparse.ArgumentParser()
     p.add_argument("--gpus", type=int, default=1)
-    p.add_argument("--steps", type=int, default=300)
-    p.add_argument("--warmup", type=int, default=20)
-    p.add_argument("--config", default="qwen3_30b_a3b")
+    p.add_argument("--steps", type=int, default=20)
+    p.add_argument("--warmup", type=int, default=5)
+    p.add_argument("--config", default=DEFAULT_WORKLOAD)
     p.add_argument("--impl", default="mok", choices=["mok", "reference"])
     p.add_argument("--tokens", type=int, default=0, help="override T (small-T sweeps)")
     p.add_argument("--cpu-sample", type=int, default=0, help="tokens of the CPU-oracle sample (0 = auto)")
     p.add_argument("--no-cpu-baseline", action="store_true")
+    p.add_argument("--per-config", default="auto",
+                   help="'auto' (the other workloads when the default one is benchmarked on one GPU), 'none', or a "
+                        "comma-separated list of workload names")
+    p.add_argument("--no-sweep", action="store_true", help="skip the small-T sweep of the default workload")
+    p.add_argument("--no-e2e", action="store_true", help="skip the host-buffer (end-to-end) legs")
+    p.add_argument("--no-counters", action="store_true", help="skip the device-side counter pass")
     p.add_argument("--gather-mode", type=int, default=0, help="0 auto, 1 fused into the GEMM, 2 separate kernel")
     p.add_argument("--cta-group", type=int, default=0, help="0 default, 1 single CTAs, 2 CTA pairs")
     p.add_argument("--gemm", type=int, default=0, help="0 tcgen05 (tokens on M), 2 tcgen05 (tokens on N), 1 SIMT")
@@ -60,51 +78,77 @@ def peaks():
 
 
 class ClockSampler:
-    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
-    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+    """nvidia-smi clock / throttle-reason samples with timestamps, taken in the background for the whole run;
+    window(t0, t1) summarises the samples that fall into one timed region (host wall-clock seconds)."""
+    Q = ("timestamp,index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
+    NAMES = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
 
     def __init__(self, gpu_index):
         self.gpu = gpu_index
         self.proc = None
+        self.samples = None
 
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "50"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
 
     def stop(self):
+        self.samples = []
         if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.06)
+            return
+        time.sleep(0.05)
         self.proc.terminate()
-        out, _ = self.proc.communicate(timeout=10)
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            out, _ = self.proc.communicate(timeout=10)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
         for line in out.strip().splitlines():
             f = [v.strip() for v in line.split(",")]
-            if len(f) < 9:
+            if len(f) < 10:
                 continue
             try:
-                sm.append(float(f[1]))
-                mx.append(float(f[2]))
+                ts = datetime.datetime.strptime(f[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                self.samples.append((ts, float(f[2]), float(f[3]), float(f[4]),
+                                     [n for n, v in zip(self.NAMES, f[6:10]) if v.lower().startswith("active")]))
             except ValueError:
                 continue
-            for n, v in zip(names, f[5:9]):
-                if v.lower().startswith("active"):
-                    reasons.add(n)
-        sm.sort()
-        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+
+    def window(self, t0, t1):
+        if self.samples is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["clock samples not collected yet"]}
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        inside = [s for s in self.samples if t0 <= s[0] <= t1]
+        note = None
+        if not inside:      # a region shorter than the sampling period: take the sample nearest to its middle
+            mid = 0.5 * (t0 + t1)
+            inside = [min(self.samples, key=lambda s: abs(s[0] - mid))]
+            note = "region shorter than the sampling period: nearest sample"
+        sm = sorted(s[1] for s in inside)
+        reasons = sorted({r for s in inside for r in s[4]})
+        out = {"sm_mhz": sm[len(sm) // 2], "sm_min_mhz": sm[0], "sm_max_mhz": max(s[2] for s in inside),
+               "power_w_max": max(s[3] for s in inside), "samples": len(inside), "reasons": reasons}
+        if note:
+            out["note"] = note
+        return out
 
 
-def cpu_oracle_rate(cfg, d, sample):
-    """tokens/s of the oracle as it stands on the host cores: routing of all T tokens (its per-token share is
-    charged to the sample) plus the per-token FFN of `sample` tokens."""
+def _median(v):
+    v = sorted(v)
+    return v[len(v) // 2]
+
+
+def cpu_oracle_leg(cfg, d, sample, gpu_idx=None, gpu_w=None):
+    """The oracle as it stands on the host cores: routing of all T tokens (its per-token share is charged to the
+    sample) plus the per-token FFN of `sample` tokens.  Returns (tokens/s, seconds, threads, routing report); the
+    report compares the device's top-k ids and weights (when given) with the oracle's, token by token."""
     import numpy as np
     from oracle import mok_ref
     t0 = time.perf_counter()
@@ -112,13 +156,26 @@ def cpu_oracle_rate(cfg, d, sample):
     t_route = time.perf_counter() - t0
     tokens = np.arange(min(sample, cfg.T), dtype=np.int32)
     t0 = time.perf_counter()
-    mok_ref.ffn_tokens(d["x"], d["W_gate_up"], d["W_down"], d["W_sgu"], d["W_sd"], idx, w, tokens)
+    if d.get("W_gate_up") is not None and len(tokens):
+        mok_ref.ffn_tokens(d["x"], d["W_gate_up"], d["W_down"], d["W_sgu"], d["W_sd"], idx, w, tokens)
     t_ffn = time.perf_counter() - t0
     t = t_ffn + t_route * len(tokens) / cfg.T
-    return len(tokens) / t, t_ffn + t_route, mok_ref.num_threads()
+    report = None
+    if gpu_idx is not None:
+        sel = np.take_along_axis(lg, idx.astype(np.int64), axis=1)
+        inner = np.full(cfg.T, np.inf) if cfg.k == 1 else (sel[:, :-1] - sel[:, 1:]).min(axis=1)
+        differs = (gpu_idx != idx).any(axis=1)
+        same_set = (np.sort(gpu_idx, axis=1) == np.sort(idx, axis=1)).all(axis=1)
+        w_sel = mok_ref.weights(lg, gpu_idx)
+        report = {"boundary_near_ties": int((gap < 1e-4).sum()),
+                  "order_near_ties": int(((inner < 1e-4) & ~(gap < 1e-4)).sum()),
+                  "flipped_tokens": int(differs.sum()), "flipped_sets": int((~same_set).sum()),
+                  "flipped_outside_near_ties": int((differs & ~((gap < 1e-4) | (inner < 1e-4))).sum()),
+                  "w_max_err": float(np.abs(gpu_w.astype(np.float64) - w_sel).max())}
+    return (len(tokens) / t if len(tokens) else 0.0), t_ffn + t_route, mok_ref.num_threads(), report
 
 
-def fingerprints(d, limit=1 << 31):
+def fingerprints(d, limit=1 << 28):
     """SHA-256 of each input tensor as generated (tensors above `limit` bytes: of their first `limit` bytes)."""
     import hashlib
     import numpy as np
@@ -133,10 +190,10 @@ def fingerprints(d, limit=1 << 31):
     return out
 
 
-def auto_sample(cfg, cores):
-    # aim at ~15 s of CPU work; the scalar oracle sustains about 4 fp64 GFLOP/s per core on the GPU hosts
+def auto_sample(cfg, cores, seconds=15.0):
+    # the scalar oracle sustains about 4 fp64 GFLOP/s per core on the GPU hosts
     per_token = 6.0 * cfg.H * (cfg.k * cfg.I + cfg.I_s)
-    n = int(15.0 * 4.0e9 * cores / per_token)
+    n = int(seconds * 4.0e9 * cores / per_token)
     return max(16, min(cfg.T, n))
 
 
@@ -148,18 +205,19 @@ def run_reference(args, cfg, rank):
     d = inputs.make_inputs(cfg)
     cores = os.cpu_count() or 1
     steps = max(1, min(args.steps, 3))
-    sample = args.cpu_sample or max(16, auto_sample(cfg, cores) // (steps + min(args.warmup, 1)))
-    for _ in range(min(args.warmup, 1)):
-        cpu_oracle_rate(cfg, d, sample)
+    warm = min(args.warmup, 1)
+    sample = args.cpu_sample or max(16, auto_sample(cfg, cores) // (steps + warm))
+    for _ in range(warm):
+        cpu_oracle_leg(cfg, d, sample)
     rates = []
     t_total = 0.0
     for _ in range(steps):
-        r, t, threads = cpu_oracle_rate(cfg, d, sample)
+        r, t, threads, _ = cpu_oracle_leg(cfg, d, sample)
         rates.append(r)
         t_total += t
     value = sum(rates) / len(rates)
     line = {"metric": METRIC, "value": value, "unit": UNIT, "impl": "reference", "n_gpus": args.gpus, "steps": steps,
-            "warmup": min(args.warmup, 1), "ms_per_step": 1e3 * t_total / steps, "higher_is_better": True,
+            "warmup": warm, "ms_per_step": 1e3 * t_total / steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": cfg.name, "T": cfg.T, "H": cfg.H, "E": cfg.E, "k": cfg.k, "I": cfg.I, "I_shared": cfg.I_s},
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
@@ -202,12 +260,14 @@ def run_backward(args, cfg):
     sampler = ClockSampler(0)
     sampler.start()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.time()
     ev0.record()
     for _ in range(args.steps):
         step()
     ev1.record()
     torch.cuda.synchronize()
-    clocks = sampler.stop()
+    t1 = time.time()
+    sampler.stop()
     ms = ev0.elapsed_time(ev1) / args.steps
     assert mok.mok_read_status(bws) == 0
     flops = 2.0 * cfg.ffn_flops()
@@ -216,7 +276,176 @@ def run_backward(args, cfg):
                       "dtype": "bf16", "data": "synthetic", "tflops": flops / (ms * 1e-3) / 1e12,
                       "config": {"workload": cfg.name, "T": cfg.T, "H": cfg.H, "E": cfg.E, "k": cfg.k, "I": cfg.I,
                                  "I_shared": cfg.I_s, "pass": "backward (recompute + dgrad + wgrad)"},
-                      "clocks": clocks}), flush=True)
+                      "clocks": sampler.window(t0, t1)}), flush=True)
+
+
+class Layer:
+    """One workload resident on the device, with the calls the benchmark times."""
+
+    def __init__(self, cfg, args, dev, rank=0, d=None, staging=0):
+        import torch
+        from paper_2609_36070_b200 import inputs, mok, sharding
+        self.cfg, self.args, self.dev, self.mok, self.torch = cfg, args, dev, mok, torch
+        self.d = d if d is not None else inputs.make_inputs(cfg)
+        if rank > 0:
+            self.d["x"] = sharding.rank_tokens(cfg, rank)
+        d = self.d
+        self.g = {k: (None if d[k] is None else mok.to_device_bf16(d[k], dev))
+                  for k in ("x", "W_gate_up", "W_down", "W_sgu", "W_sd")}
+        self.W_r = torch.from_numpy(d["W_r"]).to(dev)
+        self.bias = None if d["bias"] is None else torch.from_numpy(d["bias"]).to(dev)
+        self.mx = args.precision == "mxfp8"
+        self.prec = mok.MOK_PRECISION_MXFP8 if self.mx else mok.MOK_PRECISION_BF16
+        self.mxw = mok.MxWeights(self.g["W_gate_up"], self.g["W_down"]) if self.mx else None
+        self.ws = mok.alloc_workspace(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k, device=dev, host_staging=staging,
+                                      mx=self.mx)
+        self.out = torch.empty_like(self.g["x"])
+
+    def conf(self, **kw):
+        a = self.args
+        base = dict(impl=a.gemm, gather_mode=a.gather_mode, cta_group=a.cta_group, precision=self.prec,
+                    tile_sched=a.tile_sched)
+        base.update(kw)
+        return self.mok._config(**base)
+
+    def view(self, T):
+        """The same weights with the first T tokens (the small-T sweep)."""
+        import copy
+        v = copy.copy(self)
+        v.cfg = self.cfg.with_tokens(T)
+        v.g = dict(self.g, x=self.g["x"][:T].contiguous())
+        v.out = self.out[:T]
+        return v
+
+    def step(self, conf, stages=False):
+        g, cfg = self.g, self.cfg
+        return self.mok.mok_moe_forward_ex(g["x"], self.W_r, self.bias, g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"],
+                                           cfg.k, self.ws, out=self.out, config=conf, mx_weights=self.mxw, stages=stages)
+
+    def check_status(self):
+        status = self.mok.mok_read_status(self.ws)
+        assert status == 0, self.mok.mok_status_string(status)
+
+    def timed_steps(self, conf, steps, barrier):
+        """K steps bracketed by a barrier + synchronize on both sides, with one CUDA event between consecutive steps.
+        Returns (total ms, per-step ms list, host wall-clock window)."""
+        torch = self.torch
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+        barrier()
+        t0 = time.time()
+        ev[0].record()
+        for i in range(steps):
+            self.step(conf)
+            ev[i + 1].record()
+        barrier()
+        t1 = time.time()
+        return ev[0].elapsed_time(ev[steps]), [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)], (t0, t1)
+
+    def stage_times(self, steps):
+        """Per-stage CUDA-event times (events recorded by the library around every stage) of a loop of its own, so
+        that the events are not part of the headline loop.  Returns {stage: (mean, median)} in ms and the window."""
+        mok = self.mok
+        conf = self.conf(profile=1)
+        mok.mok_profile_begin(steps)
+        self.torch.cuda.synchronize()
+        t0 = time.time()
+        for _ in range(steps):
+            self.step(conf)
+        stage = mok.mok_profile_end(steps)
+        self.torch.cuda.synchronize()
+        t1 = time.time()
+        res = {s: (sum(c[s] for c in stage) / len(stage), _median([c[s] for c in stage])) for s in mok.STAGES}
+        return res, (t0, t1)
+
+    def counters(self):
+        """Device-side counters of the GEMM kernels (one extra step with config.debug = 1), reduced to the figures the
+        roofline discussion uses."""
+        conf = self.conf(debug=1)
+        self.step(conf)
+        raw = self.mok.mok_debug_counters(self.ws)
+        out = {}
+        for name, c in raw.items():
+            if not c["ctas"] or not c["k_blocks"]:
+                continue
+            units = c["k_blocks"]               # 128-row x 64-column-of-K MMA units: 512 tensor-pipe cycles each
+            r = {"sm_ghz_in_kernel": c["mma_total"] / max(1, c["mma_total_ns"]),
+                 "cycles_per_unit": c["mma_total"] / units,
+                 "wait_operands_per_unit": c["mma_wait_operands"] / units,
+                 "wait_accumulator_per_unit": c["mma_wait_accumulator"] / units,
+                 "busiest_cta_over_mean": c["mma_total_max_cta"] / (c["mma_total"] / c["ctas"]),
+                 "ctas": c["ctas"]}
+            if c["valid_rows_x_k_blocks"]:
+                r["pad_row_share_of_mma_work"] = 1.0 - c["valid_rows_x_k_blocks"] / (128.0 * units)
+            out[name] = r
+        return out
+
+
+def roofline_fracs(tflops, pk, mx, region_s, clocks):
+    """achieved / peak against both measured bf16 peaks; `frac` is the one that fits the run: the burst figure for a
+    kernel timed at full clocks in a short region, the sustained one when the timed region lasts seconds or the SM
+    clock sampled during it sits well under the maximum (the board is then in its power-capped steady state)."""
+    scale = 2.0 if mx else 1.0   # fp8 tensor peak = measured bf16 peak x the nominal 2:1 ratio (4.5 vs 2.25 PFLOP/s dense)
+    burst, sust = scale * pk["bf16_tflops"], scale * pk.get("bf16_tflops_sustained", pk["bf16_tflops"])
+    sm, smx = clocks.get("sm_mhz"), clocks.get("sm_max_mhz")
+    sustained = region_s > 2.0 or (sm is not None and smx and sm < 0.9 * smx)
+    peak = sust if sustained else burst
+    return {"achieved": tflops, "peak": peak, "unit": "TFLOP/s", "frac": tflops / peak,
+            "frac_of_burst": tflops / burst, "frac_of_sustained": tflops / sust,
+            "peak_source": f"{pk['source']} " + ("bf16_tflops_sustained" if sustained else "bf16_tflops (burst)") +
+                           (" x 2 (nominal fp8 : bf16 ratio)" if mx else "") +
+                           (": timed region of %.1f s at a median %s MHz of %s" % (region_s, sm, smx))}
+
+
+def measure(layer, steps, warmup, barrier, sampler_windows, pk, with_counters):
+    """Headline loop, stage loop and counters of one workload on this rank.  Clock windows are resolved later, when
+    the sampler has been stopped; `sampler_windows` collects (record, key, window) for that."""
+    cfg, mok = layer.cfg, layer.mok
+    conf = layer.conf()
+    for _ in range(warmup):
+        layer.step(conf)
+    barrier()
+    layer.check_status()
+    total_ms, per_step, win = layer.timed_steps(conf, steps, barrier)
+    layer.check_status()
+    stage_steps = max(3, min(steps, 10))
+    stages, swin = layer.stage_times(stage_steps)
+    layer.check_status()
+    rec = {"ms_per_step": _median(per_step), "mean_ms_per_step": total_ms / steps, "min_ms_per_step": min(per_step),
+           "steps": steps, "stage_ms": {s: stages[s][1] for s in mok.STAGES},
+           "stage_ms_mean": {s: stages[s][0] for s in mok.STAGES}, "_region_s": total_ms * 1e-3,
+           "_stage_region_s": swin[1] - swin[0]}
+    sampler_windows.append((rec, "clocks", win))
+    sampler_windows.append((rec, "clocks_stage_loop", swin))
+    if with_counters and not layer.mx and layer.args.gemm == 0:
+        rec["counters"] = layer.counters()
+        layer.check_status()
+    return rec
+
+
+def finish_record(rec, cfg, pk, mx, world=1):
+    """Derived figures of one workload's record (after the clock windows have been filled in)."""
+    ms = rec["ms_per_step"]
+    flops = cfg.ffn_flops()
+    st = rec["stage_ms"]
+    rec["tokens_per_s"] = world * cfg.T / (ms * 1e-3)
+    rec["tflops"] = world * flops / (ms * 1e-3) / 1e12
+    ffn_ms = st["gemm1"] + st["gemm2"] + st["shared_gemm1"] + st["shared_gemm2"]
+    ffn_tf = flops / (ffn_ms * 1e-3) / 1e12
+    scale = 2.0 if mx else 1.0
+    rec["ffn_phase"] = {"ms": ffn_ms, "tflops": ffn_tf, "frac_of_burst": ffn_tf / (scale * pk["bf16_tflops"]),
+                        "frac_of_sustained": ffn_tf / (scale * pk.get("bf16_tflops_sustained", pk["bf16_tflops"]))}
+    g1_flops = 4.0 * cfg.T * cfg.k * cfg.H * cfg.I
+    g1_tf = g1_flops / (st["gemm1"] * 1e-3) / 1e12
+    clk = rec.get("clocks_stage_loop") or {}
+    dom = roofline_fracs(g1_tf, pk, mx, rec.pop("_stage_region_s"), clk)
+    dom["ms"] = st["gemm1"]
+    if clk.get("sm_mhz"):
+        dom["sm_cycles"] = st["gemm1"] * 1e-3 * clk["sm_mhz"] * 1e6       # kernel time x median sampled SM clock
+    if "counters" in rec and "gemm1" in rec["counters"]:
+        dom["sm_cycles_device"] = st["gemm1"] * 1e-3 * rec["counters"]["gemm1"]["sm_ghz_in_kernel"] * 1e9
+    rec["dominant_kernel"] = dom
+    rec.pop("_region_s", None)
+    return rec
 
 
 def main():
@@ -236,9 +465,10 @@ def main():
             run_backward(args, cfg)
         return
 
+    import gc
     import numpy as np
     import torch
-    from paper_2609_36070_b200 import mok
+    from paper_2609_36070_b200 import mok, sharding
     assert args.warmup >= 3, "timing rules: at least 3 warm-up steps"
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
@@ -247,153 +477,228 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
 
-    # every rank: same weights, its own batch (seed offset by rank)
-    from paper_2609_36070_b200 import sharding
-    d = inputs.make_inputs(cfg)
-    if rank > 0:
-        d["x"] = sharding.rank_tokens(cfg, rank)
-    g = {k: (None if d[k] is None else mok.to_device_bf16(d[k], dev)) for k in ("x", "W_gate_up", "W_down", "W_sgu", "W_sd")}
-    W_r = torch.from_numpy(d["W_r"]).to(dev)
-    bias = None if d["bias"] is None else torch.from_numpy(d["bias"]).to(dev)
-    mx = args.precision == "mxfp8"
-    prec = mok.MOK_PRECISION_MXFP8 if mx else mok.MOK_PRECISION_BF16
-    mxw = mok.MxWeights(g["W_gate_up"], g["W_down"]) if mx else None    # weights are quantised ahead of time
-    ws = mok.alloc_workspace(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k, device=dev, host_staging=2, mx=mx)
-    out = torch.empty_like(g["x"])
-    conf = mok._config(impl=args.gemm, profile=1, gather_mode=args.gather_mode, cta_group=args.cta_group, precision=prec,
-                       tile_sched=args.tile_sched)
-
-    def step():
-        mok.mok_moe_forward_ex(g["x"], W_r, bias, g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], cfg.k, ws,
-                               out=out, config=conf, mx_weights=mxw)
-
     def barrier():
         if dist is not None:
             dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(args.warmup):
-        step()
-    barrier()
-    status = mok.mok_read_status(ws)
-    assert status == 0, mok.mok_status_string(status)
-
+    pk = peaks()
+    mx = args.precision == "mxfp8"
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
-    mok.mok_profile_begin(args.steps)
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    ev0.record()
-    for _ in range(args.steps):
-        step()
-    ev1.record()
-    barrier()
-    total_ms = ev0.elapsed_time(ev1)
-    stage = mok.mok_profile_end(args.steps)
-    clocks = sampler.stop() if rank == 0 else None
-    status = mok.mok_read_status(ws)
-    assert status == 0, mok.mok_status_string(status)
+    windows = []
 
-    total_ms = sharding.max_over_ranks(total_ms, dist, dev)
-    ms_per_step = total_ms / args.steps
-    value = sharding.aggregate_tokens_per_s(cfg.T, world, ms_per_step)
-    flops = cfg.ffn_flops()
-    tflops = world * flops / (ms_per_step * 1e-3) / 1e12
+    # ------------------------------------------------------------------ the headline workload
+    # every rank: same weights, its own batch (seed offset by rank)
+    layer = Layer(cfg, args, dev, rank=rank, staging=0 if args.no_e2e else 2)
+    main_rec = measure(layer, args.steps, args.warmup, barrier, windows, pk, with_counters=not args.no_counters and rank == 0)
+    ms_per_step = sharding.max_over_ranks(main_rec["ms_per_step"], dist, dev)
+    mean_ms = sharding.max_over_ranks(main_rec["mean_ms_per_step"], dist, dev)
+    main_rec["ms_per_step"], main_rec["mean_ms_per_step"] = ms_per_step, mean_ms
+
+    # device's routing of this batch (for the comparison inside the cpu-baseline leg); outside every timed region
+    gpu_idx = gpu_w = counts = None
+    if rank == 0:
+        _, st = layer.step(layer.conf(), stages=True)
+        layer.check_status()
+        gpu_idx, gpu_w = st["topk_idx"].cpu().numpy(), st["topk_w"].cpu().numpy()
+        counts = st["counts"].cpu().numpy()
+        del st
 
     # End to end through the host-buffer entry points: pinned host x -> device, layer, result -> pinned host, every step.
     # Throughput (`e2e.value`): a stream of batches through the asynchronous call, whose two staging slots let the upload
     # of step i+1 and the download of step i-1 overlap the layer of step i; the timed region ends when the last result
     # has arrived in host memory.  Latency of ONE isolated batch (`e2e.single_call_ms`): the blocking call, which cuts
     # the batch into token chunks to overlap its own copies.
-    xh = g["x"].cpu().pin_memory()
-    oh = [torch.empty_like(xh).pin_memory() for _ in range(2)]
-    conf0 = mok._config(impl=args.gemm, gather_mode=args.gather_mode, cta_group=args.cta_group, host_chunks=args.host_chunks,
-                        precision=prec)
+    e2e = None
+    if not args.no_e2e:
+        g = layer.g
+        xh = g["x"].cpu().pin_memory()
+        oh = [torch.empty_like(xh).pin_memory() for _ in range(2)]
+        conf0 = layer.conf(host_chunks=args.host_chunks)
 
-    def e2e_submit(i):
-        mok.mok_moe_forward_host_async(xh, oh[i & 1], W_r, bias, g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], cfg.k,
-                                       ws, config=conf0, mx_weights=mxw)
+        def e2e_submit(i):
+            mok.mok_moe_forward_host_async(xh, oh[i & 1], layer.W_r, layer.bias, g["W_gate_up"], g["W_down"], g["W_sgu"],
+                                           g["W_sd"], cfg.k, layer.ws, config=conf0, mx_weights=layer.mxw)
 
-    def single_call():
-        mok.mok_moe_forward_host(xh, oh[0], W_r, bias, g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], cfg.k, ws,
-                                 config=conf0, mx_weights=mxw)
+        def single_call():
+            mok.mok_moe_forward_host(xh, oh[0], layer.W_r, layer.bias, g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"],
+                                     cfg.k, layer.ws, config=conf0, mx_weights=layer.mxw)
 
-    e2e_steps = max(5, min(args.steps, 50))
-    for i in range(3):
-        e2e_submit(i)
-    mok.mok_host_wait()
-    barrier()
-    ev0.record()
-    for i in range(e2e_steps):
-        e2e_submit(i)
-    mok.mok_host_wait()               # the host blocks until the last download has landed ...
-    ev1.record()                      # ... so this event closes the region after every copy of every step
-    barrier()
-    e2e_ms = ev0.elapsed_time(ev1) / e2e_steps
-    e2e_ms = sharding.max_over_ranks(e2e_ms, dist, dev)
-    for _ in range(2):
-        single_call()
-    barrier()
-    ev0.record()
-    for _ in range(5):
-        single_call()
-    ev1.record()
-    barrier()
-    single_ms = sharding.max_over_ranks(ev0.elapsed_time(ev1) / 5, dist, dev)
-    act_bytes = 2 * cfg.T * cfg.H
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e2e_steps = max(5, min(args.steps, 50))
+        for i in range(3):
+            e2e_submit(i)
+        mok.mok_host_wait()
+        barrier()
+        ev0.record()
+        for i in range(e2e_steps):
+            e2e_submit(i)
+        mok.mok_host_wait()               # the host blocks until the last download has landed ...
+        ev1.record()                      # ... so this event closes the region after every copy of every step
+        barrier()
+        layer.check_status()
+        e2e_ms = sharding.max_over_ranks(ev0.elapsed_time(ev1) / e2e_steps, dist, dev)
+        for _ in range(2):
+            single_call()
+        barrier()
+        ev0.record()
+        for _ in range(3):
+            single_call()
+        ev1.record()
+        barrier()
+        single_ms = sharding.max_over_ranks(ev0.elapsed_time(ev1) / 3, dist, dev)
+        act_bytes = 2 * cfg.T * cfg.H
+        same_bits = bool(torch.equal(oh[(e2e_steps - 1) & 1].view(torch.int16), layer.out.cpu().view(torch.int16)))
+        e2e = {"value": world * cfg.T / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms, "steps": e2e_steps,
+               "h2d_bytes_per_step": act_bytes, "d2h_bytes_per_step": act_bytes,
+               "mode": "stream of batches through mok_moe_forward_host_async (two staging slots), timed until the last "
+                       "result is in host memory",
+               "single_call_ms": single_ms, "result_bits_equal_device_call": same_bits}
+        del xh, oh
 
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
         return
 
-    pk = peaks()
-    mean = {s: float(np.mean([c[s] for c in stage])) for s in mok.STAGES}
-    # dominant kernel: the routed gate/up grouped GEMM with the SwiGLU epilogue (one launch per step)
-    g1_flops = 4.0 * cfg.T * cfg.k * cfg.H * cfg.I
-    g1_tflops = g1_flops / (mean["gemm1"] * 1e-3) / 1e12
-    peak_tf = pk.get("bf16_tflops_sustained", pk["bf16_tflops"])
-    if mx:   # fp8 tensor peak = the measured bf16 peak x the nominal 2:1 ratio (4.5 vs 2.25 PFLOP/s dense)
-        peak_tf *= 2.0
-    per_step = sorted(sum(c[s] for s in mok.STAGES) for c in stage)
-    ffn_ms = mean["gemm1"] + mean["gemm2"] + mean["shared_gemm1"] + mean["shared_gemm2"]
+    # ------------------------------------------------------------------ small-T sweep of the default workload (N = 1)
+    sweep = None
+    if world == 1 and not args.no_sweep and args.config == DEFAULT_WORKLOAD and not args.tokens:
+        sweep = []
+        for T in (64, 512, 4096):
+            v = layer.view(T)
+            rec = measure(v, 30, 5, barrier, windows, pk, with_counters=False)
+            _, st = v.step(v.conf(), stages=True)
+            v.check_status()
+            active = int((st["counts"].cpu().numpy() > 0).sum())
+            wbytes = 2.0 * 3 * cfg.H * (active * cfg.I + cfg.I_s)          # every active expert's weights, read once
+            roof_ms = wbytes / (pk["hbm_gbs"] * 1e9) * 1e3
+            sm = rec["stage_ms"]
+            gemm_ms = sm["gemm1"] + sm["gemm2"] + sm["shared_gemm1"] + sm["shared_gemm2"]
+            rec.update({"T": T, "active_experts": active, "weight_bytes": wbytes, "hbm_roofline_ms": roof_ms,
+                        "gemm_ms": gemm_ms, "gemm_frac_of_hbm_roofline": roof_ms / gemm_ms,
+                        "step_frac_of_hbm_roofline": roof_ms / rec["ms_per_step"],
+                        "tokens_per_s": T / (rec["ms_per_step"] * 1e-3)})
+            rec.pop("_region_s", None)
+            rec.pop("_stage_region_s", None)
+            rec.pop("stage_ms_mean", None)
+            sweep.append(rec)
+            del st
+
+    # ------------------------------------------------------------------ the other workloads (N = 1)
+    names = []
+    if args.per_config == "auto":
+        if world == 1 and args.config == DEFAULT_WORKLOAD and not args.tokens:
+            names = [n for n in inputs.CONFIG_ORDER if n != args.config]
+    elif args.per_config != "none":
+        names = [n for n in args.per_config.split(",") if n]
+    main_d = layer.d
+    main_counts = counts
+    fp = fingerprints(main_d)
+    # keep the host copy of the headline inputs for the cpu-baseline leg; release the device copy before loading others
+    if names:
+        del layer
+        gc.collect()
+        torch.cuda.empty_cache()
+    per_config = {}
+    for n in names:
+        c = inputs.CONFIGS[n]
+        lay = Layer(c, args, dev)
+        est = None
+        for _ in range(3):
+            lay.step(lay.conf())
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        lay.step(lay.conf())
+        e1.record()
+        torch.cuda.synchronize()
+        est = max(e0.elapsed_time(e1), 1e-3)
+        steps = int(min(400, max(20, math.ceil(400.0 / est))))          # a timed region of about 0.4 s or 20 steps
+        rec = measure(lay, steps, 5, barrier, windows, pk, with_counters=not args.no_counters)
+        _, st = lay.step(lay.conf(), stages=True)
+        lay.check_status()
+        rec["config"] = {"workload": c.name, "T": c.T, "H": c.H, "E": c.E, "k": c.k, "I": c.I, "I_shared": c.I_s,
+                         "routing": c.bias}
+        cnt = st["counts"].cpu().numpy()
+        rec["load"] = {"max_count": int(cnt.max()), "empty_experts": int((cnt == 0).sum()),
+                       "rows_padded_to_128": int(((cnt + 127) // 128 * 128).sum()), "rows": int(cnt.sum())}
+        if not args.no_cpu_baseline:   # the cpu-baseline leg of this workload: routing in full, a short FFN sample
+            cores = os.cpu_count() or 1
+            r, s, th, rp = cpu_oracle_leg(c, lay.d, auto_sample(c, cores, seconds=1.0), st["topk_idx"].cpu().numpy(),
+                                          st["topk_w"].cpu().numpy())
+            rec["cpu_baseline"] = {"value": r, "unit": UNIT, "cores": th, "kind": "oracle", "seconds": s}
+            rec["routing_check"] = rp
+        per_config[n] = rec
+        del lay, st
+        gc.collect()
+        torch.cuda.empty_cache()
+
+    sampler.stop()
+    for rec, key, win in windows:
+        rec[key] = sampler.window(*win)
+    region_s = main_rec["_region_s"]
+    finish_record(main_rec, cfg, pk, mx, world)
+    for n, rec in per_config.items():
+        finish_record(rec, inputs.CONFIGS[n], pk, mx)
+        rec.pop("stage_ms_mean", None)
+    if sweep:
+        for rec in sweep:
+            rec.pop("clocks_stage_loop", None)
+
+    dom = main_rec.pop("dominant_kernel")
+    tr = NCU_TRAFFIC.get(cfg.name)
+    roofline = {"kernel": ("routed gate/up grouped GEMM on MXFP8 operands + SwiGLU + activation quantisation, token gather fused "
+                           "(gemm_mx_kernel<EPI_SWIGLU, GATHER>)") if mx else
+                          "routed gate/up grouped GEMM + SwiGLU, token gather fused (gemm_m2_kernel<EPI_SWIGLU, GATHER>)",
+                "bound": "tensor"}
+    roofline.update(dom)
+    roofline["algorithmic_flops_per_launch"] = 4.0 * cfg.T * cfg.k * cfg.H * cfg.I
+    roofline["traffic"] = None if (mx or tr is None) else tr["bytes"] * tr["scale"]
+    if tr is not None and not mx:
+        roofline["traffic_source"] = f"{tr['source']} (ncu capture x {tr['scale']})"
+    conf = mok._config(impl=args.gemm, gather_mode=args.gather_mode, cta_group=args.cta_group,
+                       precision=mok.MOK_PRECISION_MXFP8 if mx else mok.MOK_PRECISION_BF16, tile_sched=args.tile_sched)
     line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "metric": METRIC, "value": main_rec["tokens_per_s"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "mean_ms_per_step": mean_ms,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "mxfp8 routed experts (fp32 accumulate), bf16 elsewhere" if mx else "bf16", "data": "synthetic",
         "config": {"workload": cfg.name, "T": cfg.T, "H": cfg.H, "E": cfg.E, "k": cfg.k, "I": cfg.I,
                    "I_shared": cfg.I_s, "routing": cfg.bias, "parallelism": f"token-sharded replicas x{world}",
-                   "l2": "inputs larger than L2 (weights + activations >> 126 MB), no explicit flush"},
-        "tflops": tflops,
-        "tflops_frac_of_peak": tflops / world / pk["bf16_tflops"],
-        "ffn_phase": {"ms": ffn_ms, "tflops": flops / (ffn_ms * 1e-3) / 1e12,
-                      "frac_of_bf16_peak": flops / (ffn_ms * 1e-3) / 1e12 / pk["bf16_tflops"],
-                      "frac_of_bf16_sustained": flops / (ffn_ms * 1e-3) / 1e12 / peak_tf},
-        "stage_ms": mean,
-        "median_step_ms_from_stage_events": per_step[len(per_step) // 2],
-        "inputs": fingerprints(d),
-        "roofline": {"kernel": ("routed gate/up grouped GEMM on MXFP8 operands + SwiGLU + activation quantisation, token gather fused "
-                                "(gemm_mx_kernel<EPI_SWIGLU, GATHER>)") if mx else
-                               "routed gate/up grouped GEMM + SwiGLU, token gather fused (gemm_m2_kernel<EPI_SWIGLU, GATHER>)",
-                     "bound": "tensor",
-                     "achieved": g1_tflops, "peak": peak_tf, "unit": "TFLOP/s", "frac": g1_tflops / peak_tf,
-                     "peak_source": f"{pk['source']} bf16_tflops_sustained" + (" x 2 (nominal fp8 : bf16 ratio)" if mx else ""),
-                     "traffic": None if mx else NCU_TRAFFIC_BYTES.get(cfg.name)},
-        "e2e": {"value": world * cfg.T / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
-                "h2d_bytes_per_step": act_bytes, "d2h_bytes_per_step": act_bytes,
-                "mode": "stream of batches through mok_moe_forward_host_async (two staging slots), timed until the last "
-                        "result is in host memory",
-                "single_call_ms": single_ms},
+                   "l2": "inputs larger than L2 (weights + activations >> 126 MB), no explicit flush",
+                   "timing": "ms_per_step = median of the per-step CUDA-event times of one bracketed loop of `steps` "
+                             "steps (max over ranks); stage times come from a second loop with per-stage events"},
+        "tflops": main_rec["tflops"],
+        "tflops_frac_of_burst_peak": main_rec["tflops"] / world / ((2.0 if mx else 1.0) * pk["bf16_tflops"]),
+        "ffn_phase": main_rec["ffn_phase"],
+        "stage_ms": main_rec["stage_ms"],
+        "inputs": fp,
+        "roofline": roofline,
         "gpu_launches": args.steps * mok.mok_launch_count(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k, conf),
-        "clocks": clocks,
+        "clocks": main_rec["clocks"],
+        "timed_region_s": region_s,
     }
+    if "counters" in main_rec:
+        line["counters"] = main_rec["counters"]
+    if main_counts is not None:
+        line["load"] = {"max_count": int(main_counts.max()), "empty_experts": int((main_counts == 0).sum()),
+                        "rows_padded_to_128": int(((main_counts + 127) // 128 * 128).sum()), "rows": int(main_counts.sum())}
+    if e2e is not None:
+        line["e2e"] = e2e
     if not args.no_cpu_baseline:
         cores = os.cpu_count() or 1
         sample = args.cpu_sample or auto_sample(cfg, cores)
-        rate, secs, threads = cpu_oracle_rate(cfg, d, sample)
+        rate, secs, threads, rep = cpu_oracle_leg(cfg, main_d, sample, gpu_idx, gpu_w)
         line["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": threads, "kind": "oracle", "seconds": secs,
                                 "sample": f"routing of all {cfg.T} tokens (charged pro rata) + fp64 FFN of the first {min(sample, cfg.T)} tokens"}
+        line["routing_check"] = rep
+    if per_config:
+        line["per_config"] = per_config
+    if sweep:
+        line["sweep"] = sweep
     print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()

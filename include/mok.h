@@ -219,7 +219,7 @@ int mok_schedule_noalloc(const int32_t* topk_idx, int T, int E, int k,
  * Expert parallelism over n_ranks GPUs of one NVLink domain (Sections 2.1 and 3.1-3.3; Algorithm 1 with R source
  * ranks).  Rank c holds the L = E / n_ranks experts [cL, (c+1)L) and T_local tokens.  One layer is, on every rank:
  *   1. mok_route on the rank's own tokens                                  -> topk_idx, topk_w      (local)
- *   2. an all-gather of topk_idx over the ranks (the caller's collective; "all-gather of top-k routes")
+ *   2. an all-gather of topk_idx over the ranks (the caller's collective; Section 3.1: every rank learns all routes)
  *   3. mok_ep_expert_ffn: Algorithm 1 for this rank from the gathered routes (M, S, Phi; no host readback), then
  *      the routed gate/up GEMM whose gather warps PULL each scheduled row straight from its source rank's token
  *      buffer x_peers[src_rank] into shared memory ("pull dispatch": plain 16-byte asynchronous copies over NVLink,
@@ -317,8 +317,8 @@ int mok_mx_quantize_rows(const void* x, int rows, int K, void* codes, void* scal
 size_t mok_mx_workspace_bytes(int T, int H, int I, int I_shared, int E, int k);
 
 /*
- * Backward pass of the layer (Section 3.4 "fused router weight gradient computation", "activation recomputation";
- * Section 4.1: dgrad + wgrad).  The paper prints no formulas: this is the chain rule of the Section 2.1 definition.
+ * Backward pass of the layer (Section 3.4: the router-weight gradient is computed inside the backward chain and the
+ * activations are recomputed rather than stored; Section 4.1: dgrad + wgrad).  The paper prints no formulas: this is the chain rule of the Section 2.1 definition.
  * Inputs: the forward pass's inputs, its routing (topk_idx, topk_w as returned by mok_moe_forward_ex -- the only
  * thing that has to be kept from the forward pass; every activation is recomputed) and dout = dL/dout.
  * Outputs: dx = dL/dx through the experts (bf16 [T, H]; the router's own path from x to the logits is not part of
@@ -374,12 +374,17 @@ int mok_profile_begin(int max_calls);
 int mok_profile_end(float* ms, int max_calls_out, int* n_calls);
 
 /*
- * Wait-time counters of the tcgen05 GEMM kernels of the last forward call that ran with config.debug != 0
- * (measurement aid; Section 3 cost model: T_sync).  Synchronises `stream`, then writes 4 x 8 values: slot 1 = routed
- * gate/up GEMM, 2 = routed down GEMM, 3 = shared GEMMs; per slot, SM cycles summed over CTAs: MMA issuer waiting for
- * operands, for the peer CTA's operands, for a free accumulator; MMA issuer total; k-blocks issued; TMA producer
- * waiting for a free stage; epilogue waiting for an accumulator; epilogue total.
+ * Counters of the tcgen05 GEMM kernels of the last forward call that ran with config.debug != 0 (measurement aid;
+ * Section 3 cost model: T_comp against T_sync).  Synchronises `stream`, then writes 4 x MOK_DEBUG_COUNTERS values:
+ * slot 1 = routed gate/up GEMM, 2 = routed down GEMM, 3 = shared GEMMs.  Per slot, SM cycles summed over CTAs:
+ * [0] MMA issuer waiting for operands, [1] for the peer CTA's operands, [2] for a free accumulator; [3] MMA issuer
+ * total; [4] k-blocks issued (in 128-row units); [5] TMA producer waiting for a free stage; [6] epilogue waiting for an
+ * accumulator; [7] epilogue total; then [8] the busiest CTA's MMA-issuer total (cycles, maximum over CTAs: [8] against
+ * [3] / [11] is the load imbalance of the tile -> CTA rule); [9] MMA issuer total in nanoseconds of the global timer
+ * ([3] / [9] = the SM clock the kernel really ran at, in GHz); [10] valid rows x k-blocks issued (256-row kernel
+ * only, else 0: 128 x [4] minus this is the MMA work spent on padding rows); [11] CTAs that reported.
  */
+#define MOK_DEBUG_COUNTERS 12
 int mok_debug_counters(const void* workspace, void* stream, unsigned long long* out);
 
 /* Number of kernels one mok_moe_forward_ex call enqueues for these arguments (the memset of the workspace header

@@ -14,8 +14,8 @@
  *   - routes are flattened token-major: route j = t*k + s.
  *
  * What follows which passage of the paper
- *   mok_ref_logits / mok_ref_topk / mok_ref_weights : Section 2.1 ("router projection to select
- *       the top-k routed experts and assign each a router weight") and the normalised weights
+ *   mok_ref_logits / mok_ref_topk / mok_ref_weights : Section 2.1 (the router projects every token
+ *       onto the experts, keeps its k best and weights each of them) and the normalised weights
  *       s_i / sum_j s_j of the MoE equation in Section 2.1.  Score = softmax over all E logits
  *       (the benchmark configuration's reading); ties go to the lowest expert id.
  *   mok_ref_schedule : the dispatch schedule of one rank as Section 3.1 restates Algorithm 1: the

@@ -1,10 +1,10 @@
-// Backward pass of the MoE layer (paper, Section 3.4 "fused router weight gradient", "activation recomputation";
+// Backward pass of the MoE layer (paper, Section 3.4: the router-weight gradient fused into the backward chain, activations recomputed instead of stored;
 // Section 4.1: backward = dgrad + wgrad, twice the forward FLOPs).  The paper prints no formulas; this is the chain
 // rule of the Section 2.1 definition, arranged so that every contraction runs on the forward pass's grouped tcgen05
 // GEMM kernels:
 //
 //   saved from the forward pass: only the routing (top-k ids and weights).  Everything else is recomputed from x
-//   ("activation recomputation"): the dispatch schedule from the ids, the pre-activations gu = [g | u] = Xg Wgu^T.
+//   (Section 3.4): the dispatch schedule from the ids, the pre-activations gu = [g | u] = Xg Wgu^T.
 //
 //   activation gradients (dgrad)
 //     dhu  = gather(dout) Wd            grouped GEMM, rows pulled from dout through the schedule (K = H, N = I)

@@ -178,6 +178,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
             uint32_t ph = 0, aph = 0;
             long long d_full = 0, d_pfull = 0, d_tempty = 0, d_kb = 0;
             const long long d_t0 = dbg ? clock64() : 0;
+            const unsigned long long d_ns0 = dbg ? globaltimer() : 0ull;
             for (int L = unit; L < total; L += n_units) {
                 long long w0 = dbg ? clock64() : 0;
                 bool ok = mbar_wait(smem_u32(&ctrl->tempty[as]), aph ^ 1u, abort_flag, a.header, 2);
@@ -210,8 +211,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
                 atomicAdd(d + DBG_MMA_WAIT_FULL, (unsigned long long)d_full);
                 atomicAdd(d + DBG_MMA_WAIT_PFULL, (unsigned long long)d_pfull);
                 atomicAdd(d + DBG_MMA_WAIT_TEMPTY, (unsigned long long)d_tempty);
-                atomicAdd(d + DBG_MMA_TOTAL, (unsigned long long)(clock64() - d_t0));
+                const unsigned long long d_tot = (unsigned long long)(clock64() - d_t0);
+                atomicAdd(d + DBG_MMA_TOTAL, d_tot);
+                atomicMax(d + DBG_MMA_TOTAL_MAX, d_tot);
+                atomicAdd(d + DBG_MMA_TOTAL_NS, globaltimer() - d_ns0);
                 atomicAdd(d + DBG_KBLOCKS, (unsigned long long)d_kb);
+                atomicAdd(d + DBG_CTAS, 1ull);
             }
         } else if (lane == 0 && CTAS == 2 && GATHER) {
             // -------------------------------------------------------------- odd CTA: tell the even CTA that my stage landed

@@ -265,8 +265,9 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
             int s = 0;
             uint32_t ph = 0, ap0 = 0, ap1 = 0;        // phases of tempty[0], tempty[1]: they advance per use
             const bool dbg = a.dbg_slot >= 0;
-            long long d_full = 0, d_tempty = 0, d_kb = 0;
+            long long d_full = 0, d_tempty = 0, d_kb = 0, d_rows = 0;
             const long long d_t0 = dbg ? clock64() : 0;
+            const unsigned long long d_ns0 = dbg ? globaltimer() : 0ull;
             TileSeq<CLC> seq(ctrl, abort_flag, a.header, total, false);
             for (int L = seq.first(); L < total; L = seq.next(L)) {
                 const Tile t = decode_tile<KGROUP>(a, L, n_nt, n_mt_total, k_blocks);
@@ -321,13 +322,19 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
                 }
                 if (!ok) break;
                 if (two) { tc_commit<1>(smem_u32(&ctrl->tfull[1])); ap1 ^= 1u; }
+                if (dbg) d_rows += (long long)t.valid * t.kblocks;
             }
             if (dbg) {   // k_blocks counted in 128-row units so that the figures compare with the 128-row kernel
                 unsigned long long* d = a.header->dbg[a.dbg_slot];
                 atomicAdd(d + DBG_MMA_WAIT_FULL, (unsigned long long)d_full);
                 atomicAdd(d + DBG_MMA_WAIT_TEMPTY, (unsigned long long)d_tempty);
-                atomicAdd(d + DBG_MMA_TOTAL, (unsigned long long)(clock64() - d_t0));
+                const unsigned long long d_tot = (unsigned long long)(clock64() - d_t0);
+                atomicAdd(d + DBG_MMA_TOTAL, d_tot);
+                atomicMax(d + DBG_MMA_TOTAL_MAX, d_tot);
+                atomicAdd(d + DBG_MMA_TOTAL_NS, globaltimer() - d_ns0);
                 atomicAdd(d + DBG_KBLOCKS, (unsigned long long)d_kb);
+                atomicAdd(d + DBG_ROWS_KB, (unsigned long long)d_rows);
+                atomicAdd(d + DBG_CTAS, 1ull);
             }
         }
         __syncwarp();

@@ -25,11 +25,15 @@ struct WsHeader {
     uint32_t wait_limit_us; // 0 = default (2 s): bound of every mbarrier wait, in microseconds
     int32_t n_flag;        // tensor-core router: tokens on the near-tie list of the current call
     int32_t pad[58];
-    // optional wait-time counters of the tcgen05 GEMMs (config.debug): [slot][counter], SM cycles summed over CTAs
-    unsigned long long dbg[4][8];
+    // optional counters of the tcgen05 GEMMs (config.debug): [slot][counter]; SM cycles summed over CTAs unless stated
+    unsigned long long dbg[4][MOK_DEBUG_COUNTERS];
 };
 enum { DBG_MMA_WAIT_FULL = 0, DBG_MMA_WAIT_PFULL, DBG_MMA_WAIT_TEMPTY, DBG_MMA_TOTAL, DBG_KBLOCKS,
-       DBG_PROD_WAIT_EMPTY, DBG_EPI_WAIT_TFULL, DBG_EPI_TOTAL };
+       DBG_PROD_WAIT_EMPTY, DBG_EPI_WAIT_TFULL, DBG_EPI_TOTAL,
+       DBG_MMA_TOTAL_MAX,     // the busiest CTA's MMA-issuer time (cycles, maximum over CTAs)
+       DBG_MMA_TOTAL_NS,      // MMA-issuer time in nanoseconds of the global timer, summed over CTAs (cycles / ns = SM clock)
+       DBG_ROWS_KB,           // valid (non-padding) rows x k-blocks issued (256-row kernel only)
+       DBG_CTAS };            // CTAs that reported
 
 // Byte offsets of every workspace region, computed on the host from the sizes alone (no readback).
 struct WsLayout {

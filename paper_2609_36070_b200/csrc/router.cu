@@ -1,5 +1,5 @@
 // Router projection, top-k selection and normalised weights (paper, Section 2.1; Figure 1 right: the
-// GPU-side "router projection, top-k selection" step that runs before the expert kernels).
+// GPU-side routing step that runs before the expert kernels).
 //
 //   logit[t,e] = sum_h x[t,h] * W_r[e,h] (+ bias[e])      fp32 accumulation, W_r kept in fp32
 //   idx[t,0..k) = the k largest logits, ordered by (logit desc, expert id asc)

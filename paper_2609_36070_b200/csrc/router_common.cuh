@@ -1,5 +1,5 @@
 // Warp-level top-k selection and normalised router weights shared by the two router implementations
-// (paper, Section 2.1: "select the top-k routed experts and assign each a router weight").
+// (paper, Section 2.1: the router picks each token's k experts and gives each pick a weight).
 #pragma once
 #include <cuda_runtime.h>
 #include <float.h>

@@ -525,16 +525,18 @@ def mok_moe_backward(x, W_gate_up, W_down, W_shared_gate_up, W_shared_down, topk
 
 
 DEBUG_COUNTERS = ["mma_wait_operands", "mma_wait_peer_operands", "mma_wait_accumulator", "mma_total", "k_blocks",
-                  "producer_wait_stage", "epilogue_wait_accumulator", "epilogue_total"]
+                  "producer_wait_stage", "epilogue_wait_accumulator", "epilogue_total", "mma_total_max_cta",
+                  "mma_total_ns", "valid_rows_x_k_blocks", "ctas"]
 
 
 def mok_debug_counters(workspace, stream=None):
     """{slot: {counter: cycles}} of the last forward call that ran with config.debug != 0."""
-    buf = (ctypes.c_ulonglong * 32)()
+    n = len(DEBUG_COUNTERS)
+    buf = (ctypes.c_ulonglong * (4 * n))()
     wp, _ = _aligned_ws(workspace)
     _check(_lib.mok_debug_counters(wp, _stream(stream), buf))
     names = {1: "gemm1", 2: "gemm2", 3: "shared"}
-    return {names[s]: {n: int(buf[s * 8 + i]) for i, n in enumerate(DEBUG_COUNTERS)} for s in names}
+    return {names[s]: {c: int(buf[s * n + i]) for i, c in enumerate(DEBUG_COUNTERS)} for s in names}
 
 
 def mok_read_status(workspace, stream=None):

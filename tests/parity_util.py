@@ -1,9 +1,11 @@
 """Shared helpers of the GPU parity tests: run the CUDA layer through the C-ABI binding and compare every stage
-with the CPU oracle on the same seeded inputs.  Tolerances (stated by the benchmark spec):
-  * top-k indices, counts, offsets, perm, inv_perm: bit-exact, except tokens whose k-th/(k+1)-th logit gap is
-    < 1e-4, or whose selected logits contain an adjacent pair closer than 1e-4 (which decides the slot order)
-    (near-ties; counted and reported, and the schedule is then checked against the oracle's schedule of
-    the device's own selection);
+with the CPU oracle on the same seeded inputs.  Tolerances:
+  * top-k indices, counts, offsets, perm, inv_perm: bit-exact, with two counted exceptions, both decided on the
+    oracle's fp64 logits: (a) BOUNDARY near-ties -- tokens whose k-th / (k+1)-th logit gap is < 1e-4 may select the
+    other candidate; (b) ORDER near-ties -- tokens whose selected logits contain an adjacent pair closer than 1e-4 may
+    come out with those slots swapped, but must select the same SET of experts as the oracle unless (a) also holds.
+    The two classes are reported separately; whenever a token differs, the schedule is checked against the oracle's
+    schedule of the device's own selection;
   * router weights: |w_gpu - w_ref| <= 5e-5 (the tensor-core logits carry an accumulation bias of up to ~5e-5 at
     H = 7168, and dw <= dlogit / 4; tokens whose candidates are closer than that bias are re-decided exactly);
   * outputs: max|gpu - ref| <= 1e-2 * max|ref| and mean|gpu - ref| / mean|ref| <= 5e-3.
@@ -51,14 +53,19 @@ def check_routing_and_schedule(cfg, d, st):
     idx_gpu = st["topk_idx"].cpu().numpy()
     w_gpu = st["topk_w"].cpu().numpy().astype(np.float64)
     differs = (idx_gpu != idx_ref).any(axis=1)
-    # Near-ties.  The selection is decided at the k-th/(k+1)-th boundary (gap); the slot ORDER inside the selection
-    # is decided by the same kind of comparison between adjacent selected logits, so the same 1e-4 rule applies:
-    # a token whose closest adjacent pair among its top-(k+1) logits is nearer than 1e-4 may differ, and is counted.
+    # Near-ties, two classes.  The selection is decided at the k-th/(k+1)-th boundary (gap); the slot ORDER inside the
+    # selection is decided by the same kind of comparison between adjacent selected logits, so the same 1e-4 applies.
     sel = np.take_along_axis(lg, idx_ref.astype(np.int64), axis=1)           # descending
     inner = np.full(cfg.T, np.inf) if cfg.k == 1 else (sel[:, :-1] - sel[:, 1:]).min(axis=1)
-    near = np.minimum(gap, inner) < NEAR_TIE
+    boundary = gap < NEAR_TIE
+    order = inner < NEAR_TIE
+    near = boundary | order
     bad = differs & ~near
     assert not bad.any(), f"{bad.sum()} tokens with a different top-k that are not near-ties, first {np.flatnonzero(bad)[:5]}"
+    # away from a boundary near-tie the selected SET must be the oracle's: only the slot order is excused by class (b)
+    same_set = (np.sort(idx_gpu, axis=1) == np.sort(idx_ref, axis=1)).all(axis=1)
+    bad_set = ~same_set & ~boundary
+    assert not bad_set.any(), f"{bad_set.sum()} tokens select another set of experts without a boundary near-tie"
     # a flipped near-tie must still be a valid selection in a valid order, both up to the tolerance
     for t in np.flatnonzero(differs):
         lsel = lg[t, idx_gpu[t]]
@@ -73,7 +80,9 @@ def check_routing_and_schedule(cfg, d, st):
     assert np.array_equal(st["offsets"].cpu().numpy(), offsets)
     assert np.array_equal(st["perm"].cpu().numpy(), perm)
     assert np.array_equal(st["inv_perm"].cpu().numpy(), inv)
-    report = {"near_tie_tokens": int(near.sum()), "flipped_tokens": int(differs.sum()), "w_max_err": float(werr),
+    report = {"near_tie_tokens": int(near.sum()), "boundary_near_ties": int(boundary.sum()),
+              "order_near_ties": int((order & ~boundary).sum()), "flipped_tokens": int(differs.sum()),
+              "flipped_sets": int((~same_set).sum()), "w_max_err": float(werr),
               "empty_experts": int((counts == 0).sum()), "max_count": int(counts.max())}
     return idx_gpu, w_sel, report
 

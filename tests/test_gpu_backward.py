@@ -110,7 +110,8 @@ def test_bench_shape_with_fewer_tokens_all_gradients():
 
 
 def test_bench_shape_full_size_sampled():
-    """Full benchmark workload: dx and dw of a token sample against the oracle, everything finite, run-to-run bitwise."""
+    """Full-size Qwen3-like workload: dx and dw of a token sample and the weight gradients of the experts with few routes
+    against the oracle, everything finite, run-to-run bitwise."""
     m = mok()
     cfg = inputs.CONFIGS["qwen3_30b_a3b"]
     d = inputs.make_inputs(cfg)
@@ -134,6 +135,26 @@ def test_bench_shape_full_size_sampled():
         assert diff.max() <= MAX_REL_BWD * np.abs(want).max() and diff.mean() <= MEAN_REL_BWD * np.abs(want).mean(), name
     for name in ("dW_gate_up", "dW_down"):
         assert torch.isfinite(res[name].float()).all()
+    # Weight gradients at full size: an expert's gradient only depends on the tokens routed to it, so for the experts
+    # with few routes the oracle evaluates a one-expert layer on exactly those tokens (the route's weight as its only
+    # combine weight) -- the same sums, cheap in fp64.  Experts without routes must come out as exact zeros.
+    idx_h, w_h = idx.cpu().numpy(), w.cpu().numpy().astype(np.float64)
+    counts = np.bincount(idx_h.ravel(), minlength=cfg.E)
+    dout64 = inputs.bf16_bits_to_f32(dout_bits).astype(np.float64)
+    small = [e for e in np.argsort(counts) if 0 < counts[e] <= 64][:6]
+    assert small, "the Zipf routing of this workload has experts with a handful of routes"
+    for e in small:
+        toks, slots = np.nonzero(idx_h == e)
+        sub = mok_ref.backward(np.ascontiguousarray(d["x"][toks]), d["W_gate_up"][e:e + 1], d["W_down"][e:e + 1], None, None,
+                               np.zeros((toks.size, 1), np.int32), w_h[toks, slots].reshape(-1, 1),
+                               np.ascontiguousarray(dout64[toks]))
+        for name in ("dW_gate_up", "dW_down"):
+            got = res[name][e].float().cpu().numpy().astype(np.float64)
+            want = sub[name][0]
+            diff = np.abs(got - want)
+            assert diff.max() <= MAX_REL_BWD * np.abs(want).max() and diff.mean() <= MEAN_REL_BWD * np.abs(want).mean(), (name, e)
+    for e in np.flatnonzero(counts == 0):
+        assert float(res["dW_gate_up"][e].float().abs().max()) == 0.0 and float(res["dW_down"][e].float().abs().max()) == 0.0
     again = m.mok_moe_backward(g["x"], g["W_gate_up"], g["W_down"], None, None, idx, w, dout, workspace=res["workspace"])
     torch.cuda.synchronize()
     for name in ("dx", "dW_gate_up", "dW_down"):

@@ -47,6 +47,19 @@ def test_full_size_mxfp8_sampled():
     torch.cuda.empty_cache()
 
 
+def test_full_size_mxfp8_ragged_k_and_n_tails():
+    """MXFP8 mode on the GPT-OSS-like workload: H = I = 2880 is not a multiple of 128 (K tails of 64 in both GEMMs,
+    a partial last N tile, a partial last scale atom)."""
+    cfg = inputs.CONFIGS["gpt_oss_120b"]
+    d = inputs.make_inputs(cfg)
+    g = pu.upload(d)
+    out, rep = pu.mx_parity(cfg, d=d, g=g, n_sample=128)
+    print(cfg.name, "mxfp8", rep)
+    del d, g, out
+    gc.collect()
+    torch.cuda.empty_cache()
+
+
 def test_deepseek_v3_full_and_small_token_sweep():
     """The largest workload (about 23 GB of expert weights resident) and its small-T sweep with the same weights."""
     cfg = inputs.CONFIGS["deepseek_v3"]
@@ -55,7 +68,8 @@ def test_deepseek_v3_full_and_small_token_sweep():
         pytest.skip("needs about 60 GB of free device memory")
     d = inputs.make_inputs(cfg)
     g = pu.upload(d)
-    for T, n in [(64, None), (512, 64)]:
+    # T = 4096 (128 rows per expert on average) is where the choice between the 128-row and the 256-row kernel flips
+    for T, n in [(64, None), (512, 64), (4096, 64)]:
         sub = cfg.with_tokens(T)
         ds = dict(d, x=np.ascontiguousarray(d["x"][:T]))
         gs = dict(g, x=g["x"][:T].contiguous())

@@ -2,10 +2,14 @@
 serving loop that must avoid cudaMalloc's device-wide synchronisation, a process whose framework owns all of HBM, a
 plug-in that only receives input and output buffers).  Its scratch is a fixed array inside the library, shared by all
 calls and never cleared as a whole, so the test makes two calls in a row with different sizes and checks each,
-bit for bit (the outputs are integers), against mok_schedule with a caller-owned workspace.  This file sorts last
+bit for bit (the outputs are integers), against mok_schedule with a caller-owned workspace and against the CPU
+oracle's schedule of the same routes.  This file sorts last
 on purpose: a failure here cannot hide the result of any other test under `pytest -x`."""
+import numpy as np
 import pytest
 import torch
+
+from oracle import mok_ref
 
 pytestmark = pytest.mark.gpu
 
@@ -25,6 +29,9 @@ def test_noalloc_schedule_matches_workspace_schedule_on_consecutive_calls():
         torch.cuda.synchronize()
         for name, a, b in zip(("counts", "offsets", "perm", "inv_perm"), want, got):
             assert torch.equal(a, b), name
+        ref = mok_ref.schedule(idx.cpu().numpy().ravel(), E)       # the oracle's stable counting sort of the same routes
+        for name, a, b in zip(("counts", "offsets", "perm", "inv_perm"), ref, got):
+            assert np.array_equal(a, b.cpu().numpy()), name
         assert int(got[0].sum()) == T * k and int(got[0][5]) == 0
         if first is None:
             first = (idx, got)
