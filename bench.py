@@ -57,6 +57,8 @@ def parse():
     p.add_argument("--no-sweep", action="store_true", help="skip the small-T sweep of the default workload")
     p.add_argument("--no-e2e", action="store_true", help="skip the host-buffer (end-to-end) legs")
     p.add_argument("--no-counters", action="store_true", help="skip the device-side counter pass")
+    p.add_argument("--sustain-seconds", type=float, default=2.0,
+                   help="length of the extra loop that shows the power-capped steady state (0 = skip)")
     p.add_argument("--gather-mode", type=int, default=0, help="0 auto, 1 fused into the GEMM, 2 separate kernel")
     p.add_argument("--cta-group", type=int, default=0, help="0 default, 1 single CTAs, 2 CTA pairs")
     p.add_argument("--gemm", type=int, default=0, help="0 tcgen05 (tokens on M), 2 tcgen05 (tokens on N), 1 SIMT")
@@ -91,10 +93,14 @@ class ClockSampler:
         self.samples = None
 
     def start(self):
+        import tempfile
+        self.t_start = time.time()
+        # into a file: a pipe that nobody drains fills up after a few hundred lines and stops nvidia-smi
+        self.log = tempfile.NamedTemporaryFile("w+", prefix="mok_clocks_", suffix=".csv", delete=False)
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.Q}",
                                           "--format=csv,noheader,nounits", "-lms", "20"],
-                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                                         stdout=self.log, stderr=subprocess.DEVNULL)
         except OSError:
             self.proc = None
 
@@ -105,10 +111,18 @@ class ClockSampler:
         time.sleep(0.05)
         self.proc.terminate()
         try:
-            out, _ = self.proc.communicate(timeout=10)
+            self.proc.wait(timeout=10)
         except subprocess.TimeoutExpired:
             self.proc.kill()
-            out, _ = self.proc.communicate()
+            self.proc.wait()
+        self.log.flush()
+        self.log.seek(0)
+        out = self.log.read()
+        self.log.close()
+        try:
+            os.unlink(self.log.name)
+        except OSError:
+            pass
         for line in out.strip().splitlines():
             f = [v.strip() for v in line.split(",")]
             if len(f) < 10:
@@ -119,6 +133,12 @@ class ClockSampler:
                                      [n for n, v in zip(self.NAMES, f[6:10]) if v.lower().startswith("active")]))
             except ValueError:
                 continue
+        # nvidia-smi prints local time and time.time() counts from the UTC epoch: where the two disagree about the
+        # time zone the difference is a whole number of quarter hours, which the first sample reveals
+        if self.samples:
+            off = round((self.samples[0][0] - self.t_start) / 900.0) * 900.0
+            if off:
+                self.samples = [(s[0] - off,) + s[1:] for s in self.samples]
 
     def window(self, t0, t1):
         if self.samples is None:
@@ -299,6 +319,11 @@ class Layer:
         self.mxw = mok.MxWeights(self.g["W_gate_up"], self.g["W_down"]) if self.mx else None
         self.ws = mok.alloc_workspace(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k, device=dev, host_staging=staging,
                                       mx=self.mx)
+        # the router weights are split once, as a caller of the library would do at load time
+        try:
+            self.split = mok.mok_router_prepare(self.W_r, cfg.k, self.conf())
+        except mok.MokError:
+            self.split = None
         self.out = torch.empty_like(self.g["x"])
 
     def conf(self, **kw):
@@ -320,7 +345,8 @@ class Layer:
     def step(self, conf, stages=False):
         g, cfg = self.g, self.cfg
         return self.mok.mok_moe_forward_ex(g["x"], self.W_r, self.bias, g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"],
-                                           cfg.k, self.ws, out=self.out, config=conf, mx_weights=self.mxw, stages=stages)
+                                           cfg.k, self.ws, out=self.out, config=conf, mx_weights=self.mxw, stages=stages,
+                                           router_split=self.split)
 
     def check_status(self):
         status = self.mok.mok_read_status(self.ws)
@@ -341,9 +367,10 @@ class Layer:
         t1 = time.time()
         return ev[0].elapsed_time(ev[steps]), [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)], (t0, t1)
 
-    def stage_times(self, steps):
+    def stage_times(self, steps, second_half=False):
         """Per-stage CUDA-event times (events recorded by the library around every stage) of a loop of its own, so
-        that the events are not part of the headline loop.  Returns {stage: (mean, median)} in ms and the window."""
+        that the events are not part of the headline loop.  Returns {stage: (mean, median)} in ms and the window;
+        second_half: statistics over the second half of the loop only (the steady state of a long loop)."""
         mok = self.mok
         conf = self.conf(profile=1)
         mok.mok_profile_begin(steps)
@@ -354,6 +381,9 @@ class Layer:
         stage = mok.mok_profile_end(steps)
         self.torch.cuda.synchronize()
         t1 = time.time()
+        if second_half:
+            stage = stage[len(stage) // 2:]
+            t0 = 0.5 * (t0 + t1)
         res = {s: (sum(c[s] for c in stage) / len(stage), _median([c[s] for c in stage])) for s in mok.STAGES}
         return res, (t0, t1)
 
@@ -416,6 +446,17 @@ def measure(layer, steps, warmup, barrier, sampler_windows, pk, with_counters):
            "_stage_region_s": swin[1] - swin[0]}
     sampler_windows.append((rec, "clocks", win))
     sampler_windows.append((rec, "clocks_stage_loop", swin))
+    # The steady state under the board's power cap: a loop of a few seconds, statistics over its second half, and the
+    # device-side counters (in-kernel SM clock) right behind it while the board is still in that state.
+    secs = layer.args.sustain_seconds
+    if secs > 0:
+        n = int(max(10, min(5000, secs * 1e3 / rec["ms_per_step"])))
+        sstages, ssw = layer.stage_times(n, second_half=True)
+        layer.check_status()
+        srec = {"steps": n, "stage_ms": {s: sstages[s][0] for s in mok.STAGES}}
+        srec["ms_per_step"] = sum(srec["stage_ms"].values())
+        rec["sustained"] = srec
+        sampler_windows.append((srec, "clocks", ssw))
     if with_counters and not layer.mx and layer.args.gemm == 0:
         rec["counters"] = layer.counters()
         layer.check_status()
@@ -445,6 +486,18 @@ def finish_record(rec, cfg, pk, mx, world=1):
         dom["sm_cycles_device"] = st["gemm1"] * 1e-3 * rec["counters"]["gemm1"]["sm_ghz_in_kernel"] * 1e9
     rec["dominant_kernel"] = dom
     rec.pop("_region_s", None)
+    if "sustained" in rec:
+        s = rec["sustained"]
+        sst = s["stage_ms"]
+        sffn = sst["gemm1"] + sst["gemm2"] + sst["shared_gemm1"] + sst["shared_gemm2"]
+        sust_peak = scale * pk.get("bf16_tflops_sustained", pk["bf16_tflops"])
+        s["tokens_per_s"] = world * cfg.T / (s["ms_per_step"] * 1e-3)
+        s["tflops"] = world * flops / (s["ms_per_step"] * 1e-3) / 1e12
+        s["ffn_phase"] = {"ms": sffn, "tflops": flops / (sffn * 1e-3) / 1e12,
+                          "frac_of_sustained": flops / (sffn * 1e-3) / 1e12 / sust_peak,
+                          "frac_of_burst": flops / (sffn * 1e-3) / 1e12 / (scale * pk["bf16_tflops"])}
+        s["dominant_kernel"] = {"ms": sst["gemm1"], "tflops": g1_flops / (sst["gemm1"] * 1e-3) / 1e12,
+                                "frac_of_sustained": g1_flops / (sst["gemm1"] * 1e-3) / 1e12 / sust_peak}
     return rec
 
 
@@ -569,7 +622,10 @@ def main():
         sweep = []
         for T in (64, 512, 4096):
             v = layer.view(T)
+            keep = args.sustain_seconds
+            args.sustain_seconds = 0.0
             rec = measure(v, 30, 5, barrier, windows, pk, with_counters=False)
+            args.sustain_seconds = keep
             _, st = v.step(v.conf(), stages=True)
             v.check_status()
             active = int((st["counts"].cpu().numpy() > 0).sum())
@@ -616,7 +672,7 @@ def main():
         e1.record()
         torch.cuda.synchronize()
         est = max(e0.elapsed_time(e1), 1e-3)
-        steps = int(min(400, max(20, math.ceil(400.0 / est))))          # a timed region of about 0.4 s or 20 steps
+        steps = int(min(200, max(20, math.ceil(50.0 / est))))           # a short timed region: about 50 ms or 20 steps
         rec = measure(lay, steps, 5, barrier, windows, pk, with_counters=not args.no_counters)
         _, st = lay.step(lay.conf(), stages=True)
         lay.check_status()
@@ -656,6 +712,8 @@ def main():
                 "bound": "tensor"}
     roofline.update(dom)
     roofline["algorithmic_flops_per_launch"] = 4.0 * cfg.T * cfg.k * cfg.H * cfg.I
+    if "sustained" in main_rec:
+        roofline["sustained_run"] = main_rec["sustained"]["dominant_kernel"]
     roofline["traffic"] = None if (mx or tr is None) else tr["bytes"] * tr["scale"]
     if tr is not None and not mx:
         roofline["traffic_source"] = f"{tr['source']} (ncu capture x {tr['scale']})"
@@ -681,6 +739,8 @@ def main():
         "clocks": main_rec["clocks"],
         "timed_region_s": region_s,
     }
+    if "sustained" in main_rec:
+        line["sustained"] = main_rec["sustained"]
     if "counters" in main_rec:
         line["counters"] = main_rec["counters"]
     if main_counts is not None:

@@ -131,6 +131,9 @@ typedef struct mok_args {
     const void* W_gate_up_scales;   /* E8M0 scale atoms of the 2E matrices [I, H] */
     const void* W_down_codes;       /* E4M3 [E, H, I] */
     const void* W_down_scales;      /* E8M0 scale atoms of the E matrices [H, I] */
+    /* optional: W_router split ahead of time by mok_router_prepare (same E, H, k and config.router_impl as this call);
+       NULL = the split is redone inside every call.  W_router is still needed (near-ties are re-decided in fp32). */
+    const void* W_router_split;
 } mok_args;
 
 /*
@@ -151,6 +154,19 @@ size_t mok_workspace_bytes(int T, int H, int I, int I_shared, int E, int k);
 
 /* Same layer with a router bias, caller-owned workspace, stage outputs and knobs (see mok_args). */
 int mok_moe_forward_ex(const mok_args* args);
+
+/*
+ * Router weights prepared once (Section 2.1 router projection; Figure 1, right: the routing step precedes the expert
+ * kernels on every call, but W_router is a weight).  The tensor-core router multiplies x by an exact three-way bf16
+ * split of the fp32 W_router (hi + mid + lo); mok_router_prepare writes that split for the given E, H, k and
+ * config->router_impl into `out` (device, 16-byte aligned, at least mok_router_prepared_bytes(E, H) bytes; the
+ * caller owns it), and mok_args.W_router_split hands it to later forward calls, which then skip their own split
+ * kernel.  Same result bits either way.  MOK_ERR_UNSUPPORTED when the configuration routes with the fp32-FMA kernel
+ * (config->router_impl = 1, config->impl = MOK_IMPL_SIMT with router_impl = 0, or k > 28), which has no split.
+ */
+size_t mok_router_prepared_bytes(int E, int H);
+int mok_router_prepare(const float* W_router, int E, int H, int k, const mok_config* config, void* out, size_t out_bytes,
+                       void* stream);
 
 /*
  * Same layer with the activations in HOST memory: x_host (bf16 [T,H]) is copied to the device, the layer

@@ -162,11 +162,17 @@ struct TileSeq {
 template <int EPI, bool GATHER, int MODE, bool CLC>
 __global__ void __launch_bounds__(THREADS + (GATHER ? GATHER_THREADS : 0) + (CLC ? 32 : 0), 1)
 gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
-               const __grid_constant__ CUtensorMap tmapC, const __grid_constant__ GemmArgs a, const int n_nt, const int k_blocks) {
+               const __grid_constant__ CUtensorMap tmapC, const __grid_constant__ CUtensorMap tmapB64,
+               const __grid_constant__ GemmArgs a, const int n_nt, const int k_blocks) {
     constexpr bool SWIGLU = (EPI == EPI_SWIGLU);
     // MODE 3: the K-range mode with BOTH operands read MN-major: A = [rows of the dispatch space, M] and
     // B = [rows, N] as the backward pass produces them, no transposed copies
     constexpr bool KGROUP = (MODE == 1 || MODE == 3), BMN = (MODE == 2 || MODE == 3), AMN = (MODE == 3);
+    // SwiGLU tiles are [gate 128 | up 128] weight rows.  When the last N tile has at most 64 real columns (I mod 128 in
+    // 1..64) it is loaded as [gate 64 | up 64] through a 64-row box and issued as an N = 128 MMA: half the tensor-pipe
+    // time and half the weight bytes for the same outputs.
+    const int last_cols = SWIGLU ? a.N - (n_nt - 1) * (BN / 2) : 0;
+    const bool narrow_last = SWIGLU && MODE == 0 && last_cols <= BN / 4;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -231,7 +237,8 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
                     const uint32_t sa = base + s * STAGE_BYTES, sb = sa + 2 * A_BYTES;
                     // GATHER: the gather warps bring A (forward layout), or in MODE 3 the operand a.gather_mn names
                     const bool gA = GATHER && (!AMN || a.gather_mn == 1), gB = GATHER && AMN && a.gather_mn == 2;
-                    mbar_expect_tx(full, (gB ? 0 : B_BYTES) + (gA ? 0 : (two ? 2 : 1) * A_BYTES));
+                    const bool narrow = narrow_last && t.n == n_nt - 1;
+                    mbar_expect_tx(full, (gB ? 0 : (narrow ? B_BYTES / 2 : B_BYTES)) + (gA ? 0 : (two ? 2 : 1) * A_BYTES));
                     if (AMN && !gA) {   // per half two boxes of 64 M-columns x 64 K-rows (K = rows of the dispatch space)
                         tma_load_2d(sa, &tmapA, full, t.row0, t.kcol0 + kb * BK);
                         tma_load_2d(sa + A_BYTES / 2, &tmapA, full, t.row0 + 64, t.kcol0 + kb * BK);
@@ -249,6 +256,9 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
 #pragma unroll
                         for (int q = 0; q < 4; ++q)
                             tma_load_2d(sb + q * (B_BYTES / 4), &tmapB, full, t.n * BN + q * 64, krow);
+                    } else if (narrow) {
+                        tma_load_2d(sb, &tmapB64, full, t.kcol0 + kb * BK, brow0);
+                        tma_load_2d(sb + B_BYTES / 4, &tmapB64, full, t.kcol0 + kb * BK, brow1);
                     } else {
                         tma_load_2d(sb, &tmapB, full, t.kcol0 + kb * BK, brow0);
                         tma_load_2d(sb + B_BYTES / 2, &tmapB, full, t.kcol0 + kb * BK, brow1);
@@ -279,6 +289,8 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
                 uint32_t idesc = IDESC_K;
                 if (!SWIGLU && a.N - t.n * BN < BN)
                     idesc = (IDESC_K & ~(0x3Fu << 17)) | ((uint32_t)(((a.N - t.n * BN + 15) & ~15) >> 3) << 17);
+                if (narrow_last && t.n == n_nt - 1)
+                    idesc = (IDESC_K & ~(0x3Fu << 17)) | ((uint32_t)((BN / 2) >> 3) << 17);
                 long long w0 = dbg ? clock64() : 0;
                 // Accumulator 0 is needed now, accumulator 1 only after the first k-block's MMAs into accumulator 0; and
                 // accumulator 0 is published before the last k-block's MMAs into accumulator 1 are issued.  Each
@@ -380,7 +392,9 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
         // ------------------------------------------------------------------ gather warps (pull dispatch)
         // Warp gw owns rows 32 gw .. 32 gw + 31 of each half; lane = (sub-row 0..3, 16-byte chunk 0..7); pass i of half
         // h covers row 128 h + 32 gw + 4 i + sub-row.  Chunk c of row r lands at r*128 + ((c ^ (r & 7)) * 16) inside
-        // its half.  Rows past the expert's segment re-read the tile's first row (computed, never combined).
+        // its half.  Rows past the expert's segment are written as zeros: their products are never combined, and zero
+        // operands cost the tensor pipe far less power than live ones (the board runs at its power cap, so power
+        // spent on padding is clock taken from the real rows).
         const int gw = warp - (2 + EPI_WARPS), sub = lane >> 3, chunk = lane & 7;
         int s = 0;
         uint32_t ph = 0;
@@ -449,13 +463,17 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
         for (int L = seq.first(); L < total; L = seq.next(L)) {
             const Tile t = decode_tile<KGROUP>(a, L, n_nt, n_mt_total, k_blocks);
             const bool two = t.valid > BM;
-            const int tok0 = __ldg(a.row_token + t.row0);
             const __nv_bfloat16* src[16];
+            uint32_t live = 0u;                                           // bit i: row i of this thread is a real row
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
                 const int r = (i >> 3) * BM + gw * 32 + (i & 7) * 4 + sub;
-                const int tok = (r < t.valid) ? __ldg(a.row_token + t.row0 + r) : tok0;
-                src[i] = gather_row(a, tok) + chunk * 8;
+                if (r < t.valid) {
+                    src[i] = gather_row(a, __ldg(a.row_token + t.row0 + r)) + chunk * 8;
+                    live |= 1u << i;
+                } else {
+                    src[i] = a.A;
+                }
             }
             bool ok = true;
             for (int kb = 0; kb < k_blocks; ++kb) {
@@ -469,7 +487,8 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
                     if (i < 8 || two) {
                         const int rr = gw * 32 + (i & 7) * 4 + sub;       // row inside the half
                         const uint32_t dst = sa + (i >> 3) * A_BYTES + rr * 128 + ((chunk ^ (rr & 7)) << 4);
-                        cp_async_16(dst, in_k ? (const void*)(src[i] + kb * BK) : (const void*)a.A, in_k ? 16u : 0u);
+                        const bool on = in_k && ((live >> i) & 1u);
+                        cp_async_16(dst, on ? (const void*)(src[i] + kb * BK) : (const void*)a.A, on ? 16u : 0u);
                     }
                 }
                 cp_async_mbar_arrive(smem_u32(&ctrl->full[s]));
@@ -490,7 +509,7 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
         for (int L = seq.first(); L < total; L = seq.next(L)) {
             const Tile t = decode_tile<KGROUP>(a, L, n_nt, n_mt_total, k_blocks);
             if ((KGROUP && t.kblocks == 0) || (acc == 1 && t.valid <= BM)) continue;   // no rows to contract / no second half
-            bool ok = mbar_wait(smem_u32(&ctrl->tfull[acc]), aph, abort_flag, a.header, 4);
+            bool ok = mbar_wait_long(smem_u32(&ctrl->tfull[acc]), aph, abort_flag, a.header, 4, a.wait_hint_ns);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             aph ^= 1u;
@@ -557,6 +576,9 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
                 // the slab that pass p is about to overwrite, so the accumulator goes back to the MMA issuer as soon as
                 // its last column has been read, not after the stores.
                 constexpr int PASSES = SWIGLU ? 2 : 4;
+                const bool narrow = narrow_last && t.n == n_nt - 1;      // [gate 64 | up 64]: one pass, up at column 64
+                const int passes = narrow ? 1 : PASSES;
+                const uint32_t up_off = narrow ? BN / 4 : BN / 2;
                 const int c0 = SWIGLU ? t.n * (BN / 2) : t.n * BN;
                 uint32_t cur[32], nxt[32];                    // one pass = 64 columns = 32 packed bf16 pairs per row
                 auto hand_back = [&]() {                       // the accumulator goes back to the MMA issuer
@@ -570,9 +592,9 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
                         if (SWIGLU) {
                             uint32_t g[32], u[32];
                             tc_ld32(taddr + pass * 64 + c, g);
-                            tc_ld32(taddr + BN / 2 + pass * 64 + c, u);
+                            tc_ld32(taddr + up_off + pass * 64 + c, u);
                             tc_wait_ld();
-                            if (pass == PASSES - 1 && c == 32) hand_back();   // the tile's last TMEM read: arithmetic comes after
+                            if (pass == passes - 1 && c == 32) hand_back();   // the tile's last TMEM read: arithmetic comes after
 #pragma unroll
                             for (int i = 0; i < 16; ++i)
                                 o[(c >> 1) + i] = pack_bf16(swiglu(__uint_as_float(g[2 * i]), __uint_as_float(u[2 * i])),
@@ -581,7 +603,7 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
                             uint32_t r[32];
                             tc_ld32(taddr + pass * 64 + c, r);
                             tc_wait_ld();
-                            if (pass == PASSES - 1 && c == 32) hand_back();
+                            if (pass == passes - 1 && c == 32) hand_back();
 #pragma unroll
                             for (int i = 0; i < 16; ++i)
                                 o[(c >> 1) + i] = pack_bf16(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
@@ -591,9 +613,10 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
                 load_pass(0, nxt);
 #pragma unroll
                 for (int pass = 0; pass < PASSES; ++pass) {
+                    if (pass >= passes) break;
 #pragma unroll
                     for (int i = 0; i < 32; ++i) cur[i] = nxt[i];
-                    if (pass + 1 < PASSES) {
+                    if (pass + 1 < passes) {
                         load_pass(pass + 1, nxt);
                     }
                     if (lane == 0) tma_store_wait_read();     // the slab's previous store has been read out
@@ -634,8 +657,8 @@ static bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t co
 }
 
 template <int EPI, bool GATHER, int MODE = 0, bool CLC = false>
-static cudaError_t launch_one(const CUtensorMap& mA, const CUtensorMap& mB, const CUtensorMap& mC, const GemmArgs& a,
-                              int n_nt, int k_blocks, int grid, cudaStream_t s) {
+static cudaError_t launch_one(const CUtensorMap& mA, const CUtensorMap& mB, const CUtensorMap& mC, const CUtensorMap& mB64,
+                              const GemmArgs& a, int n_nt, int k_blocks, int grid, cudaStream_t s) {
     static PerDevice configured;      // per device: SM count once this instantiation has its shared-memory opt-in there
     int dev = 0, sm_count = 0;
     cudaError_t e = current_device(&dev);
@@ -656,7 +679,7 @@ static cudaError_t launch_one(const CUtensorMap& mA, const CUtensorMap& mB, cons
         grid = sm_count;
     }
     gemm_m2_kernel<EPI, GATHER, MODE, CLC><<<grid, THREADS + (GATHER ? GATHER_THREADS : 0) + (CLC ? 32 : 0), SMEM_BYTES, s>>>(
-        mA, mB, mC, a, n_nt, k_blocks);
+        mA, mB, mC, mB64, a, n_nt, k_blocks);
     return cudaGetLastError();
 }
 
@@ -681,26 +704,29 @@ cudaError_t launch_gemm_m2(const GemmArgs& a, int epi, int grid, cudaStream_t s)
     else if (a.b_mn) {   // W viewed as [E * K, N], N contiguous: boxes of 64 columns x 64 rows
         if (!make_map(&mB, a.B, (uint64_t)a.E * a.K, (uint64_t)a.N, 64, (uint64_t)a.N)) return cudaErrorInvalidValue;
     } else if (!make_map(&mB, a.B, a.kgroup_rows > 0 ? (uint64_t)a.N : b_rows, (uint64_t)a.K, BN / 2, ldb)) return cudaErrorInvalidValue;
+    // the SwiGLU kernels' 64-row box over the same weights (narrow last N tile); a copy of mB where it is not used
+    CUtensorMap mB64 = mB;
+    if (swiglu && a.kgroup_rows == 0 && !a.b_mn && !make_map(&mB64, a.B, b_rows, (uint64_t)a.K, BN / 4, ldb)) return cudaErrorInvalidValue;
     if (epi == EPI_F32) mC = mB;      // the fp32 epilogue stores directly
     else if (!make_map(&mC, a.C, (uint64_t)a.rows_pad, (uint64_t)a.N, 32, (uint64_t)a.ldc)) return cudaErrorInvalidValue;
     const int n_nt = swiglu ? (a.N + BN / 2 - 1) / (BN / 2) : (a.N + BN - 1) / BN;
     const int k_blocks = (a.K + BK - 1) / BK;
-    if (a.kgroup_rows > 0 && a.b_mn && gather) return launch_one<EPI_BF16, true, 3>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
-    if (a.kgroup_rows > 0 && a.b_mn) return launch_one<EPI_BF16, false, 3>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
-    if (a.kgroup_rows > 0) return launch_one<EPI_BF16, false, 1>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
+    if (a.kgroup_rows > 0 && a.b_mn && gather) return launch_one<EPI_BF16, true, 3>(mA, mB, mC, mB64, a, n_nt, k_blocks, grid, s);
+    if (a.kgroup_rows > 0 && a.b_mn) return launch_one<EPI_BF16, false, 3>(mA, mB, mC, mB64, a, n_nt, k_blocks, grid, s);
+    if (a.kgroup_rows > 0) return launch_one<EPI_BF16, false, 1>(mA, mB, mC, mB64, a, n_nt, k_blocks, grid, s);
     if (a.b_mn) {
         if (epi != EPI_BF16) return cudaErrorInvalidValue;
-        return gather ? launch_one<EPI_BF16, true, 2>(mA, mB, mC, a, n_nt, k_blocks, grid, s)
-                      : launch_one<EPI_BF16, false, 2>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
+        return gather ? launch_one<EPI_BF16, true, 2>(mA, mB, mC, mB64, a, n_nt, k_blocks, grid, s)
+                      : launch_one<EPI_BF16, false, 2>(mA, mB, mC, mB64, a, n_nt, k_blocks, grid, s);
     }
     const bool stolen = a.tile_sched == 1 && a.dense_rows == 0;   // hardware tile stealing: routed forward GEMMs only
-    if (stolen && epi == EPI_SWIGLU && gather) return launch_one<EPI_SWIGLU, true, 0, true>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
-    if (stolen && epi == EPI_BF16 && !gather) return launch_one<EPI_BF16, false, 0, true>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
-    if (epi == EPI_SWIGLU && gather) return launch_one<EPI_SWIGLU, true>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
-    if (epi == EPI_SWIGLU) return launch_one<EPI_SWIGLU, false>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
-    if (epi == EPI_BF16 && !gather) return launch_one<EPI_BF16, false>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
-    if (epi == EPI_BF16) return launch_one<EPI_BF16, true>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
-    if (epi == EPI_F32 && !gather) return launch_one<EPI_F32, false>(mA, mB, mC, a, n_nt, k_blocks, grid, s);
+    if (stolen && epi == EPI_SWIGLU && gather) return launch_one<EPI_SWIGLU, true, 0, true>(mA, mB, mC, mB64, a, n_nt, k_blocks, grid, s);
+    if (stolen && epi == EPI_BF16 && !gather) return launch_one<EPI_BF16, false, 0, true>(mA, mB, mC, mB64, a, n_nt, k_blocks, grid, s);
+    if (epi == EPI_SWIGLU && gather) return launch_one<EPI_SWIGLU, true>(mA, mB, mC, mB64, a, n_nt, k_blocks, grid, s);
+    if (epi == EPI_SWIGLU) return launch_one<EPI_SWIGLU, false>(mA, mB, mC, mB64, a, n_nt, k_blocks, grid, s);
+    if (epi == EPI_BF16 && !gather) return launch_one<EPI_BF16, false>(mA, mB, mC, mB64, a, n_nt, k_blocks, grid, s);
+    if (epi == EPI_BF16) return launch_one<EPI_BF16, true>(mA, mB, mC, mB64, a, n_nt, k_blocks, grid, s);
+    if (epi == EPI_F32 && !gather) return launch_one<EPI_F32, false>(mA, mB, mC, mB64, a, n_nt, k_blocks, grid, s);
     return cudaErrorInvalidValue;
 }
 

@@ -4,6 +4,7 @@
 // mok_moe_forward_host, which say so.
 #include "mok_internal.cuh"
 #include <string.h>
+#include <stdlib.h>
 
 namespace mok {
 
@@ -111,6 +112,7 @@ static int validate(const mok_args* a, WsLayout* L, size_t extra_ws) {
     } else if (!a->W_gate_up || !a->W_down) {
         return MOK_ERR_NULL;
     }
+    if (!aligned16(a->W_router_split)) return MOK_ERR_ALIGN;
     if (!aligned16(a->W_router) || !aligned16(a->W_gate_up) || !aligned16(a->W_down) ||
         !aligned16(a->W_shared_gate_up) || !aligned16(a->W_shared_down))
         return MOK_ERR_ALIGN;
@@ -178,6 +180,11 @@ static bool use_m2(const mok_config* cfg, int K, int tile_m, long long rows, int
 
 int run_gemm(GemmArgs g, bool swiglu, const mok_config* cfg, const WsLayout& L, char* ws, cudaStream_t s) {
     const int epi = swiglu ? EPI_SWIGLU : EPI_BF16, grid = cfg ? cfg->grid : 0;
+    {
+        static int hint = -1;
+        if (hint < 0) { const char* v = getenv("MOK_WAIT_HINT_NS"); hint = v ? atoi(v) : 0; }
+        g.wait_hint_ns = (uint32_t)hint;
+    }
     if (use_m2(cfg, g.K, g.tile_m, g.dense_rows > 0 ? g.dense_rows : g.total_rows, g.dense_rows > 0 ? 1 : g.E)) {
         WsHeader* hdr = reinterpret_cast<WsHeader*>(ws + L.header);
         g.n_mtiles = &hdr->n_mtiles2;
@@ -202,7 +209,8 @@ static int route_stage(const mok_args* a, const WsLayout& L, char* ws, const __n
                              reinterpret_cast<WsHeader*>(ws + L.header), a->config ? a->config->grid : 0,
                              tile_rows(a->config, a->I > 0 ? a->I : 8),
                              use_tn(a->config) ? 2 : use_m2(a->config, a->H, tile_rows(a->config, a->I > 0 ? a->I : 8), a->T, 1) ? 3 : 0,
-                             use_fused_router(a->config, a->E, a->k), idx, w, s);
+                             use_fused_router(a->config, a->E, a->k), idx, w, s,
+                             reinterpret_cast<const __nv_bfloat16*>(a->W_router_split));
     if (e != cudaSuccess) return cuda_fail(e);
     if (a->topk_idx) {
         e = cudaMemcpyAsync(a->topk_idx, idx, sizeof(int32_t) * (size_t)L.R, cudaMemcpyDeviceToDevice, s);
@@ -412,6 +420,27 @@ int mok_mx_quantize_rows(const void* x, int rows, int K, void* codes, void* scal
 size_t mok_workspace_bytes(int T, int H, int I, int I_shared, int E, int k) {
     WsLayout L;
     return ws_layout(T, H, I, I_shared, E, k, &L) ? L.total : 0;
+}
+
+size_t mok_router_prepared_bytes(int E, int H) {
+    if (E <= 0 || E > MAX_E || H <= 0 || (H % 8)) return 0;
+    return align_up(2 * (size_t)3 * ((E + 31) / 32 * 32) * H, 256);      // either layout fits: 3 * E rows rounded up
+}
+
+int mok_router_prepare(const float* W_router, int E, int H, int k, const mok_config* config, void* out, size_t out_bytes,
+                       void* stream) {
+    if (!W_router || !out) return MOK_ERR_NULL;
+    const size_t need = mok_router_prepared_bytes(E, H);
+    if (need == 0 || k < 1 || k > E || k > MAX_K) return MOK_ERR_SHAPE;
+    if (use_simt_router(config, k)) return MOK_ERR_UNSUPPORTED;        // the fp32-FMA router reads W_router itself
+    if (!aligned16(W_router) || !aligned16(out)) return MOK_ERR_ALIGN;
+    if (out_bytes < need) return MOK_ERR_WORKSPACE;
+    WsLayout L;
+    memset(&L, 0, sizeof(L));
+    cudaError_t e = launch_router_tc(nullptr, W_router, nullptr, 0, H, E, k, L, nullptr, nullptr, 0, TILE_M, 0,
+                                     use_fused_router(config, E, k), nullptr, nullptr,
+                                     reinterpret_cast<cudaStream_t>(stream), reinterpret_cast<const __nv_bfloat16*>(out), true);
+    return e == cudaSuccess ? MOK_OK : cuda_fail(e);
 }
 
 int mok_moe_forward_ex(const mok_args* a) {
@@ -707,6 +736,7 @@ int mok_launch_count(int T, int H, int I, int I_shared, int E, int k, const mok_
     // 2 routed GEMMs, (2 shared GEMMs), combine
     // (MXFP8 mode: the token-row quantiser instead of the gather kernel; its two memsets are not counted)
     const int pre = use_mx(config) ? 1 : (fused_gather(config, I) ? 0 : 1);
+    // (with mok_args.W_router_split the router's split kernel is not launched: one launch less than counted here)
     return (use_simt_router(config, k) ? 1 : use_fused_router(config, E, k) ? 3 : 4) + 3 + pre + 2 + (I_shared > 0 ? 2 : 0) + 1;
 }
 

@@ -79,6 +79,7 @@ struct GemmArgs {
     int32_t dbg_slot;            // >= 0: accumulate wait-time counters into header->dbg[dbg_slot]
     int32_t starve;              // test hook: the TMA producer issues nothing, so the kernel's waits run out
     int32_t tile_sched;          // 256-row kernel, routed forward GEMMs: 1 = tiles handed out by cluster launch control
+    uint32_t wait_hint_ns;       // 256-row kernel: suspend-time hint of the roles that wait long (0 = plain polling)
     // K-range mode of the 256-row kernel (weight gradients): C holds E matrices [kgroup_rows, N]; A is ONE matrix
     // [kgroup_rows, K extent] and B ONE matrix [N, K extent] whose columns are the rows of the dispatch space; expert e
     // contracts over its padded segment [pad_offsets[e], pad_offsets[e+1]) (dense_rows > 0: one group over columns
@@ -142,7 +143,8 @@ cudaError_t launch_mx_quantize_atoms(const __nv_bfloat16* in, int groups, int ro
                                      uint8_t* scales, cudaStream_t s);
 cudaError_t launch_router_tc(const __nv_bfloat16* x, const float* Wr, const float* bias, int T, int H, int E, int k,
                              const WsLayout& L, char* ws, WsHeader* hdr, int grid, int tile_m, int variant, bool fused,
-                             int32_t* idx, float* w, cudaStream_t s);
+                             int32_t* idx, float* w, cudaStream_t s, const __nv_bfloat16* presplit = nullptr,
+                             bool split_only = false);
 bool router_fused_ok(int E, int k);     // the one-kernel projection + top-k serves this shape
 cudaError_t launch_router_fused(const __nv_bfloat16* x, const __nv_bfloat16* split, const float* bias, int T, int H, int E,
                                 int k, float* rows, int32_t* flagged, WsHeader* hdr, int grid, int32_t* idx, float* w,

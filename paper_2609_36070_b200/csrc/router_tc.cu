@@ -22,7 +22,7 @@ namespace mok {
 __global__ void __launch_bounds__(256)
 router_split_kernel(const float* __restrict__ Wr, int E, int estride, int H, int rows, __nv_bfloat16* __restrict__ out,
                     WsHeader* hdr) {
-    if (blockIdx.x == 0 && threadIdx.x == 0) hdr->n_flag = 0;   // the near-tie list of this call starts empty
+    if (hdr && blockIdx.x == 0 && threadIdx.x == 0) hdr->n_flag = 0;   // the near-tie list of this call starts empty
     const size_t n = (size_t)rows * H;
     for (size_t i = (size_t)blockIdx.x * 256 + threadIdx.x; i < n; i += (size_t)gridDim.x * 256) {
         const int row = (int)(i / H), h = (int)(i - (size_t)row * H);
@@ -243,21 +243,30 @@ static cudaError_t launch_topk(const float* part, const float* bias, const __nv_
 
 cudaError_t launch_router_tc(const __nv_bfloat16* x, const float* Wr, const float* bias, int T, int H, int E, int k,
                              const WsLayout& L, char* ws, WsHeader* hdr, int grid, int tile_m, int variant, bool fused,
-                             int32_t* idx, float* w, cudaStream_t s) {
+                             int32_t* idx, float* w, cudaStream_t s, const __nv_bfloat16* presplit, bool split_only) {
     fused = fused && router_fused_ok(E, k);
     const int ep = (E + 31) / 32 * 32;
     const int ldl = fused ? ep : (3 * E + 7) / 8 * 8;       // row stride of the logits buffer
     const int split_rows = fused ? 3 * ep : ldl;
-    __nv_bfloat16* split = reinterpret_cast<__nv_bfloat16*>(ws + L.wr_split);
+    // W_r is a weight: its split can be made once (mok_router_prepare) and handed in, or is made here on every call
+    const __nv_bfloat16* split = presplit && !split_only ? presplit : reinterpret_cast<const __nv_bfloat16*>(ws + L.wr_split);
     float* part = reinterpret_cast<float*>(ws + L.logits);
     // the near-tie list lives in the schedule's `perm` region (T*k entries), which is not written before the schedule runs
     int32_t* flagged = reinterpret_cast<int32_t*>(ws + L.perm);
     size_t n = (size_t)split_rows * H;
     int blocks = (int)((n + 255) / 256);
     if (blocks > 148 * 8) blocks = 148 * 8;
-    router_split_kernel<<<blocks, 256, 0, s>>>(Wr, E, fused ? ep : E, H, split_rows, split, hdr);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
+    cudaError_t e = cudaSuccess;
+    if (split_only) {     // mok_router_prepare: `presplit` is the destination, no workspace is involved
+        router_split_kernel<<<blocks, 256, 0, s>>>(Wr, E, fused ? ep : E, H, split_rows, const_cast<__nv_bfloat16*>(presplit), nullptr);
+        return cudaGetLastError();
+    }
+    if (!presplit) {
+        router_split_kernel<<<blocks, 256, 0, s>>>(Wr, E, fused ? ep : E, H, split_rows,
+                                                   reinterpret_cast<__nv_bfloat16*>(ws + L.wr_split), hdr);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
     if (fused) {
         e = launch_router_fused(x, split, bias, T, H, E, k, part, flagged, hdr, grid, idx, w, s);
     } else {

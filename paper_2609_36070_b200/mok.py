@@ -25,7 +25,8 @@ EXPORTS = ["mok_moe_forward", "mok_workspace_bytes", "mok_moe_forward_ex", "mok_
            "mok_version", "mok_profile_begin", "mok_profile_end", "mok_schedule_noalloc", "mok_debug_counters",
            "mok_ep_workspace_bytes", "mok_ep_y_rows", "mok_ep_expert_ffn", "mok_ep_combine",
            "mok_mx_scale_bytes", "mok_mx_quantize_weights", "mok_mx_quantize_rows", "mok_mx_workspace_bytes",
-           "mok_ep_mx_workspace_bytes", "mok_bwd_workspace_bytes", "mok_moe_backward", "mok_selftest_per_device"]
+           "mok_ep_mx_workspace_bytes", "mok_bwd_workspace_bytes", "mok_moe_backward", "mok_selftest_per_device",
+           "mok_router_prepared_bytes", "mok_router_prepare"]
 MOK_PRECISION_BF16, MOK_PRECISION_MXFP8 = 0, 1
 MOK_MAX_RANKS = 16
 MOK_NOALLOC_MAX_ROUTES = 32768
@@ -51,7 +52,8 @@ class mok_args(ctypes.Structure):
                 ("offsets", ctypes.c_void_p), ("perm", ctypes.c_void_p), ("inv_perm", ctypes.c_void_p),
                 ("config", ctypes.POINTER(mok_config)), ("stream", ctypes.c_void_p),
                 ("W_gate_up_codes", ctypes.c_void_p), ("W_gate_up_scales", ctypes.c_void_p),
-                ("W_down_codes", ctypes.c_void_p), ("W_down_scales", ctypes.c_void_p)]
+                ("W_down_codes", ctypes.c_void_p), ("W_down_scales", ctypes.c_void_p),
+                ("W_router_split", ctypes.c_void_p)]
 
 
 class mok_ep_args(ctypes.Structure):
@@ -144,6 +146,11 @@ _lib.mok_last_cuda_error.restype = ctypes.c_int
 _lib.mok_status_string.restype = ctypes.c_char_p
 _lib.mok_status_string.argtypes = [ctypes.c_int]
 _lib.mok_version.restype = ctypes.c_int
+_lib.mok_router_prepared_bytes.restype = ctypes.c_size_t
+_lib.mok_router_prepared_bytes.argtypes = [ctypes.c_int] * 2
+_lib.mok_router_prepare.restype = ctypes.c_int
+_lib.mok_router_prepare.argtypes = ([ctypes.c_void_p] + [ctypes.c_int] * 3 + [ctypes.POINTER(mok_config), ctypes.c_void_p,
+                                    ctypes.c_size_t, ctypes.c_void_p])
 _lib.mok_selftest_per_device.restype = ctypes.c_int
 _lib.mok_selftest_per_device.argtypes = []
 _lib.mok_profile_begin.restype = ctypes.c_int
@@ -319,8 +326,20 @@ def _fill_args(x_shape, W_router, router_bias, W_gate_up, W_down, W_shared_gate_
     return a, res
 
 
+def mok_router_prepare(W_router, k, config=None, stream=None):
+    """The exact three-way bf16 split of W_router, made once; pass the result as router_split= to the forward calls."""
+    E, H = W_router.shape
+    n = int(_lib.mok_router_prepared_bytes(E, H))
+    if n == 0:
+        raise MokError(MOK_ERR_SHAPE)
+    out = torch.empty(n, dtype=torch.uint8, device=W_router.device)
+    _check(_lib.mok_router_prepare(_p(W_router), E, H, k, None if config is None else ctypes.pointer(config), _p(out), n,
+                                   _stream(stream)))
+    return out
+
+
 def mok_moe_forward_ex(x, W_router, router_bias, W_gate_up, W_down, W_shared_gate_up, W_shared_down, k, workspace,
-                       out=None, stages=False, config=None, stream=None, mx_weights=None):
+                       out=None, stages=False, config=None, stream=None, mx_weights=None, router_split=None):
     """The layer with router bias, caller-owned workspace, optional stage outputs and knobs.
 
     Returns out, or (out, dict of stage tensors) when stages=True.
@@ -330,6 +349,8 @@ def mok_moe_forward_ex(x, W_router, router_bias, W_gate_up, W_down, W_shared_gat
     a, res = _fill_args(x.shape, W_router, router_bias, W_gate_up, W_down, W_shared_gate_up, W_shared_down, k,
                         workspace, stages, config, stream, x.device)
     a.x, a.out = x.data_ptr(), out.data_ptr()
+    if router_split is not None:
+        a.W_router_split = router_split.data_ptr()
     if mx_weights is not None:
         a.W_gate_up_codes, a.W_gate_up_scales = mx_weights.gate_up_codes.data_ptr(), mx_weights.gate_up_scales.data_ptr()
         a.W_down_codes, a.W_down_scales = mx_weights.down_codes.data_ptr(), mx_weights.down_scales.data_ptr()

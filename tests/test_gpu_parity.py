@@ -103,6 +103,34 @@ def test_one_kernel_router_against_oracle_and_three_kernel_router(cfg):
     assert torch.equal(st["topk_w"].view(torch.int32), stg["topk_w"].view(torch.int32))
 
 
+@pytest.mark.parametrize("name,router_impl", [("r_e128", 0), ("r_e128", 2), ("r_e161", 0), ("r_e6", 0)])
+def test_router_weights_prepared_once_give_the_same_bits(name, router_impl):
+    """mok_router_prepare splits W_router once; forward calls that are handed the split skip their own split kernel and
+    must produce the same routing and output bits, for the one-kernel and the three-kernel layout of the split."""
+    m = mok()
+    cfg = next(c for c in ROUTER_SHAPES if c.name == name)
+    d = inputs.make_inputs(cfg)
+    g = pu.upload(d)
+    conf = m._config(router_impl=router_impl)
+    out, st = pu.run_gpu(cfg, g, config=conf)
+    split = m.mok_router_prepare(g["W_r"], cfg.k, conf)
+    ws = m.alloc_workspace(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k)
+    ws.zero_()                                                   # the workspace's own split region stays empty
+    out2, st2 = m.mok_moe_forward_ex(g["x"], g["W_r"], g["bias"], g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], cfg.k,
+                                     ws, stages=True, config=conf, router_split=split)
+    assert m.mok_read_status(ws) == 0
+    assert torch.equal(st["topk_idx"], st2["topk_idx"])
+    assert torch.equal(st["topk_w"].view(torch.int32), st2["topk_w"].view(torch.int32))
+    assert torch.equal(out.view(torch.int16), out2.view(torch.int16))
+    # a second call with the same prepared split (the near-tie list must start empty each time)
+    out3, st3 = m.mok_moe_forward_ex(g["x"], g["W_r"], g["bias"], g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], cfg.k,
+                                     ws, stages=True, config=conf, router_split=split)
+    assert torch.equal(st["topk_idx"], st3["topk_idx"]) and torch.equal(out.view(torch.int16), out3.view(torch.int16))
+    with pytest.raises(m.MokError) as ei:                        # the fp32-FMA router has no split
+        m.mok_router_prepare(g["W_r"], cfg.k, m._config(router_impl=1))
+    assert ei.value.status == m.MOK_ERR_UNSUPPORTED
+
+
 def test_one_kernel_router_lists_near_ties_for_the_exact_fix_up():
     """Duplicate expert rows give exact ties and rows that differ in the last bit give logits closer than the tensor
     cores' accumulation error: both must come out as the oracle decides them (lowest id first on exact ties)."""
