@@ -57,6 +57,8 @@ def parse():
     p.add_argument("--no-sweep", action="store_true", help="skip the small-T sweep of the default workload")
     p.add_argument("--no-e2e", action="store_true", help="skip the host-buffer (end-to-end) legs")
     p.add_argument("--no-counters", action="store_true", help="skip the device-side counter pass")
+    p.add_argument("--cooldown", type=float, default=2.0,
+                   help="idle seconds before each workload's warm-up, so that every workload starts from the same board state")
     p.add_argument("--sustain-seconds", type=float, default=2.0,
                    help="length of the extra loop that shows the power-capped steady state (0 = skip)")
     p.add_argument("--gather-mode", type=int, default=0, help="0 auto, 1 fused into the GEMM, 2 separate kernel")
@@ -384,7 +386,8 @@ class Layer:
         if second_half:
             stage = stage[len(stage) // 2:]
             t0 = 0.5 * (t0 + t1)
-        res = {s: (sum(c[s] for c in stage) / len(stage), _median([c[s] for c in stage])) for s in mok.STAGES}
+        res = {s: (sum(c[s] for c in stage) / len(stage), _median([c[s] for c in stage]), min(c[s] for c in stage))
+               for s in mok.STAGES}
         return res, (t0, t1)
 
     def counters(self):
@@ -431,6 +434,9 @@ def measure(layer, steps, warmup, barrier, sampler_windows, pk, with_counters):
     the sampler has been stopped; `sampler_windows` collects (record, key, window) for that."""
     cfg, mok = layer.cfg, layer.mok
     conf = layer.conf()
+    if layer.args.cooldown > 0:
+        layer.torch.cuda.synchronize()
+        time.sleep(layer.args.cooldown)
     for _ in range(warmup):
         layer.step(conf)
     barrier()
@@ -442,7 +448,8 @@ def measure(layer, steps, warmup, barrier, sampler_windows, pk, with_counters):
     layer.check_status()
     rec = {"ms_per_step": _median(per_step), "mean_ms_per_step": total_ms / steps, "min_ms_per_step": min(per_step),
            "steps": steps, "stage_ms": {s: stages[s][1] for s in mok.STAGES},
-           "stage_ms_mean": {s: stages[s][0] for s in mok.STAGES}, "_region_s": total_ms * 1e-3,
+           "stage_ms_mean": {s: stages[s][0] for s in mok.STAGES}, "stage_ms_min": {s: stages[s][2] for s in mok.STAGES},
+           "_region_s": total_ms * 1e-3,
            "_stage_region_s": swin[1] - swin[0]}
     sampler_windows.append((rec, "clocks", win))
     sampler_windows.append((rec, "clocks_stage_loop", swin))
@@ -480,6 +487,10 @@ def finish_record(rec, cfg, pk, mx, world=1):
     clk = rec.get("clocks_stage_loop") or {}
     dom = roofline_fracs(g1_tf, pk, mx, rec.pop("_stage_region_s"), clk)
     dom["ms"] = st["gemm1"]
+    # the fastest single launch of the loop against the burst peak (itself the best of ten single launches)
+    best = rec.pop("stage_ms_min")["gemm1"]
+    dom["best_launch_ms"] = best
+    dom["best_launch_frac_of_burst"] = g1_flops / (best * 1e-3) / 1e12 / (scale * pk["bf16_tflops"])
     if clk.get("sm_mhz"):
         dom["sm_cycles"] = st["gemm1"] * 1e-3 * clk["sm_mhz"] * 1e6       # kernel time x median sampled SM clock
     if "counters" in rec and "gemm1" in rec["counters"]:
@@ -640,6 +651,7 @@ def main():
             rec.pop("_region_s", None)
             rec.pop("_stage_region_s", None)
             rec.pop("stage_ms_mean", None)
+            rec.pop("stage_ms_min", None)
             sweep.append(rec)
             del st
 

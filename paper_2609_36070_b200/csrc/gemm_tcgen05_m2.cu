@@ -465,15 +465,17 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
             const bool two = t.valid > BM;
             const __nv_bfloat16* src[16];
             uint32_t live = 0u;                                           // bit i: row i of this thread is a real row
+            int tok[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {   // sixteen independent loads (a pad row reads the tile's last real row id)
+                const int r = (i >> 3) * BM + gw * 32 + (i & 7) * 4 + sub;
+                tok[i] = __ldg(a.row_token + t.row0 + min(r, t.valid - 1));
+            }
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
                 const int r = (i >> 3) * BM + gw * 32 + (i & 7) * 4 + sub;
-                if (r < t.valid) {
-                    src[i] = gather_row(a, __ldg(a.row_token + t.row0 + r)) + chunk * 8;
-                    live |= 1u << i;
-                } else {
-                    src[i] = a.A;
-                }
+                src[i] = gather_row(a, tok[i]) + chunk * 8;
+                if (r < t.valid) live |= 1u << i;
             }
             bool ok = true;
             for (int kb = 0; kb < k_blocks; ++kb) {
@@ -509,7 +511,7 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
         for (int L = seq.first(); L < total; L = seq.next(L)) {
             const Tile t = decode_tile<KGROUP>(a, L, n_nt, n_mt_total, k_blocks);
             if ((KGROUP && t.kblocks == 0) || (acc == 1 && t.valid <= BM)) continue;   // no rows to contract / no second half
-            bool ok = mbar_wait_long(smem_u32(&ctrl->tfull[acc]), aph, abort_flag, a.header, 4, a.wait_hint_ns);
+            bool ok = mbar_wait(smem_u32(&ctrl->tfull[acc]), aph, abort_flag, a.header, 4);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             aph ^= 1u;

@@ -4,7 +4,6 @@
 // mok_moe_forward_host, which say so.
 #include "mok_internal.cuh"
 #include <string.h>
-#include <stdlib.h>
 
 namespace mok {
 
@@ -180,11 +179,6 @@ static bool use_m2(const mok_config* cfg, int K, int tile_m, long long rows, int
 
 int run_gemm(GemmArgs g, bool swiglu, const mok_config* cfg, const WsLayout& L, char* ws, cudaStream_t s) {
     const int epi = swiglu ? EPI_SWIGLU : EPI_BF16, grid = cfg ? cfg->grid : 0;
-    {
-        static int hint = -1;
-        if (hint < 0) { const char* v = getenv("MOK_WAIT_HINT_NS"); hint = v ? atoi(v) : 0; }
-        g.wait_hint_ns = (uint32_t)hint;
-    }
     if (use_m2(cfg, g.K, g.tile_m, g.dense_rows > 0 ? g.dense_rows : g.total_rows, g.dense_rows > 0 ? 1 : g.E)) {
         WsHeader* hdr = reinterpret_cast<WsHeader*>(ws + L.header);
         g.n_mtiles = &hdr->n_mtiles2;

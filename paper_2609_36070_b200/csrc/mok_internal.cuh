@@ -79,7 +79,6 @@ struct GemmArgs {
     int32_t dbg_slot;            // >= 0: accumulate wait-time counters into header->dbg[dbg_slot]
     int32_t starve;              // test hook: the TMA producer issues nothing, so the kernel's waits run out
     int32_t tile_sched;          // 256-row kernel, routed forward GEMMs: 1 = tiles handed out by cluster launch control
-    uint32_t wait_hint_ns;       // 256-row kernel: suspend-time hint of the roles that wait long (0 = plain polling)
     // K-range mode of the 256-row kernel (weight gradients): C holds E matrices [kgroup_rows, N]; A is ONE matrix
     // [kgroup_rows, K extent] and B ONE matrix [N, K extent] whose columns are the rows of the dispatch space; expert e
     // contracts over its padded segment [pad_offsets[e], pad_offsets[e+1]) (dense_rows > 0: one group over columns

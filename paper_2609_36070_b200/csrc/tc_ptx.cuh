@@ -48,18 +48,6 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// The same test with a suspend-time hint: the thread may sleep inside the instruction for up to `ns` nanoseconds and is
-// woken when the phase completes, so a role that waits for a long time (an epilogue warp during a tile's k-loop)
-// polls far less often.
-__device__ __forceinline__ bool mbar_try_wait_hint(uint32_t bar, uint32_t parity, uint32_t ns) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity), "r"(ns) : "memory");
-    return ok != 0;
-}
 // Bounded wait.  Returns false if the CTA is aborting (this or another thread ran out of time).
 static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
                                             WsHeader* hdr, int site) {
@@ -83,27 +71,6 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
                                           WsHeader* hdr, int site) {
     if (mbar_try_wait(bar, parity)) return true;
     return mbar_wait_slow(bar, parity, abort_flag, hdr, site);
-}
-// Bounded wait of a role that expects to wait long: polls with a suspend-time hint (hint_ns > 0).
-static __device__ __noinline__ bool mbar_wait_long(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                                   WsHeader* hdr, int site, uint32_t hint_ns) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if (hint_ns == 0) return mbar_wait_slow(bar, parity, abort_flag, hdr, site);
-    const unsigned long long t0 = globaltimer();
-    uint32_t spins = 0;
-    while (!mbar_try_wait_hint(bar, parity, hint_ns)) {
-        if ((++spins & 15u) == 0u) {
-            if (*abort_flag) return false;
-            const unsigned long long limit = hdr->wait_limit_us ? 1000ull * hdr->wait_limit_us : WAIT_LIMIT_NS;
-            if (globaltimer() - t0 > limit) {
-                *abort_flag = 1u;
-                atomicCAS(&hdr->status, 0, (int)MOK_ERR_TIMEOUT);
-                hdr->where = site;
-                return false;
-            }
-        }
-    }
-    return true;
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
