@@ -87,13 +87,23 @@ typedef struct mok_config {
                              work stealing).  The hardware refuses the request while work of a higher stream priority
                              waits for an SM; the CTA then leaves and the tiles nobody stole start as CTAs of their own
                              afterwards, so such work gets onto the SMs at the next tile boundary instead of at the end
-                             of the kernel.  Same bits either way. */
+                             of the kernel.  Same bits either way.  2 = only with fused_ffn: static stride over the
+                             one-launch tile list instead of the dynamic draw. */
     int32_t macrobatch_tokens; /* mok_moe_forward_ex: > 0 and < T: the tokens pass through the workspace in macrobatches of
                              this many tokens, one after the other (Section 3.3: a fixed-size buffer through which the
                              tokens cycle, instead of buffers sized for the whole batch).  The workspace then only needs
                              mok_workspace_bytes(macrobatch_tokens, ...); every macrobatch streams the expert weights
                              again.  Same bits as the single pass; counts / offsets / perm / inv_perm (tables of ONE
                              schedule) cannot be returned: MOK_ERR_UNSUPPORTED. */
+    int32_t fused_ffn;    /* routed experts, bf16: 0 = choose by shape, 1 = gate/up GEMM and down GEMM as two launches,
+                             2 = ONE persistent launch over a list of gate/up tiles and down tiles; a down tile runs
+                             once a per-row-tile completion counter, advanced by the gate/up epilogues, shows that its
+                             rows of the gated activation exist (Section 3.2: megakernel, GPU-local synchronisation
+                             instead of kernel boundaries).  Same bits either way. */
+    int32_t fused_window; /* fused_ffn: list positions between a row group's gate/up tiles and its down tiles (0 = two
+                             grids' worth of tiles; -1 = none: directly behind them, which makes every down tile wait --
+                             a test setting).  The list is handed out dynamically (each CTA draws the next position
+                             from a global counter) unless tile_sched = 2, which walks it with stride grid. */
 } mok_config;
 
 /*
@@ -392,7 +402,9 @@ int mok_profile_end(float* ms, int max_calls_out, int* n_calls);
 /*
  * Counters of the tcgen05 GEMM kernels of the last forward call that ran with config.debug != 0 (measurement aid;
  * Section 3 cost model: T_comp against T_sync).  Synchronises `stream`, then writes 4 x MOK_DEBUG_COUNTERS values:
- * slot 1 = routed gate/up GEMM, 2 = routed down GEMM, 3 = shared GEMMs.  Per slot, SM cycles summed over CTAs:
+ * slot 1 = routed gate/up GEMM, 2 = routed down GEMM, 3 = shared GEMMs (with config.fused_ffn the routed GEMMs are one
+ * launch: slots 1 and 2 hold its gate/up tiles and its down tiles, [5] of slot 2 the time its producers waited for
+ * gate/up tiles to complete, and slot 0 the whole kernel: [3], [8], [9], [11]).  Per slot, SM cycles summed over CTAs:
  * [0] MMA issuer waiting for operands, [1] for the peer CTA's operands, [2] for a free accumulator; [3] MMA issuer
  * total; [4] k-blocks issued (in 128-row units); [5] TMA producer waiting for a free stage; [6] epilogue waiting for an
  * accumulator; [7] epilogue total; then [8] the busiest CTA's MMA-issuer total (cycles, maximum over CTAs: [8] against

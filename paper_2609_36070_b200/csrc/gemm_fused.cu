@@ -1,0 +1,730 @@
+// Routed expert FFN in ONE persistent launch: gate/up grouped GEMM + SwiGLU and the down grouped GEMM of the same rows
+// (paper, Section 3.2 "Megakernel": the stages of an expert's FFN run depth-first inside one kernel and synchronise
+// through GPU-local completion counters instead of kernel boundaries; Figure 1, left).
+//
+// The work is ONE list of 256-row tiles of two kinds:
+//   G  gate/up tile: rows gathered from x through the schedule (pull dispatch, Section 3.1), weights [gate 128 | up 128]
+//      by TMA, K = H; epilogue silu(g) * u -> h (bf16, TMA store), then the epilogue warps wait until their stores have
+//      completed and add one arrival each to ready[M tile]
+//   D  down tile: h rows and W_down by TMA, K = I; epilogue -> y (bf16, TMA store).  Its producer first waits until
+//      ready[M tile] shows every gate/up tile of those rows (bounded wait; a time-out reports MOK_ERR_TIMEOUT)
+// The list is built on the device by fused_tiles_kernel from the schedule's per-expert tables: M tiles are grouped
+// (eight per group, one expert per group) and a group's tiles are laid out [N tile][M tile] so that CTAs working side
+// by side share a weight tile in L2.  A group's D tiles are placed `window` M tiles behind its G tiles: with the
+// persistent grid walking the list in order (tile L -> CTA L mod grid), the gate/up tiles a down tile depends on are
+// then normally complete when its producer asks, and h is consumed while it is still in L2.
+//
+// No deadlock: every tile a D tile depends on has a smaller list index; a CTA works through its tiles in increasing
+// order; the launch is cooperative, so all CTAs of the grid are resident.  Take the unfinished tile with the smallest
+// index: everything it waits for is finished, so it makes progress.
+//
+// Two ways of handing out the list.  STATIC: tile L -> CTA L mod grid (cooperative launch: every CTA resident).  Gate/up
+// and down tiles differ in length (K = H against K = I), so CTAs drift apart along the list and down tiles do wait.
+// DYNAMIC: a scheduler warp per CTA draws the next list position from one global counter (a plain atomic add, a few
+// tiles ahead of the CTA's other roles, which read the ids from a small queue in shared memory), so a CTA that got
+// short tiles simply draws more of them and all CTAs stay within about one tile of each other.  The argument above
+// holds unchanged: whoever drew a position runs, and everything it waits for was drawn earlier.
+// (Tried and dropped: two draw counters with "the next down tile if its rows are complete, else a gate/up tile",
+// claimed by compare-and-swap so that a claimed down tile never waits.  Correct, but a compare-and-swap chain hands
+// out about one tile per L2 round trip for the whole GPU, an order of magnitude below the ~7 tiles per microsecond the
+// grid consumes: the layer ran three times slower.)
+//
+// Determinism: every output element is still produced by exactly one tile with a fixed k order, so the bits equal
+// those of the two separate launches whatever the interleaving (tested).
+//
+// Warp roles, shared-memory ring, tensor-memory use and the epilogue are those of gemm_tcgen05_m2.cu; during D tiles
+// the gather warps only keep the ring's arrival counts complete.
+#include "mok_internal.cuh"
+#include "tc_ptx.cuh"
+#include "tensor_map.cuh"
+
+namespace mok {
+namespace ff {
+
+using namespace tc;
+
+constexpr int BM = 128, BN = 256, BK = 64, UMMA_K = 16, STAGES = 3;
+constexpr int A_BYTES = BM * BK * 2;
+constexpr int B_BYTES = BN * BK * 2;
+constexpr int STAGE_BYTES = 2 * A_BYTES + B_BYTES;
+constexpr int TM = 2 * BM;
+constexpr int TMEM_COLS = 512;
+constexpr int EPI_WARPS = 8;
+constexpr int GATHER_THREADS = 128;
+constexpr int THREADS = 64 + 32 * EPI_WARPS + GATHER_THREADS;     // 448
+constexpr int GROUP_TILES = 8;
+constexpr int SLAB_BYTES = 4096;
+constexpr int SMEM_CTRL = 256;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_WARPS * SLAB_BYTES + SMEM_CTRL + 1024;
+constexpr int QSLOTS = 4;                       // tile ids drawn ahead by the scheduler warp (dynamic mode)
+constexpr int ROLE_READERS = 2 + EPI_WARPS + GATHER_THREADS / 32;      // one arrival per role warp and queue entry
+
+struct Ctrl {
+    uint64_t full[STAGES], empty[STAGES];
+    uint64_t tfull[2], tempty[2];
+    uint64_t q_full[QSLOTS], q_empty[QSLOTS];
+    int32_t q_tile[QSLOTS];
+    uint32_t tmem_base, abort;
+};
+static_assert(sizeof(Ctrl) <= SMEM_CTRL, "control block too large");
+
+constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+__device__ __forceinline__ uint32_t idesc_n(int n) { return (IDESC & ~(0x3Fu << 17)) | ((uint32_t)(n >> 3) << 17); }
+
+struct Tile { int row0, valid, kind, e, n, mt; };
+__device__ __forceinline__ Tile read_tile(const int4* tiles, int L) {
+    const int4 d = __ldg(tiles + L);
+    Tile t;
+    t.row0 = d.x;
+    t.valid = d.y & 0xFFFF;
+    t.kind = (d.y >> 16) & 1;
+    t.e = d.z & 0xFFFF;
+    t.n = (d.z >> 16) & 0xFFFF;
+    t.mt = d.w;
+    return t;
+}
+
+// How a role walks over its tiles: static stride, or ids read from the scheduler warp's queue (bounded waits; an entry
+// is released once every role has read it; a negative id ends the kernel).
+template <bool DYN>
+struct TileSeq {
+    Ctrl* ctrl;
+    volatile uint32_t* abort_flag;
+    WsHeader* hdr;
+    int total, slot;
+    uint32_t ph;
+    bool warp_role;       // all 32 lanes call next() together / one lane calls it
+    __device__ __forceinline__ TileSeq(Ctrl* c, volatile uint32_t* af, WsHeader* h, int tot, bool wr)
+        : ctrl(c), abort_flag(af), hdr(h), total(tot), slot(0), ph(0), warp_role(wr) {}
+    __device__ __forceinline__ int first() { return DYN ? next(0) : (int)blockIdx.x; }
+    __device__ __forceinline__ int next(int L) {
+        if (!DYN) return L + gridDim.x;
+        bool ok = mbar_wait(smem_u32(&ctrl->q_full[slot]), ph, abort_flag, hdr, 30);
+        if (warp_role) ok = __all_sync(0xffffffffu, ok);
+        if (!ok) return total;
+        const int t = *reinterpret_cast<volatile int32_t*>(&ctrl->q_tile[slot]);
+        if (warp_role) __syncwarp();
+        if (!warp_role || (threadIdx.x & 31) == 0) mbar_arrive(smem_u32(&ctrl->q_empty[slot]));
+        if (++slot == QSLOTS) { slot = 0; ph ^= 1u; }
+        return t < 0 ? total : t;
+    }
+};
+
+__device__ __forceinline__ int ld_acquire(const int32_t* p) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// ---------------------------------------------------------------------------------------------------------------
+// Tile list.  One block of MAX_E threads per launch-grid slot; every block rebuilds the (tiny) per-expert group
+// offsets in shared memory, then its warps take groups g = warp id, + number of warps, ...
+//   ME(g) = M tiles up to and including group g;  MB(g) = ME(g - 1)
+//   j(g)  = first group j >= g with ME(j) >= ME(g) + window (last group if none): D(g) follows G(j(g))
+//   c(j)  = number of groups whose D tiles precede G(j) = #{g : ME(g) <= MB(j) - window}
+//   pos_G(j) = n1 * MB(j) + n2 * MB(c(j));   pos_D(g) = n1 * ME(j(g)) + n2 * MB(g)
+__global__ void __launch_bounds__(MAX_E)
+fused_tiles_kernel(const int32_t* __restrict__ counts, const int32_t* __restrict__ pad_offsets,
+                   const int32_t* __restrict__ mt_start2, int E, int n1, int n2, int window, int max_tiles,
+                   int4* __restrict__ tiles, int32_t* __restrict__ ready, WsHeader* __restrict__ hdr) {
+    __shared__ int32_t s_mt[MAX_E + 1], s_gofs[MAX_E + 1], s_wtot[32];
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5, n_warps = blockDim.x >> 5;
+    int mc = 0;
+    if (tid < E) {
+        const int m0 = mt_start2[tid], m1 = mt_start2[tid + 1];
+        s_mt[tid] = m0;
+        if (tid == E - 1) s_mt[E] = m1;
+        mc = m1 - m0;
+    }
+    const int ng = (mc + GROUP_TILES - 1) / GROUP_TILES;
+    int inc = ng;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, inc, off);
+        if (lane >= off) inc += t;
+    }
+    if (lane == 31) s_wtot[wid] = inc;
+    __syncthreads();
+    if (wid == 0) {
+        const int mine = lane < n_warps ? s_wtot[lane] : 0;
+        int run = mine;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, run, off);
+            if (lane >= off) run += t;
+        }
+        s_wtot[lane] = run - mine;
+    }
+    __syncthreads();
+    if (tid < E) {
+        s_gofs[tid] = s_wtot[wid] + inc - ng;
+        if (tid == E - 1) s_gofs[E] = s_wtot[wid] + inc;
+    }
+    __syncthreads();
+    const int NG = s_gofs[E], NMT = s_mt[E];
+    const long long total = (long long)NMT * (n1 + n2);
+    if (blockIdx.x == 0 && tid == 0) {
+        hdr->n_ftiles = total <= max_tiles ? (int32_t)total : 0;
+        hdr->next_tile = 0;
+        if (total > max_tiles) atomicCAS(&hdr->status, 0, (int)MOK_ERR_SCHEDULE);
+    }
+    if (total > max_tiles) return;
+    for (int i = blockIdx.x * blockDim.x + tid; i < NMT; i += gridDim.x * blockDim.x) ready[i] = 0;
+
+    // largest e in [0, E) with s_mt[e] <= v and a non-empty tail (the expert that holds M tile index v), for 0 <= v < NMT
+    auto expert_of_tile = [&](int v) {
+        int lo = 0, hi = E;                       // invariant: s_mt[lo] <= v < s_mt[hi]
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (s_mt[mid] <= v) lo = mid; else hi = mid;
+        }
+        return lo;
+    };
+    for (int g = blockIdx.x * n_warps + wid; g < NG; g += gridDim.x * n_warps) {
+        // expert and position of group g: the last e with s_gofs[e] <= g (empty experts have no groups and are skipped
+        // by taking the LAST such e)
+        int lo = 0, hi = E;
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (s_gofs[mid] <= g) lo = mid; else hi = mid;
+        }
+        const int e = lo, gi = g - s_gofs[e], m0 = gi * GROUP_TILES;
+        const int mcnt = s_mt[e + 1] - s_mt[e];
+        const int gm = min(GROUP_TILES, mcnt - m0);              // M tiles of this group
+        const int MB = s_mt[e] + m0, ME = MB + gm;
+        // j(g): the group in which the cumulative M-tile count first reaches ME + window
+        int MEj;
+        {
+            const int target = ME + window;
+            if (window == 0) {
+                MEj = ME;
+            } else if (target > NMT) {
+                MEj = NMT;                                       // the last group
+            } else {
+                const int ej = expert_of_tile(target - 1);       // expert holding the target-th M tile
+                const int within = target - s_mt[ej];            // 1 .. its M-tile count
+                const int gj = (within + GROUP_TILES - 1) / GROUP_TILES;     // groups of ej needed to reach it
+                MEj = s_mt[ej] + min(gj * GROUP_TILES, s_mt[ej + 1] - s_mt[ej]);
+            }
+        }
+        // c(g): groups whose D tiles come before G(g): those ending at or before MB - window
+        int MBc;                                                 // = MB(c(g)): M tiles of those groups
+        {
+            const int v = MB - window;
+            if (v <= 0) {
+                MBc = 0;
+            } else if (window == 0) {
+                MBc = MB;
+            } else {
+                const int ec = expert_of_tile(v - 1);            // expert holding the v-th M tile
+                const int within = v - s_mt[ec];                 // M tiles of ec among the first v
+                const int mce = s_mt[ec + 1] - s_mt[ec];
+                // whole groups of ec inside the first v tiles (its last, partial group counts once all its tiles are in)
+                MBc = s_mt[ec] + (within == mce ? mce : within / GROUP_TILES * GROUP_TILES);
+            }
+        }
+        const long long posG = (long long)n1 * MB + (long long)n2 * MBc;
+        const long long posD = (long long)n1 * MEj + (long long)n2 * MB;
+        const int cnt = counts[e], pad0 = pad_offsets[e];
+        for (int i = lane; i < (n1 + n2) * gm; i += 32) {
+            const int kind = i >= n1 * gm;
+            const int r = kind ? i - n1 * gm : i;
+            const int n = r / gm, m = m0 + (r - n * gm);
+            int4 d;
+            d.x = pad0 + m * TM;
+            d.y = min(TM, cnt - m * TM) | (kind << 16);
+            d.z = e | (n << 16);
+            d.w = s_mt[e] + m;
+            tiles[(kind ? posD : posG) + r] = d;
+        }
+    }
+}
+
+struct FusedArgs {
+    const __nv_bfloat16* x;        // [T, H] token rows (gathered through row_token)
+    const int32_t* row_token;      // padded row -> token
+    const int4* tiles;             // the tile list
+    const int32_t* n_tiles;        // device: its length
+    int32_t* next_tile;            // device: dynamic mode's draw counter (zeroed by the tile-list kernel)
+    int32_t* ready;                // per 256-row M tile: epilogue-warp arrivals of its gate/up tiles
+    int32_t max_tiles;
+    int32_t H, I, E;
+    int32_t n1, n2;                // N tiles of a gate/up row tile (ceil(I / 128)) and of a down row tile (ceil(H / 256))
+    int32_t kb1, kb2;              // k-blocks of the two kinds
+    int32_t dbg;                   // != 0: counters into header->dbg[1] (gate/up tiles) and [2] (down tiles)
+    int32_t starve;                // test hook: the producer issues nothing
+    WsHeader* header;
+};
+
+template <bool DYN>
+__global__ void __launch_bounds__(THREADS + (DYN ? 32 : 0), 1)
+fused_ffn_kernel(const __grid_constant__ CUtensorMap mapWgu, const __grid_constant__ CUtensorMap mapWgu64,
+                 const __grid_constant__ CUtensorMap mapHst, const __grid_constant__ CUtensorMap mapHld,
+                 const __grid_constant__ CUtensorMap mapWd, const __grid_constant__ CUtensorMap mapY,
+                 const __grid_constant__ FusedArgs a) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t* smem = smem_raw + (base - raw);
+    Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem + STAGES * STAGE_BYTES + EPI_WARPS * SLAB_BYTES);
+    volatile uint32_t* abort_flag = &ctrl->abort;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    int total = *a.n_tiles;
+    if (total > a.max_tiles) total = a.max_tiles;
+    const int last_cols = a.I - (a.n1 - 1) * (BN / 2);
+    const bool narrow_last = last_cols <= BN / 4;          // last gate/up N tile as [gate 64 | up 64], N = 128
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(smem_u32(&ctrl->full[s]), 1 + GATHER_THREADS);
+            mbar_init(smem_u32(&ctrl->empty[s]), 1);
+        }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(smem_u32(&ctrl->tfull[s]), 1);
+            mbar_init(smem_u32(&ctrl->tempty[s]), 4);
+        }
+        if (DYN) {
+            for (int q = 0; q < QSLOTS; ++q) {
+                mbar_init(smem_u32(&ctrl->q_full[q]), 1);
+                mbar_init(smem_u32(&ctrl->q_empty[q]), ROLE_READERS);
+            }
+        }
+        ctrl->abort = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&ctrl->tmem_base)), "r"((uint32_t)TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = ctrl->tmem_base;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0 && !a.starve) {
+            int s = 0;
+            uint32_t ph = 0;
+            long long d_ready = 0;
+            TileSeq<DYN> seq(ctrl, abort_flag, a.header, total, false);
+            for (int L = seq.first(); L < total; L = seq.next(L)) {
+                const Tile t = read_tile(a.tiles, L);
+                const bool two = t.valid > BM;
+                bool ok = true;
+                if (t.kind) {
+                    // every gate/up tile of these rows has stored h: n1 tiles x 4 epilogue warps per 128-row half
+                    const int need = a.n1 * (two ? 8 : 4);
+                    const int32_t* flag = a.ready + t.mt;
+                    if (ld_acquire(flag) < need) {
+                        const long long w0 = a.dbg ? clock64() : 0;
+                        const unsigned long long t0 = globaltimer();
+                        uint32_t spins = 0;
+                        while (ld_acquire(flag) < need) {
+                            __nanosleep(64);
+                            if ((++spins & 63u) == 0u) {
+                                if (*abort_flag) { ok = false; break; }
+                                const unsigned long long limit =
+                                    a.header->wait_limit_us ? 1000ull * a.header->wait_limit_us : WAIT_LIMIT_NS;
+                                if (globaltimer() - t0 > limit) {
+                                    *abort_flag = 1u;
+                                    atomicCAS(&a.header->status, 0, (int)MOK_ERR_TIMEOUT);
+                                    a.header->where = 40;
+                                    ok = false;
+                                    break;
+                                }
+                            }
+                        }
+                        if (a.dbg) d_ready += clock64() - w0;
+                    }
+                    if (!ok) break;
+                    // the rows were written through the async proxy by other CTAs and are read through it below
+                    asm volatile("fence.proxy.async;" ::: "memory");
+                }
+                const int kblocks = t.kind ? a.kb2 : a.kb1;
+                const bool narrow = !t.kind && narrow_last && t.n == a.n1 - 1;
+                const int brow0 = t.kind ? t.e * a.H + t.n * BN : t.e * 2 * a.I + t.n * (BN / 2);
+                const int brow1 = t.kind ? brow0 + BN / 2 : brow0 + a.I;
+                for (int kb = 0; kb < kblocks; ++kb) {
+                    ok = mbar_wait(smem_u32(&ctrl->empty[s]), ph ^ 1u, abort_flag, a.header, 1);
+                    if (!ok) break;
+                    const uint32_t full = smem_u32(&ctrl->full[s]);
+                    const uint32_t sa = base + s * STAGE_BYTES, sb = sa + 2 * A_BYTES;
+                    if (t.kind) {
+                        mbar_expect_tx(full, B_BYTES + (two ? 2 : 1) * A_BYTES);
+                        tma_load_2d(sa, &mapHld, full, kb * BK, t.row0);
+                        if (two) tma_load_2d(sa + A_BYTES, &mapHld, full, kb * BK, t.row0 + BM);
+                        tma_load_2d(sb, &mapWd, full, kb * BK, brow0);
+                        tma_load_2d(sb + B_BYTES / 2, &mapWd, full, kb * BK, brow1);
+                    } else if (narrow) {
+                        mbar_expect_tx(full, B_BYTES / 2);
+                        tma_load_2d(sb, &mapWgu64, full, kb * BK, brow0);
+                        tma_load_2d(sb + B_BYTES / 4, &mapWgu64, full, kb * BK, brow1);
+                    } else {
+                        mbar_expect_tx(full, B_BYTES);
+                        tma_load_2d(sb, &mapWgu, full, kb * BK, brow0);
+                        tma_load_2d(sb + B_BYTES / 2, &mapWgu, full, kb * BK, brow1);
+                    }
+                    if (++s == STAGES) { s = 0; ph ^= 1u; }
+                }
+                if (!ok) break;
+            }
+            if (a.dbg) atomicAdd(&a.header->dbg[2][DBG_PROD_WAIT_EMPTY], (unsigned long long)d_ready);
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            int s = 0;
+            uint32_t ph = 0, ap0 = 0, ap1 = 0;
+            const bool dbg = a.dbg != 0;
+            long long d_full[2] = {0, 0}, d_tempty[2] = {0, 0}, d_kb[2] = {0, 0}, d_rows[2] = {0, 0}, d_tot[2] = {0, 0};
+            const unsigned long long d_ns0 = dbg ? globaltimer() : 0ull;
+            const long long d_c0 = dbg ? clock64() : 0;
+            TileSeq<DYN> seq(ctrl, abort_flag, a.header, total, false);
+            for (int L = seq.first(); L < total; L = seq.next(L)) {
+                const Tile t = read_tile(a.tiles, L);
+                const bool two = t.valid > BM;
+                const int kblocks = t.kind ? a.kb2 : a.kb1;
+                uint32_t idesc = IDESC;
+                if (t.kind) {
+                    if (a.H - t.n * BN < BN) idesc = idesc_n((a.H - t.n * BN + 15) & ~15);
+                } else if (narrow_last && t.n == a.n1 - 1) {
+                    idesc = idesc_n(BN / 2);
+                }
+                const long long tile0 = dbg ? clock64() : 0;
+                long long w0 = tile0;
+                bool ok = mbar_wait(smem_u32(&ctrl->tempty[0]), ap0 ^ 1u, abort_flag, a.header, 2);
+                if (dbg) d_tempty[t.kind] += clock64() - w0;
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t d0 = tmem_base, d1 = tmem_base + BN;
+                for (int kb = 0; kb < kblocks; ++kb) {
+                    if (dbg) w0 = clock64();
+                    ok = mbar_wait(smem_u32(&ctrl->full[s]), ph, abort_flag, a.header, 3);
+                    if (dbg) { d_full[t.kind] += clock64() - w0; d_kb[t.kind] += two ? 2 : 1; }
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t sa = base + s * STAGE_BYTES;
+                    const uint64_t a0 = make_smem_desc(sa), a1 = make_smem_desc(sa + A_BYTES);
+                    const uint64_t bd = make_smem_desc(sa + 2 * A_BYTES);
+#pragma unroll
+                    for (int j = 0; j < BK / UMMA_K; ++j)
+                        tc_mma<1>(d0, a0 + (uint64_t)(j * 2), bd + (uint64_t)(j * 2), idesc, (kb | j) ? 1u : 0u);
+                    if (kb == kblocks - 1) { tc_commit<1>(smem_u32(&ctrl->tfull[0])); ap0 ^= 1u; }
+                    if (two) {
+                        if (kb == 0) {
+                            if (dbg) w0 = clock64();
+                            ok = mbar_wait(smem_u32(&ctrl->tempty[1]), ap1 ^ 1u, abort_flag, a.header, 8);
+                            if (dbg) d_tempty[t.kind] += clock64() - w0;
+                            if (!ok) break;
+                            tc_fence_after();
+                        }
+#pragma unroll
+                        for (int j = 0; j < BK / UMMA_K; ++j)
+                            tc_mma<1>(d1, a1 + (uint64_t)(j * 2), bd + (uint64_t)(j * 2), idesc, (kb | j) ? 1u : 0u);
+                    }
+                    tc_commit<1>(smem_u32(&ctrl->empty[s]));
+                    if (++s == STAGES) { s = 0; ph ^= 1u; }
+                }
+                if (!ok) break;
+                if (two) { tc_commit<1>(smem_u32(&ctrl->tfull[1])); ap1 ^= 1u; }
+                if (dbg) { d_rows[t.kind] += (long long)t.valid * kblocks; d_tot[t.kind] += clock64() - tile0; }
+            }
+            if (dbg) {
+                const unsigned long long ns = globaltimer() - d_ns0, cyc = (unsigned long long)(clock64() - d_c0);
+                {   // slot 0: the whole kernel (imbalance of the tile -> CTA rule, clock)
+                    unsigned long long* d = a.header->dbg[0];
+                    atomicAdd(d + DBG_MMA_TOTAL, cyc);
+                    atomicMax(d + DBG_MMA_TOTAL_MAX, cyc);
+                    atomicAdd(d + DBG_MMA_TOTAL_NS, ns);
+                    atomicAdd(d + DBG_CTAS, 1ull);
+                }
+                for (int q = 0; q < 2; ++q) {
+                    unsigned long long* d = a.header->dbg[1 + q];
+                    // the CTA's time is split between the two kinds in proportion to the cycles spent in their tiles
+                    const unsigned long long share = d_tot[0] + d_tot[1] > 0 ? (unsigned long long)d_tot[q] : 0ull;
+                    const unsigned long long ns_q = d_tot[0] + d_tot[1] > 0
+                        ? (unsigned long long)((double)ns * (double)d_tot[q] / (double)(d_tot[0] + d_tot[1])) : 0ull;
+                    atomicAdd(d + DBG_MMA_WAIT_FULL, (unsigned long long)d_full[q]);
+                    atomicAdd(d + DBG_MMA_WAIT_TEMPTY, (unsigned long long)d_tempty[q]);
+                    atomicAdd(d + DBG_MMA_TOTAL, share);
+                    atomicMax(d + DBG_MMA_TOTAL_MAX, share);
+                    atomicAdd(d + DBG_MMA_TOTAL_NS, ns_q);
+                    atomicAdd(d + DBG_KBLOCKS, (unsigned long long)d_kb[q]);
+                    atomicAdd(d + DBG_ROWS_KB, (unsigned long long)d_rows[q]);
+                    atomicAdd(d + DBG_CTAS, 1ull);
+                }
+            }
+        }
+        __syncwarp();
+    } else if (DYN && warp == THREADS / 32) {
+        // ------------------------------------------------------------------ scheduler warp (dynamic mode)
+        if (lane == 0) {
+            // draws list positions in order from one global counter, a few tiles ahead of the roles.  Whoever draws a
+            // position runs, and everything a down tile waits for sits at smaller positions, which were drawn before.
+            int slot = 0;
+            uint32_t qph = 0;
+            for (;;) {
+                const int L = atomicAdd(a.next_tile, 1);
+                if (!mbar_wait(smem_u32(&ctrl->q_empty[slot]), qph ^ 1u, abort_flag, a.header, 32)) break;
+                *reinterpret_cast<volatile int32_t*>(&ctrl->q_tile[slot]) = L < total ? L : -1;
+                mbar_arrive(smem_u32(&ctrl->q_full[slot]));
+                if (++slot == QSLOTS) { slot = 0; qph ^= 1u; }
+                if (L >= total) break;
+            }
+        }
+        __syncwarp();
+    } else if (warp >= 2 + EPI_WARPS) {
+        // ------------------------------------------------------------------ gather warps (pull dispatch)
+        const int gw = warp - (2 + EPI_WARPS), sub = lane >> 3, chunk = lane & 7;
+        int s = 0;
+        uint32_t ph = 0;
+        TileSeq<DYN> seq(ctrl, abort_flag, a.header, total, true);
+        for (int L = seq.first(); L < total; L = seq.next(L)) {
+            const Tile t = read_tile(a.tiles, L);
+            bool ok = true;
+            if (t.kind) {
+                // down tile: both operands come by TMA; these threads only complete the ring's arrival counts
+                for (int kb = 0; kb < a.kb2; ++kb) {
+                    ok = mbar_wait(smem_u32(&ctrl->empty[s]), ph ^ 1u, abort_flag, a.header, 5);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    mbar_arrive(smem_u32(&ctrl->full[s]));
+                    if (++s == STAGES) { s = 0; ph ^= 1u; }
+                }
+                if (!ok) break;
+                continue;
+            }
+            const bool two = t.valid > BM;
+            const __nv_bfloat16* src[16];
+            uint32_t live = 0u;
+            int tok[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const int r = (i >> 3) * BM + gw * 32 + (i & 7) * 4 + sub;
+                tok[i] = __ldg(a.row_token + t.row0 + min(r, t.valid - 1));
+            }
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const int r = (i >> 3) * BM + gw * 32 + (i & 7) * 4 + sub;
+                src[i] = a.x + (size_t)tok[i] * a.H + chunk * 8;
+                if (r < t.valid) live |= 1u << i;
+            }
+            for (int kb = 0; kb < a.kb1; ++kb) {
+                ok = mbar_wait(smem_u32(&ctrl->empty[s]), ph ^ 1u, abort_flag, a.header, 5);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                const uint32_t sa = base + s * STAGE_BYTES;
+                const bool in_k = (kb * BK + chunk * 8) < a.H;
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    if (i < 8 || two) {
+                        const int rr = gw * 32 + (i & 7) * 4 + sub;
+                        const uint32_t dst = sa + (i >> 3) * A_BYTES + rr * 128 + ((chunk ^ (rr & 7)) << 4);
+                        const bool on = in_k && ((live >> i) & 1u);
+                        cp_async_16(dst, on ? (const void*)(src[i] + kb * BK) : (const void*)a.x, on ? 16u : 0u);
+                    }
+                }
+                cp_async_mbar_arrive(smem_u32(&ctrl->full[s]));
+                if (++s == STAGES) { s = 0; ph ^= 1u; }
+            }
+            if (!ok) break;
+        }
+        asm volatile("cp.async.wait_all;" ::: "memory");
+    } else {
+        // ------------------------------------------------------------------ epilogue warps
+        const int acc = (warp - 2) >> 2;
+        const int quad = warp & 3;
+        const uint32_t slab = base + STAGES * STAGE_BYTES + (warp - 2) * SLAB_BYTES;
+        uint32_t aph = 0;
+        TileSeq<DYN> seq(ctrl, abort_flag, a.header, total, true);
+        for (int L = seq.first(); L < total; L = seq.next(L)) {
+            const Tile t = read_tile(a.tiles, L);
+            if (acc == 1 && t.valid <= BM) continue;
+            bool ok = mbar_wait(smem_u32(&ctrl->tfull[acc]), aph, abort_flag, a.header, 4);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            aph ^= 1u;
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * BN);
+            const int row = t.row0 + acc * BM + quad * 32;
+            const bool swiglu = !t.kind;
+            const bool narrow = swiglu && narrow_last && t.n == a.n1 - 1;
+            const int passes = swiglu ? (narrow ? 1 : 2) : 4;
+            const uint32_t up_off = narrow ? BN / 4 : BN / 2;
+            const int c0 = swiglu ? t.n * (BN / 2) : t.n * BN;
+            const int n_cols = swiglu ? a.I : a.H;
+            const CUtensorMap* mapC = swiglu ? &mapHst : &mapY;
+            uint32_t cur[32], nxt[32];
+            auto hand_back = [&]() {
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&ctrl->tempty[acc]));
+            };
+            auto load_pass = [&](int pass, uint32_t (&o)[32]) {
+#pragma unroll
+                for (int c = 0; c < 64; c += 32) {
+                    if (swiglu) {
+                        uint32_t g[32], u[32];
+                        tc_ld32(taddr + pass * 64 + c, g);
+                        tc_ld32(taddr + up_off + pass * 64 + c, u);
+                        tc_wait_ld();
+                        if (pass == passes - 1 && c == 32) hand_back();
+#pragma unroll
+                        for (int i = 0; i < 16; ++i)
+                            o[(c >> 1) + i] = pack_bf16(tc::swiglu(__uint_as_float(g[2 * i]), __uint_as_float(u[2 * i])),
+                                                        tc::swiglu(__uint_as_float(g[2 * i + 1]), __uint_as_float(u[2 * i + 1])));
+                    } else {
+                        uint32_t r[32];
+                        tc_ld32(taddr + pass * 64 + c, r);
+                        tc_wait_ld();
+                        if (pass == passes - 1 && c == 32) hand_back();
+#pragma unroll
+                        for (int i = 0; i < 16; ++i)
+                            o[(c >> 1) + i] = pack_bf16(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
+                    }
+                }
+            };
+            load_pass(0, nxt);
+#pragma unroll
+            for (int pass = 0; pass < 4; ++pass) {
+                if (pass >= passes) break;
+#pragma unroll
+                for (int i = 0; i < 32; ++i) cur[i] = nxt[i];
+                if (pass + 1 < passes) load_pass(pass + 1, nxt);
+                if (lane == 0) tma_store_wait_read();
+                __syncwarp();
+                const uint32_t line = slab + lane * 128;
+#pragma unroll
+                for (int v = 0; v < 8; ++v)
+                    st_shared_v4(line + ((v ^ (lane & 7)) << 4), cur[4 * v], cur[4 * v + 1], cur[4 * v + 2], cur[4 * v + 3]);
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) {
+                    const int col = c0 + pass * 64;
+                    if (col < n_cols) tma_store_2d(mapC, slab, col, row);
+                    tma_store_commit();
+                }
+            }
+            if (swiglu && lane == 0) {
+                // h of this warp's 32 rows is on its way: wait until the stores have completed (not only left shared
+                // memory), then publish one arrival for the M tile.  Release at GPU scope after a proxy fence: the down
+                // tiles read these rows through the async proxy from other SMs.
+                tma_store_wait_all();
+                asm volatile("fence.proxy.async;" ::: "memory");
+                __threadfence();
+                asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(a.ready + t.mt) : "memory");
+            }
+            __syncwarp();
+        }
+        if (lane == 0) tma_store_wait_all();
+        __syncwarp();
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    if (*abort_flag) {   // failure path only: give copies and MMAs already in flight time to land before leaving
+        const unsigned long long t0 = globaltimer();
+        while (globaltimer() - t0 < 200000ull) { }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS) : "memory");
+    }
+}
+
+}  // namespace ff
+
+template <bool DYN>
+static cudaError_t launch_kernel(int grid, cudaStream_t s, const CUtensorMap& m0, const CUtensorMap& m1, const CUtensorMap& m2,
+                                 const CUtensorMap& m3, const CUtensorMap& m4, const CUtensorMap& m5, const ff::FusedArgs& a) {
+    using namespace ff;
+    static PerDevice configured;
+    int dev = 0, sm_count = 0;
+    cudaError_t e = current_device(&dev);
+    if (e != cudaSuccess) return e;
+    e = configured.get(dev, &sm_count, [](int d, int* sms) {
+        cudaError_t e2 = cudaFuncSetAttribute(fused_ffn_kernel<DYN>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+        return e2 != cudaSuccess ? e2 : device_sm_count(d, sms);
+    });
+    if (e != cudaSuccess) return e;
+    if (grid <= 0 || grid > sm_count) grid = sm_count;
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    // static list: tiles wait for tiles of other CTAs, so every CTA of the grid must be resident (cooperative launch).
+    // Dynamic draw: a position is only drawn by a CTA that runs: plain launch.
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(THREADS + (DYN ? 32 : 0));
+    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cfg.stream = s;
+    cfg.attrs = attr;
+    cfg.numAttrs = DYN ? 0 : 1;
+    return cudaLaunchKernelEx(&cfg, fused_ffn_kernel<DYN>, m0, m1, m2, m3, m4, m5, a);
+}
+
+// Host side.  `window_tiles`: distance (in list positions) between a group's gate/up tiles and its down tiles; 0 = the
+// default of two grids' worth of tiles, -1 = none (a group's down tiles directly behind its gate/up tiles).
+cudaError_t launch_fused_ffn(const __nv_bfloat16* x, int T, int H, int I, int E, const __nv_bfloat16* Wgu,
+                             const __nv_bfloat16* Wd, const WsLayout& L, char* ws, int grid, int window_tiles, bool dynamic,
+                             bool dbg, bool starve, cudaStream_t s) {
+    using namespace ff;
+    int dev = 0, sm_count = 0;
+    cudaError_t e = current_device(&dev);
+    if (e != cudaSuccess) return e;
+    if ((e = device_sm_count(dev, &sm_count)) != cudaSuccess) return e;
+    if (grid <= 0 || grid > sm_count) grid = sm_count;
+    WsHeader* hdr = reinterpret_cast<WsHeader*>(ws + L.header);
+    const int n1 = (I + BN / 2 - 1) / (BN / 2), n2 = (H + BN - 1) / BN;
+    if (window_tiles == 0) window_tiles = 2 * grid;
+    const int window = window_tiles < 0 ? 0 : (window_tiles + n1 - 1) / n1;      // in M tiles
+    int4* tiles = reinterpret_cast<int4*>(ws + L.ftiles);
+    int32_t* ready = reinterpret_cast<int32_t*>(ws + L.ready);
+    // enough blocks for one warp per group of a large batch; every block rebuilds the per-expert offsets itself
+    int tblocks = (int)((L.max_mt / 2 / GROUP_TILES + E) / (MAX_E / 32)) + 1;
+    if (tblocks > sm_count) tblocks = sm_count;
+    fused_tiles_kernel<<<tblocks, MAX_E, 0, s>>>(reinterpret_cast<const int32_t*>(ws + L.counts),
+                                                 reinterpret_cast<const int32_t*>(ws + L.pad_offsets),
+                                                 reinterpret_cast<const int32_t*>(ws + L.mt_start2), E, n1, n2, window,
+                                                 L.max_ftiles, tiles, ready, hdr);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+
+    CUtensorMap mWgu, mWgu64, mHst, mHld, mWd, mY;
+    void* h = ws + L.h;
+    void* y = ws + L.y;
+    if (!tmap::bf16_sw128(&mWgu, Wgu, (uint64_t)E * 2 * I, (uint64_t)H, BN / 2) ||
+        !tmap::bf16_sw128(&mWgu64, Wgu, (uint64_t)E * 2 * I, (uint64_t)H, BN / 4) ||
+        !tmap::bf16_sw128(&mHst, h, (uint64_t)L.Rpad, (uint64_t)I, 32) ||
+        !tmap::bf16_sw128(&mHld, h, (uint64_t)L.Rpad, (uint64_t)I, BM) ||
+        !tmap::bf16_sw128(&mWd, Wd, (uint64_t)E * H, (uint64_t)I, BN / 2) ||
+        !tmap::bf16_sw128(&mY, y, (uint64_t)L.Rpad, (uint64_t)H, 32))
+        return cudaErrorInvalidValue;
+    FusedArgs a;
+    a.x = x;
+    a.row_token = reinterpret_cast<const int32_t*>(ws + L.row_token);
+    a.tiles = tiles;
+    a.n_tiles = &hdr->n_ftiles;
+    a.next_tile = &hdr->next_tile;
+    a.ready = ready;
+    a.max_tiles = L.max_ftiles;
+    a.H = H; a.I = I; a.E = E;
+    a.n1 = n1; a.n2 = n2;
+    a.kb1 = (H + BK - 1) / BK;
+    a.kb2 = (I + BK - 1) / BK;
+    a.dbg = dbg ? 1 : 0;
+    a.starve = starve ? 1 : 0;
+    a.header = hdr;
+    (void)T;
+
+    return dynamic ? launch_kernel<true>(grid, s, mWgu, mWgu64, mHst, mHld, mWd, mY, a)
+                   : launch_kernel<false>(grid, s, mWgu, mWgu64, mHst, mHld, mWd, mY, a);
+}
+
+}  // namespace mok

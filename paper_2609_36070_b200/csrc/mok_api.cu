@@ -74,6 +74,13 @@ bool ws_layout(int T, int H, int I, int Is, int E, int k, WsLayout* L, bool mx) 
     L->xg = take(2 * (size_t)Rpad * H);
     L->h = take(2 * (size_t)Rpad * I);
     L->y = take(2 * (size_t)Rpad * H);
+    {   // fused expert-FFN kernel: every 256-row tile times (gate/up N tiles + down N tiles), one counter per row tile
+        const long long mt2 = Rpad / (2 * TILE_M), per = (I + 127) / 128 + (H + 255) / 256;
+        const long long nt = mt2 * per;
+        L->max_ftiles = nt < (1ll << 30) ? (int32_t)nt : 0;
+        L->ftiles = take(sizeof(int4) * (size_t)L->max_ftiles);
+        L->ready = take(sizeof(int32_t) * (size_t)mt2);
+    }
     L->hs = take(Is > 0 ? 2 * (size_t)L->Tpad * Is : 0);
     L->ysh = take(Is > 0 ? 2 * (size_t)L->Tpad * H : 0);
     if (mx) {
@@ -95,7 +102,7 @@ static bool mx_pairs(const mok_config* cfg) { return cfg && cfg->cta_group == 2;
 static int validate(const mok_args* a, WsLayout* L, size_t extra_ws) {
     if (!a) return MOK_ERR_NULL;
     if (a->config && (a->config->precision < 0 || a->config->precision > 1)) return MOK_ERR_SHAPE;
-    if (a->config && (a->config->tile_sched < 0 || a->config->tile_sched > 1)) return MOK_ERR_SHAPE;
+    if (a->config && (a->config->tile_sched < 0 || a->config->tile_sched > 2)) return MOK_ERR_SHAPE;
     const bool mx = use_mx(a->config);
     if (mx && a->config->impl != MOK_IMPL_TCGEN05) return MOK_ERR_SHAPE;
     if (!ws_layout(a->T, a->H, a->I, a->I_shared, a->E, a->k, L, mx)) return MOK_ERR_SHAPE;
@@ -121,7 +128,8 @@ static int validate(const mok_args* a, WsLayout* L, size_t extra_ws) {
                       a->config->router_impl < 0 || a->config->router_impl > 2 ||
                       a->config->gather_mode < 0 || a->config->gather_mode > 2 ||
                       a->config->cta_group < 0 || a->config->cta_group > 3 ||
-                      a->config->host_chunks < 0 || a->config->host_chunks > MOK_MAX_HOST_CHUNKS))
+                      a->config->host_chunks < 0 || a->config->host_chunks > MOK_MAX_HOST_CHUNKS ||
+                      a->config->fused_ffn < 0 || a->config->fused_ffn > 2 || a->config->fused_window < -1))
         return MOK_ERR_SHAPE;
     return MOK_OK;
 }
@@ -175,6 +183,18 @@ static bool use_m2(const mok_config* cfg, int K, int tile_m, long long rows, int
     // once: there the 128-row kernel, whose four stages are all weight and activation bytes, is the faster one
     // (measured on the DeepSeek-like shape: 3.39 vs 3.62 ms at 2 rows per expert, 5.58 vs 5.31 ms at 128).
     return K >= M2_MIN_K && rows >= 96ll * experts;
+}
+
+// Routed gate/up + SwiGLU + down as ONE persistent launch (gemm_fused.cu).  It is the 256-row-tile kernel's work, so it
+// is chosen where that kernel would serve both GEMMs (fused_ffn = 0), can be switched off (1: two launches) or forced
+// for any shape with the token gather fused (2).
+static bool use_fused_ffn(const mok_config* cfg, int H, int I, int tile_m, long long rows, int experts, int max_ftiles) {
+    if (use_simt(cfg) || use_tn(cfg) || use_mx(cfg) || tile_m != TILE_M || max_ftiles <= 0) return false;
+    if (cfg && (cfg->cta_group == 1 || cfg->cta_group == 2 || cfg->fused_ffn == 1)) return false;
+    if (cfg && cfg->tile_sched == 1 && cfg->fused_ffn != 2) return false;   // (tile stealing belongs to the two-launch path)
+    if (!fused_gather(cfg, I)) return false;
+    if (cfg && cfg->fused_ffn == 2) return true;
+    return use_m2(cfg, H, tile_m, rows, experts) && use_m2(cfg, I, tile_m, rows, experts);
 }
 
 int run_gemm(GemmArgs g, bool swiglu, const mok_config* cfg, const WsLayout& L, char* ws, cudaStream_t s) {
@@ -331,7 +351,14 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
         g.K = a->H; g.N = a->I; g.ldc = a->I; g.E = a->E; g.rows_pad = L.Rpad; g.dense_rows = 0;
         g.total_rows = L.R;
         g.tile_sched = a->config ? a->config->tile_sched : 0;
-        if ((rc = run_gemm(g, true, a->config, L, ws, s))) return rc;
+        const bool fused = !simt && use_fused_ffn(a->config, a->H, a->I, tile_m, L.R, a->E, L.max_ftiles);
+        if (fused) {
+            e = launch_fused_ffn(x, a->T, a->H, a->I, a->E, reinterpret_cast<const __nv_bfloat16*>(a->W_gate_up),
+                                 reinterpret_cast<const __nv_bfloat16*>(a->W_down), L, ws, a->config ? a->config->grid : 0,
+                                 a->config ? a->config->fused_window : 0, !(a->config && a->config->tile_sched == 2), dbg,
+                                 g.starve != 0, s);
+            if (e != cudaSuccess) return cuda_fail(e);
+        } else if ((rc = run_gemm(g, true, a->config, L, ws, s))) return rc;
         g.row_token = nullptr;
         g.starve = 0;
         g.a_rows = L.Rpad;
@@ -341,7 +368,7 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
         g.B = reinterpret_cast<const __nv_bfloat16*>(a->W_down);
         g.C = ws + L.y;
         g.K = a->I; g.N = a->H; g.ldc = a->H;
-        if ((rc = run_gemm(g, false, a->config, L, ws, s))) return rc;
+        if (!fused && (rc = run_gemm(g, false, a->config, L, ws, s))) return rc;
         g.tile_sched = 0;
     }
     MOK_MARK(MOK_STAGE_GEMM2 + 1);

@@ -24,7 +24,9 @@ struct WsHeader {
     int32_t where;         // diagnostic: which wait gave up (site number inside the kernel)
     uint32_t wait_limit_us; // 0 = default (2 s): bound of every mbarrier wait, in microseconds
     int32_t n_flag;        // tensor-core router: tokens on the near-tie list of the current call
-    int32_t pad[58];
+    int32_t n_ftiles;      // length of the fused expert-FFN kernel's tile list (gate/up tiles + down tiles)
+    int32_t next_tile;     // its dynamic hand-out: the next list position to draw
+    int32_t pad[56];
     // optional counters of the tcgen05 GEMMs (config.debug): [slot][counter]; SM cycles summed over CTAs unless stated
     unsigned long long dbg[4][MOK_DEBUG_COUNTERS];
 };
@@ -45,6 +47,8 @@ struct WsLayout {
                           // 3 * (E rounded up to 32) if larger: the one-kernel router pads each part to 32 rows)
     size_t xg, h, y, hs, ysh;
     size_t x8, sx, h8, sh;   // MXFP8 mode: quantised token rows + row-major scales, quantised gated activation + scale atoms
+    size_t ftiles, ready;    // fused expert-FFN kernel: tile list (int4 per tile) and per-M-tile completion counters
+    int32_t max_ftiles;
     size_t total;
     int32_t R;            // T*k
     int32_t Rpad;         // upper bound on padded rows for either tile_m (multiple of 256)
@@ -136,6 +140,10 @@ cudaError_t launch_gemm_tc(const GemmArgs& a, int epi, int grid, cudaStream_t s)
 cudaError_t launch_gemm_tn(const GemmArgs& a, int epi, int grid, cudaStream_t s);   // tokens on the MMA's N side
 cudaError_t launch_gemm_m2(const GemmArgs& a, int epi, int grid, cudaStream_t s);   // 256-row tiles, two accumulators
 cudaError_t launch_gemm_mx(const GemmArgs& a, int epi, int grid, cudaStream_t s);   // MXFP8 operands, block-scaled MMA
+// routed gate/up + SwiGLU + down in one persistent launch (tile list + kernel); needs the schedule's 256-row tile table
+cudaError_t launch_fused_ffn(const __nv_bfloat16* x, int T, int H, int I, int E, const __nv_bfloat16* Wgu,
+                             const __nv_bfloat16* Wd, const WsLayout& L, char* ws, int grid, int window_tiles, bool dynamic,
+                             bool dbg, bool starve, cudaStream_t s);
 cudaError_t launch_mx_quantize_rows(const __nv_bfloat16* in, long long rows, int K, uint8_t* codes, uint8_t* scales,
                                     cudaStream_t s);
 cudaError_t launch_mx_quantize_atoms(const __nv_bfloat16* in, int groups, int rows_per_group, int K, uint8_t* codes,

@@ -38,7 +38,8 @@ class mok_config(ctypes.Structure):
     _fields_ = [("impl", ctypes.c_int32), ("grid", ctypes.c_int32), ("router_impl", ctypes.c_int32),
                 ("profile", ctypes.c_int32), ("gather_mode", ctypes.c_int32), ("cta_group", ctypes.c_int32),
                 ("debug", ctypes.c_int32), ("host_chunks", ctypes.c_int32), ("precision", ctypes.c_int32),
-                ("tile_sched", ctypes.c_int32), ("macrobatch_tokens", ctypes.c_int32)]
+                ("tile_sched", ctypes.c_int32), ("macrobatch_tokens", ctypes.c_int32),
+                ("fused_ffn", ctypes.c_int32), ("fused_window", ctypes.c_int32)]
 
 
 class mok_args(ctypes.Structure):
@@ -184,8 +185,9 @@ def _stream(stream):
 
 
 def _config(impl=0, grid=0, router_impl=0, profile=0, gather_mode=0, cta_group=0, debug=0, host_chunks=0,
-            precision=0, tile_sched=0, macrobatch_tokens=0):
+            precision=0, tile_sched=0, macrobatch_tokens=0, fused_ffn=0, fused_window=0):
     c = mok_config()
+    c.fused_ffn, c.fused_window = fused_ffn, fused_window
     c.precision = precision
     c.tile_sched = tile_sched
     c.macrobatch_tokens = macrobatch_tokens
@@ -556,7 +558,7 @@ def mok_debug_counters(workspace, stream=None):
     buf = (ctypes.c_ulonglong * (4 * n))()
     wp, _ = _aligned_ws(workspace)
     _check(_lib.mok_debug_counters(wp, _stream(stream), buf))
-    names = {1: "gemm1", 2: "gemm2", 3: "shared"}
+    names = {0: "fused", 1: "gemm1", 2: "gemm2", 3: "shared"}
     return {names[s]: {c: int(buf[s * n + i]) for i, c in enumerate(DEBUG_COUNTERS)} for s in names}
 
 

@@ -30,7 +30,8 @@ SMALL = [
 
 
 @pytest.mark.parametrize("cfg", SMALL, ids=[c.name for c in SMALL])
-@pytest.mark.parametrize("impl", ["tcgen05_fused_gather", "tcgen05_separate_gather", "tcgen05_single_cta", "tcgen05_256_row_tiles", "tcgen05_tokens_as_n", "simt"])
+@pytest.mark.parametrize("impl", ["tcgen05_fused_gather", "tcgen05_separate_gather", "tcgen05_single_cta", "tcgen05_256_row_tiles",
+                                  "tcgen05_tokens_as_n", "simt", "tcgen05_one_launch_ffn", "tcgen05_one_launch_ffn_no_window"])
 def test_small_shapes_every_token(cfg, impl):
     m = mok()
     conf = {"simt": m._config(impl=m.MOK_IMPL_SIMT),
@@ -38,6 +39,8 @@ def test_small_shapes_every_token(cfg, impl):
             "tcgen05_separate_gather": m._config(gather_mode=2),
             "tcgen05_single_cta": m._config(cta_group=1),
             "tcgen05_256_row_tiles": m._config(cta_group=3),
+            "tcgen05_one_launch_ffn": m._config(fused_ffn=2),
+            "tcgen05_one_launch_ffn_no_window": m._config(fused_ffn=2, fused_window=-1),
             "tcgen05_tokens_as_n": m._config(impl=m.MOK_IMPL_TCGEN05_TN)}[impl]
     out, st, rep = pu.full_parity(cfg, config=conf)
     print(cfg.name, impl, rep)
@@ -332,10 +335,37 @@ def test_argument_errors_launch_nothing():
     assert out0.shape == (0, cfg.H)
 
 
-def test_bounded_waits_report_a_timeout_and_leave_the_context_usable():
+MID = [
+    # several row groups per expert, ragged last tiles, a narrow last gate/up tile (I mod 128 = 64), an empty expert
+    MoEConfig("mid_groups", T=3000, H=512, E=6, k=3, I=320, I_s=0, bias="zipf", seed=91),
+    MoEConfig("mid_many", T=2048, H=576, E=40, k=4, I=256, I_s=128, bias="normal", seed=92),
+]
+
+
+@pytest.mark.parametrize("cfg", MID, ids=[c.name for c in MID])
+def test_one_launch_ffn_gives_the_bits_of_two_launches(cfg):
+    """Gate/up + SwiGLU + down in ONE persistent launch (down tiles wait on completion counters of the gate/up tiles):
+    every token against the oracle, and bit for bit the output of the two-launch path -- whatever the grid size and
+    the distance between a row group's gate/up tiles and its down tiles (none: every down tile has to wait; huge:
+    all down tiles at the end of the list)."""
+    m = mok()
+    d = inputs.make_inputs(cfg)
+    g = pu.upload(d)
+    out2, st, rep = pu.full_parity(cfg, d=d, g=g, config=m._config(fused_ffn=1, cta_group=3))
+    print(cfg.name, rep)
+    for kw in ({}, {"fused_window": -1}, {"fused_window": 1}, {"fused_window": 1 << 20}, {"grid": 1}, {"grid": 7},
+               {"grid": 37, "fused_window": -1}, {"tile_sched": 2}, {"tile_sched": 2, "fused_window": -1},
+               {"tile_sched": 2, "grid": 5, "fused_window": 40}):
+        out1 = pu.run_gpu(cfg, g, config=m._config(fused_ffn=2, **kw), stages=False)
+        assert torch.equal(out1.view(torch.int16), out2.view(torch.int16)), kw
+
+
+@pytest.mark.parametrize("fused,sched", [(0, 0), (2, 0), (2, 2)])
+def test_bounded_waits_report_a_timeout_and_leave_the_context_usable(fused, sched):
     """Failure detection without a fault: the test hook silences the gate/up GEMM's TMA producer, so its MMA issuer
     waits for operands that never come.  Every wait is bounded (2 ms here), the kernel records MOK_ERR_TIMEOUT, frees
-    its tensor memory and returns; the next call on the same context must be correct again."""
+    its tensor memory and returns; the next call on the same context must be correct again.  fused = 2: the same on
+    the one-launch expert FFN, where the down tiles' producers additionally wait for gate/up tiles that never finish."""
     m = mok()
     cfg = inputs.CONFIGS["tiny"]
     d = inputs.make_inputs(cfg)
@@ -343,7 +373,7 @@ def test_bounded_waits_report_a_timeout_and_leave_the_context_usable():
     ws = m.alloc_workspace(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k)
     good = pu.run_gpu(cfg, g, ws=ws, stages=False).clone()
     m.mok_moe_forward_ex(g["x"], g["W_r"], g["bias"], g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], cfg.k, ws,
-                         config=m._config(debug=m.MOK_DEBUG_STARVE))
+                         config=m._config(debug=m.MOK_DEBUG_STARVE, fused_ffn=fused, tile_sched=sched))
     assert m.mok_read_status(ws) == m.MOK_ERR_TIMEOUT
     again = pu.run_gpu(cfg, g, ws=ws, stages=False)
     assert torch.equal(good.view(torch.int16), again.view(torch.int16))
