@@ -95,12 +95,12 @@ typedef struct mok_config {
                              mok_workspace_bytes(macrobatch_tokens, ...); every macrobatch streams the expert weights
                              again.  Same bits as the single pass; counts / offsets / perm / inv_perm (tables of ONE
                              schedule) cannot be returned: MOK_ERR_UNSUPPORTED. */
-    int32_t fused_ffn;    /* routed experts, bf16: 0 = choose by shape, 1 = gate/up GEMM and down GEMM as two launches,
+    int32_t fused_ffn;    /* routed experts, bf16: 0 or 1 = gate/up GEMM and down GEMM as two launches (the default),
                              2 = ONE persistent launch over a list of gate/up tiles and down tiles; a down tile runs
                              once a per-row-tile completion counter, advanced by the gate/up epilogues, shows that its
                              rows of the gated activation exist (Section 3.2: megakernel, GPU-local synchronisation
                              instead of kernel boundaries).  Same bits either way. */
-    int32_t fused_window; /* fused_ffn: list positions between a row group's gate/up tiles and its down tiles (0 = two
+    int32_t fused_window; /* fused_ffn: list positions between a row group's gate/up tiles and its down tiles (0 = eight
                              grids' worth of tiles; -1 = none: directly behind them, which makes every down tile wait --
                              a test setting).  The list is handed out dynamically (each CTA draws the next position
                              from a global counter) unless tile_sched = 2, which walks it with stride grid. */

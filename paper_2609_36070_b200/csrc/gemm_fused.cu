@@ -32,8 +32,8 @@
 // Determinism: every output element is still produced by exactly one tile with a fixed k order, so the bits equal
 // those of the two separate launches whatever the interleaving (tested).
 //
-// Warp roles, shared-memory ring, tensor-memory use and the epilogue are those of gemm_tcgen05_m2.cu; during D tiles
-// the gather warps only keep the ring's arrival counts complete.
+// Shared-memory ring, tensor-memory use and the epilogue arithmetic are those of gemm_tcgen05_m2.cu; during D tiles the
+// gather warps skip ahead and the producer makes their arrivals on the ring's barriers.
 #include "mok_internal.cuh"
 #include "tc_ptx.cuh"
 #include "tensor_map.cuh"
@@ -51,7 +51,7 @@ constexpr int TM = 2 * BM;
 constexpr int TMEM_COLS = 512;
 constexpr int EPI_WARPS = 8;
 constexpr int GATHER_THREADS = 128;
-constexpr int THREADS = 64 + 32 * EPI_WARPS + GATHER_THREADS;     // 448
+constexpr int THREADS = 128 + 32 * EPI_WARPS + GATHER_THREADS;    // 512: four groups of four warps (see the kernel)
 constexpr int GROUP_TILES = 8;
 constexpr int SLAB_BYTES = 4096;
 constexpr int SMEM_CTRL = 256;
@@ -72,8 +72,7 @@ constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >
 __device__ __forceinline__ uint32_t idesc_n(int n) { return (IDESC & ~(0x3Fu << 17)) | ((uint32_t)(n >> 3) << 17); }
 
 struct Tile { int row0, valid, kind, e, n, mt; };
-__device__ __forceinline__ Tile read_tile(const int4* tiles, int L) {
-    const int4 d = __ldg(tiles + L);
+__device__ __forceinline__ Tile decode_tile(const int4 d) {
     Tile t;
     t.row0 = d.x;
     t.valid = d.y & 0xFFFF;
@@ -82,6 +81,27 @@ __device__ __forceinline__ Tile read_tile(const int4* tiles, int L) {
     t.n = (d.z >> 16) & 0xFFFF;
     t.mt = d.w;
     return t;
+}
+
+// The bounded mbarrier wait of tc_ptx.cuh, inlined: this kernel changes the register allocation of its warps
+// (setmaxnreg), and a real function call from regions with different register counts does not compile.
+__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, WsHeader* hdr, int site) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = globaltimer();
+    uint32_t spins = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++spins & 127u) == 0u) {
+            if (*abort_flag) return false;
+            const unsigned long long limit = hdr->wait_limit_us ? 1000ull * hdr->wait_limit_us : WAIT_LIMIT_NS;
+            if (globaltimer() - t0 > limit) {
+                *abort_flag = 1u;
+                atomicCAS(&hdr->status, 0, (int)MOK_ERR_TIMEOUT);
+                hdr->where = site;
+                return false;
+            }
+        }
+    }
+    return true;
 }
 
 // How a role walks over its tiles: static stride, or ids read from the scheduler warp's queue (bounded waits; an entry
@@ -99,7 +119,7 @@ struct TileSeq {
     __device__ __forceinline__ int first() { return DYN ? next(0) : (int)blockIdx.x; }
     __device__ __forceinline__ int next(int L) {
         if (!DYN) return L + gridDim.x;
-        bool ok = mbar_wait(smem_u32(&ctrl->q_full[slot]), ph, abort_flag, hdr, 30);
+        bool ok = wait_bar(smem_u32(&ctrl->q_full[slot]), ph, abort_flag, hdr, 30);
         if (warp_role) ok = __all_sync(0xffffffffu, ok);
         if (!ok) return total;
         const int t = *reinterpret_cast<volatile int32_t*>(&ctrl->q_tile[slot]);
@@ -107,6 +127,33 @@ struct TileSeq {
         if (!warp_role || (threadIdx.x & 31) == 0) mbar_arrive(smem_u32(&ctrl->q_empty[slot]));
         if (++slot == QSLOTS) { slot = 0; ph ^= 1u; }
         return t < 0 ? total : t;
+    }
+};
+
+// A role's walk over its tiles with the NEXT tile's descriptor already on its way: the 16-byte descriptor load of tile
+// i + 1 is issued when the role starts tile i, so no role stalls on it at a tile boundary.
+template <bool DYN>
+struct TileWalk {
+    TileSeq<DYN> seq;
+    const int4* tiles;
+    int total, L, Ln;
+    int4 d, dn;
+    __device__ __forceinline__ int4 fetch(int l) const { return l < total ? __ldg(tiles + l) : make_int4(0, 0, 0, 0); }
+    __device__ __forceinline__ TileWalk(Ctrl* c, volatile uint32_t* af, WsHeader* h, const int4* tl, int tot, bool wr)
+        : seq(c, af, h, tot, wr), tiles(tl), total(tot) {
+        L = seq.first();
+        d = fetch(L);
+        Ln = L < total ? seq.next(L) : total;
+        dn = fetch(Ln);
+    }
+    __device__ __forceinline__ bool valid() const { return L < total; }
+    __device__ __forceinline__ void advance() {
+        L = Ln;
+        d = dn;
+        if (L < total) {
+            Ln = seq.next(L);
+            dn = fetch(Ln);
+        }
     }
 };
 
@@ -256,8 +303,20 @@ struct FusedArgs {
     WsHeader* header;
 };
 
+// Registers are handed from the light roles to the epilogue (setmaxnreg, per group of four warps): the producer /
+// issuer / scheduler group and the gather group give up most of theirs, and the two epilogue groups get enough to hold
+// a whole 256-column accumulator row, so that an accumulator goes back to the MMA issuer right after its last TMEM read.
+template <int N>
+__device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N>
+__device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+constexpr int REGS_CONTROL = 56, REGS_GATHER = 88, REGS_EPILOGUE = 184;      // (56 + 88 + 2 * 184) * 128 = 65536
+
+//   warp 0 TMA producer | warp 1 MMA issuer (+ tensor-memory allocation) | warp 2 scheduler (dynamic mode) | warp 3 idle
+//   warps 4..7  epilogue of accumulator 0 (rows 0..127 of a tile)     warps 8..11 epilogue of accumulator 1
+//   warps 12..15 gather
 template <bool DYN>
-__global__ void __launch_bounds__(THREADS + (DYN ? 32 : 0), 1)
+__global__ void __launch_bounds__(THREADS, 1)
 fused_ffn_kernel(const __grid_constant__ CUtensorMap mapWgu, const __grid_constant__ CUtensorMap mapWgu64,
                  const __grid_constant__ CUtensorMap mapHst, const __grid_constant__ CUtensorMap mapHld,
                  const __grid_constant__ CUtensorMap mapWd, const __grid_constant__ CUtensorMap mapY,
@@ -304,196 +363,212 @@ fused_ffn_kernel(const __grid_constant__ CUtensorMap mapWgu, const __grid_consta
     tc_fence_after();
     const uint32_t tmem_base = ctrl->tmem_base;
 
-    if (warp == 0) {
-        // ------------------------------------------------------------------ TMA producer
-        if (lane == 0 && !a.starve) {
-            int s = 0;
-            uint32_t ph = 0;
-            long long d_ready = 0;
-            TileSeq<DYN> seq(ctrl, abort_flag, a.header, total, false);
-            for (int L = seq.first(); L < total; L = seq.next(L)) {
-                const Tile t = read_tile(a.tiles, L);
-                const bool two = t.valid > BM;
-                bool ok = true;
-                if (t.kind) {
-                    // every gate/up tile of these rows has stored h: n1 tiles x 4 epilogue warps per 128-row half
-                    const int need = a.n1 * (two ? 8 : 4);
-                    const int32_t* flag = a.ready + t.mt;
-                    if (ld_acquire(flag) < need) {
-                        const long long w0 = a.dbg ? clock64() : 0;
-                        const unsigned long long t0 = globaltimer();
-                        uint32_t spins = 0;
-                        while (ld_acquire(flag) < need) {
-                            __nanosleep(64);
-                            if ((++spins & 63u) == 0u) {
-                                if (*abort_flag) { ok = false; break; }
-                                const unsigned long long limit =
-                                    a.header->wait_limit_us ? 1000ull * a.header->wait_limit_us : WAIT_LIMIT_NS;
-                                if (globaltimer() - t0 > limit) {
-                                    *abort_flag = 1u;
-                                    atomicCAS(&a.header->status, 0, (int)MOK_ERR_TIMEOUT);
-                                    a.header->where = 40;
-                                    ok = false;
-                                    break;
+    if (warp < 4) {
+        reg_dec<REGS_CONTROL>();
+        if (warp == 0) {
+            // -------------------------------------------------------------- TMA producer
+            if (lane == 0 && !a.starve) {
+                int s = 0;
+                uint32_t ph = 0;
+                long long d_ready = 0;
+                int peek = 0;            // completion counter of the NEXT tile's rows, read during the current tile
+                TileWalk<DYN> w(ctrl, abort_flag, a.header, a.tiles, total, false);
+                for (; w.valid(); w.advance()) {
+                    const Tile t = decode_tile(w.d);
+                    const bool two = t.valid > BM;
+                    bool ok = true;
+                    if (t.kind) {
+                        // every gate/up tile of these rows has stored h: n1 tiles x 4 epilogue warps per 128-row half
+                        const int need = a.n1 * (two ? 8 : 4);
+                        const int32_t* flag = a.ready + t.mt;
+                        if (peek < need && ld_acquire(flag) < need) {
+                            const long long w0 = a.dbg ? clock64() : 0;
+                            const unsigned long long t0 = globaltimer();
+                            uint32_t spins = 0;
+                            while (ld_acquire(flag) < need) {
+                                __nanosleep(64);
+                                if ((++spins & 63u) == 0u) {
+                                    if (*abort_flag) { ok = false; break; }
+                                    const unsigned long long limit =
+                                        a.header->wait_limit_us ? 1000ull * a.header->wait_limit_us : WAIT_LIMIT_NS;
+                                    if (globaltimer() - t0 > limit) {
+                                        *abort_flag = 1u;
+                                        atomicCAS(&a.header->status, 0, (int)MOK_ERR_TIMEOUT);
+                                        a.header->where = 40;
+                                        ok = false;
+                                        break;
+                                    }
                                 }
                             }
+                            if (a.dbg) d_ready += clock64() - w0;
                         }
-                        if (a.dbg) d_ready += clock64() - w0;
+                        if (!ok) break;
+                        // the rows were written through the async proxy by other CTAs and are read through it below
+                        asm volatile("fence.proxy.async;" ::: "memory");
+                    }
+                    const int kblocks = t.kind ? a.kb2 : a.kb1;
+                    const bool narrow = !t.kind && narrow_last && t.n == a.n1 - 1;
+                    const int brow0 = t.kind ? t.e * a.H + t.n * BN : t.e * 2 * a.I + t.n * (BN / 2);
+                    const int brow1 = t.kind ? brow0 + BN / 2 : brow0 + a.I;
+                    peek = 0;
+                    for (int kb = 0; kb < kblocks; ++kb) {
+                        if (kb == (kblocks >> 1) && w.Ln < total) {   // the next tile's descriptor has arrived by now
+                            const Tile tn = decode_tile(w.dn);
+                            if (tn.kind) peek = ld_acquire(a.ready + tn.mt);
+                        }
+                        ok = wait_bar(smem_u32(&ctrl->empty[s]), ph ^ 1u, abort_flag, a.header, 1);
+                        if (!ok) break;
+                        const uint32_t full = smem_u32(&ctrl->full[s]);
+                        const uint32_t sa = base + s * STAGE_BYTES, sb = sa + 2 * A_BYTES;
+                        if (t.kind) {
+                            // (the gather threads have nothing to bring: their arrivals on the stage are made here)
+                            asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0], %1;" ::"r"(full), "r"((uint32_t)GATHER_THREADS) : "memory");
+                            mbar_expect_tx(full, B_BYTES + (two ? 2 : 1) * A_BYTES);
+                            tma_load_2d(sa, &mapHld, full, kb * BK, t.row0);
+                            if (two) tma_load_2d(sa + A_BYTES, &mapHld, full, kb * BK, t.row0 + BM);
+                            tma_load_2d(sb, &mapWd, full, kb * BK, brow0);
+                            tma_load_2d(sb + B_BYTES / 2, &mapWd, full, kb * BK, brow1);
+                        } else if (narrow) {
+                            mbar_expect_tx(full, B_BYTES / 2);
+                            tma_load_2d(sb, &mapWgu64, full, kb * BK, brow0);
+                            tma_load_2d(sb + B_BYTES / 4, &mapWgu64, full, kb * BK, brow1);
+                        } else {
+                            mbar_expect_tx(full, B_BYTES);
+                            tma_load_2d(sb, &mapWgu, full, kb * BK, brow0);
+                            tma_load_2d(sb + B_BYTES / 2, &mapWgu, full, kb * BK, brow1);
+                        }
+                        if (++s == STAGES) { s = 0; ph ^= 1u; }
                     }
                     if (!ok) break;
-                    // the rows were written through the async proxy by other CTAs and are read through it below
-                    asm volatile("fence.proxy.async;" ::: "memory");
                 }
-                const int kblocks = t.kind ? a.kb2 : a.kb1;
-                const bool narrow = !t.kind && narrow_last && t.n == a.n1 - 1;
-                const int brow0 = t.kind ? t.e * a.H + t.n * BN : t.e * 2 * a.I + t.n * (BN / 2);
-                const int brow1 = t.kind ? brow0 + BN / 2 : brow0 + a.I;
-                for (int kb = 0; kb < kblocks; ++kb) {
-                    ok = mbar_wait(smem_u32(&ctrl->empty[s]), ph ^ 1u, abort_flag, a.header, 1);
-                    if (!ok) break;
-                    const uint32_t full = smem_u32(&ctrl->full[s]);
-                    const uint32_t sa = base + s * STAGE_BYTES, sb = sa + 2 * A_BYTES;
-                    if (t.kind) {
-                        mbar_expect_tx(full, B_BYTES + (two ? 2 : 1) * A_BYTES);
-                        tma_load_2d(sa, &mapHld, full, kb * BK, t.row0);
-                        if (two) tma_load_2d(sa + A_BYTES, &mapHld, full, kb * BK, t.row0 + BM);
-                        tma_load_2d(sb, &mapWd, full, kb * BK, brow0);
-                        tma_load_2d(sb + B_BYTES / 2, &mapWd, full, kb * BK, brow1);
-                    } else if (narrow) {
-                        mbar_expect_tx(full, B_BYTES / 2);
-                        tma_load_2d(sb, &mapWgu64, full, kb * BK, brow0);
-                        tma_load_2d(sb + B_BYTES / 4, &mapWgu64, full, kb * BK, brow1);
-                    } else {
-                        mbar_expect_tx(full, B_BYTES);
-                        tma_load_2d(sb, &mapWgu, full, kb * BK, brow0);
-                        tma_load_2d(sb + B_BYTES / 2, &mapWgu, full, kb * BK, brow1);
-                    }
-                    if (++s == STAGES) { s = 0; ph ^= 1u; }
-                }
-                if (!ok) break;
+                if (a.dbg) atomicAdd(&a.header->dbg[2][DBG_PROD_WAIT_EMPTY], (unsigned long long)d_ready);
             }
-            if (a.dbg) atomicAdd(&a.header->dbg[2][DBG_PROD_WAIT_EMPTY], (unsigned long long)d_ready);
-        }
-        __syncwarp();
-    } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            int s = 0;
-            uint32_t ph = 0, ap0 = 0, ap1 = 0;
-            const bool dbg = a.dbg != 0;
-            long long d_full[2] = {0, 0}, d_tempty[2] = {0, 0}, d_kb[2] = {0, 0}, d_rows[2] = {0, 0}, d_tot[2] = {0, 0};
-            const unsigned long long d_ns0 = dbg ? globaltimer() : 0ull;
-            const long long d_c0 = dbg ? clock64() : 0;
-            TileSeq<DYN> seq(ctrl, abort_flag, a.header, total, false);
-            for (int L = seq.first(); L < total; L = seq.next(L)) {
-                const Tile t = read_tile(a.tiles, L);
-                const bool two = t.valid > BM;
-                const int kblocks = t.kind ? a.kb2 : a.kb1;
-                uint32_t idesc = IDESC;
-                if (t.kind) {
-                    if (a.H - t.n * BN < BN) idesc = idesc_n((a.H - t.n * BN + 15) & ~15);
-                } else if (narrow_last && t.n == a.n1 - 1) {
-                    idesc = idesc_n(BN / 2);
-                }
-                const long long tile0 = dbg ? clock64() : 0;
-                long long w0 = tile0;
-                bool ok = mbar_wait(smem_u32(&ctrl->tempty[0]), ap0 ^ 1u, abort_flag, a.header, 2);
-                if (dbg) d_tempty[t.kind] += clock64() - w0;
-                if (!ok) break;
-                tc_fence_after();
-                const uint32_t d0 = tmem_base, d1 = tmem_base + BN;
-                for (int kb = 0; kb < kblocks; ++kb) {
-                    if (dbg) w0 = clock64();
-                    ok = mbar_wait(smem_u32(&ctrl->full[s]), ph, abort_flag, a.header, 3);
-                    if (dbg) { d_full[t.kind] += clock64() - w0; d_kb[t.kind] += two ? 2 : 1; }
+        } else if (warp == 1) {
+            // -------------------------------------------------------------- MMA issuer
+            if (lane == 0) {
+                int s = 0;
+                uint32_t ph = 0, ap0 = 0, ap1 = 0;
+                const bool dbg = a.dbg != 0;
+                // debug counters: index 0 = gate/up tiles, 1 = down tiles
+                long long d_full0 = 0, d_full1 = 0, d_te0 = 0, d_te1 = 0, d_kb0 = 0, d_kb1 = 0, d_rows0 = 0, d_rows1 = 0,
+                          d_tot0 = 0, d_tot1 = 0;
+                const unsigned long long d_ns0 = dbg ? globaltimer() : 0ull;
+                const long long d_c0 = dbg ? clock64() : 0;
+                TileWalk<DYN> w(ctrl, abort_flag, a.header, a.tiles, total, false);
+                for (; w.valid(); w.advance()) {
+                    const Tile t = decode_tile(w.d);
+                    const bool two = t.valid > BM;
+                    const int kblocks = t.kind ? a.kb2 : a.kb1;
+                    uint32_t idesc = IDESC;
+                    if (t.kind) {
+                        if (a.H - t.n * BN < BN) idesc = idesc_n((a.H - t.n * BN + 15) & ~15);
+                    } else if (narrow_last && t.n == a.n1 - 1) {
+                        idesc = idesc_n(BN / 2);
+                    }
+                    const long long tile0 = dbg ? clock64() : 0;
+                    long long w0 = tile0, w_full = 0, w_te = 0;
+                    bool ok = wait_bar(smem_u32(&ctrl->tempty[0]), ap0 ^ 1u, abort_flag, a.header, 2);
+                    if (dbg) w_te += clock64() - w0;
                     if (!ok) break;
                     tc_fence_after();
-                    const uint32_t sa = base + s * STAGE_BYTES;
-                    const uint64_t a0 = make_smem_desc(sa), a1 = make_smem_desc(sa + A_BYTES);
-                    const uint64_t bd = make_smem_desc(sa + 2 * A_BYTES);
-#pragma unroll
-                    for (int j = 0; j < BK / UMMA_K; ++j)
-                        tc_mma<1>(d0, a0 + (uint64_t)(j * 2), bd + (uint64_t)(j * 2), idesc, (kb | j) ? 1u : 0u);
-                    if (kb == kblocks - 1) { tc_commit<1>(smem_u32(&ctrl->tfull[0])); ap0 ^= 1u; }
-                    if (two) {
-                        if (kb == 0) {
-                            if (dbg) w0 = clock64();
-                            ok = mbar_wait(smem_u32(&ctrl->tempty[1]), ap1 ^ 1u, abort_flag, a.header, 8);
-                            if (dbg) d_tempty[t.kind] += clock64() - w0;
-                            if (!ok) break;
-                            tc_fence_after();
-                        }
+                    const uint32_t d0 = tmem_base, d1 = tmem_base + BN;
+                    for (int kb = 0; kb < kblocks; ++kb) {
+                        if (dbg) w0 = clock64();
+                        ok = wait_bar(smem_u32(&ctrl->full[s]), ph, abort_flag, a.header, 3);
+                        if (dbg) w_full += clock64() - w0;
+                        if (!ok) break;
+                        tc_fence_after();
+                        const uint32_t sa = base + s * STAGE_BYTES;
+                        const uint64_t a0 = make_smem_desc(sa), a1 = make_smem_desc(sa + A_BYTES);
+                        const uint64_t bd = make_smem_desc(sa + 2 * A_BYTES);
 #pragma unroll
                         for (int j = 0; j < BK / UMMA_K; ++j)
-                            tc_mma<1>(d1, a1 + (uint64_t)(j * 2), bd + (uint64_t)(j * 2), idesc, (kb | j) ? 1u : 0u);
+                            tc_mma<1>(d0, a0 + (uint64_t)(j * 2), bd + (uint64_t)(j * 2), idesc, (kb | j) ? 1u : 0u);
+                        if (kb == kblocks - 1) { tc_commit<1>(smem_u32(&ctrl->tfull[0])); ap0 ^= 1u; }
+                        if (two) {
+                            if (kb == 0) {
+                                if (dbg) w0 = clock64();
+                                ok = wait_bar(smem_u32(&ctrl->tempty[1]), ap1 ^ 1u, abort_flag, a.header, 8);
+                                if (dbg) w_te += clock64() - w0;
+                                if (!ok) break;
+                                tc_fence_after();
+                            }
+#pragma unroll
+                            for (int j = 0; j < BK / UMMA_K; ++j)
+                                tc_mma<1>(d1, a1 + (uint64_t)(j * 2), bd + (uint64_t)(j * 2), idesc, (kb | j) ? 1u : 0u);
+                        }
+                        tc_commit<1>(smem_u32(&ctrl->empty[s]));
+                        if (++s == STAGES) { s = 0; ph ^= 1u; }
                     }
-                    tc_commit<1>(smem_u32(&ctrl->empty[s]));
-                    if (++s == STAGES) { s = 0; ph ^= 1u; }
+                    if (!ok) break;
+                    if (two) { tc_commit<1>(smem_u32(&ctrl->tfull[1])); ap1 ^= 1u; }
+                    if (dbg) {
+                        const long long dt = clock64() - tile0, units = (long long)(two ? 2 : 1) * kblocks;
+                        if (t.kind) { d_full1 += w_full; d_te1 += w_te; d_kb1 += units; d_rows1 += (long long)t.valid * kblocks; d_tot1 += dt; }
+                        else        { d_full0 += w_full; d_te0 += w_te; d_kb0 += units; d_rows0 += (long long)t.valid * kblocks; d_tot0 += dt; }
+                    }
                 }
-                if (!ok) break;
-                if (two) { tc_commit<1>(smem_u32(&ctrl->tfull[1])); ap1 ^= 1u; }
-                if (dbg) { d_rows[t.kind] += (long long)t.valid * kblocks; d_tot[t.kind] += clock64() - tile0; }
+                if (dbg) {
+                    const unsigned long long ns = globaltimer() - d_ns0, cyc = (unsigned long long)(clock64() - d_c0);
+                    {   // slot 0: the whole kernel (imbalance of the tile hand-out, clock)
+                        unsigned long long* d = a.header->dbg[0];
+                        atomicAdd(d + DBG_MMA_TOTAL, cyc);
+                        atomicMax(d + DBG_MMA_TOTAL_MAX, cyc);
+                        atomicAdd(d + DBG_MMA_TOTAL_NS, ns);
+                        atomicAdd(d + DBG_CTAS, 1ull);
+                    }
+                    const double both = (double)(d_tot0 + d_tot1);
+                    for (int q = 0; q < 2; ++q) {
+                        unsigned long long* d = a.header->dbg[1 + q];
+                        const long long tot = q ? d_tot1 : d_tot0;
+                        // the CTA's wall time is split between the two kinds in proportion to the cycles spent in their tiles
+                        atomicAdd(d + DBG_MMA_WAIT_FULL, (unsigned long long)(q ? d_full1 : d_full0));
+                        atomicAdd(d + DBG_MMA_WAIT_TEMPTY, (unsigned long long)(q ? d_te1 : d_te0));
+                        atomicAdd(d + DBG_MMA_TOTAL, (unsigned long long)tot);
+                        atomicMax(d + DBG_MMA_TOTAL_MAX, (unsigned long long)tot);
+                        atomicAdd(d + DBG_MMA_TOTAL_NS, both > 0 ? (unsigned long long)((double)ns * (double)tot / both) : 0ull);
+                        atomicAdd(d + DBG_KBLOCKS, (unsigned long long)(q ? d_kb1 : d_kb0));
+                        atomicAdd(d + DBG_ROWS_KB, (unsigned long long)(q ? d_rows1 : d_rows0));
+                        atomicAdd(d + DBG_CTAS, 1ull);
+                    }
+                }
             }
-            if (dbg) {
-                const unsigned long long ns = globaltimer() - d_ns0, cyc = (unsigned long long)(clock64() - d_c0);
-                {   // slot 0: the whole kernel (imbalance of the tile -> CTA rule, clock)
-                    unsigned long long* d = a.header->dbg[0];
-                    atomicAdd(d + DBG_MMA_TOTAL, cyc);
-                    atomicMax(d + DBG_MMA_TOTAL_MAX, cyc);
-                    atomicAdd(d + DBG_MMA_TOTAL_NS, ns);
-                    atomicAdd(d + DBG_CTAS, 1ull);
-                }
-                for (int q = 0; q < 2; ++q) {
-                    unsigned long long* d = a.header->dbg[1 + q];
-                    // the CTA's time is split between the two kinds in proportion to the cycles spent in their tiles
-                    const unsigned long long share = d_tot[0] + d_tot[1] > 0 ? (unsigned long long)d_tot[q] : 0ull;
-                    const unsigned long long ns_q = d_tot[0] + d_tot[1] > 0
-                        ? (unsigned long long)((double)ns * (double)d_tot[q] / (double)(d_tot[0] + d_tot[1])) : 0ull;
-                    atomicAdd(d + DBG_MMA_WAIT_FULL, (unsigned long long)d_full[q]);
-                    atomicAdd(d + DBG_MMA_WAIT_TEMPTY, (unsigned long long)d_tempty[q]);
-                    atomicAdd(d + DBG_MMA_TOTAL, share);
-                    atomicMax(d + DBG_MMA_TOTAL_MAX, share);
-                    atomicAdd(d + DBG_MMA_TOTAL_NS, ns_q);
-                    atomicAdd(d + DBG_KBLOCKS, (unsigned long long)d_kb[q]);
-                    atomicAdd(d + DBG_ROWS_KB, (unsigned long long)d_rows[q]);
-                    atomicAdd(d + DBG_CTAS, 1ull);
+        } else if (DYN && warp == 2) {
+            // -------------------------------------------------------------- scheduler (dynamic mode)
+            if (lane == 0) {
+                // draws list positions in order from one global counter, a few tiles ahead of the roles.  Whoever draws
+                // a position runs, and everything a down tile waits for sits at smaller positions, which were drawn before.
+                int slot = 0;
+                uint32_t qph = 0;
+                for (;;) {
+                    const int L = atomicAdd(a.next_tile, 1);
+                    if (!wait_bar(smem_u32(&ctrl->q_empty[slot]), qph ^ 1u, abort_flag, a.header, 32)) break;
+                    *reinterpret_cast<volatile int32_t*>(&ctrl->q_tile[slot]) = L < total ? L : -1;
+                    mbar_arrive(smem_u32(&ctrl->q_full[slot]));
+                    if (++slot == QSLOTS) { slot = 0; qph ^= 1u; }
+                    if (L >= total) break;
                 }
             }
         }
         __syncwarp();
-    } else if (DYN && warp == THREADS / 32) {
-        // ------------------------------------------------------------------ scheduler warp (dynamic mode)
-        if (lane == 0) {
-            // draws list positions in order from one global counter, a few tiles ahead of the roles.  Whoever draws a
-            // position runs, and everything a down tile waits for sits at smaller positions, which were drawn before.
-            int slot = 0;
-            uint32_t qph = 0;
-            for (;;) {
-                const int L = atomicAdd(a.next_tile, 1);
-                if (!mbar_wait(smem_u32(&ctrl->q_empty[slot]), qph ^ 1u, abort_flag, a.header, 32)) break;
-                *reinterpret_cast<volatile int32_t*>(&ctrl->q_tile[slot]) = L < total ? L : -1;
-                mbar_arrive(smem_u32(&ctrl->q_full[slot]));
-                if (++slot == QSLOTS) { slot = 0; qph ^= 1u; }
-                if (L >= total) break;
-            }
-        }
-        __syncwarp();
-    } else if (warp >= 2 + EPI_WARPS) {
+    } else if (warp >= 4 + EPI_WARPS) {
         // ------------------------------------------------------------------ gather warps (pull dispatch)
-        const int gw = warp - (2 + EPI_WARPS), sub = lane >> 3, chunk = lane & 7;
+        reg_dec<REGS_GATHER>();
+        const int gw = warp - (4 + EPI_WARPS), sub = lane >> 3, chunk = lane & 7;
         int s = 0;
         uint32_t ph = 0;
-        TileSeq<DYN> seq(ctrl, abort_flag, a.header, total, true);
-        for (int L = seq.first(); L < total; L = seq.next(L)) {
-            const Tile t = read_tile(a.tiles, L);
+        TileWalk<DYN> w(ctrl, abort_flag, a.header, a.tiles, total, true);
+        for (; w.valid(); w.advance()) {
+            const Tile t = decode_tile(w.d);
             bool ok = true;
             if (t.kind) {
-                // down tile: both operands come by TMA; these threads only complete the ring's arrival counts
+                // down tile: both operands come by TMA and the producer makes these threads' arrivals for them.  The warp
+                // still follows the ring stage by stage (one polling lane): a parity wait is only meaningful while the
+                // waiter is at most one phase ahead of the barrier, so it must not jump over the tile's stages.
                 for (int kb = 0; kb < a.kb2; ++kb) {
-                    ok = mbar_wait(smem_u32(&ctrl->empty[s]), ph ^ 1u, abort_flag, a.header, 5);
-                    ok = __all_sync(0xffffffffu, ok);
+                    if (lane == 0) ok = wait_bar(smem_u32(&ctrl->empty[s]), ph ^ 1u, abort_flag, a.header, 5);
+                    ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
                     if (!ok) break;
-                    mbar_arrive(smem_u32(&ctrl->full[s]));
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
                 if (!ok) break;
@@ -504,7 +579,7 @@ fused_ffn_kernel(const __grid_constant__ CUtensorMap mapWgu, const __grid_consta
             uint32_t live = 0u;
             int tok[16];
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
+            for (int i = 0; i < 16; ++i) {   // sixteen independent loads (a pad row reads the tile's last real row id)
                 const int r = (i >> 3) * BM + gw * 32 + (i & 7) * 4 + sub;
                 tok[i] = __ldg(a.row_token + t.row0 + min(r, t.valid - 1));
             }
@@ -515,7 +590,7 @@ fused_ffn_kernel(const __grid_constant__ CUtensorMap mapWgu, const __grid_consta
                 if (r < t.valid) live |= 1u << i;
             }
             for (int kb = 0; kb < a.kb1; ++kb) {
-                ok = mbar_wait(smem_u32(&ctrl->empty[s]), ph ^ 1u, abort_flag, a.header, 5);
+                ok = wait_bar(smem_u32(&ctrl->empty[s]), ph ^ 1u, abort_flag, a.header, 5);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 const uint32_t sa = base + s * STAGE_BYTES;
@@ -525,7 +600,7 @@ fused_ffn_kernel(const __grid_constant__ CUtensorMap mapWgu, const __grid_consta
                     if (i < 8 || two) {
                         const int rr = gw * 32 + (i & 7) * 4 + sub;
                         const uint32_t dst = sa + (i >> 3) * A_BYTES + rr * 128 + ((chunk ^ (rr & 7)) << 4);
-                        const bool on = in_k && ((live >> i) & 1u);
+                        const bool on = in_k && ((live >> i) & 1u);    // pad rows and the K tail are written as zeros
                         cp_async_16(dst, on ? (const void*)(src[i] + kb * BK) : (const void*)a.x, on ? 16u : 0u);
                     }
                 }
@@ -537,89 +612,99 @@ fused_ffn_kernel(const __grid_constant__ CUtensorMap mapWgu, const __grid_consta
         asm volatile("cp.async.wait_all;" ::: "memory");
     } else {
         // ------------------------------------------------------------------ epilogue warps
-        const int acc = (warp - 2) >> 2;
-        const int quad = warp & 3;
-        const uint32_t slab = base + STAGES * STAGE_BYTES + (warp - 2) * SLAB_BYTES;
+        reg_inc<REGS_EPILOGUE>();
+        const int acc = (warp - 4) >> 2;
+        const int quad = warp & 3;                            // TMEM lane quadrant this warp may access
+        const uint32_t slab = base + STAGES * STAGE_BYTES + (warp - 4) * SLAB_BYTES;
         uint32_t aph = 0;
-        TileSeq<DYN> seq(ctrl, abort_flag, a.header, total, true);
-        for (int L = seq.first(); L < total; L = seq.next(L)) {
-            const Tile t = read_tile(a.tiles, L);
+        auto hand_back = [&]() {                               // the accumulator goes back to the MMA issuer
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&ctrl->tempty[acc]));
+        };
+        // one pass: 32 rows x 64 columns of packed bf16 through this warp's swizzled slab and out by TMA
+        auto store_pass = [&](const uint32_t* v, const CUtensorMap* map, int col, int n_cols, int row) {
+            if (lane == 0) tma_store_wait_read();             // the slab's previous store has been read out
+            __syncwarp();
+            const uint32_t line = slab + lane * 128;
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+                st_shared_v4(line + ((q ^ (lane & 7)) << 4), v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) {
+                if (col < n_cols) tma_store_2d(map, slab, col, row);
+                tma_store_commit();
+            }
+        };
+        TileWalk<DYN> w(ctrl, abort_flag, a.header, a.tiles, total, true);
+        for (; w.valid(); w.advance()) {
+            const Tile t = decode_tile(w.d);
             if (acc == 1 && t.valid <= BM) continue;
-            bool ok = mbar_wait(smem_u32(&ctrl->tfull[acc]), aph, abort_flag, a.header, 4);
+            bool ok = wait_bar(smem_u32(&ctrl->tfull[acc]), aph, abort_flag, a.header, 4);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             aph ^= 1u;
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * BN);
             const int row = t.row0 + acc * BM + quad * 32;
-            const bool swiglu = !t.kind;
-            const bool narrow = swiglu && narrow_last && t.n == a.n1 - 1;
-            const int passes = swiglu ? (narrow ? 1 : 2) : 4;
-            const uint32_t up_off = narrow ? BN / 4 : BN / 2;
-            const int c0 = swiglu ? t.n * (BN / 2) : t.n * BN;
-            const int n_cols = swiglu ? a.I : a.H;
-            const CUtensorMap* mapC = swiglu ? &mapHst : &mapY;
-            uint32_t cur[32], nxt[32];
-            auto hand_back = [&]() {
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&ctrl->tempty[acc]));
-            };
-            auto load_pass = [&](int pass, uint32_t (&o)[32]) {
+            if (t.kind) {
+                // down tile: the whole 256-column accumulator row is read and packed first, the accumulator goes back to
+                // the MMA issuer, and only then do the four 64-column passes through the slab start
+                uint32_t o[128];
 #pragma unroll
-                for (int c = 0; c < 64; c += 32) {
-                    if (swiglu) {
+                for (int c = 0; c < BN; c += 32) {
+                    uint32_t r[32];
+                    tc_ld32(taddr + c, r);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 16; ++i)
+                        o[(c >> 1) + i] = pack_bf16(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
+                }
+                hand_back();
+#pragma unroll
+                for (int pass = 0; pass < 4; ++pass) store_pass(o + pass * 32, &mapY, t.n * BN + pass * 64, a.H, row);
+            } else {
+                // gate/up tile: silu(g) * u from columns c and c + 128 (c + 64 of a narrow last tile), 64 output columns
+                // per pass; the next pass is read and computed before waiting for the slab of the current one
+                const bool narrow = narrow_last && t.n == a.n1 - 1;
+                const int passes = narrow ? 1 : 2;
+                const uint32_t up_off = narrow ? BN / 4 : BN / 2;
+                uint32_t cur[32], nxt[32];
+                auto load_pass = [&](int pass, uint32_t (&o)[32]) {
+#pragma unroll
+                    for (int c = 0; c < 64; c += 32) {
                         uint32_t g[32], u[32];
                         tc_ld32(taddr + pass * 64 + c, g);
                         tc_ld32(taddr + up_off + pass * 64 + c, u);
                         tc_wait_ld();
-                        if (pass == passes - 1 && c == 32) hand_back();
+                        if (pass == passes - 1 && c == 32) hand_back();   // the tile's last TMEM read: arithmetic comes after
 #pragma unroll
                         for (int i = 0; i < 16; ++i)
-                            o[(c >> 1) + i] = pack_bf16(tc::swiglu(__uint_as_float(g[2 * i]), __uint_as_float(u[2 * i])),
-                                                        tc::swiglu(__uint_as_float(g[2 * i + 1]), __uint_as_float(u[2 * i + 1])));
-                    } else {
-                        uint32_t r[32];
-                        tc_ld32(taddr + pass * 64 + c, r);
-                        tc_wait_ld();
-                        if (pass == passes - 1 && c == 32) hand_back();
-#pragma unroll
-                        for (int i = 0; i < 16; ++i)
-                            o[(c >> 1) + i] = pack_bf16(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
+                            o[(c >> 1) + i] = pack_bf16(swiglu(__uint_as_float(g[2 * i]), __uint_as_float(u[2 * i])),
+                                                        swiglu(__uint_as_float(g[2 * i + 1]), __uint_as_float(u[2 * i + 1])));
                     }
+                };
+                load_pass(0, nxt);
+#pragma unroll
+                for (int pass = 0; pass < 2; ++pass) {
+                    if (pass >= passes) break;
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) cur[i] = nxt[i];
+                    if (pass + 1 < passes) load_pass(pass + 1, nxt);
+                    store_pass(cur, &mapHst, t.n * (BN / 2) + pass * 64, a.I, row);
                 }
-            };
-            load_pass(0, nxt);
-#pragma unroll
-            for (int pass = 0; pass < 4; ++pass) {
-                if (pass >= passes) break;
-#pragma unroll
-                for (int i = 0; i < 32; ++i) cur[i] = nxt[i];
-                if (pass + 1 < passes) load_pass(pass + 1, nxt);
-                if (lane == 0) tma_store_wait_read();
-                __syncwarp();
-                const uint32_t line = slab + lane * 128;
-#pragma unroll
-                for (int v = 0; v < 8; ++v)
-                    st_shared_v4(line + ((v ^ (lane & 7)) << 4), cur[4 * v], cur[4 * v + 1], cur[4 * v + 2], cur[4 * v + 3]);
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                __syncwarp();
                 if (lane == 0) {
-                    const int col = c0 + pass * 64;
-                    if (col < n_cols) tma_store_2d(mapC, slab, col, row);
-                    tma_store_commit();
+                    // h of this warp's 32 rows is on its way: wait until the stores have completed (not only left shared
+                    // memory), then publish one arrival for the M tile.  Release at GPU scope after a proxy fence: the
+                    // down tiles read these rows through the async proxy from other SMs.
+                    tma_store_wait_all();
+                    asm volatile("fence.proxy.async;" ::: "memory");
+                    __threadfence();
+                    asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(a.ready + t.mt) : "memory");
                 }
+                __syncwarp();
             }
-            if (swiglu && lane == 0) {
-                // h of this warp's 32 rows is on its way: wait until the stores have completed (not only left shared
-                // memory), then publish one arrival for the M tile.  Release at GPU scope after a proxy fence: the down
-                // tiles read these rows through the async proxy from other SMs.
-                tma_store_wait_all();
-                asm volatile("fence.proxy.async;" ::: "memory");
-                __threadfence();
-                asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(a.ready + t.mt) : "memory");
-            }
-            __syncwarp();
         }
         if (lane == 0) tma_store_wait_all();
         __syncwarp();
@@ -661,7 +746,7 @@ static cudaError_t launch_kernel(int grid, cudaStream_t s, const CUtensorMap& m0
     attr[0].id = cudaLaunchAttributeCooperative;
     attr[0].val.cooperative = 1;
     cfg.gridDim = dim3(grid);
-    cfg.blockDim = dim3(THREADS + (DYN ? 32 : 0));
+    cfg.blockDim = dim3(THREADS);
     cfg.dynamicSmemBytes = SMEM_BYTES;
     cfg.stream = s;
     cfg.attrs = attr;
@@ -670,7 +755,8 @@ static cudaError_t launch_kernel(int grid, cudaStream_t s, const CUtensorMap& m0
 }
 
 // Host side.  `window_tiles`: distance (in list positions) between a group's gate/up tiles and its down tiles; 0 = the
-// default of two grids' worth of tiles, -1 = none (a group's down tiles directly behind its gate/up tiles).
+// default of eight grids' worth of tiles (measured: the down tiles then never wait and still find h in L2), -1 = none
+// (a group's down tiles directly behind its gate/up tiles).
 cudaError_t launch_fused_ffn(const __nv_bfloat16* x, int T, int H, int I, int E, const __nv_bfloat16* Wgu,
                              const __nv_bfloat16* Wd, const WsLayout& L, char* ws, int grid, int window_tiles, bool dynamic,
                              bool dbg, bool starve, cudaStream_t s) {
@@ -682,7 +768,7 @@ cudaError_t launch_fused_ffn(const __nv_bfloat16* x, int T, int H, int I, int E,
     if (grid <= 0 || grid > sm_count) grid = sm_count;
     WsHeader* hdr = reinterpret_cast<WsHeader*>(ws + L.header);
     const int n1 = (I + BN / 2 - 1) / (BN / 2), n2 = (H + BN - 1) / BN;
-    if (window_tiles == 0) window_tiles = 2 * grid;
+    if (window_tiles == 0) window_tiles = 8 * grid;
     const int window = window_tiles < 0 ? 0 : (window_tiles + n1 - 1) / n1;      // in M tiles
     int4* tiles = reinterpret_cast<int4*>(ws + L.ftiles);
     int32_t* ready = reinterpret_cast<int32_t*>(ws + L.ready);
