@@ -49,6 +49,10 @@ def parse():
     p.add_argument("--config", default=DEFAULT_WORKLOAD)
     p.add_argument("--impl", default="mok", choices=["mok", "reference"])
     p.add_argument("--tokens", type=int, default=0, help="override T (small-T sweeps)")
+    p.add_argument("--experts", type=int, default=0,
+                   help="override E: with --tokens, a scaled copy of a workload (same H, I, k and rows per expert) that is "
+                        "small enough for a profiler capture")
+    p.add_argument("--fused-ffn", type=int, default=0, help="2: routed gate/up + down GEMM as one persistent launch")
     p.add_argument("--cpu-sample", type=int, default=0, help="tokens of the CPU-oracle sample (0 = auto)")
     p.add_argument("--no-cpu-baseline", action="store_true")
     p.add_argument("--per-config", default="auto",
@@ -331,7 +335,7 @@ class Layer:
     def conf(self, **kw):
         a = self.args
         base = dict(impl=a.gemm, gather_mode=a.gather_mode, cta_group=a.cta_group, precision=self.prec,
-                    tile_sched=a.tile_sched)
+                    tile_sched=a.tile_sched, fused_ffn=a.fused_ffn)
         base.update(kw)
         return self.mok._config(**base)
 
@@ -389,6 +393,40 @@ class Layer:
         res = {s: (sum(c[s] for c in stage) / len(stage), _median([c[s] for c in stage]), min(c[s] for c in stage))
                for s in mok.STAGES}
         return res, (t0, t1)
+
+    def one_launch_ab(self, rounds=3, block_s=0.3):
+        """The routed expert FFN as two launches (gate/up GEMM, down GEMM) against ONE persistent launch
+        (config.fused_ffn = 2), alternating in blocks of about `block_s` seconds so that both see the same board state.
+        Returns mean step times in ms (first round dropped), or None where the one-launch kernel does not apply."""
+        torch = self.torch
+        a = self.args
+        if self.mx or a.gemm != 0 or a.cta_group in (1, 2) or a.tile_sched == 1 or (self.cfg.I + 127) // 128 > 32:
+            return None
+        confs = {"two_launches": self.conf(fused_ffn=1), "one_launch": self.conf(fused_ffn=2)}
+        for c in confs.values():
+            self.step(c)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        self.step(confs["two_launches"])
+        e1.record()
+        torch.cuda.synchronize()
+        n = int(max(3, min(500, block_s * 1e3 / max(e0.elapsed_time(e1), 1e-3))))
+        acc = {k: [] for k in confs}
+        for r in range(rounds + 1):
+            for name, c in confs.items():
+                e0.record()
+                for _ in range(n):
+                    self.step(c)
+                e1.record()
+                torch.cuda.synchronize()
+                if r > 0:
+                    acc[name].append(e0.elapsed_time(e1) / n)
+        self.check_status()
+        out = {k + "_ms": sum(v) / len(v) for k, v in acc.items()}
+        out.update({"rounds": rounds, "steps_per_block": n,
+                    "how": "blocks of the two variants alternate in one process; whole-step time, mean over the rounds"})
+        return out
 
     def counters(self):
         """Device-side counters of the GEMM kernels (one extra step with config.debug = 1), reduced to the figures the
@@ -467,6 +505,9 @@ def measure(layer, steps, warmup, barrier, sampler_windows, pk, with_counters):
     if with_counters and not layer.mx and layer.args.gemm == 0:
         rec["counters"] = layer.counters()
         layer.check_status()
+        ab = layer.one_launch_ab()
+        if ab is not None:
+            rec["one_launch_ffn"] = ab
     return rec
 
 
@@ -521,6 +562,9 @@ def main():
     cfg = inputs.CONFIGS[args.config]
     if args.tokens:
         cfg = cfg.with_tokens(args.tokens)
+    if args.experts:
+        import dataclasses
+        cfg = dataclasses.replace(cfg, E=args.experts, name=f"{cfg.name}_E{args.experts}")
     if args.impl == "reference":
         run_reference(args, cfg, rank)
         return
@@ -629,7 +673,7 @@ def main():
 
     # ------------------------------------------------------------------ small-T sweep of the default workload (N = 1)
     sweep = None
-    if world == 1 and not args.no_sweep and args.config == DEFAULT_WORKLOAD and not args.tokens:
+    if world == 1 and not args.no_sweep and args.config == DEFAULT_WORKLOAD and not args.tokens and not args.experts:
         sweep = []
         for T in (64, 512, 4096):
             v = layer.view(T)
@@ -658,7 +702,7 @@ def main():
     # ------------------------------------------------------------------ the other workloads (N = 1)
     names = []
     if args.per_config == "auto":
-        if world == 1 and args.config == DEFAULT_WORKLOAD and not args.tokens:
+        if world == 1 and args.config == DEFAULT_WORKLOAD and not args.tokens and not args.experts:
             names = [n for n in inputs.CONFIG_ORDER if n != args.config]
     elif args.per_config != "none":
         names = [n for n in args.per_config.split(",") if n]
@@ -729,7 +773,7 @@ def main():
     roofline["traffic"] = None if (mx or tr is None) else tr["bytes"] * tr["scale"]
     if tr is not None and not mx:
         roofline["traffic_source"] = f"{tr['source']} (ncu capture x {tr['scale']})"
-    conf = mok._config(impl=args.gemm, gather_mode=args.gather_mode, cta_group=args.cta_group,
+    conf = mok._config(impl=args.gemm, gather_mode=args.gather_mode, cta_group=args.cta_group, fused_ffn=args.fused_ffn,
                        precision=mok.MOK_PRECISION_MXFP8 if mx else mok.MOK_PRECISION_BF16, tile_sched=args.tile_sched)
     line = {
         "metric": METRIC, "value": main_rec["tokens_per_s"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -755,6 +799,8 @@ def main():
         line["sustained"] = main_rec["sustained"]
     if "counters" in main_rec:
         line["counters"] = main_rec["counters"]
+    if "one_launch_ffn" in main_rec:
+        line["one_launch_ffn"] = main_rec["one_launch_ffn"]
     if main_counts is not None:
         line["load"] = {"max_count": int(main_counts.max()), "empty_experts": int((main_counts == 0).sum()),
                         "rows_padded_to_128": int(((main_counts + 127) // 128 * 128).sum()), "rows": int(main_counts.sum())}
