@@ -104,6 +104,11 @@ typedef struct mok_config {
                              grids' worth of tiles; -1 = none: directly behind them, which makes every down tile wait --
                              a test setting).  The list is handed out dynamically (each CTA draws the next position
                              from a global counter) unless tile_sched = 2, which walks it with stride grid. */
+    int32_t gang_sync;    /* 256-row-tile GEMM kernel: the row tiles of an expert that use the same weight tile start that
+                             tile together (a counter per such gang, bounded wait, cooperative launch), so that the weight
+                             tile is read from DRAM once and shared through L2 instead of once per row tile.
+                             0 = where it pays (large expert matrices, fewer than eight row tiles per expert), 1 = never,
+                             2 = always (grids of fewer than eight CTAs excepted).  Same bits. */
 } mok_config;
 
 /*

@@ -7,7 +7,12 @@
 //      by TMA, K = H; epilogue silu(g) * u -> h (bf16, TMA store), then the epilogue warps wait until their stores have
 //      completed and add one arrival each to ready[M tile]
 //   D  down tile: h rows and W_down by TMA, K = I; epilogue -> y (bf16, TMA store).  Its producer first waits until
-//      ready[M tile] shows every gate/up tile of those rows (bounded wait; a time-out reports MOK_ERR_TIMEOUT)
+//      ready[M tile] shows every gate/up tile of those rows (bounded wait; a time-out reports MOK_ERR_TIMEOUT).
+//      One D entry of the list covers q = round(H / I) consecutive N tiles of its rows, so that an entry of either kind
+//      keeps a CTA busy for about the same time.  That matters for DRAM traffic, not for balance: CTAs that work on
+//      the same weight tile for different row tiles share it through L2 only while they stay in step, and they only
+//      stay in step if the entries before them took equally long (measured with entries of unequal length: 43 % more
+//      DRAM reads than the two-launch path, and a lower clock under the power cap)
 // The list is built on the device by fused_tiles_kernel from the schedule's per-expert tables: M tiles are grouped
 // (eight per group, one expert per group) and a group's tiles are laid out [N tile][M tile] so that CTAs working side
 // by side share a weight tile in L2.  A group's D tiles are placed `window` M tiles behind its G tiles: with the
@@ -71,12 +76,13 @@ static_assert(sizeof(Ctrl) <= SMEM_CTRL, "control block too large");
 constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 __device__ __forceinline__ uint32_t idesc_n(int n) { return (IDESC & ~(0x3Fu << 17)) | ((uint32_t)(n >> 3) << 17); }
 
-struct Tile { int row0, valid, kind, e, n, mt; };
+struct Tile { int row0, valid, kind, cnt, e, n, mt; };   // cnt: N tiles n .. n + cnt - 1 covered by this list entry
 __device__ __forceinline__ Tile decode_tile(const int4 d) {
     Tile t;
     t.row0 = d.x;
     t.valid = d.y & 0xFFFF;
     t.kind = (d.y >> 16) & 1;
+    t.cnt = (d.y >> 20) & 0xFF;
     t.e = d.z & 0xFFFF;
     t.n = (d.z >> 16) & 0xFFFF;
     t.mt = d.w;
@@ -172,9 +178,10 @@ __device__ __forceinline__ int ld_acquire(const int32_t* p) {
 //   pos_G(j) = n1 * MB(j) + n2 * MB(c(j));   pos_D(g) = n1 * ME(j(g)) + n2 * MB(g)
 __global__ void __launch_bounds__(MAX_E)
 fused_tiles_kernel(const int32_t* __restrict__ counts, const int32_t* __restrict__ pad_offsets,
-                   const int32_t* __restrict__ mt_start2, int E, int n1, int n2, int window, int max_tiles,
+                   const int32_t* __restrict__ mt_start2, int E, int n1, int n2_tiles, int q, int window, int max_tiles,
                    int4* __restrict__ tiles, int32_t* __restrict__ ready, WsHeader* __restrict__ hdr) {
     __shared__ int32_t s_mt[MAX_E + 1], s_gofs[MAX_E + 1], s_wtot[32];
+    const int n2 = (n2_tiles + q - 1) / q;           // down entries per M tile: each covers up to q N tiles
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5, n_warps = blockDim.x >> 5;
     int mc = 0;
     if (tid < E) {
@@ -276,10 +283,12 @@ fused_tiles_kernel(const int32_t* __restrict__ counts, const int32_t* __restrict
         for (int i = lane; i < (n1 + n2) * gm; i += 32) {
             const int kind = i >= n1 * gm;
             const int r = kind ? i - n1 * gm : i;
-            const int n = r / gm, m = m0 + (r - n * gm);
+            const int nc = r / gm, m = m0 + (r - nc * gm);
+            const int n = kind ? nc * q : nc;                       // first N tile of the entry
+            const int span = kind ? min(q, n2_tiles - n) : 1;       // N tiles it covers
             int4 d;
             d.x = pad0 + m * TM;
-            d.y = min(TM, cnt - m * TM) | (kind << 16);
+            d.y = min(TM, cnt - m * TM) | (kind << 16) | (span << 20);
             d.z = e | (n << 16);
             d.w = s_mt[e] + m;
             tiles[(kind ? posD : posG) + r] = d;
@@ -407,12 +416,14 @@ fused_ffn_kernel(const __grid_constant__ CUtensorMap mapWgu, const __grid_consta
                         asm volatile("fence.proxy.async;" ::: "memory");
                     }
                     const int kblocks = t.kind ? a.kb2 : a.kb1;
-                    const bool narrow = !t.kind && narrow_last && t.n == a.n1 - 1;
-                    const int brow0 = t.kind ? t.e * a.H + t.n * BN : t.e * 2 * a.I + t.n * (BN / 2);
-                    const int brow1 = t.kind ? brow0 + BN / 2 : brow0 + a.I;
                     peek = 0;
+                    for (int sub = 0; sub < t.cnt && ok; ++sub) {
+                    const int n = t.n + sub;
+                    const bool narrow = !t.kind && narrow_last && n == a.n1 - 1;
+                    const int brow0 = t.kind ? t.e * a.H + n * BN : t.e * 2 * a.I + n * (BN / 2);
+                    const int brow1 = t.kind ? brow0 + BN / 2 : brow0 + a.I;
                     for (int kb = 0; kb < kblocks; ++kb) {
-                        if (kb == (kblocks >> 1) && w.Ln < total) {   // the next tile's descriptor has arrived by now
+                        if (sub == t.cnt - 1 && kb == (kblocks >> 1) && w.Ln < total) {   // the next entry's descriptor has arrived by now
                             const Tile tn = decode_tile(w.dn);
                             if (tn.kind) peek = ld_acquire(a.ready + tn.mt);
                         }
@@ -439,6 +450,7 @@ fused_ffn_kernel(const __grid_constant__ CUtensorMap mapWgu, const __grid_consta
                         }
                         if (++s == STAGES) { s = 0; ph ^= 1u; }
                     }
+                    }
                     if (!ok) break;
                 }
                 if (a.dbg) atomicAdd(&a.header->dbg[2][DBG_PROD_WAIT_EMPTY], (unsigned long long)d_ready);
@@ -459,15 +471,19 @@ fused_ffn_kernel(const __grid_constant__ CUtensorMap mapWgu, const __grid_consta
                     const Tile t = decode_tile(w.d);
                     const bool two = t.valid > BM;
                     const int kblocks = t.kind ? a.kb2 : a.kb1;
-                    uint32_t idesc = IDESC;
-                    if (t.kind) {
-                        if (a.H - t.n * BN < BN) idesc = idesc_n((a.H - t.n * BN + 15) & ~15);
-                    } else if (narrow_last && t.n == a.n1 - 1) {
-                        idesc = idesc_n(BN / 2);
-                    }
                     const long long tile0 = dbg ? clock64() : 0;
                     long long w0 = tile0, w_full = 0, w_te = 0;
-                    bool ok = wait_bar(smem_u32(&ctrl->tempty[0]), ap0 ^ 1u, abort_flag, a.header, 2);
+                    bool ok = true;
+                    for (int sub = 0; sub < t.cnt && ok; ++sub) {
+                    const int n = t.n + sub;
+                    uint32_t idesc = IDESC;
+                    if (t.kind) {
+                        if (a.H - n * BN < BN) idesc = idesc_n((a.H - n * BN + 15) & ~15);
+                    } else if (narrow_last && n == a.n1 - 1) {
+                        idesc = idesc_n(BN / 2);
+                    }
+                    if (dbg) w0 = clock64();
+                    ok = wait_bar(smem_u32(&ctrl->tempty[0]), ap0 ^ 1u, abort_flag, a.header, 2);
                     if (dbg) w_te += clock64() - w0;
                     if (!ok) break;
                     tc_fence_after();
@@ -502,9 +518,11 @@ fused_ffn_kernel(const __grid_constant__ CUtensorMap mapWgu, const __grid_consta
                     }
                     if (!ok) break;
                     if (two) { tc_commit<1>(smem_u32(&ctrl->tfull[1])); ap1 ^= 1u; }
+                    }
+                    if (!ok) break;
                     if (dbg) {
-                        const long long dt = clock64() - tile0, units = (long long)(two ? 2 : 1) * kblocks;
-                        if (t.kind) { d_full1 += w_full; d_te1 += w_te; d_kb1 += units; d_rows1 += (long long)t.valid * kblocks; d_tot1 += dt; }
+                        const long long dt = clock64() - tile0, units = (long long)(two ? 2 : 1) * kblocks * t.cnt;
+                        if (t.kind) { d_full1 += w_full; d_te1 += w_te; d_kb1 += units; d_rows1 += (long long)t.valid * kblocks * t.cnt; d_tot1 += dt; }
                         else        { d_full0 += w_full; d_te0 += w_te; d_kb0 += units; d_rows0 += (long long)t.valid * kblocks; d_tot0 += dt; }
                     }
                 }
@@ -565,7 +583,7 @@ fused_ffn_kernel(const __grid_constant__ CUtensorMap mapWgu, const __grid_consta
                 // down tile: both operands come by TMA and the producer makes these threads' arrivals for them.  The warp
                 // still follows the ring stage by stage (one polling lane): a parity wait is only meaningful while the
                 // waiter is at most one phase ahead of the barrier, so it must not jump over the tile's stages.
-                for (int kb = 0; kb < a.kb2; ++kb) {
+                for (int kb = 0; kb < a.kb2 * t.cnt; ++kb) {
                     if (lane == 0) ok = wait_bar(smem_u32(&ctrl->empty[s]), ph ^ 1u, abort_flag, a.header, 5);
                     ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
                     if (!ok) break;
@@ -641,7 +659,10 @@ fused_ffn_kernel(const __grid_constant__ CUtensorMap mapWgu, const __grid_consta
         for (; w.valid(); w.advance()) {
             const Tile t = decode_tile(w.d);
             if (acc == 1 && t.valid <= BM) continue;
-            bool ok = wait_bar(smem_u32(&ctrl->tfull[acc]), aph, abort_flag, a.header, 4);
+            bool ok = true;
+            for (int sub = 0; sub < t.cnt; ++sub) {
+            const int n = t.n + sub;
+            ok = wait_bar(smem_u32(&ctrl->tfull[acc]), aph, abort_flag, a.header, 4);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             aph ^= 1u;
@@ -663,11 +684,11 @@ fused_ffn_kernel(const __grid_constant__ CUtensorMap mapWgu, const __grid_consta
                 }
                 hand_back();
 #pragma unroll
-                for (int pass = 0; pass < 4; ++pass) store_pass(o + pass * 32, &mapY, t.n * BN + pass * 64, a.H, row);
+                for (int pass = 0; pass < 4; ++pass) store_pass(o + pass * 32, &mapY, n * BN + pass * 64, a.H, row);
             } else {
                 // gate/up tile: silu(g) * u from columns c and c + 128 (c + 64 of a narrow last tile), 64 output columns
                 // per pass; the next pass is read and computed before waiting for the slab of the current one
-                const bool narrow = narrow_last && t.n == a.n1 - 1;
+                const bool narrow = narrow_last && n == a.n1 - 1;
                 const int passes = narrow ? 1 : 2;
                 const uint32_t up_off = narrow ? BN / 4 : BN / 2;
                 uint32_t cur[32], nxt[32];
@@ -692,7 +713,7 @@ fused_ffn_kernel(const __grid_constant__ CUtensorMap mapWgu, const __grid_consta
 #pragma unroll
                     for (int i = 0; i < 32; ++i) cur[i] = nxt[i];
                     if (pass + 1 < passes) load_pass(pass + 1, nxt);
-                    store_pass(cur, &mapHst, t.n * (BN / 2) + pass * 64, a.I, row);
+                    store_pass(cur, &mapHst, n * (BN / 2) + pass * 64, a.I, row);
                 }
                 if (lane == 0) {
                     // h of this warp's 32 rows is on its way: wait until the stores have completed (not only left shared
@@ -705,6 +726,8 @@ fused_ffn_kernel(const __grid_constant__ CUtensorMap mapWgu, const __grid_consta
                 }
                 __syncwarp();
             }
+            }
+            if (!ok) break;
         }
         if (lane == 0) tma_store_wait_all();
         __syncwarp();
@@ -768,6 +791,10 @@ cudaError_t launch_fused_ffn(const __nv_bfloat16* x, int T, int H, int I, int E,
     if (grid <= 0 || grid > sm_count) grid = sm_count;
     WsHeader* hdr = reinterpret_cast<WsHeader*>(ws + L.header);
     const int n1 = (I + BN / 2 - 1) / (BN / 2), n2 = (H + BN - 1) / BN;
+    // N tiles per down entry: as many as make its k-blocks about those of a gate/up entry (K = H against K = I)
+    int q = ((H + BK - 1) / BK + (I + BK - 1) / BK / 2) / ((I + BK - 1) / BK);
+    if (q < 1) q = 1;
+    if (q > n2) q = n2;
     if (window_tiles == 0) window_tiles = 8 * grid;
     const int window = window_tiles < 0 ? 0 : (window_tiles + n1 - 1) / n1;      // in M tiles
     int4* tiles = reinterpret_cast<int4*>(ws + L.ftiles);
@@ -777,7 +804,7 @@ cudaError_t launch_fused_ffn(const __nv_bfloat16* x, int T, int H, int I, int E,
     if (tblocks > sm_count) tblocks = sm_count;
     fused_tiles_kernel<<<tblocks, MAX_E, 0, s>>>(reinterpret_cast<const int32_t*>(ws + L.counts),
                                                  reinterpret_cast<const int32_t*>(ws + L.pad_offsets),
-                                                 reinterpret_cast<const int32_t*>(ws + L.mt_start2), E, n1, n2, window,
+                                                 reinterpret_cast<const int32_t*>(ws + L.mt_start2), E, n1, n2, q, window,
                                                  L.max_ftiles, tiles, ready, hdr);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;

@@ -59,7 +59,7 @@ constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >
 // valid: real rows of this tile (1..256); > 128 => both halves.  row0: first A row and first C row.  In the
 // K-range mode (weight gradients, see GemmArgs::kgroup_rows) the A rows and the C rows differ and the contraction
 // runs over kcol0 .. kcol0 + 64 kblocks of the operands' column space.
-struct Tile { int e, n, row0, valid, crow0, kcol0, kblocks; };
+struct Tile { int e, n, row0, valid, crow0, kcol0, kblocks, gang_first, gang_size; };
 
 template <bool KGROUP>
 __device__ __forceinline__ Tile decode_tile(const GemmArgs& a, int L, int n_nt, int n_mt_total, int k_blocks) {
@@ -75,6 +75,8 @@ __device__ __forceinline__ Tile decode_tile(const GemmArgs& a, int L, int n_nt, 
         t.row0 = m * TM;
         t.crow0 = t.e * a.kgroup_rows + m * TM;
         t.valid = min(TM, a.kgroup_rows - m * TM);
+        t.gang_first = L;
+        t.gang_size = 1;
         if (a.dense_rows > 0) {            // one group over all rows (shared expert)
             t.kcol0 = 0;
             t.kblocks = (a.dense_rows + 63) / 64;
@@ -101,6 +103,8 @@ __device__ __forceinline__ Tile decode_tile(const GemmArgs& a, int L, int n_nt, 
     const int in_group = min(GROUP_TILES, m_cnt - g * GROUP_TILES);
     t.n = rem / in_group;
     const int m = g * GROUP_TILES + (rem - t.n * in_group);
+    t.gang_first = L - (rem - t.n * in_group);     // the in_group tiles [N tile][M tile 0 .. in_group) use one weight tile
+    t.gang_size = in_group;
     t.row0 = pad0 + m * TM;
     t.crow0 = t.row0;
     t.valid = min(TM, cnt - m * TM);
@@ -225,6 +229,42 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
             for (int L = seq.first(); L < total; L = seq.next(L)) {
                 const Tile t = decode_tile<KGROUP>(a, L, n_nt, n_mt_total, k_blocks);
                 const bool two = t.valid > BM;
+                if (!KGROUP && !CLC && a.gang && t.gang_size > 1) {
+                    // The row tiles of one expert that use the same weight tile sit at consecutive list positions, i.e.
+                    // on neighbouring CTAs.  They only share that weight tile through L2 if they stream it at the same
+                    // time; tiles of different length (an expert's last, half-empty row tile) pull the CTAs apart, each
+                    // then fetches its own copy from DRAM, the extra traffic shortens the time a line stays in L2, and
+                    // the grid never finds back (measured on the DeepSeek-like layer: 67 GB read per launch for 20 GB
+                    // of operands).  So the producers of such a gang start the tile together: one arrival each on the
+                    // gang's counter, then a bounded wait for the others.  No deadlock: a gang's members (consecutive
+                    // list positions, at most GROUP_TILES of them) are on different CTAs because the grid is at
+                    // least that large (the launcher checks), every CTA walks its tiles in list order, and the launch
+                    // is cooperative (all CTAs resident) -- the first gang that is not yet complete only waits for
+                    // CTAs that are busy with tiles of gangs before it.
+                    int32_t* cnt = a.gang + t.gang_first;
+                    asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(cnt) : "memory");
+                    const unsigned long long t0 = globaltimer();
+                    uint32_t spins = 0;
+                    bool alive = true;
+                    int seen;
+                    for (;;) {
+                        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(cnt) : "memory");
+                        if (seen >= t.gang_size) break;
+                        if ((++spins & 63u) == 0u) {
+                            if (*abort_flag) { alive = false; break; }
+                            const unsigned long long limit =
+                                a.header->wait_limit_us ? 1000ull * a.header->wait_limit_us : WAIT_LIMIT_NS;
+                            if (globaltimer() - t0 > limit) {
+                                *abort_flag = 1u;
+                                atomicCAS(&a.header->status, 0, (int)MOK_ERR_TIMEOUT);
+                                a.header->where = 42;
+                                alive = false;
+                                break;
+                            }
+                        }
+                    }
+                    if (!alive) break;
+                }
                 // weight rows of this tile; in the K-range mode B is an activation matrix shared by all experts
                 const int brow0 = KGROUP ? t.n * BN
                                                       : t.e * b_rows_per_expert + (SWIGLU ? t.n * (BN / 2) : t.n * BN);
@@ -679,6 +719,28 @@ static cudaError_t launch_one(const CUtensorMap& mA, const CUtensorMap& mB, cons
         if (grid < 1) grid = 1;
     } else if (grid <= 0 || grid > sm_count) {
         grid = sm_count;
+    }
+    if (a.gang && !CLC && MODE == 0 && grid < GROUP_TILES) {
+        // a gang's (up to GROUP_TILES) tiles must sit on different CTAs, or a CTA would wait for its own later tile
+        GemmArgs b = a;
+        b.gang = nullptr;
+        gemm_m2_kernel<EPI, GATHER, MODE, CLC><<<grid, THREADS + (GATHER ? GATHER_THREADS : 0), SMEM_BYTES, s>>>(
+            mA, mB, mC, mB64, b, n_nt, k_blocks);
+        return cudaGetLastError();
+    }
+    if (a.gang && !CLC && MODE == 0) {
+        // gang starts wait for tiles of other CTAs: every CTA of the grid has to be resident (cooperative launch)
+        cudaLaunchConfig_t cfg = {};
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeCooperative;
+        attr[0].val.cooperative = 1;
+        cfg.gridDim = dim3(grid);
+        cfg.blockDim = dim3(THREADS + (GATHER ? GATHER_THREADS : 0));
+        cfg.dynamicSmemBytes = SMEM_BYTES;
+        cfg.stream = s;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        return cudaLaunchKernelEx(&cfg, gemm_m2_kernel<EPI, GATHER, MODE, CLC>, mA, mB, mC, mB64, a, n_nt, k_blocks);
     }
     gemm_m2_kernel<EPI, GATHER, MODE, CLC><<<grid, THREADS + (GATHER ? GATHER_THREADS : 0) + (CLC ? 32 : 0), SMEM_BYTES, s>>>(
         mA, mB, mC, mB64, a, n_nt, k_blocks);

@@ -81,6 +81,14 @@ bool ws_layout(int T, int H, int I, int Is, int E, int k, WsLayout* L, bool mx) 
         L->ftiles = take(sizeof(int4) * (size_t)L->max_ftiles);
         L->ready = take(sizeof(int32_t) * (size_t)mt2);
     }
+    {   // gang-start counters of the 256-row kernel: one per tile of the largest of the four GEMMs
+        const long long mt2 = Rpad / (2 * TILE_M), mts = L->Tpad / (2 * TILE_M);
+        long long n_r = (I + 127) / 128 > (H + 255) / 256 ? (I + 127) / 128 : (H + 255) / 256;
+        long long n_s = (Is + 127) / 128 > (H + 255) / 256 ? (Is + 127) / 128 : (H + 255) / 256;
+        long long tiles = mt2 * n_r > mts * n_s ? mt2 * n_r : mts * n_s;
+        L->gang_bytes = sizeof(int32_t) * (size_t)tiles;
+        L->gang = take(L->gang_bytes);
+    }
     L->hs = take(Is > 0 ? 2 * (size_t)L->Tpad * Is : 0);
     L->ysh = take(Is > 0 ? 2 * (size_t)L->Tpad * H : 0);
     if (mx) {
@@ -129,7 +137,8 @@ static int validate(const mok_args* a, WsLayout* L, size_t extra_ws) {
                       a->config->gather_mode < 0 || a->config->gather_mode > 2 ||
                       a->config->cta_group < 0 || a->config->cta_group > 3 ||
                       a->config->host_chunks < 0 || a->config->host_chunks > MOK_MAX_HOST_CHUNKS ||
-                      a->config->fused_ffn < 0 || a->config->fused_ffn > 2 || a->config->fused_window < -1))
+                      a->config->fused_ffn < 0 || a->config->fused_ffn > 2 || a->config->fused_window < -1 ||
+                      a->config->gang_sync < 0 || a->config->gang_sync > 2))
         return MOK_ERR_SHAPE;
     return MOK_OK;
 }
@@ -201,6 +210,28 @@ int run_gemm(GemmArgs g, bool swiglu, const mok_config* cfg, const WsLayout& L, 
     const int epi = swiglu ? EPI_SWIGLU : EPI_BF16, grid = cfg ? cfg->grid : 0;
     if (use_m2(cfg, g.K, g.tile_m, g.dense_rows > 0 ? g.dense_rows : g.total_rows, g.dense_rows > 0 ? 1 : g.E)) {
         WsHeader* hdr = reinterpret_cast<WsHeader*>(ws + L.header);
+        // synchronised starts of the row tiles that share a weight tile (see the kernel); not with stolen tiles, and
+        // off with gang_sync = 1
+        // Chosen (gang_sync = 0) where it pays: an expert's weight matrix is large against L2 (>= 16 MB: a few experts'
+        // tiles in flight fill it, so a tile only survives in L2 while its users run in step) and an expert has fewer
+        // than eight full row tiles (the half-empty last tile is what pulls CTAs apart).  Measured on B200, layer time
+        // with / without: DeepSeek-like -13 %, GPT-OSS-like -4 %; Qwen3-like (6 MB per expert) +2 %, Mixtral-like
+        // (eight equal row tiles per expert) +1.5 %.
+        const long long w_bytes = 2ll * (swiglu ? 2 : 1) * g.N * g.K;
+        const long long rows_all = g.dense_rows > 0 ? g.dense_rows : g.total_rows;
+        const bool pays = w_bytes >= (16ll << 20) && rows_all < 8ll * 256 * (g.dense_rows > 0 ? 1 : g.E);
+        const int mode = cfg ? cfg->gang_sync : 0;
+        if (L.gang_bytes > 0 && g.kgroup_rows == 0 && !g.b_mn && g.tile_sched != 1 && g.peer_tokens == 0 &&
+            (mode == 2 || (mode == 0 && pays))) {
+            const long long rows = g.dense_rows > 0 ? g.dense_rows : g.rows_pad;
+            const long long n_nt = swiglu ? (g.N + 127) / 128 : (g.N + 255) / 256;
+            const size_t bytes = sizeof(int32_t) * (size_t)((rows + 255) / 256 * n_nt);
+            if (bytes <= L.gang_bytes) {        // (a GEMM with more tiles than the region was sized for runs without)
+                cudaError_t eg = cudaMemsetAsync(ws + L.gang, 0, bytes, s);
+                if (eg != cudaSuccess) return cuda_fail(eg);
+                g.gang = reinterpret_cast<int32_t*>(ws + L.gang);
+            }
+        }
         g.n_mtiles = &hdr->n_mtiles2;
         g.mt_start = reinterpret_cast<const int32_t*>(ws + L.mt_start2);
         g.tile_expert = reinterpret_cast<const int32_t*>(ws + L.tile_expert2);

@@ -48,6 +48,8 @@ struct WsLayout {
     size_t xg, h, y, hs, ysh;
     size_t x8, sx, h8, sh;   // MXFP8 mode: quantised token rows + row-major scales, quantised gated activation + scale atoms
     size_t ftiles, ready;    // fused expert-FFN kernel: tile list (int4 per tile) and per-M-tile completion counters
+    size_t gang;             // 256-row kernel: gang-start counters, one int32 per list position of the largest GEMM
+    size_t gang_bytes;
     int32_t max_ftiles;
     size_t total;
     int32_t R;            // T*k
@@ -83,6 +85,8 @@ struct GemmArgs {
     int32_t dbg_slot;            // >= 0: accumulate wait-time counters into header->dbg[dbg_slot]
     int32_t starve;              // test hook: the TMA producer issues nothing, so the kernel's waits run out
     int32_t tile_sched;          // 256-row kernel, routed forward GEMMs: 1 = tiles handed out by cluster launch control
+    int32_t* gang;               // 256-row kernel, forward layout: per list position, arrivals of the row tiles that share
+                                 // one weight tile (zeroed before the launch), or NULL: no synchronised tile starts
     // K-range mode of the 256-row kernel (weight gradients): C holds E matrices [kgroup_rows, N]; A is ONE matrix
     // [kgroup_rows, K extent] and B ONE matrix [N, K extent] whose columns are the rows of the dispatch space; expert e
     // contracts over its padded segment [pad_offsets[e], pad_offsets[e+1]) (dense_rows > 0: one group over columns

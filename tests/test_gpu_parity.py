@@ -360,6 +360,24 @@ def test_one_launch_ffn_gives_the_bits_of_two_launches(cfg):
         assert torch.equal(out1.view(torch.int16), out2.view(torch.int16)), kw
 
 
+@pytest.mark.parametrize("cfg", MID + [SMALL[0], SMALL[6]], ids=[c.name for c in MID + [SMALL[0], SMALL[6]]])
+def test_synchronised_tile_starts_give_the_same_bits(cfg):
+    """The 256-row kernel can make the row tiles that share a weight tile start together (config.gang_sync; chosen
+    automatically for large expert matrices).  Forced on here: every token against the oracle, the same bits as without
+    it, for the smallest grid that allows it, a ragged one and the full one; a grid below eight CTAs falls back to
+    unsynchronised starts instead of deadlocking."""
+    m = mok()
+    d = inputs.make_inputs(cfg)
+    g = pu.upload(d)
+    out0, st, rep = pu.full_parity(cfg, d=d, g=g, config=m._config(cta_group=3, gang_sync=2))
+    print(cfg.name, rep)
+    ref = pu.run_gpu(cfg, g, config=m._config(cta_group=3, gang_sync=1), stages=False)
+    assert torch.equal(out0.view(torch.int16), ref.view(torch.int16))
+    for grid in (3, 8, 11, 148):
+        out = pu.run_gpu(cfg, g, config=m._config(cta_group=3, gang_sync=2, grid=grid), stages=False)
+        assert torch.equal(out.view(torch.int16), ref.view(torch.int16)), grid
+
+
 @pytest.mark.parametrize("fused,sched", [(0, 0), (2, 0), (2, 2)])
 def test_bounded_waits_report_a_timeout_and_leave_the_context_usable(fused, sched):
     """Failure detection without a fault: the test hook silences the gate/up GEMM's TMA producer, so its MMA issuer
