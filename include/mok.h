@@ -87,23 +87,25 @@ typedef struct mok_config {
                              work stealing).  The hardware refuses the request while work of a higher stream priority
                              waits for an SM; the CTA then leaves and the tiles nobody stole start as CTAs of their own
                              afterwards, so such work gets onto the SMs at the next tile boundary instead of at the end
-                             of the kernel.  Same bits either way.  2 = only with fused_ffn: static stride over the
-                             one-launch tile list instead of the dynamic draw. */
+                             of the kernel.  Same bits either way.  With the one-launch expert FFN (fused_ffn): 1 = dynamic
+                             draw of list positions, 2 = static stride. */
     int32_t macrobatch_tokens; /* mok_moe_forward_ex: > 0 and < T: the tokens pass through the workspace in macrobatches of
                              this many tokens, one after the other (Section 3.3: a fixed-size buffer through which the
                              tokens cycle, instead of buffers sized for the whole batch).  The workspace then only needs
                              mok_workspace_bytes(macrobatch_tokens, ...); every macrobatch streams the expert weights
                              again.  Same bits as the single pass; counts / offsets / perm / inv_perm (tables of ONE
                              schedule) cannot be returned: MOK_ERR_UNSUPPORTED. */
-    int32_t fused_ffn;    /* routed experts, bf16: 0 or 1 = gate/up GEMM and down GEMM as two launches (the default),
+    int32_t fused_ffn;    /* routed experts, bf16: 1 = gate/up GEMM and down GEMM as two launches, 0 = choose (the one launch
+                             where synchronised tile starts pay, see gang_sync; else the two launches),
                              2 = ONE persistent launch over a list of gate/up tiles and down tiles; a down tile runs
                              once a per-row-tile completion counter, advanced by the gate/up epilogues, shows that its
                              rows of the gated activation exist (Section 3.2: megakernel, GPU-local synchronisation
                              instead of kernel boundaries).  Same bits either way. */
-    int32_t fused_window; /* fused_ffn: list positions between a row group's gate/up tiles and its down tiles (0 = eight
-                             grids' worth of tiles; -1 = none: directly behind them, which makes every down tile wait --
-                             a test setting).  The list is handed out dynamically (each CTA draws the next position
-                             from a global counter) unless tile_sched = 2, which walks it with stride grid. */
+    int32_t fused_window; /* fused_ffn: list positions between a row group's gate/up tiles and its down tiles (0 = a
+                             default of two to eight grids' worth of tiles; -1 = none: directly behind them, which makes
+                             every down tile wait -- a test setting).  The list is walked with stride grid and
+                             synchronised tile starts where those pay, else handed out dynamically (each CTA draws the
+                             next position from a global counter); tile_sched = 1 / 2 force the draw / the stride. */
     int32_t gang_sync;    /* 256-row-tile GEMM kernel: the row tiles of an expert that use the same weight tile start that
                              tile together (a counter per such gang, bounded wait, cooperative launch), so that the weight
                              tile is read from DRAM once and shared through L2 instead of once per row tile.

@@ -76,11 +76,15 @@ static_assert(sizeof(Ctrl) <= SMEM_CTRL, "control block too large");
 constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 __device__ __forceinline__ uint32_t idesc_n(int n) { return (IDESC & ~(0x3Fu << 17)) | ((uint32_t)(n >> 3) << 17); }
 
-struct Tile { int row0, valid, kind, cnt, e, n, mt; };   // cnt: N tiles n .. n + cnt - 1 covered by this list entry
+struct Tile { int row0, valid, kind, cnt, e, n, mt, gang_m, gang_size; };
+// cnt: N tiles n .. n + cnt - 1 covered by this list entry; gang: the gang_size entries [L - gang_m, ...) use the same
+// weight tiles (one per row tile of the group)
 __device__ __forceinline__ Tile decode_tile(const int4 d) {
     Tile t;
     t.row0 = d.x;
-    t.valid = d.y & 0xFFFF;
+    t.valid = d.y & 0x1FF;
+    t.gang_m = (d.y >> 9) & 7;
+    t.gang_size = ((d.y >> 12) & 7) + 1;
     t.kind = (d.y >> 16) & 1;
     t.cnt = (d.y >> 20) & 0xFF;
     t.e = d.z & 0xFFFF;
@@ -288,7 +292,7 @@ fused_tiles_kernel(const int32_t* __restrict__ counts, const int32_t* __restrict
             const int span = kind ? min(q, n2_tiles - n) : 1;       // N tiles it covers
             int4 d;
             d.x = pad0 + m * TM;
-            d.y = min(TM, cnt - m * TM) | (kind << 16) | (span << 20);
+            d.y = min(TM, cnt - m * TM) | ((m - m0) << 9) | ((gm - 1) << 12) | (kind << 16) | (span << 20);
             d.z = e | (n << 16);
             d.w = s_mt[e] + m;
             tiles[(kind ? posD : posG) + r] = d;
@@ -302,6 +306,8 @@ struct FusedArgs {
     const int4* tiles;             // the tile list
     const int32_t* n_tiles;        // device: its length
     int32_t* next_tile;            // device: dynamic mode's draw counter (zeroed by the tile-list kernel)
+    int32_t* gang;                 // static mode: per list position, arrivals of the entries that share weight tiles
+                                   // (zeroed before the launch), or NULL: unsynchronised starts
     int32_t* ready;                // per 256-row M tile: epilogue-warp arrivals of its gate/up tiles
     int32_t max_tiles;
     int32_t H, I, E;
@@ -386,6 +392,29 @@ fused_ffn_kernel(const __grid_constant__ CUtensorMap mapWgu, const __grid_consta
                     const Tile t = decode_tile(w.d);
                     const bool two = t.valid > BM;
                     bool ok = true;
+                    if (!DYN && a.gang && t.gang_size > 1) {
+                        // entries that stream the same weight tiles start together (see gemm_tcgen05_m2.cu): with the
+                        // static stride they sit on different CTAs (grid >= 8, checked by the launcher)
+                        int32_t* cnt = a.gang + (w.L - t.gang_m);
+                        asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(cnt) : "memory");
+                        const unsigned long long t0 = globaltimer();
+                        uint32_t spins = 0;
+                        while (ld_acquire(cnt) < t.gang_size) {
+                            if ((++spins & 63u) == 0u) {
+                                if (*abort_flag) { ok = false; break; }
+                                const unsigned long long limit =
+                                    a.header->wait_limit_us ? 1000ull * a.header->wait_limit_us : WAIT_LIMIT_NS;
+                                if (globaltimer() - t0 > limit) {
+                                    *abort_flag = 1u;
+                                    atomicCAS(&a.header->status, 0, (int)MOK_ERR_TIMEOUT);
+                                    a.header->where = 43;
+                                    ok = false;
+                                    break;
+                                }
+                            }
+                        }
+                        if (!ok) break;
+                    }
                     if (t.kind) {
                         // every gate/up tile of these rows has stored h: n1 tiles x 4 epilogue warps per 128-row half
                         const int need = a.n1 * (two ? 8 : 4);
@@ -778,11 +807,11 @@ static cudaError_t launch_kernel(int grid, cudaStream_t s, const CUtensorMap& m0
 }
 
 // Host side.  `window_tiles`: distance (in list positions) between a group's gate/up tiles and its down tiles; 0 = the
-// default of eight grids' worth of tiles (measured: the down tiles then never wait and still find h in L2), -1 = none
+// default (eight grids' worth of tiles with the dynamic draw, two with the static stride: measured best), -1 = none
 // (a group's down tiles directly behind its gate/up tiles).
 cudaError_t launch_fused_ffn(const __nv_bfloat16* x, int T, int H, int I, int E, const __nv_bfloat16* Wgu,
                              const __nv_bfloat16* Wd, const WsLayout& L, char* ws, int grid, int window_tiles, bool dynamic,
-                             bool dbg, bool starve, cudaStream_t s) {
+                             bool gang_sync, bool dbg, bool starve, cudaStream_t s) {
     using namespace ff;
     int dev = 0, sm_count = 0;
     cudaError_t e = current_device(&dev);
@@ -795,7 +824,7 @@ cudaError_t launch_fused_ffn(const __nv_bfloat16* x, int T, int H, int I, int E,
     int q = ((H + BK - 1) / BK + (I + BK - 1) / BK / 2) / ((I + BK - 1) / BK);
     if (q < 1) q = 1;
     if (q > n2) q = n2;
-    if (window_tiles == 0) window_tiles = 8 * grid;
+    if (window_tiles == 0) window_tiles = dynamic ? 8 * grid : 2 * grid;
     const int window = window_tiles < 0 ? 0 : (window_tiles + n1 - 1) / n1;      // in M tiles
     int4* tiles = reinterpret_cast<int4*>(ws + L.ftiles);
     int32_t* ready = reinterpret_cast<int32_t*>(ws + L.ready);
@@ -825,6 +854,12 @@ cudaError_t launch_fused_ffn(const __nv_bfloat16* x, int T, int H, int I, int E,
     a.tiles = tiles;
     a.n_tiles = &hdr->n_ftiles;
     a.next_tile = &hdr->next_tile;
+    a.gang = nullptr;
+    if (!dynamic && gang_sync && grid >= GROUP_TILES && L.gang_bytes >= sizeof(int32_t) * (size_t)L.max_ftiles) {
+        e = cudaMemsetAsync(ws + L.gang, 0, sizeof(int32_t) * (size_t)L.max_ftiles, s);
+        if (e != cudaSuccess) return e;
+        a.gang = reinterpret_cast<int32_t*>(ws + L.gang);
+    }
     a.ready = ready;
     a.max_tiles = L.max_ftiles;
     a.H = H; a.I = I; a.E = E;

@@ -86,6 +86,7 @@ bool ws_layout(int T, int H, int I, int Is, int E, int k, WsLayout* L, bool mx) 
         long long n_r = (I + 127) / 128 > (H + 255) / 256 ? (I + 127) / 128 : (H + 255) / 256;
         long long n_s = (Is + 127) / 128 > (H + 255) / 256 ? (Is + 127) / 128 : (H + 255) / 256;
         long long tiles = mt2 * n_r > mts * n_s ? mt2 * n_r : mts * n_s;
+        if (L->max_ftiles > tiles) tiles = L->max_ftiles;       // the one-launch FFN's list (static hand-out)
         L->gang_bytes = sizeof(int32_t) * (size_t)tiles;
         L->gang = take(L->gang_bytes);
     }
@@ -194,16 +195,34 @@ static bool use_m2(const mok_config* cfg, int K, int tile_m, long long rows, int
     return K >= M2_MIN_K && rows >= 96ll * experts;
 }
 
-// Routed gate/up + SwiGLU + down as ONE persistent launch (gemm_fused.cu): on request (fused_ffn = 2), for any shape
-// whose token gather is fused into the GEMM.  It is not chosen by default: measured on B200 with the two variants
-// alternating in one process, it needs 8-10 % fewer SM cycles than the two launches, but the board runs at its power
-// cap and settles at a correspondingly lower clock, so the layer's time moves by -4 % (H = I = 2880) to +3 %
-// (H = 7168, I = 2048) only.
+// Whether synchronised tile starts (gemm_tcgen05_m2.cu, "gang") pay for a grouped GEMM whose experts own weight matrices
+// of `w_bytes` bytes and `rows` rows in total: an expert's matrix is large against L2 (>= 12 MB: a few experts' tiles in
+// flight fill it, so a tile only survives in L2 while its users run in step) and an expert has fewer than eight full
+// row tiles (the half-empty last tile is what pulls CTAs apart).  Measured on B200, layer time with / without:
+// DeepSeek-like -13 %, GPT-OSS-like -4 %; Qwen3-like (6 MB per expert) +2 %, Mixtral-like (eight equal row tiles per
+// expert) +1.5 %.
+static bool gang_pays(long long w_bytes, long long rows, int experts) {
+    return w_bytes >= (12ll << 20) && rows < 8ll * 256 * experts;
+}
+
+// Routed gate/up + SwiGLU + down as ONE persistent launch (gemm_fused.cu).  Chosen by default where synchronised tile
+// starts pay for both GEMMs (there it equals or beats the two launches: DeepSeek-like -1.6 %, GPT-OSS-like -4 %, two
+// variants alternating in one process); elsewhere the two launches are 1-2 % faster and stay the default.
+// fused_ffn = 1 / 2 force the two launches / the one launch.
+static bool fused_gang(const mok_config* cfg, int H, int I, long long rows, int experts) {
+    const int mode = cfg ? cfg->gang_sync : 0;
+    if (mode == 1) return false;
+    if (mode == 2) return true;
+    return gang_pays(4ll * I * H, rows, experts) && gang_pays(2ll * H * I, rows, experts);
+}
 static bool use_fused_ffn(const mok_config* cfg, int H, int I, int tile_m, long long rows, int experts, int max_ftiles) {
-    (void)H; (void)rows; (void)experts;
     if (use_simt(cfg) || use_tn(cfg) || use_mx(cfg) || tile_m != TILE_M || max_ftiles <= 0) return false;
-    if (!cfg || cfg->fused_ffn != 2 || cfg->cta_group == 1 || cfg->cta_group == 2 || cfg->tile_sched == 1) return false;
-    return fused_gather(cfg, I);
+    if (cfg && (cfg->fused_ffn == 1 || cfg->cta_group == 1 || cfg->cta_group == 2)) return false;
+    if (!fused_gather(cfg, I)) return false;
+    if (cfg && cfg->fused_ffn == 2) return true;
+    if (cfg && cfg->tile_sched == 1) return false;          // (tile stealing belongs to the two-launch path)
+    return use_m2(cfg, H, tile_m, rows, experts) && use_m2(cfg, I, tile_m, rows, experts) &&
+           fused_gang(cfg, H, I, rows, experts);
 }
 
 int run_gemm(GemmArgs g, bool swiglu, const mok_config* cfg, const WsLayout& L, char* ws, cudaStream_t s) {
@@ -212,14 +231,9 @@ int run_gemm(GemmArgs g, bool swiglu, const mok_config* cfg, const WsLayout& L, 
         WsHeader* hdr = reinterpret_cast<WsHeader*>(ws + L.header);
         // synchronised starts of the row tiles that share a weight tile (see the kernel); not with stolen tiles, and
         // off with gang_sync = 1
-        // Chosen (gang_sync = 0) where it pays: an expert's weight matrix is large against L2 (>= 16 MB: a few experts'
-        // tiles in flight fill it, so a tile only survives in L2 while its users run in step) and an expert has fewer
-        // than eight full row tiles (the half-empty last tile is what pulls CTAs apart).  Measured on B200, layer time
-        // with / without: DeepSeek-like -13 %, GPT-OSS-like -4 %; Qwen3-like (6 MB per expert) +2 %, Mixtral-like
-        // (eight equal row tiles per expert) +1.5 %.
         const long long w_bytes = 2ll * (swiglu ? 2 : 1) * g.N * g.K;
         const long long rows_all = g.dense_rows > 0 ? g.dense_rows : g.total_rows;
-        const bool pays = w_bytes >= (16ll << 20) && rows_all < 8ll * 256 * (g.dense_rows > 0 ? 1 : g.E);
+        const bool pays = gang_pays(w_bytes, rows_all, g.dense_rows > 0 ? 1 : g.E);
         const int mode = cfg ? cfg->gang_sync : 0;
         if (L.gang_bytes > 0 && g.kgroup_rows == 0 && !g.b_mn && g.tile_sched != 1 && g.peer_tokens == 0 &&
             (mode == 2 || (mode == 0 && pays))) {
@@ -383,11 +397,14 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
         g.total_rows = L.R;
         g.tile_sched = a->config ? a->config->tile_sched : 0;
         const bool fused = !simt && use_fused_ffn(a->config, a->H, a->I, tile_m, L.R, a->E, L.max_ftiles);
+        // its hand-out: synchronised starts need the static stride (a CTA that draws ahead could hold two tiles of a gang)
+        const bool fused_sync = fused_gang(a->config, a->H, a->I, L.R, a->E);
+        const int sched = a->config ? a->config->tile_sched : 0;
+        const bool fused_dynamic = sched == 1 || (sched == 0 && !fused_sync);
         if (fused) {
             e = launch_fused_ffn(x, a->T, a->H, a->I, a->E, reinterpret_cast<const __nv_bfloat16*>(a->W_gate_up),
                                  reinterpret_cast<const __nv_bfloat16*>(a->W_down), L, ws, a->config ? a->config->grid : 0,
-                                 a->config ? a->config->fused_window : 0, !(a->config && a->config->tile_sched == 2), dbg,
-                                 g.starve != 0, s);
+                                 a->config ? a->config->fused_window : 0, fused_dynamic, fused_sync, dbg, g.starve != 0, s);
             if (e != cudaSuccess) return cuda_fail(e);
         } else if ((rc = run_gemm(g, true, a->config, L, ws, s))) return rc;
         g.row_token = nullptr;

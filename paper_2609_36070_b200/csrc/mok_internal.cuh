@@ -147,7 +147,7 @@ cudaError_t launch_gemm_mx(const GemmArgs& a, int epi, int grid, cudaStream_t s)
 // routed gate/up + SwiGLU + down in one persistent launch (tile list + kernel); needs the schedule's 256-row tile table
 cudaError_t launch_fused_ffn(const __nv_bfloat16* x, int T, int H, int I, int E, const __nv_bfloat16* Wgu,
                              const __nv_bfloat16* Wd, const WsLayout& L, char* ws, int grid, int window_tiles, bool dynamic,
-                             bool dbg, bool starve, cudaStream_t s);
+                             bool gang_sync, bool dbg, bool starve, cudaStream_t s);
 cudaError_t launch_mx_quantize_rows(const __nv_bfloat16* in, long long rows, int K, uint8_t* codes, uint8_t* scales,
                                     cudaStream_t s);
 cudaError_t launch_mx_quantize_atoms(const __nv_bfloat16* in, int groups, int rows_per_group, int K, uint8_t* codes,

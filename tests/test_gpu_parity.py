@@ -355,7 +355,11 @@ def test_one_launch_ffn_gives_the_bits_of_two_launches(cfg):
     print(cfg.name, rep)
     for kw in ({}, {"fused_window": -1}, {"fused_window": 1}, {"fused_window": 1 << 20}, {"grid": 1}, {"grid": 7},
                {"grid": 37, "fused_window": -1}, {"tile_sched": 2}, {"tile_sched": 2, "fused_window": -1},
-               {"tile_sched": 2, "grid": 5, "fused_window": 40}):
+               {"tile_sched": 2, "grid": 5, "fused_window": 40},
+               # static stride with synchronised tile starts (what large expert matrices get by default)
+               {"gang_sync": 2}, {"gang_sync": 2, "fused_window": -1}, {"gang_sync": 2, "grid": 8},
+               {"gang_sync": 2, "grid": 11, "fused_window": 40}, {"gang_sync": 2, "grid": 3},
+               {"gang_sync": 2, "tile_sched": 1}):
         out1 = pu.run_gpu(cfg, g, config=m._config(fused_ffn=2, **kw), stages=False)
         assert torch.equal(out1.view(torch.int16), out2.view(torch.int16)), kw
 
@@ -378,8 +382,8 @@ def test_synchronised_tile_starts_give_the_same_bits(cfg):
         assert torch.equal(out.view(torch.int16), ref.view(torch.int16)), grid
 
 
-@pytest.mark.parametrize("fused,sched", [(0, 0), (2, 0), (2, 2)])
-def test_bounded_waits_report_a_timeout_and_leave_the_context_usable(fused, sched):
+@pytest.mark.parametrize("fused,sched,gang", [(1, 0, 0), (2, 0, 0), (2, 2, 0), (2, 0, 2), (1, 0, 2)])
+def test_bounded_waits_report_a_timeout_and_leave_the_context_usable(fused, sched, gang):
     """Failure detection without a fault: the test hook silences the gate/up GEMM's TMA producer, so its MMA issuer
     waits for operands that never come.  Every wait is bounded (2 ms here), the kernel records MOK_ERR_TIMEOUT, frees
     its tensor memory and returns; the next call on the same context must be correct again.  fused = 2: the same on
@@ -391,7 +395,8 @@ def test_bounded_waits_report_a_timeout_and_leave_the_context_usable(fused, sche
     ws = m.alloc_workspace(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k)
     good = pu.run_gpu(cfg, g, ws=ws, stages=False).clone()
     m.mok_moe_forward_ex(g["x"], g["W_r"], g["bias"], g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], cfg.k, ws,
-                         config=m._config(debug=m.MOK_DEBUG_STARVE, fused_ffn=fused, tile_sched=sched))
+                         config=m._config(debug=m.MOK_DEBUG_STARVE, fused_ffn=fused, tile_sched=sched, gang_sync=gang,
+                                          cta_group=3 if fused == 1 else 0))
     assert m.mok_read_status(ws) == m.MOK_ERR_TIMEOUT
     again = pu.run_gpu(cfg, g, ws=ws, stages=False)
     assert torch.equal(good.view(torch.int16), again.view(torch.int16))
