@@ -38,6 +38,9 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 NCU_TRAFFIC = {
     # one-pass captures at full size (dram__bytes_read.sum + dram__bytes_write.sum of one launch)
     "deepseek_v3": {"bytes": 20.57e9, "scale": 1, "source": "profiles/gemm_kernels_deepseek_v3.md"},
+    # the routed expert FFN as one persistent launch (the default where synchronised tile starts pay)
+    "deepseek_v3+one_launch": {"bytes": 38.01e9, "scale": 1, "source": "profiles/gemm_kernels_deepseek_v3.md"},
+    "gpt_oss_120b+one_launch": {"bytes": 8.34e9, "scale": 1, "source": "profiles/gemm_kernels_other_workloads.md"},
     "qwen3_30b_a3b": {"bytes": 1.415e9, "scale": 1, "source": "profiles/gemm_kernels_other_workloads.md"},
     "mixtral_8x7b": {"bytes": 3.553e9, "scale": 1, "source": "profiles/gemm_kernels_other_workloads.md"},
     "gpt_oss_120b": {"bytes": 5.136e9, "scale": 1, "source": "profiles/gemm_kernels_other_workloads.md"},
@@ -439,6 +442,11 @@ class Layer:
         raw = self.mok.mok_debug_counters(self.ws)
         out = {}
         for name, c in raw.items():
+            if name == "fused" and c["ctas"]:      # the one-launch expert FFN: whole-kernel clock and imbalance
+                out[name] = {"sm_ghz_in_kernel": c["mma_total"] / max(1, c["mma_total_ns"]),
+                             "busiest_cta_over_mean": c["mma_total_max_cta"] / (c["mma_total"] / c["ctas"]), "ctas": c["ctas"],
+                             "producer_wait_for_rows_share": raw["gemm2"]["producer_wait_stage"] / max(1, c["mma_total"])}
+                continue
             if not c["ctas"] or not c["k_blocks"]:
                 continue
             units = c["k_blocks"]               # 128-row x 64-column-of-K MMA units: 512 tensor-pipe cycles each
@@ -533,22 +541,35 @@ def finish_record(rec, cfg, pk, mx, world=1):
     scale = 2.0 if mx else 1.0
     rec["ffn_phase"] = {"ms": ffn_ms, "tflops": ffn_tf, "frac_of_burst": ffn_tf / (scale * pk["bf16_tflops"]),
                         "frac_of_sustained": ffn_tf / (scale * pk.get("bf16_tflops_sustained", pk["bf16_tflops"]))}
-    g1_flops = 4.0 * cfg.T * cfg.k * cfg.H * cfg.I
+    # The dominant kernel: the routed gate/up grouped GEMM -- or, where the library runs the routed expert FFN as ONE
+    # persistent launch (its default for large expert matrices), that kernel, which holds the gate/up AND the down
+    # tiles (the stage events then show the whole launch under gemm1 and nothing under gemm2).
+    one_launch = st["gemm2"] < 0.01 * st["gemm1"]
+    g1_flops = (6.0 if one_launch else 4.0) * cfg.T * cfg.k * cfg.H * cfg.I
     g1_tf = g1_flops / (st["gemm1"] * 1e-3) / 1e12
     clk = rec.get("clocks_stage_loop") or {}
     dom = roofline_fracs(g1_tf, pk, mx, rec.pop("_stage_region_s"), clk)
     dom["ms"] = st["gemm1"]
+    dom["kernel"] = ("routed expert FFN in one persistent launch: gate/up tiles + SwiGLU and down tiles, token gather fused "
+                     "(fused_ffn_kernel)") if one_launch else \
+                    "routed gate/up grouped GEMM + SwiGLU, token gather fused (gemm_m2_kernel<EPI_SWIGLU, GATHER>)"
+    dom["algorithmic_flops_per_launch"] = g1_flops
     # the fastest single launch of the loop against the burst peak (itself the best of ten single launches)
     best = rec.pop("stage_ms_min")["gemm1"]
     dom["best_launch_ms"] = best
     dom["best_launch_frac_of_burst"] = g1_flops / (best * 1e-3) / 1e12 / (scale * pk["bf16_tflops"])
     if clk.get("sm_mhz"):
         dom["sm_cycles"] = st["gemm1"] * 1e-3 * clk["sm_mhz"] * 1e6       # kernel time x median sampled SM clock
-    if "counters" in rec and "gemm1" in rec["counters"]:
-        dom["sm_cycles_device"] = st["gemm1"] * 1e-3 * rec["counters"]["gemm1"]["sm_ghz_in_kernel"] * 1e9
-    tr = NCU_TRAFFIC.get(cfg.name)
-    dom["algorithmic_bytes"] = 2.0 * (2 * cfg.I * cfg.H * cfg.E + cfg.T * cfg.k * (cfg.H + cfg.I))
+    ck = "fused" if one_launch else "gemm1"
+    if "counters" in rec and ck in rec["counters"]:
+        dom["sm_cycles_device"] = st["gemm1"] * 1e-3 * rec["counters"][ck]["sm_ghz_in_kernel"] * 1e9
+    tr = NCU_TRAFFIC.get(cfg.name + ("+one_launch" if one_launch else ""))
+    # weights once per expert, rows gathered once per route, h written (and, in the one launch, read back from L2), y written
+    dom["algorithmic_bytes"] = 2.0 * (2 * cfg.I * cfg.H * cfg.E + cfg.T * cfg.k * (cfg.H + cfg.I)) + \
+        (2.0 * (cfg.I * cfg.H * cfg.E + cfg.T * cfg.k * cfg.H) if one_launch else 0.0)
     dom["traffic"] = None if (mx or tr is None) else tr["bytes"] * tr["scale"]
+    if tr is not None and not mx:
+        dom["traffic_source"] = f"{tr['source']} (ncu capture x {tr['scale']})"
     rec["dominant_kernel"] = dom
     rec.pop("_region_s", None)
     if "sustained" in rec:
@@ -561,8 +582,9 @@ def finish_record(rec, cfg, pk, mx, world=1):
         s["ffn_phase"] = {"ms": sffn, "tflops": flops / (sffn * 1e-3) / 1e12,
                           "frac_of_sustained": flops / (sffn * 1e-3) / 1e12 / sust_peak,
                           "frac_of_burst": flops / (sffn * 1e-3) / 1e12 / (scale * pk["bf16_tflops"])}
-        s["dominant_kernel"] = {"ms": sst["gemm1"], "tflops": g1_flops / (sst["gemm1"] * 1e-3) / 1e12,
-                                "frac_of_sustained": g1_flops / (sst["gemm1"] * 1e-3) / 1e12 / sust_peak}
+        s_flops = (6.0 if sst["gemm2"] < 0.01 * sst["gemm1"] else 4.0) * cfg.T * cfg.k * cfg.H * cfg.I
+        s["dominant_kernel"] = {"ms": sst["gemm1"], "tflops": s_flops / (sst["gemm1"] * 1e-3) / 1e12,
+                                "frac_of_sustained": s_flops / (sst["gemm1"] * 1e-3) / 1e12 / sust_peak}
     return rec
 
 
@@ -774,19 +796,13 @@ def main():
             rec.pop("clocks_stage_loop", None)
 
     dom = main_rec.pop("dominant_kernel")
-    tr = NCU_TRAFFIC.get(cfg.name)
-    roofline = {"kernel": ("routed gate/up grouped GEMM on MXFP8 operands + SwiGLU + activation quantisation, token gather fused "
-                           "(gemm_mx_kernel<EPI_SWIGLU, GATHER>)") if mx else
-                          "routed gate/up grouped GEMM + SwiGLU, token gather fused (gemm_m2_kernel<EPI_SWIGLU, GATHER>)",
-                "bound": "tensor"}
+    roofline = {"kernel": dom.pop("kernel"), "bound": "tensor"}
+    if mx:
+        roofline["kernel"] = ("routed gate/up grouped GEMM on MXFP8 operands + SwiGLU + activation quantisation, token gather "
+                              "fused (gemm_mx_kernel<EPI_SWIGLU, GATHER>)")
     roofline.update(dom)
-    roofline["algorithmic_flops_per_launch"] = 4.0 * cfg.T * cfg.k * cfg.H * cfg.I
     if "sustained" in main_rec:
         roofline["sustained_run"] = main_rec["sustained"]["dominant_kernel"]
-    roofline["traffic"] = None if (mx or tr is None) else tr["bytes"] * tr["scale"]
-    roofline["algorithmic_bytes"] = 2.0 * (2 * cfg.I * cfg.H * cfg.E + cfg.T * cfg.k * (cfg.H + cfg.I))
-    if tr is not None and not mx:
-        roofline["traffic_source"] = f"{tr['source']} (ncu capture x {tr['scale']})"
     conf = mok._config(impl=args.gemm, gather_mode=args.gather_mode, cta_group=args.cta_group, fused_ffn=args.fused_ffn,
                        precision=mok.MOK_PRECISION_MXFP8 if mx else mok.MOK_PRECISION_BF16, tile_sched=args.tile_sched)
     line = {
