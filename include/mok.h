@@ -111,6 +111,9 @@ typedef struct mok_config {
                              tile is read from DRAM once and shared through L2 instead of once per row tile.
                              0 = where it pays (large expert matrices, fewer than eight row tiles per expert), 1 = never,
                              2 = always (grids of fewer than eight CTAs excepted).  Same bits. */
+    int32_t serial_launches; /* 0 = the kernels of a forward call are launched with programmatic stream serialization (a
+                             kernel's CTAs are scheduled while its predecessor still runs; every kernel waits for its
+                             predecessors' completion before it touches their data), 1 = plain launches.  Same bits. */
 } mok_config;
 
 /*

@@ -39,6 +39,7 @@ combine_kernel(const __nv_bfloat16* __restrict__ y, const __nv_bfloat16* __restr
                int T, int H, int k, __nv_bfloat16* __restrict__ out) {
     __shared__ int32_t s_pos[MAX_K];
     __shared__ float s_w[MAX_K];
+    pdl_enter();
     const int t = blockIdx.x;
     if (threadIdx.x < k) {
         s_pos[threadIdx.x] = pos[(size_t)t * k + threadIdx.x];
@@ -97,11 +98,10 @@ cudaError_t launch_gather(const __nv_bfloat16* x, int H, int k, int tile_m, cons
 
 cudaError_t launch_combine(const WsLayout& L, char* ws, int T, int H, int k, bool shared, __nv_bfloat16* out,
                            cudaStream_t s, bool unit_weights) {
-    combine_kernel<<<T, 128, 0, s>>>(reinterpret_cast<const __nv_bfloat16*>(ws + L.y),
-                                     shared ? reinterpret_cast<const __nv_bfloat16*>(ws + L.ysh) : nullptr,
-                                     reinterpret_cast<const int32_t*>(ws + L.pos),
-                                     unit_weights ? nullptr : reinterpret_cast<const float*>(ws + L.w), T, H, k, out);
-    return cudaGetLastError();
+    return launch_pdl(combine_kernel, dim3(T), dim3(128), 0, s, reinterpret_cast<const __nv_bfloat16*>(ws + L.y),
+                      shared ? reinterpret_cast<const __nv_bfloat16*>(ws + L.ysh) : (const __nv_bfloat16*)nullptr,
+                      reinterpret_cast<const int32_t*>(ws + L.pos),
+                      unit_weights ? (const float*)nullptr : reinterpret_cast<const float*>(ws + L.w), T, H, k, out);
 }
 
 }  // namespace mok

@@ -185,6 +185,7 @@ fused_tiles_kernel(const int32_t* __restrict__ counts, const int32_t* __restrict
                    const int32_t* __restrict__ mt_start2, int E, int n1, int n2_tiles, int q, int window, int max_tiles,
                    int4* __restrict__ tiles, int32_t* __restrict__ ready, WsHeader* __restrict__ hdr) {
     __shared__ int32_t s_mt[MAX_E + 1], s_gofs[MAX_E + 1], s_wtot[32];
+    pdl_enter();
     const int n2 = (n2_tiles + q - 1) / q;           // down entries per M tile: each covers up to q N tiles
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5, n_warps = blockDim.x >> 5;
     int mc = 0;
@@ -337,6 +338,7 @@ fused_ffn_kernel(const __grid_constant__ CUtensorMap mapWgu, const __grid_consta
                  const __grid_constant__ CUtensorMap mapWd, const __grid_constant__ CUtensorMap mapY,
                  const __grid_constant__ FusedArgs a) {
     extern __shared__ uint8_t smem_raw[];
+    pdl_enter();
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t* smem = smem_raw + (base - raw);
@@ -791,10 +793,11 @@ static cudaError_t launch_kernel(int grid, cudaStream_t s, const CUtensorMap& m0
     });
     if (e != cudaSuccess) return e;
     if (grid <= 0 || grid > sm_count) grid = sm_count;
+    // Dynamic draw: a position is only drawn by a CTA that runs: an ordinary (programmatically serialised) launch.
+    if (DYN) return launch_pdl(fused_ffn_kernel<DYN>, dim3(grid), dim3(THREADS), (size_t)SMEM_BYTES, s, m0, m1, m2, m3, m4, m5, a);
+    // static list: tiles wait for tiles of other CTAs, so every CTA of the grid must be resident (cooperative launch).
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
-    // static list: tiles wait for tiles of other CTAs, so every CTA of the grid must be resident (cooperative launch).
-    // Dynamic draw: a position is only drawn by a CTA that runs: plain launch.
     attr[0].id = cudaLaunchAttributeCooperative;
     attr[0].val.cooperative = 1;
     cfg.gridDim = dim3(grid);
@@ -802,7 +805,7 @@ static cudaError_t launch_kernel(int grid, cudaStream_t s, const CUtensorMap& m0
     cfg.dynamicSmemBytes = SMEM_BYTES;
     cfg.stream = s;
     cfg.attrs = attr;
-    cfg.numAttrs = DYN ? 0 : 1;
+    cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, fused_ffn_kernel<DYN>, m0, m1, m2, m3, m4, m5, a);
 }
 
@@ -831,11 +834,9 @@ cudaError_t launch_fused_ffn(const __nv_bfloat16* x, int T, int H, int I, int E,
     // enough blocks for one warp per group of a large batch; every block rebuilds the per-expert offsets itself
     int tblocks = (int)((L.max_mt / 2 / GROUP_TILES + E) / (MAX_E / 32)) + 1;
     if (tblocks > sm_count) tblocks = sm_count;
-    fused_tiles_kernel<<<tblocks, MAX_E, 0, s>>>(reinterpret_cast<const int32_t*>(ws + L.counts),
-                                                 reinterpret_cast<const int32_t*>(ws + L.pad_offsets),
-                                                 reinterpret_cast<const int32_t*>(ws + L.mt_start2), E, n1, n2, q, window,
-                                                 L.max_ftiles, tiles, ready, hdr);
-    e = cudaGetLastError();
+    e = launch_pdl(fused_tiles_kernel, dim3(tblocks), dim3(MAX_E), 0, s, reinterpret_cast<const int32_t*>(ws + L.counts),
+                   reinterpret_cast<const int32_t*>(ws + L.pad_offsets), reinterpret_cast<const int32_t*>(ws + L.mt_start2), E,
+                   n1, n2, q, window, L.max_ftiles, tiles, ready, hdr);
     if (e != cudaSuccess) return e;
 
     CUtensorMap mWgu, mWgu64, mHst, mHld, mWd, mY;

@@ -80,6 +80,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
     constexpr int TM = BM * CTAS;                           // rows of one (pair) tile
     static_assert(STAGES * STAGE_BYTES == RING_BYTES, "ring size");
     extern __shared__ uint8_t smem_raw[];
+    pdl_enter();
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t* smem = smem_raw + (base - raw);
@@ -416,6 +417,12 @@ static cudaError_t launch_one(const CUtensorMap& mA, const CUtensorMap& mB, cons
     cfg.dynamicSmemBytes = SMEM_BYTES;
     cfg.stream = s;
     cfg.numAttrs = 0;
+    if (CTAS == 1 && g_pdl) {     // single CTAs: programmatically serialised with the kernel before (see pdl_enter)
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+    }
     if (CTAS == 2) {
         attr[0].id = cudaLaunchAttributeClusterDimension;
         attr[0].val.clusterDim.x = 2;

@@ -172,6 +172,7 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
     // MODE 3: the K-range mode with BOTH operands read MN-major: A = [rows of the dispatch space, M] and
     // B = [rows, N] as the backward pass produces them, no transposed copies
     constexpr bool KGROUP = (MODE == 1 || MODE == 3), BMN = (MODE == 2 || MODE == 3), AMN = (MODE == 3);
+    pdl_enter();
     // SwiGLU tiles are [gate 128 | up 128] weight rows.  When the last N tile has at most 64 real columns (I mod 128 in
     // 1..64) it is loaded as [gate 64 | up 64] through a 64-row box and issued as an N = 128 MMA: half the tensor-pipe
     // time and half the weight bytes for the same outputs.
@@ -742,9 +743,13 @@ static cudaError_t launch_one(const CUtensorMap& mA, const CUtensorMap& mB, cons
         cfg.numAttrs = 1;
         return cudaLaunchKernelEx(&cfg, gemm_m2_kernel<EPI, GATHER, MODE, CLC>, mA, mB, mC, mB64, a, n_nt, k_blocks);
     }
-    gemm_m2_kernel<EPI, GATHER, MODE, CLC><<<grid, THREADS + (GATHER ? GATHER_THREADS : 0) + (CLC ? 32 : 0), SMEM_BYTES, s>>>(
-        mA, mB, mC, mB64, a, n_nt, k_blocks);
-    return cudaGetLastError();
+    if (CLC) {   // (tile stealing cancels CTAs that have not started: kept as a plain launch)
+        gemm_m2_kernel<EPI, GATHER, MODE, CLC><<<grid, THREADS + (GATHER ? GATHER_THREADS : 0) + 32, SMEM_BYTES, s>>>(
+            mA, mB, mC, mB64, a, n_nt, k_blocks);
+        return cudaGetLastError();
+    }
+    return launch_pdl(gemm_m2_kernel<EPI, GATHER, MODE, CLC>, dim3(grid), dim3(THREADS + (GATHER ? GATHER_THREADS : 0)),
+                      (size_t)SMEM_BYTES, s, mA, mB, mC, mB64, a, n_nt, k_blocks);
 }
 
 }  // namespace m2

@@ -8,6 +8,7 @@
 namespace mok {
 
 static thread_local int g_last_cuda_error = 0;
+thread_local bool g_pdl = true;
 constexpr int M2_MIN_K = 512;    // shortest K for which the 256-row-tile kernel is chosen by default
 
 int cuda_fail(cudaError_t e) {
@@ -139,7 +140,8 @@ static int validate(const mok_args* a, WsLayout* L, size_t extra_ws) {
                       a->config->cta_group < 0 || a->config->cta_group > 3 ||
                       a->config->host_chunks < 0 || a->config->host_chunks > MOK_MAX_HOST_CHUNKS ||
                       a->config->fused_ffn < 0 || a->config->fused_ffn > 2 || a->config->fused_window < -1 ||
-                      a->config->gang_sync < 0 || a->config->gang_sync > 2))
+                      a->config->gang_sync < 0 || a->config->gang_sync > 2 || a->config->serial_launches < 0 ||
+                      a->config->serial_launches > 1))
         return MOK_ERR_SHAPE;
     return MOK_OK;
 }
@@ -294,6 +296,7 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
     cudaError_t e = reset_header ? cudaMemsetAsync(hdr, 0, sizeof(WsHeader), s)
                                  : cudaMemsetAsync(&hdr->n_flag, 0, sizeof(hdr->n_flag), s);
     if (e != cudaSuccess) return cuda_fail(e);
+    g_pdl = !(a->config && a->config->serial_launches);
     cudaEvent_t* pev = profile_slot(a->config);
 #define MOK_MARK(i) do { if (pev) cudaEventRecord(pev[i], s); } while (0)
     MOK_MARK(0);

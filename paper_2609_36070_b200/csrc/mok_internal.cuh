@@ -163,6 +163,33 @@ cudaError_t launch_router_fused(const __nv_bfloat16* x, const __nv_bfloat16* spl
 
 inline __host__ __device__ size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// Programmatic dependent launch: the kernels of one forward call are launched with the "programmatic stream
+// serialization" attribute, so that a kernel's CTAs are scheduled (launch latency, parameter fetch) while its
+// predecessor in the stream is still running.  Device side, first thing in every such kernel: let the successor be
+// scheduled in turn, then wait until every predecessor grid has completed and its memory is visible.  Without the
+// attribute both instructions do nothing.
+__device__ __forceinline__ void pdl_enter() {
+#if defined(__CUDA_ARCH__)
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+#endif
+}
+extern thread_local bool g_pdl;       // set per forward call from config.serial_launches
+template <class... P, class... A>
+inline cudaError_t launch_pdl(void (*kernel)(P...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, A&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cfg.attrs = attr;
+    cfg.numAttrs = g_pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<P>(args)...);
+}
+
 // Launch state that belongs to ONE device.  cudaFuncSetAttribute (the opt-in to more than 48 KB of dynamic shared
 // memory) applies to the device that is current when it is called, and the SM count is a property of that device, so
 // a launcher that remembers "configured" per process would launch unconfigured kernels on a second GPU of the same

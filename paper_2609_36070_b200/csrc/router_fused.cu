@@ -81,6 +81,7 @@ router_fused_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_cons
     constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
     constexpr int N1 = (3 * EP > 256) ? 256 : 3 * EP, N2 = 3 * EP - N1;
     extern __shared__ uint8_t smem_raw[];
+    pdl_enter();
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t* smem = smem_raw + (base - raw);
@@ -296,8 +297,7 @@ static cudaError_t launch_one(const CUtensorMap& mA, const CUtensorMap& mB, Args
     a.tmem_cols = 3 * EP <= 128 ? 128u : 3 * EP <= 256 ? 256u : 512u;
     int blocks = a.n_tiles < sms ? a.n_tiles : sms;
     if (grid > 0 && grid < blocks) blocks = grid;
-    router_fused_kernel<NJ><<<blocks, THREADS, smem_bytes, s>>>(mA, mB, a);
-    return cudaGetLastError();
+    return launch_pdl(router_fused_kernel<NJ>, dim3(blocks), dim3(THREADS), (size_t)smem_bytes, s, mA, mB, a);
 }
 
 }  // namespace rf

@@ -140,6 +140,7 @@ template <int VPL>
 __global__ void __launch_bounds__(256)
 router_topk_kernel(const float* __restrict__ part, const float* __restrict__ bias, int T, int H, int E, int k, int ldl,
                    int32_t* __restrict__ idx, float* __restrict__ w, WsHeader* hdr, int32_t* __restrict__ flagged) {
+    pdl_enter();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_check = (k + 1 < E) ? k + 1 : E;        // slots compared pairwise
     const float guard_scale = (float)H * 1.4901161e-8f; // H * 2^-26
@@ -171,6 +172,7 @@ router_fixup_kernel(const float* __restrict__ part, const float* __restrict__ bi
                     const int32_t* __restrict__ flagged) {
     __shared__ int s_e[32];
     __shared__ float s_ex[32];
+    pdl_enter();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     int n_cand = (k + 4 < E) ? k + 4 : E;               // candidates recomputed
     if (n_cand > 32) n_cand = 32;
@@ -232,13 +234,13 @@ static cudaError_t launch_topk(const float* part, const float* bias, const __nv_
     if (!fused) {
         int tblocks = (T + 7) / 8;
         if (tblocks > 148 * 16) tblocks = 148 * 16;
-        router_topk_kernel<VPL><<<tblocks, 256, 0, s>>>(part, bias, T, H, E, k, ldl, idx, w, hdr, flagged);
-        cudaError_t e = cudaGetLastError();
+        cudaError_t e = launch_pdl(router_topk_kernel<VPL>, dim3(tblocks), dim3(256), 0, s, part, bias, T, H, E, k, ldl, idx, w,
+                                   hdr, flagged);
         if (e != cudaSuccess) return e;
     }
     // one block per listed token; 8 blocks fit on an SM at once, and blocks beyond the list's length leave at once
-    router_fixup_kernel<VPL><<<148 * 8, 256, 0, s>>>(part, bias, x, Wr, H, E, k, ldl, fused, idx, w, hdr, flagged);
-    return cudaGetLastError();
+    return launch_pdl(router_fixup_kernel<VPL>, dim3(148 * 8), dim3(256), 0, s, part, bias, x, Wr, H, E, k, ldl, fused, idx, w,
+                      (const WsHeader*)hdr, (const int32_t*)flagged);
 }
 
 cudaError_t launch_router_tc(const __nv_bfloat16* x, const float* Wr, const float* bias, int T, int H, int E, int k,

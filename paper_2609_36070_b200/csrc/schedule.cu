@@ -20,6 +20,7 @@ namespace mok {
 __global__ void __launch_bounds__(SCHED_THREADS)
 sched_hist_kernel(const int32_t* __restrict__ a, int n, int E, int32_t* __restrict__ blk_hist) {
     __shared__ int32_t hist[MAX_E];
+    pdl_enter();
     for (int e = threadIdx.x; e < E; e += SCHED_THREADS) hist[e] = 0;
     __syncthreads();
     int base = blockIdx.x * SCHED_CHUNK;
@@ -40,6 +41,7 @@ sched_scan_kernel(int32_t* __restrict__ blk_hist, int n_blk, int E, int max_mt, 
                   int32_t* __restrict__ mt_start2, int32_t* __restrict__ tile_expert2, WsHeader* __restrict__ hdr,
                   int32_t* __restrict__ counts_out, int32_t* __restrict__ offsets_out) {
     __shared__ int32_t s_cnt[MAX_E], s_off[MAX_E + 1], s_mt[MAX_E + 1], s_pad[MAX_E + 1], s_mt2[MAX_E + 1];
+    pdl_enter();
     const int e = threadIdx.x;
     int32_t total = 0;
     if (e < E) {
@@ -68,6 +70,7 @@ sched_scatter_kernel(const int32_t* __restrict__ a, int n, int E,
                      int32_t* __restrict__ row_token, int k,
                      int32_t* __restrict__ perm_out, int32_t* __restrict__ inv_out, int32_t* __restrict__ row_route) {
     extern __shared__ int32_t ssm[];                 // [SCHED_WARPS][E] running counters per warp
+    pdl_enter();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     int32_t* mine = ssm + warp * E;
     for (int e = threadIdx.x; e < SCHED_WARPS * E; e += SCHED_THREADS) ssm[e] = 0;
@@ -132,15 +135,17 @@ cudaError_t launch_schedule(const int32_t* idx, int T, int E, int k, int tile_m,
     int32_t* mt_start = reinterpret_cast<int32_t*>(ws + L.mt_start);
     int32_t* tile_expert = reinterpret_cast<int32_t*>(ws + L.tile_expert);
     WsHeader* hdr = reinterpret_cast<WsHeader*>(ws + L.header);
-    sched_hist_kernel<<<L.n_blk, SCHED_THREADS, 0, s>>>(idx, n, E, blk_hist);
-    sched_scan_kernel<<<1, MAX_E, 0, s>>>(blk_hist, L.n_blk, E, L.max_mt, tile_m, pad_m, counts, offsets, pad_offsets, mt_start,
-                                          tile_expert, reinterpret_cast<int32_t*>(ws + L.mt_start2),
-                                          reinterpret_cast<int32_t*>(ws + L.tile_expert2), hdr, counts_out, offsets_out);
-    sched_scatter_kernel<<<L.n_blk, SCHED_THREADS, sizeof(int32_t) * SCHED_WARPS * E, s>>>(
-        idx, n, E, blk_hist, offsets, pad_offsets,
-        reinterpret_cast<int32_t*>(ws + L.perm), reinterpret_cast<int32_t*>(ws + L.inv),
-        reinterpret_cast<int32_t*>(ws + L.pos), reinterpret_cast<int32_t*>(ws + L.row_token), k, perm_out, inv_out, row_route);
-    return cudaGetLastError();
+    cudaError_t e = launch_pdl(sched_hist_kernel, dim3(L.n_blk), dim3(SCHED_THREADS), 0, s, idx, n, E, blk_hist);
+    if (e != cudaSuccess) return e;
+    e = launch_pdl(sched_scan_kernel, dim3(1), dim3(MAX_E), 0, s, blk_hist, L.n_blk, E, L.max_mt, tile_m, pad_m, counts, offsets,
+                   pad_offsets, mt_start, tile_expert, reinterpret_cast<int32_t*>(ws + L.mt_start2),
+                   reinterpret_cast<int32_t*>(ws + L.tile_expert2), hdr, counts_out, offsets_out);
+    if (e != cudaSuccess) return e;
+    return launch_pdl(sched_scatter_kernel, dim3(L.n_blk), dim3(SCHED_THREADS), sizeof(int32_t) * SCHED_WARPS * E, s,
+                      idx, n, E, blk_hist, offsets, pad_offsets,
+                      reinterpret_cast<int32_t*>(ws + L.perm), reinterpret_cast<int32_t*>(ws + L.inv),
+                      reinterpret_cast<int32_t*>(ws + L.pos), reinterpret_cast<int32_t*>(ws + L.row_token), k, perm_out,
+                      inv_out, row_route);
 }
 
 }  // namespace mok
