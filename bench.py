@@ -78,6 +78,10 @@ def parse():
     p.add_argument("--host-chunks", type=int, default=0, help="token chunks of the host-buffer call (0 = auto)")
     p.add_argument("--precision", default="bf16", choices=["bf16", "mxfp8"],
                    help="routed experts in bf16 (the headline workload) or MXFP8 with pre-quantised weights")
+    p.add_argument("--parallelism", default="replicas", choices=["replicas", "ep"],
+                   help="replicas: every GPU holds all experts and its own batch (no data-path collective); ep: expert "
+                        "parallelism, every GPU holds E / N experts and its own batch of T tokens, rows are pulled from "
+                        "the peers' token buffers and combined by the token's owner")
     p.add_argument("--pass", dest="which", default="forward", choices=["forward", "backward"],
                    help="forward (the headline metric) or the backward pass of the same workload (bf16)")
     return p.parse_args()
@@ -588,6 +592,127 @@ def finish_record(rec, cfg, pk, mx, world=1):
     return rec
 
 
+def run_ep(args, cfg, rank, local_rank, world):
+    """`--parallelism ep`: the expert-parallel layer (Sections 2.1, 3.1-3.3) with one process per GPU.  Every rank keeps
+    T tokens of its own (weak scaling: N * T tokens per step in total) and E / N experts; per step it routes its tokens,
+    all-gathers the routes, builds Algorithm 1's schedule for its experts, runs their FFNs on rows pulled from the
+    owners' token buffers, and after one barrier combines its own tokens' rows from the serving ranks' buffers.
+    Same timing rules and JSON line as the replicated mode; `value` = N * T / the slowest rank's median step time."""
+    import statistics
+    import torch
+    import torch.distributed as dist
+    from paper_2609_36070_b200 import ep, inputs, mok, sharding
+    assert args.warmup >= 3, "timing rules: at least 3 warm-up steps"
+    assert cfg.E % world == 0, "the experts must divide over the ranks"
+    os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+    os.environ.setdefault("MASTER_PORT", "29543")
+    os.environ.setdefault("TORCH_SYMM_MEM_DISABLE_MULTICAST", "1")     # plain peer pointers only
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist.init_process_group("nccl", rank=rank, world_size=world, device_id=dev)
+    pk = peaks()
+    mx = args.precision == "mxfp8"
+    L = cfg.E // world
+    d = inputs.make_inputs(cfg, expert_range=(rank * L, (rank + 1) * L))
+    if rank > 0:
+        d["x"] = sharding.rank_tokens(cfg, rank)
+    g = {k: (None if d[k] is None else mok.to_device_bf16(d[k], dev)) for k in ("x", "W_gate_up", "W_down", "W_sgu", "W_sd")}
+    W_r = torch.from_numpy(d["W_r"]).to(dev)
+    bias = None if d["bias"] is None else torch.from_numpy(d["bias"]).to(dev)
+    mxw = mok.MxWeights(g["W_gate_up"], g["W_down"]) if mx else None
+    layer = ep.DistributedLayer(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k, dev, mx=mx)
+    out = torch.empty_like(g["x"])
+    conf = mok._config(cta_group=args.cta_group)
+
+    def step(x, timeline=None):
+        layer.forward(x, W_r, bias, g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], out=out, config=conf,
+                      mx_weights=mxw, timeline=timeline)
+
+    def barrier():
+        dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps):
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+        barrier()
+        t0 = time.time()
+        ev[0].record()
+        for i in range(steps):
+            fn(i)
+            ev[i + 1].record()
+        barrier()
+        return [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)], (t0, time.time())
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    for _ in range(args.warmup):
+        step(g["x"])
+    per, win = timed(lambda i: step(g["x"]), args.steps)
+    ms = sharding.max_over_ranks(statistics.median(per), dist, dev)
+    mean_ms = sharding.max_over_ranks(sum(per) / len(per), dist, dev)
+    assert layer.status() == 0, mok.mok_status_string(layer.status())
+    # phases, from a loop of their own with an event after each
+    phases = {}
+    n_ph = max(3, min(args.steps, 10))
+    for _ in range(n_ph):
+        tl = []
+        step(g["x"], tl)
+        torch.cuda.synchronize()
+        for (_, a), (name, b) in zip(tl, tl[1:]):
+            phases.setdefault(name, []).append(a.elapsed_time(b))
+    phases = {k: sharding.max_over_ranks(statistics.median(v), dist, dev) for k, v in phases.items()}
+    # end to end: the rank's tokens start in pinned host memory and its output ends there, every step
+    xh = g["x"].cpu().pin_memory()
+    oh = torch.empty_like(xh).pin_memory()
+
+    def e2e_step(i):
+        step(xh)
+        oh.copy_(out, non_blocking=True)
+
+    for _ in range(3):
+        e2e_step(0)
+    e2e_steps = max(5, min(args.steps, 50))
+    per_e, _ = timed(e2e_step, e2e_steps)
+    e2e_ms = sharding.max_over_ranks(statistics.median(per_e), dist, dev)
+    same_bits = bool(torch.equal(oh.view(torch.int16), out.cpu().view(torch.int16)))
+    sampler.stop() if rank == 0 else None
+    if rank == 0:
+        flops = 6.0 * cfg.T * cfg.H * (cfg.k * cfg.I + cfg.I_s)          # per rank: its experts serve N*T*k/N rows on average
+        peak = (2.0 if mx else 1.0) * pk["bf16_tflops"]
+        ffn_ms = phases["expert_ffn"]
+        act = 2 * cfg.T * cfg.H
+        clocks = sampler.window(*win)
+        line = {
+            "metric": METRIC, "value": world * cfg.T / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms, "mean_ms_per_step": mean_ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None,
+            "dtype": "mxfp8 routed experts (fp32 accumulate), bf16 elsewhere" if mx else "bf16", "data": "synthetic",
+            "config": {"workload": cfg.name, "T_per_gpu": cfg.T, "T_total": world * cfg.T, "H": cfg.H, "E": cfg.E,
+                       "experts_per_gpu": L, "k": cfg.k, "I": cfg.I, "I_shared": cfg.I_s, "routing": cfg.bias,
+                       "parallelism": f"ep{world}",
+                       "l2": "inputs larger than L2 (weights + activations >> 126 MB), no explicit flush",
+                       "timing": "ms_per_step = median of the per-step CUDA-event times of one bracketed loop (max over "
+                                 "ranks); phase times come from a second loop with an event after every phase"},
+            "tflops": world * flops / (ms * 1e-3) / 1e12,
+            "phase_ms": phases,
+            "roofline": {"kernel": "the rank's expert FFN call (Algorithm 1 schedule, routed gate/up with the pull gather "
+                                   "fused, down, shared expert)", "bound": "tensor",
+                         "achieved": flops / (ffn_ms * 1e-3) / 1e12, "peak": peak, "unit": "TFLOP/s",
+                         "frac": flops / (ffn_ms * 1e-3) / 1e12 / peak, "peak_kind": "burst (of measured)"
+                         if pk["source"] == "measured" else "burst (of fallback)", "traffic": None, "ms": ffn_ms},
+            "gpu_launches": args.steps * (mok.mok_launch_count(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k, conf) + 1),
+            "clocks": clocks,
+            "e2e": {"value": world * cfg.T / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms, "steps": e2e_steps,
+                    "h2d_bytes_per_step": act, "d2h_bytes_per_step": act,
+                    "mode": "per step: pinned host x -> the rank's peer-visible token buffer, the expert-parallel layer, "
+                            "out -> pinned host", "result_bits_equal_device_call": same_bits},
+        }
+        print(json.dumps(line), flush=True)
+    dist.barrier()
+    dist.destroy_process_group()
+
+
 def main():
     args = parse()
     rank = int(os.environ.get("RANK", "0"))
@@ -606,6 +731,9 @@ def main():
     if args.which == "backward":
         if rank == 0:
             run_backward(args, cfg)
+        return
+    if args.parallelism == "ep":
+        run_ep(args, cfg, rank, local_rank, world)
         return
 
     import gc

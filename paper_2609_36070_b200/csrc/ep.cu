@@ -259,6 +259,14 @@ static bool ep_layout(int n_ranks, int T_local, int H, int I, int Is, int E, int
     L->row_token = take(sizeof(int32_t) * (size_t)Rpad);
     L->h = take(2 * (size_t)Rpad * I);
     L->hs = take(Is > 0 ? 2 * (size_t)L->Tpad * Is : 0);
+    {   // gang-start counters of the 256-row kernel: one per tile of the largest of the four GEMMs
+        const long long mt2 = Rpad / (2 * TILE_M), mts = L->Tpad / (2 * TILE_M);
+        const long long n_r = (I + 127) / 128 > (H + 255) / 256 ? (I + 127) / 128 : (H + 255) / 256;
+        const long long n_s = (Is + 127) / 128 > (H + 255) / 256 ? (Is + 127) / 128 : (H + 255) / 256;
+        const long long tiles = mt2 * n_r > mts * n_s ? mt2 * n_r : mts * n_s;
+        L->gang_bytes = sizeof(int32_t) * (size_t)tiles;
+        L->gang = take(L->gang_bytes);
+    }
     if (mx) {
         if ((H % 32) || (I % 32)) return false;
         L->h8 = take((size_t)Rpad * I);
@@ -346,7 +354,7 @@ int mok_ep_expert_ffn(const mok_ep_args* a) {
 
     mok_config cfg;
     memset(&cfg, 0, sizeof(cfg));
-    if (a->config) { cfg.grid = a->config->grid; cfg.cta_group = a->config->cta_group; }
+    if (a->config) { cfg.grid = a->config->grid; cfg.cta_group = a->config->cta_group; cfg.gang_sync = a->config->gang_sync; }
     const __nv_bfloat16* x_own = reinterpret_cast<const __nv_bfloat16*>(a->x_peers[a->rank]);   // (may be NULL in MXFP8 mode without a shared expert)
     GemmArgs g;
     memset(&g, 0, sizeof(g));

@@ -239,7 +239,7 @@ int run_gemm(GemmArgs g, bool swiglu, const mok_config* cfg, const WsLayout& L, 
         const long long rows_all = g.dense_rows > 0 ? g.dense_rows : g.total_rows;
         const bool pays = gang_pays(w_bytes, rows_all, g.dense_rows > 0 ? 1 : g.E);
         const int mode = cfg ? cfg->gang_sync : 0;
-        if (L.gang_bytes > 0 && g.kgroup_rows == 0 && !g.b_mn && g.tile_sched != 1 && g.peer_tokens == 0 &&
+        if (L.gang_bytes > 0 && g.kgroup_rows == 0 && !g.b_mn && g.tile_sched != 1 &&
             (mode == 2 || (mode == 0 && pays))) {
             const long long rows = g.dense_rows > 0 ? g.dense_rows : g.rows_pad;
             const long long n_nt = swiglu ? (g.N + 127) / 128 : (g.N + 255) / 256;

@@ -151,11 +151,22 @@ class DistributedLayer:
         self.idx_all.copy_(torch.stack(parts))
 
     def forward(self, x_local, W_router, router_bias, W_gate_up_local, W_down_local, W_shared_gate_up, W_shared_down,
-                out=None, config=None, mx_weights=None):
-        """mx_weights: this rank's experts pre-quantised (mok.MxWeights) when the layer was built with mx=True."""
+                out=None, config=None, mx_weights=None, timeline=None):
+        """x_local: this rank's tokens, bf16 [T_local, H], on the device or in pinned host memory (it is copied into
+        the peer-visible buffer either way).  mx_weights: this rank's experts pre-quantised (mok.MxWeights) when the
+        layer was built with mx=True.  timeline: a list that receives (phase name, CUDA event recorded after it)."""
         st = self.st
+
+        def mark(name):
+            if timeline is not None:
+                ev = torch.cuda.Event(enable_timing=True)
+                ev.record()
+                timeline.append((name, ev))
+
+        mark("start")
         self._barrier()                         # peers have finished reading the previous layer's x / y / pos
-        self.x.copy_(x_local)
+        self.x.copy_(x_local, non_blocking=True)
+        mark("stage_x")
         if self.mx:                             # this rank's token rows as the peers' gather warps will pull them
             codes, scales = mok.mok_mx_quantize_rows(self.x)
             st.x_codes.copy_(codes)
@@ -164,14 +175,19 @@ class DistributedLayer:
             config.precision = mok.MOK_PRECISION_MXFP8
         st.idx, st.w = mok.mok_route(self.x, W_router, router_bias, self.k, st.route_ws)
         # the all-gather of the routes also orders every rank's x before any rank's pulls
+        mark("route")
         self._gather_routes(st.idx)
+        mark("gather_routes")
         mok.mok_ep_expert_ffn(self.rank, self.x_ptrs, self.idx_all, W_gate_up_local, W_down_local, W_shared_gate_up,
                               W_shared_down, self.E, self.k, st.y, st.pos, st.y_shared, st.ws, self.H, config=config,
                               mx_weights=mx_weights, x_codes_ptrs=self.xc_ptrs, x_scales_ptrs=self.xs_ptrs)
+        mark("expert_ffn")
         self._barrier()                         # every rank's y and pos are complete
+        mark("barrier")
         if out is None:
-            out = torch.empty_like(x_local)
+            out = torch.empty_like(self.x)
         mok.mok_ep_combine(self.rank, self.R, st.idx, st.w, self.y_ptrs, self.pos_ptrs, st.y_shared, self.E, out)
+        mark("combine")
         return out
 
     def status(self):

@@ -107,12 +107,13 @@ def make_x(cfg: MoEConfig) -> np.ndarray:
     return out
 
 
-def make_inputs(cfg: MoEConfig, threads: int = 0, experts: bool = True) -> dict:
+def make_inputs(cfg: MoEConfig, threads: int = 0, experts: bool = True, expert_range=None) -> dict:
     """All tensors of a workload as numpy arrays.
 
     Keys: x, W_r, bias, W_gate_up [E,2I,H], W_down [E,H,I], W_sgu [2I_s,H] | None, W_sd [H,I_s] | None.
     Expert weights are generated one expert per Philox stream, in a thread pool.  experts=False skips the
-    routed expert weights (for routing-only tests).
+    routed expert weights (for routing-only tests); expert_range=(lo, hi) generates only experts lo..hi-1 (the shard
+    of one expert-parallel rank: the same values as rows lo..hi-1 of the full tensors).
     """
     W_r, bias = make_router(cfg)
     d = {"x": make_x(cfg), "W_r": W_r, "bias": bias, "W_gate_up": None, "W_down": None,
@@ -121,19 +122,20 @@ def make_inputs(cfg: MoEConfig, threads: int = 0, experts: bool = True) -> dict:
         d["W_sgu"] = _normal_bf16(cfg.seed, _SGU, 0, (2 * cfg.I_s, cfg.H), 0.02)
         d["W_sd"] = _normal_bf16(cfg.seed, _SD, 0, (cfg.H, cfg.I_s), 0.02)
     if experts:
-        Wgu = np.empty((cfg.E, 2 * cfg.I, cfg.H), np.uint16)
-        Wd = np.empty((cfg.E, cfg.H, cfg.I), np.uint16)
+        lo, hi = expert_range if expert_range is not None else (0, cfg.E)
+        Wgu = np.empty((hi - lo, 2 * cfg.I, cfg.H), np.uint16)
+        Wd = np.empty((hi - lo, cfg.H, cfg.I), np.uint16)
 
         def one(e):
-            _normal_bf16(cfg.seed, _WGU, e, (2 * cfg.I, cfg.H), 0.02, out=Wgu[e])
-            _normal_bf16(cfg.seed, _WD, e, (cfg.H, cfg.I), 0.02, out=Wd[e])
+            _normal_bf16(cfg.seed, _WGU, e, (2 * cfg.I, cfg.H), 0.02, out=Wgu[e - lo])
+            _normal_bf16(cfg.seed, _WD, e, (cfg.H, cfg.I), 0.02, out=Wd[e - lo])
 
         n = threads or min(32, os.cpu_count() or 1)
-        if n > 1 and cfg.E > 1:
+        if n > 1 and hi - lo > 1:
             with ThreadPoolExecutor(n) as ex:
-                list(ex.map(one, range(cfg.E)))
+                list(ex.map(one, range(lo, hi)))
         else:
-            for e in range(cfg.E):
+            for e in range(lo, hi):
                 one(e)
         d["W_gate_up"], d["W_down"] = Wgu, Wd
     return d

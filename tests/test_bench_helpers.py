@@ -53,3 +53,17 @@ def test_reference_arm_prints_the_contract_line_on_the_smallest_workload():
     assert line["config"]["workload"] == "tiny" and line["value"] > 0 and line["higher_is_better"] is True
     assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["cores"] >= 1
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["e2e"]["value"] == line["value"]
+
+
+def test_expert_parallel_shard_of_the_inputs_equals_the_rows_of_the_full_tensors():
+    """make_inputs(expert_range=...) is what an expert-parallel rank generates: the same values as its rows of the
+    full expert tensors."""
+    import numpy as np
+    from paper_2609_36070_b200 import inputs
+    cfg = inputs.CONFIGS["tiny"]
+    full = inputs.make_inputs(cfg)
+    lo, hi = cfg.E // 2, cfg.E
+    part = inputs.make_inputs(cfg, expert_range=(lo, hi))
+    assert np.array_equal(part["W_gate_up"], full["W_gate_up"][lo:hi])
+    assert np.array_equal(part["W_down"], full["W_down"][lo:hi])
+    assert np.array_equal(part["x"], full["x"]) and np.array_equal(part["W_r"], full["W_r"])

@@ -162,6 +162,26 @@ def test_distributed_driver_with_a_world_of_one_rank():
     assert line["bitwise_equal_to_one_rank_layer"] and line["n_ranks"] == 1
 
 
+def test_bench_expert_parallel_mode_as_a_world_of_one_rank():
+    """`bench.py --parallelism ep` (one process per GPU, symmetric memory, NCCL) run alone: it prints the bench's JSON
+    line with the expert-parallel phases, and its host-buffer leg returns the bits of the device-resident leg."""
+    import json
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ, MASTER_ADDR="127.0.0.1", MASTER_PORT="29549", RANK="0", WORLD_SIZE="1", LOCAL_RANK="0",
+               NCCL_NVLS_ENABLE="0", TORCH_SYMM_MEM_DISABLE_MULTICAST="1")
+    r = subprocess.run([sys.executable, "bench.py", "--parallelism", "ep", "--config", "tiny", "--steps", "5",
+                        "--warmup", "3"], cwd=root, env=env, capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
+    line = json.loads([l for l in r.stdout.splitlines() if l.startswith("{")][-1])
+    assert line["config"]["parallelism"] == "ep1" and line["n_gpus"] == 1 and line["value"] > 0
+    assert set(line["phase_ms"]) == {"stage_x", "route", "gather_routes", "expert_ffn", "barrier", "combine"}
+    assert line["e2e"]["result_bits_equal_device_call"] and line["e2e"]["h2d_bytes_per_step"] > 0
+    assert line["gpu_launches"] > 0 and line["roofline"]["frac"] > 0
+
+
 @pytest.mark.parametrize("world,mx", [(2, False), (4, False), (2, True)], ids=["2_ranks", "4_ranks", "2_ranks_mxfp8"])
 def test_ranks_as_separate_processes_on_one_gpu(world, mx):
     """Real cross-process peer pointers: every rank is its own process on GPU 0, maps the other ranks' x / y / pos
