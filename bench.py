@@ -82,6 +82,9 @@ def parse():
                    help="replicas: every GPU holds all experts and its own batch (no data-path collective); ep: expert "
                         "parallelism, every GPU holds E / N experts and its own batch of T tokens, rows are pulled from "
                         "the peers' token buffers and combined by the token's owner")
+    p.add_argument("--ep-check", action="store_true",
+                   help="--parallelism ep with several ranks: compare with the one-rank layer even when that means "
+                        "loading all experts on every rank")
     p.add_argument("--pass", dest="which", default="forward", choices=["forward", "backward"],
                    help="forward (the headline metric) or the backward pass of the same workload (bf16)")
     return p.parse_args()
@@ -676,6 +679,22 @@ def run_ep(args, cfg, rank, local_rank, world):
     per_e, _ = timed(e2e_step, e2e_steps)
     e2e_ms = sharding.max_over_ranks(statistics.median(per_e), dist, dev)
     same_bits = bool(torch.equal(oh.view(torch.int16), out.cpu().view(torch.int16)))
+    # the bits of the one-rank layer: a token's output depends only on its own row and the weights, so every rank can
+    # run the replicated layer on its own tokens with all experts and compare.  Needs all experts on every rank, so
+    # with more than one rank it runs for workloads of at most 8 GB of expert weights, or when asked for.
+    bits_equal = None
+    w_bytes = 6.0 * cfg.E * cfg.H * cfg.I
+    if not mx and (world == 1 or args.ep_check or w_bytes <= 8e9):
+        full = g if world == 1 else {k: (None if v is None else mok.to_device_bf16(v, dev)) for k, v in
+                                     inputs.make_inputs(cfg).items() if k in ("W_gate_up", "W_down")}
+        ws1 = mok.alloc_workspace(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k, device=dev)
+        step(g["x"])
+        one = mok.mok_moe_forward_ex(g["x"], W_r, bias, full["W_gate_up"], full["W_down"], g["W_sgu"], g["W_sd"], cfg.k, ws1)
+        ok = torch.tensor([int(torch.equal(out.view(torch.int16), one.view(torch.int16)) and mok.mok_read_status(ws1) == 0)],
+                          device=dev)
+        dist.all_reduce(ok, op=dist.ReduceOp.MIN)
+        bits_equal = bool(ok.item())
+        del full, ws1, one
     sampler.stop() if rank == 0 else None
     if rank == 0:
         flops = 6.0 * cfg.T * cfg.H * (cfg.k * cfg.I + cfg.I_s)          # per rank: its experts serve N*T*k/N rows on average
@@ -695,6 +714,7 @@ def run_ep(args, cfg, rank, local_rank, world):
                        "timing": "ms_per_step = median of the per-step CUDA-event times of one bracketed loop (max over "
                                  "ranks); phase times come from a second loop with an event after every phase"},
             "tflops": world * flops / (ms * 1e-3) / 1e12,
+            "bitwise_equal_to_one_rank_layer": bits_equal,
             "phase_ms": phases,
             "roofline": {"kernel": "the rank's expert FFN call (Algorithm 1 schedule, routed gate/up with the pull gather "
                                    "fused, down, shared expert)", "bound": "tensor",

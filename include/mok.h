@@ -100,7 +100,10 @@ typedef struct mok_config {
                              2 = ONE persistent launch over a list of gate/up tiles and down tiles; a down tile runs
                              once a per-row-tile completion counter, advanced by the gate/up epilogues, shows that its
                              rows of the gated activation exist (Section 3.2: megakernel, GPU-local synchronisation
-                             instead of kernel boundaries).  Same bits either way. */
+                             instead of kernel boundaries).  3 = as 2, and the combine runs at the end of the same launch:
+                             the shared expert is then computed first, every epilogue warp reports its last store on a
+                             grid-wide counter, waits (bounded) for all of them and combines its share of the tokens in
+                             the slot order of the separate combine kernel.  Same bits in every mode. */
     int32_t fused_window; /* fused_ffn: list positions between a row group's gate/up tiles and its down tiles (0 = a
                              default of two to eight grids' worth of tiles; -1 = none: directly behind them, which makes
                              every down tile wait -- a test setting).  The list is walked with stride grid and

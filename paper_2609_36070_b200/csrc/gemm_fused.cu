@@ -39,6 +39,12 @@
 //
 // Shared-memory ring, tensor-memory use and the epilogue arithmetic are those of gemm_tcgen05_m2.cu; during D tiles the
 // gather warps skip ahead and the producer makes their arrivals on the ring's barriers.
+//
+// Optionally the COMBINE (Section 2.1: out[t] = shared[t] + sum_s w[t,s] * y[pos[t,s]]) runs in the same launch: a token's
+// k rows lie anywhere in y, so it can only start when every down tile has been stored.  Every epilogue warp adds one
+// arrival to a grid-wide counter once its last store has completed, waits (bounded) until all epilogue warps of the grid
+// have arrived; then the epilogue and gather warps draw tokens from a global counter and combine them, one token per
+// warp at a time, in the fixed slot order of the separate combine kernel (same bits).
 #include "mok_internal.cuh"
 #include "tc_ptx.cuh"
 #include "tensor_map.cuh"
@@ -225,6 +231,8 @@ fused_tiles_kernel(const int32_t* __restrict__ counts, const int32_t* __restrict
     if (blockIdx.x == 0 && tid == 0) {
         hdr->n_ftiles = total <= max_tiles ? (int32_t)total : 0;
         hdr->next_tile = 0;
+        hdr->ffn_done = 0;
+        hdr->combine_next = 0;
         if (total > max_tiles) atomicCAS(&hdr->status, 0, (int)MOK_ERR_SCHEDULE);
     }
     if (total > max_tiles) return;
@@ -317,7 +325,123 @@ struct FusedArgs {
     int32_t dbg;                   // != 0: counters into header->dbg[1] (gate/up tiles) and [2] (down tiles)
     int32_t starve;                // test hook: the producer issues nothing
     WsHeader* header;
+    // combine in the same launch (out != NULL)
+    const __nv_bfloat16* y;        // [Rpad, H] rows of the down tiles
+    const __nv_bfloat16* ysh;      // [T, H] shared expert's output, or NULL
+    const int32_t* pos;            // [T * k] padded row of every route
+    const float* w;                // [T * k] router weights
+    __nv_bfloat16* out;            // [T, H], or NULL: no combine in this launch
+    int32_t T, k;
 };
+
+// The combine of this launch, run warp by warp after a warp's last tile.  An epilogue warp first adds its arrival to the
+// grid-wide counter (its stores have completed); every participating warp then waits (bounded) for all
+// EPI_WARPS * gridDim.x arrivals and draws tokens from a global counter, one token per warp at a time: 16 bytes per
+// lane and row, CH chunks of a row per pass with the k rows of every chunk loaded before the first multiply-add,
+// accumulation in fp32 in slot order on top of the shared expert's row.
+template <int CH>
+__device__ __forceinline__ void combine_tokens(const FusedArgs& a, int lane, volatile uint32_t* abort_flag, bool arrive) {
+    int32_t* done = &a.header->ffn_done;
+    const int need = EPI_WARPS * (int)gridDim.x;
+    int ok = 1;
+    if (lane == 0) {
+        if (arrive) {
+            // (the warp's TMA stores have completed: make them visible to generic-proxy reads of other SMs, then arrive)
+            asm volatile("fence.proxy.async;" ::: "memory");
+            __threadfence();
+            asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(done) : "memory");
+        }
+        const unsigned long long t0 = globaltimer();
+        uint32_t spins = 0;
+        while (ld_acquire(done) < need) {
+            __nanosleep(128);
+            if ((++spins & 63u) == 0u) {
+                if (*abort_flag) { ok = 0; break; }
+                const unsigned long long limit = a.header->wait_limit_us ? 1000ull * a.header->wait_limit_us : WAIT_LIMIT_NS;
+                if (globaltimer() - t0 > limit) {
+                    *abort_flag = 1u;
+                    atomicCAS(&a.header->status, 0, (int)MOK_ERR_TIMEOUT);
+                    a.header->where = 44;
+                    ok = 0;
+                    break;
+                }
+            }
+        }
+    }
+    ok = __shfl_sync(0xffffffffu, ok, 0);
+    if (!ok) return;
+    const int chunks = a.H >> 3, k = a.k;
+    for (;;) {
+        int t = 0;
+        if (lane == 0) t = atomicAdd(&a.header->combine_next, 1);
+        t = __shfl_sync(0xffffffffu, t, 0);
+        if (t >= a.T) break;
+        int my_pos = 0;
+        float my_w = 0.f;
+        if (lane < k) {
+            my_pos = __ldg(a.pos + (size_t)t * k + lane);
+            my_w = __ldg(a.w + (size_t)t * k + lane);
+        }
+        // (the trip count is the same for every lane: the loop body exchanges values between lanes)
+        for (int c0 = 0; c0 < chunks; c0 += 32 * CH) {
+            float acc[CH][8];
+#pragma unroll
+            for (int u = 0; u < CH; ++u) {
+                const int c = c0 + u * 32 + lane;
+                if (a.ysh && c < chunks) {
+                    const uint4 raw = __ldcg(reinterpret_cast<const uint4*>(a.ysh + (size_t)t * a.H) + c);
+                    const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&raw);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const float2 f = __bfloat1622float2(p2[i]);
+                        acc[u][2 * i] = f.x;
+                        acc[u][2 * i + 1] = f.y;
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) acc[u][i] = 0.f;
+                }
+            }
+            for (int s0 = 0; s0 < k; s0 += 8) {
+                uint4 v[CH][8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const int row = __shfl_sync(0xffffffffu, my_pos, (s0 + j) & 31);
+#pragma unroll
+                    for (int u = 0; u < CH; ++u) {
+                        const int c = c0 + u * 32 + lane;
+                        if (c < chunks && s0 + j < k) v[u][j] = __ldcg(reinterpret_cast<const uint4*>(a.y + (size_t)row * a.H) + c);
+                    }
+                }
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const float wv = __shfl_sync(0xffffffffu, my_w, (s0 + j) & 31);
+#pragma unroll
+                    for (int u = 0; u < CH; ++u) {
+                        if (c0 + u * 32 + lane < chunks && s0 + j < k) {
+                            const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&v[u][j]);
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                const float2 f = __bfloat1622float2(p2[i]);
+                                acc[u][2 * i] = fmaf(wv, f.x, acc[u][2 * i]);
+                                acc[u][2 * i + 1] = fmaf(wv, f.y, acc[u][2 * i + 1]);
+                            }
+                        }
+                    }
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < CH; ++u) {
+                const int c = c0 + u * 32 + lane;
+                uint4 o;
+                __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&o);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) o2[i] = __floats2bfloat162_rn(acc[u][2 * i], acc[u][2 * i + 1]);
+                if (c < chunks) *(reinterpret_cast<uint4*>(a.out + (size_t)t * a.H) + c) = o;
+            }
+        }
+    }
+}
 
 // Registers are handed from the light roles to the epilogue (setmaxnreg, per group of four warps): the producer /
 // issuer / scheduler group and the gather group give up most of theirs, and the two epilogue groups get enough to hold
@@ -659,6 +783,8 @@ fused_ffn_kernel(const __grid_constant__ CUtensorMap mapWgu, const __grid_consta
             if (!ok) break;
         }
         asm volatile("cp.async.wait_all;" ::: "memory");
+        // (the gather warps help with the combine: more bytes in flight per SM)
+        if (__all_sync(0xffffffffu, a.out != nullptr && !*abort_flag)) combine_tokens<1>(a, lane, abort_flag, false);
     } else {
         // ------------------------------------------------------------------ epilogue warps
         reg_inc<REGS_EPILOGUE>();
@@ -762,6 +888,8 @@ fused_ffn_kernel(const __grid_constant__ CUtensorMap mapWgu, const __grid_consta
         }
         if (lane == 0) tma_store_wait_all();
         __syncwarp();
+        // (one decision per warp: the combine exchanges values between lanes)
+        if (__all_sync(0xffffffffu, a.out != nullptr && !*abort_flag)) combine_tokens<2>(a, lane, abort_flag, true);
     }
 
     // ---------------------------------------------------------------------- teardown
@@ -814,7 +942,8 @@ static cudaError_t launch_kernel(int grid, cudaStream_t s, const CUtensorMap& m0
 // (a group's down tiles directly behind its gate/up tiles).
 cudaError_t launch_fused_ffn(const __nv_bfloat16* x, int T, int H, int I, int E, const __nv_bfloat16* Wgu,
                              const __nv_bfloat16* Wd, const WsLayout& L, char* ws, int grid, int window_tiles, bool dynamic,
-                             bool gang_sync, bool dbg, bool starve, cudaStream_t s) {
+                             bool gang_sync, bool dbg, bool starve, cudaStream_t s, __nv_bfloat16* combine_out, int k,
+                             bool shared) {
     using namespace ff;
     int dev = 0, sm_count = 0;
     cudaError_t e = current_device(&dev);
@@ -870,7 +999,13 @@ cudaError_t launch_fused_ffn(const __nv_bfloat16* x, int T, int H, int I, int E,
     a.dbg = dbg ? 1 : 0;
     a.starve = starve ? 1 : 0;
     a.header = hdr;
-    (void)T;
+    a.y = reinterpret_cast<const __nv_bfloat16*>(y);
+    a.ysh = shared ? reinterpret_cast<const __nv_bfloat16*>(ws + L.ysh) : nullptr;
+    a.pos = reinterpret_cast<const int32_t*>(ws + L.pos);
+    a.w = reinterpret_cast<const float*>(ws + L.w);
+    a.out = combine_out;
+    a.T = T;
+    a.k = k;
 
     return dynamic ? launch_kernel<true>(grid, s, mWgu, mWgu64, mHst, mHld, mWd, mY, a)
                    : launch_kernel<false>(grid, s, mWgu, mWgu64, mHst, mHld, mWd, mY, a);

@@ -18,14 +18,35 @@ int cuda_fail(cudaError_t e) {
 
 // Event sets of the per-stage profiler (mok_profile_begin / mok_profile_end).
 struct Profiler {
-    cudaEvent_t* ev = nullptr;      // [max_calls][MOK_STAGE_COUNT + 1]
+    cudaEvent_t* ev = nullptr;      // [max_calls][MOK_STAGE_COUNT + 1]: event 0 opens the call, event st + 1 closes stage st
+    uint8_t* pred = nullptr;        // [max_calls][MOK_STAGE_COUNT]: the event recorded just before stage st's closing event
+                                    // (stages do not always run in the order of their numbers)
     int max_calls = 0, n_calls = 0;
 };
 static Profiler g_prof;
 
-static cudaEvent_t* profile_slot(const mok_config* cfg) {
-    if (!cfg || !cfg->profile || !g_prof.ev || g_prof.n_calls >= g_prof.max_calls) return nullptr;
-    return g_prof.ev + (size_t)(g_prof.n_calls++) * (MOK_STAGE_COUNT + 1);
+struct ProfileMarks {
+    cudaEvent_t* ev = nullptr;
+    uint8_t* pred = nullptr;
+    int last = 0;
+    cudaStream_t s = nullptr;
+    void open() { if (ev) cudaEventRecord(ev[0], s); }
+    void close(int stage) {
+        if (!ev) return;
+        cudaEventRecord(ev[stage + 1], s);
+        pred[stage] = (uint8_t)last;
+        last = stage + 1;
+    }
+};
+
+static ProfileMarks profile_slot(const mok_config* cfg, cudaStream_t s) {
+    ProfileMarks m;
+    if (!cfg || !cfg->profile || !g_prof.ev || g_prof.n_calls >= g_prof.max_calls) return m;
+    const int c = g_prof.n_calls++;
+    m.ev = g_prof.ev + (size_t)c * (MOK_STAGE_COUNT + 1);
+    m.pred = g_prof.pred + (size_t)c * MOK_STAGE_COUNT;
+    m.s = s;
+    return m;
 }
 
 static bool sizes_ok(int T, int H, int I, int Is, int E, int k) {
@@ -139,7 +160,7 @@ static int validate(const mok_args* a, WsLayout* L, size_t extra_ws) {
                       a->config->gather_mode < 0 || a->config->gather_mode > 2 ||
                       a->config->cta_group < 0 || a->config->cta_group > 3 ||
                       a->config->host_chunks < 0 || a->config->host_chunks > MOK_MAX_HOST_CHUNKS ||
-                      a->config->fused_ffn < 0 || a->config->fused_ffn > 2 || a->config->fused_window < -1 ||
+                      a->config->fused_ffn < 0 || a->config->fused_ffn > 3 || a->config->fused_window < -1 ||
                       a->config->gang_sync < 0 || a->config->gang_sync > 2 || a->config->serial_launches < 0 ||
                       a->config->serial_launches > 1))
         return MOK_ERR_SHAPE;
@@ -210,7 +231,7 @@ static bool gang_pays(long long w_bytes, long long rows, int experts) {
 // Routed gate/up + SwiGLU + down as ONE persistent launch (gemm_fused.cu).  Chosen by default where synchronised tile
 // starts pay for both GEMMs (there it equals or beats the two launches: DeepSeek-like -1.6 %, GPT-OSS-like -4 %, two
 // variants alternating in one process); elsewhere the two launches are 1-2 % faster and stay the default.
-// fused_ffn = 1 / 2 force the two launches / the one launch.
+// fused_ffn = 1 / 2 force the two launches / the one launch; 3 = the one launch with the combine at its end.
 static bool fused_gang(const mok_config* cfg, int H, int I, long long rows, int experts) {
     const int mode = cfg ? cfg->gang_sync : 0;
     if (mode == 1) return false;
@@ -221,7 +242,7 @@ static bool use_fused_ffn(const mok_config* cfg, int H, int I, int tile_m, long 
     if (use_simt(cfg) || use_tn(cfg) || use_mx(cfg) || tile_m != TILE_M || max_ftiles <= 0) return false;
     if (cfg && (cfg->fused_ffn == 1 || cfg->cta_group == 1 || cfg->cta_group == 2)) return false;
     if (!fused_gather(cfg, I)) return false;
-    if (cfg && cfg->fused_ffn == 2) return true;
+    if (cfg && cfg->fused_ffn >= 2) return true;
     if (cfg && cfg->tile_sched == 1) return false;          // (tile stealing belongs to the two-launch path)
     // (at least two row tiles per expert on average: with single tiles there is nothing to start together, and the
     //  weight-streaming regime of small batches is served better by the two launches: 4.64 vs 4.80 ms at 128 rows)
@@ -297,9 +318,9 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
                                  : cudaMemsetAsync(&hdr->n_flag, 0, sizeof(hdr->n_flag), s);
     if (e != cudaSuccess) return cuda_fail(e);
     g_pdl = !(a->config && a->config->serial_launches);
-    cudaEvent_t* pev = profile_slot(a->config);
-#define MOK_MARK(i) do { if (pev) cudaEventRecord(pev[i], s); } while (0)
-    MOK_MARK(0);
+    ProfileMarks marks = profile_slot(a->config, s);
+#define MOK_MARK(i) marks.close((i) - 1)
+    marks.open();
     int rc = route_stage(a, L, ws, x, s);
     if (rc) return rc;
     MOK_MARK(MOK_STAGE_ROUTER + 1);
@@ -344,6 +365,38 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
         if (e != cudaSuccess) return cuda_fail(e);
         g.starve = 1;
     }
+    bool combine_in_launch = false;
+    // shared expert: every token in natural order, no gather.  Runs after the routed experts, or before them when the
+    // routed experts' launch ends with the combine
+    auto shared_expert = [&]() -> int {
+        GemmArgs gs = g;
+        gs.dbg_slot = dbg ? 3 : -1;
+        gs.row_token = nullptr;
+        gs.starve = 0;
+        gs.tile_sched = 0;
+        gs.sfa = gs.sfb = nullptr;
+        gs.sfc = nullptr;
+        int rcs = MOK_OK;
+        if (a->I_shared > 0) {
+            gs.A = x;
+            gs.B = reinterpret_cast<const __nv_bfloat16*>(a->W_shared_gate_up);
+            gs.C = ws + L.hs;
+            gs.K = a->H; gs.N = a->I_shared; gs.ldc = a->I_shared; gs.E = 1; gs.rows_pad = L.Tpad; gs.a_rows = a->T;
+            gs.dense_rows = a->T;
+            if ((rcs = run_gemm(gs, true, a->config, L, ws, s))) return rcs;
+            MOK_MARK(MOK_STAGE_SHARED_GEMM1 + 1);
+            gs.A = reinterpret_cast<const __nv_bfloat16*>(ws + L.hs);
+            gs.B = reinterpret_cast<const __nv_bfloat16*>(a->W_shared_down);
+            gs.C = ws + L.ysh;
+            gs.K = a->I_shared; gs.N = a->H; gs.ldc = a->H; gs.a_rows = L.Tpad;
+            if ((rcs = run_gemm(gs, false, a->config, L, ws, s))) return rcs;
+            MOK_MARK(MOK_STAGE_SHARED_GEMM2 + 1);
+        } else {
+            MOK_MARK(MOK_STAGE_SHARED_GEMM1 + 1);
+            MOK_MARK(MOK_STAGE_SHARED_GEMM2 + 1);
+        }
+        return rcs;
+    };
     if (mx) {
         // routed experts on MXFP8 operands (Section 3.4): h = Q(silu(Q(x) Wg_q^T) * (Q(x) Wu_q^T));  y = h Wd_q^T
         const int grid = a->config->grid;
@@ -402,6 +455,8 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
         g.total_rows = L.R;
         g.tile_sched = a->config ? a->config->tile_sched : 0;
         const bool fused = !simt && use_fused_ffn(a->config, a->H, a->I, tile_m, L.R, a->E, L.max_ftiles);
+        combine_in_launch = fused && a->config && a->config->fused_ffn == 3;
+        if (combine_in_launch && (rc = shared_expert())) return rc;       // its output is an input of that launch
         // its hand-out: synchronised starts need the static stride (a CTA that draws ahead could hold two tiles of a gang)
         const bool fused_sync = fused_gang(a->config, a->H, a->I, L.R, a->E);
         const int sched = a->config ? a->config->tile_sched : 0;
@@ -409,7 +464,8 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
         if (fused) {
             e = launch_fused_ffn(x, a->T, a->H, a->I, a->E, reinterpret_cast<const __nv_bfloat16*>(a->W_gate_up),
                                  reinterpret_cast<const __nv_bfloat16*>(a->W_down), L, ws, a->config ? a->config->grid : 0,
-                                 a->config ? a->config->fused_window : 0, fused_dynamic, fused_sync, dbg, g.starve != 0, s);
+                                 a->config ? a->config->fused_window : 0, fused_dynamic, fused_sync, dbg, g.starve != 0, s,
+                                 combine_in_launch ? out : nullptr, a->k, a->I_shared > 0);
             if (e != cudaSuccess) return cuda_fail(e);
         } else if ((rc = run_gemm(g, true, a->config, L, ws, s))) return rc;
         g.row_token = nullptr;
@@ -425,26 +481,11 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
         g.tile_sched = 0;
     }
     MOK_MARK(MOK_STAGE_GEMM2 + 1);
-    g.dbg_slot = dbg ? 3 : -1;
-    if (a->I_shared > 0) {   // shared expert: every token in natural order, no gather
-        g.A = x;
-        g.B = reinterpret_cast<const __nv_bfloat16*>(a->W_shared_gate_up);
-        g.C = ws + L.hs;
-        g.K = a->H; g.N = a->I_shared; g.ldc = a->I_shared; g.E = 1; g.rows_pad = L.Tpad; g.a_rows = a->T; g.dense_rows = a->T;
-        if ((rc = run_gemm(g, true, a->config, L, ws, s))) return rc;
-        MOK_MARK(MOK_STAGE_SHARED_GEMM1 + 1);
-        g.A = reinterpret_cast<const __nv_bfloat16*>(ws + L.hs);
-        g.B = reinterpret_cast<const __nv_bfloat16*>(a->W_shared_down);
-        g.C = ws + L.ysh;
-        g.K = a->I_shared; g.N = a->H; g.ldc = a->H; g.a_rows = L.Tpad;
-        if ((rc = run_gemm(g, false, a->config, L, ws, s))) return rc;
-        MOK_MARK(MOK_STAGE_SHARED_GEMM2 + 1);
-    } else {
-        MOK_MARK(MOK_STAGE_SHARED_GEMM1 + 1);
-        MOK_MARK(MOK_STAGE_SHARED_GEMM2 + 1);
+    if (!combine_in_launch) {
+        if ((rc = shared_expert())) return rc;
+        e = launch_combine(L, ws, a->T, a->H, a->k, a->I_shared > 0, out, s);
+        if (e != cudaSuccess) return cuda_fail(e);
     }
-    e = launch_combine(L, ws, a->T, a->H, a->k, a->I_shared > 0, out, s);
-    if (e != cudaSuccess) return cuda_fail(e);
     MOK_MARK(MOK_STAGE_COMBINE + 1);
 #undef MOK_MARK
     return MOK_OK;
@@ -812,7 +853,10 @@ int mok_launch_count(int T, int H, int I, int I_shared, int E, int k, const mok_
     const int pre = use_mx(config) ? 1 : (fused_gather(config, I) ? 0 : 1);
     // (with mok_args.W_router_split the router's split kernel is not launched: one launch less than counted here;
     //  with config.fused_ffn = 2 the two routed GEMMs are the tile-list kernel + ONE persistent kernel: the same count)
-    return (use_simt_router(config, k) ? 1 : use_fused_router(config, E, k) ? 3 : 4) + 3 + pre + 2 + (I_shared > 0 ? 2 : 0) + 1;
+    //  with config.fused_ffn = 3 that kernel also does the combine: one launch less)
+    const int tile_m = use_mx(config) ? TILE_M : tile_rows(config, I);
+    const int combine = config && config->fused_ffn == 3 && use_fused_ffn(config, H, I, tile_m, L.R, E, L.max_ftiles) ? 0 : 1;
+    return (use_simt_router(config, k) ? 1 : use_fused_router(config, E, k) ? 3 : 4) + 3 + pre + 2 + (I_shared > 0 ? 2 : 0) + combine;
 }
 
 int mok_profile_begin(int max_calls) {
@@ -829,6 +873,8 @@ int mok_profile_begin(int max_calls) {
             return cuda_fail(e);
         }
     }
+    g_prof.pred = new uint8_t[(size_t)max_calls * MOK_STAGE_COUNT];
+    for (size_t i = 0; i < (size_t)max_calls * MOK_STAGE_COUNT; ++i) g_prof.pred[i] = (uint8_t)(i % MOK_STAGE_COUNT);
     g_prof.max_calls = max_calls;
     g_prof.n_calls = 0;
     return MOK_OK;
@@ -846,7 +892,7 @@ int mok_profile_end(float* ms, int max_calls_out, int* n_calls) {
         cudaEvent_t* ev = g_prof.ev + (size_t)c * (MOK_STAGE_COUNT + 1);
         for (int st = 0; st < MOK_STAGE_COUNT; ++st) {
             float t = 0.f;
-            cudaError_t e = cudaEventElapsedTime(&t, ev[st], ev[st + 1]);
+            cudaError_t e = cudaEventElapsedTime(&t, ev[g_prof.pred[(size_t)c * MOK_STAGE_COUNT + st]], ev[st + 1]);
             if (e != cudaSuccess) { rc = cuda_fail(e); break; }
             ms[(size_t)c * MOK_STAGE_COUNT + st] = t;
         }
@@ -855,6 +901,7 @@ int mok_profile_end(float* ms, int max_calls_out, int* n_calls) {
     const size_t total = (size_t)g_prof.max_calls * (MOK_STAGE_COUNT + 1);
     for (size_t i = 0; i < total; ++i) cudaEventDestroy(g_prof.ev[i]);
     delete[] g_prof.ev;
+    delete[] g_prof.pred;
     g_prof = Profiler();
     return rc;
 }

@@ -26,7 +26,9 @@ struct WsHeader {
     int32_t n_flag;        // tensor-core router: tokens on the near-tie list of the current call
     int32_t n_ftiles;      // length of the fused expert-FFN kernel's tile list (gate/up tiles + down tiles)
     int32_t next_tile;     // its dynamic hand-out: the next list position to draw
-    int32_t pad[56];
+    int32_t ffn_done;      // that kernel's epilogue warps whose last store has completed (gate of its in-launch combine)
+    int32_t combine_next;  // its in-launch combine: the next token to draw
+    int32_t pad[54];
     // optional counters of the tcgen05 GEMMs (config.debug): [slot][counter]; SM cycles summed over CTAs unless stated
     unsigned long long dbg[4][MOK_DEBUG_COUNTERS];
 };
@@ -147,7 +149,8 @@ cudaError_t launch_gemm_mx(const GemmArgs& a, int epi, int grid, cudaStream_t s)
 // routed gate/up + SwiGLU + down in one persistent launch (tile list + kernel); needs the schedule's 256-row tile table
 cudaError_t launch_fused_ffn(const __nv_bfloat16* x, int T, int H, int I, int E, const __nv_bfloat16* Wgu,
                              const __nv_bfloat16* Wd, const WsLayout& L, char* ws, int grid, int window_tiles, bool dynamic,
-                             bool gang_sync, bool dbg, bool starve, cudaStream_t s);
+                             bool gang_sync, bool dbg, bool starve, cudaStream_t s, __nv_bfloat16* combine_out = nullptr,
+                             int k = 0, bool shared = false);   // combine_out != NULL: the combine runs in the same launch
 cudaError_t launch_mx_quantize_rows(const __nv_bfloat16* in, long long rows, int K, uint8_t* codes, uint8_t* scales,
                                     cudaStream_t s);
 cudaError_t launch_mx_quantize_atoms(const __nv_bfloat16* in, int groups, int rows_per_group, int K, uint8_t* codes,

@@ -177,6 +177,7 @@ def test_bench_expert_parallel_mode_as_a_world_of_one_rank():
     assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
     line = json.loads([l for l in r.stdout.splitlines() if l.startswith("{")][-1])
     assert line["config"]["parallelism"] == "ep1" and line["n_gpus"] == 1 and line["value"] > 0
+    assert line["bitwise_equal_to_one_rank_layer"] is True
     assert set(line["phase_ms"]) == {"stage_x", "route", "gather_routes", "expert_ffn", "barrier", "combine"}
     assert line["e2e"]["result_bits_equal_device_call"] and line["e2e"]["h2d_bytes_per_step"] > 0
     assert line["gpu_launches"] > 0 and line["roofline"]["frac"] > 0

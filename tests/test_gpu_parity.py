@@ -359,9 +359,23 @@ def test_one_launch_ffn_gives_the_bits_of_two_launches(cfg):
                # static stride with synchronised tile starts (what large expert matrices get by default)
                {"gang_sync": 2}, {"gang_sync": 2, "fused_window": -1}, {"gang_sync": 2, "grid": 8},
                {"gang_sync": 2, "grid": 11, "fused_window": 40}, {"gang_sync": 2, "grid": 3},
-               {"gang_sync": 2, "tile_sched": 1}):
-        out1 = pu.run_gpu(cfg, g, config=m._config(fused_ffn=2, **kw), stages=False)
+               {"gang_sync": 2, "tile_sched": 1},
+               # the combine at the end of the same launch (the shared expert then runs first)
+               {"fused_ffn": 3}, {"fused_ffn": 3, "grid": 1}, {"fused_ffn": 3, "fused_window": -1, "grid": 37},
+               {"fused_ffn": 3, "tile_sched": 2, "grid": 5}, {"fused_ffn": 3, "gang_sync": 2},
+               {"fused_ffn": 3, "gang_sync": 2, "grid": 11, "fused_window": 40}):
+        out1 = pu.run_gpu(cfg, g, config=m._config(**(dict(fused_ffn=2) | kw)), stages=False)
         assert torch.equal(out1.view(torch.int16), out2.view(torch.int16)), kw
+    # ... and against the oracle with the stage outputs requested, and under the per-stage profiler (the stages then run
+    # in another order than their numbers: every stage time must still be a non-negative interval)
+    out3, st3, rep3 = pu.full_parity(cfg, d=d, g=g, config=m._config(fused_ffn=3))
+    assert torch.equal(out3.view(torch.int16), out2.view(torch.int16))
+    m.mok_profile_begin(2)
+    for _ in range(2):
+        pu.run_gpu(cfg, g, config=m._config(fused_ffn=3, profile=1), stages=False)
+    ms = m.mok_profile_end(2)
+    assert len(ms) == 2 and all(v >= 0.0 for call in ms for v in call.values()), ms
+    assert all(call["combine"] < 0.05 and call["gemm1"] > 0.0 for call in ms), ms
 
 
 @pytest.mark.parametrize("cfg", MID + [SMALL[0], SMALL[6]], ids=[c.name for c in MID + [SMALL[0], SMALL[6]]])
@@ -382,7 +396,7 @@ def test_synchronised_tile_starts_give_the_same_bits(cfg):
         assert torch.equal(out.view(torch.int16), ref.view(torch.int16)), grid
 
 
-@pytest.mark.parametrize("fused,sched,gang", [(1, 0, 0), (2, 0, 0), (2, 2, 0), (2, 0, 2), (1, 0, 2)])
+@pytest.mark.parametrize("fused,sched,gang", [(1, 0, 0), (2, 0, 0), (2, 2, 0), (2, 0, 2), (1, 0, 2), (3, 0, 0), (3, 2, 0)])
 def test_bounded_waits_report_a_timeout_and_leave_the_context_usable(fused, sched, gang):
     """Failure detection without a fault: the test hook silences the gate/up GEMM's TMA producer, so its MMA issuer
     waits for operands that never come.  Every wait is bounded (2 ms here), the kernel records MOK_ERR_TIMEOUT, frees
