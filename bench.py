@@ -58,7 +58,10 @@ def parse():
     p.add_argument("--experts", type=int, default=0,
                    help="override E: with --tokens, a scaled copy of a workload (same H, I, k and rows per expert) that is "
                         "small enough for a profiler capture")
-    p.add_argument("--fused-ffn", type=int, default=0, help="2: routed gate/up + down GEMM as one persistent launch")
+    p.add_argument("--fused-ffn", type=int, default=0, help="2: routed gate/up + down GEMM as one persistent launch; 3: and the combine")
+    p.add_argument("--h-ring", type=int, default=0,
+                   help="slots (256 rows each, >= 24) of a ring that holds the gated activation, in the smaller workspace "
+                        "that goes with it (0 = a row for every route)")
     p.add_argument("--cpu-sample", type=int, default=0, help="tokens of the CPU-oracle sample (0 = auto)")
     p.add_argument("--no-cpu-baseline", action="store_true")
     p.add_argument("--per-config", default="auto",
@@ -337,7 +340,7 @@ class Layer:
         self.prec = mok.MOK_PRECISION_MXFP8 if self.mx else mok.MOK_PRECISION_BF16
         self.mxw = mok.MxWeights(self.g["W_gate_up"], self.g["W_down"]) if self.mx else None
         self.ws = mok.alloc_workspace(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k, device=dev, host_staging=staging,
-                                      mx=self.mx)
+                                      mx=self.mx, h_ring_tiles=args.h_ring)
         # the router weights are split once, as a caller of the library would do at load time
         try:
             self.split = mok.mok_router_prepare(self.W_r, cfg.k, self.conf())
@@ -348,7 +351,7 @@ class Layer:
     def conf(self, **kw):
         a = self.args
         base = dict(impl=a.gemm, gather_mode=a.gather_mode, cta_group=a.cta_group, precision=self.prec,
-                    tile_sched=a.tile_sched, fused_ffn=a.fused_ffn)
+                    tile_sched=a.tile_sched, fused_ffn=a.fused_ffn, h_ring_tiles=a.h_ring)
         base.update(kw)
         return self.mok._config(**base)
 
@@ -788,6 +791,8 @@ def main():
     mean_ms = sharding.max_over_ranks(main_rec["mean_ms_per_step"], dist, dev)
     main_rec["ms_per_step"], main_rec["mean_ms_per_step"] = ms_per_step, mean_ms
 
+    ws_bytes = (mok.mok_workspace_bytes_ring(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k, args.h_ring) if args.h_ring else
+                mok.mok_workspace_bytes(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k))
     # device's routing of this batch (for the comparison inside the cpu-baseline leg); outside every timed region
     gpu_idx = gpu_w = counts = None
     if rank == 0:
@@ -952,6 +957,7 @@ def main():
     if "sustained" in main_rec:
         roofline["sustained_run"] = main_rec["sustained"]["dominant_kernel"]
     conf = mok._config(impl=args.gemm, gather_mode=args.gather_mode, cta_group=args.cta_group, fused_ffn=args.fused_ffn,
+                       h_ring_tiles=args.h_ring,
                        precision=mok.MOK_PRECISION_MXFP8 if mx else mok.MOK_PRECISION_BF16, tile_sched=args.tile_sched)
     line = {
         "metric": METRIC, "value": main_rec["tokens_per_s"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -960,6 +966,7 @@ def main():
         "dtype": "mxfp8 routed experts (fp32 accumulate), bf16 elsewhere" if mx else "bf16", "data": "synthetic",
         "config": {"workload": cfg.name, "T": cfg.T, "H": cfg.H, "E": cfg.E, "k": cfg.k, "I": cfg.I,
                    "I_shared": cfg.I_s, "routing": cfg.bias, "parallelism": f"token-sharded replicas x{world}",
+                   "h_ring_tiles": args.h_ring, "workspace_bytes": int(ws_bytes),
                    "l2": "inputs larger than L2 (weights + activations >> 126 MB), no explicit flush",
                    "timing": "ms_per_step = median of the per-step CUDA-event times of one bracketed loop of `steps` "
                              "steps (max over ranks); stage times come from a second loop with per-stage events"},

@@ -117,7 +117,18 @@ typedef struct mok_config {
     int32_t serial_launches; /* 0 = the kernels of a forward call are launched with programmatic stream serialization (a
                              kernel's CTAs are scheduled while its predecessor still runs; every kernel waits for its
                              predecessors' completion before it touches their data), 1 = plain launches.  Same bits. */
+    int32_t h_ring_tiles; /* 0 = the gated activation h has a row for every padded route.  > 0: h is a RING of that many
+                             256-row slots (at least MOK_H_RING_MIN_TILES) that the row tiles in flight reuse (Section 3.3:
+                             fixed-size buffers; Section 3.2: the intermediate is consumed depth-first and stays in the
+                             caches).  Only the one-launch expert FFN can do that (it is then used whatever fused_ffn says;
+                             MOK_ERR_UNSUPPORTED where it cannot run: MXFP8, impl != 0, cta_group 1 / 2, a separate gather
+                             kernel): a gate/up tile stores into its slot once every down tile of the slot's previous
+                             rows has loaded them (completion counters, bounded waits); the distance between a row
+                             group's gate/up and down tiles is cut to the ring size minus 16 tiles.  The workspace is
+                             then the smaller one of mok_workspace_bytes_ring (no h rows beyond the ring, no gathered
+                             copy of x).  Same bits. */
 } mok_config;
+#define MOK_H_RING_MIN_TILES 24
 
 /*
  * Arguments of mok_moe_forward_ex.  Zero-initialise, then fill.  Shapes follow the paper's notation:
@@ -174,6 +185,10 @@ int mok_moe_forward(const void* x, const float* W_router,
 
 /* Bytes of scratch mok_moe_forward_ex needs for these sizes (0 if the sizes are invalid). */
 size_t mok_workspace_bytes(int T, int H, int I, int I_shared, int E, int k);
+/* The same for calls with config.h_ring_tiles = h_ring_tiles > 0 (Section 3.3: buffers of fixed size): the gated
+ * activation takes min(h_ring_tiles * 256, padded routes) rows and the gathered copy of x does not exist.  0 if the sizes
+ * are invalid or h_ring_tiles < MOK_H_RING_MIN_TILES.  A workspace of mok_workspace_bytes is always large enough too. */
+size_t mok_workspace_bytes_ring(int T, int H, int I, int I_shared, int E, int k, int h_ring_tiles);
 
 /* Same layer with a router bias, caller-owned workspace, stage outputs and knobs (see mok_args). */
 int mok_moe_forward_ex(const mok_args* args);

@@ -40,6 +40,14 @@
 // Shared-memory ring, tensor-memory use and the epilogue arithmetic are those of gemm_tcgen05_m2.cu; during D tiles the
 // gather warps skip ahead and the producer makes their arrivals on the ring's barriers.
 //
+// Optionally `h` is a RING of `ring` 256-row slots (Section 3.3: fixed-size buffers reused by the minibatches in flight):
+// row tile mt lives in slot mt mod ring.  A gate/up tile of row tile mt >= ring may only store once every down entry of
+// row tile mt - ring has loaded its rows: the MMA issuer adds one arrival to consumed[mt'] when all TMA loads of a down
+// entry of mt' have landed, and the gate/up epilogue waits (bounded) for all entries' arrivals.  No deadlock: with
+// ring >= window + 2 * GROUP_TILES (the launcher shortens the window to make it so) every down entry of row tile
+// mt - ring sits at a smaller list position than every gate/up tile of row tile mt, so the argument above still holds.
+// With the static window of two grids' worth of tiles the slots are rewritten while still in L2.
+//
 // Optionally the COMBINE (Section 2.1: out[t] = shared[t] + sum_s w[t,s] * y[pos[t,s]]) runs in the same launch: a token's
 // k rows lie anywhere in y, so it can only start when every down tile has been stored.  Every epilogue warp adds one
 // arrival to a grid-wide counter once its last store has completed, waits (bounded) until all epilogue warps of the grid
@@ -189,7 +197,8 @@ __device__ __forceinline__ int ld_acquire(const int32_t* p) {
 __global__ void __launch_bounds__(MAX_E)
 fused_tiles_kernel(const int32_t* __restrict__ counts, const int32_t* __restrict__ pad_offsets,
                    const int32_t* __restrict__ mt_start2, int E, int n1, int n2_tiles, int q, int window, int max_tiles,
-                   int4* __restrict__ tiles, int32_t* __restrict__ ready, WsHeader* __restrict__ hdr) {
+                   int4* __restrict__ tiles, int32_t* __restrict__ ready, int32_t* __restrict__ consumed,
+                   WsHeader* __restrict__ hdr) {
     __shared__ int32_t s_mt[MAX_E + 1], s_gofs[MAX_E + 1], s_wtot[32];
     pdl_enter();
     const int n2 = (n2_tiles + q - 1) / q;           // down entries per M tile: each covers up to q N tiles
@@ -236,7 +245,10 @@ fused_tiles_kernel(const int32_t* __restrict__ counts, const int32_t* __restrict
         if (total > max_tiles) atomicCAS(&hdr->status, 0, (int)MOK_ERR_SCHEDULE);
     }
     if (total > max_tiles) return;
-    for (int i = blockIdx.x * blockDim.x + tid; i < NMT; i += gridDim.x * blockDim.x) ready[i] = 0;
+    for (int i = blockIdx.x * blockDim.x + tid; i < NMT; i += gridDim.x * blockDim.x) {
+        ready[i] = 0;
+        consumed[i] = 0;
+    }
 
     // largest e in [0, E) with s_mt[e] <= v and a non-empty tail (the expert that holds M tile index v), for 0 <= v < NMT
     auto expert_of_tile = [&](int v) {
@@ -318,6 +330,9 @@ struct FusedArgs {
     int32_t* gang;                 // static mode: per list position, arrivals of the entries that share weight tiles
                                    // (zeroed before the launch), or NULL: unsynchronised starts
     int32_t* ready;                // per 256-row M tile: epilogue-warp arrivals of its gate/up tiles
+    int32_t* consumed;             // per 256-row M tile: down entries whose loads of h have landed (ring mode)
+    int32_t ring;                  // > 0: h holds `ring` 256-row slots, row tile mt in slot mt % ring
+    int32_t need_d;                // down entries per row tile
     int32_t max_tiles;
     int32_t H, I, E;
     int32_t n1, n2;                // N tiles of a gate/up row tile (ceil(I / 128)) and of a down row tile (ceil(H / 256))
@@ -590,8 +605,9 @@ fused_ffn_kernel(const __grid_constant__ CUtensorMap mapWgu, const __grid_consta
                             // (the gather threads have nothing to bring: their arrivals on the stage are made here)
                             asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0], %1;" ::"r"(full), "r"((uint32_t)GATHER_THREADS) : "memory");
                             mbar_expect_tx(full, B_BYTES + (two ? 2 : 1) * A_BYTES);
-                            tma_load_2d(sa, &mapHld, full, kb * BK, t.row0);
-                            if (two) tma_load_2d(sa + A_BYTES, &mapHld, full, kb * BK, t.row0 + BM);
+                            const int hrow = a.ring ? (t.mt % a.ring) * TM : t.row0;
+                            tma_load_2d(sa, &mapHld, full, kb * BK, hrow);
+                            if (two) tma_load_2d(sa + A_BYTES, &mapHld, full, kb * BK, hrow + BM);
                             tma_load_2d(sb, &mapWd, full, kb * BK, brow0);
                             tma_load_2d(sb + B_BYTES / 2, &mapWd, full, kb * BK, brow1);
                         } else if (narrow) {
@@ -675,6 +691,9 @@ fused_ffn_kernel(const __grid_constant__ CUtensorMap mapWgu, const __grid_consta
                     if (two) { tc_commit<1>(smem_u32(&ctrl->tfull[1])); ap1 ^= 1u; }
                     }
                     if (!ok) break;
+                    // ring mode: every load of h of this down entry has landed (its stages' full barriers were passed)
+                    if (a.ring && t.kind)
+                        asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(a.consumed + t.mt) : "memory");
                     if (dbg) {
                         const long long dt = clock64() - tile0, units = (long long)(two ? 2 : 1) * kblocks * t.cnt;
                         if (t.kind) { d_full1 += w_full; d_te1 += w_te; d_kb1 += units; d_rows1 += (long long)t.valid * kblocks * t.cnt; d_tot1 += dt; }
@@ -845,6 +864,39 @@ fused_ffn_kernel(const __grid_constant__ CUtensorMap mapWgu, const __grid_consta
             } else {
                 // gate/up tile: silu(g) * u from columns c and c + 128 (c + 64 of a narrow last tile), 64 output columns
                 // per pass; the next pass is read and computed before waiting for the slab of the current one
+                int hrow = row;
+                if (a.ring) {
+                    hrow = (t.mt % a.ring) * TM + acc * BM + quad * 32;
+                    if (t.mt >= a.ring) {
+                        // the slot's previous rows (row tile mt - ring) must have been loaded by all their down entries
+                        int free_ = 1;
+                        if (lane == 0) {
+                            const int32_t* c = a.consumed + (t.mt - a.ring);
+                            if (ld_acquire(c) < a.need_d) {
+                                const unsigned long long t0 = globaltimer();
+                                uint32_t spins = 0;
+                                while (ld_acquire(c) < a.need_d) {
+                                    __nanosleep(64);
+                                    if ((++spins & 63u) == 0u) {
+                                        if (*abort_flag) { free_ = 0; break; }
+                                        const unsigned long long limit =
+                                            a.header->wait_limit_us ? 1000ull * a.header->wait_limit_us : WAIT_LIMIT_NS;
+                                        if (globaltimer() - t0 > limit) {
+                                            *abort_flag = 1u;
+                                            atomicCAS(&a.header->status, 0, (int)MOK_ERR_TIMEOUT);
+                                            a.header->where = 45;
+                                            free_ = 0;
+                                            break;
+                                        }
+                                    }
+                                }
+                            }
+                            asm volatile("fence.proxy.async;" ::: "memory");
+                        }
+                        ok = __shfl_sync(0xffffffffu, free_, 0) != 0;
+                        if (!ok) break;
+                    }
+                }
                 const bool narrow = narrow_last && n == a.n1 - 1;
                 const int passes = narrow ? 1 : 2;
                 const uint32_t up_off = narrow ? BN / 4 : BN / 2;
@@ -870,7 +922,7 @@ fused_ffn_kernel(const __grid_constant__ CUtensorMap mapWgu, const __grid_consta
 #pragma unroll
                     for (int i = 0; i < 32; ++i) cur[i] = nxt[i];
                     if (pass + 1 < passes) load_pass(pass + 1, nxt);
-                    store_pass(cur, &mapHst, n * (BN / 2) + pass * 64, a.I, row);
+                    store_pass(cur, &mapHst, n * (BN / 2) + pass * 64, a.I, hrow);
                 }
                 if (lane == 0) {
                     // h of this warp's 32 rows is on its way: wait until the stores have completed (not only left shared
@@ -943,7 +995,7 @@ static cudaError_t launch_kernel(int grid, cudaStream_t s, const CUtensorMap& m0
 cudaError_t launch_fused_ffn(const __nv_bfloat16* x, int T, int H, int I, int E, const __nv_bfloat16* Wgu,
                              const __nv_bfloat16* Wd, const WsLayout& L, char* ws, int grid, int window_tiles, bool dynamic,
                              bool gang_sync, bool dbg, bool starve, cudaStream_t s, __nv_bfloat16* combine_out, int k,
-                             bool shared) {
+                             bool shared, int h_ring_tiles) {
     using namespace ff;
     int dev = 0, sm_count = 0;
     cudaError_t e = current_device(&dev);
@@ -957,7 +1009,12 @@ cudaError_t launch_fused_ffn(const __nv_bfloat16* x, int T, int H, int I, int E,
     if (q < 1) q = 1;
     if (q > n2) q = n2;
     if (window_tiles == 0) window_tiles = dynamic ? 8 * grid : 2 * grid;
-    const int window = window_tiles < 0 ? 0 : (window_tiles + n1 - 1) / n1;      // in M tiles
+    int window = window_tiles < 0 ? 0 : (window_tiles + n1 - 1) / n1;      // in M tiles
+    // ring of h: only as many slots as there are row tiles are ever used; the window must leave 2 * GROUP_TILES slots
+    const int max_mt2 = L.max_mt / 2;
+    const int ring = h_ring_tiles > 0 && h_ring_tiles < max_mt2 ? h_ring_tiles : 0;
+    if (ring > 0 && ring < H_RING_MIN_TILES) return cudaErrorInvalidValue;
+    if (ring > 0 && window > ring - 2 * GROUP_TILES) window = ring - 2 * GROUP_TILES;
     int4* tiles = reinterpret_cast<int4*>(ws + L.ftiles);
     int32_t* ready = reinterpret_cast<int32_t*>(ws + L.ready);
     // enough blocks for one warp per group of a large batch; every block rebuilds the per-expert offsets itself
@@ -965,7 +1022,7 @@ cudaError_t launch_fused_ffn(const __nv_bfloat16* x, int T, int H, int I, int E,
     if (tblocks > sm_count) tblocks = sm_count;
     e = launch_pdl(fused_tiles_kernel, dim3(tblocks), dim3(MAX_E), 0, s, reinterpret_cast<const int32_t*>(ws + L.counts),
                    reinterpret_cast<const int32_t*>(ws + L.pad_offsets), reinterpret_cast<const int32_t*>(ws + L.mt_start2), E,
-                   n1, n2, q, window, L.max_ftiles, tiles, ready, hdr);
+                   n1, n2, q, window, L.max_ftiles, tiles, ready, ready + max_mt2, hdr);
     if (e != cudaSuccess) return e;
 
     CUtensorMap mWgu, mWgu64, mHst, mHld, mWd, mY;
@@ -973,8 +1030,8 @@ cudaError_t launch_fused_ffn(const __nv_bfloat16* x, int T, int H, int I, int E,
     void* y = ws + L.y;
     if (!tmap::bf16_sw128(&mWgu, Wgu, (uint64_t)E * 2 * I, (uint64_t)H, BN / 2) ||
         !tmap::bf16_sw128(&mWgu64, Wgu, (uint64_t)E * 2 * I, (uint64_t)H, BN / 4) ||
-        !tmap::bf16_sw128(&mHst, h, (uint64_t)L.Rpad, (uint64_t)I, 32) ||
-        !tmap::bf16_sw128(&mHld, h, (uint64_t)L.Rpad, (uint64_t)I, BM) ||
+        !tmap::bf16_sw128(&mHst, h, (uint64_t)(ring ? ring * TM : L.Rpad), (uint64_t)I, 32) ||
+        !tmap::bf16_sw128(&mHld, h, (uint64_t)(ring ? ring * TM : L.Rpad), (uint64_t)I, BM) ||
         !tmap::bf16_sw128(&mWd, Wd, (uint64_t)E * H, (uint64_t)I, BN / 2) ||
         !tmap::bf16_sw128(&mY, y, (uint64_t)L.Rpad, (uint64_t)H, 32))
         return cudaErrorInvalidValue;
@@ -991,6 +1048,9 @@ cudaError_t launch_fused_ffn(const __nv_bfloat16* x, int T, int H, int I, int E,
         a.gang = reinterpret_cast<int32_t*>(ws + L.gang);
     }
     a.ready = ready;
+    a.consumed = ready + max_mt2;
+    a.ring = ring;
+    a.need_d = (n2 + q - 1) / q;
     a.max_tiles = L.max_ftiles;
     a.H = H; a.I = I; a.E = E;
     a.n1 = n1; a.n2 = n2;

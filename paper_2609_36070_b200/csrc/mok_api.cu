@@ -57,10 +57,12 @@ static bool sizes_ok(int T, int H, int I, int Is, int E, int k) {
     return true;
 }
 
-bool ws_layout(int T, int H, int I, int Is, int E, int k, WsLayout* L, bool mx) {
+bool ws_layout(int T, int H, int I, int Is, int E, int k, WsLayout* L, bool mx, int h_ring_tiles) {
     if (!sizes_ok(T, H, I, Is, E, k)) return false;
     if (mx && ((H % 32) || (I % 32))) return false;
+    if (h_ring_tiles < 0 || (h_ring_tiles > 0 && (h_ring_tiles < H_RING_MIN_TILES || mx))) return false;
     memset(L, 0, sizeof(*L));
+    L->h_ring = h_ring_tiles;
     const long long R = (long long)T * k;
     const long long nonempty_max = R < E ? R : E;
     long long Rpad = (R + nonempty_max * (2 * TILE_M - 1) + 2 * TILE_M - 1) / (2 * TILE_M) * (2 * TILE_M);
@@ -93,15 +95,17 @@ bool ws_layout(int T, int H, int I, int Is, int E, int k, WsLayout* L, bool mx) 
     if (ldl < 3 * (size_t)((E + 31) / 32 * 32)) ldl = 3 * (size_t)((E + 31) / 32 * 32);
     L->wr_split = take(2 * ldl * H);
     L->logits = take(sizeof(float) * (size_t)L->Tpad * ldl);
-    L->xg = take(2 * (size_t)Rpad * H);
-    L->h = take(2 * (size_t)Rpad * I);
+    // (a ring of the gated activation belongs to the one-launch expert FFN, which gathers its rows itself: no copy of x)
+    L->xg = take(h_ring_tiles > 0 ? 0 : 2 * (size_t)Rpad * H);
+    const long long h_rows = h_ring_tiles > 0 && (long long)h_ring_tiles * 2 * TILE_M < Rpad ? (long long)h_ring_tiles * 2 * TILE_M : Rpad;
+    L->h = take(2 * (size_t)h_rows * I);
     L->y = take(2 * (size_t)Rpad * H);
     {   // fused expert-FFN kernel: every 256-row tile times (gate/up N tiles + down N tiles), one counter per row tile
         const long long mt2 = Rpad / (2 * TILE_M), per = (I + 127) / 128 + (H + 255) / 256;
         const long long nt = mt2 * per;
         L->max_ftiles = nt < (1ll << 30) ? (int32_t)nt : 0;
         L->ftiles = take(sizeof(int4) * (size_t)L->max_ftiles);
-        L->ready = take(sizeof(int32_t) * (size_t)mt2);
+        L->ready = take(2 * sizeof(int32_t) * (size_t)mt2);
     }
     {   // gang-start counters of the 256-row kernel: one per tile of the largest of the four GEMMs
         const long long mt2 = Rpad / (2 * TILE_M), mts = L->Tpad / (2 * TILE_M);
@@ -136,7 +140,10 @@ static int validate(const mok_args* a, WsLayout* L, size_t extra_ws) {
     if (a->config && (a->config->tile_sched < 0 || a->config->tile_sched > 2)) return MOK_ERR_SHAPE;
     const bool mx = use_mx(a->config);
     if (mx && a->config->impl != MOK_IMPL_TCGEN05) return MOK_ERR_SHAPE;
-    if (!ws_layout(a->T, a->H, a->I, a->I_shared, a->E, a->k, L, mx)) return MOK_ERR_SHAPE;
+    const int ring = a->config ? a->config->h_ring_tiles : 0;
+    if (ring < 0 || (ring > 0 && ring < H_RING_MIN_TILES)) return MOK_ERR_SHAPE;
+    if (ring > 0 && mx) return MOK_ERR_UNSUPPORTED;
+    if (!ws_layout(a->T, a->H, a->I, a->I_shared, a->E, a->k, L, mx, ring)) return MOK_ERR_SHAPE;
     if ((a->I_shared > 0) != (a->W_shared_gate_up != nullptr) || (a->I_shared > 0) != (a->W_shared_down != nullptr))
         return MOK_ERR_SHAPE;
     if (a->T == 0) return MOK_OK;
@@ -162,7 +169,7 @@ static int validate(const mok_args* a, WsLayout* L, size_t extra_ws) {
                       a->config->host_chunks < 0 || a->config->host_chunks > MOK_MAX_HOST_CHUNKS ||
                       a->config->fused_ffn < 0 || a->config->fused_ffn > 3 || a->config->fused_window < -1 ||
                       a->config->gang_sync < 0 || a->config->gang_sync > 2 || a->config->serial_launches < 0 ||
-                      a->config->serial_launches > 1))
+                      a->config->serial_launches > 1 || a->config->h_ring_tiles < 0))
         return MOK_ERR_SHAPE;
     return MOK_OK;
 }
@@ -242,7 +249,7 @@ static bool use_fused_ffn(const mok_config* cfg, int H, int I, int tile_m, long 
     if (use_simt(cfg) || use_tn(cfg) || use_mx(cfg) || tile_m != TILE_M || max_ftiles <= 0) return false;
     if (cfg && (cfg->fused_ffn == 1 || cfg->cta_group == 1 || cfg->cta_group == 2)) return false;
     if (!fused_gather(cfg, I)) return false;
-    if (cfg && cfg->fused_ffn >= 2) return true;
+    if (cfg && (cfg->fused_ffn >= 2 || cfg->h_ring_tiles > 0)) return true;
     if (cfg && cfg->tile_sched == 1) return false;          // (tile stealing belongs to the two-launch path)
     // (at least two row tiles per expert on average: with single tiles there is nothing to start together, and the
     //  weight-streaming regime of small batches is served better by the two launches: 4.64 vs 4.80 ms at 128 rows)
@@ -332,6 +339,7 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
     MOK_MARK(MOK_STAGE_SCHEDULE + 1);
     const bool mx = use_mx(a->config);
     const bool simt = !mx && !fused_gather(a->config, a->I);
+    if (L.h_ring > 0 && (simt || mx)) return MOK_ERR_UNSUPPORTED;   // (that layout has no room for a copy of x)
     if (simt) {   // materialise the expert-sorted copy of x
         e = launch_gather(x, a->H, a->k, tile_m, L, ws, s);
         if (e != cudaSuccess) return cuda_fail(e);
@@ -455,17 +463,20 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
         g.total_rows = L.R;
         g.tile_sched = a->config ? a->config->tile_sched : 0;
         const bool fused = !simt && use_fused_ffn(a->config, a->H, a->I, tile_m, L.R, a->E, L.max_ftiles);
+        if (L.h_ring > 0 && !fused) return MOK_ERR_UNSUPPORTED;     // the ring exists in the one-launch kernel only
         combine_in_launch = fused && a->config && a->config->fused_ffn == 3;
         if (combine_in_launch && (rc = shared_expert())) return rc;       // its output is an input of that launch
         // its hand-out: synchronised starts need the static stride (a CTA that draws ahead could hold two tiles of a gang)
         const bool fused_sync = fused_gang(a->config, a->H, a->I, L.R, a->E);
         const int sched = a->config ? a->config->tile_sched : 0;
-        const bool fused_dynamic = sched == 1 || (sched == 0 && !fused_sync);
+        // (with a ring of h the window is short; the static stride keeps a row group's tiles closest together: measured
+        //  1.29 against 1.56 ms on the Qwen3-like layer with 72 slots)
+        const bool fused_dynamic = sched == 1 || (sched == 0 && !fused_sync && L.h_ring == 0);
         if (fused) {
             e = launch_fused_ffn(x, a->T, a->H, a->I, a->E, reinterpret_cast<const __nv_bfloat16*>(a->W_gate_up),
                                  reinterpret_cast<const __nv_bfloat16*>(a->W_down), L, ws, a->config ? a->config->grid : 0,
                                  a->config ? a->config->fused_window : 0, fused_dynamic, fused_sync, dbg, g.starve != 0, s,
-                                 combine_in_launch ? out : nullptr, a->k, a->I_shared > 0);
+                                 combine_in_launch ? out : nullptr, a->k, a->I_shared > 0, L.h_ring);
             if (e != cudaSuccess) return cuda_fail(e);
         } else if ((rc = run_gemm(g, true, a->config, L, ws, s))) return rc;
         g.row_token = nullptr;
@@ -537,6 +548,12 @@ size_t mok_workspace_bytes(int T, int H, int I, int I_shared, int E, int k) {
     return ws_layout(T, H, I, I_shared, E, k, &L) ? L.total : 0;
 }
 
+size_t mok_workspace_bytes_ring(int T, int H, int I, int I_shared, int E, int k, int h_ring_tiles) {
+    WsLayout L;
+    if (h_ring_tiles < H_RING_MIN_TILES) return 0;
+    return ws_layout(T, H, I, I_shared, E, k, &L, false, h_ring_tiles) ? L.total : 0;
+}
+
 size_t mok_router_prepared_bytes(int E, int H) {
     if (E <= 0 || E > MAX_E || H <= 0 || (H % 8)) return 0;
     return align_up(2 * (size_t)3 * ((E + 31) / 32 * 32) * H, 256);      // either layout fits: 3 * E rows rounded up
@@ -579,7 +596,8 @@ int mok_moe_forward_ex(const mok_args* a) {
         __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(a->out);
         for (int t0 = 0; t0 < a->T; t0 += mb) {
             ac.T = a->T - t0 < mb ? a->T - t0 : mb;
-            if (!ws_layout(ac.T, a->H, a->I, a->I_shared, a->E, a->k, &L, use_mx(a->config))) return MOK_ERR_SHAPE;
+            if (!ws_layout(ac.T, a->H, a->I, a->I_shared, a->E, a->k, &L, use_mx(a->config), a->config->h_ring_tiles))
+                return MOK_ERR_SHAPE;
             ac.topk_idx = a->topk_idx ? a->topk_idx + (size_t)t0 * a->k : nullptr;
             ac.topk_w = a->topk_w ? a->topk_w + (size_t)t0 * a->k : nullptr;
             rc = forward_device(&ac, L, x + (size_t)t0 * a->H, out + (size_t)t0 * a->H, t0 == 0);
@@ -690,7 +708,8 @@ int mok_moe_forward_host(const mok_args* a, const void* x_host, void* out_host) 
         mok_args ac = *a;
         ac.T = tc;
         WsLayout Lc;
-        if (!ws_layout(tc, a->H, a->I, a->I_shared, a->E, a->k, &Lc, use_mx(a->config))) return MOK_ERR_SHAPE;
+        if (!ws_layout(tc, a->H, a->I, a->I_shared, a->E, a->k, &Lc, use_mx(a->config), a->config ? a->config->h_ring_tiles : 0))
+            return MOK_ERR_SHAPE;
         if ((e = cudaStreamWaitEvent(s, p->in_done[c], 0)) != cudaSuccess) return cuda_fail(e);
         // only the first chunk clears the header: a device-side failure of any chunk stays in the status word
         rc = forward_device(&ac, Lc, xd + (size_t)t0 * a->H, od + (size_t)t0 * a->H, c == 0);

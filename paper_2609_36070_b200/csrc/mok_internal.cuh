@@ -50,6 +50,8 @@ struct WsLayout {
     size_t xg, h, y, hs, ysh;
     size_t x8, sx, h8, sh;   // MXFP8 mode: quantised token rows + row-major scales, quantised gated activation + scale atoms
     size_t ftiles, ready;    // fused expert-FFN kernel: tile list (int4 per tile) and per-M-tile completion counters
+                             // (two int32 per 256-row tile: gate/up arrivals, then down-tile arrivals at + max_mt / 2)
+    int32_t h_ring;          // > 0: `h` holds only this many 256-row tiles (a ring), and there is no `xg` region
     size_t gang;             // 256-row kernel: gang-start counters, one int32 per list position of the largest GEMM
     size_t gang_bytes;
     int32_t max_ftiles;
@@ -61,7 +63,7 @@ struct WsLayout {
     int32_t n_blk;        // schedule blocks
 };
 
-bool ws_layout(int T, int H, int I, int Is, int E, int k, WsLayout* L, bool mx = false);
+bool ws_layout(int T, int H, int I, int Is, int E, int k, WsLayout* L, bool mx = false, int h_ring_tiles = 0);
 
 // Arguments of the grouped GEMM (both implementations).  Rows live in a padded space: expert e owns rows
 // [128*mt_start[e], 128*mt_start[e+1]); tile q belongs to expert tile_expert[q].  In dense mode (shared
@@ -150,7 +152,9 @@ cudaError_t launch_gemm_mx(const GemmArgs& a, int epi, int grid, cudaStream_t s)
 cudaError_t launch_fused_ffn(const __nv_bfloat16* x, int T, int H, int I, int E, const __nv_bfloat16* Wgu,
                              const __nv_bfloat16* Wd, const WsLayout& L, char* ws, int grid, int window_tiles, bool dynamic,
                              bool gang_sync, bool dbg, bool starve, cudaStream_t s, __nv_bfloat16* combine_out = nullptr,
-                             int k = 0, bool shared = false);   // combine_out != NULL: the combine runs in the same launch
+                             int k = 0, bool shared = false,    // combine_out != NULL: the combine runs in the same launch
+                             int h_ring_tiles = 0);             // > 0: h is a ring of that many 256-row tiles
+constexpr int H_RING_MIN_TILES = 24;     // smallest ring of the gated activation (see gemm_fused.cu)
 cudaError_t launch_mx_quantize_rows(const __nv_bfloat16* in, long long rows, int K, uint8_t* codes, uint8_t* scales,
                                     cudaStream_t s);
 cudaError_t launch_mx_quantize_atoms(const __nv_bfloat16* in, int groups, int rows_per_group, int K, uint8_t* codes,

@@ -19,7 +19,7 @@ MOK_ERR_NULL, MOK_ERR_SHAPE, MOK_ERR_ALIGN, MOK_ERR_WORKSPACE = -1, -2, -3, -4
 MOK_ERR_CUDA, MOK_ERR_TIMEOUT, MOK_ERR_SCHEDULE, MOK_ERR_UNSUPPORTED = -5, -6, -7, -8
 MOK_IMPL_TCGEN05, MOK_IMPL_SIMT, MOK_IMPL_TCGEN05_TN = 0, 1, 2
 
-EXPORTS = ["mok_moe_forward", "mok_workspace_bytes", "mok_moe_forward_ex", "mok_moe_forward_host",
+EXPORTS = ["mok_moe_forward", "mok_workspace_bytes", "mok_workspace_bytes_ring", "mok_moe_forward_ex", "mok_moe_forward_host",
            "mok_moe_forward_host_async", "mok_host_wait", "mok_route",
            "mok_schedule", "mok_read_status", "mok_launch_count", "mok_last_cuda_error", "mok_status_string",
            "mok_version", "mok_profile_begin", "mok_profile_end", "mok_schedule_noalloc", "mok_debug_counters",
@@ -28,6 +28,7 @@ EXPORTS = ["mok_moe_forward", "mok_workspace_bytes", "mok_moe_forward_ex", "mok_
            "mok_ep_mx_workspace_bytes", "mok_bwd_workspace_bytes", "mok_moe_backward", "mok_selftest_per_device",
            "mok_router_prepared_bytes", "mok_router_prepare"]
 MOK_PRECISION_BF16, MOK_PRECISION_MXFP8 = 0, 1
+MOK_H_RING_MIN_TILES = 24
 MOK_MAX_RANKS = 16
 MOK_NOALLOC_MAX_ROUTES = 32768
 MOK_DEBUG_STARVE = 2
@@ -40,7 +41,7 @@ class mok_config(ctypes.Structure):
                 ("debug", ctypes.c_int32), ("host_chunks", ctypes.c_int32), ("precision", ctypes.c_int32),
                 ("tile_sched", ctypes.c_int32), ("macrobatch_tokens", ctypes.c_int32),
                 ("fused_ffn", ctypes.c_int32), ("fused_window", ctypes.c_int32), ("gang_sync", ctypes.c_int32),
-                ("serial_launches", ctypes.c_int32)]
+                ("serial_launches", ctypes.c_int32), ("h_ring_tiles", ctypes.c_int32)]
 
 
 class mok_args(ctypes.Structure):
@@ -112,6 +113,8 @@ _lib.mok_ep_combine.restype = ctypes.c_int
 _lib.mok_ep_combine.argtypes = [ctypes.POINTER(mok_ep_combine_args)]
 _lib.mok_workspace_bytes.restype = ctypes.c_size_t
 _lib.mok_workspace_bytes.argtypes = [ctypes.c_int] * 6
+_lib.mok_workspace_bytes_ring.restype = ctypes.c_size_t
+_lib.mok_workspace_bytes_ring.argtypes = [ctypes.c_int] * 7
 _lib.mok_mx_workspace_bytes.restype = ctypes.c_size_t
 _lib.mok_mx_workspace_bytes.argtypes = [ctypes.c_int] * 6
 _lib.mok_mx_scale_bytes.restype = ctypes.c_size_t
@@ -186,9 +189,11 @@ def _stream(stream):
 
 
 def _config(impl=0, grid=0, router_impl=0, profile=0, gather_mode=0, cta_group=0, debug=0, host_chunks=0,
-            precision=0, tile_sched=0, macrobatch_tokens=0, fused_ffn=0, fused_window=0, gang_sync=0, serial_launches=0):
+            precision=0, tile_sched=0, macrobatch_tokens=0, fused_ffn=0, fused_window=0, gang_sync=0, serial_launches=0,
+            h_ring_tiles=0):
     c = mok_config()
     c.serial_launches = serial_launches
+    c.h_ring_tiles = h_ring_tiles
     c.gang_sync = gang_sync
     c.fused_ffn, c.fused_window = fused_ffn, fused_window
     c.precision = precision
@@ -230,6 +235,10 @@ def mok_workspace_bytes(T, H, I, I_shared, E, k):
     return int(_lib.mok_workspace_bytes(T, H, I, I_shared, E, k))
 
 
+def mok_workspace_bytes_ring(T, H, I, I_shared, E, k, h_ring_tiles):
+    return int(_lib.mok_workspace_bytes_ring(T, H, I, I_shared, E, k, h_ring_tiles))
+
+
 def mok_launch_count(T, H, I, I_shared, E, k, config=None):
     return int(_lib.mok_launch_count(T, H, I, I_shared, E, k, None if config is None else ctypes.pointer(config)))
 
@@ -269,10 +278,14 @@ def mok_mx_quantize_rows(x, stream=None):
     return codes, scales
 
 
-def alloc_workspace(T, H, I, I_shared, E, k, device="cuda", host_staging=False, mx=False):
+def alloc_workspace(T, H, I, I_shared, E, k, device="cuda", host_staging=False, mx=False, h_ring_tiles=0):
     """A torch uint8 buffer large enough for mok_moe_forward_ex (plus the x/out staging copies of the host variant;
-    mx=True: plus the MXFP8 mode's quantised activations)."""
-    n = (mok_mx_workspace_bytes if mx else mok_workspace_bytes)(T, H, I, I_shared, E, k)
+    mx=True: plus the MXFP8 mode's quantised activations; h_ring_tiles > 0: the smaller workspace of calls whose config
+    has that h_ring_tiles)."""
+    if h_ring_tiles:
+        n = mok_workspace_bytes_ring(T, H, I, I_shared, E, k, h_ring_tiles)
+    else:
+        n = (mok_mx_workspace_bytes if mx else mok_workspace_bytes)(T, H, I, I_shared, E, k)
     if n == 0:
         raise MokError(MOK_ERR_SHAPE)
     if host_staging:    # True / 1: the blocking host call; 2: the two slots of the asynchronous one

@@ -99,11 +99,11 @@ def check_output(cfg, d, out_gpu, idx, w, tokens):
     return {"max_rel": float(max_rel), "mean_rel": float(mean_rel), "tokens_checked": int(len(tokens))}
 
 
-def full_parity(cfg, d=None, g=None, n_sample=None, config=None):
+def full_parity(cfg, d=None, g=None, n_sample=None, config=None, ws=None):
     """End-to-end parity of one workload.  n_sample=None checks every token."""
     d = d if d is not None else inputs.make_inputs(cfg)
     g = g if g is not None else upload(d)
-    out, st = run_gpu(cfg, g, config=config)
+    out, st = run_gpu(cfg, g, ws=ws, config=config)
     idx, w, rep = check_routing_and_schedule(cfg, d, st)
     tokens = np.arange(cfg.T, dtype=np.int32) if n_sample is None else inputs.sample_tokens(cfg, idx, n_sample)
     rep.update(check_output(cfg, d, out, idx, w, tokens))

@@ -378,6 +378,50 @@ def test_one_launch_ffn_gives_the_bits_of_two_launches(cfg):
     assert all(call["combine"] < 0.05 and call["gemm1"] > 0.0 for call in ms), ms
 
 
+RING = MID + [
+    # about 270 row tiles of 256 rows: a ring of 24 slots is rewritten eleven times
+    MoEConfig("ring_long", T=16384, H=512, E=16, k=4, I=256, I_s=0, bias="zipf", seed=93),
+]
+
+
+@pytest.mark.parametrize("cfg", RING, ids=[c.name for c in RING])
+def test_gated_activation_in_a_ring_gives_the_same_bits(cfg):
+    """config.h_ring_tiles: the gated activation lives in a ring of 256-row slots that the row tiles in flight reuse
+    (Section 3.3), in a workspace without the rows beyond the ring.  A gate/up tile stores into its slot only after
+    the slot's previous rows were loaded by all their down tiles.  Every token against the oracle, and bit for bit
+    the two-launch path, for the smallest ring and larger ones, both hand-outs, several grids and windows, and with
+    the combine in the same launch."""
+    m = mok()
+    d = inputs.make_inputs(cfg)
+    g = pu.upload(d)
+    ref = pu.run_gpu(cfg, g, config=m._config(fused_ffn=1, cta_group=3), stages=False)
+    full = m.mok_workspace_bytes(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k)
+    ring = m.MOK_H_RING_MIN_TILES
+    assert 0 < m.mok_workspace_bytes_ring(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k, ring) < full
+    assert m.mok_workspace_bytes_ring(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k, ring - 1) == 0
+    ws = m.alloc_workspace(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k, h_ring_tiles=ring)
+    out, st, rep = pu.full_parity(cfg, d=d, g=g, config=m._config(h_ring_tiles=ring), ws=ws)
+    print(cfg.name, rep)
+    assert torch.equal(out.view(torch.int16), ref.view(torch.int16))
+    for kw in ({"grid": 1}, {"grid": 7}, {"fused_window": -1}, {"fused_window": 1 << 20}, {"tile_sched": 1},
+               {"tile_sched": 2, "grid": 5}, {"gang_sync": 2}, {"gang_sync": 2, "grid": 11}, {"fused_ffn": 3},
+               {"fused_ffn": 3, "tile_sched": 2, "gang_sync": 2}):
+        out1 = pu.run_gpu(cfg, g, ws=ws, config=m._config(h_ring_tiles=ring, **kw), stages=False)
+        assert torch.equal(out1.view(torch.int16), ref.view(torch.int16)), kw
+    for r in (32, 100, 1 << 20):      # (a ring with more slots than row tiles is the plain layout)
+        wr = m.alloc_workspace(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k, h_ring_tiles=r)
+        out1 = pu.run_gpu(cfg, g, ws=wr, config=m._config(h_ring_tiles=r), stages=False)
+        assert torch.equal(out1.view(torch.int16), ref.view(torch.int16)), r
+    # what cannot run with a ring says so: the two-launch kernels on request, a ring below the minimum
+    args = (g["x"], g["W_r"], g["bias"], g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], cfg.k, ws)
+    with pytest.raises(m.MokError) as e:
+        m.mok_moe_forward_ex(*args, config=m._config(h_ring_tiles=ring, cta_group=1))
+    assert e.value.status == m.MOK_ERR_UNSUPPORTED
+    with pytest.raises(m.MokError) as e:
+        m.mok_moe_forward_ex(*args, config=m._config(h_ring_tiles=ring - 1))
+    assert e.value.status == m.MOK_ERR_SHAPE
+
+
 @pytest.mark.parametrize("cfg", MID + [SMALL[0], SMALL[6]], ids=[c.name for c in MID + [SMALL[0], SMALL[6]]])
 def test_synchronised_tile_starts_give_the_same_bits(cfg):
     """The 256-row kernel can make the row tiles that share a weight tile start together (config.gang_sync; chosen
@@ -396,8 +440,9 @@ def test_synchronised_tile_starts_give_the_same_bits(cfg):
         assert torch.equal(out.view(torch.int16), ref.view(torch.int16)), grid
 
 
-@pytest.mark.parametrize("fused,sched,gang", [(1, 0, 0), (2, 0, 0), (2, 2, 0), (2, 0, 2), (1, 0, 2), (3, 0, 0), (3, 2, 0)])
-def test_bounded_waits_report_a_timeout_and_leave_the_context_usable(fused, sched, gang):
+@pytest.mark.parametrize("fused,sched,gang,ring", [(1, 0, 0, 0), (2, 0, 0, 0), (2, 2, 0, 0), (2, 0, 2, 0), (1, 0, 2, 0),
+                                                  (3, 0, 0, 0), (3, 2, 0, 0), (2, 0, 0, 24), (2, 2, 0, 24)])
+def test_bounded_waits_report_a_timeout_and_leave_the_context_usable(fused, sched, gang, ring):
     """Failure detection without a fault: the test hook silences the gate/up GEMM's TMA producer, so its MMA issuer
     waits for operands that never come.  Every wait is bounded (2 ms here), the kernel records MOK_ERR_TIMEOUT, frees
     its tensor memory and returns; the next call on the same context must be correct again.  fused = 2: the same on
@@ -410,7 +455,7 @@ def test_bounded_waits_report_a_timeout_and_leave_the_context_usable(fused, sche
     good = pu.run_gpu(cfg, g, ws=ws, stages=False).clone()
     m.mok_moe_forward_ex(g["x"], g["W_r"], g["bias"], g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], cfg.k, ws,
                          config=m._config(debug=m.MOK_DEBUG_STARVE, fused_ffn=fused, tile_sched=sched, gang_sync=gang,
-                                          cta_group=3 if fused == 1 else 0))
+                                          cta_group=3 if fused == 1 else 0, h_ring_tiles=ring))
     assert m.mok_read_status(ws) == m.MOK_ERR_TIMEOUT
     again = pu.run_gpu(cfg, g, ws=ws, stages=False)
     assert torch.equal(good.view(torch.int16), again.view(torch.int16))
