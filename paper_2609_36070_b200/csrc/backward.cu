@@ -264,7 +264,7 @@ int mok_moe_backward(const mok_bwd_args* a) {
     auto bf = [&](size_t off) { return reinterpret_cast<__nv_bfloat16*>(ws + off); };
     mok_config cfg;
     memset(&cfg, 0, sizeof(cfg));
-    if (a->config) { cfg.grid = a->config->grid; cfg.cta_group = a->config->cta_group; }
+    if (a->config) { cfg.grid = a->config->grid; cfg.cta_group = a->config->cta_group; cfg.gang_sync = a->config->gang_sync; }
     cudaError_t e = cudaMemsetAsync(hdr, 0, sizeof(WsHeader), s);
     if (e != cudaSuccess) return cuda_fail(e);
     // the dispatch schedule again, from the saved routing (no host readback)
@@ -288,8 +288,11 @@ int mok_moe_backward(const mok_bwd_args* a) {
             q.mt_start = reinterpret_cast<const int32_t*>(ws + L.mt_start2);
             q.tile_expert = reinterpret_cast<const int32_t*>(ws + L.tile_expert2);
         }
+        // (the row tiles of an expert share a tile of W here as in the forward products: synchronised starts where they pay)
+        const int rcg = gang_prepare(q, false, &cfg, L, ws, s);
+        if (rcg) return rcg;
         cudaError_t ee = launch_gemm_m2(q, EPI_BF16, cfg.grid, s);
-        q.n_mtiles = &h2->n_mtiles; q.mt_start = mt; q.tile_expert = te; q.b_mn = 0;
+        q.n_mtiles = &h2->n_mtiles; q.mt_start = mt; q.tile_expert = te; q.b_mn = 0; q.gang = nullptr;
         return ee == cudaSuccess ? MOK_OK : cuda_fail(ee);
     };
 

@@ -721,7 +721,8 @@ static cudaError_t launch_one(const CUtensorMap& mA, const CUtensorMap& mB, cons
     } else if (grid <= 0 || grid > sm_count) {
         grid = sm_count;
     }
-    if (a.gang && !CLC && MODE == 0 && grid < GROUP_TILES) {
+    constexpr bool ROW_TILES = MODE == 0 || MODE == 2;     // tiles of expert rows against a weight tile (not K ranges)
+    if (a.gang && !CLC && ROW_TILES && grid < GROUP_TILES) {
         // a gang's (up to GROUP_TILES) tiles must sit on different CTAs, or a CTA would wait for its own later tile
         GemmArgs b = a;
         b.gang = nullptr;
@@ -729,7 +730,7 @@ static cudaError_t launch_one(const CUtensorMap& mA, const CUtensorMap& mB, cons
             mA, mB, mC, mB64, b, n_nt, k_blocks);
         return cudaGetLastError();
     }
-    if (a.gang && !CLC && MODE == 0) {
+    if (a.gang && !CLC && ROW_TILES) {
         // gang starts wait for tiles of other CTAs: every CTA of the grid has to be resident (cooperative launch)
         cudaLaunchConfig_t cfg = {};
         cudaLaunchAttribute attr[1];

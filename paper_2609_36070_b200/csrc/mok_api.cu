@@ -257,27 +257,34 @@ static bool use_fused_ffn(const mok_config* cfg, int H, int I, int tile_m, long 
            rows >= 512ll * experts && fused_gang(cfg, H, I, rows, experts);
 }
 
+// Synchronised starts of the row tiles that share a weight tile (see gemm_tcgen05_m2.cu) for one launch of the 256-row
+// kernel: where they pay (or are forced), the gang counters are cleared and handed to the kernel.  Not with stolen
+// tiles, not for the K-range products of the backward pass, and off with gang_sync = 1.
+int gang_prepare(GemmArgs& g, bool swiglu, const mok_config* cfg, const WsLayout& L, char* ws, cudaStream_t s) {
+    const long long w_bytes = 2ll * (swiglu ? 2 : 1) * g.N * g.K;
+    const long long rows_all = g.dense_rows > 0 ? g.dense_rows : g.total_rows;
+    const bool pays = gang_pays(w_bytes, rows_all, g.dense_rows > 0 ? 1 : g.E);
+    const int mode = cfg ? cfg->gang_sync : 0;
+    g.gang = nullptr;
+    if (L.gang_bytes > 0 && g.kgroup_rows == 0 && g.tile_sched != 1 && (mode == 2 || (mode == 0 && pays))) {
+        const long long rows = g.dense_rows > 0 ? g.dense_rows : g.rows_pad;
+        const long long n_nt = swiglu ? (g.N + 127) / 128 : (g.N + 255) / 256;
+        const size_t bytes = sizeof(int32_t) * (size_t)((rows + 255) / 256 * n_nt);
+        if (bytes <= L.gang_bytes) {        // (a GEMM with more tiles than the region was sized for runs without)
+            cudaError_t eg = cudaMemsetAsync(ws + L.gang, 0, bytes, s);
+            if (eg != cudaSuccess) return cuda_fail(eg);
+            g.gang = reinterpret_cast<int32_t*>(ws + L.gang);
+        }
+    }
+    return MOK_OK;
+}
+
 int run_gemm(GemmArgs g, bool swiglu, const mok_config* cfg, const WsLayout& L, char* ws, cudaStream_t s) {
     const int epi = swiglu ? EPI_SWIGLU : EPI_BF16, grid = cfg ? cfg->grid : 0;
     if (use_m2(cfg, g.K, g.tile_m, g.dense_rows > 0 ? g.dense_rows : g.total_rows, g.dense_rows > 0 ? 1 : g.E)) {
         WsHeader* hdr = reinterpret_cast<WsHeader*>(ws + L.header);
-        // synchronised starts of the row tiles that share a weight tile (see the kernel); not with stolen tiles, and
-        // off with gang_sync = 1
-        const long long w_bytes = 2ll * (swiglu ? 2 : 1) * g.N * g.K;
-        const long long rows_all = g.dense_rows > 0 ? g.dense_rows : g.total_rows;
-        const bool pays = gang_pays(w_bytes, rows_all, g.dense_rows > 0 ? 1 : g.E);
-        const int mode = cfg ? cfg->gang_sync : 0;
-        if (L.gang_bytes > 0 && g.kgroup_rows == 0 && !g.b_mn && g.tile_sched != 1 &&
-            (mode == 2 || (mode == 0 && pays))) {
-            const long long rows = g.dense_rows > 0 ? g.dense_rows : g.rows_pad;
-            const long long n_nt = swiglu ? (g.N + 127) / 128 : (g.N + 255) / 256;
-            const size_t bytes = sizeof(int32_t) * (size_t)((rows + 255) / 256 * n_nt);
-            if (bytes <= L.gang_bytes) {        // (a GEMM with more tiles than the region was sized for runs without)
-                cudaError_t eg = cudaMemsetAsync(ws + L.gang, 0, bytes, s);
-                if (eg != cudaSuccess) return cuda_fail(eg);
-                g.gang = reinterpret_cast<int32_t*>(ws + L.gang);
-            }
-        }
+        const int rcg = gang_prepare(g, swiglu, cfg, L, ws, s);
+        if (rcg) return rcg;
         g.n_mtiles = &hdr->n_mtiles2;
         g.mt_start = reinterpret_cast<const int32_t*>(ws + L.mt_start2);
         g.tile_expert = reinterpret_cast<const int32_t*>(ws + L.tile_expert2);

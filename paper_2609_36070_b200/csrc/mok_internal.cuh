@@ -139,6 +139,7 @@ cudaError_t launch_ep_schedule(const int32_t* idx_all, int n_ranks, int rank, in
                                int experts_local, int tile_m, const WsLayout& L, char* ws, int32_t* pos_out, int32_t* M_out,
                                int32_t* S_out, int32_t* phi_rank_out, int32_t* phi_index_out, cudaStream_t s);
 int run_gemm(GemmArgs g, bool swiglu, const mok_config* cfg, const WsLayout& L, char* ws, cudaStream_t s);
+int gang_prepare(GemmArgs& g, bool swiglu, const mok_config* cfg, const WsLayout& L, char* ws, cudaStream_t s);
 int tile_rows(const mok_config* cfg, int I);
 bool fused_gather(const mok_config* cfg, int I);
 int cuda_fail(cudaError_t e);
