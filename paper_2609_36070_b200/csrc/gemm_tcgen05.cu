@@ -94,6 +94,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
     int n_mt_total = (a.dense_rows > 0) ? (a.dense_rows + TM - 1) / TM : *a.n_mtiles;
     if (n_mt_total > a.max_mt) n_mt_total = a.max_mt;
     const int total = n_mt_total * n_nt;
+    // columns of an N tile: 256, or fewer for the fp32 epilogue on single CTAs (GemmArgs::n_tile: more, narrower tiles
+    // when a GEMM has too few tiles to fill the GPU; every output element is still one accumulation over K)
+    const int n_width = (EPI == EPI_F32 && CTAS == 1 && a.n_tile > 0) ? a.n_tile : BN;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -140,7 +143,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
                 const Tile t = decode_tile(a, L, n_nt, n_mt_total, TM);
                 // weight rows of this tile: [gate 128 | up 128] for SwiGLU, 256 consecutive rows otherwise; a CTA
                 // of a pair stages only its half (rank 0: first 128 rows, rank 1: second 128 rows)
-                const int brow0 = t.e * b_rows_per_expert + (SWIGLU ? t.n * (BN / 2) : t.n * BN);
+                const int brow0 = t.e * b_rows_per_expert + (SWIGLU ? t.n * (BN / 2) : t.n * n_width);
                 const int brow1 = SWIGLU ? brow0 + a.N : brow0 + BN / 2;
                 bool ok = true;
                 for (int kb = 0; kb < k_blocks; ++kb) {
@@ -150,7 +153,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
                     if (!ok) break;
                     const uint32_t full = smem_u32(&ctrl->full[s]);
                     const uint32_t sa = base + s * STAGE_BYTES, sb = sa + A_BYTES;
-                    if (CTAS == 1) {
+                    if (CTAS == 1 && n_width <= BN / 2) {
+                        // narrow N tile (fp32 epilogue only): one box of n_width weight rows
+                        mbar_expect_tx(full, (GATHER ? 0 : A_BYTES) + n_width * BK * 2);
+                        if (!GATHER) tma_load_2d(sa, &tmapA, full, kb * BK, t.row0);
+                        tma_load_2d(sb, &tmapB, full, kb * BK, brow0);
+                    } else if (CTAS == 1) {
                         mbar_expect_tx(full, GATHER ? B_STAGE : STAGE_BYTES);
                         if (!GATHER) tma_load_2d(sa, &tmapA, full, kb * BK, t.row0);
                         tma_load_2d(sb, &tmapB, full, kb * BK, brow0);
@@ -174,7 +182,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
     } else if (warp == 1) {
         if (lane == 0 && rank == 0) {
             // -------------------------------------------------------------- MMA issuer (even CTA of a pair)
-            constexpr uint32_t idesc = make_idesc<CTAS>();
+            const uint32_t idesc = (make_idesc<CTAS>() & ~(0x3Fu << 17)) | ((uint32_t)(n_width >> 3) << 17);
             int s = 0, as = 0;
             uint32_t ph = 0, aph = 0;
             long long d_full = 0, d_pfull = 0, d_tempty = 0, d_kb = 0;
@@ -296,9 +304,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
             const int row = t.row0 + rank * BM + quad * 32;
             if (EPI == EPI_F32) {
                 float* frow = reinterpret_cast<float*>(a.C) + (size_t)(row + lane) * a.ldc;
-                const int c0 = t.n * BN;
+                const int c0 = t.n * n_width;
 #pragma unroll 1
-                for (int c = 0; c < BN; c += 32) {
+                for (int c = 0; c < n_width; c += 32) {
                     uint32_t r[32];
                     tc_ld32(taddr + c, r);
                     tc_wait_ld();
@@ -467,10 +475,15 @@ cudaError_t launch_gemm_tc(const GemmArgs& a, int epi, int grid, cudaStream_t s)
     CUtensorMap mA, mB, mC;
     const uint64_t b_rows = (uint64_t)a.E * (swiglu ? 2 : 1) * a.N;
     if (!make_map(&mA, a.A, (uint64_t)a.a_rows, (uint64_t)a.K, BM)) return cudaErrorInvalidValue;
-    if (!make_map(&mB, a.B, b_rows, (uint64_t)a.K, BN / 2)) return cudaErrorInvalidValue;
+    int n_width = BN;
+    if (a.n_tile > 0) {     // narrower N tiles: fp32 epilogue, single CTAs, 32 / 64 / 128 columns
+        if (epi != EPI_F32 || pair || gather || (a.n_tile != 32 && a.n_tile != 64 && a.n_tile != 128)) return cudaErrorInvalidValue;
+        n_width = a.n_tile;
+    }
+    if (!make_map(&mB, a.B, b_rows, (uint64_t)a.K, n_width < BN / 2 ? n_width : BN / 2)) return cudaErrorInvalidValue;
     if (epi == EPI_F32) mC = mB;      // the fp32 epilogue stores directly
     else if (!make_map(&mC, a.C, (uint64_t)a.rows_pad, (uint64_t)a.N, 32, (uint64_t)a.ldc)) return cudaErrorInvalidValue;
-    const int n_nt = swiglu ? (a.N + BN / 2 - 1) / (BN / 2) : (a.N + BN - 1) / BN;
+    const int n_nt = swiglu ? (a.N + BN / 2 - 1) / (BN / 2) : (a.N + n_width - 1) / n_width;
     const int k_blocks = (a.K + BK - 1) / BK;
     if (pair) {
         if (epi == EPI_SWIGLU && gather) return launch_one<EPI_SWIGLU, true, 2>(mA, mB, mC, a, n_nt, k_blocks, grid, s);

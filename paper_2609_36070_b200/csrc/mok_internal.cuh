@@ -88,6 +88,7 @@ struct GemmArgs {
     int32_t tile_m;              // rows of one tile of the padded row space: 128, or 256 for CTA pairs
     int32_t dbg_slot;            // >= 0: accumulate wait-time counters into header->dbg[dbg_slot]
     int32_t starve;              // test hook: the TMA producer issues nothing, so the kernel's waits run out
+    int32_t n_tile;              // 128-row kernel, fp32 epilogue: columns per N tile (32 / 64 / 128; 0 = 256)
     int32_t tile_sched;          // 256-row kernel, routed forward GEMMs: 1 = tiles handed out by cluster launch control
     int32_t* gang;               // 256-row kernel, forward layout: per list position, arrivals of the row tiles that share
                                  // one weight tile (zeroed before the launch), or NULL: no synchronised tile starts

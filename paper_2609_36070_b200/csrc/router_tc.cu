@@ -282,6 +282,14 @@ cudaError_t launch_router_tc(const __nv_bfloat16* x, const float* Wr, const floa
         g.tile_m = tile_m;
         g.dbg_slot = -1;
         g.header = hdr;
+        // Few tokens give few tiles (T = 64 with 256 experts: three tiles of 128 x 256, each streaming a third of the split
+        // weights through one SM): up to 16 row tiles the 128-row kernel runs with N tiles of 32 to 128 columns instead.  An
+        // output element is the same accumulation over K whatever the tile width, so the logits keep their bits.
+        const int row_tiles = (T + TILE_M - 1) / TILE_M;
+        if (variant != 2 && tile_m == TILE_M && row_tiles <= 16) {
+            g.n_tile = row_tiles <= 4 ? 32 : row_tiles <= 8 ? 64 : 128;
+            variant = 0;
+        }
         e = variant == 2 ? launch_gemm_tn(g, EPI_F32, grid, s)
             : variant == 3 ? launch_gemm_m2(g, EPI_F32, grid, s) : launch_gemm_tc(g, EPI_F32, grid, s);
     }

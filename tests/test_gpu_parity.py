@@ -8,6 +8,7 @@ from paper_2609_36070_b200 import inputs
 from paper_2609_36070_b200.inputs import MoEConfig
 
 import parity_util as pu
+from oracle import mok_ref
 
 pytestmark = pytest.mark.gpu
 
@@ -132,6 +133,30 @@ def test_router_weights_prepared_once_give_the_same_bits(name, router_impl):
     with pytest.raises(m.MokError) as ei:                        # the fp32-FMA router has no split
         m.mok_router_prepare(g["W_r"], cfg.k, m._config(router_impl=1))
     assert ei.value.status == m.MOK_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("E,router_impl", [(192, 0), (96, 2)])
+def test_router_bits_do_not_depend_on_the_batch_a_token_is_in(E, router_impl):
+    """The three-kernel tensor-core router cuts its projection into narrower tiles when there are few tokens (more CTAs
+    streaming the router weights).  A token's logits are one accumulation over H whatever the tile shape, so its
+    experts and weights must have the same bits alone, in a small batch and inside a large one; and they must be the
+    oracle's selection."""
+    m = mok()
+    cfg = MoEConfig("router_only", T=2560, H=1024, E=E, k=6, I=64, I_s=0, bias="normal", seed=95)
+    d = inputs.make_inputs(cfg, experts=False)
+    x = m.to_device_bf16(d["x"], "cuda")
+    W_r = torch.from_numpy(d["W_r"]).cuda()
+    bias = None if d["bias"] is None else torch.from_numpy(d["bias"]).cuda()
+    conf = m._config(router_impl=router_impl)
+    ws = m.alloc_workspace(cfg.T, cfg.H, 64, 0, cfg.E, cfg.k)
+    idx_all, w_all = m.mok_route(x, W_r, bias, cfg.k, ws, config=conf)          # 20 row tiles: full-width tiles
+    idx_ref, w_ref, gap, lg = mok_ref.route(d["x"], d["W_r"], d["bias"], cfg.k)
+    far = gap > 1e-3
+    assert np.array_equal(np.sort(idx_all.cpu().numpy()[far], axis=1), np.sort(idx_ref[far], axis=1))
+    for T in (1, 64, 130, 900, 1900, 2048):                                     # 1 .. 16 row tiles: narrower tiles
+        idx, w = m.mok_route(x[:T].contiguous(), W_r, bias, cfg.k, ws, config=conf)
+        assert torch.equal(idx, idx_all[:T]), T
+        assert torch.equal(w.view(torch.int32), w_all[:T].view(torch.int32)), T
 
 
 def test_one_kernel_router_lists_near_ties_for_the_exact_fix_up():
