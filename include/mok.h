@@ -406,6 +406,65 @@ size_t mok_bwd_workspace_bytes(int T, int H, int I, int I_shared, int E, int k);
 int mok_moe_backward(const mok_bwd_args* args);
 
 /*
+ * Backward pass under expert parallelism (Section 3.1: the backward pass moves the same rows the other way -- the rank
+ * that serves a route pulls the row of dL/dout from the token's owner, the owner pulls dL/d(gathered x) from the
+ * serving rank; Section 3.4: router-weight gradient inside the chain, activations recomputed).  Two calls per rank,
+ * mirroring mok_ep_expert_ffn / mok_ep_combine, with a barrier over the ranks between them:
+ *   mok_ep_expert_bwd : Algorithm 1 for this rank's experts from the all-gathered routes (the forward pass's tables and
+ *       positions), then the one-rank chain on the rows served here -- x and dout rows pulled from the owners' buffers
+ *       inside the GEMMs -- which leaves dL/d(gathered x) in dxg, dL/dw of the served routes in dw_routes (indexed by
+ *       source rank * T_local * k + route; other entries untouched), the shared expert's dx of this rank's own tokens
+ *       in dx_shared, and the weight gradients of the local experts (all four NULL: activation gradients only).
+ *   mok_ep_bwd_combine : the owner sums the k rows of dxg it pulls from the serving ranks (through their pos tables)
+ *       on top of dx_shared, in slot order in fp32, and fetches its routes' dw.
+ * dx and dw equal the one-rank backward pass on the concatenated batch bit for bit; the weight gradients sum an
+ * expert's rows in Algorithm 1's order, so they agree with it up to fp32 summation order.  bf16 mode only; H, I and
+ * I_shared multiples of 32.  The paper prints no formulas for the backward pass: this is the chain rule of Section 2.1.
+ */
+typedef struct mok_ep_bwd_args {
+    int32_t rank, n_ranks;
+    int32_t T_local, H, I, I_shared, E, k;
+    const void* x_peers[MOK_MAX_RANKS];      /* every rank's token rows, bf16 [T_local, H] (device addresses) */
+    const void* dout_peers[MOK_MAX_RANKS];   /* every rank's dL/dout, bf16 [T_local, H] */
+    const int32_t* idx_all;                  /* int32 [n_ranks, T_local * k]: all-gathered routes */
+    const float* w_all;                      /* fp32 [n_ranks, T_local * k]: all-gathered router weights */
+    const void* W_gate_up;                   /* bf16 [E / n_ranks, 2I, H]: this rank's experts */
+    const void* W_down;                      /* bf16 [E / n_ranks, H, I] */
+    const void* W_shared_gate_up;            /* bf16 [2 * I_shared, H] or NULL */
+    const void* W_shared_down;               /* bf16 [H, I_shared] or NULL */
+    void* dxg;                               /* out, read by the peers: bf16 [dxg_rows, H], dxg_rows >= mok_ep_y_rows(...) */
+    long long dxg_rows;
+    int32_t* pos;                            /* out, read by the peers: int32 [n_ranks * T_local * k] */
+    float* dw_routes;                        /* out, read by the peers: fp32 [n_ranks * T_local * k] */
+    void* dx_shared;                         /* out: bf16 [T_local rounded up to 256, H], or NULL without a shared expert */
+    void* dW_gate_up;                        /* out: bf16 [E / n_ranks, 2I, H] or NULL */
+    void* dW_down;                           /* out: bf16 [E / n_ranks, H, I] or NULL */
+    void* dW_shared_gate_up;                 /* out: bf16 [2 * I_shared, H] or NULL (this rank's tokens' share) */
+    void* dW_shared_down;                    /* out: bf16 [H, I_shared] or NULL */
+    void* workspace;                         /* mok_ep_bwd_workspace_bytes(...) bytes, 256-byte aligned */
+    size_t workspace_bytes;
+    const mok_config* config;                /* grid, cta_group 0/1/3, gang_sync */
+    void* stream;
+} mok_ep_bwd_args;
+
+typedef struct mok_ep_bwd_combine_args {
+    int32_t rank, n_ranks;
+    int32_t T_local, H, E, k;
+    const int32_t* topk_idx;                 /* int32 [T_local, k]: this rank's routes */
+    const void* dxg_peers[MOK_MAX_RANKS];    /* every rank's dxg */
+    const int32_t* pos_peers[MOK_MAX_RANKS]; /* every rank's pos */
+    const float* dw_peers[MOK_MAX_RANKS];    /* every rank's dw_routes (needed when dw != NULL) */
+    const void* dx_shared;                   /* this rank's dx_shared, or NULL */
+    void* dx;                                /* out: bf16 [T_local, H] */
+    float* dw;                               /* out: fp32 [T_local, k], or NULL */
+    void* stream;
+} mok_ep_bwd_combine_args;
+
+size_t mok_ep_bwd_workspace_bytes(int n_ranks, int T_local, int H, int I, int I_shared, int E, int k);
+int mok_ep_expert_bwd(const mok_ep_bwd_args* args);
+int mok_ep_bwd_combine(const mok_ep_bwd_combine_args* args);
+
+/*
  * Reads the device-side status word of a workspace after synchronising `stream` -- the only call besides
  * mok_moe_forward_host that blocks the host.  Returns MOK_OK, MOK_ERR_TIMEOUT or MOK_ERR_SCHEDULE
  * (or MOK_ERR_CUDA if the stream itself is in error).

@@ -222,6 +222,19 @@ static bool bwd_layout(int T, int H, int I, int Is, int E, int k, BwdLayout* B) 
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// What the expert-parallel backward adds to the one-rank chain (see backward_chain).
+struct EpBwd {
+    int n_ranks, T_local;
+    long long routes_expected;                         // expected share of this rank, for the kernel choice
+    const __nv_bfloat16* x_peers[MOK_MAX_RANKS];
+    const __nv_bfloat16* dout_peers[MOK_MAX_RANKS];
+    const float* w_all;                                // [n_ranks * T_local * k] router weights of every rank's routes
+    float* dw_routes;                                  // [n_ranks * T_local * k] dL/dw of the routes served here
+    __nv_bfloat16* dxg;                                // [rows, H] dL/d(gathered x) of the rows served here
+    __nv_bfloat16* dx_shared;                          // [Tpad, H] shared expert's dx of this rank's tokens
+};
+int backward_chain(const mok_bwd_args* a, const BwdLayout& B, const WsLayout& L, const EpBwd* ep);
+
 }  // namespace mok
 
 using namespace mok;
@@ -254,7 +267,20 @@ int mok_moe_backward(const mok_bwd_args* a) {
     const bool want_w = a->dW_gate_up || a->dW_down || a->dW_shared_gate_up || a->dW_shared_down;
     if (want_w && (!a->dW_gate_up || !a->dW_down || (a->I_shared > 0 && (!a->dW_shared_gate_up || !a->dW_shared_down))))
         return MOK_ERR_NULL;
-    const WsLayout& L = B.F;
+    return backward_chain(a, B, B.F, nullptr);
+}
+
+}  // extern "C"
+
+namespace mok {
+
+// The chain of the backward pass on one rank's dispatch space.  a: the one-rank arguments (T = tokens of the shared
+// expert and of dx, E = experts of the schedule tables, x / dout = this rank's token rows).  ep == NULL: one rank -- the
+// schedule is rebuilt from a->topk_idx and the chain ends with the combine into a->dx.  ep != NULL: expert parallelism --
+// the caller has built the schedule for the local experts (row_token holds global token ids, row_route global route
+// ids), rows are pulled from the owners' buffers, and the chain leaves dL/d(gathered x) and the shared expert's dx in
+// the caller's buffers for the owners' combine.
+int backward_chain(const mok_bwd_args* a, const BwdLayout& B, const WsLayout& L, const EpBwd* ep) {
     const int T = a->T, H = a->H, I = a->I, Is = a->I_shared, E = a->E, k = a->k;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(a->stream);
     char* ws = reinterpret_cast<char*>(a->workspace);
@@ -262,18 +288,33 @@ int mok_moe_backward(const mok_bwd_args* a) {
     const __nv_bfloat16* x = reinterpret_cast<const __nv_bfloat16*>(a->x);
     const __nv_bfloat16* dout = reinterpret_cast<const __nv_bfloat16*>(a->dout);
     auto bf = [&](size_t off) { return reinterpret_cast<__nv_bfloat16*>(ws + off); };
+    const bool want_w = a->dW_gate_up || a->dW_down || a->dW_shared_gate_up || a->dW_shared_down;
     mok_config cfg;
     memset(&cfg, 0, sizeof(cfg));
     if (a->config) { cfg.grid = a->config->grid; cfg.cta_group = a->config->cta_group; cfg.gang_sync = a->config->gang_sync; }
-    cudaError_t e = cudaMemsetAsync(hdr, 0, sizeof(WsHeader), s);
-    if (e != cudaSuccess) return cuda_fail(e);
-    // the dispatch schedule again, from the saved routing (no host readback)
-    e = launch_schedule(a->topk_idx, T, E, k, TILE_M, TILE_M, L, ws, nullptr, nullptr, nullptr, nullptr, s,
-                        reinterpret_cast<int32_t*>(ws + B.row_route));
-    if (e != cudaSuccess) return cuda_fail(e);
+    cudaError_t e = cudaSuccess;
+    if (!ep) {
+        e = cudaMemsetAsync(hdr, 0, sizeof(WsHeader), s);
+        if (e != cudaSuccess) return cuda_fail(e);
+        // the dispatch schedule again, from the saved routing (no host readback)
+        e = launch_schedule(a->topk_idx, T, E, k, TILE_M, TILE_M, L, ws, nullptr, nullptr, nullptr, nullptr, s,
+                            reinterpret_cast<int32_t*>(ws + B.row_route));
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    const float* w_routes = ep ? ep->w_all : a->topk_w;
+    float* dw_routes = ep ? ep->dw_routes : a->dw;
+    __nv_bfloat16* dxg = ep ? ep->dxg : bf(L.y);
+    __nv_bfloat16* dx_shared = ep ? ep->dx_shared : bf(L.ysh);
+    // rows pulled from the owners' buffers (expert parallelism): which buffers a gathering GEMM reads
+    auto pull_from = [&](GemmArgs& q, const __nv_bfloat16* const* peers) {
+        q.peer_tokens = 0;
+        if (!ep) return;
+        q.peer_tokens = ep->T_local;
+        for (int r = 0; r < ep->n_ranks; ++r) q.peer_x[r] = peers[r];
+    };
     // The transposed products of dgrad read the weights MN-major, as they sit in memory (W[e] = [K, N], N contiguous).
     // config.gather_mode = 2 selects the older path instead: K-contiguous transposed copies made at every call.
-    const bool wT = a->config && a->config->gather_mode == 2;
+    const bool wT = !ep && a->config && a->config->gather_mode == 2;
     if (wT) {
         if ((e = launch_transpose(reinterpret_cast<const __nv_bfloat16*>(a->W_down), bf(B.WdT), E, H, I, H, s)) != cudaSuccess) return cuda_fail(e);
         if ((e = launch_transpose(reinterpret_cast<const __nv_bfloat16*>(a->W_gate_up), bf(B.WguT), E, 2 * I, H, 2 * I, s)) != cudaSuccess) return cuda_fail(e);
@@ -307,7 +348,7 @@ int mok_moe_backward(const mok_bwd_args* a) {
     g.pad_offsets = reinterpret_cast<const int32_t*>(ws + L.pad_offsets);
     g.counts = reinterpret_cast<const int32_t*>(ws + L.counts);
     g.dbg_slot = -1;
-    g.E = E; g.rows_pad = L.Rpad; g.dense_rows = 0; g.total_rows = L.R;
+    g.E = E; g.rows_pad = L.Rpad; g.dense_rows = 0; g.total_rows = ep ? ep->routes_expected : L.R;
     int rc;
     // Four products need the rows of x or dout in dispatch order.  Up to I = 2048 each of them pulls the rows through the
     // schedule's row_token table inside the GEMM, as the forward pass does (K-major for the recomputation and the dgrad
@@ -315,7 +356,7 @@ int mok_moe_backward(const mok_bwd_args* a) {
     // re-gathers its rows once per tile along the other output dimension (2I/256 or I/256 times), so for wide experts
     // the copies are made once instead (I = 14336: 13.3 vs 13.9 ms, I = 2880: 10.9 vs 11.2 ms), padding rows zero.
     const int32_t* row_token = reinterpret_cast<const int32_t*>(ws + L.row_token);
-    const bool pull = !wT && I <= 2048;
+    const bool pull = !wT && (I <= 2048 || ep);       // (expert parallelism always pulls: there is no local copy to make)
     __nv_bfloat16* XG = bf(L.xg);
     __nv_bfloat16* DG = bf(B.doutT);
     if (!wT && !pull) {
@@ -323,26 +364,28 @@ int mok_moe_backward(const mok_bwd_args* a) {
         if ((e = launch_gather(dout, H, k, TILE_M, L, ws, s, DG)) != cudaSuccess) return cuda_fail(e);
     }
     // gu = Xg Wgu^T  (activation recomputation)
-    if (wT || pull) { g.A = x; g.a_rows = T; g.row_token = row_token; }
+    if (wT || pull) { g.A = x; g.a_rows = T; g.row_token = row_token; if (ep) pull_from(g, ep->x_peers); }
     else { g.A = XG; g.a_rows = L.Rpad; g.row_token = nullptr; }
     g.B = reinterpret_cast<const __nv_bfloat16*>(a->W_gate_up);
     g.C = ws + B.gu; g.K = H; g.N = 2 * I; g.ldc = 2 * I;
     if ((rc = run_gemm(g, false, &cfg, L, ws, s))) return rc;
     // dhu = gather(dout) Wd
     g.A = (wT || pull) ? dout : DG; g.C = ws + B.dhu; g.K = H; g.N = I; g.ldc = I;
+    if (ep) pull_from(g, ep->dout_peers);
     if ((rc = dgrad_gemm(g, a->W_down, B.WdT))) return rc;
+    g.peer_tokens = 0;
     // SwiGLU backward + router-weight gradient
     {
         int blocks = (L.Rpad + 7) / 8;
         if (blocks > 148 * 16) blocks = 148 * 16;
         swiglu_bwd_kernel<<<blocks, 256, 0, s>>>(bf(B.gu), bf(B.dhu), I, 0, hdr, g.tile_expert, g.pad_offsets, g.counts,
-                                                 reinterpret_cast<const int32_t*>(ws + B.row_route), a->topk_w, bf(B.dgu),
-                                                 bf(L.h), a->dw);
+                                                 reinterpret_cast<const int32_t*>(ws + B.row_route), w_routes, bf(B.dgu),
+                                                 bf(L.h), dw_routes);
         if ((e = cudaGetLastError()) != cudaSuccess) return cuda_fail(e);
     }
     // dXg = [dg | du] Wgu
     g.row_token = nullptr;
-    g.A = bf(B.dgu); g.a_rows = L.Rpad; g.C = ws + L.y; g.K = 2 * I; g.N = H; g.ldc = H;
+    g.A = bf(B.dgu); g.a_rows = L.Rpad; g.C = dxg; g.K = 2 * I; g.N = H; g.ldc = H;
     if ((rc = dgrad_gemm(g, a->W_gate_up, B.WguT))) return rc;
     if (Is > 0) {   // shared expert: the same chain on every token, w = 1
         if (wT) {
@@ -359,12 +402,14 @@ int mok_moe_backward(const mok_bwd_args* a) {
         swiglu_bwd_kernel<<<blocks, 256, 0, s>>>(bf(B.gus), bf(B.dhus), Is, T, hdr, nullptr, nullptr, nullptr, nullptr,
                                                  nullptr, bf(B.dgus), bf(L.hs), nullptr);
         if ((e = cudaGetLastError()) != cudaSuccess) return cuda_fail(e);
-        g.A = bf(B.dgus); g.a_rows = L.Tpad; g.C = ws + L.ysh; g.K = 2 * Is; g.N = H; g.ldc = H;
+        g.A = bf(B.dgus); g.a_rows = L.Tpad; g.C = dx_shared; g.K = 2 * Is; g.N = H; g.ldc = H;
         if ((rc = dgrad_gemm(g, a->W_shared_gate_up, B.WsguT))) return rc;
     }
-    // dx[t] = dx_shared[t] + sum_s dXg[pos[t,s]]: the forward combine with unit weights, same fixed order
-    e = launch_combine(L, ws, T, H, k, Is > 0, reinterpret_cast<__nv_bfloat16*>(a->dx), s, /*unit_weights=*/true);
-    if (e != cudaSuccess) return cuda_fail(e);
+    if (!ep) {
+        // dx[t] = dx_shared[t] + sum_s dXg[pos[t,s]]: the forward combine with unit weights, same fixed order
+        e = launch_combine(L, ws, T, H, k, Is > 0, reinterpret_cast<__nv_bfloat16*>(a->dx), s, /*unit_weights=*/true);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
     if (!want_w) return MOK_OK;
 
     // ------------------------------------------------------------------ weight gradients
@@ -387,11 +432,13 @@ int mok_moe_backward(const mok_bwd_args* a) {
         if (pull) { q.row_token = row_token; q.a_rows = T; }   // dout / x stay in token order: their rows are pulled by the GEMM
         q.kgroup_rows = H; q.A = pull ? dout : DG; q.lda = H; q.gather_mn = pull ? 1 : 0; q.B = bf(L.h); q.N = I; q.ldb = I;
         q.C = a->dW_down; q.rows_pad = E * H; q.ldc = I;
+        if (ep) pull_from(q, ep->dout_peers);
         if ((e = launch_gemm_m2(q, EPI_BF16, cfg.grid, s)) != cudaSuccess) return cuda_fail(e);
         q.kgroup_rows = 2 * I; q.A = bf(B.dgu); q.lda = 2 * I; q.B = pull ? x : XG; q.N = H; q.ldb = H; q.gather_mn = pull ? 2 : 0;
         q.C = a->dW_gate_up; q.rows_pad = E * 2 * I; q.ldc = H;
+        if (ep) pull_from(q, ep->x_peers);
         if ((e = launch_gemm_m2(q, EPI_BF16, cfg.grid, s)) != cudaSuccess) return cuda_fail(e);
-        q.row_token = nullptr; q.gather_mn = 0;
+        q.row_token = nullptr; q.gather_mn = 0; q.peer_tokens = 0;
         if (Is > 0) {   // shared expert: one K range over the T tokens (rows past T are zero-filled by the tensor maps)
             q.E = 1; q.dense_rows = T; q.K = T;
             q.kgroup_rows = H; q.A = dout; q.lda = H; q.B = bf(L.hs); q.N = Is; q.ldb = Is;
@@ -430,6 +477,176 @@ int mok_moe_backward(const mok_bwd_args* a) {
         q.kgroup_rows = 2 * Is; q.A = bf(B.dguT); q.a_rows = 2 * Is; q.B = bf(B.xgT); q.N = H; q.C = a->dW_shared_gate_up;
         q.rows_pad = 2 * Is; q.ldc = H;
         if ((e = launch_gemm_m2(q, EPI_BF16, cfg.grid, s)) != cudaSuccess) return cuda_fail(e);
+    }
+    return MOK_OK;
+}
+
+}  // namespace mok
+
+namespace mok {
+
+// padded row -> global route id (source rank * routes per rank + route) from the schedule's `pos` table
+__global__ void __launch_bounds__(256)
+ep_row_route_kernel(const int32_t* __restrict__ idx_all, const int32_t* __restrict__ pos, int total_routes, int lo, int Lx,
+                    int32_t* __restrict__ row_route) {
+    for (int g = blockIdx.x * 256 + threadIdx.x; g < total_routes; g += gridDim.x * 256) {
+        const int e = idx_all[g];
+        if (e >= lo && e < lo + Lx) row_route[pos[g]] = g;
+    }
+}
+
+// dw[t, s] of this rank's routes, from the rank that served each route
+struct EpDwArgs {
+    const float* dw[MOK_MAX_RANKS];
+    const int32_t* idx;
+    float* out;
+    int32_t n, Lx, route_base;
+};
+__global__ void __launch_bounds__(256)
+ep_dw_kernel(const __grid_constant__ EpDwArgs a) {
+    for (int j = blockIdx.x * 256 + threadIdx.x; j < a.n; j += gridDim.x * 256)
+        a.out[j] = a.dw[a.idx[j] / a.Lx][(size_t)a.route_base + j];
+}
+
+static bool ep_bwd_layout(int n_ranks, int T_local, int H, int I, int Is, int E, int k, BwdLayout* B) {
+    if ((H % 32) || (I % 32) || (Is % 32)) return false;
+    if (!ep_layout(n_ranks, T_local, H, I, Is, E, k, &B->F)) return false;
+    const WsLayout& F = B->F;
+    size_t off = F.total;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    const size_t Rp = (size_t)F.Rpad, Tp = (size_t)F.Tpad;
+    B->row_route = take(sizeof(int32_t) * Rp);
+    B->gu = take(2 * Rp * 2 * I);
+    B->dhu = take(2 * Rp * I);
+    B->dgu = take(2 * Rp * 2 * I);
+    B->gus = take(2 * Tp * 2 * Is);
+    B->dhus = take(2 * Tp * Is);
+    B->dgus = take(2 * Tp * 2 * Is);
+    B->WdT = B->WguT = B->WsdT = B->WsguT = B->doutT = B->hwT = B->dguT = B->xgT = 0;    // (paths the pull mode never takes)
+    B->total = off;
+    return true;
+}
+
+}  // namespace mok
+
+extern "C" {
+
+size_t mok_ep_bwd_workspace_bytes(int n_ranks, int T_local, int H, int I, int I_shared, int E, int k) {
+    BwdLayout B;
+    return ep_bwd_layout(n_ranks, T_local, H, I, I_shared, E, k, &B) ? B.total : 0;
+}
+
+int mok_ep_expert_bwd(const mok_ep_bwd_args* a) {
+    if (!a) return MOK_ERR_NULL;
+    BwdLayout B;
+    if (a->n_ranks < 1 || a->n_ranks > MOK_MAX_RANKS || a->rank < 0 || a->rank >= a->n_ranks) return MOK_ERR_SHAPE;
+    if (!ep_bwd_layout(a->n_ranks, a->T_local, a->H, a->I, a->I_shared, a->E, a->k, &B)) return MOK_ERR_SHAPE;
+    if ((a->I_shared > 0) != (a->W_shared_gate_up != nullptr) || (a->I_shared > 0) != (a->W_shared_down != nullptr))
+        return MOK_ERR_SHAPE;
+    if (a->config && (a->config->impl != MOK_IMPL_TCGEN05 || a->config->grid < 0 || a->config->precision != MOK_PRECISION_BF16 ||
+                      (a->config->cta_group != 0 && a->config->cta_group != 1 && a->config->cta_group != 3)))
+        return MOK_ERR_SHAPE;
+    if (a->T_local == 0) return MOK_OK;
+    if (!a->idx_all || !a->w_all || !a->W_gate_up || !a->W_down || !a->dxg || !a->pos || !a->dw_routes) return MOK_ERR_NULL;
+    if (a->I_shared > 0 && !a->dx_shared) return MOK_ERR_NULL;
+    for (int r = 0; r < a->n_ranks; ++r) {
+        if (!a->x_peers[r] || !a->dout_peers[r]) return MOK_ERR_NULL;
+        if (!aligned16(a->x_peers[r]) || !aligned16(a->dout_peers[r])) return MOK_ERR_ALIGN;
+    }
+    if (!aligned16(a->W_gate_up) || !aligned16(a->W_down) || !aligned16(a->W_shared_gate_up) || !aligned16(a->W_shared_down) ||
+        !aligned16(a->dxg) || !aligned16(a->dx_shared) || !aligned16(a->dW_gate_up) || !aligned16(a->dW_down) ||
+        !aligned16(a->dW_shared_gate_up) || !aligned16(a->dW_shared_down))
+        return MOK_ERR_ALIGN;
+    const bool want_w = a->dW_gate_up || a->dW_down || a->dW_shared_gate_up || a->dW_shared_down;
+    if (want_w && (!a->dW_gate_up || !a->dW_down || (a->I_shared > 0 && (!a->dW_shared_gate_up || !a->dW_shared_down))))
+        return MOK_ERR_NULL;
+    const WsLayout& L = B.F;
+    if (a->dxg_rows < L.Rpad) return MOK_ERR_WORKSPACE;
+    if (!a->workspace || (reinterpret_cast<uintptr_t>(a->workspace) & 255u) || a->workspace_bytes < B.total)
+        return MOK_ERR_WORKSPACE;
+
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(a->stream);
+    char* ws = reinterpret_cast<char*>(a->workspace);
+    WsHeader* hdr = reinterpret_cast<WsHeader*>(ws + L.header);
+    cudaError_t e = cudaMemsetAsync(hdr, 0, sizeof(WsHeader), s);
+    if (e != cudaSuccess) return cuda_fail(e);
+    const int Lx = a->E / a->n_ranks, n = a->T_local * a->k;
+    // Algorithm 1 for this rank's experts, as in the forward pass (same tables, same positions)
+    e = launch_ep_schedule(a->idx_all, a->n_ranks, a->rank, n, a->k, a->T_local, Lx, TILE_M, L, ws, a->pos, nullptr, nullptr,
+                           nullptr, nullptr, s);
+    if (e != cudaSuccess) return cuda_fail(e);
+    {
+        const int total = a->n_ranks * n;
+        int blocks = (total + 255) / 256;
+        if (blocks > 148 * 8) blocks = 148 * 8;
+        ep_row_route_kernel<<<blocks, 256, 0, s>>>(a->idx_all, a->pos, total, a->rank * Lx, Lx,
+                                                   reinterpret_cast<int32_t*>(ws + B.row_route));
+        if ((e = cudaGetLastError()) != cudaSuccess) return cuda_fail(e);
+    }
+    EpBwd ep;
+    memset(&ep, 0, sizeof(ep));
+    ep.n_ranks = a->n_ranks;
+    ep.T_local = a->T_local;
+    ep.routes_expected = n;
+    for (int r = 0; r < a->n_ranks; ++r) {
+        ep.x_peers[r] = reinterpret_cast<const __nv_bfloat16*>(a->x_peers[r]);
+        ep.dout_peers[r] = reinterpret_cast<const __nv_bfloat16*>(a->dout_peers[r]);
+    }
+    ep.w_all = a->w_all;
+    ep.dw_routes = a->dw_routes;
+    ep.dxg = reinterpret_cast<__nv_bfloat16*>(a->dxg);
+    ep.dx_shared = reinterpret_cast<__nv_bfloat16*>(a->dx_shared);
+    mok_bwd_args b;
+    memset(&b, 0, sizeof(b));
+    b.x = a->x_peers[a->rank];
+    b.dout = a->dout_peers[a->rank];
+    b.W_gate_up = a->W_gate_up; b.W_down = a->W_down;
+    b.W_shared_gate_up = a->W_shared_gate_up; b.W_shared_down = a->W_shared_down;
+    b.T = a->T_local; b.H = a->H; b.I = a->I; b.I_shared = a->I_shared; b.E = Lx; b.k = a->k;
+    b.dW_gate_up = a->dW_gate_up; b.dW_down = a->dW_down;
+    b.dW_shared_gate_up = a->dW_shared_gate_up; b.dW_shared_down = a->dW_shared_down;
+    b.workspace = a->workspace; b.workspace_bytes = a->workspace_bytes;
+    b.config = a->config;
+    b.stream = a->stream;
+    return backward_chain(&b, B, L, &ep);
+}
+
+int mok_ep_bwd_combine(const mok_ep_bwd_combine_args* a) {
+    if (!a) return MOK_ERR_NULL;
+    if (a->n_ranks < 1 || a->n_ranks > MOK_MAX_RANKS || a->rank < 0 || a->rank >= a->n_ranks || a->T_local < 0 ||
+        a->H <= 0 || (a->H % 8) || a->E < 1 || a->E % a->n_ranks || a->k < 1 || a->k > MAX_K || a->k > a->E)
+        return MOK_ERR_SHAPE;
+    if (a->T_local == 0) return MOK_OK;
+    if (!a->topk_idx || !a->dx) return MOK_ERR_NULL;
+    // dx: the forward's owner-side combine with unit weights over the serving ranks' dL/d(gathered x) rows
+    mok_ep_combine_args c;
+    memset(&c, 0, sizeof(c));
+    c.rank = a->rank; c.n_ranks = a->n_ranks; c.T_local = a->T_local; c.H = a->H; c.E = a->E; c.k = a->k;
+    c.topk_idx = a->topk_idx;
+    c.topk_w = nullptr;                       // unit weights
+    for (int r = 0; r < a->n_ranks; ++r) { c.y_peers[r] = a->dxg_peers[r]; c.pos_peers[r] = a->pos_peers[r]; }
+    c.y_shared = a->dx_shared;
+    c.out = a->dx;
+    c.stream = a->stream;
+    int rc = ep_combine_impl(&c, true);
+    if (rc) return rc;
+    if (a->dw) {
+        EpDwArgs d;
+        memset(&d, 0, sizeof(d));
+        for (int r = 0; r < a->n_ranks; ++r) {
+            if (!a->dw_peers[r]) return MOK_ERR_NULL;
+            d.dw[r] = a->dw_peers[r];
+        }
+        d.idx = a->topk_idx;
+        d.out = a->dw;
+        d.n = a->T_local * a->k;
+        d.Lx = a->E / a->n_ranks;
+        d.route_base = a->rank * d.n;
+        int blocks = (d.n + 255) / 256;
+        if (blocks > 148 * 8) blocks = 148 * 8;
+        ep_dw_kernel<<<blocks, 256, 0, reinterpret_cast<cudaStream_t>(a->stream)>>>(d);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return cuda_fail(e);
     }
     return MOK_OK;
 }

@@ -183,7 +183,7 @@ ep_combine_kernel(const __grid_constant__ EpCombineArgs a) {
         const int c = a.idx[j] / a.Lx;
         const int32_t p = a.pos[c][(size_t)a.route_base + j];
         s_row[threadIdx.x] = a.y[c] + (size_t)p * a.H;
-        s_w[threadIdx.x] = a.w[j];
+        s_w[threadIdx.x] = a.w ? a.w[j] : 1.f;          // w == NULL: plain sum (backward pass)
     }
     __syncthreads();
     const int chunks = a.H >> 3;
@@ -224,7 +224,7 @@ ep_combine_kernel(const __grid_constant__ EpCombineArgs a) {
 
 // Workspace of one rank: the one-rank layout for n_ranks*T_local "tokens" and L experts without the router and
 // gathered-copy regions, with room for the per-(rank, block) histograms and M.
-static bool ep_layout(int n_ranks, int T_local, int H, int I, int Is, int E, int k, WsLayout* L, bool mx = false) {
+bool ep_layout(int n_ranks, int T_local, int H, int I, int Is, int E, int k, WsLayout* L, bool mx) {
     if (n_ranks < 1 || n_ranks > MOK_MAX_RANKS || T_local < 0 || E < 1 || E % n_ranks) return false;
     if (H <= 0 || I <= 0 || Is < 0 || (H % 8) || (I % 8) || (Is % 8) || k < 1 || k > MAX_K || k > E || E > MAX_E) return false;
     const int Lx = E / n_ranks;
@@ -441,13 +441,19 @@ int mok_ep_expert_ffn(const mok_ep_args* a) {
     return MOK_OK;
 }
 
-int mok_ep_combine(const mok_ep_combine_args* a) {
+int mok_ep_combine(const mok_ep_combine_args* a) { return ep_combine_impl(a, false); }
+
+}  // extern "C"
+
+namespace mok {
+
+int ep_combine_impl(const mok_ep_combine_args* a, bool unit_weights) {
     if (!a) return MOK_ERR_NULL;
     if (a->n_ranks < 1 || a->n_ranks > MOK_MAX_RANKS || a->rank < 0 || a->rank >= a->n_ranks || a->T_local < 0 ||
         a->H <= 0 || (a->H % 8) || a->E < 1 || a->E % a->n_ranks || a->k < 1 || a->k > MAX_K || a->k > a->E)
         return MOK_ERR_SHAPE;
     if (a->T_local == 0) return MOK_OK;
-    if (!a->topk_idx || !a->topk_w || !a->out) return MOK_ERR_NULL;
+    if (!a->topk_idx || (!unit_weights && !a->topk_w) || !a->out) return MOK_ERR_NULL;
     if (!aligned16(a->out) || !aligned16(a->y_shared)) return MOK_ERR_ALIGN;
     EpCombineArgs c;
     memset(&c, 0, sizeof(c));
@@ -459,7 +465,7 @@ int mok_ep_combine(const mok_ep_combine_args* a) {
     }
     c.ysh = reinterpret_cast<const __nv_bfloat16*>(a->y_shared);
     c.idx = a->topk_idx;
-    c.w = a->topk_w;
+    c.w = unit_weights ? nullptr : a->topk_w;
     c.out = reinterpret_cast<__nv_bfloat16*>(a->out);
     c.T = a->T_local; c.H = a->H; c.k = a->k; c.Lx = a->E / a->n_ranks;
     c.route_base = a->rank * a->T_local * a->k;
@@ -468,4 +474,4 @@ int mok_ep_combine(const mok_ep_combine_args* a) {
     return e == cudaSuccess ? MOK_OK : cuda_fail(e);
 }
 
-}  // extern "C"
+}  // namespace mok

@@ -482,7 +482,11 @@ gemm_m2_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
                         const int kr = gw * 16 + q * 4 + sub;
-                        const __nv_bfloat16* srow = mat + (size_t)(tok_cur[q] >= 0 ? tok_cur[q] : 0) * ld + colbase;
+                        // (expert-parallel mode: the row id names the owning rank, whose buffer holds the row)
+                        const int tk = tok_cur[q] >= 0 ? tok_cur[q] : 0;
+                        const int pr = a.peer_tokens > 0 ? tk / a.peer_tokens : 0;
+                        const __nv_bfloat16* srow = (a.peer_tokens > 0 ? a.peer_x[pr] + (size_t)(tk - pr * a.peer_tokens) * ld
+                                                                        : mat + (size_t)tk * ld) + colbase;
                         const uint32_t drow = stage + (uint32_t)kr * 128u + (uint32_t)((chunk ^ (kr & 7)) << 4);
 #pragma unroll
                         for (int g4 = 0; g4 < 4; ++g4) {

@@ -139,6 +139,10 @@ cudaError_t launch_combine(const WsLayout& L, char* ws, int T, int H, int k, boo
 cudaError_t launch_ep_schedule(const int32_t* idx_all, int n_ranks, int rank, int routes_per_rank, int k, int tokens_per_rank,
                                int experts_local, int tile_m, const WsLayout& L, char* ws, int32_t* pos_out, int32_t* M_out,
                                int32_t* S_out, int32_t* phi_rank_out, int32_t* phi_index_out, cudaStream_t s);
+// the expert-parallel owner-side combine; unit_weights: plain sum of the k rows (backward pass)
+int ep_combine_impl(const mok_ep_combine_args* a, bool unit_weights);
+// workspace layout of one expert-parallel rank (ep.cu)
+bool ep_layout(int n_ranks, int T_local, int H, int I, int Is, int E, int k, WsLayout* L, bool mx = false);
 int run_gemm(GemmArgs g, bool swiglu, const mok_config* cfg, const WsLayout& L, char* ws, cudaStream_t s);
 int gang_prepare(GemmArgs& g, bool swiglu, const mok_config* cfg, const WsLayout& L, char* ws, cudaStream_t s);
 int tile_rows(const mok_config* cfg, int I);

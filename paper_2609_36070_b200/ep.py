@@ -88,6 +88,59 @@ def forward_emulated(xs, W_router, router_bias, W_gate_up, W_down, W_shared_gate
     return (outs, tables, idx_all) if return_tables else outs
 
 
+def backward_emulated(xs, douts, idxs, ws_, W_gate_up, W_down, W_shared_gate_up, W_shared_down, config=None,
+                      weight_grads=True):
+    """The expert-parallel backward pass with all ranks on the current GPU, phase by phase (as forward_emulated).
+    xs, douts: per-rank bf16 [T_local, H]; idxs, ws_: per-rank routing of the forward pass (int32 / fp32 [T_local, k]).
+    Returns per rank {dx, dw, dW_gate_up (this rank's experts), dW_down, (dW_shared_gate_up, dW_shared_down: this rank's
+    tokens' share of the shared expert's gradient)}."""
+    R = len(xs)
+    T_local, H = xs[0].shape
+    k = idxs[0].shape[1]
+    E = W_gate_up.shape[0]
+    L = E // R
+    I = W_gate_up.shape[1] // 2
+    I_s = 0 if W_shared_gate_up is None else W_shared_gate_up.shape[0] // 2
+    dev = xs[0].device
+    idx_all = torch.stack([i.reshape(-1) for i in idxs]).contiguous()          # the "all-gather" of routes and weights
+    w_all = torch.stack([w.reshape(-1) for w in ws_]).contiguous()
+    rows = mok.mok_ep_y_rows(R, T_local, E, k)
+    tpad = max((T_local + 255) // 256 * 256, 256)
+    nbytes = mok.mok_ep_bwd_workspace_bytes(R, T_local, H, I, I_s, E, k)
+    if nbytes == 0:
+        raise mok.MokError(mok.MOK_ERR_SHAPE)
+    st = []
+    for r in range(R):
+        st.append({"ws": torch.empty(nbytes + 256, dtype=torch.uint8, device=dev),
+                   "dxg": torch.empty((rows, H), dtype=torch.bfloat16, device=dev),
+                   "pos": torch.empty((R * T_local * k,), dtype=torch.int32, device=dev),
+                   "dw_routes": torch.zeros((R * T_local * k,), dtype=torch.float32, device=dev),
+                   "dx_shared": torch.empty((tpad, H), dtype=torch.bfloat16, device=dev) if I_s else None})
+    x_ptrs = [int(x.data_ptr()) for x in xs]
+    d_ptrs = [int(d.data_ptr()) for d in douts]
+    out = []
+    for r in range(R):                                                          # serving side, every rank
+        g = mok.mok_ep_expert_bwd(r, x_ptrs, d_ptrs, idx_all, w_all, W_gate_up[r * L:(r + 1) * L].contiguous(),
+                                  W_down[r * L:(r + 1) * L].contiguous(), W_shared_gate_up, W_shared_down, E, k, H,
+                                  st[r]["dxg"], st[r]["pos"], st[r]["dw_routes"], st[r]["dx_shared"], st[r]["ws"],
+                                  weight_grads=weight_grads, config=config)
+        status = mok.mok_read_status(st[r]["ws"])
+        if status != 0:
+            raise mok.MokError(status)
+        out.append(g)
+    torch.cuda.synchronize()                                                    # the barrier over the ranks
+    dxg_ptrs = [int(s_["dxg"].data_ptr()) for s_ in st]
+    pos_ptrs = [int(s_["pos"].data_ptr()) for s_ in st]
+    dw_ptrs = [int(s_["dw_routes"].data_ptr()) for s_ in st]
+    for r in range(R):                                                          # owner side
+        dx = torch.empty_like(xs[r])
+        dw = torch.empty((T_local, k), dtype=torch.float32, device=dev)
+        mok.mok_ep_bwd_combine(r, R, idxs[r], dxg_ptrs, pos_ptrs, dw_ptrs, st[r]["dx_shared"], E, dx, dw)
+        out[r]["dx"], out[r]["dw"] = dx, dw
+    torch.cuda.synchronize()
+    return out
+
+
 class DistributedLayer:
     """One process per rank under torch.distributed.  Buffers that peers read (x, y, pos) are allocated once and
     exchanged once; `forward` then makes no allocation a peer depends on.

@@ -25,7 +25,8 @@ EXPORTS = ["mok_moe_forward", "mok_workspace_bytes", "mok_workspace_bytes_ring",
            "mok_version", "mok_profile_begin", "mok_profile_end", "mok_schedule_noalloc", "mok_debug_counters",
            "mok_ep_workspace_bytes", "mok_ep_y_rows", "mok_ep_expert_ffn", "mok_ep_combine",
            "mok_mx_scale_bytes", "mok_mx_quantize_weights", "mok_mx_quantize_rows", "mok_mx_workspace_bytes",
-           "mok_ep_mx_workspace_bytes", "mok_bwd_workspace_bytes", "mok_moe_backward", "mok_selftest_per_device",
+           "mok_ep_mx_workspace_bytes", "mok_bwd_workspace_bytes", "mok_moe_backward", "mok_ep_bwd_workspace_bytes",
+           "mok_ep_expert_bwd", "mok_ep_bwd_combine", "mok_selftest_per_device",
            "mok_router_prepared_bytes", "mok_router_prepare"]
 MOK_PRECISION_BF16, MOK_PRECISION_MXFP8 = 0, 1
 MOK_H_RING_MIN_TILES = 24
@@ -85,6 +86,32 @@ class mok_ep_combine_args(ctypes.Structure):
                 ("y_shared", ctypes.c_void_p), ("out", ctypes.c_void_p), ("stream", ctypes.c_void_p)]
 
 
+class mok_ep_bwd_args(ctypes.Structure):
+    _fields_ = [("rank", ctypes.c_int32), ("n_ranks", ctypes.c_int32),
+                ("T_local", ctypes.c_int32), ("H", ctypes.c_int32), ("I", ctypes.c_int32), ("I_shared", ctypes.c_int32),
+                ("E", ctypes.c_int32), ("k", ctypes.c_int32),
+                ("x_peers", ctypes.c_void_p * MOK_MAX_RANKS), ("dout_peers", ctypes.c_void_p * MOK_MAX_RANKS),
+                ("idx_all", ctypes.c_void_p), ("w_all", ctypes.c_void_p),
+                ("W_gate_up", ctypes.c_void_p), ("W_down", ctypes.c_void_p),
+                ("W_shared_gate_up", ctypes.c_void_p), ("W_shared_down", ctypes.c_void_p),
+                ("dxg", ctypes.c_void_p), ("dxg_rows", ctypes.c_longlong), ("pos", ctypes.c_void_p),
+                ("dw_routes", ctypes.c_void_p), ("dx_shared", ctypes.c_void_p),
+                ("dW_gate_up", ctypes.c_void_p), ("dW_down", ctypes.c_void_p),
+                ("dW_shared_gate_up", ctypes.c_void_p), ("dW_shared_down", ctypes.c_void_p),
+                ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
+                ("config", ctypes.POINTER(mok_config)), ("stream", ctypes.c_void_p)]
+
+
+class mok_ep_bwd_combine_args(ctypes.Structure):
+    _fields_ = [("rank", ctypes.c_int32), ("n_ranks", ctypes.c_int32),
+                ("T_local", ctypes.c_int32), ("H", ctypes.c_int32), ("E", ctypes.c_int32), ("k", ctypes.c_int32),
+                ("topk_idx", ctypes.c_void_p),
+                ("dxg_peers", ctypes.c_void_p * MOK_MAX_RANKS), ("pos_peers", ctypes.c_void_p * MOK_MAX_RANKS),
+                ("dw_peers", ctypes.c_void_p * MOK_MAX_RANKS),
+                ("dx_shared", ctypes.c_void_p), ("dx", ctypes.c_void_p), ("dw", ctypes.c_void_p),
+                ("stream", ctypes.c_void_p)]
+
+
 class mok_bwd_args(ctypes.Structure):
     _fields_ = [("x", ctypes.c_void_p), ("W_gate_up", ctypes.c_void_p), ("W_down", ctypes.c_void_p),
                 ("W_shared_gate_up", ctypes.c_void_p), ("W_shared_down", ctypes.c_void_p),
@@ -113,6 +140,8 @@ _lib.mok_ep_combine.restype = ctypes.c_int
 _lib.mok_ep_combine.argtypes = [ctypes.POINTER(mok_ep_combine_args)]
 _lib.mok_workspace_bytes.restype = ctypes.c_size_t
 _lib.mok_workspace_bytes.argtypes = [ctypes.c_int] * 6
+_lib.mok_ep_bwd_workspace_bytes.restype = ctypes.c_size_t
+_lib.mok_ep_bwd_workspace_bytes.argtypes = [ctypes.c_int] * 7
 _lib.mok_workspace_bytes_ring.restype = ctypes.c_size_t
 _lib.mok_workspace_bytes_ring.argtypes = [ctypes.c_int] * 7
 _lib.mok_mx_workspace_bytes.restype = ctypes.c_size_t
@@ -519,6 +548,67 @@ def mok_ep_combine(rank, n_ranks, topk_idx, topk_w, y_peer_ptrs, pos_peer_ptrs, 
     a.stream = _stream(stream).value
     _check(_lib.mok_ep_combine(ctypes.byref(a)))
     return out
+
+
+def mok_ep_bwd_workspace_bytes(n_ranks, T_local, H, I, I_shared, E, k):
+    return int(_lib.mok_ep_bwd_workspace_bytes(n_ranks, T_local, H, I, I_shared, E, k))
+
+
+def mok_ep_expert_bwd(rank, x_peer_ptrs, dout_peer_ptrs, idx_all, w_all, W_gate_up, W_down, W_shared_gate_up,
+                      W_shared_down, E, k, H, dxg, pos, dw_routes, dx_shared, workspace, weight_grads=True, config=None,
+                      stream=None):
+    """Backward chain of one expert-parallel rank on the rows it serves (see include/mok.h).  idx_all / w_all:
+    [n_ranks, T_local*k] all-gathered routes and router weights.  Fills dxg, pos, dw_routes (and dx_shared); returns
+    the local weight gradients {dW_gate_up, dW_down (, dW_shared_gate_up, dW_shared_down)} when weight_grads."""
+    n_ranks, n = idx_all.shape
+    a = mok_ep_bwd_args()
+    a.rank, a.n_ranks, a.T_local, a.H, a.E, a.k = rank, n_ranks, n // k, H, E, k
+    a.I = W_gate_up.shape[1] // 2
+    a.I_shared = 0 if W_shared_gate_up is None else W_shared_gate_up.shape[0] // 2
+    for r in range(n_ranks):
+        a.x_peers[r] = x_peer_ptrs[r]
+        a.dout_peers[r] = dout_peer_ptrs[r]
+    a.idx_all, a.w_all = idx_all.data_ptr(), w_all.data_ptr()
+    a.W_gate_up, a.W_down = W_gate_up.data_ptr(), W_down.data_ptr()
+    a.W_shared_gate_up = None if W_shared_gate_up is None else W_shared_gate_up.data_ptr()
+    a.W_shared_down = None if W_shared_down is None else W_shared_down.data_ptr()
+    a.dxg, a.dxg_rows, a.pos, a.dw_routes = dxg.data_ptr(), dxg.shape[0], pos.data_ptr(), dw_routes.data_ptr()
+    a.dx_shared = None if dx_shared is None else dx_shared.data_ptr()
+    res = {}
+    if weight_grads:
+        res["dW_gate_up"] = torch.empty_like(W_gate_up)
+        res["dW_down"] = torch.empty_like(W_down)
+        if a.I_shared:
+            res["dW_shared_gate_up"] = torch.empty_like(W_shared_gate_up)
+            res["dW_shared_down"] = torch.empty_like(W_shared_down)
+    for name, t in res.items():
+        setattr(a, name, t.data_ptr())
+    a.workspace, a.workspace_bytes = _aligned_ws(workspace)
+    if config is not None:
+        a.config = ctypes.pointer(config)
+    a.stream = _stream(stream).value
+    _check(_lib.mok_ep_expert_bwd(ctypes.byref(a)))
+    return res
+
+
+def mok_ep_bwd_combine(rank, n_ranks, topk_idx, dxg_peer_ptrs, pos_peer_ptrs, dw_peer_ptrs, dx_shared, E, dx, dw=None,
+                       stream=None):
+    """Owner side of the expert-parallel backward: dx[t] = dx_shared[t] + sum_s (row of the serving rank's dxg), and dw."""
+    a = mok_ep_bwd_combine_args()
+    a.rank, a.n_ranks = rank, n_ranks
+    a.T_local, a.k = topk_idx.shape
+    a.H, a.E = dx.shape[1], E
+    a.topk_idx = topk_idx.data_ptr()
+    for r in range(n_ranks):
+        a.dxg_peers[r] = dxg_peer_ptrs[r]
+        a.pos_peers[r] = pos_peer_ptrs[r]
+        a.dw_peers[r] = None if dw_peer_ptrs is None else dw_peer_ptrs[r]
+    a.dx_shared = None if dx_shared is None else dx_shared.data_ptr()
+    a.dx = dx.data_ptr()
+    a.dw = None if dw is None else dw.data_ptr()
+    a.stream = _stream(stream).value
+    _check(_lib.mok_ep_bwd_combine(ctypes.byref(a)))
+    return dx, dw
 
 
 def mok_bwd_workspace_bytes(T, H, I, I_shared, E, k):

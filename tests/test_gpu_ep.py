@@ -209,3 +209,55 @@ def test_expert_parallel_mxfp8_equals_the_one_rank_mxfp8_layer(R):
                                         cfg.k, mx=True))
     one, rep = pu.mx_parity(cfg, d=d, g=g)
     assert torch.equal(out.view(torch.int16), one.view(torch.int16)), rep
+
+
+EP_BWD = [
+    # name, T, H, E, k, I, I_s, bias: ragged segments, empty experts, a shared expert, several row tiles per expert
+    ("shared", 512, 256, 8, 2, 512, 256, "none"),
+    ("skewed", 1024, 512, 32, 4, 384, 0, "zipf"),
+    ("many_rows", 3072, 256, 4, 2, 160, 64, "normal"),
+]
+
+
+@pytest.mark.parametrize("R", [1, 2, 4])
+@pytest.mark.parametrize("name,T,H,E,k,I,I_s,bias", EP_BWD)
+def test_expert_parallel_backward(name, T, H, E, k, I, I_s, bias, R):
+    """The backward pass under expert parallelism (emulated ranks: serving side of every rank, barrier, owner side).
+    dx and dw must equal the one-rank backward pass on the concatenated batch bit for bit (every row goes through the
+    same products, the owner sums its k rows in slot order); the weight gradients sum an expert's rows in Algorithm 1's
+    order, so they are compared with the oracle's fp64 chain rule within the backward tolerances (and, for one rank,
+    where that order is the token order, bit for bit with the one-rank pass)."""
+    from paper_2609_36070_b200 import ep
+    m = mok()
+    cfg = inputs.MoEConfig("epbwd_" + name, T, H, E, k, I, I_s, bias=bias, seed=61)
+    d = inputs.make_inputs(cfg)
+    g = pu.upload(d)
+    out, st = pu.run_gpu(cfg, g)
+    idx, w = st["topk_idx"], st["topk_w"]
+    rng = np.random.default_rng(cfg.seed + 7)
+    dout_bits = inputs.f32_to_bf16_bits(rng.normal(0, 1, (cfg.T, cfg.H)).astype(np.float32))
+    dout = m.to_device_bf16(dout_bits)
+    one = m.mok_moe_backward(g["x"], g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], idx, w, dout)
+    Tl = T // R
+    cut = lambda t: [t[r * Tl:(r + 1) * Tl].contiguous() for r in range(R)]
+    res = ep.backward_emulated(cut(g["x"]), cut(dout), cut(idx), cut(w), g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"])
+    dx = torch.cat([r["dx"] for r in res])
+    dw = torch.cat([r["dw"] for r in res])
+    assert torch.equal(dx.view(torch.int16), one["dx"].view(torch.int16))
+    assert torch.equal(dw.view(torch.int32), one["dw"].view(torch.int32))
+    got = {"dW_gate_up": torch.cat([r["dW_gate_up"] for r in res]).float(),
+           "dW_down": torch.cat([r["dW_down"] for r in res]).float()}
+    if I_s:     # every rank holds the shared expert and contributes its own tokens' share
+        got["dW_sgu"] = sum(r["dW_shared_gate_up"].float() for r in res)
+        got["dW_sd"] = sum(r["dW_shared_down"].float() for r in res)
+    if R == 1:
+        assert torch.equal(res[0]["dW_gate_up"].view(torch.int16), one["dW_gate_up"].view(torch.int16))
+        assert torch.equal(res[0]["dW_down"].view(torch.int16), one["dW_down"].view(torch.int16))
+    ref = mok_ref.backward(d["x"], d["W_gate_up"], d["W_down"], d["W_sgu"], d["W_sd"], idx.cpu().numpy(),
+                           w.cpu().numpy().astype(np.float64), inputs.bf16_bits_to_f32(dout_bits).astype(np.float64),
+                           weights=True)
+    for name_, t in got.items():
+        a, b = t.cpu().numpy().astype(np.float64), ref[name_]
+        diff = np.abs(a - b)
+        assert np.isfinite(a).all(), name_
+        assert diff.max() <= 2e-2 * np.abs(b).max() and diff.mean() <= 1e-2 * np.abs(b).mean(), (name_, R)
