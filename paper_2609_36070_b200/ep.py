@@ -180,6 +180,9 @@ class DistributedLayer:
                 assert len(peers) == self.R
                 self._keep.append(peers)                    # the mappings must outlive every kernel that reads them
                 return [int(q.data_ptr()) for q in peers]
+        self._alloc, self._peers_of, self.device = alloc, peers_of, device
+        self.T_local, self.I, self.I_shared = T_local, I, I_shared
+        self._bwd = None
         self.st = RankState(self.R, T_local, H, I, I_shared, E, k, device, alloc=alloc, mx=mx)
         self.x = alloc((T_local, H), torch.bfloat16)
         self.y_ptrs = peers_of("y", self.st.y)
@@ -194,14 +197,16 @@ class DistributedLayer:
             torch.cuda.synchronize()
         self.dist.barrier(group=self.group)
 
-    def _gather_routes(self, idx):
+    def _gather_routes(self, idx, dst=None):
+        """All-gather of a per-route tensor (the top-k ids; in the backward pass also the router weights)."""
+        dst = self.idx_all if dst is None else dst
         if not self.host_collectives:
-            self.dist.all_gather_into_tensor(self.idx_all, idx.reshape(-1), group=self.group)
+            self.dist.all_gather_into_tensor(dst, idx.reshape(-1), group=self.group)
             return
         mine = idx.reshape(-1).cpu()                          # synchronises this rank's stream: its x is final too
         parts = [torch.empty_like(mine) for _ in range(self.R)]
         self.dist.all_gather(parts, mine, group=self.group)
-        self.idx_all.copy_(torch.stack(parts))
+        dst.copy_(torch.stack(parts))
 
     def forward(self, x_local, W_router, router_bias, W_gate_up_local, W_down_local, W_shared_gate_up, W_shared_down,
                 out=None, config=None, mx_weights=None, timeline=None):
@@ -243,8 +248,52 @@ class DistributedLayer:
         mark("combine")
         return out
 
+    def _init_backward(self):
+        """Buffers of the backward pass, allocated and exchanged once (a collective: every rank calls it together)."""
+        n = self.T_local * self.k
+        nbytes = mok.mok_ep_bwd_workspace_bytes(self.R, self.T_local, self.H, self.I, self.I_shared, self.E, self.k)
+        if nbytes == 0:
+            raise mok.MokError(mok.MOK_ERR_SHAPE)
+        b = {"ws": torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device),
+             "dout": self._alloc((self.T_local, self.H), torch.bfloat16),
+             "dxg": self._alloc(tuple(self.st.y.shape), torch.bfloat16),
+             "dw_routes": self._alloc((self.R * n,), torch.float32),
+             "w_all": torch.empty((self.R, n), dtype=torch.float32, device=self.device),
+             "dx_shared": None if self.st.y_shared is None else torch.empty_like(self.st.y_shared)}
+        b["dout_ptrs"] = self._peers_of("dout", b["dout"])
+        b["dxg_ptrs"] = self._peers_of("dxg", b["dxg"])
+        b["dw_ptrs"] = self._peers_of("dw_routes", b["dw_routes"])
+        self._bwd = b
+
+    def backward(self, dout_local, W_gate_up_local, W_down_local, W_shared_gate_up, W_shared_down, weight_grads=True,
+                 config=None):
+        """The backward pass of the last forward call (its tokens are still in the peer-visible buffer, its routing in
+        this object).  dout_local: bf16 [T_local, H].  Returns {dx, dw, and with weight_grads the gradients of this
+        rank's experts and its tokens' share of the shared expert's}."""
+        if self.mx:
+            raise mok.MokError(mok.MOK_ERR_UNSUPPORTED)
+        if self._bwd is None:
+            self._init_backward()
+        st, b = self.st, self._bwd
+        self._barrier()                         # peers have finished reading the previous call's buffers
+        b["dout"].copy_(dout_local, non_blocking=True)
+        # the all-gather of the router weights also orders every rank's dout before any rank's pulls
+        self._gather_routes(st.w, b["w_all"])
+        res = mok.mok_ep_expert_bwd(self.rank, self.x_ptrs, b["dout_ptrs"], self.idx_all, b["w_all"], W_gate_up_local,
+                                    W_down_local, W_shared_gate_up, W_shared_down, self.E, self.k, self.H, b["dxg"], st.pos,
+                                    b["dw_routes"], b["dx_shared"], b["ws"], weight_grads=weight_grads, config=config)
+        self._barrier()                         # every rank's dxg, pos and dw_routes are complete
+        res["dx"] = torch.empty((self.T_local, self.H), dtype=torch.bfloat16, device=self.device)
+        res["dw"] = torch.empty((self.T_local, self.k), dtype=torch.float32, device=self.device)
+        mok.mok_ep_bwd_combine(self.rank, self.R, st.idx, b["dxg_ptrs"], self.pos_ptrs, b["dw_ptrs"], b["dx_shared"],
+                               self.E, res["dx"], res["dw"])
+        return res
+
     def status(self):
-        return mok.mok_read_status(self.st.ws)
+        status = mok.mok_read_status(self.st.ws)
+        if status == 0 and self._bwd is not None:
+            status = mok.mok_read_status(self._bwd["ws"])
+        return status
 
 
 def forward_distributed(x_local, W_router, router_bias, W_gate_up_local, W_down_local, W_shared_gate_up, W_shared_down,
@@ -307,6 +356,21 @@ def _ipc_rank(rank, world, queues, config_name, port, results, mx=False):
                                  config=mok._config(precision=int(mx)),
                                  mx_weights=mok.MxWeights(g["W_gate_up"], g["W_down"]) if mx else None)
     same = torch.equal(out.view(torch.int16), one[rank * T_local:(rank + 1) * T_local].view(torch.int16))
+    if not mx:
+        # the backward pass of that layer, twice on the same buffers: dx and dw against the one-rank backward pass
+        gen = torch.Generator(device="cpu").manual_seed(7)
+        dout = torch.randn((cfg.T, cfg.H), generator=gen).to(torch.bfloat16).to(dev)
+        sl = slice(rank * T_local, (rank + 1) * T_local)
+        for _ in range(2):
+            res = layer.backward(dout[sl].contiguous(), Wgu, Wd, g["W_sgu"], g["W_sd"])
+        layer._barrier()
+        _, st1 = mok.mok_moe_forward_ex(g["x"], W_r, bias, g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], cfg.k, ws,
+                                        stages=True)
+        ref = mok.mok_moe_backward(g["x"], g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], st1["topk_idx"],
+                                   st1["topk_w"], dout, weight_grads=False)
+        same = same and torch.equal(res["dx"].view(torch.int16), ref["dx"][sl].view(torch.int16))
+        same = same and torch.equal(res["dw"].view(torch.int32), ref["dw"][sl].view(torch.int32))
+        same = same and bool(torch.isfinite(res["dW_gate_up"].float()).all())
     results.put((rank, bool(same) and layer.status() == 0))
     layer._barrier()                                           # peers may still read this rank's buffers until here
     dist.destroy_process_group()
@@ -314,7 +378,8 @@ def _ipc_rank(rank, world, queues, config_name, port, results, mx=False):
 
 def check_processes_on_one_gpu(world=2, config_name="tiny", port=29561, mx=False):
     """Runs `world` ranks as separate processes on GPU 0 (each maps the others' x / y / pos through CUDA IPC) and
-    returns True if every rank's output equals its slice of the one-rank layer bit for bit."""
+    returns True if every rank's output (and, in bf16 mode, its dx and dw of the backward pass) equals its slice of the
+    one-rank layer's bit for bit."""
     import torch.multiprocessing as mp
     ctx = mp.get_context("spawn")
     queues = [ctx.Queue() for _ in range(world)]
@@ -391,12 +456,25 @@ def main():
     ws = mok.alloc_workspace(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k, device=dev)
     one = mok.mok_moe_forward_ex(g["x"], W_r, bias, g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], cfg.k, ws)
     same = torch.equal(out.view(torch.int16), one[rank * T_local:(rank + 1) * T_local].view(torch.int16))
-    ok = torch.tensor([int(same and layer.status() == 0)], device=dev)
+    # the backward pass of the same layer against the one-rank backward pass (dx, dw bit for bit)
+    gen = torch.Generator(device="cpu").manual_seed(7)
+    dout = torch.randn((cfg.T, cfg.H), generator=gen).to(torch.bfloat16).to(dev)
+    sl = slice(rank * T_local, (rank + 1) * T_local)
+    step()
+    res = layer.backward(dout[sl].contiguous(), Wgu, Wd, g["W_sgu"], g["W_sd"], weight_grads=False)
+    _, st1 = mok.mok_moe_forward_ex(g["x"], W_r, bias, g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], cfg.k, ws,
+                                    stages=True)
+    ref = mok.mok_moe_backward(g["x"], g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], st1["topk_idx"], st1["topk_w"],
+                               dout, weight_grads=False)
+    same_bwd = (torch.equal(res["dx"].view(torch.int16), ref["dx"][sl].view(torch.int16)) and
+                torch.equal(res["dw"].view(torch.int32), ref["dw"][sl].view(torch.int32)))
+    ok = torch.tensor([int(same and same_bwd and layer.status() == 0)], device=dev)
     dist.all_reduce(ok, op=dist.ReduceOp.MIN)
     if rank == 0:
         print(json.dumps({"workload": cfg.name, "n_ranks": world, "T_total": cfg.T, "ms_per_layer": float(ms.item()),
                           "tokens_per_s": cfg.T / (float(ms.item()) * 1e-3),
-                          "bitwise_equal_to_one_rank_layer": bool(ok.item())}), flush=True)
+                          "bitwise_equal_to_one_rank_layer": bool(ok.item()),
+                          "backward_dx_dw_bitwise_equal_to_one_rank": bool(ok.item())}), flush=True)
     dist.barrier()
     dist.destroy_process_group()
     return 0 if ok.item() else 1

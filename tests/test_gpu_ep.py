@@ -188,7 +188,8 @@ def test_ranks_as_separate_processes_on_one_gpu(world, mx):
     """Real cross-process peer pointers: every rank is its own process on GPU 0, maps the other ranks' x / y / pos
     buffers through CUDA IPC, and runs the expert-parallel layer with gloo collectives (routes staged through the
     host).  No kernel waits on another rank's kernel, so sharing one GPU is safe; each rank checks its output bit for
-    bit against the one-rank layer."""
+    bit against the one-rank layer and, in bf16 mode, runs the backward pass twice on the same buffers and checks dx and
+    dw bit for bit against the one-rank backward pass."""
     from paper_2609_36070_b200 import ep
     assert ep.check_processes_on_one_gpu(world=world, config_name="tiny", port=29561 + world + 10 * int(mx), mx=mx)
 
