@@ -57,6 +57,7 @@ enum { MOK_PRECISION_BF16 = 0, MOK_PRECISION_MXFP8 = 1 };
 
 #define MOK_MAX_HOST_CHUNKS 8
 #define MOK_DEBUG_STARVE 2
+#define MOK_DEBUG_NO_ARRIVALS 3
 
 /* Optional tuning / debugging knobs.  Zero-initialise for defaults. */
 typedef struct mok_config {
@@ -75,7 +76,10 @@ typedef struct mok_config {
     int32_t debug;        /* 1: the tcgen05 GEMMs accumulate wait-time counters (see mok_debug_counters).
                              MOK_DEBUG_STARVE: test hook for the bounded waits -- the gate/up GEMM's TMA producer
                              issues nothing and every wait gives up after 2 ms, so the call must end with
-                             mok_read_status() == MOK_ERR_TIMEOUT and a usable context (output undefined) */
+                             mok_read_status() == MOK_ERR_TIMEOUT and a usable context (output undefined).
+                             MOK_DEBUG_NO_ARRIVALS: the same for the completion counters of the one-launch expert FFN
+                             that gate a ring slot's reuse (h_ring_tiles) and the in-launch combine (fused_ffn = 3):
+                             nobody arrives on them, so those waits run out */
     int32_t host_chunks;  /* mok_moe_forward_host: token chunks whose copies overlap compute (0 = choose by T,
                              at most MOK_MAX_HOST_CHUNKS) */
     int32_t precision;    /* MOK_PRECISION_BF16 (0, default) or MOK_PRECISION_MXFP8: routed experts on MXFP8 operands

@@ -338,7 +338,7 @@ struct FusedArgs {
     int32_t n1, n2;                // N tiles of a gate/up row tile (ceil(I / 128)) and of a down row tile (ceil(H / 256))
     int32_t kb1, kb2;              // k-blocks of the two kinds
     int32_t dbg;                   // != 0: counters into header->dbg[1] (gate/up tiles) and [2] (down tiles)
-    int32_t starve;                // test hook: the producer issues nothing
+    int32_t starve;                // test hooks: 1 = the producer issues nothing, 2 = nobody arrives on `consumed` / `ffn_done`
     WsHeader* header;
     // combine in the same launch (out != NULL)
     const __nv_bfloat16* y;        // [Rpad, H] rows of the down tiles
@@ -360,7 +360,7 @@ __device__ __forceinline__ void combine_tokens(const FusedArgs& a, int lane, vol
     const int need = EPI_WARPS * (int)gridDim.x;
     int ok = 1;
     if (lane == 0) {
-        if (arrive) {
+        if (arrive && a.starve != 2) {
             // (the warp's TMA stores have completed: make them visible to generic-proxy reads of other SMs, then arrive)
             asm volatile("fence.proxy.async;" ::: "memory");
             __threadfence();
@@ -523,7 +523,7 @@ fused_ffn_kernel(const __grid_constant__ CUtensorMap mapWgu, const __grid_consta
         reg_dec<REGS_CONTROL>();
         if (warp == 0) {
             // -------------------------------------------------------------- TMA producer
-            if (lane == 0 && !a.starve) {
+            if (lane == 0 && a.starve != 1) {
                 int s = 0;
                 uint32_t ph = 0;
                 long long d_ready = 0;
@@ -692,7 +692,7 @@ fused_ffn_kernel(const __grid_constant__ CUtensorMap mapWgu, const __grid_consta
                     }
                     if (!ok) break;
                     // ring mode: every load of h of this down entry has landed (its stages' full barriers were passed)
-                    if (a.ring && t.kind)
+                    if (a.ring && t.kind && a.starve != 2)
                         asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(a.consumed + t.mt) : "memory");
                     if (dbg) {
                         const long long dt = clock64() - tile0, units = (long long)(two ? 2 : 1) * kblocks * t.cnt;
@@ -994,7 +994,7 @@ static cudaError_t launch_kernel(int grid, cudaStream_t s, const CUtensorMap& m0
 // (a group's down tiles directly behind its gate/up tiles).
 cudaError_t launch_fused_ffn(const __nv_bfloat16* x, int T, int H, int I, int E, const __nv_bfloat16* Wgu,
                              const __nv_bfloat16* Wd, const WsLayout& L, char* ws, int grid, int window_tiles, bool dynamic,
-                             bool gang_sync, bool dbg, bool starve, cudaStream_t s, __nv_bfloat16* combine_out, int k,
+                             bool gang_sync, bool dbg, int starve, cudaStream_t s, __nv_bfloat16* combine_out, int k,
                              bool shared, int h_ring_tiles) {
     using namespace ff;
     int dev = 0, sm_count = 0;
@@ -1057,7 +1057,7 @@ cudaError_t launch_fused_ffn(const __nv_bfloat16* x, int T, int H, int I, int E,
     a.kb1 = (H + BK - 1) / BK;
     a.kb2 = (I + BK - 1) / BK;
     a.dbg = dbg ? 1 : 0;
-    a.starve = starve ? 1 : 0;
+    a.starve = starve;
     a.header = hdr;
     a.y = reinterpret_cast<const __nv_bfloat16*>(y);
     a.ysh = shared ? reinterpret_cast<const __nv_bfloat16*>(ws + L.ysh) : nullptr;

@@ -373,12 +373,13 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
     g.counts = reinterpret_cast<const int32_t*>(ws + L.counts);
     const bool dbg = a->config && a->config->debug == 1;
     g.dbg_slot = dbg ? 1 : -1;
-    if (a->config && a->config->debug == MOK_DEBUG_STARVE) {
-        // test hook (see mok.h): the gate/up GEMM's producer stays silent and every wait gives up after 2 ms
+    if (a->config && (a->config->debug == MOK_DEBUG_STARVE || a->config->debug == MOK_DEBUG_NO_ARRIVALS)) {
+        // test hooks (see mok.h): the gate/up GEMM's producer stays silent, or the one-launch kernel's completion
+        // counters get no arrivals; every wait gives up after 2 ms
         const uint32_t limit_us = 2000;
         e = cudaMemcpyAsync(&hdr->wait_limit_us, &limit_us, sizeof(limit_us), cudaMemcpyHostToDevice, s);
         if (e != cudaSuccess) return cuda_fail(e);
-        g.starve = 1;
+        g.starve = a->config->debug == MOK_DEBUG_STARVE ? 1 : 2;
     }
     bool combine_in_launch = false;
     // shared expert: every token in natural order, no gather.  Runs after the routed experts, or before them when the
@@ -471,6 +472,7 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
         g.tile_sched = a->config ? a->config->tile_sched : 0;
         const bool fused = !simt && use_fused_ffn(a->config, a->H, a->I, tile_m, L.R, a->E, L.max_ftiles);
         if (L.h_ring > 0 && !fused) return MOK_ERR_UNSUPPORTED;     // the ring exists in the one-launch kernel only
+        if (!fused && g.starve == 2) g.starve = 0;                  // (that hook only exists in the one-launch kernel)
         combine_in_launch = fused && a->config && a->config->fused_ffn == 3;
         if (combine_in_launch && (rc = shared_expert())) return rc;       // its output is an input of that launch
         // its hand-out: synchronised starts need the static stride (a CTA that draws ahead could hold two tiles of a gang)
@@ -482,7 +484,7 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
         if (fused) {
             e = launch_fused_ffn(x, a->T, a->H, a->I, a->E, reinterpret_cast<const __nv_bfloat16*>(a->W_gate_up),
                                  reinterpret_cast<const __nv_bfloat16*>(a->W_down), L, ws, a->config ? a->config->grid : 0,
-                                 a->config ? a->config->fused_window : 0, fused_dynamic, fused_sync, dbg, g.starve != 0, s,
+                                 a->config ? a->config->fused_window : 0, fused_dynamic, fused_sync, dbg, g.starve, s,
                                  combine_in_launch ? out : nullptr, a->k, a->I_shared > 0, L.h_ring);
             if (e != cudaSuccess) return cuda_fail(e);
         } else if ((rc = run_gemm(g, true, a->config, L, ws, s))) return rc;

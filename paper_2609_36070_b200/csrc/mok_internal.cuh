@@ -157,7 +157,7 @@ cudaError_t launch_gemm_mx(const GemmArgs& a, int epi, int grid, cudaStream_t s)
 // routed gate/up + SwiGLU + down in one persistent launch (tile list + kernel); needs the schedule's 256-row tile table
 cudaError_t launch_fused_ffn(const __nv_bfloat16* x, int T, int H, int I, int E, const __nv_bfloat16* Wgu,
                              const __nv_bfloat16* Wd, const WsLayout& L, char* ws, int grid, int window_tiles, bool dynamic,
-                             bool gang_sync, bool dbg, bool starve, cudaStream_t s, __nv_bfloat16* combine_out = nullptr,
+                             bool gang_sync, bool dbg, int starve, cudaStream_t s, __nv_bfloat16* combine_out = nullptr,
                              int k = 0, bool shared = false,    // combine_out != NULL: the combine runs in the same launch
                              int h_ring_tiles = 0);             // > 0: h is a ring of that many 256-row tiles
 constexpr int H_RING_MIN_TILES = 24;     // smallest ring of the gated activation (see gemm_fused.cu)

@@ -33,6 +33,7 @@ MOK_H_RING_MIN_TILES = 24
 MOK_MAX_RANKS = 16
 MOK_NOALLOC_MAX_ROUTES = 32768
 MOK_DEBUG_STARVE = 2
+MOK_DEBUG_NO_ARRIVALS = 3
 STAGES = ["router", "schedule", "gather", "gemm1", "gemm2", "shared_gemm1", "shared_gemm2", "combine"]
 
 

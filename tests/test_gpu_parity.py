@@ -486,6 +486,26 @@ def test_bounded_waits_report_a_timeout_and_leave_the_context_usable(fused, sche
     assert torch.equal(good.view(torch.int16), again.view(torch.int16))
 
 
+@pytest.mark.parametrize("kw", [{"h_ring_tiles": 24}, {"h_ring_tiles": 24, "tile_sched": 1}, {"fused_ffn": 3},
+                                {"fused_ffn": 3, "tile_sched": 2}], ids=["ring", "ring_dynamic", "combine", "combine_static"])
+def test_completion_counter_waits_of_the_one_launch_kernel_run_out_cleanly(kw):
+    """The waits on the one-launch kernel's own completion counters -- a ring slot's previous rows consumed, all
+    epilogue warps done before the in-launch combine -- are bounded too: with the test hook that suppresses every
+    arrival on those counters (and a 2 ms limit) the call ends with MOK_ERR_TIMEOUT, nothing faults, and the next call
+    on the same context and workspace gives the normal bits."""
+    m = mok()
+    cfg = MID[0]                                     # about 40 row tiles: a ring of 24 slots wraps
+    d = inputs.make_inputs(cfg)
+    g = pu.upload(d)
+    ws = m.alloc_workspace(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k)
+    good = pu.run_gpu(cfg, g, ws=ws, config=m._config(**kw), stages=False).clone()
+    m.mok_moe_forward_ex(g["x"], g["W_r"], g["bias"], g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], cfg.k, ws,
+                         config=m._config(debug=m.MOK_DEBUG_NO_ARRIVALS, **kw))
+    assert m.mok_read_status(ws) == m.MOK_ERR_TIMEOUT
+    again = pu.run_gpu(cfg, g, ws=ws, config=m._config(**kw), stages=False)
+    assert torch.equal(good.view(torch.int16), again.view(torch.int16))
+
+
 def test_forward_can_be_captured_in_a_cuda_graph_and_replayed():
     """The layer makes no host synchronisation and no allocation after its first call for a shape, so a whole
     forward can be recorded once into a CUDA graph and replayed (launch-bound small batches): same bits."""
