@@ -69,6 +69,7 @@ def parse():
                         "comma-separated list of workload names")
     p.add_argument("--no-sweep", action="store_true", help="skip the small-T sweep of the default workload")
     p.add_argument("--no-e2e", action="store_true", help="skip the host-buffer (end-to-end) legs")
+    p.add_argument("--no-backward", action="store_true", help="skip the backward-pass record of the headline workload")
     p.add_argument("--no-counters", action="store_true", help="skip the device-side counter pass")
     p.add_argument("--cooldown", type=float, default=2.0,
                    help="idle seconds before each workload's warm-up, so that every workload starts from the same board state")
@@ -269,11 +270,49 @@ def run_reference(args, cfg, rank):
     print(json.dumps(line), flush=True)
 
 
-def run_backward(args, cfg):
-    """Times mok_moe_backward (activation recomputation, dx, router-weight and weight gradients) on one GPU.  FLOPs
-    are counted as twice the forward pass's (dgrad + wgrad), as in the paper's Section 4.1; the recomputed gate/up
-    product and the transposes are extra work that is not counted."""
+def backward_record(cfg, g, idx, w, steps, warmup, cta_group=0, sampler=None):
+    """Times mok_moe_backward (activation recomputation, dx, router-weight and weight gradients) on tensors already on
+    the device; idx / w: the forward pass's routing.  FLOPs are counted as twice the forward pass's (dgrad + wgrad), as
+    in the paper's Section 4.1; the recomputed gate/up product and the transposes are extra work that is not counted."""
     import numpy as np
+    import torch
+    from paper_2609_36070_b200 import inputs, mok
+    dev = g["x"].device
+    rng = np.random.default_rng(1)
+    dout = mok.to_device_bf16(inputs.f32_to_bf16_bits(rng.standard_normal((cfg.T, cfg.H), dtype=np.float32)), dev)
+    res = mok.mok_moe_backward(g["x"], g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], idx, w, dout)
+    bws = res["workspace"]
+    conf = mok._config(cta_group=cta_group)
+
+    def step():
+        mok.mok_moe_backward(g["x"], g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], idx, w, dout, workspace=bws,
+                             config=conf)
+
+    for _ in range(max(warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    t0 = time.time()
+    ev[0].record()
+    for i in range(steps):
+        step()
+        ev[i + 1].record()
+    torch.cuda.synchronize()
+    t1 = time.time()
+    per = sorted(ev[i].elapsed_time(ev[i + 1]) for i in range(steps))
+    ms = per[len(per) // 2]
+    assert mok.mok_read_status(bws) == 0
+    flops = 2.0 * cfg.ffn_flops()
+    rec = {"ms_per_step": ms, "mean_ms_per_step": ev[0].elapsed_time(ev[steps]) / steps, "steps": steps,
+           "tokens_per_s": cfg.T / (ms * 1e-3), "tflops": flops / (ms * 1e-3) / 1e12,
+           "flops_counted": "2 x forward (dgrad + wgrad); the recomputed gate/up product is extra work, not counted",
+           "pass": "backward (recompute + dgrad + wgrad), bf16", "_window": (t0, t1)}
+    del res, bws, dout
+    return rec
+
+
+def run_backward(args, cfg):
+    """`--pass backward`: the backward pass of one workload on one GPU, one JSON line."""
     import torch
     from paper_2609_36070_b200 import inputs, mok
     dev = torch.device("cuda", 0)
@@ -285,40 +324,18 @@ def run_backward(args, cfg):
     ws = mok.alloc_workspace(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k, device=dev)
     out, st = mok.mok_moe_forward_ex(g["x"], W_r, bias, g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], cfg.k, ws,
                                      stages=True)
-    idx, w = st["topk_idx"], st["topk_w"]
-    rng = np.random.default_rng(1)
-    dout = mok.to_device_bf16(inputs.f32_to_bf16_bits(rng.standard_normal((cfg.T, cfg.H), dtype=np.float32)), dev)
-    res = mok.mok_moe_backward(g["x"], g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], idx, w, dout)
-    bws = res["workspace"]
-    conf = mok._config(cta_group=args.cta_group)
-
-    def step():
-        mok.mok_moe_backward(g["x"], g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], idx, w, dout, workspace=bws,
-                             config=conf)
-
-    for _ in range(max(args.warmup, 3)):
-        step()
-    torch.cuda.synchronize()
     sampler = ClockSampler(0)
     sampler.start()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    t0 = time.time()
-    ev0.record()
-    for _ in range(args.steps):
-        step()
-    ev1.record()
-    torch.cuda.synchronize()
-    t1 = time.time()
+    rec = backward_record(cfg, g, st["topk_idx"], st["topk_w"], args.steps, args.warmup, args.cta_group)
     sampler.stop()
-    ms = ev0.elapsed_time(ev1) / args.steps
-    assert mok.mok_read_status(bws) == 0
-    flops = 2.0 * cfg.ffn_flops()
-    print(json.dumps({"metric": "moe_layer_bwd_tokens_per_s", "value": cfg.T / (ms * 1e-3), "unit": UNIT, "n_gpus": 1,
-                      "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True,
-                      "dtype": "bf16", "data": "synthetic", "tflops": flops / (ms * 1e-3) / 1e12,
+    win = rec.pop("_window")
+    print(json.dumps({"metric": "moe_layer_bwd_tokens_per_s", "value": rec["tokens_per_s"], "unit": UNIT, "n_gpus": 1,
+                      "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": rec["ms_per_step"],
+                      "mean_ms_per_step": rec["mean_ms_per_step"], "higher_is_better": True,
+                      "dtype": "bf16", "data": "synthetic", "tflops": rec["tflops"],
                       "config": {"workload": cfg.name, "T": cfg.T, "H": cfg.H, "E": cfg.E, "k": cfg.k, "I": cfg.I,
-                                 "I_shared": cfg.I_s, "pass": "backward (recompute + dgrad + wgrad)"},
-                      "clocks": sampler.window(t0, t1)}), flush=True)
+                                 "I_shared": cfg.I_s, "pass": rec["pass"]},
+                      "clocks": sampler.window(*win)}), flush=True)
 
 
 class Layer:
@@ -859,6 +876,24 @@ def main():
             dist.destroy_process_group()
         return
 
+    # ------------------------------------------------------------------ backward pass of the headline workload (N = 1)
+    backward = None
+    if world == 1 and not args.no_backward and not mx and gpu_idx is not None:
+        free, _ = torch.cuda.mem_get_info()
+        need = (mok.mok_bwd_workspace_bytes(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k) +
+                6.0 * cfg.E * cfg.H * cfg.I + 6.0 * cfg.H * cfg.I_s + 4.0 * cfg.T * cfg.H + (2 << 30))
+        if free > need:
+            _, stb = layer.step(layer.conf(), stages=True)
+            time.sleep(args.cooldown)
+            backward = backward_record(cfg, layer.g, stb["topk_idx"], stb["topk_w"], max(5, min(args.steps, 10)), 3,
+                                       args.cta_group)
+            windows.append((backward, "clocks", backward.pop("_window")))
+            del stb
+            gc.collect()
+            torch.cuda.empty_cache()
+        else:
+            backward = {"skipped": f"needs {need / 2**30:.0f} GiB of free device memory, {free / 2**30:.0f} free"}
+
     # ------------------------------------------------------------------ small-T sweep of the default workload (N = 1)
     sweep = None
     if world == 1 and not args.no_sweep and args.config == DEFAULT_WORKLOAD and not args.tokens and not args.experts:
@@ -1009,6 +1044,8 @@ def main():
         line["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": threads, "kind": "oracle", "seconds": secs,
                                 "sample": f"routing of all {cfg.T} tokens (charged pro rata) + fp64 FFN of the first {min(sample, cfg.T)} tokens"}
         line["routing_check"] = rep
+    if backward is not None:
+        line["backward"] = backward
     if per_config:
         line["per_config"] = per_config
     if sweep:
