@@ -84,6 +84,7 @@ struct Ctrl {
     uint64_t q_full[QSLOTS], q_empty[QSLOTS];
     int32_t q_tile[QSLOTS];
     uint32_t tmem_base, abort;
+    uint32_t combine_go;                 // in-launch combine: the grid has finished its tiles (written by the CTA's poller)
 };
 static_assert(sizeof(Ctrl) <= SMEM_CTRL, "control block too large");
 
@@ -354,37 +355,44 @@ struct FusedArgs {
 // EPI_WARPS * gridDim.x arrivals and draws tokens from a global counter, one token per warp at a time: 16 bytes per
 // lane and row, CH chunks of a row per pass with the k rows of every chunk loaded before the first multiply-add,
 // accumulation in fp32 in slot order on top of the shared expert's row.
+// (every epilogue and gather warp of the CTA calls this exactly once, whatever happened before: the two named barriers
+//  below count all COMBINE_THREADS threads.  ONE thread per CTA polls the grid-wide counter: with every warp of the grid
+//  polling, the polls swamp the L2 slice that also has to take the arrivals.)
+constexpr int COMBINE_THREADS = 32 * EPI_WARPS + GATHER_THREADS;
 template <int CH>
-__device__ __forceinline__ void combine_tokens(const FusedArgs& a, int lane, volatile uint32_t* abort_flag, bool arrive) {
+__device__ __forceinline__ void combine_tokens(const FusedArgs& a, Ctrl* ctrl, int lane, bool poller,
+                                               volatile uint32_t* abort_flag, bool arrive) {
     int32_t* done = &a.header->ffn_done;
     const int need = EPI_WARPS * (int)gridDim.x;
-    int ok = 1;
-    if (lane == 0) {
-        if (arrive && a.starve != 2) {
-            // (the warp's TMA stores have completed: make them visible to generic-proxy reads of other SMs, then arrive)
-            asm volatile("fence.proxy.async;" ::: "memory");
-            __threadfence();
-            asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(done) : "memory");
-        }
+    if (lane == 0 && arrive && a.starve != 2 && !*abort_flag) {
+        // (the warp's TMA stores have completed: make them visible to generic-proxy reads of other SMs, then arrive)
+        asm volatile("fence.proxy.async;" ::: "memory");
+        __threadfence();
+        asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(done) : "memory");
+    }
+    asm volatile("bar.sync 1, %0;" ::"n"(COMBINE_THREADS) : "memory");      // this CTA's warps are through with their tiles
+    if (poller && lane == 0) {
+        uint32_t go = *abort_flag ? 0u : 1u;
         const unsigned long long t0 = globaltimer();
         uint32_t spins = 0;
-        while (ld_acquire(done) < need) {
-            __nanosleep(128);
-            if ((++spins & 63u) == 0u) {
-                if (*abort_flag) { ok = 0; break; }
+        while (go && ld_acquire(done) < need) {
+            __nanosleep(256);
+            if ((++spins & 31u) == 0u) {
+                if (*abort_flag) { go = 0u; break; }
                 const unsigned long long limit = a.header->wait_limit_us ? 1000ull * a.header->wait_limit_us : WAIT_LIMIT_NS;
                 if (globaltimer() - t0 > limit) {
                     *abort_flag = 1u;
                     atomicCAS(&a.header->status, 0, (int)MOK_ERR_TIMEOUT);
                     a.header->where = 44;
-                    ok = 0;
+                    go = 0u;
                     break;
                 }
             }
         }
+        *reinterpret_cast<volatile uint32_t*>(&ctrl->combine_go) = go;
     }
-    ok = __shfl_sync(0xffffffffu, ok, 0);
-    if (!ok) return;
+    asm volatile("bar.sync 1, %0;" ::"n"(COMBINE_THREADS) : "memory");      // the poller's verdict is in shared memory
+    if (!*reinterpret_cast<volatile uint32_t*>(&ctrl->combine_go)) return;
     const int chunks = a.H >> 3, k = a.k;
     for (;;) {
         int t = 0;
@@ -803,7 +811,7 @@ fused_ffn_kernel(const __grid_constant__ CUtensorMap mapWgu, const __grid_consta
         }
         asm volatile("cp.async.wait_all;" ::: "memory");
         // (the gather warps help with the combine: more bytes in flight per SM)
-        if (__all_sync(0xffffffffu, a.out != nullptr && !*abort_flag)) combine_tokens<1>(a, lane, abort_flag, false);
+        if (a.out != nullptr) combine_tokens<1>(a, ctrl, lane, false, abort_flag, false);
     } else {
         // ------------------------------------------------------------------ epilogue warps
         reg_inc<REGS_EPILOGUE>();
@@ -940,8 +948,7 @@ fused_ffn_kernel(const __grid_constant__ CUtensorMap mapWgu, const __grid_consta
         }
         if (lane == 0) tma_store_wait_all();
         __syncwarp();
-        // (one decision per warp: the combine exchanges values between lanes)
-        if (__all_sync(0xffffffffu, a.out != nullptr && !*abort_flag)) combine_tokens<2>(a, lane, abort_flag, true);
+        if (a.out != nullptr) combine_tokens<2>(a, ctrl, lane, warp == 4, abort_flag, true);
     }
 
     // ---------------------------------------------------------------------- teardown
