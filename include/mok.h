@@ -131,6 +131,12 @@ typedef struct mok_config {
                              group's gate/up and down tiles is cut to the ring size minus 16 tiles.  The workspace is
                              then the smaller one of mok_workspace_bytes_ring (no h rows beyond the ring, no gathered
                              copy of x).  Same bits. */
+    int32_t shared_overlap; /* shared expert: 2 = its two GEMMs run on a library-owned second stream on 16 SMs beside the
+                             router, the schedule and the routed experts (forked from and joined to `stream` by events,
+                             before the combine; the routed kernels then take the other SMs); 1 = in line, after the
+                             routed experts; 0 = beside them for small layers only (at most 160 routed rows per expert
+                             and 64 MB of expert weights), whose kernels are bound by launch and fill latency rather
+                             than by DRAM or the tensor cores (Section 3.4 "Shared Expert").  Same bits. */
 } mok_config;
 #define MOK_H_RING_MIN_TILES 24
 

@@ -169,7 +169,8 @@ static int validate(const mok_args* a, WsLayout* L, size_t extra_ws) {
                       a->config->host_chunks < 0 || a->config->host_chunks > MOK_MAX_HOST_CHUNKS ||
                       a->config->fused_ffn < 0 || a->config->fused_ffn > 3 || a->config->fused_window < -1 ||
                       a->config->gang_sync < 0 || a->config->gang_sync > 2 || a->config->serial_launches < 0 ||
-                      a->config->serial_launches > 1 || a->config->h_ring_tiles < 0))
+                      a->config->serial_launches > 1 || a->config->h_ring_tiles < 0 || a->config->shared_overlap < 0 ||
+                      a->config->shared_overlap > 2))
         return MOK_ERR_SHAPE;
     return MOK_OK;
 }
@@ -321,6 +322,49 @@ static int route_stage(const mok_args* a, const WsLayout& L, char* ws, const __n
     return MOK_OK;
 }
 
+// A second, library-owned stream per device for the shared expert (see forward_device): forked from and joined to the
+// caller's stream with two events, so the caller sees one stream's worth of ordering (and a stream capture of the call
+// captures both).
+struct SidePipe {
+    cudaStream_t stream = nullptr;
+    cudaEvent_t fork = nullptr, join = nullptr;
+    bool ready = false;
+};
+static SidePipe g_side[64];
+static int side_pipe(SidePipe** out) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (dev < 0 || dev >= 64) return MOK_ERR_UNSUPPORTED;
+    SidePipe& p = g_side[dev];
+    if (!p.ready) {
+        if ((e = cudaStreamCreateWithFlags(&p.stream, cudaStreamNonBlocking)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaEventCreateWithFlags(&p.fork, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaEventCreateWithFlags(&p.join, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
+        p.ready = true;
+    }
+    *out = &p;
+    return MOK_OK;
+}
+constexpr int SIDE_CTAS = 16;           // persistent CTAs of the shared expert's GEMMs while they run beside the routed ones
+
+// Shared expert beside the routed experts (Section 3.4 "Shared Expert": it does not depend on the dispatch, so it can
+// fill time the routed path leaves idle).  On one GPU that pays for SMALL layers only, whose kernels are a few tiles
+// each and bound by launch and pipeline-fill latency: there the shared expert's two GEMMs run while router, schedule
+// and routed GEMMs go through their own latencies (tiny workload: 47 against 60 us per layer).  It does not pay where
+// the routed GEMMs stream expert weights from DRAM (few rows per expert, large experts): a CTA pulls about 40 GB/s, so
+// that phase needs every SM to reach the DRAM bandwidth, and each SM given to the shared expert is lost to it
+// (DeepSeek-like layer at 64 / 4096 tokens: 3.59 against 3.40 ms, 6.6 against 4.9 ms).  Nor with many rows per expert,
+// where both are bound by the tensor cores or the power cap and a split of the SMs conserves the work.
+static bool shared_beside_routed(const mok_config* cfg, int H, int I, int I_shared, long long rows, int experts) {
+    if (I_shared <= 0) return false;
+    const int mode = cfg ? cfg->shared_overlap : 0;
+    if (mode == 1) return false;
+    if (cfg && (cfg->debug == MOK_DEBUG_STARVE || cfg->debug == MOK_DEBUG_NO_ARRIVALS || cfg->fused_ffn == 3)) return false;
+    if (mode == 2) return true;
+    return rows <= 160ll * experts && 6ll * experts * H * I <= (64ll << 20);
+}
+
 // The whole layer on device pointers.  x / out may differ from a->x / a->out (host-buffer variant).
 static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloat16* x, __nv_bfloat16* out,
                           bool reset_header = true) {
@@ -331,11 +375,33 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
     cudaError_t e = reset_header ? cudaMemsetAsync(hdr, 0, sizeof(WsHeader), s)
                                  : cudaMemsetAsync(&hdr->n_flag, 0, sizeof(hdr->n_flag), s);
     if (e != cudaSuccess) return cuda_fail(e);
-    g_pdl = !(a->config && a->config->serial_launches);
+    // a private copy of the knobs: the grid of the routed kernels shrinks while the shared expert runs beside them
+    mok_config cfg_main;
+    if (a->config) cfg_main = *a->config; else memset(&cfg_main, 0, sizeof(cfg_main));
+    mok_args a_main = *a;
+    a_main.config = &cfg_main;
+    a = &a_main;
+    g_pdl = !cfg_main.serial_launches;
     ProfileMarks marks = profile_slot(a->config, s);
 #define MOK_MARK(i) marks.close((i) - 1)
     marks.open();
-    int rc = route_stage(a, L, ws, x, s);
+    int rc = MOK_OK;
+    SidePipe* side = nullptr;
+    mok_config cfg_side = cfg_main;
+    if (shared_beside_routed(&cfg_main, a->H, a->I, a->I_shared, L.R, a->E)) {
+        int dev = 0, sms = 0;
+        if ((e = current_device(&dev)) != cudaSuccess || (e = device_sm_count(dev, &sms)) != cudaSuccess) return cuda_fail(e);
+        if (sms >= 4 * SIDE_CTAS) {
+            if ((rc = side_pipe(&side))) return rc;
+            cfg_side.grid = cfg_main.grid > 0 && cfg_main.grid < SIDE_CTAS ? cfg_main.grid : SIDE_CTAS;
+            cfg_side.gang_sync = 1;                                 // (the gang counters belong to the routed kernels)
+            // (forced on a layer whose routed kernels fill the GPU: those then leave the side kernels their SMs)
+            if (cfg_main.grid == 0 && cfg_main.shared_overlap == 2) cfg_main.grid = sms - SIDE_CTAS;
+            if ((e = cudaEventRecord(side->fork, s)) != cudaSuccess) return cuda_fail(e);
+            if ((e = cudaStreamWaitEvent(side->stream, side->fork, 0)) != cudaSuccess) return cuda_fail(e);
+        }
+    }
+    rc = route_stage(a, L, ws, x, s);
     if (rc) return rc;
     MOK_MARK(MOK_STAGE_ROUTER + 1);
     const int tile_m = use_mx(a->config) ? TILE_M : tile_rows(a->config, a->I);
@@ -384,7 +450,7 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
     bool combine_in_launch = false;
     // shared expert: every token in natural order, no gather.  Runs after the routed experts, or before them when the
     // routed experts' launch ends with the combine
-    auto shared_expert = [&]() -> int {
+    auto shared_expert = [&](cudaStream_t ss, const mok_config* cs, bool mark) -> int {
         GemmArgs gs = g;
         gs.dbg_slot = dbg ? 3 : -1;
         gs.row_token = nullptr;
@@ -399,20 +465,25 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
             gs.C = ws + L.hs;
             gs.K = a->H; gs.N = a->I_shared; gs.ldc = a->I_shared; gs.E = 1; gs.rows_pad = L.Tpad; gs.a_rows = a->T;
             gs.dense_rows = a->T;
-            if ((rcs = run_gemm(gs, true, a->config, L, ws, s))) return rcs;
-            MOK_MARK(MOK_STAGE_SHARED_GEMM1 + 1);
+            if ((rcs = run_gemm(gs, true, cs, L, ws, ss))) return rcs;
+            if (mark) MOK_MARK(MOK_STAGE_SHARED_GEMM1 + 1);
             gs.A = reinterpret_cast<const __nv_bfloat16*>(ws + L.hs);
             gs.B = reinterpret_cast<const __nv_bfloat16*>(a->W_shared_down);
             gs.C = ws + L.ysh;
             gs.K = a->I_shared; gs.N = a->H; gs.ldc = a->H; gs.a_rows = L.Tpad;
-            if ((rcs = run_gemm(gs, false, a->config, L, ws, s))) return rcs;
-            MOK_MARK(MOK_STAGE_SHARED_GEMM2 + 1);
-        } else {
+            if ((rcs = run_gemm(gs, false, cs, L, ws, ss))) return rcs;
+            if (mark) MOK_MARK(MOK_STAGE_SHARED_GEMM2 + 1);
+        } else if (mark) {
             MOK_MARK(MOK_STAGE_SHARED_GEMM1 + 1);
             MOK_MARK(MOK_STAGE_SHARED_GEMM2 + 1);
         }
         return rcs;
     };
+    if (side) {
+        // the shared expert's two GEMMs on the side stream, now: they need x and the weights only
+        if ((rc = shared_expert(side->stream, &cfg_side, false))) return rc;
+        if ((e = cudaEventRecord(side->join, side->stream)) != cudaSuccess) return cuda_fail(e);
+    }
     if (mx) {
         // routed experts on MXFP8 operands (Section 3.4): h = Q(silu(Q(x) Wg_q^T) * (Q(x) Wu_q^T));  y = h Wd_q^T
         const int grid = a->config->grid;
@@ -474,7 +545,7 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
         if (L.h_ring > 0 && !fused) return MOK_ERR_UNSUPPORTED;     // the ring exists in the one-launch kernel only
         if (!fused && g.starve == 2) g.starve = 0;                  // (that hook only exists in the one-launch kernel)
         combine_in_launch = fused && a->config && a->config->fused_ffn == 3;
-        if (combine_in_launch && (rc = shared_expert())) return rc;       // its output is an input of that launch
+        if (combine_in_launch && (rc = shared_expert(s, a->config, true))) return rc;   // its output is an input of that launch
         // its hand-out: synchronised starts need the static stride (a CTA that draws ahead could hold two tiles of a gang)
         const bool fused_sync = fused_gang(a->config, a->H, a->I, L.R, a->E);
         const int sched = a->config ? a->config->tile_sched : 0;
@@ -502,7 +573,11 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
     }
     MOK_MARK(MOK_STAGE_GEMM2 + 1);
     if (!combine_in_launch) {
-        if ((rc = shared_expert())) return rc;
+        if (side) {
+            MOK_MARK(MOK_STAGE_SHARED_GEMM1 + 1);
+            MOK_MARK(MOK_STAGE_SHARED_GEMM2 + 1);
+            if ((e = cudaStreamWaitEvent(s, side->join, 0)) != cudaSuccess) return cuda_fail(e);
+        } else if ((rc = shared_expert(s, a->config, true))) return rc;
         e = launch_combine(L, ws, a->T, a->H, a->k, a->I_shared > 0, out, s);
         if (e != cudaSuccess) return cuda_fail(e);
     }

@@ -506,6 +506,25 @@ def test_completion_counter_waits_of_the_one_launch_kernel_run_out_cleanly(kw):
     assert torch.equal(good.view(torch.int16), again.view(torch.int16))
 
 
+@pytest.mark.parametrize("cfg", [inputs.CONFIGS["tiny"], MID[1]], ids=["tiny", "mid_many"])
+def test_shared_expert_beside_the_routed_experts_gives_the_same_bits(cfg):
+    """config.shared_overlap: the shared expert's GEMMs on a library-owned second stream, forked from and joined to the
+    caller's stream by events (the default for small layers), against the same GEMMs in line: every token against the
+    oracle, the same bits with either order, with the one-launch expert FFN, small grids, and several calls in a row on
+    one workspace (the fork of a call waits for the previous call's combine)."""
+    m = mok()
+    d = inputs.make_inputs(cfg)
+    g = pu.upload(d)
+    inline, st, rep = pu.full_parity(cfg, d=d, g=g, config=m._config(shared_overlap=1))
+    print(cfg.name, rep)
+    ws = m.alloc_workspace(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k)
+    for kw in ({}, {"shared_overlap": 2}, {"shared_overlap": 2, "fused_ffn": 2}, {"shared_overlap": 2, "grid": 3},
+               {"shared_overlap": 2, "cta_group": 1}, {"shared_overlap": 2, "cta_group": 3, "gang_sync": 2}):
+        for _ in range(3):
+            out = pu.run_gpu(cfg, g, ws=ws, config=m._config(**kw), stages=False)
+            assert torch.equal(out.view(torch.int16), inline.view(torch.int16)), kw
+
+
 def test_forward_can_be_captured_in_a_cuda_graph_and_replayed():
     """The layer makes no host synchronisation and no allocation after its first call for a shape, so a whole
     forward can be recorded once into a CUDA graph and replayed (launch-bound small batches): same bits."""
