@@ -136,7 +136,9 @@ typedef struct mok_config {
                              before the combine; the routed kernels then take the other SMs); 1 = in line, after the
                              routed experts; 0 = beside them for small layers only (at most 160 routed rows per expert
                              and 64 MB of expert weights), whose kernels are bound by launch and fill latency rather
-                             than by DRAM or the tensor cores (Section 3.4 "Shared Expert").  Same bits. */
+                             than by DRAM or the tensor cores (Section 3.4 "Shared Expert").  Same bits.  The second
+                             stream and its two events exist once per device: host threads that call the library
+                             concurrently on one device must set 1. */
 } mok_config;
 #define MOK_H_RING_MIN_TILES 24
 
