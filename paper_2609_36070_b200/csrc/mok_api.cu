@@ -365,6 +365,41 @@ static bool shared_beside_routed(const mok_config* cfg, int H, int I, int I_shar
     return rows <= 160ll * experts && 6ll * experts * H * I <= (64ll << 20);
 }
 
+// The shared expert's two GEMMs (every token in natural order, no gather) on stream ss with the knobs cs.
+static int shared_expert_gemms(const mok_args* a, const WsLayout& L, char* ws, WsHeader* hdr, const __nv_bfloat16* x,
+                               int tile_m, bool dbg, const mok_config* cs, cudaStream_t ss, ProfileMarks* marks) {
+    if (a->I_shared <= 0) {
+        if (marks) { marks->close(MOK_STAGE_SHARED_GEMM1); marks->close(MOK_STAGE_SHARED_GEMM2); }
+        return MOK_OK;
+    }
+    GemmArgs gs;
+    memset(&gs, 0, sizeof(gs));
+    gs.header = hdr;
+    gs.n_mtiles = &hdr->n_mtiles;          // (dense mode derives its tiles from dense_rows: the schedule's tables are not read)
+    gs.tile_expert = reinterpret_cast<const int32_t*>(ws + L.tile_expert);
+    gs.mt_start = reinterpret_cast<const int32_t*>(ws + L.mt_start);
+    gs.max_mt = L.max_mt;
+    gs.tile_m = tile_m;
+    gs.pad_offsets = reinterpret_cast<const int32_t*>(ws + L.pad_offsets);
+    gs.counts = reinterpret_cast<const int32_t*>(ws + L.counts);
+    gs.dbg_slot = dbg ? 3 : -1;
+    gs.A = x;
+    gs.B = reinterpret_cast<const __nv_bfloat16*>(a->W_shared_gate_up);
+    gs.C = ws + L.hs;
+    gs.K = a->H; gs.N = a->I_shared; gs.ldc = a->I_shared; gs.E = 1; gs.rows_pad = L.Tpad; gs.a_rows = a->T;
+    gs.dense_rows = a->T;
+    int rc = run_gemm(gs, true, cs, L, ws, ss);
+    if (rc) return rc;
+    if (marks) marks->close(MOK_STAGE_SHARED_GEMM1);
+    gs.A = reinterpret_cast<const __nv_bfloat16*>(ws + L.hs);
+    gs.B = reinterpret_cast<const __nv_bfloat16*>(a->W_shared_down);
+    gs.C = ws + L.ysh;
+    gs.K = a->I_shared; gs.N = a->H; gs.ldc = a->H; gs.a_rows = L.Tpad;
+    if ((rc = run_gemm(gs, false, cs, L, ws, ss))) return rc;
+    if (marks) marks->close(MOK_STAGE_SHARED_GEMM2);
+    return MOK_OK;
+}
+
 // The whole layer on device pointers.  x / out may differ from a->x / a->out (host-buffer variant).
 static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloat16* x, __nv_bfloat16* out,
                           bool reset_header = true) {
@@ -386,6 +421,7 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
 #define MOK_MARK(i) marks.close((i) - 1)
     marks.open();
     int rc = MOK_OK;
+    const int tile_m = use_mx(a->config) ? TILE_M : tile_rows(a->config, a->I);
     SidePipe* side = nullptr;
     mok_config cfg_side = cfg_main;
     if (shared_beside_routed(&cfg_main, a->H, a->I, a->I_shared, L.R, a->E)) {
@@ -395,16 +431,21 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
             if ((rc = side_pipe(&side))) return rc;
             cfg_side.grid = cfg_main.grid > 0 && cfg_main.grid < SIDE_CTAS ? cfg_main.grid : SIDE_CTAS;
             cfg_side.gang_sync = 1;                                 // (the gang counters belong to the routed kernels)
-            // (forced on a layer whose routed kernels fill the GPU: those then leave the side kernels their SMs)
-            if (cfg_main.grid == 0 && cfg_main.shared_overlap == 2) cfg_main.grid = sms - SIDE_CTAS;
+            // The persistent kernels of the caller's stream leave the side kernels their SMs: every GEMM CTA takes a
+            // whole SM, and with programmatic launches the routed GEMM's CTAs become resident (and wait) while router
+            // and schedule still run -- a full grid of them would keep the side kernels off the GPU until it is done.
+            if (cfg_main.grid == 0) cfg_main.grid = sms - SIDE_CTAS;
             if ((e = cudaEventRecord(side->fork, s)) != cudaSuccess) return cuda_fail(e);
             if ((e = cudaStreamWaitEvent(side->stream, side->fork, 0)) != cudaSuccess) return cuda_fail(e);
+            // its two GEMMs need x and the weights only: enqueued first, so that they are on the GPU first
+            if ((rc = shared_expert_gemms(a, L, ws, hdr, x, tile_m, cfg_main.debug == 1, &cfg_side, side->stream, nullptr)))
+                return rc;
+            if ((e = cudaEventRecord(side->join, side->stream)) != cudaSuccess) return cuda_fail(e);
         }
     }
     rc = route_stage(a, L, ws, x, s);
     if (rc) return rc;
     MOK_MARK(MOK_STAGE_ROUTER + 1);
-    const int tile_m = use_mx(a->config) ? TILE_M : tile_rows(a->config, a->I);
     const int pad_m = use_tn(a->config) ? 16 : tile_m;   // tokens on the MMA's N side need 16-row granularity only
     e = launch_schedule(reinterpret_cast<const int32_t*>(ws + L.idx), a->T, a->E, a->k, tile_m, pad_m, L, ws,
                         a->counts, a->offsets, a->perm, a->inv_perm, s);
@@ -448,42 +489,6 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
         g.starve = a->config->debug == MOK_DEBUG_STARVE ? 1 : 2;
     }
     bool combine_in_launch = false;
-    // shared expert: every token in natural order, no gather.  Runs after the routed experts, or before them when the
-    // routed experts' launch ends with the combine
-    auto shared_expert = [&](cudaStream_t ss, const mok_config* cs, bool mark) -> int {
-        GemmArgs gs = g;
-        gs.dbg_slot = dbg ? 3 : -1;
-        gs.row_token = nullptr;
-        gs.starve = 0;
-        gs.tile_sched = 0;
-        gs.sfa = gs.sfb = nullptr;
-        gs.sfc = nullptr;
-        int rcs = MOK_OK;
-        if (a->I_shared > 0) {
-            gs.A = x;
-            gs.B = reinterpret_cast<const __nv_bfloat16*>(a->W_shared_gate_up);
-            gs.C = ws + L.hs;
-            gs.K = a->H; gs.N = a->I_shared; gs.ldc = a->I_shared; gs.E = 1; gs.rows_pad = L.Tpad; gs.a_rows = a->T;
-            gs.dense_rows = a->T;
-            if ((rcs = run_gemm(gs, true, cs, L, ws, ss))) return rcs;
-            if (mark) MOK_MARK(MOK_STAGE_SHARED_GEMM1 + 1);
-            gs.A = reinterpret_cast<const __nv_bfloat16*>(ws + L.hs);
-            gs.B = reinterpret_cast<const __nv_bfloat16*>(a->W_shared_down);
-            gs.C = ws + L.ysh;
-            gs.K = a->I_shared; gs.N = a->H; gs.ldc = a->H; gs.a_rows = L.Tpad;
-            if ((rcs = run_gemm(gs, false, cs, L, ws, ss))) return rcs;
-            if (mark) MOK_MARK(MOK_STAGE_SHARED_GEMM2 + 1);
-        } else if (mark) {
-            MOK_MARK(MOK_STAGE_SHARED_GEMM1 + 1);
-            MOK_MARK(MOK_STAGE_SHARED_GEMM2 + 1);
-        }
-        return rcs;
-    };
-    if (side) {
-        // the shared expert's two GEMMs on the side stream, now: they need x and the weights only
-        if ((rc = shared_expert(side->stream, &cfg_side, false))) return rc;
-        if ((e = cudaEventRecord(side->join, side->stream)) != cudaSuccess) return cuda_fail(e);
-    }
     if (mx) {
         // routed experts on MXFP8 operands (Section 3.4): h = Q(silu(Q(x) Wg_q^T) * (Q(x) Wu_q^T));  y = h Wd_q^T
         const int grid = a->config->grid;
@@ -545,7 +550,8 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
         if (L.h_ring > 0 && !fused) return MOK_ERR_UNSUPPORTED;     // the ring exists in the one-launch kernel only
         if (!fused && g.starve == 2) g.starve = 0;                  // (that hook only exists in the one-launch kernel)
         combine_in_launch = fused && a->config && a->config->fused_ffn == 3;
-        if (combine_in_launch && (rc = shared_expert(s, a->config, true))) return rc;   // its output is an input of that launch
+        // (the shared expert's output is an input of that launch: it then runs first)
+        if (combine_in_launch && (rc = shared_expert_gemms(a, L, ws, hdr, x, tile_m, dbg, a->config, s, &marks))) return rc;
         // its hand-out: synchronised starts need the static stride (a CTA that draws ahead could hold two tiles of a gang)
         const bool fused_sync = fused_gang(a->config, a->H, a->I, L.R, a->E);
         const int sched = a->config ? a->config->tile_sched : 0;
@@ -577,7 +583,7 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
             MOK_MARK(MOK_STAGE_SHARED_GEMM1 + 1);
             MOK_MARK(MOK_STAGE_SHARED_GEMM2 + 1);
             if ((e = cudaStreamWaitEvent(s, side->join, 0)) != cudaSuccess) return cuda_fail(e);
-        } else if ((rc = shared_expert(s, a->config, true))) return rc;
+        } else if ((rc = shared_expert_gemms(a, L, ws, hdr, x, tile_m, dbg, a->config, s, &marks))) return rc;
         e = launch_combine(L, ws, a->T, a->H, a->k, a->I_shared > 0, out, s);
         if (e != cudaSuccess) return cuda_fail(e);
     }
@@ -950,7 +956,7 @@ int mok_debug_counters(const void* workspace, void* stream, unsigned long long* 
 int mok_launch_count(int T, int H, int I, int I_shared, int E, int k, const mok_config* config) {
     WsLayout L;
     if (!ws_layout(T, H, I, I_shared, E, k, &L) || T == 0) return 0;
-    // router (1 fp32-FMA kernel, or split + GEMM + top-k + near-tie fix-up), 3 schedule kernels, (gather on the SIMT path),
+    // router (1 fp32-FMA kernel, or split + GEMM + top-k + near-tie fix-up), 3 schedule kernels (1 up to 2048 routes), (gather on the SIMT path),
     // 2 routed GEMMs, (2 shared GEMMs), combine
     // (MXFP8 mode: the token-row quantiser instead of the gather kernel; its two memsets are not counted)
     const int pre = use_mx(config) ? 1 : (fused_gather(config, I) ? 0 : 1);
@@ -959,7 +965,8 @@ int mok_launch_count(int T, int H, int I, int I_shared, int E, int k, const mok_
     //  with config.fused_ffn = 3 that kernel also does the combine: one launch less)
     const int tile_m = use_mx(config) ? TILE_M : tile_rows(config, I);
     const int combine = config && config->fused_ffn == 3 && use_fused_ffn(config, H, I, tile_m, L.R, E, L.max_ftiles) ? 0 : 1;
-    return (use_simt_router(config, k) ? 1 : use_fused_router(config, E, k) ? 3 : 4) + 3 + pre + 2 + (I_shared > 0 ? 2 : 0) + combine;
+    const int sched = (long long)T * k <= SCHED_CHUNK ? 1 : 3;       // small batches: the schedule is one block
+    return (use_simt_router(config, k) ? 1 : use_fused_router(config, E, k) ? 3 : 4) + sched + pre + 2 + (I_shared > 0 ? 2 : 0) + combine;
 }
 
 int mok_profile_begin(int max_calls) {
