@@ -259,11 +259,19 @@ bool ep_layout(int n_ranks, int T_local, int H, int I, int Is, int E, int k, WsL
     L->row_token = take(sizeof(int32_t) * (size_t)Rpad);
     L->h = take(2 * (size_t)Rpad * I);
     L->hs = take(Is > 0 ? 2 * (size_t)L->Tpad * Is : 0);
+    if (!mx) {   // one-launch expert FFN: its tile list and the two completion counters per 256-row tile
+        const long long mt2 = Rpad / (2 * TILE_M), per = (I + 127) / 128 + (H + 255) / 256;
+        const long long nt = mt2 * per;
+        L->max_ftiles = nt < (1ll << 30) ? (int32_t)nt : 0;
+        L->ftiles = take(sizeof(int4) * (size_t)L->max_ftiles);
+        L->ready = take(2 * sizeof(int32_t) * (size_t)mt2);
+    }
     {   // gang-start counters of the 256-row kernel: one per tile of the largest of the four GEMMs
         const long long mt2 = Rpad / (2 * TILE_M), mts = L->Tpad / (2 * TILE_M);
         const long long n_r = (I + 127) / 128 > (H + 255) / 256 ? (I + 127) / 128 : (H + 255) / 256;
         const long long n_s = (Is + 127) / 128 > (H + 255) / 256 ? (Is + 127) / 128 : (H + 255) / 256;
-        const long long tiles = mt2 * n_r > mts * n_s ? mt2 * n_r : mts * n_s;
+        long long tiles = mt2 * n_r > mts * n_s ? mt2 * n_r : mts * n_s;
+        if (L->max_ftiles > tiles) tiles = L->max_ftiles;       // the one-launch FFN's list (static hand-out)
         L->gang_bytes = sizeof(int32_t) * (size_t)tiles;
         L->gang = take(L->gang_bytes);
     }
@@ -354,7 +362,11 @@ int mok_ep_expert_ffn(const mok_ep_args* a) {
 
     mok_config cfg;
     memset(&cfg, 0, sizeof(cfg));
-    if (a->config) { cfg.grid = a->config->grid; cfg.cta_group = a->config->cta_group; cfg.gang_sync = a->config->gang_sync; }
+    if (a->config) {
+        cfg.grid = a->config->grid; cfg.cta_group = a->config->cta_group; cfg.gang_sync = a->config->gang_sync;
+        cfg.fused_ffn = a->config->fused_ffn == 3 ? 2 : a->config->fused_ffn;     // (the combine is the owners' call here)
+        cfg.fused_window = a->config->fused_window; cfg.tile_sched = a->config->tile_sched;
+    }
     const __nv_bfloat16* x_own = reinterpret_cast<const __nv_bfloat16*>(a->x_peers[a->rank]);   // (may be NULL in MXFP8 mode without a shared expert)
     GemmArgs g;
     memset(&g, 0, sizeof(g));
@@ -415,15 +427,30 @@ int mok_ep_expert_ffn(const mok_ep_args* a) {
         g.C = ws + L.h;
         g.K = a->H; g.N = a->I; g.ldc = a->I; g.E = Lx; g.rows_pad = L.Rpad; g.dense_rows = 0;
         g.total_rows = n;   // expected share of this rank, for the kernel choice
-        if ((rc = run_gemm(g, true, &cfg, L, ws, s))) return rc;
+        // the routed experts as ONE persistent launch where the one-rank layer would choose it (large expert matrices),
+        // or on request: the same kernel, its gather warps pulling from the owners' buffers, its down tiles storing
+        // into the peer-visible y
+        bool fused_sync = false;
+        const bool fused = fused_ffn_choice(&cfg, a->H, a->I, TILE_M, n, Lx, L.max_ftiles, &fused_sync);
+        if (fused) {
+            const bool dynamic = cfg.tile_sched == 1 || (cfg.tile_sched == 0 && !fused_sync);
+            e = launch_fused_ffn(x_own, a->T_local, a->H, a->I, Lx, reinterpret_cast<const __nv_bfloat16*>(a->W_gate_up),
+                                 reinterpret_cast<const __nv_bfloat16*>(a->W_down), L, ws, cfg.grid, cfg.fused_window, dynamic,
+                                 fused_sync, false, 0, s, nullptr, 0, false, 0, a->x_peers, a->T_local, a->y);
+            if (e != cudaSuccess) return cuda_fail(e);
+        } else {
+            if ((rc = run_gemm(g, true, &cfg, L, ws, s))) return rc;
+            g.row_token = nullptr;
+            g.peer_tokens = 0;
+            g.a_rows = L.Rpad;
+            g.A = reinterpret_cast<const __nv_bfloat16*>(ws + L.h);
+            g.B = reinterpret_cast<const __nv_bfloat16*>(a->W_down);
+            g.C = a->y;
+            g.K = a->I; g.N = a->H; g.ldc = a->H;
+            if ((rc = run_gemm(g, false, &cfg, L, ws, s))) return rc;
+        }
         g.row_token = nullptr;
         g.peer_tokens = 0;
-        g.a_rows = L.Rpad;
-        g.A = reinterpret_cast<const __nv_bfloat16*>(ws + L.h);
-        g.B = reinterpret_cast<const __nv_bfloat16*>(a->W_down);
-        g.C = a->y;
-        g.K = a->I; g.N = a->H; g.ldc = a->H;
-        if ((rc = run_gemm(g, false, &cfg, L, ws, s))) return rc;
     }
     if (a->I_shared > 0) {   // shared expert on the rank's own tokens, natural order
         g.A = x_own;

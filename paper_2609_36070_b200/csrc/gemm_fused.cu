@@ -56,6 +56,7 @@
 #include "mok_internal.cuh"
 #include "tc_ptx.cuh"
 #include "tensor_map.cuh"
+#include <string.h>
 
 namespace mok {
 namespace ff {
@@ -324,6 +325,10 @@ fused_tiles_kernel(const int32_t* __restrict__ counts, const int32_t* __restrict
 
 struct FusedArgs {
     const __nv_bfloat16* x;        // [T, H] token rows (gathered through row_token)
+    // expert parallelism (Section 3.1, pull dispatch): with peer_tokens > 0 the ids in row_token are global,
+    // id = source rank * peer_tokens + token, and the row is read from that rank's buffer with plain peer loads
+    int32_t peer_tokens;
+    const __nv_bfloat16* peer_x[MOK_MAX_RANKS];
     const int32_t* row_token;      // padded row -> token
     const int4* tiles;             // the tile list
     const int32_t* n_tiles;        // device: its length
@@ -786,7 +791,12 @@ fused_ffn_kernel(const __grid_constant__ CUtensorMap mapWgu, const __grid_consta
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
                 const int r = (i >> 3) * BM + gw * 32 + (i & 7) * 4 + sub;
-                src[i] = a.x + (size_t)tok[i] * a.H + chunk * 8;
+                if (a.peer_tokens > 0) {
+                    const int pr = tok[i] / a.peer_tokens;
+                    src[i] = a.peer_x[pr] + (size_t)(tok[i] - pr * a.peer_tokens) * a.H + chunk * 8;
+                } else {
+                    src[i] = a.x + (size_t)tok[i] * a.H + chunk * 8;
+                }
                 if (r < t.valid) live |= 1u << i;
             }
             for (int kb = 0; kb < a.kb1; ++kb) {
@@ -1002,7 +1012,7 @@ static cudaError_t launch_kernel(int grid, cudaStream_t s, const CUtensorMap& m0
 cudaError_t launch_fused_ffn(const __nv_bfloat16* x, int T, int H, int I, int E, const __nv_bfloat16* Wgu,
                              const __nv_bfloat16* Wd, const WsLayout& L, char* ws, int grid, int window_tiles, bool dynamic,
                              bool gang_sync, bool dbg, int starve, cudaStream_t s, __nv_bfloat16* combine_out, int k,
-                             bool shared, int h_ring_tiles) {
+                             bool shared, int h_ring_tiles, const void* const* peer_x, int peer_tokens, void* y_out) {
     using namespace ff;
     int dev = 0, sm_count = 0;
     cudaError_t e = current_device(&dev);
@@ -1034,7 +1044,7 @@ cudaError_t launch_fused_ffn(const __nv_bfloat16* x, int T, int H, int I, int E,
 
     CUtensorMap mWgu, mWgu64, mHst, mHld, mWd, mY;
     void* h = ws + L.h;
-    void* y = ws + L.y;
+    void* y = y_out ? y_out : ws + L.y;
     if (!tmap::bf16_sw128(&mWgu, Wgu, (uint64_t)E * 2 * I, (uint64_t)H, BN / 2) ||
         !tmap::bf16_sw128(&mWgu64, Wgu, (uint64_t)E * 2 * I, (uint64_t)H, BN / 4) ||
         !tmap::bf16_sw128(&mHst, h, (uint64_t)(ring ? ring * TM : L.Rpad), (uint64_t)I, 32) ||
@@ -1043,7 +1053,10 @@ cudaError_t launch_fused_ffn(const __nv_bfloat16* x, int T, int H, int I, int E,
         !tmap::bf16_sw128(&mY, y, (uint64_t)L.Rpad, (uint64_t)H, 32))
         return cudaErrorInvalidValue;
     FusedArgs a;
+    memset(&a, 0, sizeof(a));
     a.x = x;
+    a.peer_tokens = peer_x ? peer_tokens : 0;
+    for (int r = 0; peer_x && r < MOK_MAX_RANKS; ++r) a.peer_x[r] = reinterpret_cast<const __nv_bfloat16*>(peer_x[r]);
     a.row_token = reinterpret_cast<const int32_t*>(ws + L.row_token);
     a.tiles = tiles;
     a.n_tiles = &hdr->n_ftiles;

@@ -280,6 +280,11 @@ int gang_prepare(GemmArgs& g, bool swiglu, const mok_config* cfg, const WsLayout
     return MOK_OK;
 }
 
+bool fused_ffn_choice(const mok_config* cfg, int H, int I, int tile_m, long long rows, int experts, int max_ftiles, bool* sync) {
+    if (sync) *sync = fused_gang(cfg, H, I, rows, experts);
+    return use_fused_ffn(cfg, H, I, tile_m, rows, experts, max_ftiles);
+}
+
 int run_gemm(GemmArgs g, bool swiglu, const mok_config* cfg, const WsLayout& L, char* ws, cudaStream_t s) {
     const int epi = swiglu ? EPI_SWIGLU : EPI_BF16, grid = cfg ? cfg->grid : 0;
     if (use_m2(cfg, g.K, g.tile_m, g.dense_rows > 0 ? g.dense_rows : g.total_rows, g.dense_rows > 0 ? 1 : g.E)) {

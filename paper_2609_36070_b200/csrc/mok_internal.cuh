@@ -159,7 +159,11 @@ cudaError_t launch_fused_ffn(const __nv_bfloat16* x, int T, int H, int I, int E,
                              const __nv_bfloat16* Wd, const WsLayout& L, char* ws, int grid, int window_tiles, bool dynamic,
                              bool gang_sync, bool dbg, int starve, cudaStream_t s, __nv_bfloat16* combine_out = nullptr,
                              int k = 0, bool shared = false,    // combine_out != NULL: the combine runs in the same launch
-                             int h_ring_tiles = 0);             // > 0: h is a ring of that many 256-row tiles
+                             int h_ring_tiles = 0,              // > 0: h is a ring of that many 256-row tiles
+                             const void* const* peer_x = nullptr, int peer_tokens = 0,   // expert parallelism: every rank's token rows
+                             void* y_out = nullptr);            // where the down tiles go (NULL: the workspace's y)
+// whether the routed expert FFN runs as the one launch for these sizes and knobs; *sync: with synchronised tile starts
+bool fused_ffn_choice(const mok_config* cfg, int H, int I, int tile_m, long long rows, int experts, int max_ftiles, bool* sync);
 constexpr int H_RING_MIN_TILES = 24;     // smallest ring of the gated activation (see gemm_fused.cu)
 cudaError_t launch_mx_quantize_rows(const __nv_bfloat16* in, long long rows, int K, uint8_t* codes, uint8_t* scales,
                                     cudaStream_t s);

@@ -108,6 +108,19 @@ def test_expert_parallel_layer_shapes(name, T, H, E, k, I, I_s, bias, R):
     assert rep["bitwise_equal_to_one_rank"], rep
 
 
+@pytest.mark.parametrize("R", [1, 2, 4])
+@pytest.mark.parametrize("kw", [{"fused_ffn": 2}, {"fused_ffn": 2, "tile_sched": 2, "gang_sync": 2},
+                                {"fused_ffn": 2, "fused_window": -1, "grid": 7}], ids=["dynamic", "static_gang", "no_window"])
+def test_expert_parallel_layer_with_the_one_launch_expert_ffn(R, kw):
+    """The routed experts of every rank as ONE persistent launch (gate/up tiles pull their rows from the owners'
+    buffers, down tiles wait on the completion counters and store into the peer-visible y): every token against the
+    oracle and bit for bit the one-rank layer, on a shape with several row tiles per expert and a shared expert."""
+    m = mok()
+    cfg = inputs.MoEConfig("ep_one_launch", 3072, 512, 8, 3, 320, 128, bias="zipf", seed=12)
+    rep = ep_case(cfg, R, config=m._config(**kw))
+    assert rep["bitwise_equal_to_one_rank"], rep
+
+
 def test_expert_parallel_is_reproducible_and_independent_of_the_kernel_choice():
     cfg = inputs.MoEConfig("ep_repro", 1024, 512, 16, 4, 512, 0, bias="zipf", seed=5)
     m = mok()
