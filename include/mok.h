@@ -139,6 +139,15 @@ typedef struct mok_config {
                              than by DRAM or the tensor cores (Section 3.4 "Shared Expert").  Same bits.  The second
                              stream and its two events exist once per device: host threads that call the library
                              concurrently on one device must set 1. */
+    int32_t comm_ctas;    /* one-launch expert FFN (used whatever fused_ffn says; MOK_ERR_UNSUPPORTED where it cannot run, or
+                             with h_ring_tiles): that many CTAs of the grid are COMMUNICATION CTAs (Section 3.4
+                             "Computation-Communication SM Tuning"): they do no tiles but copy the token rows of one row
+                             tile after the other -- from x, under expert parallelism from the owners' buffers -- into
+                             a ring of 24 staging slots, from which the gate/up tiles then load their A operand by
+                             TMA; completion counters (bounded waits) order staging, use and reuse of a slot.  The
+                             latency of a pull is then taken by CTAs that do nothing else, a row tile ahead of its
+                             use, instead of by the gather warps of the computing CTAs.  0 = none: the gather warps
+                             pull.  Same bits. */
 } mok_config;
 #define MOK_H_RING_MIN_TILES 24
 

@@ -264,7 +264,8 @@ bool ep_layout(int n_ranks, int T_local, int H, int I, int Is, int E, int k, WsL
         const long long nt = mt2 * per;
         L->max_ftiles = nt < (1ll << 30) ? (int32_t)nt : 0;
         L->ftiles = take(sizeof(int4) * (size_t)L->max_ftiles);
-        L->ready = take(2 * sizeof(int32_t) * (size_t)mt2);
+        L->ready = take(4 * sizeof(int32_t) * (size_t)mt2);    // ready, consumed, staged, released
+        L->xg = take(2 * (size_t)FFN_COMM_SLOTS * 2 * TILE_M * H);    // staging slots of the communication CTAs
     }
     {   // gang-start counters of the 256-row kernel: one per tile of the largest of the four GEMMs
         const long long mt2 = Rpad / (2 * TILE_M), mts = L->Tpad / (2 * TILE_M);
@@ -317,7 +318,8 @@ int mok_ep_expert_ffn(const mok_ep_args* a) {
     if ((a->I_shared > 0) != (a->W_shared_gate_up != nullptr) || (a->I_shared > 0) != (a->W_shared_down != nullptr))
         return MOK_ERR_SHAPE;
     if (a->config && (a->config->impl != MOK_IMPL_TCGEN05 || a->config->grid < 0 ||
-                      (a->config->cta_group != 0 && a->config->cta_group != 1 && a->config->cta_group != 3)))
+                      (a->config->cta_group != 0 && a->config->cta_group != 1 && a->config->cta_group != 3) ||
+                      a->config->comm_ctas < 0))
         return MOK_ERR_SHAPE;
     if (a->T_local == 0) return MOK_OK;
     if (!a->idx_all || !a->pos) return MOK_ERR_NULL;
@@ -366,6 +368,7 @@ int mok_ep_expert_ffn(const mok_ep_args* a) {
         cfg.grid = a->config->grid; cfg.cta_group = a->config->cta_group; cfg.gang_sync = a->config->gang_sync;
         cfg.fused_ffn = a->config->fused_ffn == 3 ? 2 : a->config->fused_ffn;     // (the combine is the owners' call here)
         cfg.fused_window = a->config->fused_window; cfg.tile_sched = a->config->tile_sched;
+        cfg.comm_ctas = a->config->comm_ctas;
     }
     const __nv_bfloat16* x_own = reinterpret_cast<const __nv_bfloat16*>(a->x_peers[a->rank]);   // (may be NULL in MXFP8 mode without a shared expert)
     GemmArgs g;
@@ -432,11 +435,13 @@ int mok_ep_expert_ffn(const mok_ep_args* a) {
         // into the peer-visible y
         bool fused_sync = false;
         const bool fused = fused_ffn_choice(&cfg, a->H, a->I, TILE_M, n, Lx, L.max_ftiles, &fused_sync);
+        if (cfg.comm_ctas > 0 && !fused) return MOK_ERR_UNSUPPORTED;     // communication CTAs exist in that kernel only
         if (fused) {
             const bool dynamic = cfg.tile_sched == 1 || (cfg.tile_sched == 0 && !fused_sync);
             e = launch_fused_ffn(x_own, a->T_local, a->H, a->I, Lx, reinterpret_cast<const __nv_bfloat16*>(a->W_gate_up),
                                  reinterpret_cast<const __nv_bfloat16*>(a->W_down), L, ws, cfg.grid, cfg.fused_window, dynamic,
-                                 fused_sync, false, 0, s, nullptr, 0, false, 0, a->x_peers, a->T_local, a->y);
+                                 fused_sync, false, 0, s, nullptr, 0, false, 0, a->x_peers, a->T_local, a->y, cfg.comm_ctas,
+                                 cfg.comm_ctas > 0 ? ws + L.xg : nullptr);
             if (e != cudaSuccess) return cuda_fail(e);
         } else {
             if ((rc = run_gemm(g, true, &cfg, L, ws, s))) return rc;

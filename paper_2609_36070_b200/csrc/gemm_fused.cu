@@ -48,6 +48,18 @@
 // mt - ring sits at a smaller list position than every gate/up tile of row tile mt, so the argument above still holds.
 // With the static window of two grids' worth of tiles the slots are rewritten while still in L2.
 //
+// Optionally some CTAs of the grid are COMMUNICATION CTAs (Section 3.4 "Computation-Communication SM Tuning"; Figure 1:
+// dedicated SMs pull the tokens while the others compute).  They do no tiles: for row tile after row tile, in list
+// order, they copy the tile's token rows (from x, or under expert parallelism from the owners' buffers) into one of
+// COMM_SLOTS 256-row slots of a staging buffer and add an arrival to staged[mt]; the gate/up tiles of that row tile
+// then take their A operand from the slot by TMA (the gather warps idle, as for down tiles) once staged[mt] is set, and
+// the MMA issuer adds an arrival to released[mt] when a gate/up tile's loads have landed, which is what a communication
+// CTA waits for (all n1 of them) before it reuses the slot for row tile mt + COMM_SLOTS.  So the latency of a pull --
+// microseconds over NVLink -- is taken by CTAs that do nothing else, a whole row tile ahead of its use, instead of by
+// gather warps that feed a three-stage ring.  No deadlock: communication CTAs walk the row tiles in increasing order,
+// every gate/up tile of row tile mt - COMM_SLOTS has a smaller list position than any of row tile mt (COMM_SLOTS >=
+// 2 * GROUP_TILES), the launch is cooperative; the unfinished item with the smallest position can always proceed.
+//
 // Optionally the COMBINE (Section 2.1: out[t] = shared[t] + sum_s w[t,s] * y[pos[t,s]]) runs in the same launch: a token's
 // k rows lie anywhere in y, so it can only start when every down tile has been stored.  Every epilogue warp adds one
 // arrival to a grid-wide counter once its last store has completed, waits (bounded) until all epilogue warps of the grid
@@ -74,9 +86,12 @@ constexpr int GATHER_THREADS = 128;
 constexpr int THREADS = 128 + 32 * EPI_WARPS + GATHER_THREADS;    // 512: four groups of four warps (see the kernel)
 constexpr int GROUP_TILES = 8;
 constexpr int SLAB_BYTES = 4096;
-constexpr int SMEM_CTRL = 256;
+constexpr int SMEM_CTRL = 512;
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_WARPS * SLAB_BYTES + SMEM_CTRL + 1024;
 constexpr int QSLOTS = 4;                       // tile ids drawn ahead by the scheduler warp (dynamic mode)
+constexpr int COMM_SLOTS = FFN_COMM_SLOTS;      // 256-row slots of the staging buffer of the communication CTAs
+constexpr int COMM_ISSUERS = 4, COMM_BUFS = 3, COMM_PIECE = 16384;   // its copy pipelines: 4 threads x 3 buffers of 16 KB
+static_assert(COMM_SLOTS >= 2 * GROUP_TILES, "a slot must not be reused inside the row group that still needs it");
 constexpr int ROLE_READERS = 2 + EPI_WARPS + GATHER_THREADS / 32;      // one arrival per role warp and queue entry
 
 struct Ctrl {
@@ -86,6 +101,7 @@ struct Ctrl {
     int32_t q_tile[QSLOTS];
     uint32_t tmem_base, abort;
     uint32_t combine_go;                 // in-launch combine: the grid has finished its tiles (written by the CTA's poller)
+    uint64_t cbar[COMM_ISSUERS * COMM_BUFS];   // communication CTA: one barrier per staging buffer of its copy pipelines
 };
 static_assert(sizeof(Ctrl) <= SMEM_CTRL, "control block too large");
 
@@ -137,14 +153,14 @@ struct TileSeq {
     Ctrl* ctrl;
     volatile uint32_t* abort_flag;
     WsHeader* hdr;
-    int total, slot;
+    int total, slot, stride;
     uint32_t ph;
     bool warp_role;       // all 32 lanes call next() together / one lane calls it
-    __device__ __forceinline__ TileSeq(Ctrl* c, volatile uint32_t* af, WsHeader* h, int tot, bool wr)
-        : ctrl(c), abort_flag(af), hdr(h), total(tot), slot(0), ph(0), warp_role(wr) {}
+    __device__ __forceinline__ TileSeq(Ctrl* c, volatile uint32_t* af, WsHeader* h, int tot, bool wr, int str)
+        : ctrl(c), abort_flag(af), hdr(h), total(tot), slot(0), stride(str), ph(0), warp_role(wr) {}
     __device__ __forceinline__ int first() { return DYN ? next(0) : (int)blockIdx.x; }
     __device__ __forceinline__ int next(int L) {
-        if (!DYN) return L + gridDim.x;
+        if (!DYN) return L + stride;             // (the compute CTAs of the grid: communication CTAs take no tiles)
         bool ok = wait_bar(smem_u32(&ctrl->q_full[slot]), ph, abort_flag, hdr, 30);
         if (warp_role) ok = __all_sync(0xffffffffu, ok);
         if (!ok) return total;
@@ -165,8 +181,8 @@ struct TileWalk {
     int total, L, Ln;
     int4 d, dn;
     __device__ __forceinline__ int4 fetch(int l) const { return l < total ? __ldg(tiles + l) : make_int4(0, 0, 0, 0); }
-    __device__ __forceinline__ TileWalk(Ctrl* c, volatile uint32_t* af, WsHeader* h, const int4* tl, int tot, bool wr)
-        : seq(c, af, h, tot, wr), tiles(tl), total(tot) {
+    __device__ __forceinline__ TileWalk(Ctrl* c, volatile uint32_t* af, WsHeader* h, const int4* tl, int tot, bool wr, int str)
+        : seq(c, af, h, tot, wr, str), tiles(tl), total(tot) {
         L = seq.first();
         d = fetch(L);
         Ln = L < total ? seq.next(L) : total;
@@ -200,7 +216,7 @@ __global__ void __launch_bounds__(MAX_E)
 fused_tiles_kernel(const int32_t* __restrict__ counts, const int32_t* __restrict__ pad_offsets,
                    const int32_t* __restrict__ mt_start2, int E, int n1, int n2_tiles, int q, int window, int max_tiles,
                    int4* __restrict__ tiles, int32_t* __restrict__ ready, int32_t* __restrict__ consumed,
-                   WsHeader* __restrict__ hdr) {
+                   int32_t* __restrict__ staged, int32_t* __restrict__ released, WsHeader* __restrict__ hdr) {
     __shared__ int32_t s_mt[MAX_E + 1], s_gofs[MAX_E + 1], s_wtot[32];
     pdl_enter();
     const int n2 = (n2_tiles + q - 1) / q;           // down entries per M tile: each covers up to q N tiles
@@ -250,6 +266,8 @@ fused_tiles_kernel(const int32_t* __restrict__ counts, const int32_t* __restrict
     for (int i = blockIdx.x * blockDim.x + tid; i < NMT; i += gridDim.x * blockDim.x) {
         ready[i] = 0;
         consumed[i] = 0;
+        staged[i] = 0;
+        released[i] = 0;
     }
 
     // largest e in [0, E) with s_mt[e] <= v and a non-empty tail (the expert that holds M tile index v), for 0 <= v < NMT
@@ -337,6 +355,17 @@ struct FusedArgs {
                                    // (zeroed before the launch), or NULL: unsynchronised starts
     int32_t* ready;                // per 256-row M tile: epilogue-warp arrivals of its gate/up tiles
     int32_t* consumed;             // per 256-row M tile: down entries whose loads of h have landed (ring mode)
+    // communication CTAs (comm_ctas > 0): the last comm_ctas CTAs of the grid stage the token rows of every row tile
+    int32_t comm_ctas, n_compute;  // n_compute = gridDim.x - comm_ctas CTAs work on tiles
+    __nv_bfloat16* xg;             // [COMM_SLOTS * 256, H] staging slots, row tile mt in slot mt % COMM_SLOTS
+    int32_t* staged;               // per row tile: 1 once its rows are in the slot
+    int32_t* released;             // per row tile: gate/up tiles whose loads from the slot have landed
+    const int32_t* mt_start2;      // the schedule's 256-row tile tables (row tile -> expert, first row, valid rows)
+    const int32_t* tile_expert2;
+    const int32_t* counts;
+    const int32_t* pad_offsets;
+    const int32_t* n_mtiles2;
+    int32_t max_mt2;
     int32_t ring;                  // > 0: h holds `ring` 256-row slots, row tile mt in slot mt % ring
     int32_t need_d;                // down entries per row tile
     int32_t max_tiles;
@@ -368,7 +397,7 @@ template <int CH>
 __device__ __forceinline__ void combine_tokens(const FusedArgs& a, Ctrl* ctrl, int lane, bool poller,
                                                volatile uint32_t* abort_flag, bool arrive) {
     int32_t* done = &a.header->ffn_done;
-    const int need = EPI_WARPS * (int)gridDim.x;
+    const int need = EPI_WARPS * a.n_compute;
     if (lane == 0 && arrive && a.starve != 2 && !*abort_flag) {
         // (the warp's TMA stores have completed: make them visible to generic-proxy reads of other SMs, then arrive)
         asm volatile("fence.proxy.async;" ::: "memory");
@@ -488,7 +517,7 @@ __global__ void __launch_bounds__(THREADS, 1)
 fused_ffn_kernel(const __grid_constant__ CUtensorMap mapWgu, const __grid_constant__ CUtensorMap mapWgu64,
                  const __grid_constant__ CUtensorMap mapHst, const __grid_constant__ CUtensorMap mapHld,
                  const __grid_constant__ CUtensorMap mapWd, const __grid_constant__ CUtensorMap mapY,
-                 const __grid_constant__ FusedArgs a) {
+                 const __grid_constant__ CUtensorMap mapXg, const __grid_constant__ FusedArgs a) {
     extern __shared__ uint8_t smem_raw[];
     pdl_enter();
     const uint32_t raw = smem_u32(smem_raw);
@@ -518,11 +547,13 @@ fused_ffn_kernel(const __grid_constant__ CUtensorMap mapWgu, const __grid_consta
                 mbar_init(smem_u32(&ctrl->q_empty[q]), ROLE_READERS);
             }
         }
+        for (int q = 0; q < COMM_ISSUERS * COMM_BUFS; ++q) mbar_init(smem_u32(&ctrl->cbar[q]), 1);
         ctrl->abort = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (warp == 1) {
+    const bool is_comm = (int)blockIdx.x >= a.n_compute;
+    if (warp == 1 && !is_comm) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                      ::"r"(smem_u32(&ctrl->tmem_base)), "r"((uint32_t)TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -531,6 +562,130 @@ fused_ffn_kernel(const __grid_constant__ CUtensorMap mapWgu, const __grid_consta
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = ctrl->tmem_base;
+
+    if (is_comm) {
+        // ---------------------------------------------------------------------- communication CTA: stages token rows
+        // Row tiles cr, cr + comm_ctas, ... in increasing order.  The copy goes through shared memory with bulk
+        // asynchronous copies (global -> shared -> global), so that ~128 KB are in flight per SM whatever the latency of
+        // the source: COMM_ISSUERS threads (lane 0 of warps 0..3) each run a pipeline over COMM_BUFS buffers of 16 KB and
+        // take every fourth piece (a row, or 16 KB of a longer row).  Rows past the expert's count are written as zeros by
+        // the other threads.
+        const int cr = (int)blockIdx.x - a.n_compute;
+        const int n_mt = min(*a.n_mtiles2, a.max_mt2);
+        const int row_bytes = a.H * 2, ppr = (row_bytes + COMM_PIECE - 1) / COMM_PIECE;
+        int32_t* s_tok = reinterpret_cast<int32_t*>(smem + STAGES * STAGE_BYTES);       // the tile's row -> token ids
+        uint32_t cph[COMM_BUFS] = {0u, 0u, 0u};
+        for (int mt = cr; mt < n_mt; mt += a.comm_ctas) {
+            if (threadIdx.x == 0) {
+                uint32_t go = 1u;
+                if (mt >= COMM_SLOTS) {      // the slot's previous rows have been loaded by all their gate/up tiles
+                    const int32_t* c = a.released + (mt - COMM_SLOTS);
+                    const unsigned long long t0 = globaltimer();
+                    uint32_t spins = 0;
+                    while (ld_acquire(c) < a.n1) {
+                        __nanosleep(256);
+                        if ((++spins & 31u) == 0u) {
+                            const unsigned long long limit =
+                                a.header->wait_limit_us ? 1000ull * a.header->wait_limit_us : WAIT_LIMIT_NS;
+                            if (a.header->status != 0 || globaltimer() - t0 > limit) {
+                                atomicCAS(&a.header->status, 0, (int)MOK_ERR_TIMEOUT);
+                                a.header->where = 46;
+                                go = 0u;
+                                break;
+                            }
+                        }
+                    }
+                }
+                *reinterpret_cast<volatile uint32_t*>(&ctrl->combine_go) = go;
+            }
+            const int e = __ldg(a.tile_expert2 + mt);
+            const int m = mt - __ldg(a.mt_start2 + e);
+            const int row0 = __ldg(a.pad_offsets + e) + m * TM;
+            const int valid = min(TM, __ldg(a.counts + e) - m * TM);
+            const int rows = valid > BM ? TM : BM;                      // a tile with one half only loads one half
+            if ((int)threadIdx.x < valid) s_tok[threadIdx.x] = __ldg(a.row_token + row0 + threadIdx.x);
+            __syncthreads();
+            if (!*reinterpret_cast<volatile uint32_t*>(&ctrl->combine_go)) break;
+            __nv_bfloat16* dst0 = a.xg + (size_t)(mt % COMM_SLOTS) * TM * a.H;
+            bool ok = true;
+            if (warp < COMM_ISSUERS) {
+                if (lane == 0) {
+                    const int n_pieces = valid * ppr;
+                    const uint32_t buf0 = base + (uint32_t)(warp * COMM_BUFS) * COMM_PIECE;
+                    uint64_t* bars = ctrl->cbar + warp * COMM_BUFS;
+                    auto piece = [&](int q, const char*& src, char*& dst, uint32_t& bytes) {
+                        const int r = q / ppr, off = (q - r * ppr) * COMM_PIECE;
+                        const int tok = s_tok[r];
+                        const __nv_bfloat16* srow;
+                        if (a.peer_tokens > 0) {
+                            const int pr = tok / a.peer_tokens;
+                            srow = a.peer_x[pr] + (size_t)(tok - pr * a.peer_tokens) * a.H;
+                        } else {
+                            srow = a.x + (size_t)tok * a.H;
+                        }
+                        src = reinterpret_cast<const char*>(srow) + off;
+                        dst = reinterpret_cast<char*>(dst0 + (size_t)r * a.H) + off;
+                        bytes = (uint32_t)min(COMM_PIECE, row_bytes - off);
+                    };
+                    auto load = [&](int q, int b) {
+                        const char* src; char* dst; uint32_t bytes;
+                        piece(q, src, dst, bytes);
+                        const uint32_t bar = smem_u32(&bars[b]);
+                        mbar_expect_tx(bar, bytes);
+                        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                                     ::"r"(buf0 + (uint32_t)b * COMM_PIECE), "l"(src), "r"(bytes), "r"(bar) : "memory");
+                    };
+                    // this issuer's pieces: warp, warp + 4, ...; two loads ahead of the store
+                    int q_load = warp, b_load = 0;
+                    for (int pre = 0; pre < COMM_BUFS - 1 && q_load < n_pieces; ++pre) {
+                        load(q_load, b_load);
+                        q_load += COMM_ISSUERS;
+                        b_load = (b_load + 1) % COMM_BUFS;
+                    }
+                    int b = 0;
+                    for (int q = warp; q < n_pieces; q += COMM_ISSUERS) {
+                        ok = wait_bar(smem_u32(&bars[b]), cph[b], abort_flag, a.header, 48);
+                        if (!ok) break;
+                        cph[b] ^= 1u;
+                        const char* src; char* dst; uint32_t bytes;
+                        piece(q, src, dst, bytes);
+                        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                                     ::"l"(dst), "r"(buf0 + (uint32_t)b * COMM_PIECE), "r"(bytes) : "memory");
+                        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                        // the buffer of the next load held the piece before this one: its store must have left shared memory
+                        asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                        if (q_load < n_pieces) {
+                            load(q_load, b_load);
+                            q_load += COMM_ISSUERS;
+                            b_load = (b_load + 1) % COMM_BUFS;
+                        }
+                        b = (b + 1) % COMM_BUFS;
+                    }
+                    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");      // every store of this issuer has completed
+                    asm volatile("fence.proxy.async;" ::: "memory");
+                    __threadfence();
+                }
+                ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+            } else {
+                // padding rows of the tile, as zeros
+                const int chunks = a.H >> 3;
+                for (int r = valid + (warp - COMM_ISSUERS); r < rows; r += THREADS / 32 - COMM_ISSUERS) {
+                    uint4* d = reinterpret_cast<uint4*>(dst0 + (size_t)r * a.H);
+                    for (int c = lane; c < chunks; c += 32) d[c] = make_uint4(0u, 0u, 0u, 0u);
+                }
+                __threadfence();                 // visible at GPU scope before the arrival below
+            }
+            if (!__syncthreads_and((int)ok)) {
+                // failure path only: give the copies already in flight into this CTA's shared memory time to land
+                const unsigned long long t0 = globaltimer();
+                while (globaltimer() - t0 < 200000ull) { }
+                break;
+            }
+            if (threadIdx.x == 0) asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(a.staged + mt) : "memory");
+        }
+        if (warp < COMM_ISSUERS && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+        return;                                  // (no tensor memory, no tiles: nothing to tear down)
+    }
 
     if (warp < 4) {
         reg_dec<REGS_CONTROL>();
@@ -541,7 +696,7 @@ fused_ffn_kernel(const __grid_constant__ CUtensorMap mapWgu, const __grid_consta
                 uint32_t ph = 0;
                 long long d_ready = 0;
                 int peek = 0;            // completion counter of the NEXT tile's rows, read during the current tile
-                TileWalk<DYN> w(ctrl, abort_flag, a.header, a.tiles, total, false);
+                TileWalk<DYN> w(ctrl, abort_flag, a.header, a.tiles, total, false, a.n_compute);
                 for (; w.valid(); w.advance()) {
                     const Tile t = decode_tile(w.d);
                     const bool two = t.valid > BM;
@@ -598,6 +753,33 @@ fused_ffn_kernel(const __grid_constant__ CUtensorMap mapWgu, const __grid_consta
                         // the rows were written through the async proxy by other CTAs and are read through it below
                         asm volatile("fence.proxy.async;" ::: "memory");
                     }
+                    const bool staged_a = !t.kind && a.comm_ctas > 0;     // the A rows come from the communication CTAs' slot
+                    if (staged_a) {
+                        const int32_t* flag = a.staged + t.mt;
+                        if (ld_acquire(flag) < 1) {
+                            const unsigned long long t0 = globaltimer();
+                            uint32_t spins = 0;
+                            while (ld_acquire(flag) < 1) {
+                                __nanosleep(64);
+                                if ((++spins & 63u) == 0u) {
+                                    if (*abort_flag) { ok = false; break; }
+                                    const unsigned long long limit =
+                                        a.header->wait_limit_us ? 1000ull * a.header->wait_limit_us : WAIT_LIMIT_NS;
+                                    if (globaltimer() - t0 > limit) {
+                                        *abort_flag = 1u;
+                                        atomicCAS(&a.header->status, 0, (int)MOK_ERR_TIMEOUT);
+                                        a.header->where = 47;
+                                        ok = false;
+                                        break;
+                                    }
+                                }
+                            }
+                        }
+                        if (!ok) break;
+                        // the rows were written through the generic proxy by another CTA and are read through the async one
+                        asm volatile("fence.proxy.async;" ::: "memory");
+                    }
+                    const int xrow = (t.mt % COMM_SLOTS) * TM;
                     const int kblocks = t.kind ? a.kb2 : a.kb1;
                     peek = 0;
                     for (int sub = 0; sub < t.cnt && ok; ++sub) {
@@ -623,14 +805,24 @@ fused_ffn_kernel(const __grid_constant__ CUtensorMap mapWgu, const __grid_consta
                             if (two) tma_load_2d(sa + A_BYTES, &mapHld, full, kb * BK, hrow + BM);
                             tma_load_2d(sb, &mapWd, full, kb * BK, brow0);
                             tma_load_2d(sb + B_BYTES / 2, &mapWd, full, kb * BK, brow1);
-                        } else if (narrow) {
-                            mbar_expect_tx(full, B_BYTES / 2);
-                            tma_load_2d(sb, &mapWgu64, full, kb * BK, brow0);
-                            tma_load_2d(sb + B_BYTES / 4, &mapWgu64, full, kb * BK, brow1);
                         } else {
-                            mbar_expect_tx(full, B_BYTES);
-                            tma_load_2d(sb, &mapWgu, full, kb * BK, brow0);
-                            tma_load_2d(sb + B_BYTES / 2, &mapWgu, full, kb * BK, brow1);
+                            uint32_t a_bytes = 0;
+                            if (staged_a) {     // (the gather threads have nothing to bring here either)
+                                asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0], %1;" ::"r"(full), "r"((uint32_t)GATHER_THREADS) : "memory");
+                                a_bytes = (two ? 2 : 1) * A_BYTES;
+                            }
+                            mbar_expect_tx(full, (narrow ? B_BYTES / 2 : B_BYTES) + a_bytes);
+                            if (staged_a) {
+                                tma_load_2d(sa, &mapXg, full, kb * BK, xrow);
+                                if (two) tma_load_2d(sa + A_BYTES, &mapXg, full, kb * BK, xrow + BM);
+                            }
+                            if (narrow) {
+                                tma_load_2d(sb, &mapWgu64, full, kb * BK, brow0);
+                                tma_load_2d(sb + B_BYTES / 4, &mapWgu64, full, kb * BK, brow1);
+                            } else {
+                                tma_load_2d(sb, &mapWgu, full, kb * BK, brow0);
+                                tma_load_2d(sb + B_BYTES / 2, &mapWgu, full, kb * BK, brow1);
+                            }
                         }
                         if (++s == STAGES) { s = 0; ph ^= 1u; }
                     }
@@ -650,7 +842,7 @@ fused_ffn_kernel(const __grid_constant__ CUtensorMap mapWgu, const __grid_consta
                           d_tot0 = 0, d_tot1 = 0;
                 const unsigned long long d_ns0 = dbg ? globaltimer() : 0ull;
                 const long long d_c0 = dbg ? clock64() : 0;
-                TileWalk<DYN> w(ctrl, abort_flag, a.header, a.tiles, total, false);
+                TileWalk<DYN> w(ctrl, abort_flag, a.header, a.tiles, total, false, a.n_compute);
                 for (; w.valid(); w.advance()) {
                     const Tile t = decode_tile(w.d);
                     const bool two = t.valid > BM;
@@ -707,6 +899,9 @@ fused_ffn_kernel(const __grid_constant__ CUtensorMap mapWgu, const __grid_consta
                     // ring mode: every load of h of this down entry has landed (its stages' full barriers were passed)
                     if (a.ring && t.kind && a.starve != 2)
                         asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(a.consumed + t.mt) : "memory");
+                    // communication CTAs: every load of this gate/up tile from its staging slot has landed
+                    if (a.comm_ctas > 0 && !t.kind && a.starve != 2)
+                        asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(a.released + t.mt) : "memory");
                     if (dbg) {
                         const long long dt = clock64() - tile0, units = (long long)(two ? 2 : 1) * kblocks * t.cnt;
                         if (t.kind) { d_full1 += w_full; d_te1 += w_te; d_kb1 += units; d_rows1 += (long long)t.valid * kblocks * t.cnt; d_tot1 += dt; }
@@ -762,15 +957,16 @@ fused_ffn_kernel(const __grid_constant__ CUtensorMap mapWgu, const __grid_consta
         const int gw = warp - (4 + EPI_WARPS), sub = lane >> 3, chunk = lane & 7;
         int s = 0;
         uint32_t ph = 0;
-        TileWalk<DYN> w(ctrl, abort_flag, a.header, a.tiles, total, true);
+        TileWalk<DYN> w(ctrl, abort_flag, a.header, a.tiles, total, true, a.n_compute);
         for (; w.valid(); w.advance()) {
             const Tile t = decode_tile(w.d);
             bool ok = true;
-            if (t.kind) {
-                // down tile: both operands come by TMA and the producer makes these threads' arrivals for them.  The warp
+            if (t.kind || a.comm_ctas > 0) {
+                // down tile (or a gate/up tile whose rows the communication CTAs staged): both operands come by TMA and
+                // the producer makes these threads' arrivals for them.  The warp
                 // still follows the ring stage by stage (one polling lane): a parity wait is only meaningful while the
                 // waiter is at most one phase ahead of the barrier, so it must not jump over the tile's stages.
-                for (int kb = 0; kb < a.kb2 * t.cnt; ++kb) {
+                for (int kb = 0; kb < (t.kind ? a.kb2 : a.kb1) * t.cnt; ++kb) {
                     if (lane == 0) ok = wait_bar(smem_u32(&ctrl->empty[s]), ph ^ 1u, abort_flag, a.header, 5);
                     ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
                     if (!ok) break;
@@ -849,7 +1045,7 @@ fused_ffn_kernel(const __grid_constant__ CUtensorMap mapWgu, const __grid_consta
                 tma_store_commit();
             }
         };
-        TileWalk<DYN> w(ctrl, abort_flag, a.header, a.tiles, total, true);
+        TileWalk<DYN> w(ctrl, abort_flag, a.header, a.tiles, total, true, a.n_compute);
         for (; w.valid(); w.advance()) {
             const Tile t = decode_tile(w.d);
             if (acc == 1 && t.valid <= BM) continue;
@@ -978,7 +1174,8 @@ fused_ffn_kernel(const __grid_constant__ CUtensorMap mapWgu, const __grid_consta
 
 template <bool DYN>
 static cudaError_t launch_kernel(int grid, cudaStream_t s, const CUtensorMap& m0, const CUtensorMap& m1, const CUtensorMap& m2,
-                                 const CUtensorMap& m3, const CUtensorMap& m4, const CUtensorMap& m5, const ff::FusedArgs& a) {
+                                 const CUtensorMap& m3, const CUtensorMap& m4, const CUtensorMap& m5, const CUtensorMap& m6,
+                                 const ff::FusedArgs& a) {
     using namespace ff;
     static PerDevice configured;
     int dev = 0, sm_count = 0;
@@ -990,8 +1187,10 @@ static cudaError_t launch_kernel(int grid, cudaStream_t s, const CUtensorMap& m0
     });
     if (e != cudaSuccess) return e;
     if (grid <= 0 || grid > sm_count) grid = sm_count;
-    // Dynamic draw: a position is only drawn by a CTA that runs: an ordinary (programmatically serialised) launch.
-    if (DYN) return launch_pdl(fused_ffn_kernel<DYN>, dim3(grid), dim3(THREADS), (size_t)SMEM_BYTES, s, m0, m1, m2, m3, m4, m5, a);
+    // Dynamic draw: a position is only drawn by a CTA that runs: an ordinary (programmatically serialised) launch --
+    // unless tiles wait for communication CTAs, which then have to be resident like everybody else.
+    if (DYN && a.comm_ctas == 0)
+        return launch_pdl(fused_ffn_kernel<DYN>, dim3(grid), dim3(THREADS), (size_t)SMEM_BYTES, s, m0, m1, m2, m3, m4, m5, m6, a);
     // static list: tiles wait for tiles of other CTAs, so every CTA of the grid must be resident (cooperative launch).
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
@@ -1003,7 +1202,7 @@ static cudaError_t launch_kernel(int grid, cudaStream_t s, const CUtensorMap& m0
     cfg.stream = s;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, fused_ffn_kernel<DYN>, m0, m1, m2, m3, m4, m5, a);
+    return cudaLaunchKernelEx(&cfg, fused_ffn_kernel<DYN>, m0, m1, m2, m3, m4, m5, m6, a);
 }
 
 // Host side.  `window_tiles`: distance (in list positions) between a group's gate/up tiles and its down tiles; 0 = the
@@ -1012,13 +1211,19 @@ static cudaError_t launch_kernel(int grid, cudaStream_t s, const CUtensorMap& m0
 cudaError_t launch_fused_ffn(const __nv_bfloat16* x, int T, int H, int I, int E, const __nv_bfloat16* Wgu,
                              const __nv_bfloat16* Wd, const WsLayout& L, char* ws, int grid, int window_tiles, bool dynamic,
                              bool gang_sync, bool dbg, int starve, cudaStream_t s, __nv_bfloat16* combine_out, int k,
-                             bool shared, int h_ring_tiles, const void* const* peer_x, int peer_tokens, void* y_out) {
+                             bool shared, int h_ring_tiles, const void* const* peer_x, int peer_tokens, void* y_out,
+                             int comm_ctas, void* xg) {
     using namespace ff;
     int dev = 0, sm_count = 0;
     cudaError_t e = current_device(&dev);
     if (e != cudaSuccess) return e;
     if ((e = device_sm_count(dev, &sm_count)) != cudaSuccess) return e;
     if (grid <= 0 || grid > sm_count) grid = sm_count;
+    // communication CTAs come out of the grid; at least one CTA computes
+    if (comm_ctas < 0 || (comm_ctas > 0 && !xg)) return cudaErrorInvalidValue;
+    if (comm_ctas >= grid) comm_ctas = grid - 1;
+    const int total_grid = grid;
+    grid -= comm_ctas;                                  // from here on: the CTAs that work on tiles
     WsHeader* hdr = reinterpret_cast<WsHeader*>(ws + L.header);
     const int n1 = (I + BN / 2 - 1) / (BN / 2), n2 = (H + BN - 1) / BN;
     // N tiles per down entry: as many as make its k-blocks about those of a gate/up entry (K = H against K = I)
@@ -1039,10 +1244,10 @@ cudaError_t launch_fused_ffn(const __nv_bfloat16* x, int T, int H, int I, int E,
     if (tblocks > sm_count) tblocks = sm_count;
     e = launch_pdl(fused_tiles_kernel, dim3(tblocks), dim3(MAX_E), 0, s, reinterpret_cast<const int32_t*>(ws + L.counts),
                    reinterpret_cast<const int32_t*>(ws + L.pad_offsets), reinterpret_cast<const int32_t*>(ws + L.mt_start2), E,
-                   n1, n2, q, window, L.max_ftiles, tiles, ready, ready + max_mt2, hdr);
+                   n1, n2, q, window, L.max_ftiles, tiles, ready, ready + max_mt2, ready + 2 * max_mt2, ready + 3 * max_mt2, hdr);
     if (e != cudaSuccess) return e;
 
-    CUtensorMap mWgu, mWgu64, mHst, mHld, mWd, mY;
+    CUtensorMap mWgu, mWgu64, mHst, mHld, mWd, mY, mXg;
     void* h = ws + L.h;
     void* y = y_out ? y_out : ws + L.y;
     if (!tmap::bf16_sw128(&mWgu, Wgu, (uint64_t)E * 2 * I, (uint64_t)H, BN / 2) ||
@@ -1052,6 +1257,8 @@ cudaError_t launch_fused_ffn(const __nv_bfloat16* x, int T, int H, int I, int E,
         !tmap::bf16_sw128(&mWd, Wd, (uint64_t)E * H, (uint64_t)I, BN / 2) ||
         !tmap::bf16_sw128(&mY, y, (uint64_t)L.Rpad, (uint64_t)H, 32))
         return cudaErrorInvalidValue;
+    mXg = mHld;      // (unused without communication CTAs)
+    if (comm_ctas > 0 && !tmap::bf16_sw128(&mXg, xg, (uint64_t)COMM_SLOTS * TM, (uint64_t)H, BM)) return cudaErrorInvalidValue;
     FusedArgs a;
     memset(&a, 0, sizeof(a));
     a.x = x;
@@ -1069,6 +1276,17 @@ cudaError_t launch_fused_ffn(const __nv_bfloat16* x, int T, int H, int I, int E,
     }
     a.ready = ready;
     a.consumed = ready + max_mt2;
+    a.staged = ready + 2 * max_mt2;
+    a.released = ready + 3 * max_mt2;
+    a.comm_ctas = comm_ctas;
+    a.n_compute = grid;
+    a.xg = reinterpret_cast<__nv_bfloat16*>(xg);
+    a.mt_start2 = reinterpret_cast<const int32_t*>(ws + L.mt_start2);
+    a.tile_expert2 = reinterpret_cast<const int32_t*>(ws + L.tile_expert2);
+    a.counts = reinterpret_cast<const int32_t*>(ws + L.counts);
+    a.pad_offsets = reinterpret_cast<const int32_t*>(ws + L.pad_offsets);
+    a.n_mtiles2 = &hdr->n_mtiles2;
+    a.max_mt2 = max_mt2;
     a.ring = ring;
     a.need_d = (n2 + q - 1) / q;
     a.max_tiles = L.max_ftiles;
@@ -1087,8 +1305,8 @@ cudaError_t launch_fused_ffn(const __nv_bfloat16* x, int T, int H, int I, int E,
     a.T = T;
     a.k = k;
 
-    return dynamic ? launch_kernel<true>(grid, s, mWgu, mWgu64, mHst, mHld, mWd, mY, a)
-                   : launch_kernel<false>(grid, s, mWgu, mWgu64, mHst, mHld, mWd, mY, a);
+    return dynamic ? launch_kernel<true>(total_grid, s, mWgu, mWgu64, mHst, mHld, mWd, mY, mXg, a)
+                   : launch_kernel<false>(total_grid, s, mWgu, mWgu64, mHst, mHld, mWd, mY, mXg, a);
 }
 
 }  // namespace mok

@@ -105,7 +105,7 @@ bool ws_layout(int T, int H, int I, int Is, int E, int k, WsLayout* L, bool mx, 
         const long long nt = mt2 * per;
         L->max_ftiles = nt < (1ll << 30) ? (int32_t)nt : 0;
         L->ftiles = take(sizeof(int4) * (size_t)L->max_ftiles);
-        L->ready = take(2 * sizeof(int32_t) * (size_t)mt2);
+        L->ready = take(4 * sizeof(int32_t) * (size_t)mt2);    // ready, consumed, staged, released
     }
     {   // gang-start counters of the 256-row kernel: one per tile of the largest of the four GEMMs
         const long long mt2 = Rpad / (2 * TILE_M), mts = L->Tpad / (2 * TILE_M);
@@ -170,7 +170,7 @@ static int validate(const mok_args* a, WsLayout* L, size_t extra_ws) {
                       a->config->fused_ffn < 0 || a->config->fused_ffn > 3 || a->config->fused_window < -1 ||
                       a->config->gang_sync < 0 || a->config->gang_sync > 2 || a->config->serial_launches < 0 ||
                       a->config->serial_launches > 1 || a->config->h_ring_tiles < 0 || a->config->shared_overlap < 0 ||
-                      a->config->shared_overlap > 2))
+                      a->config->shared_overlap > 2 || a->config->comm_ctas < 0))
         return MOK_ERR_SHAPE;
     return MOK_OK;
 }
@@ -250,7 +250,7 @@ static bool use_fused_ffn(const mok_config* cfg, int H, int I, int tile_m, long 
     if (use_simt(cfg) || use_tn(cfg) || use_mx(cfg) || tile_m != TILE_M || max_ftiles <= 0) return false;
     if (cfg && (cfg->fused_ffn == 1 || cfg->cta_group == 1 || cfg->cta_group == 2)) return false;
     if (!fused_gather(cfg, I)) return false;
-    if (cfg && (cfg->fused_ffn >= 2 || cfg->h_ring_tiles > 0)) return true;
+    if (cfg && (cfg->fused_ffn >= 2 || cfg->h_ring_tiles > 0 || cfg->comm_ctas > 0)) return true;
     if (cfg && cfg->tile_sched == 1) return false;          // (tile stealing belongs to the two-launch path)
     // (at least two row tiles per expert on average: with single tiles there is nothing to start together, and the
     //  weight-streaming regime of small batches is served better by the two launches: 4.64 vs 4.80 ms at 128 rows)
@@ -563,11 +563,16 @@ static int forward_device(const mok_args* a, const WsLayout& L, const __nv_bfloa
         // (with a ring of h the window is short; the static stride keeps a row group's tiles closest together: measured
         //  1.29 against 1.56 ms on the Qwen3-like layer with 72 slots)
         const bool fused_dynamic = sched == 1 || (sched == 0 && !fused_sync && L.h_ring == 0);
+        // communication CTAs exist in the one-launch kernel; their staging slots take the place of the gathered copy of x
+        const int comm_ctas = a->config ? a->config->comm_ctas : 0;
+        if (comm_ctas > 0 && (!fused || L.h_ring > 0 || (long long)L.Rpad < (long long)FFN_COMM_SLOTS * 2 * TILE_M))
+            return MOK_ERR_UNSUPPORTED;
         if (fused) {
             e = launch_fused_ffn(x, a->T, a->H, a->I, a->E, reinterpret_cast<const __nv_bfloat16*>(a->W_gate_up),
                                  reinterpret_cast<const __nv_bfloat16*>(a->W_down), L, ws, a->config ? a->config->grid : 0,
                                  a->config ? a->config->fused_window : 0, fused_dynamic, fused_sync, dbg, g.starve, s,
-                                 combine_in_launch ? out : nullptr, a->k, a->I_shared > 0, L.h_ring);
+                                 combine_in_launch ? out : nullptr, a->k, a->I_shared > 0, L.h_ring, nullptr, 0, nullptr,
+                                 comm_ctas, comm_ctas > 0 ? ws + L.xg : nullptr);
             if (e != cudaSuccess) return cuda_fail(e);
         } else if ((rc = run_gemm(g, true, a->config, L, ws, s))) return rc;
         g.row_token = nullptr;

@@ -161,7 +161,9 @@ cudaError_t launch_fused_ffn(const __nv_bfloat16* x, int T, int H, int I, int E,
                              int k = 0, bool shared = false,    // combine_out != NULL: the combine runs in the same launch
                              int h_ring_tiles = 0,              // > 0: h is a ring of that many 256-row tiles
                              const void* const* peer_x = nullptr, int peer_tokens = 0,   // expert parallelism: every rank's token rows
-                             void* y_out = nullptr);            // where the down tiles go (NULL: the workspace's y)
+                             void* y_out = nullptr,             // where the down tiles go (NULL: the workspace's y)
+                             int comm_ctas = 0, void* xg = nullptr);   // communication CTAs and their staging slots
+constexpr int FFN_COMM_SLOTS = 24;       // 256-row slots of that staging buffer ([FFN_COMM_SLOTS * 256, H] bf16)
 // whether the routed expert FFN runs as the one launch for these sizes and knobs; *sync: with synchronised tile starts
 bool fused_ffn_choice(const mok_config* cfg, int H, int I, int tile_m, long long rows, int experts, int max_ftiles, bool* sync);
 constexpr int H_RING_MIN_TILES = 24;     // smallest ring of the gated activation (see gemm_fused.cu)

@@ -44,7 +44,7 @@ class mok_config(ctypes.Structure):
                 ("tile_sched", ctypes.c_int32), ("macrobatch_tokens", ctypes.c_int32),
                 ("fused_ffn", ctypes.c_int32), ("fused_window", ctypes.c_int32), ("gang_sync", ctypes.c_int32),
                 ("serial_launches", ctypes.c_int32), ("h_ring_tiles", ctypes.c_int32),
-                ("shared_overlap", ctypes.c_int32)]
+                ("shared_overlap", ctypes.c_int32), ("comm_ctas", ctypes.c_int32)]
 
 
 class mok_args(ctypes.Structure):
@@ -221,8 +221,9 @@ def _stream(stream):
 
 def _config(impl=0, grid=0, router_impl=0, profile=0, gather_mode=0, cta_group=0, debug=0, host_chunks=0,
             precision=0, tile_sched=0, macrobatch_tokens=0, fused_ffn=0, fused_window=0, gang_sync=0, serial_launches=0,
-            h_ring_tiles=0, shared_overlap=0):
+            h_ring_tiles=0, shared_overlap=0, comm_ctas=0):
     c = mok_config()
+    c.comm_ctas = comm_ctas
     c.shared_overlap = shared_overlap
     c.serial_launches = serial_launches
     c.h_ring_tiles = h_ring_tiles

@@ -110,11 +110,14 @@ def test_expert_parallel_layer_shapes(name, T, H, E, k, I, I_s, bias, R):
 
 @pytest.mark.parametrize("R", [1, 2, 4])
 @pytest.mark.parametrize("kw", [{"fused_ffn": 2}, {"fused_ffn": 2, "tile_sched": 2, "gang_sync": 2},
-                                {"fused_ffn": 2, "fused_window": -1, "grid": 7}], ids=["dynamic", "static_gang", "no_window"])
+                                {"fused_ffn": 2, "fused_window": -1, "grid": 7}, {"comm_ctas": 6},
+                                {"comm_ctas": 12, "tile_sched": 2, "gang_sync": 2}],
+                         ids=["dynamic", "static_gang", "no_window", "comm_ctas", "comm_ctas_static"])
 def test_expert_parallel_layer_with_the_one_launch_expert_ffn(R, kw):
     """The routed experts of every rank as ONE persistent launch (gate/up tiles pull their rows from the owners'
     buffers, down tiles wait on the completion counters and store into the peer-visible y): every token against the
-    oracle and bit for bit the one-rank layer, on a shape with several row tiles per expert and a shared expert."""
+    oracle and bit for bit the one-rank layer, on a shape with several row tiles per expert and a shared expert.
+    With comm_ctas the pulls are made by communication CTAs into staging slots a row tile ahead of their use."""
     m = mok()
     cfg = inputs.MoEConfig("ep_one_launch", 3072, 512, 8, 3, 320, 128, bias="zipf", seed=12)
     rep = ep_case(cfg, R, config=m._config(**kw))

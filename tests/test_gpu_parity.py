@@ -388,7 +388,11 @@ def test_one_launch_ffn_gives_the_bits_of_two_launches(cfg):
                # the combine at the end of the same launch (the shared expert then runs first)
                {"fused_ffn": 3}, {"fused_ffn": 3, "grid": 1}, {"fused_ffn": 3, "fused_window": -1, "grid": 37},
                {"fused_ffn": 3, "tile_sched": 2, "grid": 5}, {"fused_ffn": 3, "gang_sync": 2},
-               {"fused_ffn": 3, "gang_sync": 2, "grid": 11, "fused_window": 40}):
+               {"fused_ffn": 3, "gang_sync": 2, "grid": 11, "fused_window": 40},
+               # communication CTAs: some CTAs of the grid stage the token rows, the others load them by TMA
+               {"comm_ctas": 4}, {"comm_ctas": 16, "tile_sched": 2, "gang_sync": 2}, {"comm_ctas": 1, "grid": 9},
+               {"comm_ctas": 8, "fused_window": -1}, {"comm_ctas": 4, "fused_ffn": 3}, {"comm_ctas": 200},
+               {"comm_ctas": 3, "tile_sched": 1, "grid": 5}):
         out1 = pu.run_gpu(cfg, g, config=m._config(**(dict(fused_ffn=2) | kw)), stages=False)
         assert torch.equal(out1.view(torch.int16), out2.view(torch.int16)), kw
     # ... and against the oracle with the stage outputs requested, and under the per-stage profiler (the stages then run
@@ -487,10 +491,11 @@ def test_bounded_waits_report_a_timeout_and_leave_the_context_usable(fused, sche
 
 
 @pytest.mark.parametrize("kw", [{"h_ring_tiles": 24}, {"h_ring_tiles": 24, "tile_sched": 1}, {"fused_ffn": 3},
-                                {"fused_ffn": 3, "tile_sched": 2}], ids=["ring", "ring_dynamic", "combine", "combine_static"])
+                                {"fused_ffn": 3, "tile_sched": 2}, {"comm_ctas": 2}, {"comm_ctas": 2, "tile_sched": 2}],
+                         ids=["ring", "ring_dynamic", "combine", "combine_static", "comm", "comm_static"])
 def test_completion_counter_waits_of_the_one_launch_kernel_run_out_cleanly(kw):
     """The waits on the one-launch kernel's own completion counters -- a ring slot's previous rows consumed, all
-    epilogue warps done before the in-launch combine -- are bounded too: with the test hook that suppresses every
+    epilogue warps done before the in-launch combine, a staging slot released for the communication CTAs -- are bounded too: with the test hook that suppresses every
     arrival on those counters (and a 2 ms limit) the call ends with MOK_ERR_TIMEOUT, nothing faults, and the next call
     on the same context and workspace gives the normal bits."""
     m = mok()
