@@ -82,6 +82,9 @@ def parse():
     p.add_argument("--host-chunks", type=int, default=0, help="token chunks of the host-buffer call (0 = auto)")
     p.add_argument("--precision", default="bf16", choices=["bf16", "mxfp8"],
                    help="routed experts in bf16 (the headline workload) or MXFP8 with pre-quantised weights")
+    p.add_argument("--comm-ctas", type=int, default=0,
+                   help="one-launch expert FFN: CTAs that only stage token rows for the computing CTAs (0 = the gather "
+                        "warps of every CTA pull their rows themselves)")
     p.add_argument("--parallelism", default="replicas", choices=["replicas", "ep"],
                    help="replicas: every GPU holds all experts and its own batch (no data-path collective); ep: expert "
                         "parallelism, every GPU holds E / N experts and its own batch of T tokens, rows are pulled from "
@@ -368,7 +371,7 @@ class Layer:
     def conf(self, **kw):
         a = self.args
         base = dict(impl=a.gemm, gather_mode=a.gather_mode, cta_group=a.cta_group, precision=self.prec,
-                    tile_sched=a.tile_sched, fused_ffn=a.fused_ffn, h_ring_tiles=a.h_ring)
+                    tile_sched=a.tile_sched, fused_ffn=a.fused_ffn, h_ring_tiles=a.h_ring, comm_ctas=a.comm_ctas)
         base.update(kw)
         return self.mok._config(**base)
 
@@ -645,7 +648,8 @@ def run_ep(args, cfg, rank, local_rank, world):
     mxw = mok.MxWeights(g["W_gate_up"], g["W_down"]) if mx else None
     layer = ep.DistributedLayer(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k, dev, mx=mx)
     out = torch.empty_like(g["x"])
-    conf = mok._config(cta_group=args.cta_group)
+    conf = mok._config(cta_group=args.cta_group, comm_ctas=args.comm_ctas, fused_ffn=args.fused_ffn,
+                       tile_sched=args.tile_sched)
 
     def step(x, timeline=None):
         layer.forward(x, W_r, bias, g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], out=out, config=conf,
@@ -729,7 +733,7 @@ def run_ep(args, cfg, rank, local_rank, world):
             "dtype": "mxfp8 routed experts (fp32 accumulate), bf16 elsewhere" if mx else "bf16", "data": "synthetic",
             "config": {"workload": cfg.name, "T_per_gpu": cfg.T, "T_total": world * cfg.T, "H": cfg.H, "E": cfg.E,
                        "experts_per_gpu": L, "k": cfg.k, "I": cfg.I, "I_shared": cfg.I_s, "routing": cfg.bias,
-                       "parallelism": f"ep{world}",
+                       "parallelism": f"ep{world}", "comm_ctas": args.comm_ctas,
                        "l2": "inputs larger than L2 (weights + activations >> 126 MB), no explicit flush",
                        "timing": "ms_per_step = median of the per-step CUDA-event times of one bracketed loop (max over "
                                  "ranks); phase times come from a second loop with an event after every phase"},
