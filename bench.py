@@ -40,7 +40,7 @@ NCU_TRAFFIC = {
     "deepseek_v3": {"bytes": 20.57e9, "scale": 1, "source": "profiles/gemm_kernels_deepseek_v3.md"},
     # the routed expert FFN as one persistent launch (the default where synchronised tile starts pay)
     "deepseek_v3+one_launch": {"bytes": 38.01e9, "scale": 1, "source": "profiles/gemm_kernels_deepseek_v3.md"},
-    "gpt_oss_120b+one_launch": {"bytes": 8.34e9, "scale": 1, "source": "profiles/gemm_kernels_other_workloads.md"},
+    "gpt_oss_120b+one_launch": {"bytes": 9.55e9, "scale": 1, "source": "profiles/gemm_kernels_other_workloads.md"},
     "qwen3_30b_a3b": {"bytes": 1.415e9, "scale": 1, "source": "profiles/gemm_kernels_other_workloads.md"},
     "mixtral_8x7b": {"bytes": 3.553e9, "scale": 1, "source": "profiles/gemm_kernels_other_workloads.md"},
     "gpt_oss_120b": {"bytes": 5.136e9, "scale": 1, "source": "profiles/gemm_kernels_other_workloads.md"},

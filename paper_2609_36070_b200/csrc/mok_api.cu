@@ -236,15 +236,22 @@ static bool gang_pays(long long w_bytes, long long rows, int experts) {
     return w_bytes >= (12ll << 20) && rows < 8ll * 256 * experts;
 }
 
-// Routed gate/up + SwiGLU + down as ONE persistent launch (gemm_fused.cu).  Chosen by default where synchronised tile
-// starts pay for both GEMMs (there it equals or beats the two launches: DeepSeek-like -1.6 %, GPT-OSS-like -4 %, two
-// variants alternating in one process); elsewhere the two launches are 1-2 % faster and stay the default.
+// Routed gate/up + SwiGLU + down as ONE persistent launch (gemm_fused.cu).  Chosen by default for large expert
+// matrices (both GEMMs' weights of an expert >= 12 MB, fewer than eight row tiles per expert: there it equals or beats
+// the two launches: DeepSeek-like -1.6 %, GPT-OSS-like -4 to -13 %, variants alternating in one process); elsewhere the
+// two launches are 1-2 % faster from a rested board and stay the default.
 // fused_ffn = 1 / 2 force the two launches / the one launch; 3 = the one launch with the combine at its end.
+static bool large_experts(int H, int I, long long rows, int experts) {
+    return gang_pays(4ll * I * H, rows, experts) && gang_pays(2ll * H * I, rows, experts);
+}
+// ... with synchronised tile starts on the static stride where an expert has three or more row tiles on average (the
+// DeepSeek-like layer: 23.7 against 29-31 ms with the dynamic draw), with the dynamic draw and no gangs below that (the
+// GPT-OSS-like layer, two row tiles per expert and K = 2880: 3.20-3.24 against 3.41-3.48 ms under the power cap).
 static bool fused_gang(const mok_config* cfg, int H, int I, long long rows, int experts) {
     const int mode = cfg ? cfg->gang_sync : 0;
     if (mode == 1) return false;
     if (mode == 2) return true;
-    return gang_pays(4ll * I * H, rows, experts) && gang_pays(2ll * H * I, rows, experts);
+    return large_experts(H, I, rows, experts) && rows >= 768ll * experts;
 }
 static bool use_fused_ffn(const mok_config* cfg, int H, int I, int tile_m, long long rows, int experts, int max_ftiles) {
     if (use_simt(cfg) || use_tn(cfg) || use_mx(cfg) || tile_m != TILE_M || max_ftiles <= 0) return false;
@@ -255,7 +262,7 @@ static bool use_fused_ffn(const mok_config* cfg, int H, int I, int tile_m, long 
     // (at least two row tiles per expert on average: with single tiles there is nothing to start together, and the
     //  weight-streaming regime of small batches is served better by the two launches: 4.64 vs 4.80 ms at 128 rows)
     return use_m2(cfg, H, tile_m, rows, experts) && use_m2(cfg, I, tile_m, rows, experts) &&
-           rows >= 512ll * experts && fused_gang(cfg, H, I, rows, experts);
+           rows >= 512ll * experts && large_experts(H, I, rows, experts) && !(cfg && cfg->gang_sync == 1);
 }
 
 // Synchronised starts of the row tiles that share a weight tile (see gemm_tcgen05_m2.cu) for one launch of the 256-row
