@@ -100,7 +100,8 @@ typedef struct mok_config {
                              again.  Same bits as the single pass; counts / offsets / perm / inv_perm (tables of ONE
                              schedule) cannot be returned: MOK_ERR_UNSUPPORTED. */
     int32_t fused_ffn;    /* routed experts, bf16: 1 = gate/up GEMM and down GEMM as two launches, 0 = choose (the one launch
-                             where synchronised tile starts pay, see gang_sync; else the two launches),
+                             for large expert matrices -- an expert's weights of either GEMM at least 12 MB, two to
+                             eight row tiles per expert; else the two launches),
                              2 = ONE persistent launch over a list of gate/up tiles and down tiles; a down tile runs
                              once a per-row-tile completion counter, advanced by the gate/up epilogues, shows that its
                              rows of the gated activation exist (Section 3.2: megakernel, GPU-local synchronisation
@@ -111,8 +112,9 @@ typedef struct mok_config {
     int32_t fused_window; /* fused_ffn: list positions between a row group's gate/up tiles and its down tiles (0 = a
                              default of two to eight grids' worth of tiles; -1 = none: directly behind them, which makes
                              every down tile wait -- a test setting).  The list is walked with stride grid and
-                             synchronised tile starts where those pay, else handed out dynamically (each CTA draws the
-                             next position from a global counter); tile_sched = 1 / 2 force the draw / the stride. */
+                             synchronised tile starts where experts have three or more row tiles on average, else
+                             handed out dynamically (each CTA draws the next position from a global counter);
+                             tile_sched = 1 / 2 force the draw / the stride. */
     int32_t gang_sync;    /* 256-row-tile GEMM kernel: the row tiles of an expert that use the same weight tile start that
                              tile together (a counter per such gang, bounded wait, cooperative launch), so that the weight
                              tile is read from DRAM once and shared through L2 instead of once per row tile.
