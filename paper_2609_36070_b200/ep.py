@@ -313,8 +313,9 @@ def forward_distributed(x_local, W_router, router_bias, W_gate_up_local, W_down_
     return out
 
 
-def _ipc_rank(rank, world, queues, config_name, port, results, mx=False):
-    """One rank of the several-processes-on-one-GPU self-check: gloo collectives, peer buffers through CUDA IPC."""
+def _ipc_rank(rank, world, queues, config_name, port, results, mx=False, tokens=0, config_kw=None):
+    """One rank of the several-processes-on-one-GPU self-check: gloo collectives, peer buffers through CUDA IPC.
+    tokens: total tokens over the ranks (0 = the workload's); config_kw: knobs of the expert-parallel calls."""
     import os
     import torch.distributed as dist
     from . import inputs
@@ -323,7 +324,10 @@ def _ipc_rank(rank, world, queues, config_name, port, results, mx=False):
     torch.cuda.set_device(dev)
     dist.init_process_group("gloo", rank=rank, world_size=world)
     cfg = inputs.CONFIGS[config_name]
+    if tokens:
+        cfg = cfg.with_tokens(tokens)
     T_local, L = cfg.T // world, cfg.E // world
+    conf = mok._config(**config_kw) if config_kw else None
 
     def exchange(name, t):
         # every rank puts its tensor on every other rank's queue (torch.multiprocessing ships a CUDA IPC handle) and
@@ -349,7 +353,7 @@ def _ipc_rank(rank, world, queues, config_name, port, results, mx=False):
     mxw = mok.MxWeights(Wgu, Wd) if mx else None
     out = None
     for _ in range(2):                                         # twice: buffers are reused across layers
-        out = layer.forward(x_local, W_r, bias, Wgu, Wd, g["W_sgu"], g["W_sd"], mx_weights=mxw)
+        out = layer.forward(x_local, W_r, bias, Wgu, Wd, g["W_sgu"], g["W_sd"], mx_weights=mxw, config=conf)
     layer._barrier()
     ws = mok.alloc_workspace(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k, device=dev, mx=mx)
     one = mok.mok_moe_forward_ex(g["x"], W_r, bias, g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], cfg.k, ws,
@@ -376,7 +380,7 @@ def _ipc_rank(rank, world, queues, config_name, port, results, mx=False):
     dist.destroy_process_group()
 
 
-def check_processes_on_one_gpu(world=2, config_name="tiny", port=29561, mx=False):
+def check_processes_on_one_gpu(world=2, config_name="tiny", port=29561, mx=False, tokens=0, config_kw=None):
     """Runs `world` ranks as separate processes on GPU 0 (each maps the others' x / y / pos through CUDA IPC) and
     returns True if every rank's output (and, in bf16 mode, its dx and dw of the backward pass) equals its slice of the
     one-rank layer's bit for bit."""
@@ -384,7 +388,8 @@ def check_processes_on_one_gpu(world=2, config_name="tiny", port=29561, mx=False
     ctx = mp.get_context("spawn")
     queues = [ctx.Queue() for _ in range(world)]
     results = ctx.Queue()
-    procs = [ctx.Process(target=_ipc_rank, args=(r, world, queues, config_name, port, results, mx)) for r in range(world)]
+    procs = [ctx.Process(target=_ipc_rank, args=(r, world, queues, config_name, port, results, mx, tokens, config_kw))
+             for r in range(world)]
     for p in procs:
         p.start()
     ok = []

@@ -210,6 +210,16 @@ def test_ranks_as_separate_processes_on_one_gpu(world, mx):
     assert ep.check_processes_on_one_gpu(world=world, config_name="tiny", port=29561 + world + 10 * int(mx), mx=mx)
 
 
+@pytest.mark.parametrize("kw,port", [({"fused_ffn": 2}, 29591), ({"comm_ctas": 2}, 29593)], ids=["one_launch", "comm_ctas"])
+def test_ranks_as_separate_processes_with_the_one_launch_kernel(kw, port):
+    """Two processes on GPU 0, the Qwen3-like shapes with 2048 tokens, the routed experts of each rank as the one-launch
+    kernel: its gather warps (or, with comm_ctas, the bulk copies of its communication CTAs) read the other process's
+    token rows through a CUDA IPC mapping; each rank's output must equal its slice of the one-rank layer bit for bit,
+    and so must dx and dw of the backward pass."""
+    from paper_2609_36070_b200 import ep
+    assert ep.check_processes_on_one_gpu(world=2, config_name="qwen3_30b_a3b", port=port, tokens=2048, config_kw=kw)
+
+
 @pytest.mark.parametrize("R", [1, 2, 4])
 def test_expert_parallel_mxfp8_equals_the_one_rank_mxfp8_layer(R):
     """The paper's main configuration: expert parallelism with MXFP8 routed experts (Section 3.4).  Every rank quantises
