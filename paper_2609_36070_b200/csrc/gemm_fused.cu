@@ -1154,7 +1154,7 @@ fused_ffn_kernel(const __grid_constant__ CUtensorMap mapWgu, const __grid_consta
         }
         if (lane == 0) tma_store_wait_all();
         __syncwarp();
-        if (a.out != nullptr) combine_tokens<2>(a, ctrl, lane, warp == 4, abort_flag, true);
+        if (a.out != nullptr) combine_tokens<4>(a, ctrl, lane, warp == 4, abort_flag, true);
     }
 
     // ---------------------------------------------------------------------- teardown
