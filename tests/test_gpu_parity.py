@@ -530,23 +530,36 @@ def test_shared_expert_beside_the_routed_experts_gives_the_same_bits(cfg):
             assert torch.equal(out.view(torch.int16), inline.view(torch.int16)), kw
 
 
-def test_forward_can_be_captured_in_a_cuda_graph_and_replayed():
+GRAPH_CASES = [
+    ("tiny", {}),                                                     # two streams: the shared expert beside the routed ones
+    ("mid_many", {"fused_ffn": 2}),                                   # the one-launch kernel, dynamic draw
+    ("mid_many", {"fused_ffn": 2, "tile_sched": 2, "gang_sync": 2}),  # ... as a cooperative launch
+    ("mid_many", {"comm_ctas": 4}),
+    ("mid_many", {"fused_ffn": 3}),
+    ("mid_many", {"h_ring_tiles": 24}),
+]
+
+
+@pytest.mark.parametrize("name,kw", GRAPH_CASES, ids=[f"{n}-{'-'.join(k) or 'default'}" for n, k in GRAPH_CASES])
+def test_forward_can_be_captured_in_a_cuda_graph_and_replayed(name, kw):
     """The layer makes no host synchronisation and no allocation after its first call for a shape, so a whole
-    forward can be recorded once into a CUDA graph and replayed (launch-bound small batches): same bits."""
+    forward can be recorded once into a CUDA graph and replayed (launch-bound small batches): same bits.  That holds
+    for the call with a second stream inside, for the cooperative launches and for the one-launch kernel's options."""
     m = mok()
-    cfg = inputs.CONFIGS["tiny"]
+    cfg = inputs.CONFIGS["tiny"] if name == "tiny" else MID[1]
     d = inputs.make_inputs(cfg)
     g = pu.upload(d)
     ws = m.alloc_workspace(cfg.T, cfg.H, cfg.I, cfg.I_s, cfg.E, cfg.k)
     out = torch.empty_like(g["x"])
+    conf = m._config(**kw)
     args = (g["x"], g["W_r"], g["bias"], g["W_gate_up"], g["W_down"], g["W_sgu"], g["W_sd"], cfg.k, ws)
-    m.mok_moe_forward_ex(*args, out=out)                       # first call: one-time kernel attribute set-up
+    m.mok_moe_forward_ex(*args, out=out, config=conf)          # first call: one-time kernel attribute set-up
     torch.cuda.synchronize()
     want = out.clone()
     graph = torch.cuda.CUDAGraph()
     out.zero_()
     with torch.cuda.graph(graph):
-        m.mok_moe_forward_ex(*args, out=out)
+        m.mok_moe_forward_ex(*args, out=out, config=conf)
     for _ in range(3):
         out.zero_()
         graph.replay()
