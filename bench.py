@@ -550,6 +550,32 @@ def measure(layer, steps, warmup, barrier, sampler_windows, pk, with_counters):
         srec["ms_per_step"] = sum(srec["stage_ms"].values())
         rec["sustained"] = srec
         sampler_windows.append((srec, "clocks", ssw))
+    if rec["ms_per_step"] < 0.3 and not layer.mx:
+        # a launch-bound layer: the same call recorded once into a CUDA graph and replayed (what a caller with a fixed
+        # shape would do), so that the number shows the GPU's time and not the host's launch rate
+        torch = layer.torch
+        try:
+            layer.step(conf)
+            torch.cuda.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                layer.step(conf)
+            for _ in range(5):
+                graph.replay()
+            torch.cuda.synchronize()
+            n = 200
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(n):
+                graph.replay()
+            e1.record()
+            torch.cuda.synchronize()
+            layer.check_status()
+            rec["cuda_graph_replay_ms"] = e0.elapsed_time(e1) / n
+            del graph
+        except Exception as ex:                      # (informational: never fails the run)
+            rec["cuda_graph_replay_ms"] = None
+            rec["cuda_graph_note"] = str(ex)[:200]
     if with_counters and not layer.mx and layer.args.gemm == 0:
         rec["counters"] = layer.counters()
         layer.check_status()
@@ -1036,6 +1062,9 @@ def main():
         line["counters"] = main_rec["counters"]
     if "one_launch_ffn" in main_rec:
         line["one_launch_ffn"] = main_rec["one_launch_ffn"]
+    for key in ("cuda_graph_replay_ms", "cuda_graph_note"):
+        if key in main_rec:
+            line[key] = main_rec[key]
     if main_counts is not None:
         line["load"] = {"max_count": int(main_counts.max()), "empty_experts": int((main_counts == 0).sum()),
                         "rows_padded_to_128": int(((main_counts + 127) // 128 * 128).sum()), "rows": int(main_counts.sum())}
